@@ -1,0 +1,132 @@
+"""numpy front end of the CPU oracle (test infrastructure only).
+
+Only the tests, the smoke check and the CPU-baseline leg of the benchmark may
+import this package; the GPU library never does.  Arrays are dense and
+C-contiguous, laid out [B, L, H, T_cap, D]; bfloat16 data travels as uint16
+bit patterns (``dtype='bf16'``), fp32 as float32.
+"""
+import ctypes
+import os
+
+import numpy as np
+
+from . import build as _build
+
+_DT = {"f32": 0, "bf16": 1}
+_LIB = None
+
+
+def lib():
+    global _LIB
+    if _LIB is None:
+        _LIB = ctypes.CDLL(_build.build())
+        _LIB.l2kv_oracle_keep_count.restype = ctypes.c_int32
+        _LIB.l2kv_oracle_keep_count.argtypes = [ctypes.c_int32, ctypes.c_double]
+    return _LIB
+
+
+def _p(a):
+    return ctypes.c_void_p(a.ctypes.data)
+
+
+def _check(a, dtype):
+    want = np.uint16 if dtype == "bf16" else np.float32
+    if a.dtype != want or not a.flags["C_CONTIGUOUS"]:
+        raise ValueError(f"expected contiguous {want} for dtype {dtype}, got {a.dtype}")
+
+
+def _i32(x):
+    return np.ascontiguousarray(np.asarray(x, dtype=np.int32))
+
+
+def hardware_threads():
+    return int(lib().l2kv_oracle_hardware_threads())
+
+
+def keep_count(length, keep_ratio):
+    return int(lib().l2kv_oracle_keep_count(int(length), float(keep_ratio)))
+
+
+def key_sumsq(K, dtype):
+    """fp64 sum of squares of every row of K[..., D]."""
+    _check(K, dtype)
+    D = K.shape[-1]
+    out = np.empty(K.shape[:-1], dtype=np.float64)
+    lib().l2kv_oracle_key_sumsq(_p(K), _DT[dtype], ctypes.c_int64(out.size), D, _p(out))
+    return out
+
+
+def key_sumsq_f32(K, dtype):
+    """Sum of squares in the GPU library's documented fp32 summation order."""
+    _check(K, dtype)
+    D = K.shape[-1]
+    out = np.empty(K.shape[:-1], dtype=np.float32)
+    lib().l2kv_oracle_key_sumsq_f32(_p(K), _DT[dtype], ctypes.c_int64(out.size), D, _p(out))
+    return out
+
+
+def select(key, keep, policy=0):
+    """Positions (ascending) of the `keep` lowest keys of a 1-D float64 array."""
+    key = np.ascontiguousarray(key, dtype=np.float64)
+    out = np.empty(keep, dtype=np.int32)
+    lib().l2kv_oracle_select(_p(key), int(key.size), int(keep), int(policy), _p(out))
+    return out
+
+
+def compress(K, V, dtype, lens, keep, uncompressed=(), key_mode=0, policy=0, t_cap_out=None,
+             nthreads=1):
+    """Whole-cache compression.  Returns dict(K_c, V_c, idx, key, kept_len)."""
+    _check(K, dtype)
+    _check(V, dtype)
+    B, L, H, T_cap, D = K.shape
+    lens, keep, unc = _i32(lens), _i32(keep), _i32(list(uncompressed))
+    if t_cap_out is None:
+        t_cap_out = T_cap
+    K_c = np.zeros((B, L, H, t_cap_out, D), dtype=K.dtype)
+    V_c = np.zeros_like(K_c)
+    idx = np.full((B, L, H, t_cap_out), -1, dtype=np.int32)
+    key = np.full((B, L, H, t_cap_out), np.nan, dtype=np.float64)
+    kept_len = np.zeros((B, L), dtype=np.int32)
+    rc = lib().l2kv_oracle_compress(
+        _p(K), _p(V), _DT[dtype], B, L, H, T_cap, D, _p(lens), _p(keep), _p(unc), int(unc.size),
+        int(key_mode), int(policy), int(t_cap_out), _p(K_c), _p(V_c), _p(idx), _p(key),
+        _p(kept_len), int(nthreads))
+    if rc != 0:
+        raise ValueError(f"oracle compress: bad argument ({rc})")
+    return dict(K_c=K_c, V_c=V_c, idx=idx, key=key, kept_len=kept_len)
+
+
+def attention(q, K_c, V_c, dtype, cur_len, scale=0.0, nthreads=1):
+    """Decode attention, fp64 two-pass softmax.  q [B, L, Hq, D] -> float64 [B, L, Hq, D]."""
+    _check(q, dtype)
+    _check(K_c, dtype)
+    _check(V_c, dtype)
+    B, L, Hkv, T_cap, D = K_c.shape
+    Hq = q.shape[2]
+    cur_len = _i32(cur_len).reshape(B, L)
+    out = np.empty((B, L, Hq, D), dtype=np.float64)
+    rc = lib().l2kv_oracle_attention(
+        _p(q), _p(K_c), _p(V_c), _DT[dtype], B, L, Hkv, Hq, T_cap, D, _p(cur_len),
+        ctypes.c_double(scale), _p(out), int(nthreads))
+    if rc != 0:
+        raise ValueError(f"oracle attention: bad argument ({rc})")
+    return out
+
+
+def append_evict(state, dtype, budget, uncompressed, k_new, v_new, pos_new, key_mode=0):
+    """One append/evict step, in place on state = dict(K_c, V_c, idx, key, cur_len).
+
+    Returns the oracle's status (0, or -2 when a row did not fit T_cap).
+    """
+    K_c, V_c = state["K_c"], state["V_c"]
+    _check(K_c, dtype)
+    _check(k_new, dtype)
+    _check(v_new, dtype)
+    B, L, H, T_cap, D = K_c.shape
+    budget, unc, pos_new = _i32(budget), _i32(list(uncompressed)), _i32(pos_new)
+    assert state["idx"].dtype == np.int32 and state["key"].dtype == np.float64
+    assert state["cur_len"].dtype == np.int32 and state["cur_len"].shape == (B, L)
+    return int(lib().l2kv_oracle_append_evict(
+        _p(K_c), _p(V_c), _p(state["idx"]), _p(state["key"]), _DT[dtype], B, L, H, T_cap, D,
+        _p(state["cur_len"]), _p(budget), _p(unc), int(unc.size), _p(k_new), _p(v_new),
+        _p(pos_new), int(key_mode)))

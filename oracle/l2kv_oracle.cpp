@@ -1,0 +1,345 @@
+// CPU oracle for L2-norm KV-cache compression and single-query decode attention.
+//
+// TEST INFRASTRUCTURE ONLY.  This file is the slow, plain statement of what the
+// GPU library must compute.  It shares no code with the CUDA path, is never
+// called by it, and may be used only by the tests, the smoke check and the
+// CPU-baseline leg of the benchmark.
+//
+// Every routine is the definition written out:
+//   * key norm        -- the paper's compression criterion, the L2 norm of each
+//                        cached key embedding (Abstract; Section 1; Section 3).
+//                        The ordering key is the sum of squares, which orders
+//                        tokens exactly as the norm does.
+//   * selection       -- "keep only the keys with the lowest L2 norm, and the
+//                        corresponding values" (Section 1), per layer and head
+//                        as the dropped set D_{l,h} of Eq. 5 is indexed
+//                        (Section 3): a full stable sort.
+//   * compaction      -- byte copies of the kept rows, in position order.
+//   * skipped layers  -- the listed layers are left uncompressed (Section 3,
+//                        last paragraph; Section 4, default = first two).
+//   * attention       -- Eq. 2 applied to the cached keys and values as in
+//                        Eq. 4, one query per head: softmax(q K^T / sqrt(d_k)) V,
+//                        two passes, fp64.
+//   * append / evict  -- "let the KV cache grow until a pre-defined length and
+//                        subsequently discard the tokens with the highest L2
+//                        norm" (Section 4, Language Modelling).
+//
+// Readings of points the paper leaves open (ties, rounding of keep counts,
+// slot reuse after eviction, ...) are listed beside each routine.
+//
+// Parity pins (tests, CPU only): brute-force enumeration on tiny inputs, closed
+// forms for norms, selection invariants, keep-all == plain attention, one-token
+// cache, equal keys -> mean of V, shift invariance, and streaming top-k ==
+// one-shot selection.  The *quality* of the heuristic on real models (the
+// paper's accuracy figures) needs weights and datasets: parity unpinned, and
+// out of scope.
+//
+// Layout: every cache tensor is dense [B, L, H, T_cap, D] with D contiguous.
+// dtype 0 = IEEE fp32, dtype 1 = bfloat16 stored as raw uint16.
+
+#include <algorithm>
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <numeric>
+#include <thread>
+#include <vector>
+
+namespace {
+
+constexpr int kF32 = 0;
+constexpr int kBF16 = 1;
+
+inline int elem_size(int dtype) { return dtype == kBF16 ? 2 : 4; }
+
+// bfloat16 is the upper half of an fp32 bit pattern: widening is exact.
+inline float bf16_to_float(uint16_t h) {
+  uint32_t u = static_cast<uint32_t>(h) << 16;
+  float f;
+  std::memcpy(&f, &u, sizeof f);
+  return f;
+}
+
+inline float load_elem_f32(const void* base, int dtype, int64_t i) {
+  if (dtype == kBF16) return bf16_to_float(static_cast<const uint16_t*>(base)[i]);
+  return static_cast<const float*>(base)[i];
+}
+
+inline double load_elem(const void* base, int dtype, int64_t i) {
+  return static_cast<double>(load_elem_f32(base, dtype, i));
+}
+
+// Sum of squares of one row, fp64, elements taken in index order.
+double row_sumsq_f64(const void* K, int dtype, int64_t row_off, int D) {
+  double s = 0.0;
+  for (int d = 0; d < D; ++d) {
+    const double x = load_elem(K, dtype, row_off + d);
+    s += x * x;
+  }
+  return s;
+}
+
+// Sum of squares of one row in single precision, in the summation order the
+// GPU library documents for its ordering key, so that the keep/evict decision
+// can also be compared with no tolerance band at all:
+//   * the row is cut into 16-byte pieces (8 bf16 or 4 fp32 elements);
+//   * each piece is summed front to back with fused multiply-adds,
+//     acc = fma(x, x, acc), starting from 0;
+//   * the P piece sums are combined by a butterfly: for off = P/2, P/4, .., 1
+//     every p[i] becomes p[i] + p[i ^ off]; the result is p[0].
+float row_sumsq_f32_ordered(const void* K, int dtype, int64_t row_off, int D) {
+  const int per_piece = 16 / elem_size(dtype);
+  const int P = D / per_piece;
+  std::vector<float> p(P), nxt(P);
+  for (int i = 0; i < P; ++i) {
+    float acc = 0.0f;
+    for (int e = 0; e < per_piece; ++e) {
+      const float x = load_elem_f32(K, dtype, row_off + int64_t(i) * per_piece + e);
+      acc = std::fmaf(x, x, acc);
+    }
+    p[i] = acc;
+  }
+  for (int off = P / 2; off >= 1; off /= 2) {
+    for (int i = 0; i < P; ++i) nxt[i] = p[i] + p[i ^ off];
+    p.swap(nxt);
+  }
+  return p[0];
+}
+
+inline double row_key(const void* K, int dtype, int64_t row_off, int D, int key_mode) {
+  if (key_mode == 1) return static_cast<double>(row_sumsq_f32_ordered(K, dtype, row_off, D));
+  return row_sumsq_f64(K, dtype, row_off, D);
+}
+
+// The `keep` positions with the smallest key; equal keys go to the lower
+// position (reading: the paper does not say how ties break).  policy 0 keeps
+// the lowest norms (the method); policy 1 keeps the highest (the paper's
+// ablation), ties again to the lower position.  Result sorted by position.
+void select_positions(const double* key, int T, int keep, int policy, int32_t* out) {
+  std::vector<int32_t> order(T);
+  std::iota(order.begin(), order.end(), 0);
+  if (policy == 0) {
+    std::stable_sort(order.begin(), order.end(),
+                     [&](int32_t a, int32_t b) { return key[a] < key[b]; });
+  } else {
+    std::stable_sort(order.begin(), order.end(),
+                     [&](int32_t a, int32_t b) { return key[a] > key[b]; });
+  }
+  std::vector<int32_t> kept(order.begin(), order.begin() + keep);
+  std::sort(kept.begin(), kept.end());
+  std::copy(kept.begin(), kept.end(), out);
+}
+
+bool in_list(const int32_t* list, int n, int v) {
+  for (int i = 0; i < n; ++i)
+    if (list[i] == v) return true;
+  return false;
+}
+
+// Run fn(unit) for unit in [0, n) on `nthreads` threads (units are independent).
+template <class F>
+void for_each_unit(int64_t n, int nthreads, F fn) {
+  if (nthreads <= 1) {
+    for (int64_t u = 0; u < n; ++u) fn(u);
+    return;
+  }
+  std::vector<std::thread> pool;
+  for (int w = 0; w < nthreads; ++w) {
+    pool.emplace_back([=]() {
+      for (int64_t u = w; u < n; u += nthreads) fn(u);
+    });
+  }
+  for (auto& t : pool) t.join();
+}
+
+}  // namespace
+
+extern "C" {
+
+int l2kv_oracle_hardware_threads() {
+  const unsigned n = std::thread::hardware_concurrency();
+  return n == 0 ? 1 : static_cast<int>(n);
+}
+
+// a1: sum of squares (fp64) of n_rows rows of D elements.
+void l2kv_oracle_key_sumsq(const void* K, int dtype, int64_t n_rows, int D, double* sumsq) {
+  for (int64_t r = 0; r < n_rows; ++r) sumsq[r] = row_sumsq_f64(K, dtype, r * D, D);
+}
+
+// a1 in the GPU library's documented single-precision order (see above).
+void l2kv_oracle_key_sumsq_f32(const void* K, int dtype, int64_t n_rows, int D, float* sumsq) {
+  for (int64_t r = 0; r < n_rows; ++r) sumsq[r] = row_sumsq_f32_ordered(K, dtype, r * D, D);
+}
+
+// a2 on a bare key array.
+void l2kv_oracle_select(const double* key, int T, int keep, int policy, int32_t* idx_out) {
+  select_positions(key, T, keep, policy, idx_out);
+}
+
+// Reading (rounding of a keep ratio): keep = ceil(ratio * len), clamped to
+// [1, len]; the paper quotes ratios only.
+int32_t l2kv_oracle_keep_count(int32_t len, double keep_ratio) {
+  if (len <= 0) return 0;
+  double k = std::ceil(keep_ratio * static_cast<double>(len));
+  if (k < 1.0) k = 1.0;
+  if (k > len) k = len;
+  return static_cast<int32_t>(k);
+}
+
+// a1-a4: compress a whole cache.
+//   K, V        [B, L, H, T_cap, D]
+//   len[b]      valid tokens of sequence b; keep[b] tokens kept per head in
+//               every compressed layer (the paper uses one ratio for all heads)
+//   uncompressed[0..n_unc)  layers copied whole (kept_len = len, identity map)
+//   key_mode    0: fp64 sums (the definition); 1: the GPU's fp32 order
+//   outputs     K_out, V_out [B, L, H, T_cap_out, D] (rows >= kept_len untouched),
+//               idx_out int32, key_out double [B, L, H, T_cap_out], kept_len [B, L]
+// Returns 0, or -1 if an argument is out of range.
+int l2kv_oracle_compress(const void* K, const void* V, int dtype, int B, int L, int H, int T_cap,
+                         int D, const int32_t* len, const int32_t* keep,
+                         const int32_t* uncompressed, int n_unc, int key_mode, int policy,
+                         int T_cap_out, void* K_out, void* V_out, int32_t* idx_out,
+                         double* key_out, int32_t* kept_len, int nthreads) {
+  for (int b = 0; b < B; ++b) {
+    if (len[b] < 0 || len[b] > T_cap) return -1;
+    if (keep[b] < 0 || keep[b] > len[b]) return -1;
+    if (keep[b] > T_cap_out) return -1;
+    if (n_unc > 0 && len[b] > T_cap_out) return -1;
+  }
+  const int es = elem_size(dtype);
+  for (int b = 0; b < B; ++b)
+    for (int l = 0; l < L; ++l)
+      kept_len[b * L + l] = in_list(uncompressed, n_unc, l) ? len[b] : keep[b];
+
+  for_each_unit(int64_t(B) * L * H, nthreads, [=](int64_t u) {
+    const int b = static_cast<int>(u / (int64_t(L) * H));
+    const int l = static_cast<int>((u / H) % L);
+    const int T = len[b];
+    const int n_keep = kept_len[b * L + l];
+    const int64_t in_row0 = u * T_cap;        // first row of this unit, in rows
+    const int64_t out_row0 = u * T_cap_out;
+    std::vector<double> key(T);
+    for (int t = 0; t < T; ++t) key[t] = row_key(K, dtype, (in_row0 + t) * D, D, key_mode);
+    std::vector<int32_t> kept(n_keep);
+    if (in_list(uncompressed, n_unc, l)) {
+      std::iota(kept.begin(), kept.end(), 0);
+    } else if (n_keep > 0) {
+      select_positions(key.data(), T, n_keep, policy, kept.data());
+    }
+    const size_t row_bytes = size_t(D) * es;
+    for (int j = 0; j < n_keep; ++j) {
+      const int64_t src = (in_row0 + kept[j]) * int64_t(row_bytes);
+      const int64_t dst = (out_row0 + j) * int64_t(row_bytes);
+      std::memcpy(static_cast<char*>(K_out) + dst, static_cast<const char*>(K) + src, row_bytes);
+      std::memcpy(static_cast<char*>(V_out) + dst, static_cast<const char*>(V) + src, row_bytes);
+      idx_out[out_row0 + j] = kept[j];
+      key_out[out_row0 + j] = key[kept[j]];
+    }
+  });
+  return 0;
+}
+
+// a5: one query per query head over the cached rows [0, cur_len[b, l]).
+//   q [B, L, Hq, D]; K_c, V_c [B, L, Hkv, T_cap, D]; out double [B, L, Hq, D]
+// Query head j reads KV head j / (Hq / Hkv) (reading: contiguous grouping; the
+// paper cites grouped-query attention without giving the mapping).  No mask:
+// a decode query sees every cached entry (Eq. 4).  scale <= 0 means
+// 1 / sqrt(D) (Eq. 2).  An empty cache gives zeros (reading).
+int l2kv_oracle_attention(const void* q, const void* K_c, const void* V_c, int dtype, int B, int L,
+                          int Hkv, int Hq, int T_cap, int D, const int32_t* cur_len, double scale,
+                          double* out, int nthreads) {
+  if (Hkv <= 0 || Hq % Hkv != 0) return -1;
+  const int G = Hq / Hkv;
+  const double sc = scale > 0.0 ? scale : 1.0 / std::sqrt(static_cast<double>(D));
+  for_each_unit(int64_t(B) * L * Hq, nthreads, [=](int64_t u) {
+    const int hq = static_cast<int>(u % Hq);
+    const int64_t bl = u / Hq;
+    const int n = cur_len[bl];
+    const int64_t kv_row0 = (bl * Hkv + hq / G) * T_cap;
+    double* o = out + u * D;
+    for (int d = 0; d < D; ++d) o[d] = 0.0;
+    if (n <= 0) return;
+    std::vector<double> z(n);
+    double m = -INFINITY;
+    for (int j = 0; j < n; ++j) {
+      double dot = 0.0;
+      for (int d = 0; d < D; ++d)
+        dot += load_elem(q, dtype, u * D + d) * load_elem(K_c, dtype, (kv_row0 + j) * D + d);
+      z[j] = dot * sc;
+      m = std::max(m, z[j]);
+    }
+    double denom = 0.0;
+    for (int j = 0; j < n; ++j) {
+      z[j] = std::exp(z[j] - m);
+      denom += z[j];
+    }
+    for (int j = 0; j < n; ++j) {
+      const double p = z[j] / denom;
+      for (int d = 0; d < D; ++d) o[d] += p * load_elem(V_c, dtype, (kv_row0 + j) * D + d);
+    }
+  });
+  return 0;
+}
+
+// a6: append one token per (b, l, h); over budget, evict the highest norm.
+//   K_c, V_c [B, L, H, T_cap, D], idx [B, L, H, T_cap], key_c double (same
+//   shape), cur_len [B, L] in/out, budget[b], k_new / v_new [B, L, H, D],
+//   pos_new[b] = original position of the new token.
+// Readings: (i) the new token competes like any other -- if it has the highest
+// norm it is the one dropped; (ii) among equal norms the highest position goes
+// first (the mirror of keeping the lower position); (iii) the new row takes the
+// evicted slot, so the cache stays dense but is no longer position-ordered and
+// idx carries the original positions; (iv) uncompressed layers only append.
+// Returns 0, or -2 if a row would not fit T_cap (nothing is written for it).
+int l2kv_oracle_append_evict(void* K_c, void* V_c, int32_t* idx, double* key_c, int dtype, int B,
+                             int L, int H, int T_cap, int D, int32_t* cur_len,
+                             const int32_t* budget, const int32_t* uncompressed, int n_unc,
+                             const void* k_new, const void* v_new, const int32_t* pos_new,
+                             int key_mode) {
+  const size_t row_bytes = size_t(D) * elem_size(dtype);
+  int status = 0;
+  for (int b = 0; b < B; ++b) {
+    for (int l = 0; l < L; ++l) {
+      const int n = cur_len[b * L + l];
+      const bool grow = in_list(uncompressed, n_unc, l) || n < budget[b];
+      if (grow && n >= T_cap) {
+        status = -2;
+        continue;
+      }
+      for (int h = 0; h < H; ++h) {
+        const int64_t u = (int64_t(b) * L + l) * H + h;
+        const double s_new = row_key(k_new, dtype, u * D, D, key_mode);
+        int slot;
+        if (grow) {
+          slot = n;
+        } else {
+          // arg-max of (key, position) over the stored entries and the new one
+          slot = -1;  // -1 = the new token itself
+          double best = s_new;
+          int32_t best_pos = pos_new[b];
+          for (int j = 0; j < n; ++j) {
+            const double s = key_c[u * T_cap + j];
+            const int32_t p = idx[u * T_cap + j];
+            if (s > best || (s == best && p > best_pos)) {
+              best = s;
+              best_pos = p;
+              slot = j;
+            }
+          }
+          if (slot < 0) continue;  // the new token is the one discarded
+        }
+        const int64_t dst = (u * T_cap + slot) * int64_t(row_bytes);
+        std::memcpy(static_cast<char*>(K_c) + dst,
+                    static_cast<const char*>(k_new) + u * int64_t(row_bytes), row_bytes);
+        std::memcpy(static_cast<char*>(V_c) + dst,
+                    static_cast<const char*>(v_new) + u * int64_t(row_bytes), row_bytes);
+        idx[u * T_cap + slot] = pos_new[b];
+        key_c[u * T_cap + slot] = s_new;
+      }
+      if (grow) cur_len[b * L + l] = n + 1;
+    }
+  }
+  return status;
+}
+
+}  // extern "C"
