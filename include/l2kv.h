@@ -1,0 +1,153 @@
+/* l2kv -- L2-norm KV-cache compression and decode attention for NVIDIA B200 (sm_100a).
+ *
+ * C ABI of the library.  The operations are those of "A Simple and Effective L2
+ * Norm-Based Strategy for KV Cache Compression" (arXiv 2406.11430):
+ *
+ *   - keep, per layer and head, only the cached keys with the lowest L2 norm and
+ *     the corresponding values (Section 1; Section 3, the dropped set D_{l,h} of Eq. 5),
+ *     leaving a caller-given list of layers uncompressed (Section 3, last paragraph;
+ *     Section 4: the first two layers by default);
+ *   - decode attention of one query per head over the cached keys and values
+ *     (Eq. 2 applied as in Eq. 4);
+ *   - a cache that grows to a pre-defined length and then discards the token with
+ *     the highest key norm at every step (Section 4, "Language Modelling Tasks").
+ *
+ * Conventions shared by every entry point
+ *   - Pointers named *_dev, and all tensor pointers (K, V, q, outputs, workspace),
+ *     are DEVICE pointers owned by the caller.  `const l2kv_layout*` and the
+ *     `uncompressed_layers` list are HOST pointers read before the call returns.
+ *   - The library allocates nothing and keeps no state.  Calls enqueue work on
+ *     `stream` (a cudaStream_t passed as void*; NULL = the default stream) and
+ *     return at once; outputs are valid in stream order.
+ *   - Return value: L2KV_OK (0) or a negative l2kv_status.  Arguments are checked on
+ *     the host and nothing is launched when a check fails.  Conditions only the
+ *     device can see (a cache row that does not fit t_cap) are recorded in the
+ *     status word at the start of the workspace: see l2kv_read_device_status.
+ *   - A cache tensor is described by l2kv_layout: logical shape
+ *     [batch, layers, kv_heads, t_cap, head_dim], head_dim contiguous, the other
+ *     strides in ELEMENTS.  Base pointers and every row must be 16-byte aligned
+ *     (all strides * element size multiples of 16).  Supported: bf16 and fp32
+ *     elements, head_dim 64 or 128; q_heads a multiple of kv_heads with
+ *     q_heads / kv_heads in {1, 2, 4, 8}.  Query head j reads KV head
+ *     j / (q_heads / kv_heads).
+ *   - `len_dev[b]` is the number of valid tokens of sequence b; `max_len` is a host
+ *     upper bound on every length the call will meet (it sizes grids and scratch;
+ *     device lengths above it are clamped to it).
+ *   - The ordering key of a cached key row is its fp32 sum of squares (monotone in
+ *     the L2 norm), accumulated in a fixed order: the row is cut into 16-byte
+ *     pieces; each piece is summed front to back with acc = fma(x, x, acc) from 0;
+ *     the P piece sums are combined by a butterfly (for off = P/2 .. 1:
+ *     p[i] += p[i ^ off]).  Tokens are ordered by (key, position): among equal keys
+ *     the lower position counts as the smaller.
+ */
+#ifndef L2KV_H_
+#define L2KV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  L2KV_OK = 0,
+  L2KV_ERR_INVALID_ARG = -1,         /* null pointer, non-positive size, bad enum          */
+  L2KV_ERR_UNSUPPORTED = -2,         /* dtype / head_dim / group size outside the list     */
+  L2KV_ERR_MISALIGNED = -3,          /* a base pointer or stride breaks 16-byte alignment  */
+  L2KV_ERR_WORKSPACE_TOO_SMALL = -4,
+  L2KV_ERR_OUT_OF_RANGE = -5,        /* max_len > t_cap, layer index outside [0, layers)   */
+  L2KV_ERR_CUDA = -6,                /* a CUDA runtime call failed                         */
+  L2KV_ERR_DEVICE_OVERFLOW = -7      /* device status: a row did not fit t_cap             */
+} l2kv_status;
+
+typedef enum { L2KV_F32 = 0, L2KV_BF16 = 1 } l2kv_dtype;
+
+/* Which tokens survive compression.  LOWEST is the paper's method; HIGHEST is
+ * its ablation baseline (Section 4: keeping the highest-norm tokens). */
+typedef enum { L2KV_KEEP_LOWEST_NORM = 0, L2KV_KEEP_HIGHEST_NORM = 1 } l2kv_policy;
+
+typedef struct {
+  int32_t batch, layers, kv_heads, q_heads, head_dim, t_cap;
+  int32_t dtype;                                     /* l2kv_dtype                          */
+  int32_t reserved;
+  int64_t stride_b, stride_l, stride_h, stride_t;    /* in elements; stride_t >= head_dim   */
+} l2kv_layout;
+
+/* Text for a status code (static storage, never NULL). */
+const char* l2kv_status_string(int status);
+
+/* keep = clamp(ceil(keep_ratio * len), 1, len) (0 when len == 0).  keep_ratio is the
+ * fraction KEPT, i.e. 1 - the paper's compression ratio (Section 4 quotes ratios
+ * of 0 % to 90 % dropped and gives no rounding rule; this one is the library's).
+ * Host only. */
+int l2kv_keep_count(int32_t len, double keep_ratio, int32_t* keep);
+
+/* Bytes of device scratch that suffice for any call on caches of this layout with
+ * lengths up to max_len.  The first 256 bytes hold the device status word; zero
+ * the workspace once before first use.  Host only. */
+int l2kv_workspace_bytes(const l2kv_layout* lay, int32_t max_len, size_t* bytes);
+
+/* Reads (and waits for) the device status word of a workspace: *status becomes
+ * L2KV_OK or L2KV_ERR_DEVICE_OVERFLOW.  Synchronises `stream`. */
+int l2kv_read_device_status(const void* workspace, void* stream, int32_t* status);
+
+/* Key norms (Abstract; Section 3): for every valid token t < len_dev[b] of every
+ * (b, l, h), sumsq_out[b,l,h,t] = sum_d K[b,l,h,t,d]^2 in the fixed order above, and,
+ * if norm_out is not NULL, norm_out = sqrt(sumsq).  Both outputs are dense fp32
+ * [batch, layers, kv_heads, t_cap]; entries at t >= len are left untouched. */
+int l2kv_key_norms(const void* K, const l2kv_layout* lay, const int32_t* len_dev, int32_t max_len,
+                   float* sumsq_out, float* norm_out, void* stream);
+
+/* Compression (Section 1; Section 3): for every (b, l, h) with l not in
+ * uncompressed_layers, keep the keep_dev[b] tokens that come first in the order
+ * (key, position) -- last, for L2KV_KEEP_HIGHEST_NORM, with ties still to the lower
+ * position -- and write them, in increasing position, to the first rows of the
+ * output cache:  K_out[b,l,h,j] = K[b,l,h,t_j], V_out likewise (bit copies),
+ * idx_out[b,l,h,j] = t_j, sumsq_out[b,l,h,j] = key of t_j, kept_len_dev[b,l] =
+ * keep_dev[b].  Layers in uncompressed_layers (host array, may be NULL when
+ * n_uncompressed == 0) are copied whole: kept_len = len, idx = identity.
+ * Requires 0 <= keep_dev[b] <= len_dev[b] <= max_len <= in->t_cap and kept_len <=
+ * out->t_cap (the host checks what it can see: max_len and the layouts; a device
+ * value outside its range is clamped).  `in` and `out` must agree in batch, layers,
+ * kv_heads, head_dim and dtype, and the output tensors must not overlap the
+ * inputs.  idx_out / sumsq_out are dense [batch, layers, kv_heads, out->t_cap];
+ * rows at and beyond kept_len are left untouched. */
+int l2kv_select_compact(const void* K, const void* V, const l2kv_layout* in,
+                        const int32_t* len_dev, const int32_t* keep_dev, int32_t max_len,
+                        const int32_t* uncompressed_layers, int32_t n_uncompressed, int32_t policy,
+                        void* K_out, void* V_out, const l2kv_layout* out, int32_t* idx_out,
+                        float* sumsq_out, int32_t* kept_len_dev, void* workspace,
+                        size_t workspace_bytes, void* stream);
+
+/* Decode attention (Eq. 2 over the cache, Eq. 4): for every (b, l, query head j)
+ *   out[b,l,j,:] = sum_i softmax_i( scale * q[b,l,j,:] . K_c[b,l,j/G,i,:] ) * V_c[b,l,j/G,i,:]
+ * over rows i < cur_len_dev[b,l], G = q_heads / kv_heads, no mask.  q is dense
+ * [batch, layers, q_heads, head_dim] in the cache's dtype; out is dense fp32 of the
+ * same shape.  scale <= 0 selects 1 / sqrt(head_dim).  Products and sums are fp32.
+ * An empty cache (cur_len == 0) gives zeros.  cur_len <= max_len <= lay->t_cap. */
+int l2kv_decode_attention(const void* q, const void* K_c, const void* V_c, const l2kv_layout* lay,
+                          const int32_t* cur_len_dev, int32_t max_len, float scale, float* out,
+                          void* workspace, size_t workspace_bytes, void* stream);
+
+/* Budget-maintained cache (Section 4, "Language Modelling Tasks"): append one new
+ * token per (b, l, h).  If l is uncompressed or cur_len_dev[b,l] < budget_dev[b] the
+ * row is appended at slot cur_len and cur_len grows by one.  Otherwise the entry
+ * that comes last in the order (key, position) among the stored ones and the new
+ * one is discarded: if that is the new token nothing changes, else the new row
+ * overwrites the discarded slot (the cache stays dense, no longer position-
+ * ordered; idx keeps original positions).  k_new, v_new are dense
+ * [batch, layers, kv_heads, head_dim]; pos_new_dev[b] is the new token's position.
+ * K_c, V_c, idx, sumsq_c and cur_len_dev are updated in place (idx and sumsq_c dense
+ * [batch, layers, kv_heads, lay->t_cap]).  A row that would land at slot >= t_cap is
+ * not written and sets the device status word to L2KV_ERR_DEVICE_OVERFLOW. */
+int l2kv_append_evict(void* K_c, void* V_c, int32_t* idx, float* sumsq_c, const l2kv_layout* lay,
+                      int32_t* cur_len_dev, const int32_t* budget_dev,
+                      const int32_t* uncompressed_layers, int32_t n_uncompressed,
+                      const void* k_new, const void* v_new, const int32_t* pos_new_dev,
+                      void* workspace, size_t workspace_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* L2KV_H_ */

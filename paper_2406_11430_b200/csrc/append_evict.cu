@@ -1,0 +1,131 @@
+// Budget-maintained cache: append one token per (b, l, h); once a sequence holds `budget`
+// tokens, discard the entry that comes last in the order (key, position).
+//
+// One CTA per (b, l) walks that layer's KV heads, so the shared length cur_len[b, l] is
+// read before and written after all of them by the same CTA.  Per head: the new key's
+// ordering key (same fixed summation order as the norm pass), a block-wide arg-max over
+// the stored keys packed as (key bits << 32 | position), then two 16-byte-piece row copies.
+#include "common.cuh"
+
+namespace l2kv {
+
+constexpr int kAppendThreads = 256;
+
+template <typename T, int D>
+__global__ void __launch_bounds__(kAppendThreads)
+append_evict_kernel(T* __restrict__ K, T* __restrict__ V, int32_t* __restrict__ idx,
+                    float* __restrict__ sumsq, Geom g, int32_t* __restrict__ cur_len_dev,
+                    const int32_t* __restrict__ budget_dev, LayerMask unc,
+                    const T* __restrict__ k_new, const T* __restrict__ v_new,
+                    const int32_t* __restrict__ pos_new_dev, int32_t* __restrict__ status_word) {
+  constexpr int EPV = Elem<T>::kPerVec;
+  constexpr int LPR = D / EPV;
+  constexpr int NW = kAppendThreads / 32;
+  __shared__ unsigned long long s_best[NW];
+  __shared__ int s_slot;
+
+  const long long bl = blockIdx.x;
+  const int l = (int)(bl % g.L);
+  const int b = (int)(bl / g.L);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int n = max(0, min(cur_len_dev[bl], g.t_cap));
+  const bool grow = unc.test(l) || n < budget_dev[b];
+  if (grow && n >= g.t_cap) {
+    if (tid == 0) atomicExch(status_word, (int)L2KV_ERR_DEVICE_OVERFLOW);
+    return;
+  }
+  const int pos_new = pos_new_dev[b];
+
+  for (int h = 0; h < g.H; ++h) {
+    const long long unit = bl * g.H + h;
+    // Warp 0 holds the new rows: lanes < LPR own one 16-byte piece each.
+    uint4 vk = make_uint4(0, 0, 0, 0), vv = make_uint4(0, 0, 0, 0);
+    float s_new = 0.f;
+    if (warp == 0) {
+      if (lane < LPR) {
+        vk = *reinterpret_cast<const uint4*>(k_new + unit * D + lane * EPV);
+        vv = *reinterpret_cast<const uint4*>(v_new + unit * D + lane * EPV);
+      }
+      s_new = piece_sumsq_reduce<T, LPR>(vk);            // lanes < LPR end with the row's key
+      s_new = __shfl_sync(0xffffffffu, s_new, 0);
+    }
+    int slot = n;
+    if (!grow) {
+      const float* key = sumsq + unit * g.t_cap;
+      const int32_t* pos = idx + unit * g.t_cap;
+      unsigned long long best = 0ull;
+      int best_j = -1;
+      for (int j = tid; j < n; j += kAppendThreads) {
+        const unsigned long long c =
+            ((unsigned long long)__float_as_uint(key[j]) << 32) | (uint32_t)pos[j];
+        if (best_j < 0 || c > best) { best = c; best_j = j; }
+      }
+      unsigned long long wbest = best;
+#pragma unroll
+      for (int off = 16; off >= 1; off >>= 1) {
+        const unsigned long long o = __shfl_xor_sync(0xffffffffu, wbest, off);
+        wbest = o > wbest ? o : wbest;
+      }
+      if (lane == 0) s_best[warp] = wbest;
+      if (tid == 0) s_slot = -1;
+      __syncthreads();
+      unsigned long long top = s_best[0];
+#pragma unroll
+      for (int w = 1; w < NW; ++w) top = s_best[w] > top ? s_best[w] : top;
+      // (key, position) pairs are distinct, so at most one thread owns the maximum.
+      if (best_j >= 0 && best == top) s_slot = best_j;
+      __syncthreads();
+      slot = s_slot;
+      if (warp == 0) {
+        const unsigned long long c_new =
+            ((unsigned long long)__float_as_uint(s_new) << 32) | (uint32_t)pos_new;
+        if (slot < 0 || c_new > top) slot = -1;          // the newcomer is the one discarded
+      }
+      __syncthreads();                                   // s_best / s_slot are reused next head
+    }
+    if (warp == 0 && slot >= 0 && lane < LPR) {
+      const long long row = b * g.sb + l * g.sl + h * g.sh + (long long)slot * g.st + lane * EPV;
+      *reinterpret_cast<uint4*>(K + row) = vk;
+      *reinterpret_cast<uint4*>(V + row) = vv;
+      if (lane == 0) {
+        idx[unit * g.t_cap + slot] = pos_new;
+        sumsq[unit * g.t_cap + slot] = s_new;
+      }
+    }
+  }
+  if (grow && tid == 0) cur_len_dev[bl] = n + 1;
+}
+
+template <typename T, int D>
+static int launch_ae_t(void* K, void* V, int32_t* idx, float* sumsq, const Geom& g,
+                       int32_t* cur_len_dev, const int32_t* budget_dev, const LayerMask& unc,
+                       const void* k_new, const void* v_new, const int32_t* pos_new_dev,
+                       int32_t* status_word, cudaStream_t s) {
+  const long long blocks = (long long)g.B * g.L;
+  if (blocks == 0 || g.H == 0) return L2KV_OK;
+  if (blocks > 0x7fffffffLL) return L2KV_ERR_OUT_OF_RANGE;
+  append_evict_kernel<T, D><<<(unsigned)blocks, kAppendThreads, 0, s>>>(
+      static_cast<T*>(K), static_cast<T*>(V), idx, sumsq, g, cur_len_dev, budget_dev, unc,
+      static_cast<const T*>(k_new), static_cast<const T*>(v_new), pos_new_dev, status_word);
+  return cudaGetLastError() == cudaSuccess ? L2KV_OK : L2KV_ERR_CUDA;
+}
+
+int launch_append_evict(void* K, void* V, int32_t* idx, float* sumsq, const Geom& g, int dtype,
+                        int32_t* cur_len_dev, const int32_t* budget_dev, const LayerMask& unc,
+                        const void* k_new, const void* v_new, const int32_t* pos_new_dev,
+                        int32_t* status_word, cudaStream_t s) {
+#define L2KV_AE(T, D)                                                                            \
+  return launch_ae_t<T, D>(K, V, idx, sumsq, g, cur_len_dev, budget_dev, unc, k_new, v_new,      \
+                           pos_new_dev, status_word, s)
+  if (dtype == L2KV_BF16) {
+    if (g.D == 128) L2KV_AE(__nv_bfloat16, 128);
+    if (g.D == 64) L2KV_AE(__nv_bfloat16, 64);
+  } else if (dtype == L2KV_F32) {
+    if (g.D == 128) L2KV_AE(float, 128);
+    if (g.D == 64) L2KV_AE(float, 64);
+  }
+#undef L2KV_AE
+  return L2KV_ERR_UNSUPPORTED;
+}
+
+}  // namespace l2kv

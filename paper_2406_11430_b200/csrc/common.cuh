@@ -1,0 +1,149 @@
+// Shared device/host helpers of the l2kv kernels (sm_100a).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <type_traits>
+
+#include "l2kv.h"
+
+namespace l2kv {
+
+constexpr int kStatusBytes = 256;      // device status word lives at the start of a workspace
+constexpr int kMaxLayers = 1024;       // size of the uncompressed-layer bit mask
+constexpr int kGatherChunk = 512;      // input tokens per gather CTA / per scan chunk
+constexpr int kMaxChunks = 4096;       // kGatherChunk * kMaxChunks tokens per unit at most
+constexpr int kDecodeChunk = 1024;     // cached tokens per split of decode attention
+
+// Cache geometry handed to kernels by value (strides in elements).
+struct Geom {
+  int B, L, H, Hq, D, t_cap;
+  long long sb, sl, sh, st;
+};
+
+struct LayerMask {
+  uint32_t w[kMaxLayers / 32];
+  __host__ __device__ bool test(int l) const { return (w[l >> 5] >> (l & 31)) & 1u; }
+};
+
+inline Geom make_geom(const l2kv_layout& a) {
+  Geom g;
+  g.B = a.batch; g.L = a.layers; g.H = a.kv_heads; g.Hq = a.q_heads; g.D = a.head_dim;
+  g.t_cap = a.t_cap;
+  g.sb = a.stride_b; g.sl = a.stride_l; g.sh = a.stride_h; g.st = a.stride_t;
+  return g;
+}
+
+__host__ __device__ inline long long round_up_ll(long long x, long long m) {
+  return (x + m - 1) / m * m;
+}
+
+// Workspace carve-up (offsets in bytes), identical for every entry point.
+struct WorkspacePlan {
+  size_t sumsq_off;      // float  [units][ld_sumsq]         ordering keys of the input cache
+  size_t unit_off;       // uint32 [units][4]                threshold, admitted ties, kept, flags
+  size_t chunk_off;      // int32  [units][n_chunks][2]      slot base / equal-keys-before per chunk
+  size_t partial_off;    // float  [B*L*Hq][n_splits][D + 2] decode partials
+  size_t total;
+  long long ld_sumsq;
+  int n_chunks, n_splits;
+};
+
+inline WorkspacePlan plan_workspace(const l2kv_layout& a, int max_len) {
+  WorkspacePlan p;
+  const long long units = (long long)a.batch * a.layers * a.kv_heads;
+  p.ld_sumsq = round_up_ll(max_len > 0 ? max_len : 1, 64);
+  p.n_chunks = (int)((max_len + kGatherChunk - 1) / kGatherChunk);
+  if (p.n_chunks < 1) p.n_chunks = 1;
+  p.n_splits = (int)((max_len + kDecodeChunk - 1) / kDecodeChunk);
+  if (p.n_splits < 1) p.n_splits = 1;
+  size_t off = kStatusBytes;
+  p.sumsq_off = off;   off += (size_t)round_up_ll(units * p.ld_sumsq * 4, 256);
+  p.unit_off = off;    off += (size_t)round_up_ll(units * 16, 256);
+  p.chunk_off = off;   off += (size_t)round_up_ll(units * p.n_chunks * 8, 256);
+  p.partial_off = off;
+  off += (size_t)round_up_ll((long long)a.batch * a.layers * a.q_heads * p.n_splits *
+                                 (a.head_dim + 2) * 4, 256);
+  p.total = off;
+  return p;
+}
+
+// ---- element access ------------------------------------------------------------------
+
+template <typename T> struct Elem;
+template <> struct Elem<float> {
+  static constexpr int kPerVec = 4;                      // elements in a 16-byte piece
+  static constexpr int kDtype = L2KV_F32;
+  __device__ static void unpack(const uint4& v, float (&x)[4]) {
+    x[0] = __uint_as_float(v.x); x[1] = __uint_as_float(v.y);
+    x[2] = __uint_as_float(v.z); x[3] = __uint_as_float(v.w);
+  }
+};
+template <> struct Elem<__nv_bfloat16> {
+  static constexpr int kPerVec = 8;
+  static constexpr int kDtype = L2KV_BF16;
+  // bf16 is the upper half of an fp32: widening is a shift / mask, exact.
+  __device__ static void unpack(const uint4& v, float (&x)[8]) {
+    x[0] = __uint_as_float(v.x << 16); x[1] = __uint_as_float(v.x & 0xffff0000u);
+    x[2] = __uint_as_float(v.y << 16); x[3] = __uint_as_float(v.y & 0xffff0000u);
+    x[4] = __uint_as_float(v.z << 16); x[5] = __uint_as_float(v.z & 0xffff0000u);
+    x[6] = __uint_as_float(v.w << 16); x[7] = __uint_as_float(v.w & 0xffff0000u);
+  }
+};
+
+// 16-byte streaming load: read-only path, no L1 allocation.
+__device__ __forceinline__ uint4 ld_stream(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+
+__device__ __forceinline__ void st_stream(void* p, const uint4& v) {
+  asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};"
+               :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+
+// The ordering key of a row: every lane of the LPR-lane group that owns the row passes
+// its 16-byte piece; all lanes return the same sum.  Fixed order: piece front to back
+// by fma, then a butterfly over the pieces (off = LPR/2 .. 1).  Must be reached by
+// whole warps.
+template <typename T, int LPR>
+__device__ __forceinline__ float piece_sumsq_reduce(const uint4& v) {
+  float x[Elem<T>::kPerVec];
+  Elem<T>::unpack(v, x);
+  float acc = 0.f;
+#pragma unroll
+  for (int e = 0; e < Elem<T>::kPerVec; ++e) acc = __fmaf_rn(x[e], x[e], acc);
+#pragma unroll
+  for (int off = LPR / 2; off >= 1; off >>= 1) acc = acc + __shfl_xor_sync(0xffffffffu, acc, off);
+  return acc;
+}
+
+// Total order on (key bits, position) used everywhere: non-negative floats order as
+// their bit patterns.  For the keep-highest policy the bits are complemented.
+__device__ __forceinline__ uint32_t order_bits(float sumsq, int policy) {
+  const uint32_t b = __float_as_uint(sumsq);
+  return policy == L2KV_KEEP_HIGHEST_NORM ? ~b : b;
+}
+
+// Launchers, one per source file (arguments already validated by the C entry points).
+int launch_key_norms(const void* K, const Geom& g, int dtype, const int32_t* len_dev, int max_len,
+                     float* sumsq, long long ld_sumsq, float* norm_out, const LayerMask* skip,
+                     cudaStream_t s);
+int launch_select_compact(const void* K, const void* V, const Geom& gi, int dtype,
+                          const int32_t* len_dev, const int32_t* keep_dev, int max_len,
+                          const LayerMask& unc, int policy, void* K_out, void* V_out,
+                          const Geom& go, int32_t* idx_out, float* sumsq_out, int32_t* kept_len_dev,
+                          char* ws, const WorkspacePlan& plan, cudaStream_t s);
+int launch_decode_attention(const void* q, const void* K, const void* V, const Geom& g, int dtype,
+                            const int32_t* cur_len_dev, int max_len, float scale, float* out,
+                            char* ws, const WorkspacePlan& plan, cudaStream_t s);
+int launch_append_evict(void* K, void* V, int32_t* idx, float* sumsq, const Geom& g, int dtype,
+                        int32_t* cur_len_dev, const int32_t* budget_dev, const LayerMask& unc,
+                        const void* k_new, const void* v_new, const int32_t* pos_new_dev,
+                        int32_t* status_word, cudaStream_t s);
+
+}  // namespace l2kv
