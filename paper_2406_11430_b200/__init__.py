@@ -1,0 +1,10 @@
+"""l2kv: L2-norm KV-cache compression and decode attention on B200 (sm_100a).
+
+Thin Python front end of the C library ``libl2kv.so``: the functions here only
+marshal torch tensors into pointers and sizes; every step runs in the library's
+CUDA kernels.  There is no CPU fallback -- a missing library is an ImportError.
+"""
+from .binding import (L2KVError, Layout, key_norms, select_compact, decode_attention,  # noqa: F401
+                      append_evict, keep_count, workspace_bytes, new_workspace,
+                      read_device_status, status_string, library_path, lib,
+                      KEEP_LOWEST_NORM, KEEP_HIGHEST_NORM)

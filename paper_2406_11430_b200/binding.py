@@ -1,0 +1,163 @@
+"""ctypes binding of libl2kv.so: argument marshalling only."""
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libl2kv.so")
+_LIB = None
+
+KEEP_LOWEST_NORM = 0
+KEEP_HIGHEST_NORM = 1
+_DTYPE = {torch.float32: 0, torch.bfloat16: 1}
+
+
+class L2KVError(RuntimeError):
+    def __init__(self, status, where):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} ({status})")
+
+
+class _CLayout(ctypes.Structure):
+    _fields_ = [("batch", ctypes.c_int32), ("layers", ctypes.c_int32),
+                ("kv_heads", ctypes.c_int32), ("q_heads", ctypes.c_int32),
+                ("head_dim", ctypes.c_int32), ("t_cap", ctypes.c_int32),
+                ("dtype", ctypes.c_int32), ("reserved", ctypes.c_int32),
+                ("stride_b", ctypes.c_int64), ("stride_l", ctypes.c_int64),
+                ("stride_h", ctypes.c_int64), ("stride_t", ctypes.c_int64)]
+
+
+def library_path():
+    return _LIB_PATH
+
+
+def lib():
+    """The loaded C library.  Raises if it has not been built: nothing else can run."""
+    global _LIB
+    if _LIB is None:
+        if not os.path.exists(_LIB_PATH):
+            raise ImportError(f"{_LIB_PATH} is missing: run `python -m paper_2406_11430_b200.build` "
+                              "(needs nvcc); there is no fallback path")
+        L = ctypes.CDLL(_LIB_PATH)
+        vp, i32, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_size_t
+        lay = ctypes.POINTER(_CLayout)
+        L.l2kv_status_string.restype = ctypes.c_char_p
+        L.l2kv_status_string.argtypes = [ctypes.c_int]
+        L.l2kv_keep_count.argtypes = [i32, ctypes.c_double, ctypes.POINTER(i32)]
+        L.l2kv_workspace_bytes.argtypes = [lay, i32, ctypes.POINTER(sz)]
+        L.l2kv_read_device_status.argtypes = [vp, vp, ctypes.POINTER(i32)]
+        L.l2kv_key_norms.argtypes = [vp, lay, vp, i32, vp, vp, vp]
+        L.l2kv_select_compact.argtypes = [vp, vp, lay, vp, vp, i32, ctypes.POINTER(i32), i32, i32,
+                                          vp, vp, lay, vp, vp, vp, vp, sz, vp]
+        L.l2kv_decode_attention.argtypes = [vp, vp, vp, lay, vp, i32, ctypes.c_float, vp, vp, sz, vp]
+        L.l2kv_append_evict.argtypes = [vp, vp, vp, vp, lay, vp, vp, ctypes.POINTER(i32), i32,
+                                        vp, vp, vp, vp, sz, vp]
+        for name in ("l2kv_keep_count", "l2kv_workspace_bytes", "l2kv_read_device_status",
+                     "l2kv_key_norms", "l2kv_select_compact", "l2kv_decode_attention",
+                     "l2kv_append_evict"):
+            getattr(L, name).restype = ctypes.c_int
+        _LIB = L
+    return _LIB
+
+
+def status_string(status):
+    return lib().l2kv_status_string(int(status)).decode()
+
+
+def _check(rc, where):
+    if rc != 0:
+        raise L2KVError(rc, where)
+
+
+class Layout:
+    """Geometry of a cache tensor [B, L, Hkv, t_cap, D] (D contiguous), taken from a tensor."""
+
+    def __init__(self, cache, q_heads=None):
+        if cache.dim() != 5 or cache.stride(4) != 1:
+            raise ValueError("cache must be [B, L, Hkv, t_cap, D] with D contiguous")
+        if cache.dtype not in _DTYPE:
+            raise ValueError(f"unsupported dtype {cache.dtype}")
+        B, L, H, T, D = cache.shape
+        self.c = _CLayout(B, L, H, H if q_heads is None else q_heads, D, T, _DTYPE[cache.dtype], 0,
+                          cache.stride(0), cache.stride(1), cache.stride(2), cache.stride(3))
+
+    def ref(self):
+        return ctypes.byref(self.c)
+
+
+def _ptr(t):
+    return ctypes.c_void_p(0 if t is None else t.data_ptr())
+
+
+def _stream(stream):
+    if stream is None:
+        if not torch.cuda.is_available():        # host-only calls (argument checks) need no stream
+            return ctypes.c_void_p(0)
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def _layers(layers):
+    layers = list(layers or ())
+    arr = (ctypes.c_int32 * max(1, len(layers)))(*layers)
+    return arr, len(layers)
+
+
+def keep_count(length, keep_ratio):
+    out = ctypes.c_int32(0)
+    _check(lib().l2kv_keep_count(int(length), float(keep_ratio), ctypes.byref(out)), "l2kv_keep_count")
+    return out.value
+
+
+def workspace_bytes(layout, max_len):
+    out = ctypes.c_size_t(0)
+    _check(lib().l2kv_workspace_bytes(layout.ref(), int(max_len), ctypes.byref(out)),
+           "l2kv_workspace_bytes")
+    return out.value
+
+
+def new_workspace(layout, max_len, device):
+    """A zeroed device buffer large enough for any call on this layout."""
+    return torch.zeros(workspace_bytes(layout, max_len), dtype=torch.uint8, device=device)
+
+
+def read_device_status(workspace, stream=None):
+    out = ctypes.c_int32(0)
+    _check(lib().l2kv_read_device_status(_ptr(workspace), _stream(stream), ctypes.byref(out)),
+           "l2kv_read_device_status")
+    return out.value
+
+
+def key_norms(K, len_dev, max_len, sumsq_out, norm_out=None, stream=None):
+    lay = Layout(K)
+    _check(lib().l2kv_key_norms(_ptr(K), lay.ref(), _ptr(len_dev), int(max_len), _ptr(sumsq_out),
+                                _ptr(norm_out), _stream(stream)), "l2kv_key_norms")
+
+
+def select_compact(K, V, len_dev, keep_dev, max_len, uncompressed_layers, K_out, V_out, idx_out,
+                   sumsq_out, kept_len_dev, workspace, policy=KEEP_LOWEST_NORM, stream=None):
+    lin, lout = Layout(K), Layout(K_out)
+    arr, n = _layers(uncompressed_layers)
+    _check(lib().l2kv_select_compact(
+        _ptr(K), _ptr(V), lin.ref(), _ptr(len_dev), _ptr(keep_dev), int(max_len), arr, n,
+        int(policy), _ptr(K_out), _ptr(V_out), lout.ref(), _ptr(idx_out), _ptr(sumsq_out),
+        _ptr(kept_len_dev), _ptr(workspace), workspace.numel(), _stream(stream)),
+        "l2kv_select_compact")
+
+
+def decode_attention(q, K_c, V_c, cur_len_dev, max_len, out, workspace, scale=0.0, stream=None):
+    lay = Layout(K_c, q_heads=q.shape[2])
+    _check(lib().l2kv_decode_attention(
+        _ptr(q), _ptr(K_c), _ptr(V_c), lay.ref(), _ptr(cur_len_dev), int(max_len), float(scale),
+        _ptr(out), _ptr(workspace), workspace.numel(), _stream(stream)), "l2kv_decode_attention")
+
+
+def append_evict(K_c, V_c, idx, sumsq_c, cur_len_dev, budget_dev, uncompressed_layers, k_new, v_new,
+                 pos_new_dev, workspace, stream=None):
+    lay = Layout(K_c)
+    arr, n = _layers(uncompressed_layers)
+    _check(lib().l2kv_append_evict(
+        _ptr(K_c), _ptr(V_c), _ptr(idx), _ptr(sumsq_c), lay.ref(), _ptr(cur_len_dev),
+        _ptr(budget_dev), arr, n, _ptr(k_new), _ptr(v_new), _ptr(pos_new_dev), _ptr(workspace),
+        workspace.numel(), _stream(stream)), "l2kv_append_evict")
