@@ -12,7 +12,7 @@ def i32(x, device=DEV):
     return torch.tensor(np.asarray(x, dtype=np.int32), dtype=torch.int32, device=device)
 
 
-def gpu_compress(l2, K, V, lens, keep, uncompressed=(), policy=0, t_cap_out=None, max_len=None):
+def gpu_compress(l2, K, V, lens, keep, unc=(), policy=0, t_cap_out=None, max_len=None):
     """K, V: device tensors [B, L, H, T_cap, D].  Returns (device dict, numpy dict)."""
     B, L, H, T_cap, D = K.shape
     t_cap_out = T_cap if t_cap_out is None else t_cap_out
@@ -23,7 +23,7 @@ def gpu_compress(l2, K, V, lens, keep, uncompressed=(), policy=0, t_cap_out=None
     sumsq = torch.full((B, L, H, t_cap_out), float("nan"), dtype=torch.float32, device=K.device)
     kept_len = torch.zeros((B, L), dtype=torch.int32, device=K.device)
     ws = l2.new_workspace(l2.Layout(K), max_len, K.device)
-    l2.select_compact(K, V, i32(lens), i32(keep), max_len, uncompressed, K_c, V_c, idx, sumsq,
+    l2.select_compact(K, V, i32(lens), i32(keep), max_len, unc, K_c, V_c, idx, sumsq,
                       kept_len, ws, policy=policy)
     torch.cuda.synchronize()
     dev = dict(K_c=K_c, V_c=V_c, idx=idx, sumsq=sumsq, kept_len=kept_len)
