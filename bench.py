@@ -1,0 +1,389 @@
+#!/usr/bin/env python
+"""Benchmark of the l2kv hot path on B200.
+
+One step = one pass of the whole path over one synthetic batch of the Llama-3-8B
+32k-context workload: a compression pass over the full cache (key norms, selection,
+compaction; the uncompressed layers are copied) followed by the workload's 64
+single-query decode-attention steps over the compressed cache.  The metric is the
+throughput of KV bytes the algorithm has to move (GB/s), reported with the fraction
+of the HBM roofline, plus decode tokens/s.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl l2kv|reference]
+
+With N > 1 (under torchrun) every rank runs the same per-GPU workload on its own
+batch: the path shards over independent (batch, layer, head) units with no exchange,
+so there is no collective on the data path (weak scaling).
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import synth  # noqa: E402
+
+GIB = 1 << 30
+METRIC = "compress + decode GB/s of KV read and % of B200 HBM peak; decode tokens/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def workload(args):
+    w = synth.WORKLOADS[2]
+    if args.layers:
+        w = w.scaled(L=args.layers)
+    if args.context:
+        w = w.scaled(T=args.context)
+    if args.decode_steps:
+        w = w.scaled(decode_steps=args.decode_steps)
+    return w
+
+
+def algorithmic_bytes(w):
+    """Bytes the method must move, per step, from the shapes alone."""
+    e, row = w.elem_bytes, w.D * w.elem_bytes
+    keep = int(np.ceil(w.keep_ratio * w.T))
+    n_unc = len([l for l in w.uncompressed if l < w.L])
+    units_c = w.B * (w.L - n_unc) * w.Hkv
+    units_u = w.B * n_unc * w.Hkv
+    # compressed unit: read K once for the norms, read kept K and V rows, write them, plus
+    # the index map and stored keys; uncompressed unit: read and write K and V once
+    compress = units_c * (w.T * row + 4 * keep * row + 8 * keep) + units_u * (4 * w.T * row + 8 * w.T)
+    decode = (units_c * keep + units_u * w.T) * 2 * row + w.B * w.L * w.Hq * w.D * (e + 4)
+    return compress, decode, keep
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+        try:
+            self.p = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-i", str(index), "-lms", "100"], stdout=self.f, stderr=subprocess.DEVNULL)
+        except OSError:
+            pass
+
+    def stop(self):
+        if self.p is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.p.terminate()
+        self.p.wait()
+        self.f.seek(0)
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.f:
+            c = [x.strip() for x in line.split(",")]
+            if len(c) < 8:
+                continue
+            try:
+                sm.append(float(c[0])); smax.append(float(c[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, c[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        self.f.close()
+        os.unlink(self.f.name)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(smax) if smax else None, "samples": len(sm),
+                "reasons": sorted(reasons)}
+
+
+def dist_setup(n):
+    if n <= 1:
+        return 0, 1, 0
+    import torch.distributed as dist
+    rank, world = int(os.environ["RANK"]), int(os.environ["WORLD_SIZE"])
+    local = int(os.environ.get("LOCAL_RANK", rank))
+    torch.cuda.set_device(local)
+    dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    return rank, world, local
+
+
+def max_over_ranks(x, world, device):
+    if world <= 1:
+        return x
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def barrier(world):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+    torch.cuda.synchronize()
+
+
+# ------------------------------------------------------------------------------ GPU arm
+
+class Job:
+    """Device-resident state of one rank: the full cache, the compressed cache, queries."""
+
+    def __init__(self, w, device, rank):
+        import paper_2406_11430_b200 as l2
+        self.l2, self.w, self.dev = l2, w, device
+        ws = w.scaled(seed=w.seed + 1000 * rank)          # each rank its own batch
+        self.K, self.V = synth.make_cache(ws, device)
+        shape = (w.B, w.L, w.Hkv, w.T, w.D)
+        self.K_c = torch.zeros(shape, dtype=w.torch_dtype, device=device)
+        self.V_c = torch.zeros_like(self.K_c)
+        self.idx = torch.zeros(shape[:4], dtype=torch.int32, device=device)
+        self.sumsq = torch.zeros(shape[:4], dtype=torch.float32, device=device)
+        self.cur = torch.zeros((w.B, w.L), dtype=torch.int32, device=device)
+        self.keep_n = int(np.ceil(w.keep_ratio * w.T))
+        self.lens = torch.full((w.B,), w.T, dtype=torch.int32, device=device)
+        self.keep = torch.full((w.B,), self.keep_n, dtype=torch.int32, device=device)
+        self.unc = tuple(l for l in w.uncompressed if l < w.L)
+        self.q = torch.stack([synth.make_query(ws, s, device) for s in range(w.decode_steps)])
+        self.out = torch.zeros((w.decode_steps, w.B, w.L, w.Hq, w.D), dtype=torch.float32,
+                               device=device)
+        self.ws = l2.new_workspace(l2.Layout(self.K, q_heads=w.Hq), w.T, device)
+        self.launches_per_step = 3 + 2 * w.decode_steps
+
+    def compress(self):
+        self.l2.select_compact(self.K, self.V, self.lens, self.keep, self.w.T, self.unc, self.K_c,
+                               self.V_c, self.idx, self.sumsq, self.cur, self.ws)
+
+    def decode(self, s):
+        self.l2.decode_attention(self.q[s], self.K_c, self.V_c, self.cur, self.w.T, self.out[s],
+                                 self.ws)
+
+    def step(self, ev=None):
+        """One pass of the whole path.  ev: optional list collecting (start, mid, end) events."""
+        if ev is not None:
+            e0 = torch.cuda.Event(enable_timing=True); e0.record()
+        self.compress()
+        if ev is not None:
+            e1 = torch.cuda.Event(enable_timing=True); e1.record()
+        for s in range(self.w.decode_steps):
+            self.decode(s)
+        if ev is not None:
+            e2 = torch.cuda.Event(enable_timing=True); e2.record()
+            ev.append((e0, e1, e2))
+
+
+def run_gpu(args):
+    rank, world, local = dist_setup(args.gpus)
+    device = torch.device("cuda", local)
+    torch.cuda.set_device(device)
+    w = workload(args)
+    job = Job(w, device, rank)
+    cbytes, dbytes, keep = algorithmic_bytes(w)
+    step_bytes = cbytes + w.decode_steps * dbytes
+
+    for _ in range(max(args.warmup, 3)):
+        job.step()
+    barrier(world)
+    sampler = ClockSampler(local) if rank == 0 else None
+    ev = []
+    t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(args.steps):
+        job.step(ev)
+    t1.record()
+    barrier(world)
+    total_ms = max_over_ranks(t0.elapsed_time(t1), world, device)
+    clocks = sampler.stop() if sampler else None
+    c_ms = statistics.mean(a.elapsed_time(b) for a, b, _ in ev)
+    d_ms = statistics.mean(b.elapsed_time(c) for _, b, c in ev) / w.decode_steps
+    c_ms = max_over_ranks(c_ms, world, device)
+    d_ms = max_over_ranks(d_ms, world, device)
+
+    # end to end: inputs start in pinned host memory, results end there
+    e2e = None
+    if not args.no_e2e:
+        e2e = run_e2e(job, w, step_bytes, world, device, args)
+
+    if rank != 0:
+        return
+    ms_per_step = total_ms / args.steps
+    value = world * step_bytes / (ms_per_step * 1e-3) / 1e9
+    peak, peak_kind = measured_peak()
+    dec_gbs = dbytes / (d_ms * 1e-3) / 1e9
+    cmp_gbs = cbytes / (c_ms * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": round(value, 1), "unit": "GB/s", "n_gpus": world,
+        "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": round(ms_per_step, 3),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic",
+        "config": {"workload": w.name, "batch": w.B, "layers": w.L, "kv_heads": w.Hkv,
+                   "q_heads": w.Hq, "head_dim": w.D, "context": w.T, "storage": w.dtype,
+                   "keep_ratio": w.keep_ratio, "keep_per_head": keep,
+                   "uncompressed_layers": list(job.unc), "decode_steps_per_step": w.decode_steps,
+                   "l2": "inputs larger than L2 (8.5 GiB read per decode step, 16 GiB per compress)",
+                   "parallelism": f"independent replicas x{world}, no collective"},
+        "compress": {"ms": round(c_ms, 3), "GBps": round(cmp_gbs, 1), "bytes": cbytes,
+                     "frac_of_8TBps": round(cmp_gbs / NOMINAL_HBM_GBS, 4),
+                     f"frac_of_{peak_kind}": round(cmp_gbs / peak, 4)},
+        "decode": {"ms_per_decode_step": round(d_ms, 4), "GBps": round(dec_gbs, 1), "bytes": dbytes,
+                   "frac_of_8TBps": round(dec_gbs / NOMINAL_HBM_GBS, 4),
+                   f"frac_of_{peak_kind}": round(dec_gbs / peak, 4),
+                   "tokens_per_s": round(world * w.B / (d_ms * 1e-3), 1)},
+        "roofline": {"bound": "hbm", "kernel": "decode_split_kernel (+ combine, timed together)",
+                     "achieved": round(dec_gbs, 1), "peak": peak, "peak_kind": peak_kind,
+                     "unit": "GB/s", "frac": round(dec_gbs / peak, 4), "traffic": args.traffic},
+        "gpu_launches": job.launches_per_step * args.steps,
+        "clocks": clocks,
+    }
+    if e2e:
+        line["e2e"] = e2e
+    if not args.no_cpu_baseline and world == 1:
+        line["cpu_baseline"] = cpu_baseline(w, target_s=args.cpu_seconds)
+    print(json.dumps(line))
+
+
+def run_e2e(job, w, step_bytes, world, device, args):
+    """The same step with the cache arriving from pinned host memory and the attention outputs
+    returning to it, all inside the timed region."""
+    Kh = torch.empty(job.K.shape, dtype=job.K.dtype, pin_memory=True)
+    Vh = torch.empty_like(Kh, pin_memory=True)
+    qh = torch.empty(job.q.shape, dtype=job.q.dtype, pin_memory=True)
+    oh = torch.empty(job.out.shape, dtype=torch.float32, pin_memory=True)
+    Kh.copy_(job.K); Vh.copy_(job.V); qh.copy_(job.q)
+    torch.cuda.synchronize()
+    h2d = Kh.numel() * Kh.element_size() * 2 + qh.numel() * qh.element_size()
+    d2h = oh.numel() * 4
+
+    def step():
+        job.K.copy_(Kh, non_blocking=True)
+        job.V.copy_(Vh, non_blocking=True)
+        job.q.copy_(qh, non_blocking=True)
+        job.step()
+        oh.copy_(job.out, non_blocking=True)
+
+    step()
+    barrier(world)
+    n = max(1, min(args.steps, args.e2e_steps))
+    t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(n):
+        step()
+    t1.record()
+    barrier(world)
+    ms = max_over_ranks(t0.elapsed_time(t1), world, device) / n
+    del Kh, Vh
+    return {"value": round(world * step_bytes / (ms * 1e-3) / 1e9, 1), "unit": "GB/s",
+            "ms_per_step": round(ms, 2), "steps": n, "h2d_bytes_per_step": h2d,
+            "d2h_bytes_per_step": d2h}
+
+
+# ------------------------------------------------------------------------- oracle arm
+
+def oracle_sample_step(w, seed_shift=0, n_dec=2, nthreads=None):
+    """One bounded sample of the workload through the CPU oracle: sequence 0, one
+    uncompressed and one compressed layer, full context, a compression pass and n_dec
+    decode steps.  Returns (seconds, algorithmic bytes moved)."""
+    import oracle
+    nthreads = nthreads or oracle.hardware_threads()
+    layers = [l for l in (0, 2) if l < w.L] or [0]
+    ws = w.scaled(seed=w.seed + seed_shift)
+    Ks, Vs = [], []
+    for l in layers:
+        Ks.append(synth.to_numpy(synth.make_kv_slab(ws, "K", 0, l, "cpu")))
+        Vs.append(synth.to_numpy(synth.make_kv_slab(ws, "V", 0, l, "cpu")))
+    K = np.ascontiguousarray(np.stack(Ks)[None]); V = np.ascontiguousarray(np.stack(Vs)[None])
+    sub = w.scaled(B=1, L=len(layers),
+                   uncompressed=tuple(i for i, l in enumerate(layers) if l in w.uncompressed))
+    qs = [synth.to_numpy(synth.make_query(ws, s, "cpu"))[:1, layers] for s in range(n_dec)]
+    qs = [np.ascontiguousarray(q) for q in qs]
+    keep = oracle.keep_count(w.T, w.keep_ratio)
+    t0 = time.perf_counter()
+    r = oracle.compress(K, V, w.dtype, [w.T], [keep], sub.uncompressed, nthreads=nthreads)
+    for q in qs:
+        oracle.attention(q, r["K_c"], r["V_c"], w.dtype, r["kept_len"], nthreads=nthreads)
+    dt = time.perf_counter() - t0
+    cb, db, _ = algorithmic_bytes(sub.scaled(decode_steps=n_dec))
+    return dt, cb + n_dec * db, nthreads, layers
+
+
+def cpu_baseline(w, target_s=15.0):
+    dt, nbytes, nthreads, layers = oracle_sample_step(w, n_dec=1)
+    per_dec = max(dt, 1e-3)
+    n_dec = int(max(1, min(w.decode_steps, target_s / per_dec)))
+    dt, nbytes, nthreads, layers = oracle_sample_step(w, n_dec=n_dec)
+    return {"value": round(nbytes / dt / 1e9, 4), "unit": "GB/s", "cores": nthreads,
+            "kind": "oracle", "seconds": round(dt, 2),
+            "sample": f"sequence 0, layers {layers} (one uncompressed, one compressed), all "
+                      f"{w.Hkv} KV heads, full {w.T}-token context: one compression pass + "
+                      f"{n_dec} decode steps"}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = workload(args)
+    import oracle
+    n_dec = 2
+    for _ in range(min(args.warmup, 1)):
+        oracle_sample_step(w, n_dec=n_dec)
+    times, nbytes, nthreads, layers = [], 0, 0, []
+    for s in range(args.steps):
+        dt, nbytes, nthreads, layers = oracle_sample_step(w, seed_shift=s, n_dec=n_dec)
+        times.append(dt)
+    ms = 1e3 * sum(times) / len(times)
+    value = round(nbytes / (ms * 1e-3) / 1e9, 4)
+    sample = (f"per step: sequence 0, layers {layers}, all {w.Hkv} KV heads, full {w.T}-token "
+              f"context, one compression pass + {n_dec} decode steps")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": min(args.warmup, 1), "ms_per_step": round(ms, 1),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": {"workload": w.name, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": "GB/s", "cores": nthreads, "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="l2kv", choices=["l2kv", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    ap.add_argument("--layers", type=int, default=0, help="profiling aid: fewer layers")
+    ap.add_argument("--context", type=int, default=0, help="profiling aid: shorter context")
+    ap.add_argument("--decode-steps", type=int, default=0, help="profiling aid")
+    ap.add_argument("--traffic", type=float, default=None,
+                    help="DRAM bytes per launch of the dominant kernel from an ncu capture")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()
