@@ -242,6 +242,275 @@ decode_combine_kernel(const float* __restrict__ partial, const int32_t* __restri
   out[row * D + d] = ns > 0 ? num / den : 0.f;
 }
 
+// ---------------------------------------------------------------------------------------
+// bf16, head_dim 128: the same three phases with the two contractions on tensor cores.
+//
+// The CUDA-core kernel above spends ~70 warp instructions per cached token (unpack, FMA,
+// shuffles), which at G = 4 fills two thirds of the issue slots and leaves the kernel
+// latency-bound well below the HBM rate.  Here the work per token is a handful of
+// instructions, so the kernel is a pure stream:
+//   * K and V rows travel global -> shared memory with 16-byte cp.async copies through a
+//     ring of kStages stages of kStageTok tokens (16-byte pieces XOR-swizzled by row so that
+//     ldmatrix reads are conflict-free); nothing is staged in registers.
+//   * scores: S^T[token, head] = K[token, :] . Q^T -- mma.m16n8k16, A = 16 tokens x 16 dims of
+//     K (ldmatrix), B = Q^T with the G heads padded to N = 8, fp32 accumulators.
+//   * output: O^T[dim, head] = V^T[dim, token] . P^T -- A = V^T via ldmatrix.trans, B = the
+//     weights split into two bf16 terms (hi + lo carries 16 mantissa bits), fp32 accumulators.
+//     Warp w owns output dims [16w, 16w + 16) for the whole split, so no cross-warp sum.
+// bf16 x bf16 products are exact in fp32, so the arithmetic is the same as above up to the
+// summation order inside the tensor core and the 2^-17 relative split of the weights.
+constexpr int kStageTok = 128;
+constexpr int kStages = 3;
+constexpr int kRowBytes = 256;                         // 128 bf16
+constexpr int kScLd = kDecodeChunk + 4;                // floats per head row of the score buffer
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" :: "r"(dst), "l"(src), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;" :: "n"(N) : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+template <int G>
+__global__ void __launch_bounds__(kDecThreads, 2)
+decode_split_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ K,
+                        const __nv_bfloat16* __restrict__ V, Geom g,
+                        const int32_t* __restrict__ cur_len_dev, int max_len, float scale_log2e,
+                        float* __restrict__ partial, int n_splits) {
+  constexpr int D = 128;
+  constexpr int NW = kDecThreads / 32;
+  constexpr int TPT = kDecodeChunk / kDecThreads;        // tokens per thread in phase 2
+  extern __shared__ __align__(128) unsigned char smem[];
+  unsigned char* s_stage = smem;                                        // [kStages][128][256 B]
+  float* s_sc = reinterpret_cast<float*>(smem + kStages * kStageTok * kRowBytes);  // [G][kScLd]
+  __shared__ float s_red[NW][G];
+  __shared__ float s_m[G], s_l[G];
+
+  const int split = blockIdx.x % n_splits;
+  const long long unit = blockIdx.x / n_splits;          // (b * L + l) * H + h
+  const int h = (int)(unit % g.H);
+  const long long bl = unit / g.H;
+  const int l = (int)(bl % g.L);
+  const int b = (int)(bl / g.L);
+  const int n = max(0, min(cur_len_dev[bl], min(max_len, g.t_cap)));
+  const int t0 = split * kDecodeChunk;
+  if (t0 >= n) return;
+  const int nt = min(n, t0 + kDecodeChunk) - t0;
+  const int n_st = (nt + kStageTok - 1) / kStageTok;     // stages of K, and again of V
+  const int total = 2 * n_st;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int fr = lane >> 2, fc = lane & 3;               // fragment row / column-pair indices
+  const __nv_bfloat16* Kb = K + b * g.sb + l * g.sl + h * g.sh + (long long)t0 * g.st;
+  const __nv_bfloat16* Vb = V + b * g.sb + l * g.sl + h * g.sh + (long long)t0 * g.st;
+  const uint32_t stage0 = smem_u32(s_stage);
+
+  auto issue = [&](int s) {
+    const __nv_bfloat16* src = s < n_st ? Kb : Vb;
+    const int st = s < n_st ? s : s - n_st;
+    const uint32_t dst0 = stage0 + (s % kStages) * (kStageTok * kRowBytes);
+#pragma unroll
+    for (int i = 0; i < kStageTok * 16 / kDecThreads; ++i) {
+      const int id = tid + i * kDecThreads;
+      const int row = id >> 4, ch = id & 15;
+      const int tl = st * kStageTok + row;
+      const bool ok = tl < nt;                             // rows past the end are zero-filled
+      cp_async16(dst0 + row * kRowBytes + ((ch ^ (row & 7)) << 4),
+                 src + (long long)(ok ? tl : 0) * g.st + ch * 8, ok ? 16 : 0);
+    }
+  };
+
+  for (int s = 0; s < kStages - 1; ++s) {
+    if (s < total) issue(s);
+    cp_async_commit();
+  }
+
+  // Q^T fragments: lane (fr, fc) holds head fr's dims 16j + 2fc (+1) and 16j + 2fc + 8 (+9).
+  uint32_t qb[8][2];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) { qb[j][0] = 0u; qb[j][1] = 0u; }
+  if (fr < G) {
+    const __nv_bfloat16* qrow = q + (bl * g.Hq + h * G + fr) * D;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      qb[j][0] = *reinterpret_cast<const uint32_t*>(qrow + 16 * j + 2 * fc);
+      qb[j][1] = *reinterpret_cast<const uint32_t*>(qrow + 16 * j + 2 * fc + 8);
+    }
+  }
+
+  float oacc[4] = {0.f, 0.f, 0.f, 0.f};                    // O^T[16 warp + fr (+8)][2 fc (+1)]
+  for (int s = 0; s < total; ++s) {
+    cp_async_wait<kStages - 2>();
+    __syncthreads();                                       // stage s landed; stage s-1 is free
+    if (s + kStages - 1 < total) issue(s + kStages - 1);
+    cp_async_commit();
+    const uint32_t sb = stage0 + (s % kStages) * (kStageTok * kRowBytes);
+
+    if (s < n_st) {
+      // ---- phase 1: scores of tokens [16 warp, 16 warp + 16) of this stage ------------
+      const int tl0 = s * kStageTok + warp * 16;
+      if (tl0 < nt) {
+        float c[4] = {0.f, 0.f, 0.f, 0.f};
+        const int row = warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          uint32_t a[4];
+          const int ch = 2 * j + (lane >> 4);
+          ldmatrix_x4(a, sb + row * kRowBytes + ((ch ^ (row & 7)) << 4));
+          mma_bf16(c, a, qb[j][0], qb[j][1]);
+        }
+        if (2 * fc < G) {
+          s_sc[(2 * fc) * kScLd + tl0 + fr] = c[0] * scale_log2e;
+          s_sc[(2 * fc) * kScLd + tl0 + fr + 8] = c[2] * scale_log2e;
+        }
+        if (2 * fc + 1 < G) {
+          s_sc[(2 * fc + 1) * kScLd + tl0 + fr] = c[1] * scale_log2e;
+          s_sc[(2 * fc + 1) * kScLd + tl0 + fr + 8] = c[3] * scale_log2e;
+        }
+      }
+      if (s == n_st - 1) {
+        // ---- phase 2: exact maximum, weights as bf16 hi + lo, their sum -----------------
+        __syncthreads();
+        float sc[TPT][G], mx[G], sum[G];
+#pragma unroll
+        for (int gi = 0; gi < G; ++gi) mx[gi] = -INFINITY;
+#pragma unroll
+        for (int i = 0; i < TPT; ++i) {
+          const int tl = tid + i * kDecThreads;
+#pragma unroll
+          for (int gi = 0; gi < G; ++gi) {
+            sc[i][gi] = tl < nt ? s_sc[gi * kScLd + tl] : -INFINITY;
+            mx[gi] = fmaxf(mx[gi], sc[i][gi]);
+          }
+        }
+#pragma unroll
+        for (int gi = 0; gi < G; ++gi) {
+#pragma unroll
+          for (int off = 16; off >= 1; off >>= 1)
+            mx[gi] = fmaxf(mx[gi], __shfl_xor_sync(0xffffffffu, mx[gi], off));
+          if (lane == 0) s_red[warp][gi] = mx[gi];
+        }
+        __syncthreads();                                   // also: every score is in registers
+        if (tid < G) {
+          float m = s_red[0][tid];
+          for (int w = 1; w < NW; ++w) m = fmaxf(m, s_red[w][tid]);
+          s_m[tid] = m;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int gi = 0; gi < G; ++gi) { mx[gi] = s_m[gi]; sum[gi] = 0.f; }
+#pragma unroll
+        for (int i = 0; i < TPT; ++i) {
+          const int tl = tid + i * kDecThreads;
+#pragma unroll
+          for (int gi = 0; gi < G; ++gi) {
+            const float w = exp2f(sc[i][gi] - mx[gi]);     // 0 for tokens past the end
+            sum[gi] += w;
+            const __nv_bfloat16 hi = __float2bfloat16_rn(w);
+            const __nv_bfloat16 lo = __float2bfloat16_rn(w - __bfloat162float(hi));
+            __nv_bfloat16* prow = reinterpret_cast<__nv_bfloat16*>(s_sc + gi * kScLd);
+            prow[tl] = hi;                                 // hi terms: first half of the row
+            prow[kScLd + tl] = lo;                         // lo terms: second half
+          }
+        }
+#pragma unroll
+        for (int gi = 0; gi < G; ++gi) {
+#pragma unroll
+          for (int off = 16; off >= 1; off >>= 1) sum[gi] += __shfl_xor_sync(0xffffffffu, sum[gi], off);
+          if (lane == 0) s_red[warp][gi] = sum[gi];
+        }
+        __syncthreads();                                   // weights and partial sums visible
+        if (tid < G) {
+          float acc = 0.f;
+          for (int w = 0; w < NW; ++w) acc += s_red[w][tid];
+          s_l[tid] = acc;
+        }
+      }
+    } else {
+      // ---- phase 3: O^T[16 warp .. +16, head] += V^T . P^T over this stage's tokens ------
+      const int st = s - n_st;
+      const int ksteps = min(kStageTok / 16, (nt - st * kStageTok + 15) / 16);
+      const __nv_bfloat16* prow = reinterpret_cast<const __nv_bfloat16*>(s_sc + fr * kScLd);
+      for (int ks = 0; ks < ksteps; ++ks) {
+        uint32_t a[4];
+        const int row = ks * 16 + (lane & 7) + (lane >> 4) * 8;
+        const int ch = 2 * warp + ((lane >> 3) & 1);
+        ldmatrix_x4_trans(a, sb + row * kRowBytes + ((ch ^ (row & 7)) << 4));
+        uint32_t h0 = 0u, h1 = 0u, l0 = 0u, l1 = 0u;
+        if (fr < G) {
+          const int tb = st * kStageTok + ks * 16 + 2 * fc;
+          h0 = *reinterpret_cast<const uint32_t*>(prow + tb);
+          h1 = *reinterpret_cast<const uint32_t*>(prow + tb + 8);
+          l0 = *reinterpret_cast<const uint32_t*>(prow + kScLd + tb);
+          l1 = *reinterpret_cast<const uint32_t*>(prow + kScLd + tb + 8);
+        }
+        mma_bf16(oacc, a, h0, h1);
+        mma_bf16(oacc, a, l0, l1);
+      }
+    }
+  }
+  cp_async_wait<0>();
+
+  // O^T fragment: rows = dims 16 warp + fr (+8), columns = heads 2 fc (+1).
+#pragma unroll
+  for (int e = 0; e < 2; ++e) {
+    const int head = 2 * fc + e;
+    if (head < G) {
+      float* p = partial + ((bl * g.Hq + h * G + head) * n_splits + split) * (long long)(D + 2);
+      p[2 + 16 * warp + fr] = oacc[e];
+      p[2 + 16 * warp + fr + 8] = oacc[2 + e];
+    }
+  }
+  if (tid < G) {
+    float* p = partial + ((bl * g.Hq + h * G + tid) * n_splits + split) * (long long)(D + 2);
+    p[0] = s_m[tid];
+    p[1] = s_l[tid];
+  }
+}
+
+template <int G>
+static int launch_dec_mma(const void* q, const void* K, const void* V, const Geom& g,
+                          const int32_t* cur_len_dev, int max_len, float scale, float* out,
+                          char* ws, const WorkspacePlan& plan, cudaStream_t s) {
+  const long long units = (long long)g.B * g.L * g.H;
+  if (units == 0) return L2KV_OK;
+  if (units * plan.n_splits > 0x7fffffffLL) return L2KV_ERR_OUT_OF_RANGE;
+  float* partial = reinterpret_cast<float*>(ws + plan.partial_off);
+  constexpr int smem_bytes = kStages * kStageTok * kRowBytes + G * kScLd * 4;
+  if (max_len > 0) {
+    auto kern = decode_split_mma_kernel<G>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) !=
+        cudaSuccess)
+      return L2KV_ERR_CUDA;
+    kern<<<(unsigned)(units * plan.n_splits), kDecThreads, smem_bytes, s>>>(
+        static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(K),
+        static_cast<const __nv_bfloat16*>(V), g, cur_len_dev, max_len, scale * kLog2e, partial,
+        plan.n_splits);
+    if (cudaGetLastError() != cudaSuccess) return L2KV_ERR_CUDA;
+  }
+  decode_combine_kernel<128><<<(unsigned)((long long)g.B * g.L * g.Hq), 128, 0, s>>>(
+      partial, cur_len_dev, max_len, g.t_cap, g.Hq, plan.n_splits, out);
+  return cudaGetLastError() == cudaSuccess ? L2KV_OK : L2KV_ERR_CUDA;
+}
+
 template <typename T, int D, int G>
 static int launch_dec_t(const void* q, const void* K, const void* V, const Geom& g,
                         const int32_t* cur_len_dev, int max_len, float scale, float* out, char* ws,
@@ -280,7 +549,15 @@ int launch_decode_attention(const void* q, const void* K, const void* V, const G
 #define L2KV_DA(T, D) \
   return launch_dec_g<T, D>(q, K, V, g, cur_len_dev, max_len, scale, out, ws, plan, s)
   if (dtype == L2KV_BF16) {
-    if (g.D == 128) L2KV_DA(__nv_bfloat16, 128);
+    if (g.D == 128) {
+      switch (g.Hq / g.H) {
+        case 1: return launch_dec_mma<1>(q, K, V, g, cur_len_dev, max_len, scale, out, ws, plan, s);
+        case 2: return launch_dec_mma<2>(q, K, V, g, cur_len_dev, max_len, scale, out, ws, plan, s);
+        case 4: return launch_dec_mma<4>(q, K, V, g, cur_len_dev, max_len, scale, out, ws, plan, s);
+        case 8: return launch_dec_mma<8>(q, K, V, g, cur_len_dev, max_len, scale, out, ws, plan, s);
+      }
+      return L2KV_ERR_UNSUPPORTED;
+    }
     if (g.D == 64) L2KV_DA(__nv_bfloat16, 64);
   } else if (dtype == L2KV_F32) {
     if (g.D == 128) L2KV_DA(float, 128);
