@@ -35,6 +35,10 @@ GIB = 1 << 30
 METRIC = "compress + decode GB/s of KV read and % of B200 HBM peak; decode tokens/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
+# DRAM bytes (read + written) per algorithmic byte of the dominant kernel, from the ncu capture
+# summarised in profiles/decode_split_mma_kernel_llama3-8b-32k_4layers.md (a 4-layer case; the
+# traffic is proportional to the tokens streamed).  Set to None whenever that kernel changes.
+DECODE_TRAFFIC_RATIO = 1.0062
 
 
 def workload(args):
@@ -115,30 +119,24 @@ class ClockSampler:
 
 
 def dist_setup(n):
+    """One process per GPU (torchrun sets RANK / LOCAL_RANK / WORLD_SIZE)."""
+    from paper_2406_11430_b200 import sharding
     if n <= 1:
         return 0, 1, 0
-    import torch.distributed as dist
-    rank, world = int(os.environ["RANK"]), int(os.environ["WORLD_SIZE"])
-    local = int(os.environ.get("LOCAL_RANK", rank))
+    local = int(os.environ.get("LOCAL_RANK", os.environ.get("RANK", "0")))
     torch.cuda.set_device(local)
-    dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    rank, world = sharding.init("nccl", torch.device("cuda", local))
     return rank, world, local
 
 
 def max_over_ranks(x, world, device):
-    if world <= 1:
-        return x
-    import torch.distributed as dist
-    t = torch.tensor([x], dtype=torch.float64, device=device)
-    dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    return float(t.item())
+    from paper_2406_11430_b200 import sharding
+    return sharding.max_over_ranks(x, device) if world > 1 else x
 
 
 def barrier(world):
-    if world > 1:
-        import torch.distributed as dist
-        dist.barrier()
-    torch.cuda.synchronize()
+    from paper_2406_11430_b200 import sharding
+    sharding.barrier()
 
 
 # ------------------------------------------------------------------------------ GPU arm
@@ -246,9 +244,11 @@ def run_gpu(args):
                    "frac_of_8TBps": round(dec_gbs / NOMINAL_HBM_GBS, 4),
                    f"frac_of_{peak_kind}": round(dec_gbs / peak, 4),
                    "tokens_per_s": round(world * w.B / (d_ms * 1e-3), 1)},
-        "roofline": {"bound": "hbm", "kernel": "decode_split_kernel (+ combine, timed together)",
+        "roofline": {"bound": "hbm", "kernel": "decode_split_mma_kernel (+ combine, timed together)",
                      "achieved": round(dec_gbs, 1), "peak": peak, "peak_kind": peak_kind,
-                     "unit": "GB/s", "frac": round(dec_gbs / peak, 4), "traffic": args.traffic},
+                     "unit": "GB/s", "frac": round(dec_gbs / peak, 4),
+                     "traffic": args.traffic if args.traffic is not None else
+                     (round(DECODE_TRAFFIC_RATIO * dbytes) if DECODE_TRAFFIC_RATIO else None)},
         "gpu_launches": job.launches_per_step * args.steps,
         "clocks": clocks,
     }
