@@ -147,6 +147,34 @@ int l2kv_append_evict(void* K_c, void* V_c, int32_t* idx, float* sumsq_c, const 
                       const void* k_new, const void* v_new, const int32_t* pos_new_dev,
                       void* workspace, size_t workspace_bytes, void* stream);
 
+/* Decode attention without a workspace -- the paper has no counterpart to this entry
+ * point; it exists for the callers of this library that cannot allocate device memory.
+ *
+ * Same operation, arguments, result and errors as l2kv_decode_attention, but the scratch
+ * for the per-split partial results is a fixed array of L2KV_STATIC_SCRATCH_BYTES that
+ * is part of the library image: every GPU that loads the library holds that much memory
+ * until the process exits, and no call here ever runs cudaMalloc, cudaFree or any other
+ * allocating routine.  Meant for code that runs where allocation is forbidden or would
+ * stall (a thread that may not take the allocator's lock, a callback, a serving loop whose
+ * pool is already handed out) and that has no spare buffer to pass as a workspace.
+ *
+ *   - Limit: batch * layers * q_heads * ceil(max_len / 1024) * (head_dim + 2) * 4 bytes must
+ *     not exceed L2KV_STATIC_SCRATCH_BYTES (16 MiB: e.g. one layer of 32 query heads at
+ *     batch 4 up to a cache of about 250k tokens, or a whole 32-layer model at batch 4 up to 7k
+ *     tokens).  Beyond it the call returns L2KV_ERR_WORKSPACE_TOO_SMALL and launches
+ *     nothing: call per layer, or use l2kv_decode_attention with your own workspace.
+ *   - The first call on each device looks up the array's device address (a runtime
+ *     query, not an allocation), with the current device taken as the one `stream`
+ *     belongs to; make that first call outside any stream capture.
+ *   - All calls on a device share the one array, which simply keeps what the last call
+ *     left in it (nothing in it needs clearing between calls).  Two calls whose kernels can
+ *     overlap on the GPU -- different streams, no dependency -- race on it and give wrong
+ *     results: order them, or use the workspace variant for concurrent streams. */
+#define L2KV_STATIC_SCRATCH_BYTES (16u << 20)
+int l2kv_decode_attention_static(const void* q, const void* K_c, const void* V_c,
+                                 const l2kv_layout* lay, const int32_t* cur_len_dev,
+                                 int32_t max_len, float scale, float* out, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

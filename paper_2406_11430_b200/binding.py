@@ -161,3 +161,17 @@ def append_evict(K_c, V_c, idx, sumsq_c, cur_len_dev, budget_dev, uncompressed_l
         _ptr(K_c), _ptr(V_c), _ptr(idx), _ptr(sumsq_c), lay.ref(), _ptr(cur_len_dev),
         _ptr(budget_dev), arr, n, _ptr(k_new), _ptr(v_new), _ptr(pos_new_dev), _ptr(workspace),
         workspace.numel(), _stream(stream)), "l2kv_append_evict")
+
+
+def decode_attention_static(q, K_c, V_c, cur_len_dev, max_len, out, scale=0.0, stream=None):
+    """decode_attention for callers that cannot allocate: no workspace argument.  The partial
+    results go to a fixed 16 MiB array inside the library (problems that need more raise
+    L2KVError with status -4).  Calls share that array, so do not let two of them overlap on
+    the GPU; make the first call on a device outside any stream capture."""
+    fn = lib().l2kv_decode_attention_static
+    vp = ctypes.c_void_p
+    fn.restype = ctypes.c_int
+    fn.argtypes = [vp, vp, vp, ctypes.POINTER(_CLayout), vp, ctypes.c_int32, ctypes.c_float, vp, vp]
+    lay = Layout(K_c, q_heads=q.shape[2])
+    _check(fn(_ptr(q), _ptr(K_c), _ptr(V_c), lay.ref(), _ptr(cur_len_dev), int(max_len),
+              float(scale), _ptr(out), _stream(stream)), "l2kv_decode_attention_static")
