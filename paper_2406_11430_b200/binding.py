@@ -5,7 +5,8 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_LIB_PATH = os.path.join(_HERE, "libl2kv.so")
+# L2KV_LIBRARY selects another build of the same library (a tuning variant).
+_LIB_PATH = os.environ.get("L2KV_LIBRARY") or os.path.join(_HERE, "libl2kv.so")
 _LIB = None
 
 KEEP_LOWEST_NORM = 0

@@ -31,14 +31,16 @@ def _stale():
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force=False, verbose=False):
-    if not force and not _stale():
+def build(force=False, verbose=False, out=None, defines=()):
+    """out / defines: build a tuning variant (e.g. defines=["L2KV_MMA_WARPS=4"]) elsewhere."""
+    out = out or LIB
+    if out == LIB and not force and not _stale():
         return LIB
     nvcc = os.environ.get("NVCC", "nvcc")
-    cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + \
-        ["-shared", "-o", LIB] + sources()
+    cmd = [nvcc] + NVCC_FLAGS + [f"-D{d}" for d in defines] + \
+        (["-Xptxas", "-v"] if verbose else []) + ["-shared", "-o", out] + sources()
     subprocess.run(cmd, check=True)
-    return LIB
+    return out
 
 
 if __name__ == "__main__":

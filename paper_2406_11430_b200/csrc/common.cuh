@@ -15,7 +15,10 @@ constexpr int kStatusBytes = 256;      // device status word lives at the start 
 constexpr int kMaxLayers = 1024;       // size of the uncompressed-layer bit mask
 constexpr int kGatherChunk = 512;      // input tokens per gather CTA / per scan chunk
 constexpr int kMaxChunks = 4096;       // kGatherChunk * kMaxChunks tokens per unit at most
-constexpr int kDecodeChunk = 1024;     // cached tokens per split of decode attention
+#ifndef L2KV_DECODE_CHUNK
+#define L2KV_DECODE_CHUNK 1024
+#endif
+constexpr int kDecodeChunk = L2KV_DECODE_CHUNK;   // cached tokens per split of decode attention
 
 // Cache geometry handed to kernels by value (strides in elements).
 struct Geom {

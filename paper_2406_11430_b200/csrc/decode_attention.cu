@@ -259,8 +259,20 @@ decode_combine_kernel(const float* __restrict__ partial, const int32_t* __restri
 //     Warp w owns output dims [16w, 16w + 16) for the whole split, so no cross-warp sum.
 // bf16 x bf16 products are exact in fp32, so the arithmetic is the same as above up to the
 // summation order inside the tensor core and the 2^-17 relative split of the weights.
-constexpr int kStageTok = 128;
-constexpr int kStages = 3;
+#ifndef L2KV_MMA_WARPS
+#define L2KV_MMA_WARPS 8
+#endif
+#ifndef L2KV_MMA_STAGES
+#define L2KV_MMA_STAGES 3
+#endif
+#ifndef L2KV_MMA_MIN_CTAS
+#define L2KV_MMA_MIN_CTAS 2
+#endif
+constexpr int kMmaWarps = L2KV_MMA_WARPS;              // 8, 4 or 2: each warp scores 16 tokens a stage
+constexpr int kMmaThreads = 32 * kMmaWarps;
+constexpr int kStageTok = 16 * kMmaWarps;              // tokens per ring stage
+constexpr int kStages = L2KV_MMA_STAGES;
+constexpr int kDbw = 8 / kMmaWarps;                    // 16-dim output blocks per warp
 constexpr int kRowBytes = 256;                         // 128 bf16
 constexpr int kScLd = kDecodeChunk + 4;                // floats per head row of the score buffer
 
@@ -290,14 +302,14 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], 
 }
 
 template <int G>
-__global__ void __launch_bounds__(kDecThreads, 2)
+__global__ void __launch_bounds__(kMmaThreads, L2KV_MMA_MIN_CTAS)
 decode_split_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ K,
                         const __nv_bfloat16* __restrict__ V, Geom g,
                         const int32_t* __restrict__ cur_len_dev, int max_len, float scale_log2e,
                         float* __restrict__ partial, int n_splits) {
   constexpr int D = 128;
-  constexpr int NW = kDecThreads / 32;
-  constexpr int TPT = kDecodeChunk / kDecThreads;        // tokens per thread in phase 2
+  constexpr int NW = kMmaWarps;
+  constexpr int TPT = kDecodeChunk / kMmaThreads;        // tokens per thread in phase 2
   extern __shared__ __align__(128) unsigned char smem[];
   unsigned char* s_stage = smem;                                        // [kStages][128][256 B]
   float* s_sc = reinterpret_cast<float*>(smem + kStages * kStageTok * kRowBytes);  // [G][kScLd]
@@ -323,18 +335,33 @@ decode_split_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16
   const __nv_bfloat16* Vb = V + b * g.sb + l * g.sl + h * g.sh + (long long)t0 * g.st;
   const uint32_t stage0 = smem_u32(s_stage);
 
+  // Copy plan of this thread, fixed for the whole kernel: it moves the 16-byte piece c_ch of
+  // rows c_row, c_row + kRowStep, ... of every stage.  kRowStep is a multiple of 8, so the
+  // swizzled piece index is the same for all of them and only pointers advance.
+  static_assert(kMmaWarps == 4 || kMmaWarps == 8, "copy plan needs a row step that is a multiple of 8");
+  constexpr int kRowStep = kMmaThreads / 16;
+  constexpr int kCopies = kStageTok / kRowStep;            // 8 pieces per thread per stage
+  const int c_row = tid >> 4, c_ch = tid & 15;
+  const uint32_t c_dst = stage0 + c_row * kRowBytes + ((c_ch ^ (c_row & 7)) << 4);
+  const long long row_bytes = g.st * 2;                    // global bytes between cached rows
+  const char* c_k = reinterpret_cast<const char*>(Kb) + c_row * row_bytes + c_ch * 16;
+  const char* c_v = reinterpret_cast<const char*>(Vb) + c_row * row_bytes + c_ch * 16;
   auto issue = [&](int s) {
-    const __nv_bfloat16* src = s < n_st ? Kb : Vb;
     const int st = s < n_st ? s : s - n_st;
-    const uint32_t dst0 = stage0 + (s % kStages) * (kStageTok * kRowBytes);
+    const char* src = (s < n_st ? c_k : c_v) + (long long)st * kStageTok * row_bytes;
+    const uint32_t dst = c_dst + (s % kStages) * (kStageTok * kRowBytes);
+    const int rows = nt - st * kStageTok;                  // valid rows of this stage (>= 1)
+    if (rows >= kStageTok) {
 #pragma unroll
-    for (int i = 0; i < kStageTok * 16 / kDecThreads; ++i) {
-      const int id = tid + i * kDecThreads;
-      const int row = id >> 4, ch = id & 15;
-      const int tl = st * kStageTok + row;
-      const bool ok = tl < nt;                             // rows past the end are zero-filled
-      cp_async16(dst0 + row * kRowBytes + ((ch ^ (row & 7)) << 4),
-                 src + (long long)(ok ? tl : 0) * g.st + ch * 8, ok ? 16 : 0);
+      for (int i = 0; i < kCopies; ++i)
+        cp_async16(dst + i * kRowStep * kRowBytes, src + i * kRowStep * row_bytes, 16);
+    } else {
+#pragma unroll
+      for (int i = 0; i < kCopies; ++i) {
+        const bool ok = c_row + i * kRowStep < rows;       // rows past the end are zero-filled
+        cp_async16(dst + i * kRowStep * kRowBytes, ok ? src + i * kRowStep * row_bytes : src - c_row * row_bytes,
+                   ok ? 16 : 0);
+      }
     }
   };
 
@@ -356,7 +383,9 @@ decode_split_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16
     }
   }
 
-  float oacc[4] = {0.f, 0.f, 0.f, 0.f};                    // O^T[16 warp + fr (+8)][2 fc (+1)]
+  float oacc[kDbw][4];                                     // O^T[16 (kDbw warp + db) + fr (+8)][2 fc (+1)]
+#pragma unroll
+  for (int db = 0; db < kDbw; ++db) { oacc[db][0] = oacc[db][1] = oacc[db][2] = oacc[db][3] = 0.f; }
   for (int s = 0; s < total; ++s) {
     cp_async_wait<kStages - 2>();
     __syncthreads();                                       // stage s landed; stage s-1 is free
@@ -394,7 +423,7 @@ decode_split_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16
         for (int gi = 0; gi < G; ++gi) mx[gi] = -INFINITY;
 #pragma unroll
         for (int i = 0; i < TPT; ++i) {
-          const int tl = tid + i * kDecThreads;
+          const int tl = tid + i * kMmaThreads;
 #pragma unroll
           for (int gi = 0; gi < G; ++gi) {
             sc[i][gi] = tl < nt ? s_sc[gi * kScLd + tl] : -INFINITY;
@@ -419,7 +448,7 @@ decode_split_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16
         for (int gi = 0; gi < G; ++gi) { mx[gi] = s_m[gi]; sum[gi] = 0.f; }
 #pragma unroll
         for (int i = 0; i < TPT; ++i) {
-          const int tl = tid + i * kDecThreads;
+          const int tl = tid + i * kMmaThreads;
 #pragma unroll
           for (int gi = 0; gi < G; ++gi) {
             const float w = exp2f(sc[i][gi] - mx[gi]);     // 0 for tokens past the end
@@ -448,35 +477,51 @@ decode_split_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16
       // ---- phase 3: O^T[16 warp .. +16, head] += V^T . P^T over this stage's tokens ------
       const int st = s - n_st;
       const int ksteps = min(kStageTok / 16, (nt - st * kStageTok + 15) / 16);
-      const __nv_bfloat16* prow = reinterpret_cast<const __nv_bfloat16*>(s_sc + fr * kScLd);
-      for (int ks = 0; ks < ksteps; ++ks) {
-        uint32_t a[4];
-        const int row = ks * 16 + (lane & 7) + (lane >> 4) * 8;
-        const int ch = 2 * warp + ((lane >> 3) & 1);
-        ldmatrix_x4_trans(a, sb + row * kRowBytes + ((ch ^ (row & 7)) << 4));
+      // Per-lane constants: weights of head fr as packed token pairs; V^T tile addresses.
+      const uint32_t* pw = reinterpret_cast<const uint32_t*>(s_sc + fr * kScLd) +
+                           st * (kStageTok / 2) + fc;
+      const int vrow = (lane & 7) + (lane >> 4) * 8;
+      uint32_t voff[kDbw];
+#pragma unroll
+      for (int db = 0; db < kDbw; ++db) {
+        const int ch = 2 * (warp * kDbw + db) + ((lane >> 3) & 1);
+        voff[db] = sb + vrow * kRowBytes + ((ch ^ (lane & 7)) << 4);
+      }
+      auto kstep = [&](int ks) {
         uint32_t h0 = 0u, h1 = 0u, l0 = 0u, l1 = 0u;
         if (fr < G) {
-          const int tb = st * kStageTok + ks * 16 + 2 * fc;
-          h0 = *reinterpret_cast<const uint32_t*>(prow + tb);
-          h1 = *reinterpret_cast<const uint32_t*>(prow + tb + 8);
-          l0 = *reinterpret_cast<const uint32_t*>(prow + kScLd + tb);
-          l1 = *reinterpret_cast<const uint32_t*>(prow + kScLd + tb + 8);
+          h0 = pw[ks * 8];              h1 = pw[ks * 8 + 4];
+          l0 = pw[kScLd / 2 + ks * 8];  l1 = pw[kScLd / 2 + ks * 8 + 4];
         }
-        mma_bf16(oacc, a, h0, h1);
-        mma_bf16(oacc, a, l0, l1);
+#pragma unroll
+        for (int db = 0; db < kDbw; ++db) {
+          uint32_t a[4];
+          ldmatrix_x4_trans(a, voff[db] + ks * 16 * kRowBytes);
+          mma_bf16(oacc[db], a, h0, h1);
+          mma_bf16(oacc[db], a, l0, l1);
+        }
+      };
+      if (ksteps == kStageTok / 16) {
+#pragma unroll
+        for (int ks = 0; ks < kStageTok / 16; ++ks) kstep(ks);
+      } else {
+        for (int ks = 0; ks < ksteps; ++ks) kstep(ks);
       }
     }
   }
   cp_async_wait<0>();
 
-  // O^T fragment: rows = dims 16 warp + fr (+8), columns = heads 2 fc (+1).
+  // O^T fragments: rows = dims 16 (kDbw warp + db) + fr (+8), columns = heads 2 fc (+1).
 #pragma unroll
   for (int e = 0; e < 2; ++e) {
     const int head = 2 * fc + e;
     if (head < G) {
       float* p = partial + ((bl * g.Hq + h * G + head) * n_splits + split) * (long long)(D + 2);
-      p[2 + 16 * warp + fr] = oacc[e];
-      p[2 + 16 * warp + fr + 8] = oacc[2 + e];
+#pragma unroll
+      for (int db = 0; db < kDbw; ++db) {
+        p[2 + 16 * (warp * kDbw + db) + fr] = oacc[db][e];
+        p[2 + 16 * (warp * kDbw + db) + fr + 8] = oacc[db][2 + e];
+      }
     }
   }
   if (tid < G) {
@@ -500,7 +545,7 @@ static int launch_dec_mma(const void* q, const void* K, const void* V, const Geo
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) !=
         cudaSuccess)
       return L2KV_ERR_CUDA;
-    kern<<<(unsigned)(units * plan.n_splits), kDecThreads, smem_bytes, s>>>(
+    kern<<<(unsigned)(units * plan.n_splits), kMmaThreads, smem_bytes, s>>>(
         static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(K),
         static_cast<const __nv_bfloat16*>(V), g, cur_len_dev, max_len, scale * kLog2e, partial,
         plan.n_splits);
