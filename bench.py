@@ -38,7 +38,7 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes (read + written) per algorithmic byte of the dominant kernel, from the ncu capture
 # summarised in profiles/decode_split_mma_kernel_llama3-8b-32k_4layers.md (a 4-layer case; the
 # traffic is proportional to the tokens streamed).  Set to None whenever that kernel changes.
-DECODE_TRAFFIC_RATIO = 1.0062
+DECODE_TRAFFIC_RATIO = 1.0055
 
 
 def workload(args):
@@ -163,7 +163,8 @@ class Job:
         self.out = torch.zeros((w.decode_steps, w.B, w.L, w.Hq, w.D), dtype=torch.float32,
                                device=device)
         self.ws = l2.new_workspace(l2.Layout(self.K, q_heads=w.Hq), w.T, device)
-        self.launches_per_step = 3 + 2 * w.decode_steps
+        # norm pass (with the selection inside) + gather, then split + merge per decode step
+        self.launches_per_step = 2 + 2 * w.decode_steps
 
     def compress(self):
         self.l2.select_compact(self.K, self.V, self.lens, self.keep, self.w.T, self.unc, self.K_c,

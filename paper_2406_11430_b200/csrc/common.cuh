@@ -26,6 +26,11 @@ struct Geom {
   long long sb, sl, sh, st;
 };
 
+// Result of the selection for one (b, l, h) unit, consumed by the gather kernel.
+struct UnitRec { uint32_t thr; int32_t admit; int32_t n_keep; uint32_t flags; };
+constexpr uint32_t kFlagIdentity = 1u;           // every valid token is kept
+constexpr uint32_t kFlagNoKeys = 2u;             // keys were not precomputed for this unit
+
 struct LayerMask {
   uint32_t w[kMaxLayers / 32];
   __host__ __device__ bool test(int l) const { return (w[l >> 5] >> (l & 31)) & 1u; }
@@ -48,6 +53,7 @@ struct WorkspacePlan {
   size_t sumsq_off;      // float  [units][ld_sumsq]         ordering keys of the input cache
   size_t unit_off;       // uint32 [units][4]                threshold, admitted ties, kept, flags
   size_t chunk_off;      // int32  [units][n_chunks][2]      slot base / equal-keys-before per chunk
+  size_t ticket_off;     // int32  [units]                   norm CTAs finished per unit (rests at 0)
   size_t partial_off;    // float  [B*L*Hq][n_splits][D + 2] decode partials
   size_t total;
   long long ld_sumsq;
@@ -66,6 +72,7 @@ inline WorkspacePlan plan_workspace(const l2kv_layout& a, int max_len) {
   p.sumsq_off = off;   off += (size_t)round_up_ll(units * p.ld_sumsq * 4, 256);
   p.unit_off = off;    off += (size_t)round_up_ll(units * 16, 256);
   p.chunk_off = off;   off += (size_t)round_up_ll(units * p.n_chunks * 8, 256);
+  p.ticket_off = off;  off += (size_t)round_up_ll(units * 4, 256);
   p.partial_off = off;
   off += (size_t)round_up_ll((long long)a.batch * a.layers * a.q_heads * p.n_splits *
                                  (a.head_dim + 2) * 4, 256);
@@ -125,6 +132,36 @@ __device__ __forceinline__ float piece_sumsq_reduce(const uint4& v) {
   return acc;
 }
 
+// Sums N per-lane values over the LPR adjacent lanes that share a row, N <= LPR.  Halving
+// exchange: at each step a lane keeps half of its values and hands the other half to its
+// partner (lane ^ off), so N values cost N - 1 + log2(LPR / N) shuffles instead of
+// N * log2(LPR).  Every value is still summed over the lanes by the butterfly off = LPR/2 .. 1
+// (x[i] + x[i ^ off] at each level), so the result has the bits of the plain butterfly.  On
+// return d[0] is complete for value number  piece / (LPR / N).  Must be reached by whole warps.
+template <int N, int LPR>
+__device__ __forceinline__ float halving_reduce(float (&d)[N], int piece) {
+  int cnt = N;
+#pragma unroll
+  for (int off = LPR / 2; off >= 1; off >>= 1) {
+    if (cnt > 1) {
+      const int half = cnt / 2;
+      const bool upper = piece & off;
+#pragma unroll
+      for (int i = 0; i < (N > 1 ? N / 2 : 1); ++i) {
+        if (i < half) {
+          const float send = upper ? d[i] : d[i + half];
+          const float keep = upper ? d[i + half] : d[i];
+          d[i] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+        }
+      }
+      cnt = half;
+    } else {
+      d[0] += __shfl_xor_sync(0xffffffffu, d[0], off);
+    }
+  }
+  return d[0];
+}
+
 // Total order on (key bits, position) used everywhere: non-negative floats order as
 // their bit patterns.  For the keep-highest policy the bits are complemented.
 __device__ __forceinline__ uint32_t order_bits(float sumsq, int policy) {
@@ -133,8 +170,18 @@ __device__ __forceinline__ uint32_t order_bits(float sumsq, int policy) {
 }
 
 // Launchers, one per source file (arguments already validated by the C entry points).
+// Arguments of the selection that the norm pass runs for each unit as its last chunk finishes.
+struct SelectArgs {
+  const int32_t* keep_dev;
+  int out_t_cap, policy, n_chunks;
+  LayerMask unc;
+  UnitRec* unit_rec;
+  int2* chunk_rec;
+  int32_t* tickets;
+  int32_t* kept_len_dev;
+};
 int launch_key_norms(const void* K, const Geom& g, int dtype, const int32_t* len_dev, int max_len,
-                     float* sumsq, long long ld_sumsq, float* norm_out, const LayerMask* skip,
+                     float* sumsq, long long ld_sumsq, float* norm_out, const SelectArgs* select,
                      cudaStream_t s);
 int launch_select_compact(const void* K, const void* V, const Geom& gi, int dtype,
                           const int32_t* len_dev, const int32_t* keep_dev, int max_len,

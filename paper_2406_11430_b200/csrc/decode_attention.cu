@@ -19,34 +19,6 @@ constexpr int kDecThreads = 256;
 constexpr int kDecUnroll = 4;
 constexpr float kLog2e = 1.4426950408889634f;
 
-// Sums G per-lane partial dot products over the LPR lanes that share a row.  Halving
-// exchange: at each step a lane keeps half of its values and hands the other half to its
-// partner, so G values cost G - 1 + log2(LPR / G) shuffles instead of G * log2(LPR).
-// On return d[0] is complete for head  piece / (LPR / G).
-template <int G, int LPR>
-__device__ __forceinline__ float reduce_heads(float (&d)[G], int piece) {
-  int cnt = G;
-#pragma unroll
-  for (int off = LPR / 2; off >= 1; off >>= 1) {
-    if (cnt > 1) {
-      const int half = cnt / 2;
-      const bool upper = piece & off;
-#pragma unroll
-      for (int i = 0; i < G / 2; ++i) {
-        if (i < half) {
-          const float send = upper ? d[i] : d[i + half];
-          const float keep = upper ? d[i + half] : d[i];
-          d[i] = keep + __shfl_xor_sync(0xffffffffu, send, off);
-        }
-      }
-      cnt = half;
-    } else {
-      d[0] += __shfl_xor_sync(0xffffffffu, d[0], off);
-    }
-  }
-  return d[0];
-}
-
 template <typename T, int D, int G>
 __global__ void __launch_bounds__(kDecThreads)
 decode_split_kernel(const T* __restrict__ q, const T* __restrict__ K, const T* __restrict__ V,
@@ -109,7 +81,7 @@ decode_split_kernel(const T* __restrict__ q, const T* __restrict__ K, const T* _
         for (int e = 0; e < EPV; ++e) a = fmaf(qf[gi][e], x[e], a);
         d[gi] = a;
       }
-      const float s = reduce_heads<G, LPR>(d, piece);
+      const float s = halving_reduce<G, LPR>(d, piece);
       if (writer && tl < nt) s_buf[tl * G + my_head] = s;
     }
   }

@@ -2,79 +2,144 @@
 // cached key row (the ordering key of the compression) and, optionally, its square
 // root (the L2 norm itself).  HBM-bound: each byte of K is read exactly once with
 // 16-byte coalesced loads; LPR = row bytes / 16 adjacent lanes own one row.
-#include "common.cuh"
+//
+// Inside l2kv_select_compact the same pass also runs the selection: the CTA that finishes
+// the last chunk of a unit (an atomic ticket per unit, nobody waits) selects that unit's
+// threshold while the other CTAs keep streaming, so selection costs no time of its own
+// except after the very last units.
+#include "select_unit.cuh"
 
 namespace l2kv {
 
 constexpr int kNormThreads = 256;
-constexpr int kNormUnroll = 8;
+constexpr int kNormUnroll = 8;                 // rows per thread per step, all loads in flight
 constexpr int kNormRowsPerCta = 1024;
 
-template <typename T, int D>
+template <typename T, int D, bool SEL>
 __global__ void __launch_bounds__(kNormThreads)
 key_norms_kernel(const T* __restrict__ K, Geom g, const int32_t* __restrict__ len_dev,
                  float* __restrict__ sumsq, long long ld, float* __restrict__ norm_out,
-                 LayerMask skip, int use_skip, int chunks_per_unit, int max_len) {
+                 int chunks_per_unit, int max_len, SelectArgs sel) {
   constexpr int LPR = D / Elem<T>::kPerVec;            // lanes per row
-  constexpr int RPS = kNormThreads / LPR;              // rows per load step of the CTA
+  constexpr int RPS = kNormThreads / LPR;              // row groups of the CTA
+  constexpr int U = kNormUnroll;
+  static_assert(U <= LPR, "the halving reduction needs at least as many lanes as rows");
   const long long unit = blockIdx.x / chunks_per_unit;
   const int chunk = blockIdx.x % chunks_per_unit;
   const int h = (int)(unit % g.H);
   const int l = (int)((unit / g.H) % g.L);
   const int b = (int)(unit / ((long long)g.H * g.L));
-  if (use_skip && skip.test(l)) return;
-  const int len = min(len_dev[b], min(max_len, g.t_cap));
+  const int tid = threadIdx.x;
+  const int len = max(0, min(len_dev[b], min(max_len, g.t_cap)));
+
+  if constexpr (SEL) {
+    // Units that need no keys: copied layers and empty sequences get their record here.
+    const bool whole = sel.unc.test(l);
+    if (whole || len == 0) {
+      if (chunk == 0) {
+        const int keep = min(len, sel.out_t_cap);
+        identity_unit<kNormThreads>(len, keep, true, sel.unit_rec + unit,
+                                    sel.chunk_rec + unit * sel.n_chunks);
+        if (h == 0 && tid == 0) sel.kept_len_dev[b * g.L + l] = keep;
+      }
+      return;
+    }
+  }
   const int row0 = chunk * kNormRowsPerCta;
   if (row0 >= len) return;
   const int row_end = min(len, row0 + kNormRowsPerCta);
 
-  const int piece = threadIdx.x % LPR;
-  const int sub = threadIdx.x / LPR;
+  const int piece = tid % LPR;
+  const int sub = tid / LPR;
   const T* base = K + b * g.sb + l * g.sl + h * g.sh + (long long)piece * Elem<T>::kPerVec;
   float* out = sumsq + unit * ld;
   float* nout = norm_out ? norm_out + unit * ld : nullptr;
+  const int my_row = piece / (LPR / U);                // which of its U rows this lane reports
+  const bool writer = (piece % (LPR / U)) == 0;
 
-  // Loop bounds are uniform over the CTA so that the shuffles below always see full warps.
-  for (int rb = row0; rb < row_end; rb += RPS * kNormUnroll) {
-    uint4 v[kNormUnroll];
+  // Thread (sub, piece) owns piece `piece` of rows rb + sub * U + [0, U).  Loop bounds are
+  // uniform over the CTA so that the shuffles always see full warps.
+  for (int rb = row0; rb < row_end; rb += RPS * U) {
+    uint4 v[U];
+    const int t0 = rb + sub * U;
 #pragma unroll
-    for (int i = 0; i < kNormUnroll; ++i) {
-      const int t = rb + i * RPS + sub;
-      v[i] = (t < row_end) ? ld_stream(base + (long long)t * g.st) : make_uint4(0, 0, 0, 0);
+    for (int i = 0; i < U; ++i)
+      v[i] = (t0 + i < row_end) ? ld_stream(base + (long long)(t0 + i) * g.st)
+                                : make_uint4(0, 0, 0, 0);
+    float p[U];
+#pragma unroll
+    for (int i = 0; i < U; ++i) {
+      float x[Elem<T>::kPerVec];
+      Elem<T>::unpack(v[i], x);
+      float acc = 0.f;
+#pragma unroll
+      for (int e = 0; e < Elem<T>::kPerVec; ++e) acc = __fmaf_rn(x[e], x[e], acc);
+      p[i] = acc;
     }
-#pragma unroll
-    for (int i = 0; i < kNormUnroll; ++i) {
-      const int t = rb + i * RPS + sub;
-      const float s = piece_sumsq_reduce<T, LPR>(v[i]);
-      if (piece == 0 && t < row_end) {
-        out[t] = s;
-        if (nout) nout[t] = sqrtf(s);
+    const float s = halving_reduce<U, LPR>(p, piece);
+    const int t = t0 + my_row;
+    if (writer && t < row_end) {
+      out[t] = s;
+      if (nout) nout[t] = sqrtf(s);
+    }
+  }
+
+  if constexpr (SEL) {
+    __shared__ SelectSmem sm;
+    __shared__ int s_last;
+    __threadfence();                                     // this CTA's keys are visible device-wide
+    __syncthreads();
+    if (tid == 0) {
+      const int n_ctas = (len + kNormRowsPerCta - 1) / kNormRowsPerCta;
+      s_last = atomicAdd(sel.tickets + unit, 1) == n_ctas - 1;
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();                                     // see the other CTAs' keys
+    const int keep_req = max(0, min(sel.keep_dev[b], len));
+    const int keep = min(keep_req, sel.out_t_cap);       // rows that fit the output; the rest is cut
+    if (h == 0 && tid == 0) sel.kept_len_dev[b * g.L + l] = keep;
+    if (keep_req == len) {
+      identity_unit<kNormThreads>(len, keep, false, sel.unit_rec + unit,
+                                  sel.chunk_rec + unit * sel.n_chunks);
+    } else if (keep == 0) {
+      if (tid == 0) {
+        UnitRec r; r.thr = 0u; r.admit = 0; r.n_keep = 0; r.flags = 0u;
+        sel.unit_rec[unit] = r;
       }
+    } else {
+      select_unit<kNormThreads>(sm, out, len, keep, sel.policy, sel.unit_rec + unit,
+                                sel.chunk_rec + unit * sel.n_chunks);
     }
+    if (tid == 0) sel.tickets[unit] = 0;                 // the ticket rests at zero between calls
   }
 }
 
 template <typename T, int D>
 static int launch_norms_t(const void* K, const Geom& g, const int32_t* len_dev, int max_len,
-                          float* sumsq, long long ld, float* norm_out, const LayerMask* skip,
+                          float* sumsq, long long ld, float* norm_out, const SelectArgs* select,
                           cudaStream_t s) {
   const long long units = (long long)g.B * g.L * g.H;
-  const int chunks = (max_len + kNormRowsPerCta - 1) / kNormRowsPerCta;
+  int chunks = (max_len + kNormRowsPerCta - 1) / kNormRowsPerCta;
+  if (select && chunks < 1) chunks = 1;                  // records are written even for max_len 0
   if (units == 0 || chunks == 0) return L2KV_OK;
   const long long blocks = units * chunks;
   if (blocks > 0x7fffffffLL) return L2KV_ERR_OUT_OF_RANGE;
-  LayerMask m = {};
-  if (skip) m = *skip;
-  key_norms_kernel<T, D><<<(unsigned)blocks, kNormThreads, 0, s>>>(
-      static_cast<const T*>(K), g, len_dev, sumsq, ld, norm_out, m, skip ? 1 : 0, chunks, max_len);
+  if (select) {
+    key_norms_kernel<T, D, true><<<(unsigned)blocks, kNormThreads, 0, s>>>(
+        static_cast<const T*>(K), g, len_dev, sumsq, ld, norm_out, chunks, max_len, *select);
+  } else {
+    key_norms_kernel<T, D, false><<<(unsigned)blocks, kNormThreads, 0, s>>>(
+        static_cast<const T*>(K), g, len_dev, sumsq, ld, norm_out, chunks, max_len, SelectArgs{});
+  }
   return cudaGetLastError() == cudaSuccess ? L2KV_OK : L2KV_ERR_CUDA;
 }
 
 int launch_key_norms(const void* K, const Geom& g, int dtype, const int32_t* len_dev, int max_len,
-                     float* sumsq, long long ld_sumsq, float* norm_out, const LayerMask* skip,
+                     float* sumsq, long long ld_sumsq, float* norm_out, const SelectArgs* select,
                      cudaStream_t s) {
 #define L2KV_KN(T, D) \
-  return launch_norms_t<T, D>(K, g, len_dev, max_len, sumsq, ld_sumsq, norm_out, skip, s)
+  return launch_norms_t<T, D>(K, g, len_dev, max_len, sumsq, ld_sumsq, norm_out, select, s)
   if (dtype == L2KV_BF16) {
     if (g.D == 128) L2KV_KN(__nv_bfloat16, 128);
     if (g.D == 64) L2KV_KN(__nv_bfloat16, 64);

@@ -1,8 +1,8 @@
 // Selection and compaction.
 //
-//   select_kernel   one CTA per (b, l, h): exact k-th smallest of the ordering keys by a
-//                   most-significant-digit radix select (4 passes of 8 bits) over the
-//                   L2-resident key array, then per-chunk slot bases by a scan.
+//   selection       runs inside the norm pass (key_norms.cu, select_unit.cuh): exact k-th
+//                   smallest of the ordering keys by a most-significant-digit radix select
+//                   (4 passes of 8 bits), then per-chunk slot bases by a scan.
 //   gather_kernel   one CTA per (unit, chunk of input tokens): rebuilds the keep flags
 //                   from the threshold, ranks the kept tokens with a block scan and copies
 //                   their K and V rows (16-byte pieces, LPR lanes per row) to the dense,
@@ -14,140 +14,8 @@
 
 namespace l2kv {
 
-constexpr int kSelectThreads = 1024;
 constexpr int kGatherThreads = 256;
 constexpr int kGatherUnroll = 4;
-constexpr uint32_t kFlagIdentity = 1u;           // every valid token is kept
-constexpr uint32_t kFlagNoKeys = 2u;             // keys were not precomputed for this unit
-
-struct UnitRec { uint32_t thr; int32_t admit; int32_t n_keep; uint32_t flags; };
-
-__global__ void __launch_bounds__(kSelectThreads)
-select_kernel(const float* __restrict__ sumsq, long long ld, Geom g,
-              const int32_t* __restrict__ len_dev, const int32_t* __restrict__ keep_dev,
-              int max_len, int out_t_cap, LayerMask unc, int policy,
-              UnitRec* __restrict__ unit_rec, int2* __restrict__ chunk_rec, int n_chunks,
-              int32_t* __restrict__ kept_len_dev) {
-  __shared__ int hist[256];
-  __shared__ int s_bucket, s_before;
-  __shared__ int c_less[kMaxChunks];
-  __shared__ int c_eq[kMaxChunks];
-
-  const long long unit = blockIdx.x;
-  const int h = (int)(unit % g.H);
-  const int l = (int)((unit / g.H) % g.L);
-  const int b = (int)(unit / ((long long)g.H * g.L));
-  const int tid = threadIdx.x;
-  const int len = max(0, min(len_dev[b], min(max_len, g.t_cap)));
-  const bool whole = unc.test(l);
-  const int keep_req = whole ? len : max(0, min(keep_dev[b], len));
-  const bool identity = whole || keep_req == len;
-  const int keep = min(keep_req, out_t_cap);      // rows that fit the output; the rest is cut
-  if (h == 0 && tid == 0) kept_len_dev[b * g.L + l] = keep;
-
-  const int my_chunks = (len + kGatherChunk - 1) / kGatherChunk;
-  int2* crec = chunk_rec + unit * n_chunks;
-
-  if (identity) {
-    if (tid == 0) {
-      UnitRec r; r.thr = 0xffffffffu; r.admit = 0; r.n_keep = keep;
-      r.flags = kFlagIdentity | (whole ? kFlagNoKeys : 0u);
-      unit_rec[unit] = r;
-    }
-    for (int c = tid; c < my_chunks; c += kSelectThreads) crec[c] = make_int2(c * kGatherChunk, 0);
-    return;
-  }
-  if (keep == 0) {
-    if (tid == 0) {
-      UnitRec r; r.thr = 0u; r.admit = 0; r.n_keep = 0; r.flags = 0u;
-      unit_rec[unit] = r;
-    }
-    for (int c = tid; c < my_chunks; c += kSelectThreads) crec[c] = make_int2(0, 0);
-    return;
-  }
-
-  const float* key = sumsq + unit * ld;
-  uint32_t prefix = 0, mask = 0;
-  int k_rem = keep;
-  for (int shift = 24; shift >= 0; shift -= 8) {
-    if (tid < 256) hist[tid] = 0;
-    __syncthreads();
-    // Run-length accumulation: neighbouring tokens mostly share the high digits.
-    int cur = -1, cnt = 0;
-    for (int t = tid; t < len; t += kSelectThreads) {
-      const uint32_t kb = order_bits(key[t], policy);
-      if ((kb & mask) == prefix) {
-        const int d = (kb >> shift) & 255;
-        if (d == cur) {
-          ++cnt;
-        } else {
-          if (cnt) atomicAdd(&hist[cur], cnt);
-          cur = d; cnt = 1;
-        }
-      }
-    }
-    if (cnt) atomicAdd(&hist[cur], cnt);
-    __syncthreads();
-    if (tid < 32) {
-      // 8 bins per lane: lane totals -> warp scan -> locate the bin holding rank k_rem.
-      int v[8], tot = 0;
-#pragma unroll
-      for (int i = 0; i < 8; ++i) { v[i] = hist[tid * 8 + i]; tot += v[i]; }
-      int inc = tot;
-#pragma unroll
-      for (int off = 1; off < 32; off <<= 1) {
-        const int n = __shfl_up_sync(0xffffffffu, inc, off);
-        if (tid >= off) inc += n;
-      }
-      int before = inc - tot;
-      if (before < k_rem && k_rem <= inc) {
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          if (before < k_rem && k_rem <= before + v[i]) { s_bucket = tid * 8 + i; s_before = before; }
-          before += v[i];
-        }
-      }
-    }
-    __syncthreads();
-    prefix |= (uint32_t)s_bucket << shift;
-    mask |= 255u << shift;
-    k_rem -= s_before;
-    __syncthreads();
-  }
-  const uint32_t thr = prefix;      // the keep-th smallest key; k_rem of its copies are admitted
-  if (tid == 0) {
-    UnitRec r; r.thr = thr; r.admit = k_rem; r.n_keep = keep; r.flags = 0u;
-    unit_rec[unit] = r;
-  }
-
-  // Per-chunk counts of keys below / equal to the threshold, one warp per chunk.
-  const int warp = tid >> 5, lane = tid & 31;
-  for (int c = warp; c < my_chunks; c += kSelectThreads / 32) {
-    const int t0 = c * kGatherChunk;
-    int nl = 0, ne = 0;
-    for (int t = t0 + lane; t < min(len, t0 + kGatherChunk); t += 32) {
-      const uint32_t kb = order_bits(key[t], policy);
-      nl += kb < thr;
-      ne += kb == thr;
-    }
-#pragma unroll
-    for (int off = 16; off >= 1; off >>= 1) {
-      nl += __shfl_xor_sync(0xffffffffu, nl, off);
-      ne += __shfl_xor_sync(0xffffffffu, ne, off);
-    }
-    if (lane == 0) { c_less[c] = nl; c_eq[c] = ne; }
-  }
-  __syncthreads();
-  if (tid == 0) {
-    int slot = 0, eq_before = 0;
-    for (int c = 0; c < my_chunks; ++c) {
-      crec[c] = make_int2(slot, eq_before);
-      const int adm = max(0, min(c_eq[c], k_rem - eq_before));
-      slot += c_less[c] + adm;
-      eq_before += c_eq[c];
-    }
-  }
-}
 
 template <typename T, int D>
 __global__ void __launch_bounds__(kGatherThreads)
@@ -275,14 +143,16 @@ static int launch_sc_t(const void* K, const void* V, const Geom& gi, const int32
   float* sumsq = reinterpret_cast<float*>(ws + plan.sumsq_off);
   UnitRec* urec = reinterpret_cast<UnitRec*>(ws + plan.unit_off);
   int2* crec = reinterpret_cast<int2*>(ws + plan.chunk_off);
-  // Keys of the layers that are compressed (the others are copied whole).
+  // Keys of the layers that are compressed (the others are copied whole), and, as each
+  // unit's last chunk of keys lands, its selection.
+  SelectArgs sel;
+  sel.keep_dev = keep_dev; sel.out_t_cap = go.t_cap; sel.policy = policy;
+  sel.n_chunks = plan.n_chunks; sel.unc = unc; sel.unit_rec = urec; sel.chunk_rec = crec;
+  sel.tickets = reinterpret_cast<int32_t*>(ws + plan.ticket_off);
+  sel.kept_len_dev = kept_len_dev;
   const int rc = launch_key_norms(K, gi, Elem<T>::kDtype, len_dev, max_len, sumsq, plan.ld_sumsq,
-                                  nullptr, &unc, s);
+                                  nullptr, &sel, s);
   if (rc != L2KV_OK) return rc;
-  select_kernel<<<(unsigned)units, kSelectThreads, 0, s>>>(
-      sumsq, plan.ld_sumsq, gi, len_dev, keep_dev, max_len, go.t_cap, unc, policy, urec, crec,
-      plan.n_chunks, kept_len_dev);
-  if (cudaGetLastError() != cudaSuccess) return L2KV_ERR_CUDA;
   if (max_len > 0) {
     gather_kernel<T, D><<<(unsigned)(units * plan.n_chunks), kGatherThreads, 0, s>>>(
         static_cast<const T*>(K), static_cast<const T*>(V), gi, static_cast<T*>(K_out),

@@ -1,0 +1,137 @@
+// Exact k-selection for one (b, l, h) unit, run by one CTA of NT threads.
+//
+// Finds the keep-th smallest ordering key by a most-significant-digit radix select (4
+// passes of 8 bits) over the unit's key array in global memory (L2-resident: it was
+// written moments before), then counts, per gather chunk, the keys below and equal to the
+// threshold and scans those counts into slot bases.  No waiting on other CTAs anywhere.
+#pragma once
+
+#include "common.cuh"
+
+namespace l2kv {
+
+struct SelectSmem {
+  int hist[256];
+  int bucket, before;
+  int c_less[kMaxChunks];
+  int c_eq[kMaxChunks];
+};
+
+// Keys may have been written by other CTAs of the same grid: read them through L2.
+__device__ __forceinline__ uint32_t load_key_bits(const float* p, int policy) {
+  return order_bits(__ldcg(p), policy);
+}
+
+template <int NT>
+__device__ void select_unit(SelectSmem& sm, const float* __restrict__ key, int len, int keep,
+                            int policy, UnitRec* __restrict__ rec, int2* __restrict__ crec) {
+  constexpr int kBatch = 8;                      // independent key loads in flight per thread
+  const int tid = threadIdx.x;
+  const int my_chunks = (len + kGatherChunk - 1) / kGatherChunk;
+  uint32_t prefix = 0, mask = 0;
+  int k_rem = keep;
+  for (int shift = 24; shift >= 0; shift -= 8) {
+    for (int i = tid; i < 256; i += NT) sm.hist[i] = 0;
+    __syncthreads();
+    // Run-length accumulation: neighbouring tokens mostly share the high digits, so the
+    // shared-memory atomics of the first passes collapse to a few per thread.
+    int cur = -1, cnt = 0;
+    for (int base = 0; base < len; base += NT * kBatch) {
+      uint32_t kb[kBatch];
+#pragma unroll
+      for (int j = 0; j < kBatch; ++j) {
+        const int t = base + j * NT + tid;
+        kb[j] = t < len ? load_key_bits(key + t, policy) : 0u;
+      }
+#pragma unroll
+      for (int j = 0; j < kBatch; ++j) {
+        const int t = base + j * NT + tid;
+        if (t < len && (kb[j] & mask) == prefix) {
+          const int d = (kb[j] >> shift) & 255;
+          if (d == cur) {
+            ++cnt;
+          } else {
+            if (cnt) atomicAdd(&sm.hist[cur], cnt);
+            cur = d; cnt = 1;
+          }
+        }
+      }
+    }
+    if (cnt) atomicAdd(&sm.hist[cur], cnt);
+    __syncthreads();
+    if (tid < 32) {
+      // 8 bins per lane: lane totals -> warp scan -> locate the bin holding rank k_rem.
+      int v[8], tot = 0;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) { v[i] = sm.hist[tid * 8 + i]; tot += v[i]; }
+      int inc = tot;
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const int n = __shfl_up_sync(0xffffffffu, inc, off);
+        if (tid >= off) inc += n;
+      }
+      int before = inc - tot;
+      if (before < k_rem && k_rem <= inc) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          if (before < k_rem && k_rem <= before + v[i]) { sm.bucket = tid * 8 + i; sm.before = before; }
+          before += v[i];
+        }
+      }
+    }
+    __syncthreads();
+    prefix |= (uint32_t)sm.bucket << shift;
+    mask |= 255u << shift;
+    k_rem -= sm.before;
+    __syncthreads();
+  }
+  const uint32_t thr = prefix;      // the keep-th smallest key; k_rem of its copies are admitted
+  if (tid == 0) {
+    UnitRec r; r.thr = thr; r.admit = k_rem; r.n_keep = keep; r.flags = 0u;
+    *rec = r;
+  }
+  // Per-chunk counts of keys below / equal to the threshold, one warp per chunk.
+  const int warp = tid >> 5, lane = tid & 31;
+  for (int c = warp; c < my_chunks; c += NT / 32) {
+    const int t0 = c * kGatherChunk;
+    const int t1 = min(len, t0 + kGatherChunk);
+    int nl = 0, ne = 0;
+#pragma unroll 4
+    for (int t = t0 + lane; t < t1; t += 32) {
+      const uint32_t kb = load_key_bits(key + t, policy);
+      nl += kb < thr;
+      ne += kb == thr;
+    }
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) {
+      nl += __shfl_xor_sync(0xffffffffu, nl, off);
+      ne += __shfl_xor_sync(0xffffffffu, ne, off);
+    }
+    if (lane == 0) { sm.c_less[c] = nl; sm.c_eq[c] = ne; }
+  }
+  __syncthreads();
+  if (tid == 0) {
+    int slot = 0, eq_before = 0;
+    for (int c = 0; c < my_chunks; ++c) {
+      crec[c] = make_int2(slot, eq_before);
+      const int adm = max(0, min(sm.c_eq[c], k_rem - eq_before));
+      slot += sm.c_less[c] + adm;
+      eq_before += sm.c_eq[c];
+    }
+  }
+}
+
+// Record of a unit whose valid tokens are all kept (uncompressed layer, or keep == len).
+template <int NT>
+__device__ void identity_unit(int len, int keep, bool keys_missing, UnitRec* __restrict__ rec,
+                              int2* __restrict__ crec) {
+  const int my_chunks = (len + kGatherChunk - 1) / kGatherChunk;
+  if (threadIdx.x == 0) {
+    UnitRec r; r.thr = 0xffffffffu; r.admit = 0; r.n_keep = keep;
+    r.flags = kFlagIdentity | (keys_missing ? kFlagNoKeys : 0u);
+    *rec = r;
+  }
+  for (int c = threadIdx.x; c < my_chunks; c += NT) crec[c] = make_int2(c * kGatherChunk, 0);
+}
+
+}  // namespace l2kv
