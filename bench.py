@@ -170,6 +170,11 @@ class Job:
         self.l2.select_compact(self.K, self.V, self.lens, self.keep, self.w.T, self.unc, self.K_c,
                                self.V_c, self.idx, self.sumsq, self.cur, self.ws)
 
+    def compress_variant(self, policy=0, sumsq_in=None):
+        self.l2.select_compact(self.K, self.V, self.lens, self.keep, self.w.T, self.unc, self.K_c,
+                               self.V_c, self.idx, self.sumsq, self.cur, self.ws, policy=policy,
+                               seed=1, sumsq_in=sumsq_in)
+
     def decode(self, s):
         self.l2.decode_attention(self.q[s], self.K_c, self.V_c, self.cur, self.w.T, self.out[s],
                                  self.ws)
@@ -215,6 +220,8 @@ def run_gpu(args):
     c_ms = max_over_ranks(c_ms, world, device)
     d_ms = max_over_ranks(d_ms, world, device)
 
+    variants = time_variants(job, w, cbytes) if (rank == 0 and not args.no_variants) else None
+
     # end to end: inputs start in pinned host memory, results end there
     e2e = None
     if not args.no_e2e:
@@ -253,11 +260,38 @@ def run_gpu(args):
         "gpu_launches": job.launches_per_step * args.steps,
         "clocks": clocks,
     }
+    if variants:
+        line["variants"] = variants
     if e2e:
         line["e2e"] = e2e
     if not args.no_cpu_baseline and world == 1:
         line["cpu_baseline"] = cpu_baseline(w, target_s=args.cpu_seconds)
     print(json.dumps(line))
+
+
+def time_variants(job, w, cbytes, reps=5):
+    """Other forms of the compression pass, outside the main timed region: keys kept from
+    cache-write time (no pass over K), and the keep-random / keep-highest ablation policies."""
+    keys = torch.zeros((w.B, w.L, w.Hkv, w.T), dtype=torch.float32, device=job.dev)
+    job.l2.key_norms(job.K, job.lens, w.T, keys)
+    n_unc = len(job.unc)
+    norm_pass = w.B * (w.L - n_unc) * w.Hkv * w.T * w.D * w.elem_bytes
+    out = {}
+    for name, kw, nbytes in (("keys_given", dict(sumsq_in=keys), cbytes - norm_pass),
+                             ("keep_random", dict(policy=2), cbytes - norm_pass),
+                             ("keep_highest", dict(policy=1), cbytes)):
+        for _ in range(2):
+            job.compress_variant(**kw)
+        t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+        t0.record()
+        for _ in range(reps):
+            job.compress_variant(**kw)
+        t1.record(); torch.cuda.synchronize()
+        ms = t0.elapsed_time(t1) / reps
+        out[name] = {"ms": round(ms, 3), "bytes": nbytes, "GBps": round(nbytes / ms / 1e6, 1)}
+    job.compress()                     # leave the cache as the method's own policy makes it
+    torch.cuda.synchronize()
+    return out
 
 
 def run_e2e(job, w, step_bytes, world, device, args):
@@ -374,6 +408,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-variants", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--layers", type=int, default=0, help="profiling aid: fewer layers")
     ap.add_argument("--context", type=int, default=0, help="profiling aid: shorter context")

@@ -63,9 +63,19 @@ typedef enum {
 
 typedef enum { L2KV_F32 = 0, L2KV_BF16 = 1 } l2kv_dtype;
 
-/* Which tokens survive compression.  LOWEST is the paper's method; HIGHEST is
- * its ablation baseline (Section 4: keeping the highest-norm tokens). */
-typedef enum { L2KV_KEEP_LOWEST_NORM = 0, L2KV_KEEP_HIGHEST_NORM = 1 } l2kv_policy;
+/* Which tokens survive compression.  LOWEST is the paper's method; HIGHEST and
+ * RANDOM are its ablation baselines (Section 4: keeping the highest-norm tokens,
+ * keeping random tokens).  RANDOM orders the tokens of unit u = (b * layers + l) *
+ * kv_heads + h by a seeded counter-based key instead of the norm: the upper 32 bits
+ * of the SplitMix64 output function (Steele, Lea, Flood 2014) applied to the state
+ * seed + (u << 32 | t), i.e. z = state + 0x9E3779B97F4A7C15; z = (z ^ z >> 30) *
+ * 0xBF58476D1CE4E5B9; z = (z ^ z >> 27) * 0x94D049BB133111EB; z ^= z >> 31 (mod 2^64);
+ * the `keep` smallest keys are kept, equal keys going to the lower position. */
+typedef enum {
+  L2KV_KEEP_LOWEST_NORM = 0,
+  L2KV_KEEP_HIGHEST_NORM = 1,
+  L2KV_KEEP_RANDOM = 2
+} l2kv_policy;
 
 typedef struct {
   int32_t batch, layers, kv_heads, q_heads, head_dim, t_cap;
@@ -107,6 +117,10 @@ int l2kv_key_norms(const void* K, const l2kv_layout* lay, const int32_t* len_dev
  * idx_out[b,l,h,j] = t_j, sumsq_out[b,l,h,j] = key of t_j, kept_len_dev[b,l] =
  * keep_dev[b].  Layers in uncompressed_layers (host array, may be NULL when
  * n_uncompressed == 0) are copied whole: kept_len = len, idx = identity.
+ * `seed` is used by L2KV_KEEP_RANDOM only.  `sumsq_in` may be NULL; if it is given it
+ * must hold the keys of K as l2kv_key_norms writes them (dense fp32
+ * [batch, layers, kv_heads, in->t_cap], e.g. produced when the rows were written to
+ * the cache): the pass over K that computes the keys is then skipped.
  * Requires 0 <= keep_dev[b] <= len_dev[b] <= max_len <= in->t_cap and kept_len <=
  * out->t_cap (the host checks what it can see: max_len and the layouts; a device
  * value outside its range is clamped).  `in` and `out` must agree in batch, layers,
@@ -116,6 +130,7 @@ int l2kv_key_norms(const void* K, const l2kv_layout* lay, const int32_t* len_dev
 int l2kv_select_compact(const void* K, const void* V, const l2kv_layout* in,
                         const int32_t* len_dev, const int32_t* keep_dev, int32_t max_len,
                         const int32_t* uncompressed_layers, int32_t n_uncompressed, int32_t policy,
+                        uint64_t seed, const float* sumsq_in,
                         void* K_out, void* V_out, const l2kv_layout* out, int32_t* idx_out,
                         float* sumsq_out, int32_t* kept_len_dev, void* workspace,
                         size_t workspace_bytes, void* stream);

@@ -73,8 +73,16 @@ def select(key, keep, policy=0):
     return out
 
 
+def random_key(seed, unit, t):
+    """Ordering key of the keep-random policy for token t of unit (b * L + l) * H + h."""
+    f = lib().l2kv_oracle_random_key
+    f.restype = ctypes.c_uint32
+    f.argtypes = [ctypes.c_uint64, ctypes.c_uint64, ctypes.c_uint32]
+    return int(f(seed & 0xFFFFFFFFFFFFFFFF, unit, t))
+
+
 def compress(K, V, dtype, lens, keep, uncompressed=(), key_mode=0, policy=0, t_cap_out=None,
-             nthreads=1):
+             nthreads=1, seed=0):
     """Whole-cache compression.  Returns dict(K_c, V_c, idx, key, kept_len)."""
     _check(K, dtype)
     _check(V, dtype)
@@ -89,7 +97,8 @@ def compress(K, V, dtype, lens, keep, uncompressed=(), key_mode=0, policy=0, t_c
     kept_len = np.zeros((B, L), dtype=np.int32)
     rc = lib().l2kv_oracle_compress(
         _p(K), _p(V), _DT[dtype], B, L, H, T_cap, D, _p(lens), _p(keep), _p(unc), int(unc.size),
-        int(key_mode), int(policy), int(t_cap_out), _p(K_c), _p(V_c), _p(idx), _p(key),
+        int(key_mode), int(policy), ctypes.c_uint64(int(seed) & 0xFFFFFFFFFFFFFFFF), int(t_cap_out),
+        _p(K_c), _p(V_c), _p(idx), _p(key),
         _p(kept_len), int(nthreads))
     if rc != 0:
         raise ValueError(f"oracle compress: bad argument ({rc})")

@@ -130,6 +130,19 @@ void select_positions(const double* key, int T, int keep, int policy, int32_t* o
   std::copy(kept.begin(), kept.end(), out);
 }
 
+// Ordering key of the keep-random ablation (Section 4: "keeping random tokens"), made
+// reproducible: the upper 32 bits of the SplitMix64 output function (Steele, Lea, Flood,
+// "Fast splittable pseudorandom number generators", 2014) for the state
+// seed + (unit * 2^32 + t), all arithmetic modulo 2^64.
+uint32_t random_key(uint64_t seed, uint64_t unit, uint32_t t) {
+  uint64_t z = seed + (unit * 4294967296ull + t);
+  z += 0x9E3779B97F4A7C15ull;
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+  z = z ^ (z >> 31);
+  return static_cast<uint32_t>(z >> 32);
+}
+
 bool in_list(const int32_t* list, int n, int v) {
   for (int i = 0; i < n; ++i)
     if (list[i] == v) return true;
@@ -171,6 +184,10 @@ void l2kv_oracle_key_sumsq_f32(const void* K, int dtype, int64_t n_rows, int D, 
   for (int64_t r = 0; r < n_rows; ++r) sumsq[r] = row_sumsq_f32_ordered(K, dtype, r * D, D);
 }
 
+uint32_t l2kv_oracle_random_key(uint64_t seed, uint64_t unit, uint32_t t) {
+  return random_key(seed, unit, t);
+}
+
 // a2 on a bare key array.
 void l2kv_oracle_select(const double* key, int T, int keep, int policy, int32_t* idx_out) {
   select_positions(key, T, keep, policy, idx_out);
@@ -192,13 +209,15 @@ int32_t l2kv_oracle_keep_count(int32_t len, double keep_ratio) {
 //               every compressed layer (the paper uses one ratio for all heads)
 //   uncompressed[0..n_unc)  layers copied whole (kept_len = len, identity map)
 //   key_mode    0: fp64 sums (the definition); 1: the GPU's fp32 order
+//   policy      0: keep the lowest norms (the method); 1: keep the highest; 2: keep the
+//               lowest seeded random keys of unit (b * L + l) * H + h (`seed`)
 //   outputs     K_out, V_out [B, L, H, T_cap_out, D] (rows >= kept_len untouched),
 //               idx_out int32, key_out double [B, L, H, T_cap_out], kept_len [B, L]
 // Returns 0, or -1 if an argument is out of range.
 int l2kv_oracle_compress(const void* K, const void* V, int dtype, int B, int L, int H, int T_cap,
                          int D, const int32_t* len, const int32_t* keep,
                          const int32_t* uncompressed, int n_unc, int key_mode, int policy,
-                         int T_cap_out, void* K_out, void* V_out, int32_t* idx_out,
+                         uint64_t seed, int T_cap_out, void* K_out, void* V_out, int32_t* idx_out,
                          double* key_out, int32_t* kept_len, int nthreads) {
   for (int b = 0; b < B; ++b) {
     if (len[b] < 0 || len[b] > T_cap) return -1;
@@ -223,6 +242,10 @@ int l2kv_oracle_compress(const void* K, const void* V, int dtype, int B, int L, 
     std::vector<int32_t> kept(n_keep);
     if (in_list(uncompressed, n_unc, l)) {
       std::iota(kept.begin(), kept.end(), 0);
+    } else if (n_keep > 0 && policy == 2) {
+      std::vector<double> rnd(T);
+      for (int t = 0; t < T; ++t) rnd[t] = static_cast<double>(random_key(seed, uint64_t(u), uint32_t(t)));
+      select_positions(rnd.data(), T, n_keep, 0, kept.data());
     } else if (n_keep > 0) {
       select_positions(key.data(), T, n_keep, policy, kept.data());
     }

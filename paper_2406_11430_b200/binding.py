@@ -11,6 +11,7 @@ _LIB = None
 
 KEEP_LOWEST_NORM = 0
 KEEP_HIGHEST_NORM = 1
+KEEP_RANDOM = 2
 _DTYPE = {torch.float32: 0, torch.bfloat16: 1}
 
 
@@ -50,7 +51,7 @@ def lib():
         L.l2kv_read_device_status.argtypes = [vp, vp, ctypes.POINTER(i32)]
         L.l2kv_key_norms.argtypes = [vp, lay, vp, i32, vp, vp, vp]
         L.l2kv_select_compact.argtypes = [vp, vp, lay, vp, vp, i32, ctypes.POINTER(i32), i32, i32,
-                                          vp, vp, lay, vp, vp, vp, vp, sz, vp]
+                                          ctypes.c_uint64, vp, vp, vp, lay, vp, vp, vp, vp, sz, vp]
         L.l2kv_decode_attention.argtypes = [vp, vp, vp, lay, vp, i32, ctypes.c_float, vp, vp, sz, vp]
         L.l2kv_append_evict.argtypes = [vp, vp, vp, vp, lay, vp, vp, ctypes.POINTER(i32), i32,
                                         vp, vp, vp, vp, sz, vp]
@@ -137,12 +138,14 @@ def key_norms(K, len_dev, max_len, sumsq_out, norm_out=None, stream=None):
 
 
 def select_compact(K, V, len_dev, keep_dev, max_len, uncompressed_layers, K_out, V_out, idx_out,
-                   sumsq_out, kept_len_dev, workspace, policy=KEEP_LOWEST_NORM, stream=None):
+                   sumsq_out, kept_len_dev, workspace, policy=KEEP_LOWEST_NORM, seed=0,
+                   sumsq_in=None, stream=None):
     lin, lout = Layout(K), Layout(K_out)
     arr, n = _layers(uncompressed_layers)
     _check(lib().l2kv_select_compact(
         _ptr(K), _ptr(V), lin.ref(), _ptr(len_dev), _ptr(keep_dev), int(max_len), arr, n,
-        int(policy), _ptr(K_out), _ptr(V_out), lout.ref(), _ptr(idx_out), _ptr(sumsq_out),
+        int(policy), ctypes.c_uint64(int(seed) & 0xFFFFFFFFFFFFFFFF), _ptr(sumsq_in), _ptr(K_out),
+        _ptr(V_out), lout.ref(), _ptr(idx_out), _ptr(sumsq_out),
         _ptr(kept_len_dev), _ptr(workspace), workspace.numel(), _stream(stream)),
         "l2kv_select_compact")
 

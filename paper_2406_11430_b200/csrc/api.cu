@@ -104,12 +104,13 @@ int l2kv_key_norms(const void* K, const l2kv_layout* lay, const int32_t* len_dev
   if (!K || !len_dev || !sumsq_out) return L2KV_ERR_INVALID_ARG;
   if (!aligned16(K)) return L2KV_ERR_MISALIGNED;
   return launch_key_norms(K, make_geom(*lay), lay->dtype, len_dev, max_len, sumsq_out, lay->t_cap,
-                          norm_out, nullptr, static_cast<cudaStream_t>(stream));
+                          norm_out, kKeysOnly, nullptr, static_cast<cudaStream_t>(stream));
 }
 
 int l2kv_select_compact(const void* K, const void* V, const l2kv_layout* in,
                         const int32_t* len_dev, const int32_t* keep_dev, int32_t max_len,
                         const int32_t* uncompressed_layers, int32_t n_uncompressed, int32_t policy,
+                        uint64_t seed, const float* sumsq_in,
                         void* K_out, void* V_out, const l2kv_layout* out, int32_t* idx_out,
                         float* sumsq_out, int32_t* kept_len_dev, void* workspace,
                         size_t workspace_bytes, void* stream) {
@@ -120,7 +121,8 @@ int l2kv_select_compact(const void* K, const void* V, const l2kv_layout* in,
   if (in->batch != out->batch || in->layers != out->layers || in->kv_heads != out->kv_heads ||
       in->head_dim != out->head_dim || in->dtype != out->dtype)
     return L2KV_ERR_INVALID_ARG;
-  if (policy != L2KV_KEEP_LOWEST_NORM && policy != L2KV_KEEP_HIGHEST_NORM)
+  if (policy != L2KV_KEEP_LOWEST_NORM && policy != L2KV_KEEP_HIGHEST_NORM &&
+      policy != L2KV_KEEP_RANDOM)
     return L2KV_ERR_INVALID_ARG;
   if (max_len < 0) return L2KV_ERR_INVALID_ARG;
   if (max_len > in->t_cap) return L2KV_ERR_OUT_OF_RANGE;
@@ -139,7 +141,7 @@ int l2kv_select_compact(const void* K, const void* V, const l2kv_layout* in,
   const WorkspacePlan plan = plan_workspace(*in, max_len);
   if (workspace_bytes < plan.total) return L2KV_ERR_WORKSPACE_TOO_SMALL;
   return launch_select_compact(K, V, make_geom(*in), in->dtype, len_dev, keep_dev, max_len, unc,
-                               policy, K_out, V_out, make_geom(*out), idx_out, sumsq_out,
+                               policy, seed, sumsq_in, K_out, V_out, make_geom(*out), idx_out, sumsq_out,
                                kept_len_dev, static_cast<char*>(workspace), plan,
                                static_cast<cudaStream_t>(stream));
 }

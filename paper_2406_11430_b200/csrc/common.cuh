@@ -162,6 +162,17 @@ __device__ __forceinline__ float halving_reduce(float (&d)[N], int piece) {
   return d[0];
 }
 
+// Ordering key of the keep-random policy: upper half of the SplitMix64 output function
+// (Steele, Lea, Flood 2014) applied to the state seed + (unit << 32 | t).
+__host__ __device__ inline uint32_t random_key_bits(unsigned long long seed, unsigned long long unit,
+                                                    uint32_t t) {
+  unsigned long long z = seed + ((unit << 32) | t) + 0x9E3779B97F4A7C15ull;
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+  z ^= z >> 31;
+  return (uint32_t)(z >> 32);
+}
+
 // Total order on (key bits, position) used everywhere: non-negative floats order as
 // their bit patterns.  For the keep-highest policy the bits are complemented.
 __device__ __forceinline__ uint32_t order_bits(float sumsq, int policy) {
@@ -171,9 +182,11 @@ __device__ __forceinline__ uint32_t order_bits(float sumsq, int policy) {
 
 // Launchers, one per source file (arguments already validated by the C entry points).
 // Arguments of the selection that the norm pass runs for each unit as its last chunk finishes.
+enum KeyMode { kKeysOnly = 0, kKeysFromK = 1, kKeysRandom = 2, kKeysGiven = 3 };
 struct SelectArgs {
   const int32_t* keep_dev;
-  int out_t_cap, policy, n_chunks;
+  int out_t_cap, policy, n_chunks;            // policy: how key bits order (lowest / highest)
+  unsigned long long seed;                    // kKeysRandom
   LayerMask unc;
   UnitRec* unit_rec;
   int2* chunk_rec;
@@ -181,13 +194,14 @@ struct SelectArgs {
   int32_t* kept_len_dev;
 };
 int launch_key_norms(const void* K, const Geom& g, int dtype, const int32_t* len_dev, int max_len,
-                     float* sumsq, long long ld_sumsq, float* norm_out, const SelectArgs* select,
-                     cudaStream_t s);
+                     float* sumsq, long long ld_sumsq, float* norm_out, int key_mode,
+                     const SelectArgs* select, cudaStream_t s);
 int launch_select_compact(const void* K, const void* V, const Geom& gi, int dtype,
                           const int32_t* len_dev, const int32_t* keep_dev, int max_len,
-                          const LayerMask& unc, int policy, void* K_out, void* V_out,
-                          const Geom& go, int32_t* idx_out, float* sumsq_out, int32_t* kept_len_dev,
-                          char* ws, const WorkspacePlan& plan, cudaStream_t s);
+                          const LayerMask& unc, int policy, unsigned long long seed,
+                          const float* sumsq_in, void* K_out, void* V_out, const Geom& go,
+                          int32_t* idx_out, float* sumsq_out, int32_t* kept_len_dev, char* ws,
+                          const WorkspacePlan& plan, cudaStream_t s);
 int launch_decode_attention(const void* q, const void* K, const void* V, const Geom& g, int dtype,
                             const int32_t* cur_len_dev, int max_len, float scale, float* out,
                             char* ws, const WorkspacePlan& plan, cudaStream_t s);

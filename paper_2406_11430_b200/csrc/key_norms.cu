@@ -15,7 +15,7 @@ constexpr int kNormThreads = 256;
 constexpr int kNormUnroll = 8;                 // rows per thread per step, all loads in flight
 constexpr int kNormRowsPerCta = 1024;
 
-template <typename T, int D, bool SEL>
+template <typename T, int D, int MODE>
 __global__ void __launch_bounds__(kNormThreads)
 key_norms_kernel(const T* __restrict__ K, Geom g, const int32_t* __restrict__ len_dev,
                  float* __restrict__ sumsq, long long ld, float* __restrict__ norm_out,
@@ -23,6 +23,7 @@ key_norms_kernel(const T* __restrict__ K, Geom g, const int32_t* __restrict__ le
   constexpr int LPR = D / Elem<T>::kPerVec;            // lanes per row
   constexpr int RPS = kNormThreads / LPR;              // row groups of the CTA
   constexpr int U = kNormUnroll;
+  constexpr bool SEL = MODE != kKeysOnly;
   static_assert(U <= LPR, "the halving reduction needs at least as many lanes as rows");
   const long long unit = blockIdx.x / chunks_per_unit;
   const int chunk = blockIdx.x % chunks_per_unit;
@@ -45,62 +46,71 @@ key_norms_kernel(const T* __restrict__ K, Geom g, const int32_t* __restrict__ le
       return;
     }
   }
-  const int row0 = chunk * kNormRowsPerCta;
-  if (row0 >= len) return;
-  const int row_end = min(len, row0 + kNormRowsPerCta);
-
-  const int piece = tid % LPR;
-  const int sub = tid / LPR;
-  const T* base = K + b * g.sb + l * g.sl + h * g.sh + (long long)piece * Elem<T>::kPerVec;
   float* out = sumsq + unit * ld;
-  float* nout = norm_out ? norm_out + unit * ld : nullptr;
-  const int my_row = piece / (LPR / U);                // which of its U rows this lane reports
-  const bool writer = (piece % (LPR / U)) == 0;
+  if constexpr (MODE != kKeysGiven) {
+    const int row0 = chunk * kNormRowsPerCta;
+    if (row0 >= len) return;
+    const int row_end = min(len, row0 + kNormRowsPerCta);
+    if constexpr (MODE == kKeysRandom) {
+      // Keys that do not depend on K: seeded counter-based bits, stored as raw 32-bit patterns.
+      for (int t = row0 + tid; t < row_end; t += kNormThreads)
+        out[t] = __uint_as_float(random_key_bits(sel.seed, (unsigned long long)unit, (uint32_t)t));
+    } else {
+      const int piece = tid % LPR;
+      const int sub = tid / LPR;
+      const T* base = K + b * g.sb + l * g.sl + h * g.sh + (long long)piece * Elem<T>::kPerVec;
+      float* nout = norm_out ? norm_out + unit * ld : nullptr;
+      const int my_row = piece / (LPR / U);              // which of its U rows this lane reports
+      const bool writer = (piece % (LPR / U)) == 0;
 
-  // Thread (sub, piece) owns piece `piece` of rows rb + sub * U + [0, U).  Loop bounds are
-  // uniform over the CTA so that the shuffles always see full warps.
-  for (int rb = row0; rb < row_end; rb += RPS * U) {
-    uint4 v[U];
-    const int t0 = rb + sub * U;
+      // Thread (sub, piece) owns piece `piece` of rows rb + sub * U + [0, U).  Loop bounds are
+      // uniform over the CTA so that the shuffles always see full warps.
+      for (int rb = row0; rb < row_end; rb += RPS * U) {
+        uint4 v[U];
+        const int t0 = rb + sub * U;
 #pragma unroll
-    for (int i = 0; i < U; ++i)
-      v[i] = (t0 + i < row_end) ? ld_stream(base + (long long)(t0 + i) * g.st)
-                                : make_uint4(0, 0, 0, 0);
-    float p[U];
+        for (int i = 0; i < U; ++i)
+          v[i] = (t0 + i < row_end) ? ld_stream(base + (long long)(t0 + i) * g.st)
+                                    : make_uint4(0, 0, 0, 0);
+        float p[U];
 #pragma unroll
-    for (int i = 0; i < U; ++i) {
-      float x[Elem<T>::kPerVec];
-      Elem<T>::unpack(v[i], x);
-      float acc = 0.f;
+        for (int i = 0; i < U; ++i) {
+          float x[Elem<T>::kPerVec];
+          Elem<T>::unpack(v[i], x);
+          float acc = 0.f;
 #pragma unroll
-      for (int e = 0; e < Elem<T>::kPerVec; ++e) acc = __fmaf_rn(x[e], x[e], acc);
-      p[i] = acc;
-    }
-    const float s = halving_reduce<U, LPR>(p, piece);
-    const int t = t0 + my_row;
-    if (writer && t < row_end) {
-      out[t] = s;
-      if (nout) nout[t] = sqrtf(s);
+          for (int e = 0; e < Elem<T>::kPerVec; ++e) acc = __fmaf_rn(x[e], x[e], acc);
+          p[i] = acc;
+        }
+        const float s = halving_reduce<U, LPR>(p, piece);
+        const int t = t0 + my_row;
+        if (writer && t < row_end) {
+          out[t] = s;
+          if (nout) nout[t] = sqrtf(s);
+        }
+      }
     }
   }
 
   if constexpr (SEL) {
     __shared__ SelectSmem sm;
     __shared__ int s_last;
-    __threadfence();                                     // this CTA's keys are visible device-wide
-    __syncthreads();
-    if (tid == 0) {
-      const int n_ctas = (len + kNormRowsPerCta - 1) / kNormRowsPerCta;
-      s_last = atomicAdd(sel.tickets + unit, 1) == n_ctas - 1;
+    if constexpr (MODE != kKeysGiven) {
+      __threadfence();                                   // this CTA's keys are visible device-wide
+      __syncthreads();
+      if (tid == 0) {
+        const int n_ctas = (len + kNormRowsPerCta - 1) / kNormRowsPerCta;
+        s_last = atomicAdd(sel.tickets + unit, 1) == n_ctas - 1;
+      }
+      __syncthreads();
+      if (!s_last) return;
+      __threadfence();                                   // see the other CTAs' keys
     }
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();                                     // see the other CTAs' keys
     const int keep_req = max(0, min(sel.keep_dev[b], len));
     const int keep = min(keep_req, sel.out_t_cap);       // rows that fit the output; the rest is cut
     if (h == 0 && tid == 0) sel.kept_len_dev[b * g.L + l] = keep;
     if (keep_req == len) {
-      identity_unit<kNormThreads>(len, keep, false, sel.unit_rec + unit,
+      identity_unit<kNormThreads>(len, keep, MODE == kKeysRandom, sel.unit_rec + unit,
                                   sel.chunk_rec + unit * sel.n_chunks);
     } else if (keep == 0) {
       if (tid == 0) {
@@ -108,38 +118,52 @@ key_norms_kernel(const T* __restrict__ K, Geom g, const int32_t* __restrict__ le
         sel.unit_rec[unit] = r;
       }
     } else {
-      select_unit<kNormThreads>(sm, out, len, keep, sel.policy, sel.unit_rec + unit,
+      select_unit<kNormThreads>(sm, out, len, keep, sel.policy,
+                                MODE == kKeysRandom ? kFlagNoKeys : 0u, sel.unit_rec + unit,
                                 sel.chunk_rec + unit * sel.n_chunks);
     }
-    if (tid == 0) sel.tickets[unit] = 0;                 // the ticket rests at zero between calls
+    if (MODE != kKeysGiven && tid == 0) sel.tickets[unit] = 0;   // tickets rest at zero between calls
   }
 }
 
 template <typename T, int D>
 static int launch_norms_t(const void* K, const Geom& g, const int32_t* len_dev, int max_len,
-                          float* sumsq, long long ld, float* norm_out, const SelectArgs* select,
-                          cudaStream_t s) {
+                          float* sumsq, long long ld, float* norm_out, int key_mode,
+                          const SelectArgs* select, cudaStream_t s) {
   const long long units = (long long)g.B * g.L * g.H;
   int chunks = (max_len + kNormRowsPerCta - 1) / kNormRowsPerCta;
-  if (select && chunks < 1) chunks = 1;                  // records are written even for max_len 0
+  if (key_mode != kKeysOnly && chunks < 1) chunks = 1;   // records are written even for max_len 0
+  if (key_mode == kKeysGiven) chunks = 1;                // one CTA per unit: selection only
   if (units == 0 || chunks == 0) return L2KV_OK;
   const long long blocks = units * chunks;
   if (blocks > 0x7fffffffLL) return L2KV_ERR_OUT_OF_RANGE;
-  if (select) {
-    key_norms_kernel<T, D, true><<<(unsigned)blocks, kNormThreads, 0, s>>>(
-        static_cast<const T*>(K), g, len_dev, sumsq, ld, norm_out, chunks, max_len, *select);
-  } else {
-    key_norms_kernel<T, D, false><<<(unsigned)blocks, kNormThreads, 0, s>>>(
-        static_cast<const T*>(K), g, len_dev, sumsq, ld, norm_out, chunks, max_len, SelectArgs{});
+  const T* Kt = static_cast<const T*>(K);
+  const SelectArgs sa = select ? *select : SelectArgs{};
+  const unsigned nb = (unsigned)blocks;
+  switch (key_mode) {
+    case kKeysOnly:
+      key_norms_kernel<T, D, kKeysOnly><<<nb, kNormThreads, 0, s>>>(Kt, g, len_dev, sumsq, ld, norm_out, chunks, max_len, sa);
+      break;
+    case kKeysFromK:
+      key_norms_kernel<T, D, kKeysFromK><<<nb, kNormThreads, 0, s>>>(Kt, g, len_dev, sumsq, ld, norm_out, chunks, max_len, sa);
+      break;
+    case kKeysRandom:
+      key_norms_kernel<T, D, kKeysRandom><<<nb, kNormThreads, 0, s>>>(Kt, g, len_dev, sumsq, ld, norm_out, chunks, max_len, sa);
+      break;
+    case kKeysGiven:
+      key_norms_kernel<T, D, kKeysGiven><<<nb, kNormThreads, 0, s>>>(Kt, g, len_dev, sumsq, ld, norm_out, chunks, max_len, sa);
+      break;
+    default:
+      return L2KV_ERR_INVALID_ARG;
   }
   return cudaGetLastError() == cudaSuccess ? L2KV_OK : L2KV_ERR_CUDA;
 }
 
 int launch_key_norms(const void* K, const Geom& g, int dtype, const int32_t* len_dev, int max_len,
-                     float* sumsq, long long ld_sumsq, float* norm_out, const SelectArgs* select,
-                     cudaStream_t s) {
+                     float* sumsq, long long ld_sumsq, float* norm_out, int key_mode,
+                     const SelectArgs* select, cudaStream_t s) {
 #define L2KV_KN(T, D) \
-  return launch_norms_t<T, D>(K, g, len_dev, max_len, sumsq, ld_sumsq, norm_out, select, s)
+  return launch_norms_t<T, D>(K, g, len_dev, max_len, sumsq, ld_sumsq, norm_out, key_mode, select, s)
   if (dtype == L2KV_BF16) {
     if (g.D == 128) L2KV_KN(__nv_bfloat16, 128);
     if (g.D == 64) L2KV_KN(__nv_bfloat16, 64);

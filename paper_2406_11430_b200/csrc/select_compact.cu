@@ -134,29 +134,43 @@ gather_kernel(const T* __restrict__ K, const T* __restrict__ V, Geom gi, T* __re
 template <typename T, int D>
 static int launch_sc_t(const void* K, const void* V, const Geom& gi, const int32_t* len_dev,
                        const int32_t* keep_dev, int max_len, const LayerMask& unc, int policy,
-                       void* K_out, void* V_out, const Geom& go, int32_t* idx_out, float* sumsq_out,
-                       int32_t* kept_len_dev, char* ws, const WorkspacePlan& plan, cudaStream_t s) {
+                       unsigned long long seed, const float* sumsq_in, void* K_out, void* V_out,
+                       const Geom& go, int32_t* idx_out, float* sumsq_out, int32_t* kept_len_dev,
+                       char* ws, const WorkspacePlan& plan, cudaStream_t s) {
   const long long units = (long long)gi.B * gi.L * gi.H;
   if (units == 0) return L2KV_OK;
   if (plan.n_chunks > kMaxChunks) return L2KV_ERR_OUT_OF_RANGE;
   if (units * plan.n_chunks > 0x7fffffffLL) return L2KV_ERR_OUT_OF_RANGE;
-  float* sumsq = reinterpret_cast<float*>(ws + plan.sumsq_off);
   UnitRec* urec = reinterpret_cast<UnitRec*>(ws + plan.unit_off);
   int2* crec = reinterpret_cast<int2*>(ws + plan.chunk_off);
-  // Keys of the layers that are compressed (the others are copied whole), and, as each
-  // unit's last chunk of keys lands, its selection.
+  // Where the ordering keys come from: a pass over K (the default), the caller (keys kept
+  // from the time the rows were written: no pass over K at all), or a seeded hash.
+  int key_mode = kKeysFromK;
+  float* keys = reinterpret_cast<float*>(ws + plan.sumsq_off);
+  long long ld = plan.ld_sumsq;
+  if (policy == L2KV_KEEP_RANDOM) {
+    key_mode = kKeysRandom;
+  } else if (sumsq_in) {
+    key_mode = kKeysGiven;
+    keys = const_cast<float*>(sumsq_in);                 // read-only in this mode
+    ld = gi.t_cap;
+  }
   SelectArgs sel;
-  sel.keep_dev = keep_dev; sel.out_t_cap = go.t_cap; sel.policy = policy;
+  sel.keep_dev = keep_dev; sel.out_t_cap = go.t_cap;
+  sel.policy = policy == L2KV_KEEP_HIGHEST_NORM ? L2KV_KEEP_HIGHEST_NORM : L2KV_KEEP_LOWEST_NORM;
+  sel.seed = seed;
   sel.n_chunks = plan.n_chunks; sel.unc = unc; sel.unit_rec = urec; sel.chunk_rec = crec;
   sel.tickets = reinterpret_cast<int32_t*>(ws + plan.ticket_off);
   sel.kept_len_dev = kept_len_dev;
-  const int rc = launch_key_norms(K, gi, Elem<T>::kDtype, len_dev, max_len, sumsq, plan.ld_sumsq,
-                                  nullptr, &sel, s);
+  // Keys of the layers that are compressed (the others are copied whole), and, as each
+  // unit's last chunk of keys lands, its selection.
+  const int rc = launch_key_norms(K, gi, Elem<T>::kDtype, len_dev, max_len, keys, ld, nullptr,
+                                  key_mode, &sel, s);
   if (rc != L2KV_OK) return rc;
   if (max_len > 0) {
     gather_kernel<T, D><<<(unsigned)(units * plan.n_chunks), kGatherThreads, 0, s>>>(
         static_cast<const T*>(K), static_cast<const T*>(V), gi, static_cast<T*>(K_out),
-        static_cast<T*>(V_out), go, len_dev, max_len, sumsq, plan.ld_sumsq, policy, urec, crec,
+        static_cast<T*>(V_out), go, len_dev, max_len, keys, ld, sel.policy, urec, crec,
         plan.n_chunks, idx_out, sumsq_out);
     if (cudaGetLastError() != cudaSuccess) return L2KV_ERR_CUDA;
   }
@@ -165,12 +179,13 @@ static int launch_sc_t(const void* K, const void* V, const Geom& gi, const int32
 
 int launch_select_compact(const void* K, const void* V, const Geom& gi, int dtype,
                           const int32_t* len_dev, const int32_t* keep_dev, int max_len,
-                          const LayerMask& unc, int policy, void* K_out, void* V_out,
-                          const Geom& go, int32_t* idx_out, float* sumsq_out, int32_t* kept_len_dev,
-                          char* ws, const WorkspacePlan& plan, cudaStream_t s) {
-#define L2KV_SC(T, D)                                                                             \
-  return launch_sc_t<T, D>(K, V, gi, len_dev, keep_dev, max_len, unc, policy, K_out, V_out, go,   \
-                           idx_out, sumsq_out, kept_len_dev, ws, plan, s)
+                          const LayerMask& unc, int policy, unsigned long long seed,
+                          const float* sumsq_in, void* K_out, void* V_out, const Geom& go,
+                          int32_t* idx_out, float* sumsq_out, int32_t* kept_len_dev, char* ws,
+                          const WorkspacePlan& plan, cudaStream_t s) {
+#define L2KV_SC(T, D)                                                                           \
+  return launch_sc_t<T, D>(K, V, gi, len_dev, keep_dev, max_len, unc, policy, seed, sumsq_in,   \
+                           K_out, V_out, go, idx_out, sumsq_out, kept_len_dev, ws, plan, s)
   if (dtype == L2KV_BF16) {
     if (gi.D == 128) L2KV_SC(__nv_bfloat16, 128);
     if (gi.D == 64) L2KV_SC(__nv_bfloat16, 64);

@@ -24,7 +24,8 @@ __device__ __forceinline__ uint32_t load_key_bits(const float* p, int policy) {
 
 template <int NT>
 __device__ void select_unit(SelectSmem& sm, const float* __restrict__ key, int len, int keep,
-                            int policy, UnitRec* __restrict__ rec, int2* __restrict__ crec) {
+                            int policy, uint32_t flags, UnitRec* __restrict__ rec,
+                            int2* __restrict__ crec) {
   constexpr int kBatch = 8;                      // independent key loads in flight per thread
   const int tid = threadIdx.x;
   const int my_chunks = (len + kGatherChunk - 1) / kGatherChunk;
@@ -87,7 +88,7 @@ __device__ void select_unit(SelectSmem& sm, const float* __restrict__ key, int l
   }
   const uint32_t thr = prefix;      // the keep-th smallest key; k_rem of its copies are admitted
   if (tid == 0) {
-    UnitRec r; r.thr = thr; r.admit = k_rem; r.n_keep = keep; r.flags = 0u;
+    UnitRec r; r.thr = thr; r.admit = k_rem; r.n_keep = keep; r.flags = flags;
     *rec = r;
   }
   // Per-chunk counts of keys below / equal to the threshold, one warp per chunk.

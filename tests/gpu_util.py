@@ -12,7 +12,8 @@ def i32(x, device=DEV):
     return torch.tensor(np.asarray(x, dtype=np.int32), dtype=torch.int32, device=device)
 
 
-def gpu_compress(l2, K, V, lens, keep, unc=(), policy=0, t_cap_out=None, max_len=None):
+def gpu_compress(l2, K, V, lens, keep, unc=(), policy=0, t_cap_out=None, max_len=None, seed=0,
+                 sumsq_in=None):
     """K, V: device tensors [B, L, H, T_cap, D].  Returns (device dict, numpy dict)."""
     B, L, H, T_cap, D = K.shape
     t_cap_out = T_cap if t_cap_out is None else t_cap_out
@@ -24,7 +25,7 @@ def gpu_compress(l2, K, V, lens, keep, unc=(), policy=0, t_cap_out=None, max_len
     kept_len = torch.zeros((B, L), dtype=torch.int32, device=K.device)
     ws = l2.new_workspace(l2.Layout(K), max_len, K.device)
     l2.select_compact(K, V, i32(lens), i32(keep), max_len, unc, K_c, V_c, idx, sumsq,
-                      kept_len, ws, policy=policy)
+                      kept_len, ws, policy=policy, seed=seed, sumsq_in=sumsq_in)
     torch.cuda.synchronize()
     dev = dict(K_c=K_c, V_c=V_c, idx=idx, sumsq=sumsq, kept_len=kept_len)
     host = {k: synth.to_numpy(v) for k, v in dev.items()}

@@ -32,10 +32,12 @@ def make(w, t_cap=None):
     return K, V, synth.to_numpy(K), synth.to_numpy(V)
 
 
-def check_compress(l2, w, K, V, Kn, Vn, lens, keep, unc=(), policy=0, t_cap_out=None):
-    _, got = gpu_compress(l2, K, V, lens, keep, unc, policy, t_cap_out)
+def check_compress(l2, w, K, V, Kn, Vn, lens, keep, unc=(), policy=0, t_cap_out=None, seed=0,
+                   sumsq_in=None):
+    _, got = gpu_compress(l2, K, V, lens, keep, unc, policy, t_cap_out, seed=seed,
+                          sumsq_in=sumsq_in)
     exact = oracle.compress(Kn, Vn, w.dtype, lens, keep, unc, key_mode=1, policy=policy,
-                            t_cap_out=t_cap_out, nthreads=8)
+                            t_cap_out=t_cap_out, nthreads=8, seed=seed)
     assert np.array_equal(got["kept_len"], exact["kept_len"])
     assert np.array_equal(got["idx"], exact["idx"])
     assert np.array_equal(got["K_c"], exact["K_c"])
@@ -155,6 +157,29 @@ def test_compress_is_deterministic(l2):
     b = gpu_compress(l2, K, V, [4096], [2048])[1]
     for name in a:
         assert np.array_equal(a[name], b[name], equal_nan=True)
+
+
+def test_compress_random_policy(l2):
+    w = synth.WORKLOADS[1].scaled(B=2, L=3, Hkv=2, Hq=2, T=2500)
+    K, V, Kn, Vn = make(w, t_cap=2560)
+    a, _ = check_compress(l2, w, K, V, Kn, Vn, [2500, 700], [1000, 699], unc=(1,), policy=2,
+                          seed=12345, t_cap_out=2500)
+    b, _ = check_compress(l2, w, K, V, Kn, Vn, [2500, 700], [1000, 699], unc=(1,), policy=2,
+                          seed=(1 << 63) + 99, t_cap_out=2500)
+    assert not np.array_equal(a["idx"], b["idx"])
+
+
+@pytest.mark.parametrize("policy", [0, 1])
+def test_compress_with_keys_from_write_time(l2, policy):
+    # Keys computed once (as when rows are written to the cache) and handed back in: same
+    # result as letting the call compute them, without its pass over K.
+    w = synth.WORKLOADS[1].scaled(B=2, L=3, Hkv=2, Hq=2, T=2500)
+    K, V, Kn, Vn = make(w, t_cap=2560)
+    lens = [2500, 1200]
+    keys = torch.full(K.shape[:4], float("nan"), dtype=torch.float32, device=DEV)
+    l2.key_norms(K, i32(lens), 2500, keys)
+    check_compress(l2, w, K, V, Kn, Vn, lens, [1250, 7], unc=(1,), policy=policy, t_cap_out=2500,
+                   sumsq_in=keys)
 
 
 # ---------------------------------------------------------- decode attention

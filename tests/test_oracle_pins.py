@@ -372,3 +372,43 @@ def test_append_evict_cases():
     assert st["cur_len"][0, 0] == 4 and st["idx"][0, 0, 0, 3] == 6
     assert oracle.append_evict(st, "f32", [3], (0,), row(1.0), row(17), [7]) == -2  # no room
     assert st["cur_len"][0, 0] == 4
+
+
+# ------------------------------------------------- keep-random ablation policy
+
+def test_random_key_is_splitmix64():
+    g = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "splitmix64.json")))
+    gamma, mask = 0x9E3779B97F4A7C15, (1 << 64) - 1
+    for k, out in enumerate(g["outputs"]):
+        # the k-th output of the sequential generator is the output function at seed + k * gamma
+        assert oracle.random_key((g["seed"] + k * gamma) & mask, 0, 0) == int(out) >> 32
+    # the counter is seed + (unit * 2^32 + t)
+    assert oracle.random_key(5, 3, 9) == oracle.random_key(5 + (3 << 32) + 9, 0, 0)
+    assert oracle.random_key(5, 3, 9) != oracle.random_key(5, 3, 10)
+
+
+def test_random_policy_keeps_the_lowest_random_keys():
+    w, K, V = _tiny("f32", L=2, T=200)
+    keep = 50
+    r = oracle.compress(K, V, "f32", [w.T], [keep], uncompressed=(0,), policy=2, seed=77)
+    s = oracle.key_sumsq(K, "f32")
+    assert r["kept_len"].tolist() == [[w.T, keep]]
+    counts = np.zeros(w.T)
+    for h in range(w.Hkv):
+        u = (0 * w.L + 1) * w.Hkv + h
+        want = sorted(sorted(range(w.T), key=lambda t: (oracle.random_key(77, u, t), t))[:keep])
+        idx = r["idx"][0, 1, h, :keep]
+        assert idx.tolist() == want
+        assert np.array_equal(r["K_c"][0, 1, h, :keep], K[0, 1, h, idx])
+        assert np.array_equal(r["key"][0, 1, h, :keep], s[0, 1, h, idx])    # stored keys stay norms
+        counts[idx] += 1
+    again = oracle.compress(K, V, "f32", [w.T], [keep], uncompressed=(0,), policy=2, seed=77)
+    other = oracle.compress(K, V, "f32", [w.T], [keep], uncompressed=(0,), policy=2, seed=78)
+    assert np.array_equal(again["idx"], r["idx"]) and not np.array_equal(other["idx"], r["idx"])
+    assert counts.max() <= w.Hkv and 0 < (counts > 0).mean() < 1             # heads differ
+    # over many seeds every position is kept about keep / T of the time
+    freq = np.zeros(w.T)
+    for seed in range(200):
+        freq[oracle.compress(K, V, "f32", [w.T], [keep], uncompressed=(0,), policy=2,
+                             seed=seed)["idx"][0, 1, 0, :keep]] += 1
+    assert abs(freq.mean() / 200 - keep / w.T) < 1e-12 and freq.min() > 20 and freq.max() < 85
