@@ -11,6 +11,11 @@
 //   decode_combine_kernel  merges the partials of all splits of a query head.
 //
 // All arithmetic is fp32 on values widened exactly from the stored bf16 / fp32.
+#include <cuda.h>      // CUtensorMap and its enums only; the encoder is fetched from the driver at run time
+
+#include <cstdlib>
+#include <cstring>
+
 #include "common.cuh"
 
 namespace l2kv {
@@ -273,18 +278,67 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], 
                : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
-template <int G>
+// ---- mbarrier / TMA (cp.async.bulk.tensor) helpers -------------------------------------
+__device__ __forceinline__ void mbar_init(uint32_t bar, int count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"(bytes)
+               : "memory");
+}
+// Waits for the phase with the given parity; gives up after a bounded number of polls (a
+// copy that never lands must not hang the GPU) and reports that through the return value.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  for (int spin = 0; spin < (1 << 20); ++spin) {
+    uint32_t done;
+    asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; "
+                 "selp.u32 %0, 1, 0, p; }" : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    if (done) return true;
+  }
+  return false;
+}
+// One box of a rank-5 tensor map (dims: head_dim, token, kv head, layer, batch) into shared memory.
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map, uint32_t bar,
+                                            int c0, int c1, int c2, int c3, int c4) {
+  asm volatile("cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
+               "[%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+               :: "r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+               : "memory");
+}
+
+// Shared-memory address of the 16-byte piece `ch` of row `row` of a stage.  cp.async path:
+// rows of 256 bytes, piece index XORed with row & 7.  TMA path: the two halves of the head
+// dimension are separate [kStageTok][128 B] tiles, and the tensor map's 128-byte swizzle XORs
+// address bits 4..6 with address bits 7..9 (the 128-byte line number; sb is 128-byte aligned
+// and the tiles are whole multiples of 1024 bytes apart).
+template <bool TMA>
+__device__ __forceinline__ uint32_t tile_addr(uint32_t sb, int row, int ch) {
+  if constexpr (TMA) {
+    const int line = (int)(sb >> 7) + row;
+    return sb + (ch >> 3) * (kStageTok * 128) + row * 128 + (((ch & 7) ^ (line & 7)) << 4);
+  } else {
+    return sb + row * kRowBytes + ((ch ^ (row & 7)) << 4);
+  }
+}
+
+template <int G, bool TMA>
 __global__ void __launch_bounds__(kMmaThreads, L2KV_MMA_MIN_CTAS)
 decode_split_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ K,
                         const __nv_bfloat16* __restrict__ V, Geom g,
                         const int32_t* __restrict__ cur_len_dev, int max_len, float scale_log2e,
-                        float* __restrict__ partial, int n_splits) {
+                        float* __restrict__ partial, int n_splits,
+                        const __grid_constant__ CUtensorMap map_k,
+                        const __grid_constant__ CUtensorMap map_v, int32_t* __restrict__ status_word) {
   constexpr int D = 128;
   constexpr int NW = kMmaWarps;
   constexpr int TPT = kDecodeChunk / kMmaThreads;        // tokens per thread in phase 2
-  extern __shared__ __align__(128) unsigned char smem[];
-  unsigned char* s_stage = smem;                                        // [kStages][128][256 B]
-  float* s_sc = reinterpret_cast<float*>(smem + kStages * kStageTok * kRowBytes);  // [G][kScLd]
+  constexpr int kStageBytes = kStageTok * kRowBytes;
+  extern __shared__ unsigned char smem_raw[];
+  // Stages start on a 128-byte boundary (required of a tensor-copy destination).
+  unsigned char* smem = smem_raw + ((128u - (smem_u32(smem_raw) & 127u)) & 127u);
+  unsigned char* s_stage = smem;                         // [kStages][kStageTok rows of 256 B]
+  float* s_sc = reinterpret_cast<float*>(smem + kStages * kStageBytes);           // [G][kScLd]
+  __shared__ __align__(8) unsigned long long s_bar[kStages];
   __shared__ float s_red[NW][G];
   __shared__ float s_m[G], s_l[G];
 
@@ -297,6 +351,11 @@ decode_split_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16
   const int n = max(0, min(cur_len_dev[bl], min(max_len, g.t_cap)));
   const int t0 = split * kDecodeChunk;
   if (t0 >= n) return;
+  if constexpr (TMA) {
+    // A copy that timed out in an earlier CTA marks the workspace; the rest of the grid
+    // then leaves at once instead of timing out CTA by CTA.
+    if (status_word && *reinterpret_cast<volatile int32_t*>(status_word + 2) != 0) return;
+  }
   const int nt = min(n, t0 + kDecodeChunk) - t0;
   const int n_st = (nt + kStageTok - 1) / kStageTok;     // stages of K, and again of V
   const int total = 2 * n_st;
@@ -320,26 +379,47 @@ decode_split_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16
   const char* c_v = reinterpret_cast<const char*>(Vb) + c_row * row_bytes + c_ch * 16;
   auto issue = [&](int s) {
     const int st = s < n_st ? s : s - n_st;
-    const char* src = (s < n_st ? c_k : c_v) + (long long)st * kStageTok * row_bytes;
-    const uint32_t dst = c_dst + (s % kStages) * (kStageTok * kRowBytes);
-    const int rows = nt - st * kStageTok;                  // valid rows of this stage (>= 1)
-    if (rows >= kStageTok) {
-#pragma unroll
-      for (int i = 0; i < kCopies; ++i)
-        cp_async16(dst + i * kRowStep * kRowBytes, src + i * kRowStep * row_bytes, 16);
+    if constexpr (TMA) {
+      // One thread hands the whole stage to the copy engine: two boxes of kStageTok rows x
+      // 64 elements.  Rows past the tensor's t_cap arrive as zeros; rows between the valid
+      // length and t_cap arrive as stored and are masked where they could matter.
+      if (tid == 0) {
+        const uint32_t bar = smem_u32(&s_bar[s % kStages]);
+        const uint32_t dst = stage0 + (s % kStages) * kStageBytes;
+        const CUtensorMap* map = s < n_st ? &map_k : &map_v;
+        mbar_expect_tx(bar, kStageBytes);
+        tma_load_5d(dst, map, bar, 0, t0 + st * kStageTok, h, l, b);
+        tma_load_5d(dst + kStageTok * 128, map, bar, 64, t0 + st * kStageTok, h, l, b);
+      }
     } else {
+      const char* src = (s < n_st ? c_k : c_v) + (long long)st * kStageTok * row_bytes;
+      const uint32_t dst = c_dst + (s % kStages) * kStageBytes;
+      const int rows = nt - st * kStageTok;                // valid rows of this stage (>= 1)
+      if (rows >= kStageTok) {
 #pragma unroll
-      for (int i = 0; i < kCopies; ++i) {
-        const bool ok = c_row + i * kRowStep < rows;       // rows past the end are zero-filled
-        cp_async16(dst + i * kRowStep * kRowBytes, ok ? src + i * kRowStep * row_bytes : src - c_row * row_bytes,
-                   ok ? 16 : 0);
+        for (int i = 0; i < kCopies; ++i)
+          cp_async16(dst + i * kRowStep * kRowBytes, src + i * kRowStep * row_bytes, 16);
+      } else {
+#pragma unroll
+        for (int i = 0; i < kCopies; ++i) {
+          const bool ok = c_row + i * kRowStep < rows;     // rows past the end are zero-filled
+          cp_async16(dst + i * kRowStep * kRowBytes,
+                     ok ? src + i * kRowStep * row_bytes : src - c_row * row_bytes, ok ? 16 : 0);
+        }
       }
     }
   };
 
+  if constexpr (TMA) {
+    if (tid == 0) {
+      for (int i = 0; i < kStages; ++i) mbar_init(smem_u32(&s_bar[i]), 1);
+      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+  }
   for (int s = 0; s < kStages - 1; ++s) {
     if (s < total) issue(s);
-    cp_async_commit();
+    if constexpr (!TMA) cp_async_commit();
   }
 
   // Q^T fragments: lane (fr, fc) holds head fr's dims 16j + 2fc (+1) and 16j + 2fc + 8 (+9).
@@ -358,12 +438,17 @@ decode_split_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16
   float oacc[kDbw][4];                                     // O^T[16 (kDbw warp + db) + fr (+8)][2 fc (+1)]
 #pragma unroll
   for (int db = 0; db < kDbw; ++db) { oacc[db][0] = oacc[db][1] = oacc[db][2] = oacc[db][3] = 0.f; }
+  bool copy_ok = true;
   for (int s = 0; s < total; ++s) {
-    cp_async_wait<kStages - 2>();
+    if constexpr (TMA) {
+      copy_ok = mbar_wait(smem_u32(&s_bar[s % kStages]), (s / kStages) & 1) && copy_ok;
+    } else {
+      cp_async_wait<kStages - 2>();
+    }
     __syncthreads();                                       // stage s landed; stage s-1 is free
     if (s + kStages - 1 < total) issue(s + kStages - 1);
-    cp_async_commit();
-    const uint32_t sb = stage0 + (s % kStages) * (kStageTok * kRowBytes);
+    if constexpr (!TMA) cp_async_commit();
+    const uint32_t sb = stage0 + (s % kStages) * kStageBytes;
 
     if (s < n_st) {
       // ---- phase 1: scores of tokens [16 warp, 16 warp + 16) of this stage ------------
@@ -374,8 +459,7 @@ decode_split_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
           uint32_t a[4];
-          const int ch = 2 * j + (lane >> 4);
-          ldmatrix_x4(a, sb + row * kRowBytes + ((ch ^ (row & 7)) << 4));
+          ldmatrix_x4(a, tile_addr<TMA>(sb, row, 2 * j + (lane >> 4)));
           mma_bf16(c, a, qb[j][0], qb[j][1]);
         }
         if (2 * fc < G) {
@@ -453,12 +537,15 @@ decode_split_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16
       const uint32_t* pw = reinterpret_cast<const uint32_t*>(s_sc + fr * kScLd) +
                            st * (kStageTok / 2) + fc;
       const int vrow = (lane & 7) + (lane >> 4) * 8;
+      constexpr int kPitch = TMA ? 128 : kRowBytes;        // bytes between rows of a tile
       uint32_t voff[kDbw];
 #pragma unroll
-      for (int db = 0; db < kDbw; ++db) {
-        const int ch = 2 * (warp * kDbw + db) + ((lane >> 3) & 1);
-        voff[db] = sb + vrow * kRowBytes + ((ch ^ (lane & 7)) << 4);
-      }
+      for (int db = 0; db < kDbw; ++db)
+        voff[db] = tile_addr<TMA>(sb, vrow, 2 * (warp * kDbw + db) + ((lane >> 3) & 1));
+      // TMA path only: tokens of the last, partial 16-token step that lie past the valid
+      // length hold whatever the cache holds there; their V^T entries are cleared in
+      // registers so that 0 * (Inf or NaN) cannot reach the accumulators.
+      const int valid = nt - st * kStageTok;               // valid tokens of this stage
       auto kstep = [&](int ks) {
         uint32_t h0 = 0u, h1 = 0u, l0 = 0u, l1 = 0u;
         if (fr < G) {
@@ -468,7 +555,15 @@ decode_split_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16
 #pragma unroll
         for (int db = 0; db < kDbw; ++db) {
           uint32_t a[4];
-          ldmatrix_x4_trans(a, voff[db] + ks * 16 * kRowBytes);
+          ldmatrix_x4_trans(a, voff[db] + ks * 16 * kPitch);
+          if constexpr (TMA) {
+            if (ks * 16 + 16 > valid) {
+              const int t = ks * 16 + 2 * fc;              // a[0], a[1]: tokens t, t+1; a[2], a[3]: +8
+              const uint32_t m0 = (t < valid ? 0x0000ffffu : 0u) | (t + 1 < valid ? 0xffff0000u : 0u);
+              const uint32_t m1 = (t + 8 < valid ? 0x0000ffffu : 0u) | (t + 9 < valid ? 0xffff0000u : 0u);
+              a[0] &= m0; a[1] &= m0; a[2] &= m1; a[3] &= m1;
+            }
+          }
           mma_bf16(oacc[db], a, h0, h1);
           mma_bf16(oacc[db], a, l0, l1);
         }
@@ -481,7 +576,14 @@ decode_split_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16
       }
     }
   }
-  cp_async_wait<0>();
+  if constexpr (TMA) {
+    if (!copy_ok && tid == 0 && status_word) {
+      atomicExch(status_word, (int)L2KV_ERR_CUDA);
+      atomicExch(status_word + 2, 1);                      // abort mark read by later CTAs
+    }
+  } else {
+    cp_async_wait<0>();
+  }
 
   // O^T fragments: rows = dims 16 (kDbw warp + db) + fr (+8), columns = heads 2 fc (+1).
 #pragma unroll
@@ -503,6 +605,35 @@ decode_split_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16
   }
 }
 
+// Builds the rank-5 tensor map (head_dim, token, kv head, layer, batch) of a bf16 cache with a
+// box of 64 elements x kStageTok tokens and the 128-byte swizzle.  Returns false when the
+// encoder is unavailable or rejects the geometry (the caller then uses the cp.async path).
+static bool make_cache_map(CUtensorMap* map, const void* base, const Geom& g) {
+  using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+  static EncodeFn encode = []() -> EncodeFn {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult res;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &res) !=
+            cudaSuccess || res != cudaDriverEntryPointSuccess)
+      return nullptr;
+    return reinterpret_cast<EncodeFn>(fn);
+  }();
+  if (!encode) return false;
+  if (g.st <= 0 || g.sh <= 0 || g.sl <= 0 || g.sb <= 0) return false;   // broadcast views
+  const cuuint64_t dims[5] = {128, (cuuint64_t)g.t_cap, (cuuint64_t)g.H, (cuuint64_t)g.L,
+                              (cuuint64_t)g.B};
+  const cuuint64_t strides[4] = {(cuuint64_t)g.st * 2, (cuuint64_t)g.sh * 2, (cuuint64_t)g.sl * 2,
+                                 (cuuint64_t)g.sb * 2};
+  const cuuint32_t box[5] = {64, (cuuint32_t)kStageTok, 1, 1, 1};
+  const cuuint32_t elem[5] = {1, 1, 1, 1, 1};
+  return encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(base), dims, strides,
+                box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <int G>
 static int launch_dec_mma(const void* q, const void* K, const void* V, const Geom& g,
                           const int32_t* cur_len_dev, int max_len, float scale, float* out,
@@ -511,16 +642,25 @@ static int launch_dec_mma(const void* q, const void* K, const void* V, const Geo
   if (units == 0) return L2KV_OK;
   if (units * plan.n_splits > 0x7fffffffLL) return L2KV_ERR_OUT_OF_RANGE;
   float* partial = reinterpret_cast<float*>(ws + plan.partial_off);
-  constexpr int smem_bytes = kStages * kStageTok * kRowBytes + G * kScLd * 4;
+  constexpr int smem_bytes = 128 + kStages * kStageTok * kRowBytes + G * kScLd * 4;
   if (max_len > 0) {
-    auto kern = decode_split_mma_kernel<G>;
+    // K and V rows reach shared memory through TMA tensor maps; L2KV_DECODE_COPY=cpasync (or a
+    // geometry the encoder rejects) selects the per-thread cp.async copies instead.
+    alignas(64) CUtensorMap map_k, map_v;
+    std::memset(&map_k, 0, sizeof map_k);
+    std::memset(&map_v, 0, sizeof map_v);
+    const char* mode = std::getenv("L2KV_DECODE_COPY");
+    const bool want_tma = !(mode && std::strcmp(mode, "cpasync") == 0);
+    const bool tma = want_tma && make_cache_map(&map_k, K, g) && make_cache_map(&map_v, V, g);
+    auto kern = tma ? decode_split_mma_kernel<G, true> : decode_split_mma_kernel<G, false>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) !=
         cudaSuccess)
       return L2KV_ERR_CUDA;
     kern<<<(unsigned)(units * plan.n_splits), kMmaThreads, smem_bytes, s>>>(
         static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(K),
         static_cast<const __nv_bfloat16*>(V), g, cur_len_dev, max_len, scale * kLog2e, partial,
-        plan.n_splits);
+        plan.n_splits, map_k, map_v,
+        plan.partial_off >= (size_t)kStatusBytes ? reinterpret_cast<int32_t*>(ws) : nullptr);
     if (cudaGetLastError() != cudaSuccess) return L2KV_ERR_CUDA;
   }
   decode_combine_kernel<128><<<(unsigned)((long long)g.B * g.L * g.Hq), 128, 0, s>>>(

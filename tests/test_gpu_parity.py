@@ -200,6 +200,29 @@ def test_attention_ragged(l2, dtype, D, Hkv, Hq):
     assert np.sqrt(np.mean((got - want) ** 2)) <= 2e-4 * max(rms, 1e-3) + 1e-6
 
 
+def test_attention_copy_paths_agree(l2, monkeypatch):
+    # bf16 / head_dim 128 streams K and V through TMA tensor maps by default and through
+    # per-thread cp.async copies on request (or when a geometry cannot be encoded); the
+    # arithmetic is the same, so the outputs must be bit-identical.
+    w = synth.WORKLOADS[2].scaled(B=2, L=2, T=2300)
+    K, V, Kn, Vn = make(w)
+    q = synth.make_query(w, 0, DEV)
+    cur = np.array([[2300, 1030], [129, 2047]], dtype=np.int32)
+    monkeypatch.setenv("L2KV_DECODE_COPY", "tma")
+    a = gpu_attention(l2, q, K, V, cur)
+    monkeypatch.setenv("L2KV_DECODE_COPY", "cpasync")
+    b = gpu_attention(l2, q, K, V, cur)
+    assert np.array_equal(a, b)
+    assert_attention_close(a, oracle.attention(synth.to_numpy(q), Kn, Vn, "bf16", cur, nthreads=8))
+    # rows past the valid length must not leak in, whatever they hold (here: NaN and Inf)
+    Kp, Vp = K.clone(), V.clone()
+    Kp[0, 1, :, 1030:] = float("nan"); Vp[0, 1, :, 1030:] = float("inf")
+    Kp[1, 0, :, 129:] = float("inf"); Vp[1, 0, :, 129:] = float("nan")
+    for mode in ("tma", "cpasync"):
+        monkeypatch.setenv("L2KV_DECODE_COPY", mode)
+        assert np.array_equal(gpu_attention(l2, q, Kp, Vp, cur), a)
+
+
 def test_attention_special_cases(l2):
     w = synth.WORKLOADS[2].scaled(B=1, L=1, T=2048)
     K, V, Kn, Vn = make(w)
