@@ -291,7 +291,38 @@ def time_variants(job, w, cbytes, reps=5):
         out[name] = {"ms": round(ms, 3), "bytes": nbytes, "GBps": round(nbytes / ms / 1e6, 1)}
     job.compress()                     # leave the cache as the method's own policy makes it
     torch.cuda.synchronize()
+    out["append_evict"] = time_append_evict(job, w)
+    job.compress()
+    torch.cuda.synchronize()
     return out
+
+
+def time_append_evict(job, w, reps=20):
+    """One budget-maintenance step (a new K/V row per head, eviction of the highest norm) on
+    the compressed cache of this workload, every sequence at its budget.  Not part of the
+    workload's step (its cache is static); timed here so that the kernel has a number."""
+    budget = torch.full((w.B,), job.keep_n, dtype=torch.int32, device=job.dev)
+    pos = torch.full((w.B,), w.T, dtype=torch.int32, device=job.dev)
+    rows = [synth.make_new_kv(w, s, job.dev) for s in range(4)]
+    cur = job.cur.cpu()
+    stored = int(cur.sum().item()) * w.Hkv                 # (key, position) pairs scanned
+    nbytes = stored * 8 + w.B * w.L * w.Hkv * (4 * w.D * w.elem_bytes + 8)
+
+    def one(i):
+        k, v = rows[i % len(rows)]
+        # no layer list: the full-length layers 0-1 are over budget too and evict like the rest
+        job.l2.append_evict(job.K_c, job.V_c, job.idx, job.sumsq, job.cur, budget, (), k, v,
+                            pos + i, job.ws)
+    for i in range(3):
+        one(i)
+    t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for i in range(reps):
+        one(3 + i)
+    t1.record(); torch.cuda.synchronize()
+    ms = t0.elapsed_time(t1) / reps
+    return {"ms": round(ms, 4), "bytes": nbytes, "GBps": round(nbytes / ms / 1e6, 1),
+            "stored_entries": stored}
 
 
 def run_e2e(job, w, step_bytes, world, device, args):

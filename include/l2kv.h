@@ -155,7 +155,9 @@ int l2kv_decode_attention(const void* q, const void* K_c, const void* V_c, const
  * [batch, layers, kv_heads, head_dim]; pos_new_dev[b] is the new token's position.
  * K_c, V_c, idx, sumsq_c and cur_len_dev are updated in place (idx and sumsq_c dense
  * [batch, layers, kv_heads, lay->t_cap]).  A row that would land at slot >= t_cap is
- * not written and sets the device status word to L2KV_ERR_DEVICE_OVERFLOW. */
+ * not written and sets the device status word to L2KV_ERR_DEVICE_OVERFLOW.  The
+ * workspace may be the one of the other calls or a small one of its own: any zeroed
+ * buffer of at least l2kv_workspace_bytes(lay, 0) bytes. */
 int l2kv_append_evict(void* K_c, void* V_c, int32_t* idx, float* sumsq_c, const l2kv_layout* lay,
                       int32_t* cur_len_dev, const int32_t* budget_dev,
                       const int32_t* uncompressed_layers, int32_t n_uncompressed,

@@ -184,10 +184,14 @@ int l2kv_append_evict(void* K_c, void* V_c, int32_t* idx, float* sumsq_c, const 
   if (!aligned16(K_c) || !aligned16(V_c) || !aligned16(k_new) || !aligned16(v_new) ||
       !aligned16(workspace))
     return L2KV_ERR_MISALIGNED;
-  if (workspace_bytes < (size_t)kStatusBytes) return L2KV_ERR_WORKSPACE_TOO_SMALL;
+  const WorkspacePlan plan = plan_workspace(*lay, 0);    // status word and tickets only
+  if (workspace_bytes < plan.sumsq_off) return L2KV_ERR_WORKSPACE_TOO_SMALL;
+  char* ws = static_cast<char*>(workspace);
   return launch_append_evict(K_c, V_c, idx, sumsq_c, make_geom(*lay), lay->dtype, cur_len_dev,
                              budget_dev, unc, k_new, v_new, pos_new_dev,
-                             static_cast<int32_t*>(workspace), static_cast<cudaStream_t>(stream));
+                             reinterpret_cast<int32_t*>(ws),
+                             reinterpret_cast<int32_t*>(ws + plan.ticket_off),
+                             static_cast<cudaStream_t>(stream));
 }
 
 }  // extern "C"

@@ -1,15 +1,18 @@
 // Budget-maintained cache: append one token per (b, l, h); once a sequence holds `budget`
 // tokens, discard the entry that comes last in the order (key, position).
 //
-// One CTA per (b, l) walks that layer's KV heads, so the shared length cur_len[b, l] is
-// read before and written after all of them by the same CTA.  Per head: the new key's
-// ordering key (same fixed summation order as the norm pass), a block-wide arg-max over
-// the stored keys packed as (key bits << 32 | position), then two 16-byte-piece row copies.
+// One CTA per (b, l, h).  Per unit: the new key's ordering key (same fixed summation order
+// as the norm pass), a block-wide arg-max over the stored keys packed as
+// (key bits << 32 | position), then two 16-byte-piece row copies.  The length cur_len[b, l]
+// is shared by the KV heads of a layer: every CTA reads it first and takes a ticket of its
+// (b, l) when done; the CTA that takes the last ticket -- by then all heads have read the
+// old value -- stores the new length and resets the ticket.  Nobody waits.
 #include "common.cuh"
 
 namespace l2kv {
 
 constexpr int kAppendThreads = 256;
+constexpr int kAppendUnroll = 4;
 
 template <typename T, int D>
 __global__ void __launch_bounds__(kAppendThreads)
@@ -17,27 +20,26 @@ append_evict_kernel(T* __restrict__ K, T* __restrict__ V, int32_t* __restrict__ 
                     float* __restrict__ sumsq, Geom g, int32_t* __restrict__ cur_len_dev,
                     const int32_t* __restrict__ budget_dev, LayerMask unc,
                     const T* __restrict__ k_new, const T* __restrict__ v_new,
-                    const int32_t* __restrict__ pos_new_dev, int32_t* __restrict__ status_word) {
+                    const int32_t* __restrict__ pos_new_dev, int32_t* __restrict__ status_word,
+                    int32_t* __restrict__ tickets) {
   constexpr int EPV = Elem<T>::kPerVec;
   constexpr int LPR = D / EPV;
   constexpr int NW = kAppendThreads / 32;
   __shared__ unsigned long long s_best[NW];
   __shared__ int s_slot;
 
-  const long long bl = blockIdx.x;
+  const long long unit = blockIdx.x;                     // (b * L + l) * H + h
+  const int h = (int)(unit % g.H);
+  const long long bl = unit / g.H;
   const int l = (int)(bl % g.L);
   const int b = (int)(bl / g.L);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int n = max(0, min(cur_len_dev[bl], g.t_cap));
   const bool grow = unc.test(l) || n < budget_dev[b];
-  if (grow && n >= g.t_cap) {
-    if (tid == 0) atomicExch(status_word, (int)L2KV_ERR_DEVICE_OVERFLOW);
-    return;
-  }
+  const bool overflow = grow && n >= g.t_cap;
   const int pos_new = pos_new_dev[b];
 
-  for (int h = 0; h < g.H; ++h) {
-    const long long unit = bl * g.H + h;
+  if (!overflow) {
     // Warp 0 holds the new rows: lanes < LPR own one 16-byte piece each.
     uint4 vk = make_uint4(0, 0, 0, 0), vv = make_uint4(0, 0, 0, 0);
     float s_new = 0.f;
@@ -55,10 +57,20 @@ append_evict_kernel(T* __restrict__ K, T* __restrict__ V, int32_t* __restrict__ 
       const int32_t* pos = idx + unit * g.t_cap;
       unsigned long long best = 0ull;
       int best_j = -1;
-      for (int j = tid; j < n; j += kAppendThreads) {
-        const unsigned long long c =
-            ((unsigned long long)__float_as_uint(key[j]) << 32) | (uint32_t)pos[j];
-        if (best_j < 0 || c > best) { best = c; best_j = j; }
+      for (int j0 = 0; j0 < n; j0 += kAppendThreads * kAppendUnroll) {
+        uint32_t kb[kAppendUnroll], pb[kAppendUnroll];
+#pragma unroll
+        for (int u = 0; u < kAppendUnroll; ++u) {
+          const int j = j0 + u * kAppendThreads + tid;
+          kb[u] = j < n ? __float_as_uint(key[j]) : 0u;
+          pb[u] = j < n ? (uint32_t)pos[j] : 0u;
+        }
+#pragma unroll
+        for (int u = 0; u < kAppendUnroll; ++u) {
+          const int j = j0 + u * kAppendThreads + tid;
+          const unsigned long long c = ((unsigned long long)kb[u] << 32) | pb[u];
+          if (j < n && (best_j < 0 || c > best)) { best = c; best_j = j; }
+        }
       }
       unsigned long long wbest = best;
 #pragma unroll
@@ -81,7 +93,6 @@ append_evict_kernel(T* __restrict__ K, T* __restrict__ V, int32_t* __restrict__ 
             ((unsigned long long)__float_as_uint(s_new) << 32) | (uint32_t)pos_new;
         if (slot < 0 || c_new > top) slot = -1;          // the newcomer is the one discarded
       }
-      __syncthreads();                                   // s_best / s_slot are reused next head
     }
     if (warp == 0 && slot >= 0 && lane < LPR) {
       const long long row = b * g.sb + l * g.sl + h * g.sh + (long long)slot * g.st + lane * EPV;
@@ -93,30 +104,41 @@ append_evict_kernel(T* __restrict__ K, T* __restrict__ V, int32_t* __restrict__ 
       }
     }
   }
-  if (grow && tid == 0) cur_len_dev[bl] = n + 1;
+
+  // Ticket of (b, l): the last of the layer's heads to finish publishes the new length.
+  __syncthreads();
+  if (tid == 0) {
+    __threadfence();
+    if (atomicAdd(tickets + bl, 1) == g.H - 1) {
+      if (overflow) atomicExch(status_word, (int)L2KV_ERR_DEVICE_OVERFLOW);
+      else if (grow) cur_len_dev[bl] = n + 1;
+      tickets[bl] = 0;
+    }
+  }
 }
 
 template <typename T, int D>
 static int launch_ae_t(void* K, void* V, int32_t* idx, float* sumsq, const Geom& g,
                        int32_t* cur_len_dev, const int32_t* budget_dev, const LayerMask& unc,
                        const void* k_new, const void* v_new, const int32_t* pos_new_dev,
-                       int32_t* status_word, cudaStream_t s) {
-  const long long blocks = (long long)g.B * g.L;
-  if (blocks == 0 || g.H == 0) return L2KV_OK;
+                       int32_t* status_word, int32_t* tickets, cudaStream_t s) {
+  const long long blocks = (long long)g.B * g.L * g.H;
+  if (blocks == 0) return L2KV_OK;
   if (blocks > 0x7fffffffLL) return L2KV_ERR_OUT_OF_RANGE;
   append_evict_kernel<T, D><<<(unsigned)blocks, kAppendThreads, 0, s>>>(
       static_cast<T*>(K), static_cast<T*>(V), idx, sumsq, g, cur_len_dev, budget_dev, unc,
-      static_cast<const T*>(k_new), static_cast<const T*>(v_new), pos_new_dev, status_word);
+      static_cast<const T*>(k_new), static_cast<const T*>(v_new), pos_new_dev, status_word,
+      tickets);
   return cudaGetLastError() == cudaSuccess ? L2KV_OK : L2KV_ERR_CUDA;
 }
 
 int launch_append_evict(void* K, void* V, int32_t* idx, float* sumsq, const Geom& g, int dtype,
                         int32_t* cur_len_dev, const int32_t* budget_dev, const LayerMask& unc,
                         const void* k_new, const void* v_new, const int32_t* pos_new_dev,
-                        int32_t* status_word, cudaStream_t s) {
+                        int32_t* status_word, int32_t* tickets, cudaStream_t s) {
 #define L2KV_AE(T, D)                                                                            \
   return launch_ae_t<T, D>(K, V, idx, sumsq, g, cur_len_dev, budget_dev, unc, k_new, v_new,      \
-                           pos_new_dev, status_word, s)
+                           pos_new_dev, status_word, tickets, s)
   if (dtype == L2KV_BF16) {
     if (g.D == 128) L2KV_AE(__nv_bfloat16, 128);
     if (g.D == 64) L2KV_AE(__nv_bfloat16, 64);

@@ -69,10 +69,12 @@ inline WorkspacePlan plan_workspace(const l2kv_layout& a, int max_len) {
   p.n_splits = (int)((max_len + kDecodeChunk - 1) / kDecodeChunk);
   if (p.n_splits < 1) p.n_splits = 1;
   size_t off = kStatusBytes;
+  // Tickets come first so that their place does not depend on max_len (append/evict, which
+  // has no max_len, uses one ticket per (b, l); the norm pass one per unit).
+  p.ticket_off = off;  off += (size_t)round_up_ll(units * 4, 256);
   p.sumsq_off = off;   off += (size_t)round_up_ll(units * p.ld_sumsq * 4, 256);
   p.unit_off = off;    off += (size_t)round_up_ll(units * 16, 256);
   p.chunk_off = off;   off += (size_t)round_up_ll(units * p.n_chunks * 8, 256);
-  p.ticket_off = off;  off += (size_t)round_up_ll(units * 4, 256);
   p.partial_off = off;
   off += (size_t)round_up_ll((long long)a.batch * a.layers * a.q_heads * p.n_splits *
                                  (a.head_dim + 2) * 4, 256);
@@ -208,6 +210,6 @@ int launch_decode_attention(const void* q, const void* K, const void* V, const G
 int launch_append_evict(void* K, void* V, int32_t* idx, float* sumsq, const Geom& g, int dtype,
                         int32_t* cur_len_dev, const int32_t* budget_dev, const LayerMask& unc,
                         const void* k_new, const void* v_new, const int32_t* pos_new_dev,
-                        int32_t* status_word, cudaStream_t s);
+                        int32_t* status_word, int32_t* tickets, cudaStream_t s);
 
 }  // namespace l2kv
