@@ -139,3 +139,23 @@ def append_evict(state, dtype, budget, uncompressed, k_new, v_new, pos_new, key_
         _p(K_c), _p(V_c), _p(state["idx"]), _p(state["key"]), _DT[dtype], B, L, H, T_cap, D,
         _p(state["cur_len"]), _p(budget), _p(unc), int(unc.size), _p(k_new), _p(v_new),
         _p(pos_new), int(key_mode)))
+
+
+def attention_loss(q, K, dtype, cur_len, scale=0.0, key_mode=0, curves=False, nthreads=1):
+    """Attention loss of norm-based vs ideal compression (Eqs. 5-7).  Returns alr [B, L, Hq]
+    (float64) and, with curves=True, also (loss, loss_ref) [B, L, Hq, T_cap] (NaN past n)."""
+    _check(q, dtype)
+    _check(K, dtype)
+    B, L, Hkv, T_cap, D = K.shape
+    Hq = q.shape[2]
+    cur_len = _i32(cur_len).reshape(B, L)
+    alr = np.zeros((B, L, Hq), dtype=np.float64)
+    loss = np.full((B, L, Hq, T_cap), np.nan) if curves else None
+    ref = np.full((B, L, Hq, T_cap), np.nan) if curves else None
+    rc = lib().l2kv_oracle_attention_loss(
+        _p(q), _p(K), _DT[dtype], B, L, Hkv, Hq, T_cap, D, _p(cur_len), ctypes.c_double(scale),
+        int(key_mode), _p(alr), _p(loss) if curves else None, _p(ref) if curves else None,
+        int(nthreads))
+    if rc != 0:
+        raise ValueError(f"oracle attention_loss: bad argument ({rc})")
+    return (alr, loss, ref) if curves else alr

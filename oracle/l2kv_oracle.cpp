@@ -304,6 +304,63 @@ int l2kv_oracle_attention(const void* q, const void* K_c, const void* V_c, int d
   return 0;
 }
 
+// Attention loss of the norm-based compression against the ideal one (Section 3, Eqs. 5-7),
+// for one query per query head over the cached keys [0, cur_len[b, l]):
+//   a_p        = softmax_p(scale * q . k_p)                                   (Eq. 2)
+//   L^m        = sum of a_p over the m tokens the method drops first, i.e. the m largest in
+//                the order (key, position)                                     (Eq. 5)
+//   L^{m,ref}  = sum of the m smallest a_p (the ideal compression drops the lowest scores)
+//   Y^m        = L^m - L^{m,ref},   Y = sum_{m=1..n} Y^m                      (Eqs. 6, 7)
+// Outputs: alr [B, L, Hq]; optional curves loss / loss_ref [B, L, Hq, T_cap] with L^m at
+// index m - 1 (entries at and beyond n untouched).  key_mode as in compression.
+int l2kv_oracle_attention_loss(const void* q, const void* K, int dtype, int B, int L, int Hkv,
+                               int Hq, int T_cap, int D, const int32_t* cur_len, double scale,
+                               int key_mode, double* alr, double* loss, double* loss_ref,
+                               int nthreads) {
+  if (Hkv <= 0 || Hq % Hkv != 0) return -1;
+  const int G = Hq / Hkv;
+  const double sc = scale > 0.0 ? scale : 1.0 / std::sqrt(static_cast<double>(D));
+  for_each_unit(int64_t(B) * L * Hq, nthreads, [=](int64_t u) {
+    const int hq = static_cast<int>(u % Hq);
+    const int64_t bl = u / Hq;
+    const int n = cur_len[bl];
+    const int64_t kv_row0 = (bl * Hkv + hq / G) * T_cap;
+    alr[u] = 0.0;
+    if (n <= 0) return;
+    std::vector<double> a(n), key(n);
+    double m = -INFINITY;
+    for (int p = 0; p < n; ++p) {
+      double dot = 0.0;
+      for (int d = 0; d < D; ++d)
+        dot += load_elem(q, dtype, u * D + d) * load_elem(K, dtype, (kv_row0 + p) * D + d);
+      a[p] = dot * sc;
+      m = std::max(m, a[p]);
+      key[p] = row_key(K, dtype, (kv_row0 + p) * D, D, key_mode);
+    }
+    double denom = 0.0;
+    for (int p = 0; p < n; ++p) { a[p] = std::exp(a[p] - m); denom += a[p]; }
+    for (int p = 0; p < n; ++p) a[p] /= denom;
+    // drop order of the method: largest (key, position) first
+    std::vector<int32_t> by_norm(n);
+    std::iota(by_norm.begin(), by_norm.end(), 0);
+    std::sort(by_norm.begin(), by_norm.end(), [&](int32_t x, int32_t y) {
+      return key[x] > key[y] || (key[x] == key[y] && x > y);
+    });
+    std::vector<double> asc(a);
+    std::sort(asc.begin(), asc.end());
+    double lm = 0.0, lref = 0.0, y = 0.0;
+    for (int i = 0; i < n; ++i) {
+      lm += a[by_norm[i]];
+      lref += asc[i];
+      y += lm - lref;
+      if (loss) loss[u * T_cap + i] = lm;
+      if (loss_ref) loss_ref[u * T_cap + i] = lref;
+    }
+    alr[u] = y;
+  });
+  return 0;
+}
+
 // a6: append one token per (b, l, h); over budget, evict the highest norm.
 //   K_c, V_c [B, L, H, T_cap, D], idx [B, L, H, T_cap], key_c double (same
 //   shape), cur_len [B, L] in/out, budget[b], k_new / v_new [B, L, H, D],

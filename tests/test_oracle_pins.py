@@ -412,3 +412,51 @@ def test_random_policy_keeps_the_lowest_random_keys():
         freq[oracle.compress(K, V, "f32", [w.T], [keep], uncompressed=(0,), policy=2,
                              seed=seed)["idx"][0, 1, 0, :keep]] += 1
     assert abs(freq.mean() / 200 - keep / w.T) < 1e-12 and freq.min() > 20 and freq.max() < 85
+
+
+# ----------------------------------------- attention loss / ALR (Eqs. 5-7)
+
+def test_attention_loss_hand_worked():
+    g = json.load(open(GOLDEN))["attention_loss"]
+    ln = np.log([1.0, 2.0, 3.0])
+    K = np.zeros((1, 1, 1, 3, 4), np.float64)
+    K[0, 0, 0, :, 0] = ln
+    K[0, 0, 0, :, 1] = np.sqrt(np.array([4.0, 1.0, 9.0]) - ln ** 2)    # norms 2, 1, 3
+    q = np.array([2, 0, 0, 0], np.float32).reshape(1, 1, 1, 4)
+    alr, loss, ref = oracle.attention_loss(q, K.astype(np.float32), "f32", [3], curves=True)
+    np.testing.assert_allclose(loss[0, 0, 0], g["loss"], atol=1e-6)
+    np.testing.assert_allclose(ref[0, 0, 0], g["loss_ref"], atol=1e-6)
+    np.testing.assert_allclose(alr[0, 0, 0], g["alr"], atol=2e-6)
+
+
+def test_attention_loss_invariants_and_brute_force():
+    rng = np.random.default_rng(11)
+    D, n = 64, 9
+    q = rng.standard_normal((1, 1, 4, D)).astype(np.float32)
+    K = (rng.standard_normal((1, 1, 2, n, D)) * rng.uniform(0.3, 2, (1, 1, 2, n, 1))).astype(np.float32)
+    alr, loss, ref = oracle.attention_loss(q, K, "f32", [n], curves=True)
+    s = oracle.key_sumsq(K, "f32")
+    for j in range(4):
+        h = j // 2
+        z = K[0, 0, h].astype(np.float64) @ q[0, 0, j].astype(np.float64) / math.sqrt(D)
+        a = scipy.special.softmax(z)
+        drop = sorted(range(n), key=lambda t: (s[0, 0, h, t], t), reverse=True)
+        for m in range(1, n + 1):
+            np.testing.assert_allclose(loss[0, 0, j, m - 1], a[drop[:m]].sum(), rtol=1e-12)
+            # the ideal compression loses the least attention any m-subset can lose
+            best = min(sum(a[list(c)]) for c in itertools.combinations(range(n), m))
+            np.testing.assert_allclose(ref[0, 0, j, m - 1], best, rtol=1e-12)
+        assert np.all(loss[0, 0, j] >= ref[0, 0, j] - 1e-15)                    # Y^m >= 0
+        np.testing.assert_allclose(loss[0, 0, j, -1], 1.0, rtol=1e-12)
+        np.testing.assert_allclose(alr[0, 0, j], (loss[0, 0, j] - ref[0, 0, j]).sum(), rtol=1e-12)
+        # rank identity: Y = sum_p a_p (rank in ideal order - rank in the method's drop order)
+        rank_n = np.empty(n); rank_n[drop] = np.arange(1, n + 1)
+        rank_a = np.empty(n); rank_a[np.argsort(a, kind="stable")] = np.arange(1, n + 1)
+        np.testing.assert_allclose(alr[0, 0, j], (a * (rank_a - rank_n)).sum(), rtol=1e-10, atol=1e-12)
+    # a cache whose norms fall exactly as the attention rises has no loss at all
+    Kc = np.zeros((1, 1, 1, 5, D), np.float32)
+    Kc[0, 0, 0, :, 0] = [0.5, 0.4, 0.3, 0.2, 0.1]        # scores rise with ... the first coordinate
+    Kc[0, 0, 0, :, 1] = [0.0, 1.0, 2.0, 3.0, 4.0]        # norms rise the other way round
+    qc = np.zeros((1, 1, 1, D), np.float32); qc[..., 0] = 8.0
+    assert abs(oracle.attention_loss(qc, Kc, "f32", [5])[0, 0, 0]) < 1e-15
+    assert oracle.attention_loss(qc, Kc, "f32", [0])[0, 0, 0] == 0.0
