@@ -15,6 +15,7 @@ batch: the path shards over independent (batch, layer, head) units with no excha
 so there is no collective on the data path (weak scaling).
 """
 import argparse
+import ctypes
 import json
 import os
 import statistics
@@ -292,6 +293,21 @@ def time_variants(job, w, cbytes, reps=5):
     job.compress()                     # leave the cache as the method's own policy makes it
     torch.cuda.synchronize()
     out["append_evict"] = time_append_evict(job, w)
+    # attention-loss analysis (Eqs. 5-7) of the full cache: keys from above, first query
+    lens_bl = torch.full((w.B, w.L), w.T, dtype=torch.int32, device=job.dev)
+    alr = torch.zeros((w.B, w.L, w.Hq), dtype=torch.float32, device=job.dev)
+    need = ctypes.c_size_t(0)
+    job.l2.lib().l2kv_attention_loss_workspace_bytes(job.l2.Layout(job.K, q_heads=w.Hq).ref(), w.T,
+                                                     ctypes.byref(need))
+    ws_al = torch.empty(need.value, dtype=torch.uint8, device=job.dev)
+    job.l2.attention_loss(job.q[0], job.K, lens_bl, w.T, keys, alr, workspace=ws_al)
+    t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    job.l2.attention_loss(job.q[0], job.K, lens_bl, w.T, keys, alr, workspace=ws_al)
+    t1.record(); torch.cuda.synchronize()
+    out["attention_loss"] = {"ms": round(t0.elapsed_time(t1), 2), "heads": w.B * w.L * w.Hq,
+                             "tokens_per_head": w.T, "mean_alr": round(float(alr.mean().item()), 2)}
+    del ws_al
     job.compress()
     torch.cuda.synchronize()
     return out

@@ -164,6 +164,27 @@ int l2kv_append_evict(void* K_c, void* V_c, int32_t* idx, float* sumsq_c, const 
                       const void* k_new, const void* v_new, const int32_t* pos_new_dev,
                       void* workspace, size_t workspace_bytes, void* stream);
 
+/* Attention loss of the norm-based compression against the ideal one (Section 3,
+ * Eqs. 5-7), for one query per query head over the cached keys i < cur_len_dev[b,l]:
+ *   a_p       = softmax_p(scale * q . K_p)                       (attention scores, Eq. 2)
+ *   L^m       = sum of a_p over the m tokens the method drops first, i.e. the m last
+ *               in the order (key, position)                      (Eq. 5)
+ *   L^{m,ref} = sum of the m smallest a_p (the ideal compression)
+ *   Y         = sum_{m=1..n} (L^m - L^{m,ref})                     (Eqs. 6, 7)
+ * sumsq holds the keys of K as l2kv_key_norms writes them (dense fp32
+ * [batch, layers, kv_heads, t_cap]).  alr_out is dense fp32 [batch, layers, q_heads].
+ * loss_out / loss_ref_out may be NULL; otherwise dense fp32
+ * [batch, layers, q_heads, t_cap] receiving L^m / L^{m,ref} at index m - 1 (entries at
+ * and beyond n untouched).  Sums are fp64 internally.  An empty cache gives Y = 0.
+ * The workspace needs l2kv_attention_loss_workspace_bytes(lay, max_len) bytes (it is
+ * separate from, and much larger than, the one of the other calls; no zeroing needed).
+ * An analysis tool: it sorts every head's scores and is not tuned like the decode path. */
+int l2kv_attention_loss_workspace_bytes(const l2kv_layout* lay, int32_t max_len, size_t* bytes);
+int l2kv_attention_loss(const void* q, const void* K, const l2kv_layout* lay,
+                        const int32_t* cur_len_dev, int32_t max_len, float scale,
+                        const float* sumsq, float* alr_out, float* loss_out, float* loss_ref_out,
+                        void* workspace, size_t workspace_bytes, void* stream);
+
 /* Decode attention without a workspace -- the paper has no counterpart to this entry
  * point; it exists for the callers of this library that cannot allocate device memory.
  *

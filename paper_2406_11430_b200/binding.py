@@ -55,7 +55,11 @@ def lib():
         L.l2kv_decode_attention.argtypes = [vp, vp, vp, lay, vp, i32, ctypes.c_float, vp, vp, sz, vp]
         L.l2kv_append_evict.argtypes = [vp, vp, vp, vp, lay, vp, vp, ctypes.POINTER(i32), i32,
                                         vp, vp, vp, vp, sz, vp]
-        for name in ("l2kv_keep_count", "l2kv_workspace_bytes", "l2kv_read_device_status",
+        L.l2kv_attention_loss_workspace_bytes.argtypes = [lay, i32, ctypes.POINTER(sz)]
+        L.l2kv_attention_loss.argtypes = [vp, vp, lay, vp, i32, ctypes.c_float, vp, vp, vp, vp,
+                                          vp, sz, vp]
+        for name in ("l2kv_attention_loss_workspace_bytes", "l2kv_attention_loss",
+                     "l2kv_keep_count", "l2kv_workspace_bytes", "l2kv_read_device_status",
                      "l2kv_key_norms", "l2kv_select_compact", "l2kv_decode_attention",
                      "l2kv_append_evict"):
             getattr(L, name).restype = ctypes.c_int
@@ -179,3 +183,20 @@ def decode_attention_static(q, K_c, V_c, cur_len_dev, max_len, out, scale=0.0, s
     lay = Layout(K_c, q_heads=q.shape[2])
     _check(fn(_ptr(q), _ptr(K_c), _ptr(V_c), lay.ref(), _ptr(cur_len_dev), int(max_len),
               float(scale), _ptr(out), _stream(stream)), "l2kv_decode_attention_static")
+
+
+def attention_loss(q, K, cur_len_dev, max_len, sumsq, alr_out, loss_out=None, loss_ref_out=None,
+                   scale=0.0, workspace=None, stream=None):
+    """Attention loss of norm-based vs ideal compression (Eqs. 5-7); see l2kv_attention_loss.
+    Allocates the (large) scratch itself unless a workspace tensor is passed."""
+    lay = Layout(K, q_heads=q.shape[2])
+    if workspace is None:
+        need = ctypes.c_size_t(0)
+        _check(lib().l2kv_attention_loss_workspace_bytes(lay.ref(), int(max_len),
+                                                         ctypes.byref(need)),
+               "l2kv_attention_loss_workspace_bytes")
+        workspace = torch.empty(need.value, dtype=torch.uint8, device=K.device)
+    _check(lib().l2kv_attention_loss(
+        _ptr(q), _ptr(K), lay.ref(), _ptr(cur_len_dev), int(max_len), float(scale), _ptr(sumsq),
+        _ptr(alr_out), _ptr(loss_out), _ptr(loss_ref_out), _ptr(workspace), workspace.numel(),
+        _stream(stream)), "l2kv_attention_loss")

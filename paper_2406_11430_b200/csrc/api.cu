@@ -194,4 +194,32 @@ int l2kv_append_evict(void* K_c, void* V_c, int32_t* idx, float* sumsq_c, const 
                              static_cast<cudaStream_t>(stream));
 }
 
+int l2kv_attention_loss_workspace_bytes(const l2kv_layout* lay, int32_t max_len, size_t* bytes) {
+  if (!bytes || max_len < 0) return L2KV_ERR_INVALID_ARG;
+  const int rc = check_layout(lay);
+  if (rc != L2KV_OK) return rc;
+  *bytes = attention_loss_workspace(*lay, max_len);
+  return L2KV_OK;
+}
+
+int l2kv_attention_loss(const void* q, const void* K, const l2kv_layout* lay,
+                        const int32_t* cur_len_dev, int32_t max_len, float scale,
+                        const float* sumsq, float* alr_out, float* loss_out, float* loss_ref_out,
+                        void* workspace, size_t workspace_bytes, void* stream) {
+  int rc = check_layout(lay);
+  if (rc != L2KV_OK) return rc;
+  if (lay->kv_heads > 0 && lay->q_heads % lay->kv_heads) return L2KV_ERR_INVALID_ARG;
+  if (max_len < 0 || !(scale == scale)) return L2KV_ERR_INVALID_ARG;
+  if (max_len > lay->t_cap) return L2KV_ERR_OUT_OF_RANGE;
+  if ((long long)max_len > (1ll << 24)) return L2KV_ERR_OUT_OF_RANGE;
+  if (empty(lay) || lay->q_heads == 0) return L2KV_OK;
+  if (!q || !K || !cur_len_dev || !sumsq || !alr_out || !workspace) return L2KV_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(K) || !aligned16(workspace)) return L2KV_ERR_MISALIGNED;
+  if (workspace_bytes < attention_loss_workspace(*lay, max_len)) return L2KV_ERR_WORKSPACE_TOO_SMALL;
+  const float sc = scale > 0.f ? scale : 1.0f / std::sqrt((float)lay->head_dim);
+  return launch_attention_loss(q, K, make_geom(*lay), lay->dtype, cur_len_dev, max_len, sc, sumsq,
+                               alr_out, loss_out, loss_ref_out, static_cast<char*>(workspace),
+                               static_cast<cudaStream_t>(stream));
+}
+
 }  // extern "C"

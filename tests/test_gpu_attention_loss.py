@@ -1,0 +1,65 @@
+"""GPU parity of the attention-loss analysis (Eqs. 5-7) against the oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import synth
+from gpu_util import DEV, i32
+
+pytestmark = pytest.mark.gpu
+
+
+def run(l2, q, K, cur, max_len, curves=True):
+    B, L, Hkv, T_cap, D = K.shape
+    Hq = q.shape[2]
+    lens = i32(np.full(B, T_cap))
+    sumsq = torch.zeros((B, L, Hkv, T_cap), dtype=torch.float32, device=DEV)
+    l2.key_norms(K, lens, T_cap, sumsq)
+    alr = torch.full((B, L, Hq), float("nan"), dtype=torch.float32, device=DEV)
+    loss = torch.full((B, L, Hq, T_cap), float("nan"), dtype=torch.float32, device=DEV) if curves else None
+    ref = torch.full((B, L, Hq, T_cap), float("nan"), dtype=torch.float32, device=DEV) if curves else None
+    l2.attention_loss(q, K, i32(np.asarray(cur).reshape(B, L)), max_len, sumsq, alr, loss, ref)
+    torch.cuda.synchronize()
+    return alr.cpu().numpy(), (loss.cpu().numpy() if curves else None), (ref.cpu().numpy() if curves else None)
+
+
+@pytest.mark.parametrize("dtype,D,Hkv,Hq,T", [("bf16", 128, 2, 8, 5000), ("f32", 64, 4, 4, 1024),
+                                             ("bf16", 64, 2, 2, 4097), ("f32", 128, 1, 2, 700)])
+def test_attention_loss_matches_oracle(dtype, D, Hkv, Hq, T):
+    import paper_2406_11430_b200 as l2
+    w = synth.WORKLOADS[2].scaled(dtype=dtype, D=D, Hkv=Hkv, Hq=Hq, B=2, L=2, T=T)
+    K, _ = synth.make_cache(w, DEV)
+    q = synth.make_query(w, 0, DEV)
+    cur = np.array([[T, 1], [0, max(2, T // 3)]], dtype=np.int32)
+    alr, loss, ref = run(l2, q, K, cur, T)
+    want, wloss, wref = oracle.attention_loss(synth.to_numpy(q), synth.to_numpy(K), dtype, cur,
+                                              key_mode=1, curves=True, nthreads=8)
+    for b in range(2):
+        for l in range(2):
+            n = cur[b, l]
+            np.testing.assert_allclose(loss[b, l, :, :n], wloss[b, l, :, :n], rtol=0, atol=3e-5)
+            np.testing.assert_allclose(ref[b, l, :, :n], wref[b, l, :, :n], rtol=0, atol=3e-5)
+            assert np.isnan(loss[b, l, :, n:]).all()                 # untouched past n
+            np.testing.assert_allclose(alr[b, l], want[b, l], rtol=2e-4, atol=1e-4 * max(n, 1))
+    assert np.all(alr[1, 0] == 0.0) and np.all(alr[0, 1] == 0.0)      # empty / one-token caches
+    assert np.all(alr >= -1e-3)
+
+
+def test_attention_loss_planted_structure():
+    # Keys whose norm falls exactly as their score rises lose nothing against the ideal.
+    import paper_2406_11430_b200 as l2
+    n, D = 3000, 128
+    K = torch.zeros((1, 1, 1, n, D), dtype=torch.float32, device=DEV)
+    K[0, 0, 0, :, 0] = torch.linspace(1.0, 0.0, n, device=DEV)      # score falls with position
+    K[0, 0, 0, :, 1] = torch.linspace(1.0, 9.0, n, device=DEV)      # norm rises with position
+    q = torch.zeros((1, 1, 1, D), dtype=torch.float32, device=DEV)
+    q[..., 0] = 30.0
+    alr, _, _ = run(l2, q, K, [[n]], n, curves=False)
+    assert abs(alr[0, 0, 0]) < 1e-2
+    alr2, _, _ = run(l2, q, K.flip(3).contiguous(), [[n]], n, curves=False)   # same set, other slots
+    assert abs(alr2[0, 0, 0]) < 1e-2
+    # the opposite pairing (highest norm = highest score) is the worst case: loss well above 0
+    K[0, 0, 0, :, 1] = torch.linspace(9.0, 1.0, n, device=DEV)
+    alr3, _, _ = run(l2, q, K, [[n]], n, curves=False)
+    assert alr3[0, 0, 0] > 100.0
