@@ -39,7 +39,7 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes (read + written) per algorithmic byte of the dominant kernel, from the ncu capture
 # summarised in profiles/decode_split_mma_kernel_llama3-8b-32k_4layers.md (a 4-layer case; the
 # traffic is proportional to the tokens streamed).  Set to None whenever that kernel changes.
-DECODE_TRAFFIC_RATIO = None
+DECODE_TRAFFIC_RATIO = 1.0058
 
 
 def workload(args):
