@@ -43,28 +43,42 @@ DECODE_TRAFFIC_RATIO = 1.0058
 
 
 def workload(args):
-    w = synth.WORKLOADS[2]
+    """The benchmark workload: configuration 2 (Llama-3-8B, 32k context) unless --workload
+    picks another of the five; the serving workload is cut to 8 of its 32 layers, since all 32
+    padded to the longest sequence do not fit one GPU next to their compressed copy."""
+    w = synth.WORKLOADS[args.workload]
+    if w.append_steps and not args.layers:
+        w = w.scaled(L=8)
     if args.layers:
         w = w.scaled(L=args.layers)
     if args.context:
         w = w.scaled(T=args.context)
     if args.decode_steps:
-        w = w.scaled(decode_steps=args.decode_steps)
+        w = w.scaled(decode_steps=args.decode_steps,
+                     append_steps=args.decode_steps if w.append_steps else 0)
     return w
 
 
-def algorithmic_bytes(w):
-    """Bytes the method must move, per step, from the shapes alone."""
+def algorithmic_bytes(w, lens=None):
+    """Bytes the method must move, per step, from the shapes alone:
+    (compression pass, all decode-attention steps together, all append/evict steps together)."""
     e, row = w.elem_bytes, w.D * w.elem_bytes
-    keep = int(np.ceil(w.keep_ratio * w.T))
+    lens = [w.T] * w.B if lens is None else [int(n) for n in lens]
     n_unc = len([l for l in w.uncompressed if l < w.L])
-    units_c = w.B * (w.L - n_unc) * w.Hkv
-    units_u = w.B * n_unc * w.Hkv
-    # compressed unit: read K once for the norms, read kept K and V rows, write them, plus
-    # the index map and stored keys; uncompressed unit: read and write K and V once
-    compress = units_c * (w.T * row + 4 * keep * row + 8 * keep) + units_u * (4 * w.T * row + 8 * w.T)
-    decode = (units_c * keep + units_u * w.T) * 2 * row + w.B * w.L * w.Hq * w.D * (e + 4)
-    return compress, decode, keep
+    n_cmp = w.L - n_unc
+    compress = decode = append = 0
+    for n in lens:
+        keep = int(np.ceil(w.keep_ratio * n))
+        # compressed unit: read K once for the norms, read kept K and V rows, write them, plus
+        # the index map and stored keys; uncompressed unit: read and write K and V once
+        compress += w.Hkv * (n_cmp * (n * row + 4 * keep * row + 8 * keep) + n_unc * (4 * n * row + 8 * n))
+        for s in range(w.decode_steps):
+            grown = n + (s + 1 if w.append_steps else 0)          # uncompressed layers only append
+            decode += w.Hkv * (n_cmp * keep + n_unc * grown) * 2 * row
+            if w.append_steps:
+                append += w.Hkv * (n_cmp * keep * 8 + w.L * (4 * row + 8))
+    decode += w.decode_steps * w.B * w.L * w.Hq * w.D * (e + 4)
+    return compress, decode, append
 
 
 def measured_peak():
@@ -150,22 +164,30 @@ class Job:
         self.l2, self.w, self.dev = l2, w, device
         ws = w.scaled(seed=w.seed + 1000 * rank)          # each rank its own batch
         self.K, self.V = synth.make_cache(ws, device)
-        shape = (w.B, w.L, w.Hkv, w.T, w.D)
+        self.lens_host = synth.ragged_lengths(ws)
+        self.keep_host = np.ceil(w.keep_ratio * self.lens_host.astype(np.float64)).astype(np.int32)
+        self.t_cap = w.T + w.append_steps                 # uncompressed layers grow by one per step
+        shape = (w.B, w.L, w.Hkv, self.t_cap, w.D)
         self.K_c = torch.zeros(shape, dtype=w.torch_dtype, device=device)
         self.V_c = torch.zeros_like(self.K_c)
         self.idx = torch.zeros(shape[:4], dtype=torch.int32, device=device)
         self.sumsq = torch.zeros(shape[:4], dtype=torch.float32, device=device)
         self.cur = torch.zeros((w.B, w.L), dtype=torch.int32, device=device)
-        self.keep_n = int(np.ceil(w.keep_ratio * w.T))
-        self.lens = torch.full((w.B,), w.T, dtype=torch.int32, device=device)
-        self.keep = torch.full((w.B,), self.keep_n, dtype=torch.int32, device=device)
+        self.keep_n = int(self.keep_host.max())
+        self.lens = torch.tensor(self.lens_host, dtype=torch.int32, device=device)
+        self.keep = torch.tensor(self.keep_host, dtype=torch.int32, device=device)
         self.unc = tuple(l for l in w.uncompressed if l < w.L)
         self.q = torch.stack([synth.make_query(ws, s, device) for s in range(w.decode_steps)])
         self.out = torch.zeros((w.decode_steps, w.B, w.L, w.Hq, w.D), dtype=torch.float32,
                                device=device)
-        self.ws = l2.new_workspace(l2.Layout(self.K, q_heads=w.Hq), w.T, device)
-        # norm pass (with the selection inside) + gather, then split + merge per decode step
-        self.launches_per_step = 2 + 2 * w.decode_steps
+        self.ws = l2.new_workspace(l2.Layout(self.K_c, q_heads=w.Hq), self.t_cap, device)
+        self.new_rows, self.new_pos = [], []
+        for s in range(w.append_steps):                   # budget-maintained serving loop
+            self.new_rows.append(synth.make_new_kv(ws, s, device))
+            self.new_pos.append(self.lens + s)
+        # norm pass (with the selection inside) + gather; per decode step split + merge, and
+        # one append/evict launch when the workload maintains a budget
+        self.launches_per_step = 2 + (3 if w.append_steps else 2) * w.decode_steps
 
     def compress(self):
         self.l2.select_compact(self.K, self.V, self.lens, self.keep, self.w.T, self.unc, self.K_c,
@@ -177,7 +199,11 @@ class Job:
                                seed=1, sumsq_in=sumsq_in)
 
     def decode(self, s):
-        self.l2.decode_attention(self.q[s], self.K_c, self.V_c, self.cur, self.w.T, self.out[s],
+        if self.w.append_steps:
+            k, v = self.new_rows[s]
+            self.l2.append_evict(self.K_c, self.V_c, self.idx, self.sumsq, self.cur, self.keep,
+                                 self.unc, k, v, self.new_pos[s], self.ws)
+        self.l2.decode_attention(self.q[s], self.K_c, self.V_c, self.cur, self.t_cap, self.out[s],
                                  self.ws)
 
     def step(self, ev=None):
@@ -200,8 +226,10 @@ def run_gpu(args):
     torch.cuda.set_device(device)
     w = workload(args)
     job = Job(w, device, rank)
-    cbytes, dbytes, keep = algorithmic_bytes(w)
-    step_bytes = cbytes + w.decode_steps * dbytes
+    cbytes, dbytes_all, abytes_all = algorithmic_bytes(w, job.lens_host)
+    dbytes = (dbytes_all + abytes_all) / w.decode_steps   # per decode step (with its append, if any)
+    step_bytes = cbytes + dbytes_all + abytes_all
+    keep = job.keep_n
 
     for _ in range(max(args.warmup, 3)):
         job.step()
@@ -221,7 +249,9 @@ def run_gpu(args):
     c_ms = max_over_ranks(c_ms, world, device)
     d_ms = max_over_ranks(d_ms, world, device)
 
-    variants = time_variants(job, w, cbytes) if (rank == 0 and not args.no_variants) else None
+    variants = None
+    if rank == 0 and not args.no_variants and not w.append_steps and not w.ragged_lo:
+        variants = time_variants(job, w, cbytes)
 
     # end to end: inputs start in pinned host memory, results end there
     e2e = None
@@ -242,14 +272,17 @@ def run_gpu(args):
         "data": "synthetic",
         "config": {"workload": w.name, "batch": w.B, "layers": w.L, "kv_heads": w.Hkv,
                    "q_heads": w.Hq, "head_dim": w.D, "context": w.T, "storage": w.dtype,
+                   "ragged_lengths": bool(w.ragged_lo),
+                   "append_evict_per_decode_step": bool(w.append_steps),
                    "keep_ratio": w.keep_ratio, "keep_per_head": keep,
                    "uncompressed_layers": list(job.unc), "decode_steps_per_step": w.decode_steps,
-                   "l2": "inputs larger than L2 (8.5 GiB read per decode step, 16 GiB per compress)",
+                   "l2": f"inputs larger than L2 ({dbytes / GIB:.1f} GiB read per decode step, "
+                         f"{2 * job.K.numel() * w.elem_bytes / GIB:.0f} GiB of K and V per compress)",
                    "parallelism": f"independent replicas x{world}, no collective"},
-        "compress": {"ms": round(c_ms, 3), "GBps": round(cmp_gbs, 1), "bytes": cbytes,
+        "compress": {"ms": round(c_ms, 3), "GBps": round(cmp_gbs, 1), "bytes": int(cbytes),
                      "frac_of_8TBps": round(cmp_gbs / NOMINAL_HBM_GBS, 4),
                      f"frac_of_{peak_kind}": round(cmp_gbs / peak, 4)},
-        "decode": {"ms_per_decode_step": round(d_ms, 4), "GBps": round(dec_gbs, 1), "bytes": dbytes,
+        "decode": {"ms_per_decode_step": round(d_ms, 4), "GBps": round(dec_gbs, 1), "bytes": int(dbytes),
                    "frac_of_8TBps": round(dec_gbs / NOMINAL_HBM_GBS, 4),
                    f"frac_of_{peak_kind}": round(dec_gbs / peak, 4),
                    "tokens_per_s": round(world * w.B / (d_ms * 1e-3), 1)},
@@ -257,7 +290,8 @@ def run_gpu(args):
                      "achieved": round(dec_gbs, 1), "peak": peak, "peak_kind": peak_kind,
                      "unit": "GB/s", "frac": round(dec_gbs / peak, 4),
                      "traffic": args.traffic if args.traffic is not None else
-                     (round(DECODE_TRAFFIC_RATIO * dbytes) if DECODE_TRAFFIC_RATIO else None)},
+                     (round(DECODE_TRAFFIC_RATIO * dbytes)
+                      if DECODE_TRAFFIC_RATIO and args.workload == 2 and not w.append_steps else None)},
         "gpu_launches": job.launches_per_step * args.steps,
         "clocks": clocks,
     }
@@ -401,8 +435,8 @@ def oracle_sample_step(w, seed_shift=0, n_dec=2, n_comp=1, nthreads=None):
     for q in qs:
         oracle.attention(q, r["K_c"], r["V_c"], w.dtype, r["kept_len"], nthreads=nthreads)
     dt = time.perf_counter() - t0
-    cb, db, _ = algorithmic_bytes(sub.scaled(decode_steps=n_dec))
-    return dt, cb + n_dec * db, nthreads, layers
+    cb, db, _ = algorithmic_bytes(sub.scaled(decode_steps=n_dec, append_steps=0, ragged_lo=0))
+    return dt, cb + db, nthreads, layers
 
 
 def cpu_baseline(w, target_s=15.0):
@@ -457,6 +491,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-variants", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    ap.add_argument("--workload", type=int, default=2, choices=range(len(synth.WORKLOADS)),
+                    help="which of the five configurations (default 2: llama3-8b-32k)")
     ap.add_argument("--layers", type=int, default=0, help="profiling aid: fewer layers")
     ap.add_argument("--context", type=int, default=0, help="profiling aid: shorter context")
     ap.add_argument("--decode-steps", type=int, default=0, help="profiling aid")

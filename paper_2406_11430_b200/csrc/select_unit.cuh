@@ -10,11 +10,15 @@
 
 namespace l2kv {
 
+constexpr int kCandCap = 2 * kMaxChunks;        // candidate keys that fit the shared list
+
 struct SelectSmem {
   int hist[256];
-  int bucket, before;
-  int c_less[kMaxChunks];
-  int c_eq[kMaxChunks];
+  int bucket, before, in_bucket, n_cand;
+  union {
+    struct { int c_less[kMaxChunks]; int c_eq[kMaxChunks]; };   // after the passes
+    uint32_t cand[kCandCap];                                    // during the passes
+  };
 };
 
 // Keys may have been written by other CTAs of the same grid: read them through L2.
@@ -26,35 +30,47 @@ template <int NT>
 __device__ void select_unit(SelectSmem& sm, const float* __restrict__ key, int len, int keep,
                             int policy, uint32_t flags, UnitRec* __restrict__ rec,
                             int2* __restrict__ crec) {
-  constexpr int kBatch = 8;                      // independent key loads in flight per thread
+  constexpr int kBatch = 16;                     // independent key loads in flight per thread
   const int tid = threadIdx.x;
   const int my_chunks = (len + kGatherChunk - 1) / kGatherChunk;
   uint32_t prefix = 0, mask = 0;
   int k_rem = keep;
+  // Passes scan every key until the keys that still match the prefix fit the shared list;
+  // the next pass then also collects them, and the passes after that only look at the list.
+  bool collect = false, listed = false;
   for (int shift = 24; shift >= 0; shift -= 8) {
     for (int i = tid; i < 256; i += NT) sm.hist[i] = 0;
+    if (tid == 0 && collect) sm.n_cand = 0;
     __syncthreads();
     // Run-length accumulation: neighbouring tokens mostly share the high digits, so the
     // shared-memory atomics of the first passes collapse to a few per thread.
     int cur = -1, cnt = 0;
-    for (int base = 0; base < len; base += NT * kBatch) {
-      uint32_t kb[kBatch];
-#pragma unroll
-      for (int j = 0; j < kBatch; ++j) {
-        const int t = base + j * NT + tid;
-        kb[j] = t < len ? load_key_bits(key + t, policy) : 0u;
+    auto tally = [&](uint32_t kb) {
+      if ((kb & mask) != prefix) return false;
+      const int d = (kb >> shift) & 255;
+      if (d == cur) {
+        ++cnt;
+      } else {
+        if (cnt) atomicAdd(&sm.hist[cur], cnt);
+        cur = d; cnt = 1;
       }
+      return true;
+    };
+    if (listed) {
+      const int n_cand = sm.n_cand;
+      for (int i = tid; i < n_cand; i += NT) tally(sm.cand[i]);
+    } else {
+      for (int base = 0; base < len; base += NT * kBatch) {
+        uint32_t kb[kBatch];
 #pragma unroll
-      for (int j = 0; j < kBatch; ++j) {
-        const int t = base + j * NT + tid;
-        if (t < len && (kb[j] & mask) == prefix) {
-          const int d = (kb[j] >> shift) & 255;
-          if (d == cur) {
-            ++cnt;
-          } else {
-            if (cnt) atomicAdd(&sm.hist[cur], cnt);
-            cur = d; cnt = 1;
-          }
+        for (int j = 0; j < kBatch; ++j) {
+          const int t = base + j * NT + tid;
+          kb[j] = t < len ? load_key_bits(key + t, policy) : 0u;
+        }
+#pragma unroll
+        for (int j = 0; j < kBatch; ++j) {
+          const int t = base + j * NT + tid;
+          if (t < len && tally(kb[j]) && collect) sm.cand[atomicAdd(&sm.n_cand, 1)] = kb[j];
         }
       }
     }
@@ -75,7 +91,9 @@ __device__ void select_unit(SelectSmem& sm, const float* __restrict__ key, int l
       if (before < k_rem && k_rem <= inc) {
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-          if (before < k_rem && k_rem <= before + v[i]) { sm.bucket = tid * 8 + i; sm.before = before; }
+          if (before < k_rem && k_rem <= before + v[i]) {
+            sm.bucket = tid * 8 + i; sm.before = before; sm.in_bucket = v[i];
+          }
           before += v[i];
         }
       }
@@ -84,6 +102,8 @@ __device__ void select_unit(SelectSmem& sm, const float* __restrict__ key, int l
     prefix |= (uint32_t)sm.bucket << shift;
     mask |= 255u << shift;
     k_rem -= sm.before;
+    if (collect) { listed = true; collect = false; }
+    else if (!listed && sm.in_bucket <= kCandCap) collect = true;
     __syncthreads();
   }
   const uint32_t thr = prefix;      // the keep-th smallest key; k_rem of its copies are admitted
@@ -91,7 +111,8 @@ __device__ void select_unit(SelectSmem& sm, const float* __restrict__ key, int l
     UnitRec r; r.thr = thr; r.admit = k_rem; r.n_keep = keep; r.flags = flags;
     *rec = r;
   }
-  // Per-chunk counts of keys below / equal to the threshold, one warp per chunk.
+  // Per-chunk counts of keys below / equal to the threshold, one warp per chunk (the
+  // candidate list is dead by now: its storage becomes the count arrays).
   const int warp = tid >> 5, lane = tid & 31;
   for (int c = warp; c < my_chunks; c += NT / 32) {
     const int t0 = c * kGatherChunk;
