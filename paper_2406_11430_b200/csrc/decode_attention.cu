@@ -11,12 +11,10 @@
 //   decode_combine_kernel  merges the partials of all splits of a query head.
 //
 // All arithmetic is fp32 on values widened exactly from the stored bf16 / fp32.
-#include <cuda.h>      // CUtensorMap and its enums only; the encoder is fetched from the driver at run time
-
 #include <cstdlib>
 #include <cstring>
 
-#include "common.cuh"
+#include "async_copy.cuh"
 
 namespace l2kv {
 
@@ -253,9 +251,6 @@ constexpr int kDbw = 8 / kMmaWarps;                    // 16-dim output blocks p
 constexpr int kRowBytes = 256;                         // 128 bf16
 constexpr int kScLd = kDecodeChunk + 4;                // floats per head row of the score buffer
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-  return (uint32_t)__cvta_generic_to_shared(p);
-}
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int bytes) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" :: "r"(dst), "l"(src), "r"(bytes)
                : "memory");
@@ -276,34 +271,6 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], 
   asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
                : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-
-// ---- mbarrier / TMA (cp.async.bulk.tensor) helpers -------------------------------------
-__device__ __forceinline__ void mbar_init(uint32_t bar, int count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"(bytes)
-               : "memory");
-}
-// Waits for the phase with the given parity; gives up after a bounded number of polls (a
-// copy that never lands must not hang the GPU) and reports that through the return value.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  for (int spin = 0; spin < (1 << 20); ++spin) {
-    uint32_t done;
-    asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; "
-                 "selp.u32 %0, 1, 0, p; }" : "=r"(done) : "r"(bar), "r"(parity) : "memory");
-    if (done) return true;
-  }
-  return false;
-}
-// One box of a rank-5 tensor map (dims: head_dim, token, kv head, layer, batch) into shared memory.
-__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map, uint32_t bar,
-                                            int c0, int c1, int c2, int c3, int c4) {
-  asm volatile("cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
-               "[%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
-               :: "r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
-               : "memory");
 }
 
 // Shared-memory address of the 16-byte piece `ch` of row `row` of a stage.  cp.async path:
@@ -605,35 +572,6 @@ decode_split_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16
   }
 }
 
-// Builds the rank-5 tensor map (head_dim, token, kv head, layer, batch) of a bf16 cache with a
-// box of 64 elements x kStageTok tokens and the 128-byte swizzle.  Returns false when the
-// encoder is unavailable or rejects the geometry (the caller then uses the cp.async path).
-static bool make_cache_map(CUtensorMap* map, const void* base, const Geom& g) {
-  using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
-                                const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
-                                const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-  static EncodeFn encode = []() -> EncodeFn {
-    void* fn = nullptr;
-    cudaDriverEntryPointQueryResult res;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &res) !=
-            cudaSuccess || res != cudaDriverEntryPointSuccess)
-      return nullptr;
-    return reinterpret_cast<EncodeFn>(fn);
-  }();
-  if (!encode) return false;
-  if (g.st <= 0 || g.sh <= 0 || g.sl <= 0 || g.sb <= 0) return false;   // broadcast views
-  const cuuint64_t dims[5] = {128, (cuuint64_t)g.t_cap, (cuuint64_t)g.H, (cuuint64_t)g.L,
-                              (cuuint64_t)g.B};
-  const cuuint64_t strides[4] = {(cuuint64_t)g.st * 2, (cuuint64_t)g.sh * 2, (cuuint64_t)g.sl * 2,
-                                 (cuuint64_t)g.sb * 2};
-  const cuuint32_t box[5] = {64, (cuuint32_t)kStageTok, 1, 1, 1};
-  const cuuint32_t elem[5] = {1, 1, 1, 1, 1};
-  return encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(base), dims, strides,
-                box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 template <int G>
 static int launch_dec_mma(const void* q, const void* K, const void* V, const Geom& g,
                           const int32_t* cur_len_dev, int max_len, float scale, float* out,
@@ -651,7 +589,7 @@ static int launch_dec_mma(const void* q, const void* K, const void* V, const Geo
     std::memset(&map_v, 0, sizeof map_v);
     const char* mode = std::getenv("L2KV_DECODE_COPY");
     const bool want_tma = !(mode && std::strcmp(mode, "cpasync") == 0);
-    const bool tma = want_tma && make_cache_map(&map_k, K, g) && make_cache_map(&map_v, V, g);
+    const bool tma = want_tma && make_cache_map(&map_k, K, g, kStageTok) && make_cache_map(&map_v, V, g, kStageTok);
     auto kern = tma ? decode_split_mma_kernel<G, true> : decode_split_mma_kernel<G, false>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) !=
         cudaSuccess)
