@@ -164,6 +164,25 @@ int l2kv_append_evict(void* K_c, void* V_c, int32_t* idx, float* sumsq_c, const 
                       const void* k_new, const void* v_new, const int32_t* pos_new_dev,
                       void* workspace, size_t workspace_bytes, void* stream);
 
+/* Prefix attention: n_queries new queries per (b, l) -- a prefill chunk, or several draft
+ * tokens -- over the compressed cache, with the fused online-softmax formulation that the
+ * method stays compatible with because it never needs the attention scores (Abstract;
+ * Section 1).  Eq. 2 per query, over the cached rows i < cur_len_dev[b,l], no mask (every
+ * cached token precedes the new ones; attention among the new tokens themselves is the
+ * caller's, to be merged with this result through lse_out):
+ *   out[b,l,s,j,:] = sum_i softmax_i( scale * q[b,l,s,j,:] . K_c[b,l,j/G,i,:] ) * V_c[b,l,j/G,i,:]
+ * q is dense bf16 [batch, layers, n_queries, q_heads, head_dim]; out dense fp32 of the same
+ * shape; lse_out (may be NULL) dense fp32 [batch, layers, n_queries, q_heads] receives the
+ * natural-log sum of exponentials of the scaled scores.  bf16 caches with head_dim 128 only
+ * (L2KV_ERR_UNSUPPORTED otherwise, also for strides a tensor map cannot express).  Products
+ * are exact, sums fp32; the softmax weights are rounded to bf16 before they multiply V, as
+ * in FlashAttention.  An empty cache gives zeros and lse = -inf.  workspace may be NULL; if
+ * given (>= 256 bytes, zeroed) its status word reports a copy or MMA wait that gave up. */
+int l2kv_prefix_attention(const void* q, const void* K_c, const void* V_c, const l2kv_layout* lay,
+                          const int32_t* cur_len_dev, int32_t max_len, int32_t n_queries, float scale,
+                          float* out, float* lse_out, void* workspace, size_t workspace_bytes,
+                          void* stream);
+
 /* Attention loss of the norm-based compression against the ideal one (Section 3,
  * Eqs. 5-7), for one query per query head over the cached keys i < cur_len_dev[b,l]:
  *   a_p       = softmax_p(scale * q . K_p)                       (attention scores, Eq. 2)

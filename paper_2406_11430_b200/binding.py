@@ -58,7 +58,9 @@ def lib():
         L.l2kv_attention_loss_workspace_bytes.argtypes = [lay, i32, ctypes.POINTER(sz)]
         L.l2kv_attention_loss.argtypes = [vp, vp, lay, vp, i32, ctypes.c_float, vp, vp, vp, vp,
                                           vp, sz, vp]
-        for name in ("l2kv_attention_loss_workspace_bytes", "l2kv_attention_loss",
+        L.l2kv_prefix_attention.argtypes = [vp, vp, vp, lay, vp, i32, i32, ctypes.c_float, vp, vp,
+                                            vp, sz, vp]
+        for name in ("l2kv_prefix_attention", "l2kv_attention_loss_workspace_bytes", "l2kv_attention_loss",
                      "l2kv_keep_count", "l2kv_workspace_bytes", "l2kv_read_device_status",
                      "l2kv_key_norms", "l2kv_select_compact", "l2kv_decode_attention",
                      "l2kv_append_evict"):
@@ -200,3 +202,13 @@ def attention_loss(q, K, cur_len_dev, max_len, sumsq, alr_out, loss_out=None, lo
         _ptr(q), _ptr(K), lay.ref(), _ptr(cur_len_dev), int(max_len), float(scale), _ptr(sumsq),
         _ptr(alr_out), _ptr(loss_out), _ptr(loss_ref_out), _ptr(workspace), workspace.numel(),
         _stream(stream)), "l2kv_attention_loss")
+
+
+def prefix_attention(q, K_c, V_c, cur_len_dev, max_len, out, lse_out=None, scale=0.0, workspace=None,
+                     stream=None):
+    """n_queries new queries per (b, l) over the compressed cache; q [B, L, Sq, Hq, D] bf16."""
+    lay = Layout(K_c, q_heads=q.shape[3])
+    _check(lib().l2kv_prefix_attention(
+        _ptr(q), _ptr(K_c), _ptr(V_c), lay.ref(), _ptr(cur_len_dev), int(max_len), int(q.shape[2]),
+        float(scale), _ptr(out), _ptr(lse_out), _ptr(workspace),
+        0 if workspace is None else workspace.numel(), _stream(stream)), "l2kv_prefix_attention")

@@ -194,6 +194,28 @@ int l2kv_append_evict(void* K_c, void* V_c, int32_t* idx, float* sumsq_c, const 
                              static_cast<cudaStream_t>(stream));
 }
 
+int l2kv_prefix_attention(const void* q, const void* K_c, const void* V_c, const l2kv_layout* lay,
+                          const int32_t* cur_len_dev, int32_t max_len, int32_t n_queries, float scale,
+                          float* out, float* lse_out, void* workspace, size_t workspace_bytes,
+                          void* stream) {
+  int rc = check_layout(lay);
+  if (rc != L2KV_OK) return rc;
+  rc = check_groups(lay);
+  if (rc != L2KV_OK) return rc;
+  if (lay->dtype != L2KV_BF16 || lay->head_dim != 128) return L2KV_ERR_UNSUPPORTED;
+  if (max_len < 0 || n_queries < 0 || !(scale == scale)) return L2KV_ERR_INVALID_ARG;
+  if (max_len > lay->t_cap) return L2KV_ERR_OUT_OF_RANGE;
+  if (empty(lay) || n_queries == 0) return L2KV_OK;
+  if (!q || !K_c || !V_c || !cur_len_dev || !out) return L2KV_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(K_c) || !aligned16(V_c) || !aligned16(out))
+    return L2KV_ERR_MISALIGNED;
+  if (workspace && workspace_bytes < (size_t)kStatusBytes) return L2KV_ERR_WORKSPACE_TOO_SMALL;
+  const float sc = scale > 0.f ? scale : 1.0f / std::sqrt((float)lay->head_dim);
+  return launch_prefix_attention(q, K_c, V_c, make_geom(*lay), lay->dtype, n_queries, cur_len_dev,
+                                 max_len, sc, out, lse_out, static_cast<int32_t*>(workspace),
+                                 static_cast<cudaStream_t>(stream));
+}
+
 int l2kv_attention_loss_workspace_bytes(const l2kv_layout* lay, int32_t max_len, size_t* bytes) {
   if (!bytes || max_len < 0) return L2KV_ERR_INVALID_ARG;
   const int rc = check_layout(lay);

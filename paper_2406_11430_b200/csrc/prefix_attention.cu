@@ -1,0 +1,316 @@
+// Prefix attention: a block of new queries (a prefill chunk, or several draft tokens) attends
+// to the whole compressed cache.  Unlike single-query decode this is a dense contraction --
+// 4 * Sq * Hq * D flop per cached token per (b, l) -- so it runs on the Blackwell tensor cores
+// (tcgen05.mma, operands in shared memory, accumulators in tensor memory).
+//
+// One CTA (128 threads) per (b, l, kv head, tile of 128 / G queries): its 128 rows are the
+// (query, head-of-the-group) pairs that share one KV head.  Per block of 128 cached tokens:
+//   K block  -- TMA --> shared memory (128-byte swizzle)
+//   S = Q . K^T            8 x tcgen05.mma (M 128, N 128, K 16), fp32 in tensor memory
+//   thread r reads row r of S (tcgen05.ld): running maximum, weights 2^(s - m) as bf16 back
+//   to shared memory (over the K block, which is no longer needed), running sum
+//   V block  -- TMA --> shared memory;  O_blk = P . V   8 x tcgen05.mma (V as an N-major operand)
+//   thread r reads row r of O_blk and folds it into its fp32 accumulator row (rescaled by
+//   2^(m_old - m_new)), FlashAttention style.
+// Every wait on an mbarrier is bounded (a wait that gives up ends the CTA's loop and marks
+// the status word); tensor memory is released on every path.
+#include <cstring>
+
+#include "async_copy.cuh"
+
+namespace l2kv {
+
+constexpr int kPfThreads = 128;
+constexpr int kPfRows = 128;                    // query rows per CTA, cached tokens per block
+constexpr int kPfHalf = kPfRows * 128;          // one [128 rows][64 bf16] swizzled tile: 16 KB
+constexpr int kPfTileBytes = 2 * kPfHalf;       // both halves of the head dimension: 32 KB
+constexpr int kPfTmemCols = 256;                // S: columns 0..127, O_blk: columns 128..255
+constexpr int kPfPolls = 18;                    // log2 of the polls a wait may take
+constexpr float kPfLog2e = 1.4426950408889634f;
+
+// Instruction descriptor of tcgen05.mma kind::f16: fp32 accumulate (bits 4-5 = 1), bf16 A and B
+// (bits 7-9 and 10-12 = 1), A/B major-ness (bits 15, 16; 0 = K-major), N / 8 (bits 17-22),
+// M / 16 (bits 24-28).
+constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+constexpr uint32_t kIdescPV = kIdescQK | (1u << 16);       // V is N-major (head_dim contiguous)
+
+// Shared-memory matrix descriptor: start address, leading / stride byte offsets (all / 16),
+// descriptor version 1 (bit 46), 128-byte swizzle (layout type 2 in bits 61-63).
+__device__ __forceinline__ uint64_t umma_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) |
+         ((uint64_t)(sbo_bytes >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
+                                          uint32_t idesc, uint32_t accumulate) {
+  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+               "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+               :: "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u)
+               : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+               :: "r"(bar) : "memory");
+}
+// 32 consecutive fp32 columns of this thread's tensor-memory lane.  Whole warps only.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+               "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+               "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
+                 "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]),
+                 "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]),
+                 "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+                 "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]),
+                 "=r"(r[31])
+               : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void proxy_fence() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+__device__ __forceinline__ void st_shared16(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" :: "r"(addr), "r"(a), "r"(b), "r"(c), "r"(d)
+               : "memory");
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&v);
+}
+
+template <int G>
+__global__ void __launch_bounds__(kPfThreads, 2)
+prefix_attention_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n_queries,
+                        const int32_t* __restrict__ cur_len_dev, int max_len, float scale_log2e,
+                        float* __restrict__ out, float* __restrict__ lse_out,
+                        const __grid_constant__ CUtensorMap map_k,
+                        const __grid_constant__ CUtensorMap map_v, int32_t* __restrict__ status_word) {
+  constexpr int D = 128;
+  constexpr int QT = kPfRows / G;                       // queries per CTA
+  extern __shared__ unsigned char smem_raw[];
+  __shared__ __align__(8) unsigned long long s_bar[3];  // K landed, V landed, MMA done
+  __shared__ uint32_t s_tmem;
+
+  const int q_tiles = (n_queries + QT - 1) / QT;
+  const int qt = blockIdx.x % q_tiles;
+  const long long unit = blockIdx.x / q_tiles;          // (b * L + l) * H + h
+  const int h = (int)(unit % g.H);
+  const long long bl = unit / g.H;
+  const int l = (int)(bl % g.L), b = (int)(bl / g.L);
+  const int n = max(0, min(cur_len_dev[bl], min(max_len, g.t_cap)));
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const int s_idx = qt * QT + tid / G;                  // this thread's query and head
+  const int head = h * G + tid % G;
+  const bool row_valid = s_idx < n_queries;
+  const long long row_off = ((bl * n_queries + s_idx) * g.Hq + head);
+  if (n == 0) {                                         // empty cache: zeros, log-sum-exp = -inf
+    if (row_valid) {
+      for (int d = 0; d < D; ++d) out[row_off * D + d] = 0.f;
+      if (lse_out) lse_out[row_off] = -INFINITY;
+    }
+    return;
+  }
+  // A wait that gave up in an earlier CTA marks the workspace; the rest of the grid leaves.
+  if (status_word && *reinterpret_cast<volatile int32_t*>(status_word + 2) != 0) return;
+  const int n_blocks = (n + kPfRows - 1) / kPfRows;
+
+  // Tiles start on a 1024-byte boundary (the period of the 128-byte swizzle, which the matrix
+  // descriptors assume).
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t sQ = base, sKP = base + kPfTileBytes, sV = base + 2 * kPfTileBytes;
+  const uint32_t bar_k = smem_u32(&s_bar[0]), bar_v = smem_u32(&s_bar[1]), bar_m = smem_u32(&s_bar[2]);
+
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 :: "r"(smem_u32(&s_tmem)), "r"(kPfTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  if (tid == 0) {
+    mbar_init(bar_k, 1); mbar_init(bar_v, 1); mbar_init(bar_m, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncwarp();
+  // Q rows of this tile into shared memory, K-major with the 128-byte swizzle.
+  {
+    const uint4* src = reinterpret_cast<const uint4*>(q + row_off * D);
+#pragma unroll
+    for (int c = 0; c < 16; ++c) {
+      const uint4 v = row_valid ? src[c] : make_uint4(0, 0, 0, 0);
+      st_shared16(sQ + (c >> 3) * kPfHalf + tid * 128 + (((c & 7) ^ (tid & 7)) << 4), v.x, v.y, v.z, v.w);
+    }
+  }
+  proxy_fence();
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = s_tmem;
+  const uint32_t t_row = tmem + ((uint32_t)(warp * 32) << 16);      // this warp's lane quarter
+
+  auto load_block = [&](int kb) {                       // thread 0 only
+    mbar_expect_tx(bar_k, kPfTileBytes);
+    tma_load_5d(sKP, &map_k, bar_k, 0, kb * kPfRows, h, l, b);
+    tma_load_5d(sKP + kPfHalf, &map_k, bar_k, 64, kb * kPfRows, h, l, b);
+    mbar_expect_tx(bar_v, kPfTileBytes);
+    tma_load_5d(sV, &map_v, bar_v, 0, kb * kPfRows, h, l, b);
+    tma_load_5d(sV + kPfHalf, &map_v, bar_v, 64, kb * kPfRows, h, l, b);
+  };
+  if (tid == 0) load_block(0);
+  __syncwarp();
+
+  float o[D];
+#pragma unroll
+  for (int d = 0; d < D; ++d) o[d] = 0.f;
+  float m_run = -INFINITY, l_run = 0.f;
+  __shared__ int s_fail;
+  if (tid == 0) s_fail = 0;
+  uint32_t mma_phase = 0;
+
+  for (int kb = 0; kb < n_blocks; ++kb) {
+    const int valid = min(kPfRows, n - kb * kPfRows);   // valid tokens of this block
+    // ---- S = Q K^T ---------------------------------------------------------------------
+    if (tid == 0) {
+      if (!mbar_wait<kPfPolls>(bar_k, kb & 1)) s_fail = 1;
+      tc_fence_after();
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const uint32_t off = (k >> 2) * kPfHalf + (k & 3) * 32;
+        umma_bf16(tmem, umma_desc(sQ + off, 16, 1024), umma_desc(sKP + off, 16, 1024), kIdescQK, k > 0);
+      }
+      umma_commit(bar_m);
+      if (!mbar_wait<kPfPolls>(bar_m, mma_phase)) s_fail = 1;
+    }
+    mma_phase ^= 1;
+    __syncthreads();                                    // S is complete (thread 0 saw the commit)
+    if (s_fail) break;
+    tc_fence_after();
+    // ---- softmax of this thread's row ------------------------------------------------------
+    float bmax = -INFINITY;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      uint32_t r[32];
+      tmem_ld32(t_row + c * 32, r);
+#pragma unroll
+      for (int i = 0; i < 32; ++i)
+        if (c * 32 + i < valid) bmax = fmaxf(bmax, __uint_as_float(r[i]) * scale_log2e);
+    }
+    const float m_new = fmaxf(m_run, bmax);
+    const float alpha = exp2f(m_run - m_new);           // 0 on the first block
+    float rowsum = 0.f;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      uint32_t r[32];
+      tmem_ld32(t_row + c * 32, r);
+      uint32_t pk[16];
+#pragma unroll
+      for (int i = 0; i < 32; i += 2) {
+        const float p0 = c * 32 + i < valid ? exp2f(__uint_as_float(r[i]) * scale_log2e - m_new) : 0.f;
+        const float p1 = c * 32 + i + 1 < valid ? exp2f(__uint_as_float(r[i + 1]) * scale_log2e - m_new) : 0.f;
+        rowsum += p0 + p1;
+        pk[i >> 1] = pack_bf16(p0, p1);
+      }
+      // tokens 32c .. 32c+31 of row tid: four 16-byte pieces of the K-major swizzled P tile
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int ch = c * 4 + j;                       // piece index 0..15 along the tokens
+        st_shared16(sKP + (ch >> 3) * kPfHalf + tid * 128 + (((ch & 7) ^ (tid & 7)) << 4),
+                    pk[4 * j], pk[4 * j + 1], pk[4 * j + 2], pk[4 * j + 3]);
+      }
+    }
+    l_run = l_run * alpha + rowsum;
+    m_run = m_new;
+    // ---- O_blk = P V -----------------------------------------------------------------------
+    if (tid == 0 && !mbar_wait<kPfPolls>(bar_v, kb & 1)) s_fail = 1;
+    __syncthreads();                                    // V landed (thread 0 saw it)
+    if (s_fail) break;
+    if (valid < kPfRows && tid >= valid) {
+      // Rows past the valid length hold whatever the cache holds there: clear them so that a
+      // zero weight times Inf/NaN cannot reach the accumulators.
+#pragma unroll
+      for (int c = 0; c < 16; ++c) st_shared16(sV + (c >> 3) * kPfHalf + tid * 128 + ((c & 7) << 4), 0, 0, 0, 0);
+    }
+    proxy_fence();                                      // P (and cleared rows) visible to the MMA
+    tc_fence_before();
+    __syncthreads();
+    if (tid == 0) {
+      tc_fence_after();
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        umma_bf16(tmem + 128, umma_desc(sKP + (k >> 2) * kPfHalf + (k & 3) * 32, 16, 1024),
+                  umma_desc(sV + k * 2048, kPfHalf, 1024), kIdescPV, k > 0);
+      }
+      umma_commit(bar_m);
+      if (!mbar_wait<kPfPolls>(bar_m, mma_phase)) s_fail = 1;
+      else if (kb + 1 < n_blocks) load_block(kb + 1);   // both buffers are free again
+    }
+    mma_phase ^= 1;
+    __syncthreads();                                    // O_blk is complete
+    if (s_fail) break;
+    tc_fence_after();
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      uint32_t r[32];
+      tmem_ld32(t_row + 128 + c * 32, r);
+#pragma unroll
+      for (int i = 0; i < 32; ++i) o[c * 32 + i] = fmaf(o[c * 32 + i], alpha, __uint_as_float(r[i]));
+    }
+    tc_fence_before();
+    __syncthreads();                                    // tensor memory free for the next block
+  }
+
+  const bool failed = s_fail != 0;
+  if (row_valid && !failed) {
+    const float inv = 1.f / l_run;
+    float4* dst = reinterpret_cast<float4*>(out + row_off * D);
+#pragma unroll
+    for (int d = 0; d < D; d += 4) dst[d >> 2] = make_float4(o[d] * inv, o[d + 1] * inv, o[d + 2] * inv, o[d + 3] * inv);
+    if (lse_out) lse_out[row_off] = (m_run + log2f(l_run)) * 0.6931471805599453f;
+  }
+  if (failed && tid == 0 && status_word) {
+    atomicExch(status_word, (int)L2KV_ERR_CUDA);
+    atomicExch(status_word + 2, 1);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0)
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem), "r"(kPfTmemCols)
+                 : "memory");
+}
+
+template <int G>
+static int launch_pf(const void* q, const void* K, const void* V, const Geom& g, int n_queries,
+                     const int32_t* cur_len_dev, int max_len, float scale, float* out,
+                     float* lse_out, int32_t* status_word, cudaStream_t s) {
+  constexpr int QT = kPfRows / G;
+  const long long units = (long long)g.B * g.L * g.H;
+  const long long blocks = units * ((n_queries + QT - 1) / QT);
+  if (blocks == 0) return L2KV_OK;
+  if (blocks > 0x7fffffffLL) return L2KV_ERR_OUT_OF_RANGE;
+  alignas(64) CUtensorMap map_k, map_v;
+  std::memset(&map_k, 0, sizeof map_k);
+  std::memset(&map_v, 0, sizeof map_v);
+  if (!make_cache_map(&map_k, K, g, kPfRows) || !make_cache_map(&map_v, V, g, kPfRows))
+    return L2KV_ERR_UNSUPPORTED;
+  constexpr int smem_bytes = 1024 + 3 * kPfTileBytes;
+  auto kern = prefix_attention_kernel<G>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) != cudaSuccess)
+    return L2KV_ERR_CUDA;
+  kern<<<(unsigned)blocks, kPfThreads, smem_bytes, s>>>(
+      static_cast<const __nv_bfloat16*>(q), g, n_queries, cur_len_dev, max_len, scale * kPfLog2e, out,
+      lse_out, map_k, map_v, status_word);
+  return cudaGetLastError() == cudaSuccess ? L2KV_OK : L2KV_ERR_CUDA;
+}
+
+int launch_prefix_attention(const void* q, const void* K, const void* V, const Geom& g, int dtype,
+                            int n_queries, const int32_t* cur_len_dev, int max_len, float scale,
+                            float* out, float* lse_out, int32_t* status_word, cudaStream_t s) {
+  if (dtype != L2KV_BF16 || g.D != 128) return L2KV_ERR_UNSUPPORTED;
+  switch (g.Hq / g.H) {
+    case 1: return launch_pf<1>(q, K, V, g, n_queries, cur_len_dev, max_len, scale, out, lse_out, status_word, s);
+    case 2: return launch_pf<2>(q, K, V, g, n_queries, cur_len_dev, max_len, scale, out, lse_out, status_word, s);
+    case 4: return launch_pf<4>(q, K, V, g, n_queries, cur_len_dev, max_len, scale, out, lse_out, status_word, s);
+    case 8: return launch_pf<8>(q, K, V, g, n_queries, cur_len_dev, max_len, scale, out, lse_out, status_word, s);
+  }
+  return L2KV_ERR_UNSUPPORTED;
+}
+
+}  // namespace l2kv
