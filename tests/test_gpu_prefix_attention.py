@@ -1,0 +1,66 @@
+"""GPU parity of prefix attention (several new queries over the compressed cache; tensor-core
+contractions) against the oracle's single-query attention applied query by query."""
+import numpy as np
+import pytest
+import scipy.special
+import torch
+
+import oracle
+import synth
+from gpu_util import DEV, i32, assert_attention_close, gpu_attention
+
+pytestmark = pytest.mark.gpu
+
+
+def make_queries(w, n_q, seed):
+    g = torch.Generator().manual_seed(seed)
+    return torch.randn((w.B, w.L, n_q, w.Hq, w.D), generator=g).to(torch.bfloat16).to(DEV)
+
+
+def run(l2, q, K, V, cur, max_len, scale=0.0):
+    out = torch.full(q.shape, float("nan"), dtype=torch.float32, device=DEV)
+    lse = torch.full(q.shape[:4], float("nan"), dtype=torch.float32, device=DEV)
+    ws = torch.zeros(256, dtype=torch.uint8, device=DEV)
+    l2.prefix_attention(q, K, V, i32(np.asarray(cur)), max_len, out, lse, scale=scale, workspace=ws)
+    torch.cuda.synchronize()
+    assert l2.read_device_status(ws) == 0
+    return out.cpu().numpy(), lse.cpu().numpy()
+
+
+@pytest.mark.parametrize("Hkv,Hq,n_q,T", [(2, 8, 40, 300), (2, 2, 130, 257), (1, 8, 1, 1000),
+                                          (2, 4, 64, 128)])
+def test_prefix_attention_matches_oracle(Hkv, Hq, n_q, T):
+    import paper_2406_11430_b200 as l2
+    w = synth.WORKLOADS[2].scaled(B=2, L=2, Hkv=Hkv, Hq=Hq, T=T)
+    K, V = synth.make_cache(w, DEV)
+    q = make_queries(w, n_q, 3)
+    cur = np.array([[T, 128], [0, min(T, 129)]], dtype=np.int32)
+    out, lse = run(l2, q, K, V, cur, T)
+    Kn, Vn = synth.to_numpy(K), synth.to_numpy(V)
+    G = Hq // Hkv
+    for s in range(n_q):
+        want = oracle.attention(synth.to_numpy(q[:, :, s].contiguous()), Kn, Vn, "bf16", cur, nthreads=8)
+        assert_attention_close(out[:, :, s], want)
+    assert not out[1, 0].any() and np.all(np.isneginf(lse[1, 0]))          # empty cache
+    # log-sum-exp against a library routine on a few rows
+    qf, Kf = q.float().cpu().numpy().astype(np.float64), K.float().cpu().numpy().astype(np.float64)
+    for (b, l, s, j) in [(0, 0, 0, 0), (0, 1, n_q - 1, Hq - 1), (1, 1, n_q // 2, Hq // 2)]:
+        z = Kf[b, l, j // G, :cur[b, l]] @ qf[b, l, s, j] / np.sqrt(w.D)
+        np.testing.assert_allclose(lse[b, l, s, j], scipy.special.logsumexp(z), rtol=1e-5, atol=1e-4)
+
+
+def test_prefix_attention_agrees_with_decode_and_ignores_rows_past_the_length():
+    import paper_2406_11430_b200 as l2
+    w = synth.WORKLOADS[2].scaled(B=1, L=2, T=700)
+    K, V = synth.make_cache(w, DEV)
+    q = make_queries(w, 5, 9)
+    cur = np.array([[700, 333]], dtype=np.int32)
+    out, _ = run(l2, q, K, V, cur, 700, scale=0.07)
+    for s in range(5):
+        dec = gpu_attention(l2, q[:, :, s].contiguous(), K, V, cur, scale=0.07)
+        np.testing.assert_allclose(out[:, :, s], dec, rtol=1e-2, atol=2e-3)
+    Kp, Vp = K.clone(), V.clone()
+    Kp[0, 1, :, 333:] = float("nan")
+    Vp[0, 1, :, 333:] = float("inf")
+    out2, _ = run(l2, q, Kp, Vp, cur, 700, scale=0.07)
+    assert np.array_equal(out, out2)
