@@ -160,7 +160,7 @@ prefix_attention_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n_queri
   float o[D];
 #pragma unroll
   for (int d = 0; d < D; ++d) o[d] = 0.f;
-  float m_run = -INFINITY, l_run = 0.f;
+  float m_run = -INFINITY, l_run = 0.f, l_exact = 0.f;   // sums of rounded / unrounded weights
   __shared__ int s_fail;
   if (tid == 0) s_fail = 0;
   uint32_t mma_phase = 0;
@@ -195,7 +195,7 @@ prefix_attention_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n_queri
     }
     const float m_new = fmaxf(m_run, bmax);
     const float alpha = exp2f(m_run - m_new);           // 0 on the first block
-    float rowsum = 0.f;
+    float rowsum = 0.f, rowsum_exact = 0.f;
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
       uint32_t r[32];
@@ -205,8 +205,12 @@ prefix_attention_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n_queri
       for (int i = 0; i < 32; i += 2) {
         const float p0 = c * 32 + i < valid ? exp2f(__uint_as_float(r[i]) * scale_log2e - m_new) : 0.f;
         const float p1 = c * 32 + i + 1 < valid ? exp2f(__uint_as_float(r[i + 1]) * scale_log2e - m_new) : 0.f;
-        rowsum += p0 + p1;
-        pk[i >> 1] = pack_bf16(p0, p1);
+        const __nv_bfloat162 pr = __floats2bfloat162_rn(p0, p1);
+        // The sum is taken over the rounded weights, the ones V is multiplied with, so that
+        // numerator and denominator stay consistent (a dominant token still gives its V row).
+        rowsum += __low2float(pr) + __high2float(pr);
+        rowsum_exact += p0 + p1;
+        pk[i >> 1] = *reinterpret_cast<const uint32_t*>(&pr);
       }
       // tokens 32c .. 32c+31 of row tid: four 16-byte pieces of the K-major swizzled P tile
 #pragma unroll
@@ -217,6 +221,7 @@ prefix_attention_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n_queri
       }
     }
     l_run = l_run * alpha + rowsum;
+    l_exact = l_exact * alpha + rowsum_exact;
     m_run = m_new;
     // ---- O_blk = P V -----------------------------------------------------------------------
     if (tid == 0 && !mbar_wait<kPfPolls>(bar_v, kb & 1)) s_fail = 1;
@@ -263,7 +268,7 @@ prefix_attention_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n_queri
     float4* dst = reinterpret_cast<float4*>(out + row_off * D);
 #pragma unroll
     for (int d = 0; d < D; d += 4) dst[d >> 2] = make_float4(o[d] * inv, o[d + 1] * inv, o[d + 2] * inv, o[d + 3] * inv);
-    if (lse_out) lse_out[row_off] = (m_run + log2f(l_run)) * 0.6931471805599453f;
+    if (lse_out) lse_out[row_off] = (m_run + log2f(l_exact)) * 0.6931471805599453f;
   }
   if (failed && tid == 0 && status_word) {
     atomicExch(status_word, (int)L2KV_ERR_CUDA);

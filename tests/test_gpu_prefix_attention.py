@@ -1,5 +1,10 @@
 """GPU parity of prefix attention (several new queries over the compressed cache; tensor-core
-contractions) against the oracle's single-query attention applied query by query."""
+contractions) against the oracle's single-query attention applied query by query.
+
+Tolerance: the softmax weights are rounded to bf16 before they multiply V (relative error
+up to 2^-9 per weight, the FlashAttention arrangement), on top of the decode path's bf16
+inputs / fp32 accumulation; the absolute term is therefore 4e-3 instead of 2e-3, the relative
+term stays 1e-2, and the RMS error is bounded separately."""
 import numpy as np
 import pytest
 import scipy.special
@@ -40,7 +45,8 @@ def test_prefix_attention_matches_oracle(Hkv, Hq, n_q, T):
     G = Hq // Hkv
     for s in range(n_q):
         want = oracle.attention(synth.to_numpy(q[:, :, s].contiguous()), Kn, Vn, "bf16", cur, nthreads=8)
-        assert_attention_close(out[:, :, s], want)
+        assert_attention_close(out[:, :, s], want, atol=4e-3)
+        assert np.sqrt(np.mean((out[:, :, s] - want) ** 2)) <= 3e-3 * max(np.sqrt(np.mean(want ** 2)), 0.05)
     assert not out[1, 0].any() and np.all(np.isneginf(lse[1, 0]))          # empty cache
     # log-sum-exp against a library routine on a few rows
     qf, Kf = q.float().cpu().numpy().astype(np.float64), K.float().cpu().numpy().astype(np.float64)
