@@ -3,11 +3,11 @@
 // 4 * Sq * Hq * D flop per cached token per (b, l) -- so it runs on the Blackwell tensor cores
 // (tcgen05.mma, operands in shared memory, accumulators in tensor memory).
 //
-// One CTA (128 threads) per (b, l, kv head, tile of 128 / G queries): its 128 rows are the
+// One CTA (256 threads, two per row) per (b, l, kv head, tile of 128 / G queries): its 128 rows are the
 // (query, head-of-the-group) pairs that share one KV head.  Per block of 128 cached tokens:
 //   K block  -- TMA --> shared memory (128-byte swizzle)
 //   S = Q . K^T            8 x tcgen05.mma (M 128, N 128, K 16), fp32 in tensor memory
-//   thread r reads row r of S (tcgen05.ld): running maximum, weights 2^(s - m) as bf16 back
+//   the two threads of row r read it from S (tcgen05.ld): running maximum, weights 2^(s - m) as bf16 back
 //   to shared memory (over the K block, which is no longer needed), running sum
 //   V block  -- TMA --> shared memory;  O_blk = P . V   8 x tcgen05.mma (V as an N-major operand)
 //   thread r reads row r of O_blk and folds it into its fp32 accumulator row (rescaled by
@@ -20,7 +20,7 @@
 
 namespace l2kv {
 
-constexpr int kPfThreads = 128;
+constexpr int kPfThreads = 256;                // two threads per query row
 constexpr int kPfRows = 128;                    // query rows per CTA, cached tokens per block
 constexpr int kPfHalf = kPfRows * 128;          // one [128 rows][64 bf16] swizzled tile: 16 KB
 constexpr int kPfTileBytes = 2 * kPfHalf;       // both halves of the head dimension: 32 KB
@@ -78,6 +78,13 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<const uint32_t*>(&v);
 }
 
+// 2^x by the hardware approximation (one MUFU instruction; x <= 0 here, -inf gives 0).
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
 template <int G>
 __global__ void __launch_bounds__(kPfThreads, 2)
 prefix_attention_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n_queries,
@@ -90,6 +97,8 @@ prefix_attention_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n_queri
   extern __shared__ unsigned char smem_raw[];
   __shared__ __align__(8) unsigned long long s_bar[3];  // K landed, V landed, MMA done
   __shared__ uint32_t s_tmem;
+  __shared__ int s_fail;
+  __shared__ float s_x[2][kPfRows];                     // row maxima / sums of the two column halves
 
   const int q_tiles = (n_queries + QT - 1) / QT;
   const int qt = blockIdx.x % q_tiles;
@@ -98,15 +107,18 @@ prefix_attention_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n_queri
   const long long bl = unit / g.H;
   const int l = (int)(bl % g.L), b = (int)(bl / g.L);
   const int n = max(0, min(cur_len_dev[bl], min(max_len, g.t_cap)));
+  // Two threads per query row: thread (row, hf) owns score columns and output dims
+  // [64 hf, 64 hf + 64).  Warps w and w + 4 share a tensor-memory lane quarter.
   const int tid = threadIdx.x, warp = tid >> 5;
-  const int s_idx = qt * QT + tid / G;                  // this thread's query and head
-  const int head = h * G + tid % G;
+  const int row = tid & (kPfRows - 1), hf = tid >> 7;
+  const int s_idx = qt * QT + row / G;                  // this row's query and head
+  const int head = h * G + row % G;
   const bool row_valid = s_idx < n_queries;
   const long long row_off = ((bl * n_queries + s_idx) * g.Hq + head);
   if (n == 0) {                                         // empty cache: zeros, log-sum-exp = -inf
     if (row_valid) {
-      for (int d = 0; d < D; ++d) out[row_off * D + d] = 0.f;
-      if (lse_out) lse_out[row_off] = -INFINITY;
+      for (int d = 0; d < 64; ++d) out[row_off * D + hf * 64 + d] = 0.f;
+      if (lse_out && hf == 0) lse_out[row_off] = -INFINITY;
     }
     return;
   }
@@ -128,15 +140,17 @@ prefix_attention_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n_queri
   if (tid == 0) {
     mbar_init(bar_k, 1); mbar_init(bar_v, 1); mbar_init(bar_m, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    s_fail = 0;
   }
   __syncwarp();
-  // Q rows of this tile into shared memory, K-major with the 128-byte swizzle.
+  // Q rows of this tile into shared memory, K-major with the 128-byte swizzle (this thread:
+  // the eight 16-byte pieces of half hf of its row).
   {
-    const uint4* src = reinterpret_cast<const uint4*>(q + row_off * D);
+    const uint4* src = reinterpret_cast<const uint4*>(q + row_off * D) + hf * 8;
 #pragma unroll
-    for (int c = 0; c < 16; ++c) {
+    for (int c = 0; c < 8; ++c) {
       const uint4 v = row_valid ? src[c] : make_uint4(0, 0, 0, 0);
-      st_shared16(sQ + (c >> 3) * kPfHalf + tid * 128 + (((c & 7) ^ (tid & 7)) << 4), v.x, v.y, v.z, v.w);
+      st_shared16(sQ + hf * kPfHalf + row * 128 + ((c ^ (row & 7)) << 4), v.x, v.y, v.z, v.w);
     }
   }
   proxy_fence();
@@ -144,7 +158,7 @@ prefix_attention_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n_queri
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = s_tmem;
-  const uint32_t t_row = tmem + ((uint32_t)(warp * 32) << 16);      // this warp's lane quarter
+  const uint32_t t_row = tmem + ((uint32_t)((warp & 3) * 32) << 16) + hf * 64;   // lane quarter, column half
 
   auto load_block = [&](int kb) {                       // thread 0 only
     mbar_expect_tx(bar_k, kPfTileBytes);
@@ -157,16 +171,14 @@ prefix_attention_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n_queri
   if (tid == 0) load_block(0);
   __syncwarp();
 
-  float o[D];
+  float o[64];
 #pragma unroll
-  for (int d = 0; d < D; ++d) o[d] = 0.f;
-  float m_run = -INFINITY, l_run = 0.f, l_exact = 0.f;   // sums of rounded / unrounded weights
-  __shared__ int s_fail;
-  if (tid == 0) s_fail = 0;
+  for (int d = 0; d < 64; ++d) o[d] = 0.f;
+  float m_run = -INFINITY, l_run = 0.f, l_exact = 0.f;  // sums (of this half) of rounded / unrounded weights
   uint32_t mma_phase = 0;
 
   for (int kb = 0; kb < n_blocks; ++kb) {
-    const int valid = min(kPfRows, n - kb * kPfRows);   // valid tokens of this block
+    const int valid = min(kPfRows, n - kb * kPfRows) - hf * 64;   // valid tokens among this thread's 64
     // ---- S = Q K^T ---------------------------------------------------------------------
     if (tid == 0) {
       if (!mbar_wait<kPfPolls>(bar_k, kb & 1)) s_fail = 1;
@@ -183,28 +195,30 @@ prefix_attention_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n_queri
     __syncthreads();                                    // S is complete (thread 0 saw the commit)
     if (s_fail) break;
     tc_fence_after();
-    // ---- softmax of this thread's row ------------------------------------------------------
+    // ---- softmax of this thread's half row -------------------------------------------------
     float bmax = -INFINITY;
 #pragma unroll
-    for (int c = 0; c < 4; ++c) {
+    for (int c = 0; c < 2; ++c) {
       uint32_t r[32];
       tmem_ld32(t_row + c * 32, r);
 #pragma unroll
       for (int i = 0; i < 32; ++i)
-        if (c * 32 + i < valid) bmax = fmaxf(bmax, __uint_as_float(r[i]) * scale_log2e);
+        if (c * 32 + i < valid) bmax = fmaxf(bmax, __uint_as_float(r[i]));
     }
-    const float m_new = fmaxf(m_run, bmax);
-    const float alpha = exp2f(m_run - m_new);           // 0 on the first block
+    s_x[hf][row] = bmax * scale_log2e;                  // scale > 0: the maximum commutes with it
+    __syncthreads();
+    const float m_new = fmaxf(m_run, fmaxf(s_x[0][row], s_x[1][row]));
+    const float alpha = fast_exp2(m_run - m_new);       // 0 on the first block
     float rowsum = 0.f, rowsum_exact = 0.f;
 #pragma unroll
-    for (int c = 0; c < 4; ++c) {
+    for (int c = 0; c < 2; ++c) {
       uint32_t r[32];
       tmem_ld32(t_row + c * 32, r);
       uint32_t pk[16];
 #pragma unroll
       for (int i = 0; i < 32; i += 2) {
-        const float p0 = c * 32 + i < valid ? exp2f(__uint_as_float(r[i]) * scale_log2e - m_new) : 0.f;
-        const float p1 = c * 32 + i + 1 < valid ? exp2f(__uint_as_float(r[i + 1]) * scale_log2e - m_new) : 0.f;
+        const float p0 = c * 32 + i < valid ? fast_exp2(fmaf(__uint_as_float(r[i]), scale_log2e, -m_new)) : 0.f;
+        const float p1 = c * 32 + i + 1 < valid ? fast_exp2(fmaf(__uint_as_float(r[i + 1]), scale_log2e, -m_new)) : 0.f;
         const __nv_bfloat162 pr = __floats2bfloat162_rn(p0, p1);
         // The sum is taken over the rounded weights, the ones V is multiplied with, so that
         // numerator and denominator stay consistent (a dominant token still gives its V row).
@@ -212,11 +226,11 @@ prefix_attention_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n_queri
         rowsum_exact += p0 + p1;
         pk[i >> 1] = *reinterpret_cast<const uint32_t*>(&pr);
       }
-      // tokens 32c .. 32c+31 of row tid: four 16-byte pieces of the K-major swizzled P tile
+      // tokens 64 hf + 32 c .. + 31 of this row: four 16-byte pieces of the swizzled P tile
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        const int ch = c * 4 + j;                       // piece index 0..15 along the tokens
-        st_shared16(sKP + (ch >> 3) * kPfHalf + tid * 128 + (((ch & 7) ^ (tid & 7)) << 4),
+        const int ch = c * 4 + j;                       // piece index 0..7 inside half hf
+        st_shared16(sKP + hf * kPfHalf + row * 128 + ((ch ^ (row & 7)) << 4),
                     pk[4 * j], pk[4 * j + 1], pk[4 * j + 2], pk[4 * j + 3]);
       }
     }
@@ -227,11 +241,11 @@ prefix_attention_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n_queri
     if (tid == 0 && !mbar_wait<kPfPolls>(bar_v, kb & 1)) s_fail = 1;
     __syncthreads();                                    // V landed (thread 0 saw it)
     if (s_fail) break;
-    if (valid < kPfRows && tid >= valid) {
+    if (row >= min(kPfRows, n - kb * kPfRows)) {
       // Rows past the valid length hold whatever the cache holds there: clear them so that a
       // zero weight times Inf/NaN cannot reach the accumulators.
 #pragma unroll
-      for (int c = 0; c < 16; ++c) st_shared16(sV + (c >> 3) * kPfHalf + tid * 128 + ((c & 7) << 4), 0, 0, 0, 0);
+      for (int c = 0; c < 8; ++c) st_shared16(sV + hf * kPfHalf + row * 128 + (c << 4), 0, 0, 0, 0);
     }
     proxy_fence();                                      // P (and cleared rows) visible to the MMA
     tc_fence_before();
@@ -252,7 +266,7 @@ prefix_attention_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n_queri
     if (s_fail) break;
     tc_fence_after();
 #pragma unroll
-    for (int c = 0; c < 4; ++c) {
+    for (int c = 0; c < 2; ++c) {
       uint32_t r[32];
       tmem_ld32(t_row + 128 + c * 32, r);
 #pragma unroll
@@ -263,12 +277,21 @@ prefix_attention_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n_queri
   }
 
   const bool failed = s_fail != 0;
+  // the two halves of a row share the maximum; their weight sums add up
+  __syncthreads();
+  s_x[hf][row] = l_run;
+  __syncthreads();
+  const float l_tot = s_x[0][row] + s_x[1][row];
+  __syncthreads();
+  s_x[hf][row] = l_exact;
+  __syncthreads();
+  const float l_tot_exact = s_x[0][row] + s_x[1][row];
   if (row_valid && !failed) {
-    const float inv = 1.f / l_run;
-    float4* dst = reinterpret_cast<float4*>(out + row_off * D);
+    const float inv = 1.f / l_tot;
+    float4* dst = reinterpret_cast<float4*>(out + row_off * D + hf * 64);
 #pragma unroll
-    for (int d = 0; d < D; d += 4) dst[d >> 2] = make_float4(o[d] * inv, o[d + 1] * inv, o[d + 2] * inv, o[d + 3] * inv);
-    if (lse_out) lse_out[row_off] = (m_run + log2f(l_exact)) * 0.6931471805599453f;
+    for (int d = 0; d < 64; d += 4) dst[d >> 2] = make_float4(o[d] * inv, o[d + 1] * inv, o[d + 2] * inv, o[d + 3] * inv);
+    if (lse_out && hf == 0) lse_out[row_off] = (m_run + log2f(l_tot_exact)) * 0.6931471805599453f;
   }
   if (failed && tid == 0 && status_word) {
     atomicExch(status_word, (int)L2KV_ERR_CUDA);
