@@ -464,9 +464,9 @@ def oracle_sample_step(w, seed_shift=0, n_dec=2, n_comp=1, nthreads=None):
 
 def cpu_baseline(w, target_s=15.0):
     """The oracle, as it stands, on the host cores: a sample sized to about target_s seconds."""
-    probe, _, _, _ = oracle_sample_step(w, n_dec=4, n_comp=1)
-    per_layer_full = max(probe, 1e-3) * w.decode_steps / 4.0     # one (unc + comp) pair, all steps
-    n_comp = int(max(1, min(w.L - len(w.uncompressed), 12, round(target_s / per_layer_full))))
+    probe, _, _, _ = oracle_sample_step(w, n_dec=w.decode_steps, n_comp=1)   # one layer pair, all steps
+    # the uncompressed layer of the pair costs about two compressed ones (twice the rows)
+    n_comp = int(max(1, min(w.L - len(w.uncompressed), round(3 * target_s / max(probe, 1e-3) - 2))))
     dt, nbytes, nthreads, layers = oracle_sample_step(w, n_dec=w.decode_steps, n_comp=n_comp)
     return {"value": round(nbytes / dt / 1e9, 4), "unit": "GB/s", "cores": nthreads,
             "kind": "oracle", "seconds": round(dt, 2),
