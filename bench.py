@@ -301,6 +301,7 @@ def run_gpu(args):
         line["e2e"] = e2e
     if not args.no_cpu_baseline and world == 1:
         line["cpu_baseline"] = cpu_baseline(w, target_s=args.cpu_seconds)
+        line["tie_band"] = tie_band_report(job, w)
     print(json.dumps(line))
 
 
@@ -473,6 +474,35 @@ def cpu_baseline(w, target_s=15.0):
             "sample": f"sequence 0, layers {layers} (first one uncompressed), all {w.Hkv} KV "
                       f"heads, full {w.T}-token context: one compression pass + "
                       f"{w.decode_steps} decode steps"}
+
+
+def tie_band_report(job, w, n_units=6, band=1e-6):
+    """Part of the CPU leg: the kept sets of a few compressed units against the oracle's fp64
+    selection.  Tokens may differ only where the fp64 norm lies within `band` (relative) of the
+    unit's threshold norm; such swaps are counted, anything else is reported as a mismatch."""
+    import oracle
+    job.compress()
+    torch.cuda.synchronize()
+    comp = [l for l in range(w.L) if l not in job.unc]
+    if not comp:
+        return {"units_checked": 0, "swaps_inside_band": 0, "mismatches_outside_band": 0, "band": band}
+    swaps = bad = 0
+    for i in range(n_units):
+        b, l, h = i % w.B, comp[(i * 7) % len(comp)], (i * 3) % w.Hkv
+        n_in, keep = int(job.lens_host[b]), int(job.keep_host[b])
+        Kn = synth.to_numpy(job.K[b, l, h, :n_in])[None, None, None]
+        key = oracle.key_sumsq(Kn, w.dtype)[0, 0, 0]
+        want = set(oracle.select(key, keep).tolist())
+        got = set(job.idx[b, l, h, :keep].cpu().tolist())
+        norm = np.sqrt(key)
+        thr = np.sort(norm)[keep - 1]
+        for t in got ^ want:
+            if abs(norm[t] - thr) <= band * thr:
+                swaps += 1
+            else:
+                bad += 1
+    return {"units_checked": n_units, "swaps_inside_band": swaps // 2,
+            "mismatches_outside_band": bad, "band": band}
 
 
 def run_reference(args):
