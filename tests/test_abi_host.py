@@ -82,3 +82,31 @@ def test_validation_rejects_before_launch():
     with pytest.raises(l2.L2KVError) as e:          # null output
         l2.decode_attention(_fake((1, 2, 4, 128)), K, K, kl, 128, None, ws)
     assert e.value.status == -1
+
+
+def test_validation_of_the_analysis_and_prefix_entry_points():
+    K = _fake((1, 2, 4, 128, 128))
+    kl = torch.zeros((1, 2), dtype=torch.int32)
+    q = _fake((1, 2, 5, 8, 128))
+    out = _fake((1, 2, 5, 8, 128), torch.float32)
+    with pytest.raises(l2.L2KVError) as e:          # fp32 caches are not served by the tensor-core path
+        l2.prefix_attention(q.float(), K.float(), K.float(), kl, 128, out)
+    assert e.value.status == -2
+    with pytest.raises(l2.L2KVError) as e:          # max_len beyond t_cap
+        l2.prefix_attention(q, K, K, kl, 129, out)
+    assert e.value.status == -5
+    with pytest.raises(l2.L2KVError) as e:          # 12 query heads over 4 KV heads
+        l2.prefix_attention(_fake((1, 2, 5, 12, 128)), K, K, kl, 128, out)
+    assert e.value.status == -2
+    with pytest.raises(l2.L2KVError) as e:          # status workspace too small
+        l2.prefix_attention(q, K, K, kl, 128, out, workspace=_fake((16,), torch.uint8))
+    assert e.value.status == -4
+    sumsq = _fake((1, 2, 4, 128), torch.float32)
+    alr = _fake((1, 2, 8), torch.float32)
+    qd = _fake((1, 2, 8, 128))
+    with pytest.raises(l2.L2KVError) as e:          # workspace too small for the sorts
+        l2.attention_loss(qd, K, kl, 128, sumsq, alr, workspace=_fake((1024,), torch.uint8))
+    assert e.value.status == -4
+    with pytest.raises(l2.L2KVError) as e:          # keys are required
+        l2.attention_loss(qd, K, kl, 128, None, alr, workspace=_fake((1 << 20,), torch.uint8))
+    assert e.value.status == -1
