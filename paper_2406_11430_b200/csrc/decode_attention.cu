@@ -633,7 +633,9 @@ static int launch_dec_g(const void* q, const void* K, const void* V, const Geom&
     case 1: return launch_dec_t<T, D, 1>(q, K, V, g, cur_len_dev, max_len, scale, out, ws, plan, s);
     case 2: return launch_dec_t<T, D, 2>(q, K, V, g, cur_len_dev, max_len, scale, out, ws, plan, s);
     case 4: return launch_dec_t<T, D, 4>(q, K, V, g, cur_len_dev, max_len, scale, out, ws, plan, s);
+#if L2KV_DECODE_CHUNK <= 1024   /* the score buffer of 8 heads x a longer split exceeds static shared memory */
     case 8: return launch_dec_t<T, D, 8>(q, K, V, g, cur_len_dev, max_len, scale, out, ws, plan, s);
+#endif
   }
   return L2KV_ERR_UNSUPPORTED;
 }
