@@ -11,9 +11,15 @@
 
 namespace l2kv {
 
-constexpr int kNormThreads = 256;
+#ifndef L2KV_NORM_THREADS
+#define L2KV_NORM_THREADS 256
+#endif
+#ifndef L2KV_NORM_ROWS
+#define L2KV_NORM_ROWS 1024
+#endif
+constexpr int kNormThreads = L2KV_NORM_THREADS;
 constexpr int kNormUnroll = 8;                 // rows per thread per step, all loads in flight
-constexpr int kNormRowsPerCta = 1024;
+constexpr int kNormRowsPerCta = L2KV_NORM_ROWS;
 
 template <typename T, int D, int MODE>
 __global__ void __launch_bounds__(kNormThreads)

@@ -30,7 +30,8 @@ template <int NT>
 __device__ void select_unit(SelectSmem& sm, const float* __restrict__ key, int len, int keep,
                             int policy, uint32_t flags, UnitRec* __restrict__ rec,
                             int2* __restrict__ crec) {
-  constexpr int kBatch = 16;                     // independent key loads in flight per thread
+  constexpr int kBatch = 8;                      // independent key loads in flight per thread
+  const bool vec = (reinterpret_cast<uintptr_t>(key) & 15u) == 0;   // caller-provided keys may not be
   const int tid = threadIdx.x;
   const int my_chunks = (len + kGatherChunk - 1) / kGatherChunk;
   uint32_t prefix = 0, mask = 0;
@@ -60,17 +61,41 @@ __device__ void select_unit(SelectSmem& sm, const float* __restrict__ key, int l
       const int n_cand = sm.n_cand;
       for (int i = tid; i < n_cand; i += NT) tally(sm.cand[i]);
     } else {
-      for (int base = 0; base < len; base += NT * kBatch) {
-        uint32_t kb[kBatch];
+      auto visit = [&](uint32_t kb) {
+        if (tally(kb) && collect) sm.cand[atomicAdd(&sm.n_cand, 1)] = kb;
+      };
+      if (vec) {
+        // 16-byte loads, kBatch of them in flight per thread: the pass is bound by how many
+        // bytes one CTA keeps outstanding towards L2.
+        const int n4 = len >> 2;
+        const float4* key4 = reinterpret_cast<const float4*>(key);
+        for (int base = 0; base < n4; base += NT * kBatch) {
+          float4 v[kBatch];
 #pragma unroll
-        for (int j = 0; j < kBatch; ++j) {
-          const int t = base + j * NT + tid;
-          kb[j] = t < len ? load_key_bits(key + t, policy) : 0u;
+          for (int j = 0; j < kBatch; ++j) {
+            const int i = base + j * NT + tid;
+            v[j] = i < n4 ? __ldcg(key4 + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+          }
+#pragma unroll
+          for (int j = 0; j < kBatch; ++j) {
+            if (base + j * NT + tid < n4) {
+              visit(order_bits(v[j].x, policy)); visit(order_bits(v[j].y, policy));
+              visit(order_bits(v[j].z, policy)); visit(order_bits(v[j].w, policy));
+            }
+          }
         }
+        if (tid < (len & 3)) visit(load_key_bits(key + (n4 << 2) + tid, policy));
+      } else {
+        for (int base = 0; base < len; base += NT * kBatch) {
+          uint32_t kb[kBatch];
 #pragma unroll
-        for (int j = 0; j < kBatch; ++j) {
-          const int t = base + j * NT + tid;
-          if (t < len && tally(kb[j]) && collect) sm.cand[atomicAdd(&sm.n_cand, 1)] = kb[j];
+          for (int j = 0; j < kBatch; ++j) {
+            const int t = base + j * NT + tid;
+            kb[j] = t < len ? load_key_bits(key + t, policy) : 0u;
+          }
+#pragma unroll
+          for (int j = 0; j < kBatch; ++j)
+            if (base + j * NT + tid < len) visit(kb[j]);
         }
       }
     }
@@ -118,11 +143,20 @@ __device__ void select_unit(SelectSmem& sm, const float* __restrict__ key, int l
     const int t0 = c * kGatherChunk;
     const int t1 = min(len, t0 + kGatherChunk);
     int nl = 0, ne = 0;
+    auto count = [&](uint32_t kb) { nl += kb < thr; ne += kb == thr; };
+    if (vec && t1 == t0 + kGatherChunk) {
+      const float4* key4 = reinterpret_cast<const float4*>(key + t0);
+      float4 v[kGatherChunk / 128];
+#pragma unroll
+      for (int j = 0; j < kGatherChunk / 128; ++j) v[j] = __ldcg(key4 + j * 32 + lane);
+#pragma unroll
+      for (int j = 0; j < kGatherChunk / 128; ++j) {
+        count(order_bits(v[j].x, policy)); count(order_bits(v[j].y, policy));
+        count(order_bits(v[j].z, policy)); count(order_bits(v[j].w, policy));
+      }
+    } else {
 #pragma unroll 4
-    for (int t = t0 + lane; t < t1; t += 32) {
-      const uint32_t kb = load_key_bits(key + t, policy);
-      nl += kb < thr;
-      ne += kb == thr;
+      for (int t = t0 + lane; t < t1; t += 32) count(load_key_bits(key + t, policy));
     }
 #pragma unroll
     for (int off = 16; off >= 1; off >>= 1) {
