@@ -57,7 +57,36 @@ append_evict_kernel(T* __restrict__ K, T* __restrict__ V, int32_t* __restrict__ 
       const int32_t* pos = idx + unit * g.t_cap;
       unsigned long long best = 0ull;
       int best_j = -1;
-      for (int j0 = 0; j0 < n; j0 += kAppendThreads * kAppendUnroll) {
+      auto consider = [&](uint32_t kb, uint32_t pb, int j) {
+        const unsigned long long c = ((unsigned long long)kb << 32) | pb;
+        if (best_j < 0 || c > best) { best = c; best_j = j; }
+      };
+      int j_done = 0;
+      if (((reinterpret_cast<uintptr_t>(key) | reinterpret_cast<uintptr_t>(pos)) & 15u) == 0) {
+        // 16-byte loads of four (key, position) pairs, kAppendUnroll of them in flight per thread
+        const int n4 = n >> 2;
+        const uint4* key4 = reinterpret_cast<const uint4*>(key);
+        const uint4* pos4 = reinterpret_cast<const uint4*>(pos);
+        for (int i0 = 0; i0 < n4; i0 += kAppendThreads * kAppendUnroll) {
+          uint4 kv[kAppendUnroll], pv[kAppendUnroll];
+#pragma unroll
+          for (int u = 0; u < kAppendUnroll; ++u) {
+            const int i = i0 + u * kAppendThreads + tid;
+            kv[u] = i < n4 ? key4[i] : make_uint4(0, 0, 0, 0);
+            pv[u] = i < n4 ? pos4[i] : make_uint4(0, 0, 0, 0);
+          }
+#pragma unroll
+          for (int u = 0; u < kAppendUnroll; ++u) {
+            const int i = i0 + u * kAppendThreads + tid;
+            if (i < n4) {
+              consider(kv[u].x, pv[u].x, 4 * i); consider(kv[u].y, pv[u].y, 4 * i + 1);
+              consider(kv[u].z, pv[u].z, 4 * i + 2); consider(kv[u].w, pv[u].w, 4 * i + 3);
+            }
+          }
+        }
+        j_done = n4 << 2;
+      }
+      for (int j0 = j_done; j0 < n; j0 += kAppendThreads * kAppendUnroll) {
         uint32_t kb[kAppendUnroll], pb[kAppendUnroll];
 #pragma unroll
         for (int u = 0; u < kAppendUnroll; ++u) {
@@ -68,8 +97,7 @@ append_evict_kernel(T* __restrict__ K, T* __restrict__ V, int32_t* __restrict__ 
 #pragma unroll
         for (int u = 0; u < kAppendUnroll; ++u) {
           const int j = j0 + u * kAppendThreads + tid;
-          const unsigned long long c = ((unsigned long long)kb[u] << 32) | pb[u];
-          if (j < n && (best_j < 0 || c > best)) { best = c; best_j = j; }
+          if (j < n) consider(kb[u], pb[u], j);
         }
       }
       unsigned long long wbest = best;
