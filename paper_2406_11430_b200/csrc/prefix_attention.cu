@@ -14,6 +14,7 @@
 //   2^(m_old - m_new)), FlashAttention style.
 // Every wait on an mbarrier is bounded (a wait that gives up ends the CTA's loop and marks
 // the status word); tensor memory is released on every path.
+#include <cstdlib>
 #include <cstring>
 
 #include "async_copy.cuh"
@@ -65,6 +66,28 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
                : "r"(taddr));
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
+// A operand taken from tensor memory (bf16 pairs packed two per 32-bit column, row = lane).
+__device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc,
+                                             uint32_t idesc, uint32_t accumulate) {
+  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+               "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+               :: "r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u)
+               : "memory");
+}
+// Stores 32 consecutive 32-bit columns of this thread's tensor-memory lane.  Whole warps only.
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+               "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+               "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+               :: "r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]),
+                  "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]),
+                  "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]),
+                  "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]),
+                  "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+               : "memory");
+}
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void proxy_fence() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
@@ -304,6 +327,246 @@ prefix_attention_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n_queri
                  : "memory");
 }
 
+// Second formulation of the same kernel, the one the entry point uses: the weights never go
+// to shared memory.  They are written as bf16 pairs into the tensor-memory columns that held
+// the scores and feed the second contraction from there (tcgen05.mma with A in tensor
+// memory), the output accumulates in tensor memory across blocks and is rescaled only when
+// a row's maximum has grown by more than 2^8 since the last rescale (weights stay <= 2^8, well
+// inside bf16 / fp32 range), and K and V each have their own shared-memory tile, so the next
+// K block is fetched while the softmax and the second contraction of the current one run.
+constexpr float kPfRescaleGap = 8.f;            // log2 units a maximum may drift before O is rescaled
+
+template <int G>
+__global__ void __launch_bounds__(kPfThreads, 2)
+prefix_attention_kernel_v2(const __nv_bfloat16* __restrict__ q, Geom g, int n_queries,
+                           const int32_t* __restrict__ cur_len_dev, int max_len, float scale_log2e,
+                           float* __restrict__ out, float* __restrict__ lse_out,
+                           const __grid_constant__ CUtensorMap map_k,
+                           const __grid_constant__ CUtensorMap map_v,
+                           int32_t* __restrict__ status_word) {
+  constexpr int D = 128;
+  constexpr int QT = kPfRows / G;                       // queries per CTA
+  extern __shared__ unsigned char smem_raw[];
+  __shared__ __align__(8) unsigned long long s_bar[4];  // K landed, V landed, QK done, PV done
+  __shared__ uint32_t s_tmem;
+  __shared__ int s_fail;
+  __shared__ float s_x[2][kPfRows];                     // row maxima / sums of the two column halves
+
+  const int q_tiles = (n_queries + QT - 1) / QT;
+  const int qt = blockIdx.x % q_tiles;
+  const long long unit = blockIdx.x / q_tiles;          // (b * L + l) * H + h
+  const int h = (int)(unit % g.H);
+  const long long bl = unit / g.H;
+  const int l = (int)(bl % g.L), b = (int)(bl / g.L);
+  const int n = max(0, min(cur_len_dev[bl], min(max_len, g.t_cap)));
+  // Two threads per query row: thread (row, hf) owns score columns and output dims
+  // [64 hf, 64 hf + 64).  Warps w and w + 4 share a tensor-memory lane quarter.
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const int row = tid & (kPfRows - 1), hf = tid >> 7;
+  const int s_idx = qt * QT + row / G;                  // this row's query and head
+  const int head = h * G + row % G;
+  const bool row_valid = s_idx < n_queries;
+  const long long row_off = ((bl * n_queries + s_idx) * g.Hq + head);
+  if (n == 0) {                                         // empty cache: zeros, log-sum-exp = -inf
+    if (row_valid) {
+      for (int d = 0; d < 64; ++d) out[row_off * D + hf * 64 + d] = 0.f;
+      if (lse_out && hf == 0) lse_out[row_off] = -INFINITY;
+    }
+    return;
+  }
+  // A wait that gave up in an earlier CTA marks the workspace; the rest of the grid leaves.
+  if (status_word && *reinterpret_cast<volatile int32_t*>(status_word + 2) != 0) return;
+  const int n_blocks = (n + kPfRows - 1) / kPfRows;
+
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;   // 1024-byte aligned tiles
+  const uint32_t sQ = base, sK = base + kPfTileBytes, sV = base + 2 * kPfTileBytes;
+  const uint32_t bar_k = smem_u32(&s_bar[0]), bar_v = smem_u32(&s_bar[1]);
+  const uint32_t bar_s = smem_u32(&s_bar[2]), bar_o = smem_u32(&s_bar[3]);
+
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 :: "r"(smem_u32(&s_tmem)), "r"(kPfTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  if (tid == 0) {
+    mbar_init(bar_k, 1); mbar_init(bar_v, 1); mbar_init(bar_s, 1); mbar_init(bar_o, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    s_fail = 0;
+  }
+  __syncwarp();
+  {                                                     // Q rows, K-major, 128-byte swizzle
+    const uint4* src = reinterpret_cast<const uint4*>(q + row_off * D) + hf * 8;
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+      const uint4 v = row_valid ? src[c] : make_uint4(0, 0, 0, 0);
+      st_shared16(sQ + hf * kPfHalf + row * 128 + ((c ^ (row & 7)) << 4), v.x, v.y, v.z, v.w);
+    }
+  }
+  proxy_fence();
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = s_tmem;
+  const uint32_t t_lane = tmem + ((uint32_t)((warp & 3) * 32) << 16);   // this warp's lane quarter
+  const uint32_t t_s = t_lane + hf * 64;                // scores of this thread's 64 tokens
+  const uint32_t t_p = t_lane + hf * 32;                // their weights, two per column
+  const uint32_t t_o = t_lane + 128 + hf * 64;          // this thread's 64 output dims
+
+  auto load_k = [&](int kb) {                           // thread 0 only
+    mbar_expect_tx(bar_k, kPfTileBytes);
+    tma_load_5d(sK, &map_k, bar_k, 0, kb * kPfRows, h, l, b);
+    tma_load_5d(sK + kPfHalf, &map_k, bar_k, 64, kb * kPfRows, h, l, b);
+  };
+  auto load_v = [&](int kb) {
+    mbar_expect_tx(bar_v, kPfTileBytes);
+    tma_load_5d(sV, &map_v, bar_v, 0, kb * kPfRows, h, l, b);
+    tma_load_5d(sV + kPfHalf, &map_v, bar_v, 64, kb * kPfRows, h, l, b);
+  };
+  if (tid == 0) { load_k(0); load_v(0); }
+  __syncwarp();
+
+  float m_ref = -INFINITY, l_run = 0.f, l_exact = 0.f;  // reference maximum; sums of this half's weights
+
+  for (int kb = 0; kb < n_blocks; ++kb) {
+    const int valid_all = min(kPfRows, n - kb * kPfRows);   // valid tokens of this block
+    const int valid = valid_all - hf * 64;                   // ... among this thread's 64
+    // ---- S = Q K^T; fetch V for this block and K for the next as their tiles come free ---
+    if (tid == 0) {
+      if (!mbar_wait<kPfPolls>(bar_k, kb & 1)) s_fail = 1;
+      tc_fence_after();
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const uint32_t off = (k >> 2) * kPfHalf + (k & 3) * 32;
+        umma_bf16(tmem, umma_desc(sQ + off, 16, 1024), umma_desc(sK + off, 16, 1024), kIdescQK, k > 0);
+      }
+      umma_commit(bar_s);
+      if (kb > 0) {                                      // P.V of the previous block is done:
+        if (!mbar_wait<kPfPolls>(bar_o, (kb - 1) & 1)) s_fail = 1;   // O is quiet, the V tile is free
+        else load_v(kb);
+      }
+      if (!mbar_wait<kPfPolls>(bar_s, kb & 1)) s_fail = 1;
+      else if (kb + 1 < n_blocks) load_k(kb + 1);        // the K tile is free again
+    }
+    __syncthreads();                                     // S is complete (thread 0 saw the commit)
+    if (s_fail) break;
+    tc_fence_after();
+    // ---- this thread's 64 scores (log2 domain), kept in registers ---------------------------
+    float sv[64];
+    float bmax = -INFINITY;
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+      uint32_t r[32];
+      tmem_ld32(t_s + c * 32, r);
+#pragma unroll
+      for (int i = 0; i < 32; ++i) {
+        sv[c * 32 + i] = c * 32 + i < valid ? __uint_as_float(r[i]) * scale_log2e : -INFINITY;
+        bmax = fmaxf(bmax, sv[c * 32 + i]);
+      }
+    }
+    s_x[hf][row] = bmax;
+    tc_fence_before();
+    __syncthreads();                                     // maxima exchanged; every score has been read
+    tc_fence_after();
+    const float m_new = fmaxf(m_ref, fmaxf(s_x[0][row], s_x[1][row]));
+    if (kb == 0) m_ref = m_new;
+    // ---- rescale O only when this row's maximum has drifted far from the reference ----------
+    const bool need = m_new > m_ref + kPfRescaleGap;
+    if (__any_sync(0xffffffffu, need)) {
+      const float factor = need ? fast_exp2(m_ref - m_new) : 1.f;
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        uint32_t r[32];
+        tmem_ld32(t_o + c * 32, r);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * factor);
+        tmem_st32(t_o + c * 32, r);
+      }
+      tmem_wait_st();
+      if (need) { l_run *= factor; l_exact *= factor; m_ref = m_new; }
+    }
+    // ---- weights 2^(s - m_ref) as bf16 pairs over the score columns -------------------------
+    {
+      uint32_t pk[32];
+      float rowsum = 0.f, rowsum_exact = 0.f;
+#pragma unroll
+      for (int i = 0; i < 64; i += 2) {
+        const float p0 = fast_exp2(sv[i] - m_ref), p1 = fast_exp2(sv[i + 1] - m_ref);   // -inf -> 0
+        const __nv_bfloat162 pr = __floats2bfloat162_rn(p0, p1);
+        // the normalising sum uses the rounded weights, the ones V is multiplied with
+        rowsum += __low2float(pr) + __high2float(pr);
+        rowsum_exact += p0 + p1;
+        pk[i >> 1] = *reinterpret_cast<const uint32_t*>(&pr);
+      }
+      tmem_st32(t_p, pk);
+      tmem_wait_st();
+      l_run += rowsum;
+      l_exact += rowsum_exact;
+    }
+    if (valid_all < kPfRows) {
+      // Last, partial block: rows of the V tile past the valid length hold whatever the cache
+      // holds there; clear them so that a zero weight times Inf/NaN cannot reach O.
+      if (tid == 0 && !mbar_wait<kPfPolls>(bar_v, kb & 1)) s_fail = 1;
+      __syncthreads();
+      if (row >= valid_all) {
+#pragma unroll
+        for (int c = 0; c < 8; ++c) st_shared16(sV + hf * kPfHalf + row * 128 + (c << 4), 0, 0, 0, 0);
+      }
+      proxy_fence();
+    }
+    tc_fence_before();
+    __syncthreads();                                     // all weights are in tensor memory
+    // ---- O += P V ----------------------------------------------------------------------------
+    if (tid == 0) {
+      if (valid_all == kPfRows && !mbar_wait<kPfPolls>(bar_v, kb & 1)) s_fail = 1;
+      tc_fence_after();
+#pragma unroll
+      for (int k = 0; k < 8; ++k)
+        umma_bf16_ts(tmem + 128, tmem + k * 8, umma_desc(sV + k * 2048, kPfHalf, 1024), kIdescPV,
+                     (kb > 0 || k > 0) ? 1u : 0u);
+      umma_commit(bar_o);
+    }
+  }
+
+  if (tid == 0 && !s_fail && !mbar_wait<kPfPolls>(bar_o, (n_blocks - 1) & 1)) s_fail = 1;
+  __syncthreads();                                       // O is complete
+  tc_fence_after();
+  const bool failed = s_fail != 0;
+  // the two halves of a row share the reference maximum; their weight sums add up
+  s_x[hf][row] = l_run;
+  __syncthreads();
+  const float l_tot = s_x[0][row] + s_x[1][row];
+  __syncthreads();
+  s_x[hf][row] = l_exact;
+  __syncthreads();
+  const float l_tot_exact = s_x[0][row] + s_x[1][row];
+  if (!failed) {
+    const float inv = 1.f / l_tot;
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+      uint32_t r[32];
+      tmem_ld32(t_o + c * 32, r);
+      if (row_valid) {
+        float4* dst = reinterpret_cast<float4*>(out + row_off * D + hf * 64 + c * 32);
+#pragma unroll
+        for (int i = 0; i < 32; i += 4)
+          dst[i >> 2] = make_float4(__uint_as_float(r[i]) * inv, __uint_as_float(r[i + 1]) * inv,
+                                    __uint_as_float(r[i + 2]) * inv, __uint_as_float(r[i + 3]) * inv);
+      }
+    }
+    if (row_valid && lse_out && hf == 0)
+      lse_out[row_off] = (m_ref + log2f(l_tot_exact)) * 0.6931471805599453f;
+  }
+  if (failed && tid == 0 && status_word) {
+    atomicExch(status_word, (int)L2KV_ERR_CUDA);
+    atomicExch(status_word + 2, 1);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0)
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem), "r"(kPfTmemCols)
+                 : "memory");
+}
+
 template <int G>
 static int launch_pf(const void* q, const void* K, const void* V, const Geom& g, int n_queries,
                      const int32_t* cur_len_dev, int max_len, float scale, float* out,
@@ -319,7 +582,10 @@ static int launch_pf(const void* q, const void* K, const void* V, const Geom& g,
   if (!make_cache_map(&map_k, K, g, kPfRows) || !make_cache_map(&map_v, V, g, kPfRows))
     return L2KV_ERR_UNSUPPORTED;
   constexpr int smem_bytes = 1024 + 3 * kPfTileBytes;
-  auto kern = prefix_attention_kernel<G>;
+  // L2KV_PREFIX_KERNEL=v1 selects the first formulation (weights through shared memory).
+  const char* which = std::getenv("L2KV_PREFIX_KERNEL");
+  const bool v1 = which && std::strcmp(which, "v1") == 0;
+  auto kern = v1 ? prefix_attention_kernel<G> : prefix_attention_kernel_v2<G>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) != cudaSuccess)
     return L2KV_ERR_CUDA;
   kern<<<(unsigned)blocks, kPfThreads, smem_bytes, s>>>(
