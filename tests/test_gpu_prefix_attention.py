@@ -55,8 +55,11 @@ def test_prefix_attention_matches_oracle(Hkv, Hq, n_q, T):
         np.testing.assert_allclose(lse[b, l, s, j], scipy.special.logsumexp(z), rtol=1e-5, atol=1e-4)
 
 
-def test_prefix_attention_agrees_with_decode_and_ignores_rows_past_the_length():
+@pytest.mark.parametrize("kernel", ["v2", "v1"])
+def test_prefix_attention_agrees_with_decode_and_ignores_rows_past_the_length(kernel, monkeypatch):
+    # both formulations of the kernel (weights in tensor memory / through shared memory)
     import paper_2406_11430_b200 as l2
+    monkeypatch.setenv("L2KV_PREFIX_KERNEL", kernel)
     w = synth.WORKLOADS[2].scaled(B=1, L=2, T=700)
     K, V = synth.make_cache(w, DEV)
     q = make_queries(w, 5, 9)
