@@ -83,11 +83,17 @@ def random_key(seed, unit, t):
 
 def compress(K, V, dtype, lens, keep, uncompressed=(), key_mode=0, policy=0, t_cap_out=None,
              nthreads=1, seed=0):
-    """Whole-cache compression.  Returns dict(K_c, V_c, idx, key, kept_len)."""
+    """Whole-cache compression.  Returns dict(K_c, V_c, idx, key, kept_len).  `keep` is [B],
+    or [B, L, H] for a keep count per head; kept_len is then [B, L, H] too."""
     _check(K, dtype)
     _check(V, dtype)
     B, L, H, T_cap, D = K.shape
     lens, keep, unc = _i32(lens), _i32(keep), _i32(list(uncompressed))
+    per_head = keep.ndim == 3
+    if per_head:
+        assert keep.shape == (B, L, H)
+        keep_unit, keep = keep, np.zeros(B, dtype=np.int32)
+        kept_len_unit = np.zeros((B, L, H), dtype=np.int32)
     if t_cap_out is None:
         t_cap_out = T_cap
     K_c = np.zeros((B, L, H, t_cap_out, D), dtype=K.dtype)
@@ -99,24 +105,32 @@ def compress(K, V, dtype, lens, keep, uncompressed=(), key_mode=0, policy=0, t_c
         _p(K), _p(V), _DT[dtype], B, L, H, T_cap, D, _p(lens), _p(keep), _p(unc), int(unc.size),
         int(key_mode), int(policy), ctypes.c_uint64(int(seed) & 0xFFFFFFFFFFFFFFFF), int(t_cap_out),
         _p(K_c), _p(V_c), _p(idx), _p(key),
-        _p(kept_len), int(nthreads))
+        _p(kept_len), _p(keep_unit) if per_head else None,
+        _p(kept_len_unit) if per_head else None, int(nthreads))
     if rc != 0:
         raise ValueError(f"oracle compress: bad argument ({rc})")
-    return dict(K_c=K_c, V_c=V_c, idx=idx, key=key, kept_len=kept_len)
+    return dict(K_c=K_c, V_c=V_c, idx=idx, key=key,
+                kept_len=kept_len_unit if per_head else kept_len)
 
 
 def attention(q, K_c, V_c, dtype, cur_len, scale=0.0, nthreads=1):
-    """Decode attention, fp64 two-pass softmax.  q [B, L, Hq, D] -> float64 [B, L, Hq, D]."""
+    """Decode attention, fp64 two-pass softmax.  q [B, L, Hq, D] -> float64 [B, L, Hq, D].
+    cur_len is [B, L], or [B, L, Hkv] for a length per KV head."""
     _check(q, dtype)
     _check(K_c, dtype)
     _check(V_c, dtype)
     B, L, Hkv, T_cap, D = K_c.shape
     Hq = q.shape[2]
-    cur_len = _i32(cur_len).reshape(B, L)
+    cur_len = _i32(cur_len)
+    per_head = cur_len.ndim == 3
+    if per_head:
+        cur_len_unit, cur_len = cur_len.reshape(B, L, Hkv), np.zeros((B, L), dtype=np.int32)
+    else:
+        cur_len = cur_len.reshape(B, L)
     out = np.empty((B, L, Hq, D), dtype=np.float64)
     rc = lib().l2kv_oracle_attention(
         _p(q), _p(K_c), _p(V_c), _DT[dtype], B, L, Hkv, Hq, T_cap, D, _p(cur_len),
-        ctypes.c_double(scale), _p(out), int(nthreads))
+        ctypes.c_double(scale), _p(out), _p(cur_len_unit) if per_head else None, int(nthreads))
     if rc != 0:
         raise ValueError(f"oracle attention: bad argument ({rc})")
     return out

@@ -213,28 +213,48 @@ int32_t l2kv_oracle_keep_count(int32_t len, double keep_ratio) {
 //               lowest seeded random keys of unit (b * L + l) * H + h (`seed`)
 //   outputs     K_out, V_out [B, L, H, T_cap_out, D] (rows >= kept_len untouched),
 //               idx_out int32, key_out double [B, L, H, T_cap_out], kept_len [B, L]
+//   keep_unit   optional [B, L, H]: a keep count of its own for every head (the per-head
+//               ratios that the paper's discussion of future work names); it replaces
+//               keep[b] in compressed layers, and kept_len_unit [B, L, H] then receives
+//               every unit's length (kept_len holds head 0's)
 // Returns 0, or -1 if an argument is out of range.
 int l2kv_oracle_compress(const void* K, const void* V, int dtype, int B, int L, int H, int T_cap,
                          int D, const int32_t* len, const int32_t* keep,
                          const int32_t* uncompressed, int n_unc, int key_mode, int policy,
                          uint64_t seed, int T_cap_out, void* K_out, void* V_out, int32_t* idx_out,
-                         double* key_out, int32_t* kept_len, int nthreads) {
+                         double* key_out, int32_t* kept_len, const int32_t* keep_unit,
+                         int32_t* kept_len_unit, int nthreads) {
+  if (keep_unit != nullptr && kept_len_unit == nullptr) return -1;
   for (int b = 0; b < B; ++b) {
     if (len[b] < 0 || len[b] > T_cap) return -1;
-    if (keep[b] < 0 || keep[b] > len[b]) return -1;
-    if (keep[b] > T_cap_out) return -1;
+    if (keep_unit == nullptr) {
+      if (keep[b] < 0 || keep[b] > len[b]) return -1;
+      if (keep[b] > T_cap_out) return -1;
+    } else {
+      for (int64_t u = int64_t(b) * L * H; u < int64_t(b + 1) * L * H; ++u)
+        if (keep_unit[u] < 0 || keep_unit[u] > len[b] || keep_unit[u] > T_cap_out) return -1;
+    }
     if (n_unc > 0 && len[b] > T_cap_out) return -1;
   }
   const int es = elem_size(dtype);
+  std::vector<int32_t> unit_keep_store(size_t(B) * L * H);
+  int32_t* unit_keep = unit_keep_store.data();
   for (int b = 0; b < B; ++b)
     for (int l = 0; l < L; ++l)
-      kept_len[b * L + l] = in_list(uncompressed, n_unc, l) ? len[b] : keep[b];
+      for (int h = 0; h < H; ++h) {
+        const int64_t u = (int64_t(b) * L + l) * H + h;
+        unit_keep[u] = in_list(uncompressed, n_unc, l) ? len[b]
+                       : keep_unit != nullptr          ? keep_unit[u]
+                                                       : keep[b];
+        if (kept_len_unit != nullptr) kept_len_unit[u] = unit_keep[u];
+        if (h == 0) kept_len[b * L + l] = unit_keep[u];
+      }
 
   for_each_unit(int64_t(B) * L * H, nthreads, [=](int64_t u) {
     const int b = static_cast<int>(u / (int64_t(L) * H));
     const int l = static_cast<int>((u / H) % L);
     const int T = len[b];
-    const int n_keep = kept_len[b * L + l];
+    const int n_keep = unit_keep[u];
     const int64_t in_row0 = u * T_cap;        // first row of this unit, in rows
     const int64_t out_row0 = u * T_cap_out;
     std::vector<double> key(T);
@@ -267,17 +287,18 @@ int l2kv_oracle_compress(const void* K, const void* V, int dtype, int B, int L, 
 // Query head j reads KV head j / (Hq / Hkv) (reading: contiguous grouping; the
 // paper cites grouped-query attention without giving the mapping).  No mask:
 // a decode query sees every cached entry (Eq. 4).  scale <= 0 means
-// 1 / sqrt(D) (Eq. 2).  An empty cache gives zeros (reading).
+// 1 / sqrt(D) (Eq. 2).  An empty cache gives zeros (reading).  cur_len_unit, when not
+// null, is [B, L, Hkv] and replaces cur_len (caches compressed with per-head keep counts).
 int l2kv_oracle_attention(const void* q, const void* K_c, const void* V_c, int dtype, int B, int L,
                           int Hkv, int Hq, int T_cap, int D, const int32_t* cur_len, double scale,
-                          double* out, int nthreads) {
+                          double* out, const int32_t* cur_len_unit, int nthreads) {
   if (Hkv <= 0 || Hq % Hkv != 0) return -1;
   const int G = Hq / Hkv;
   const double sc = scale > 0.0 ? scale : 1.0 / std::sqrt(static_cast<double>(D));
   for_each_unit(int64_t(B) * L * Hq, nthreads, [=](int64_t u) {
     const int hq = static_cast<int>(u % Hq);
     const int64_t bl = u / Hq;
-    const int n = cur_len[bl];
+    const int n = cur_len_unit != nullptr ? cur_len_unit[bl * Hkv + hq / G] : cur_len[bl];
     const int64_t kv_row0 = (bl * Hkv + hq / G) * T_cap;
     double* o = out + u * D;
     for (int d = 0; d < D; ++d) o[d] = 0.0;

@@ -219,6 +219,35 @@ def test_ragged_lengths_and_per_sequence_keep():
         oracle.compress(K, V, "bf16", [300, 1, 1], [2, 2, 1])
 
 
+def test_per_head_keep_counts():
+    """A keep count per (b, l, h): every unit is the sort-and-cut of its own keys; the
+    uncompressed layer ignores the counts."""
+    w, K, V = _tiny("bf16", B=2, L=3, T=200)
+    lens = [200, 61]
+    rng = np.random.default_rng(11)
+    keep = np.stack([rng.integers(0, lens[b] + 1, size=(w.L, w.Hkv)) for b in range(2)])
+    keep[0, 0, 0], keep[1, 2, 1] = 0, 61                                   # empty and whole
+    r = oracle.compress(K, V, "bf16", lens, keep, uncompressed=(1,))
+    s = oracle.key_sumsq(K, "bf16")
+    assert r["kept_len"].shape == (2, w.L, w.Hkv)
+    for b, l, h in itertools.product(range(2), range(w.L), range(w.Hkv)):
+        n = lens[b] if l == 1 else keep[b, l, h]
+        assert r["kept_len"][b, l, h] == n
+        want = sorted(sorted(range(lens[b]), key=lambda t: (s[b, l, h, t], t))[:n])
+        assert r["idx"][b, l, h, :n].tolist() == want
+        assert np.all(r["idx"][b, l, h, n:] == -1)
+        assert np.array_equal(r["V_c"][b, l, h, :n], V[b, l, h, want])
+    # equal counts in every head are the per-sequence call
+    same = oracle.compress(K, V, "bf16", lens, np.broadcast_to(np.array([90, 30])[:, None, None],
+                                                               (2, w.L, w.Hkv)).copy())
+    ref = oracle.compress(K, V, "bf16", lens, [90, 30])
+    assert np.array_equal(same["idx"], ref["idx"]) and np.array_equal(same["K_c"], ref["K_c"])
+    bad = keep.copy()
+    bad[1, 0, 0] = 62
+    with pytest.raises(ValueError):
+        oracle.compress(K, V, "bf16", lens, bad)
+
+
 # ------------------------------------------------------------ a5: attention
 
 def _textbook_attention(q, K, V, G):
@@ -257,6 +286,24 @@ def test_attention_matches_textbook_and_gqa_mapping(dtype):
                                V[0, 0, :, :50].float().numpy(), 4)
     np.testing.assert_allclose(out2[0, 0], want, rtol=1e-11, atol=1e-13)
     assert not out2[0, 1].any()                                            # empty cache -> zeros
+
+
+def test_attention_with_a_length_per_kv_head():
+    w = synth.WORKLOADS[0].scaled(dtype="bf16", L=2, Hkv=2, Hq=8, T=200)
+    K, V = synth.make_cache(w, "cpu")
+    q = synth.make_query(w, 0, "cpu")
+    lens = np.array([[[200, 37], [0, 1]]])
+    out = oracle.attention(synth.to_numpy(q), synth.to_numpy(K), synth.to_numpy(V), "bf16", lens)
+    for l, h in itertools.product(range(2), range(2)):
+        n = lens[0, l, h]
+        got = out[0, l, 4 * h:4 * h + 4]
+        if n == 0:
+            assert not got.any()
+            continue
+        want = _textbook_attention(q[0, l, 4 * h:4 * h + 4].float().numpy(),
+                                   K[0, l, h:h + 1, :n].float().numpy(),
+                                   V[0, l, h:h + 1, :n].float().numpy(), 4)
+        np.testing.assert_allclose(got, want, rtol=1e-11, atol=1e-13)
 
 
 def test_keep_everything_reproduces_uncompressed_attention():
