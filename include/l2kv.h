@@ -145,6 +145,27 @@ int l2kv_decode_attention(const void* q, const void* K_c, const void* V_c, const
                           const int32_t* cur_len_dev, int32_t max_len, float scale, float* out,
                           void* workspace, size_t workspace_bytes, void* stream);
 
+/* A keep count of its own for every head -- the per-head compression ratios that the paper
+ * names as future work (Limitations section); the method itself uses one ratio for all
+ * heads.  l2kv_select_compact_per_head is l2kv_select_compact with keep_unit_dev dense
+ * int32 [batch, layers, kv_heads] in place of keep_dev (0 <= keep_unit_dev[b,l,h] <=
+ * len_dev[b]; layers in uncompressed_layers ignore it) and kept_len_unit_dev of the same
+ * shape in place of kept_len_dev.  l2kv_decode_attention_per_head is l2kv_decode_attention
+ * over rows i < cur_len_unit_dev[b,l,j/G] (dense int32 [batch, layers, kv_heads]).  All
+ * other arguments, layouts, ownership and errors are those of the per-sequence calls. */
+int l2kv_select_compact_per_head(const void* K, const void* V, const l2kv_layout* in,
+                                 const int32_t* len_dev, const int32_t* keep_unit_dev,
+                                 int32_t max_len, const int32_t* uncompressed_layers,
+                                 int32_t n_uncompressed, int32_t policy, uint64_t seed,
+                                 const float* sumsq_in, void* K_out, void* V_out,
+                                 const l2kv_layout* out, int32_t* idx_out, float* sumsq_out,
+                                 int32_t* kept_len_unit_dev, void* workspace,
+                                 size_t workspace_bytes, void* stream);
+int l2kv_decode_attention_per_head(const void* q, const void* K_c, const void* V_c,
+                                   const l2kv_layout* lay, const int32_t* cur_len_unit_dev,
+                                   int32_t max_len, float scale, float* out, void* workspace,
+                                   size_t workspace_bytes, void* stream);
+
 /* Budget-maintained cache (Section 4, "Language Modelling Tasks"): append one new
  * token per (b, l, h).  If l is uncompressed or cur_len_dev[b,l] < budget_dev[b] the
  * row is appended at slot cur_len and cur_len grows by one.  Otherwise the entry

@@ -52,7 +52,9 @@ def lib():
         L.l2kv_key_norms.argtypes = [vp, lay, vp, i32, vp, vp, vp]
         L.l2kv_select_compact.argtypes = [vp, vp, lay, vp, vp, i32, ctypes.POINTER(i32), i32, i32,
                                           ctypes.c_uint64, vp, vp, vp, lay, vp, vp, vp, vp, sz, vp]
+        L.l2kv_select_compact_per_head.argtypes = L.l2kv_select_compact.argtypes
         L.l2kv_decode_attention.argtypes = [vp, vp, vp, lay, vp, i32, ctypes.c_float, vp, vp, sz, vp]
+        L.l2kv_decode_attention_per_head.argtypes = L.l2kv_decode_attention.argtypes
         L.l2kv_append_evict.argtypes = [vp, vp, vp, vp, lay, vp, vp, ctypes.POINTER(i32), i32,
                                         vp, vp, vp, vp, sz, vp]
         L.l2kv_attention_loss_workspace_bytes.argtypes = [lay, i32, ctypes.POINTER(sz)]
@@ -63,7 +65,8 @@ def lib():
         for name in ("l2kv_prefix_attention", "l2kv_attention_loss_workspace_bytes", "l2kv_attention_loss",
                      "l2kv_keep_count", "l2kv_workspace_bytes", "l2kv_read_device_status",
                      "l2kv_key_norms", "l2kv_select_compact", "l2kv_decode_attention",
-                     "l2kv_append_evict"):
+                     "l2kv_append_evict", "l2kv_select_compact_per_head",
+                     "l2kv_decode_attention_per_head"):
             getattr(L, name).restype = ctypes.c_int
         _LIB = L
     return _LIB
@@ -154,6 +157,30 @@ def select_compact(K, V, len_dev, keep_dev, max_len, uncompressed_layers, K_out,
         _ptr(V_out), lout.ref(), _ptr(idx_out), _ptr(sumsq_out),
         _ptr(kept_len_dev), _ptr(workspace), workspace.numel(), _stream(stream)),
         "l2kv_select_compact")
+
+
+def select_compact_per_head(K, V, len_dev, keep_unit_dev, max_len, uncompressed_layers, K_out,
+                            V_out, idx_out, sumsq_out, kept_len_unit_dev, workspace,
+                            policy=KEEP_LOWEST_NORM, seed=0, sumsq_in=None, stream=None):
+    """select_compact with a keep count and a result length per (b, l, h)."""
+    lin, lout = Layout(K), Layout(K_out)
+    arr, n = _layers(uncompressed_layers)
+    _check(lib().l2kv_select_compact_per_head(
+        _ptr(K), _ptr(V), lin.ref(), _ptr(len_dev), _ptr(keep_unit_dev), int(max_len), arr, n,
+        int(policy), ctypes.c_uint64(int(seed) & 0xFFFFFFFFFFFFFFFF), _ptr(sumsq_in), _ptr(K_out),
+        _ptr(V_out), lout.ref(), _ptr(idx_out), _ptr(sumsq_out),
+        _ptr(kept_len_unit_dev), _ptr(workspace), workspace.numel(), _stream(stream)),
+        "l2kv_select_compact_per_head")
+
+
+def decode_attention_per_head(q, K_c, V_c, cur_len_unit_dev, max_len, out, workspace, scale=0.0,
+                              stream=None):
+    """decode_attention with a cache length per (b, l, kv head)."""
+    lay = Layout(K_c, q_heads=q.shape[2])
+    _check(lib().l2kv_decode_attention_per_head(
+        _ptr(q), _ptr(K_c), _ptr(V_c), lay.ref(), _ptr(cur_len_unit_dev), int(max_len),
+        float(scale), _ptr(out), _ptr(workspace), workspace.numel(), _stream(stream)),
+        "l2kv_decode_attention_per_head")
 
 
 def decode_attention(q, K_c, V_c, cur_len_dev, max_len, out, workspace, scale=0.0, stream=None):

@@ -107,13 +107,15 @@ int l2kv_key_norms(const void* K, const l2kv_layout* lay, const int32_t* len_dev
                           norm_out, kKeysOnly, nullptr, static_cast<cudaStream_t>(stream));
 }
 
-int l2kv_select_compact(const void* K, const void* V, const l2kv_layout* in,
-                        const int32_t* len_dev, const int32_t* keep_dev, int32_t max_len,
-                        const int32_t* uncompressed_layers, int32_t n_uncompressed, int32_t policy,
-                        uint64_t seed, const float* sumsq_in,
-                        void* K_out, void* V_out, const l2kv_layout* out, int32_t* idx_out,
-                        float* sumsq_out, int32_t* kept_len_dev, void* workspace,
-                        size_t workspace_bytes, void* stream) {
+// Both forms of the compression call: keep counts and result lengths per sequence
+// (per_head false: keep [B], kept_len [B, L]) or per head (keep and kept_len [B, L, H]).
+static int select_compact_impl(bool per_head, const void* K, const void* V, const l2kv_layout* in,
+                               const int32_t* len_dev, const int32_t* keep_dev, int32_t max_len,
+                               const int32_t* uncompressed_layers, int32_t n_uncompressed,
+                               int32_t policy, uint64_t seed, const float* sumsq_in, void* K_out,
+                               void* V_out, const l2kv_layout* out, int32_t* idx_out,
+                               float* sumsq_out, int32_t* kept_len_dev, void* workspace,
+                               size_t workspace_bytes, void* stream) {
   int rc = check_layout(in);
   if (rc != L2KV_OK) return rc;
   rc = check_layout(out);
@@ -140,15 +142,45 @@ int l2kv_select_compact(const void* K, const void* V, const l2kv_layout* in,
     return L2KV_ERR_MISALIGNED;
   const WorkspacePlan plan = plan_workspace(*in, max_len);
   if (workspace_bytes < plan.total) return L2KV_ERR_WORKSPACE_TOO_SMALL;
-  return launch_select_compact(K, V, make_geom(*in), in->dtype, len_dev, keep_dev, max_len, unc,
-                               policy, seed, sumsq_in, K_out, V_out, make_geom(*out), idx_out, sumsq_out,
-                               kept_len_dev, static_cast<char*>(workspace), plan,
+  return launch_select_compact(K, V, make_geom(*in), in->dtype, len_dev,
+                               per_head ? nullptr : keep_dev, per_head ? keep_dev : nullptr,
+                               max_len, unc, policy, seed, sumsq_in, K_out, V_out,
+                               make_geom(*out), idx_out, sumsq_out,
+                               per_head ? nullptr : kept_len_dev, per_head ? kept_len_dev : nullptr,
+                               static_cast<char*>(workspace), plan,
                                static_cast<cudaStream_t>(stream));
 }
 
-int l2kv_decode_attention(const void* q, const void* K_c, const void* V_c, const l2kv_layout* lay,
-                          const int32_t* cur_len_dev, int32_t max_len, float scale, float* out,
-                          void* workspace, size_t workspace_bytes, void* stream) {
+int l2kv_select_compact(const void* K, const void* V, const l2kv_layout* in,
+                        const int32_t* len_dev, const int32_t* keep_dev, int32_t max_len,
+                        const int32_t* uncompressed_layers, int32_t n_uncompressed, int32_t policy,
+                        uint64_t seed, const float* sumsq_in,
+                        void* K_out, void* V_out, const l2kv_layout* out, int32_t* idx_out,
+                        float* sumsq_out, int32_t* kept_len_dev, void* workspace,
+                        size_t workspace_bytes, void* stream) {
+  return select_compact_impl(false, K, V, in, len_dev, keep_dev, max_len, uncompressed_layers,
+                             n_uncompressed, policy, seed, sumsq_in, K_out, V_out, out, idx_out,
+                             sumsq_out, kept_len_dev, workspace, workspace_bytes, stream);
+}
+
+int l2kv_select_compact_per_head(const void* K, const void* V, const l2kv_layout* in,
+                                 const int32_t* len_dev, const int32_t* keep_unit_dev,
+                                 int32_t max_len, const int32_t* uncompressed_layers,
+                                 int32_t n_uncompressed, int32_t policy, uint64_t seed,
+                                 const float* sumsq_in, void* K_out, void* V_out,
+                                 const l2kv_layout* out, int32_t* idx_out, float* sumsq_out,
+                                 int32_t* kept_len_unit_dev, void* workspace,
+                                 size_t workspace_bytes, void* stream) {
+  return select_compact_impl(true, K, V, in, len_dev, keep_unit_dev, max_len,
+                             uncompressed_layers, n_uncompressed, policy, seed, sumsq_in, K_out,
+                             V_out, out, idx_out, sumsq_out, kept_len_unit_dev, workspace,
+                             workspace_bytes, stream);
+}
+
+static int decode_attention_impl(bool per_head, const void* q, const void* K_c, const void* V_c,
+                                 const l2kv_layout* lay, const int32_t* cur_len_dev,
+                                 int32_t max_len, float scale, float* out, void* workspace,
+                                 size_t workspace_bytes, void* stream) {
   int rc = check_layout(lay);
   if (rc != L2KV_OK) return rc;
   rc = check_groups(lay);
@@ -162,9 +194,25 @@ int l2kv_decode_attention(const void* q, const void* K_c, const void* V_c, const
   const WorkspacePlan plan = plan_workspace(*lay, max_len);
   if (workspace_bytes < plan.total) return L2KV_ERR_WORKSPACE_TOO_SMALL;
   const float sc = scale > 0.f ? scale : 1.0f / std::sqrt((float)lay->head_dim);
-  return launch_decode_attention(q, K_c, V_c, make_geom(*lay), lay->dtype, cur_len_dev, max_len, sc,
+  const LenView lens{cur_len_dev, per_head ? 1 : 0};
+  return launch_decode_attention(q, K_c, V_c, make_geom(*lay), lay->dtype, lens, max_len, sc,
                                  out, static_cast<char*>(workspace), plan,
                                  static_cast<cudaStream_t>(stream));
+}
+
+int l2kv_decode_attention(const void* q, const void* K_c, const void* V_c, const l2kv_layout* lay,
+                          const int32_t* cur_len_dev, int32_t max_len, float scale, float* out,
+                          void* workspace, size_t workspace_bytes, void* stream) {
+  return decode_attention_impl(false, q, K_c, V_c, lay, cur_len_dev, max_len, scale, out,
+                               workspace, workspace_bytes, stream);
+}
+
+int l2kv_decode_attention_per_head(const void* q, const void* K_c, const void* V_c,
+                                   const l2kv_layout* lay, const int32_t* cur_len_unit_dev,
+                                   int32_t max_len, float scale, float* out, void* workspace,
+                                   size_t workspace_bytes, void* stream) {
+  return decode_attention_impl(true, q, K_c, V_c, lay, cur_len_unit_dev, max_len, scale, out,
+                               workspace, workspace_bytes, stream);
 }
 
 int l2kv_append_evict(void* K_c, void* V_c, int32_t* idx, float* sumsq_c, const l2kv_layout* lay,

@@ -36,6 +36,16 @@ struct LayerMask {
   __host__ __device__ bool test(int l) const { return (w[l >> 5] >> (l & 31)) & 1u; }
 };
 
+// Valid lengths, one per (b, l) or, for caches compressed with a keep count per head, one
+// per (b, l, h).
+struct LenView {
+  const int32_t* p;
+  int per_head;
+  __device__ __forceinline__ int at(long long bl, int h, int H) const {
+    return p[per_head ? bl * H + h : bl];
+  }
+};
+
 inline Geom make_geom(const l2kv_layout& a) {
   Geom g;
   g.B = a.batch; g.L = a.layers; g.H = a.kv_heads; g.Hq = a.q_heads; g.D = a.head_dim;
@@ -186,26 +196,30 @@ __device__ __forceinline__ uint32_t order_bits(float sumsq, int policy) {
 // Arguments of the selection that the norm pass runs for each unit as its last chunk finishes.
 enum KeyMode { kKeysOnly = 0, kKeysFromK = 1, kKeysRandom = 2, kKeysGiven = 3 };
 struct SelectArgs {
-  const int32_t* keep_dev;
+  const int32_t* keep_dev;                    // [B], or null when keep_unit_dev is given
+  const int32_t* keep_unit_dev;               // [B, L, H] or null
+  int32_t* kept_len_unit_dev;                 // [B, L, H] or null
   int out_t_cap, policy, n_chunks;            // policy: how key bits order (lowest / highest)
   unsigned long long seed;                    // kKeysRandom
   LayerMask unc;
   UnitRec* unit_rec;
   int2* chunk_rec;
   int32_t* tickets;
-  int32_t* kept_len_dev;
+  int32_t* kept_len_dev;                      // [B, L] (head 0's length) or null
 };
 int launch_key_norms(const void* K, const Geom& g, int dtype, const int32_t* len_dev, int max_len,
                      float* sumsq, long long ld_sumsq, float* norm_out, int key_mode,
                      const SelectArgs* select, cudaStream_t s);
 int launch_select_compact(const void* K, const void* V, const Geom& gi, int dtype,
-                          const int32_t* len_dev, const int32_t* keep_dev, int max_len,
+                          const int32_t* len_dev, const int32_t* keep_dev,
+                          const int32_t* keep_unit_dev, int max_len,
                           const LayerMask& unc, int policy, unsigned long long seed,
                           const float* sumsq_in, void* K_out, void* V_out, const Geom& go,
-                          int32_t* idx_out, float* sumsq_out, int32_t* kept_len_dev, char* ws,
+                          int32_t* idx_out, float* sumsq_out, int32_t* kept_len_dev,
+                          int32_t* kept_len_unit_dev, char* ws,
                           const WorkspacePlan& plan, cudaStream_t s);
 int launch_decode_attention(const void* q, const void* K, const void* V, const Geom& g, int dtype,
-                            const int32_t* cur_len_dev, int max_len, float scale, float* out,
+                            const LenView& cur_len_dev, int max_len, float scale, float* out,
                             char* ws, const WorkspacePlan& plan, cudaStream_t s);
 int launch_append_evict(void* K, void* V, int32_t* idx, float* sumsq, const Geom& g, int dtype,
                         int32_t* cur_len_dev, const int32_t* budget_dev, const LayerMask& unc,

@@ -25,7 +25,7 @@ constexpr float kLog2e = 1.4426950408889634f;
 template <typename T, int D, int G>
 __global__ void __launch_bounds__(kDecThreads)
 decode_split_kernel(const T* __restrict__ q, const T* __restrict__ K, const T* __restrict__ V,
-                    Geom g, const int32_t* __restrict__ cur_len_dev, int max_len,
+                    Geom g, LenView cur_len_dev, int max_len,
                     float scale_log2e, float* __restrict__ partial, int n_splits) {
   constexpr int EPV = Elem<T>::kPerVec;
   constexpr int LPR = D / EPV;
@@ -42,7 +42,7 @@ decode_split_kernel(const T* __restrict__ q, const T* __restrict__ K, const T* _
   const long long bl = unit / g.H;
   const int l = (int)(bl % g.L);
   const int b = (int)(bl / g.L);
-  const int n = max(0, min(cur_len_dev[bl], min(max_len, g.t_cap)));
+  const int n = max(0, min(cur_len_dev.at(bl, h, g.H), min(max_len, g.t_cap)));
   const int t0 = split * kDecodeChunk;
   if (t0 >= n) return;
   const int t_end = min(n, t0 + kDecodeChunk);
@@ -198,11 +198,13 @@ decode_split_kernel(const T* __restrict__ q, const T* __restrict__ K, const T* _
 
 template <int D>
 __global__ void __launch_bounds__(D)
-decode_combine_kernel(const float* __restrict__ partial, const int32_t* __restrict__ cur_len_dev,
-                      int max_len, int t_cap, int Hq, int n_splits, float* __restrict__ out) {
+decode_combine_kernel(const float* __restrict__ partial, LenView cur_len_dev,
+                      int max_len, int t_cap, int H, int Hq, int n_splits,
+                      float* __restrict__ out) {
   const long long row = blockIdx.x;                      // (b * L + l) * Hq + hq
   const long long bl = row / Hq;
-  const int n = max(0, min(cur_len_dev[bl], min(max_len, t_cap)));
+  const int h = (int)(row % Hq) / (Hq / H);
+  const int n = max(0, min(cur_len_dev.at(bl, h, H), min(max_len, t_cap)));
   const int ns = (n + kDecodeChunk - 1) / kDecodeChunk;
   const int d = threadIdx.x;
   const float* p = partial + row * n_splits * (long long)(D + 2);
@@ -292,7 +294,7 @@ template <int G, bool TMA>
 __global__ void __launch_bounds__(kMmaThreads, L2KV_MMA_MIN_CTAS)
 decode_split_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ K,
                         const __nv_bfloat16* __restrict__ V, Geom g,
-                        const int32_t* __restrict__ cur_len_dev, int max_len, float scale_log2e,
+                        LenView cur_len_dev, int max_len, float scale_log2e,
                         float* __restrict__ partial, int n_splits,
                         const __grid_constant__ CUtensorMap map_k,
                         const __grid_constant__ CUtensorMap map_v, int32_t* __restrict__ status_word) {
@@ -315,7 +317,7 @@ decode_split_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16
   const long long bl = unit / g.H;
   const int l = (int)(bl % g.L);
   const int b = (int)(bl / g.L);
-  const int n = max(0, min(cur_len_dev[bl], min(max_len, g.t_cap)));
+  const int n = max(0, min(cur_len_dev.at(bl, h, g.H), min(max_len, g.t_cap)));
   const int t0 = split * kDecodeChunk;
   if (t0 >= n) return;
   if constexpr (TMA) {
@@ -574,7 +576,7 @@ decode_split_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16
 
 template <int G>
 static int launch_dec_mma(const void* q, const void* K, const void* V, const Geom& g,
-                          const int32_t* cur_len_dev, int max_len, float scale, float* out,
+                          const LenView& cur_len_dev, int max_len, float scale, float* out,
                           char* ws, const WorkspacePlan& plan, cudaStream_t s) {
   const long long units = (long long)g.B * g.L * g.H;
   if (units == 0) return L2KV_OK;
@@ -602,13 +604,13 @@ static int launch_dec_mma(const void* q, const void* K, const void* V, const Geo
     if (cudaGetLastError() != cudaSuccess) return L2KV_ERR_CUDA;
   }
   decode_combine_kernel<128><<<(unsigned)((long long)g.B * g.L * g.Hq), 128, 0, s>>>(
-      partial, cur_len_dev, max_len, g.t_cap, g.Hq, plan.n_splits, out);
+      partial, cur_len_dev, max_len, g.t_cap, g.H, g.Hq, plan.n_splits, out);
   return cudaGetLastError() == cudaSuccess ? L2KV_OK : L2KV_ERR_CUDA;
 }
 
 template <typename T, int D, int G>
 static int launch_dec_t(const void* q, const void* K, const void* V, const Geom& g,
-                        const int32_t* cur_len_dev, int max_len, float scale, float* out, char* ws,
+                        const LenView& cur_len_dev, int max_len, float scale, float* out, char* ws,
                         const WorkspacePlan& plan, cudaStream_t s) {
   const long long units = (long long)g.B * g.L * g.H;
   if (units == 0) return L2KV_OK;
@@ -621,13 +623,13 @@ static int launch_dec_t(const void* q, const void* K, const void* V, const Geom&
     if (cudaGetLastError() != cudaSuccess) return L2KV_ERR_CUDA;
   }
   decode_combine_kernel<D><<<(unsigned)((long long)g.B * g.L * g.Hq), D, 0, s>>>(
-      partial, cur_len_dev, max_len, g.t_cap, g.Hq, plan.n_splits, out);
+      partial, cur_len_dev, max_len, g.t_cap, g.H, g.Hq, plan.n_splits, out);
   return cudaGetLastError() == cudaSuccess ? L2KV_OK : L2KV_ERR_CUDA;
 }
 
 template <typename T, int D>
 static int launch_dec_g(const void* q, const void* K, const void* V, const Geom& g,
-                        const int32_t* cur_len_dev, int max_len, float scale, float* out, char* ws,
+                        const LenView& cur_len_dev, int max_len, float scale, float* out, char* ws,
                         const WorkspacePlan& plan, cudaStream_t s) {
   switch (g.Hq / g.H) {
     case 1: return launch_dec_t<T, D, 1>(q, K, V, g, cur_len_dev, max_len, scale, out, ws, plan, s);
@@ -641,7 +643,7 @@ static int launch_dec_g(const void* q, const void* K, const void* V, const Geom&
 }
 
 int launch_decode_attention(const void* q, const void* K, const void* V, const Geom& g, int dtype,
-                            const int32_t* cur_len_dev, int max_len, float scale, float* out,
+                            const LenView& cur_len_dev, int max_len, float scale, float* out,
                             char* ws, const WorkspacePlan& plan, cudaStream_t s) {
 #define L2KV_DA(T, D) \
   return launch_dec_g<T, D>(q, K, V, g, cur_len_dev, max_len, scale, out, ws, plan, s)

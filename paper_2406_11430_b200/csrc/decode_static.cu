@@ -72,7 +72,8 @@ extern "C" int l2kv_decode_attention_static(const void* q, const void* K_c, cons
   const float sc = scale > 0.f ? scale : 1.0f / sqrtf((float)lay->head_dim);
   // Nothing in the scratch has to start at zero: every partial that the merge step reads is
   // written by the split step of the same call.
-  return launch_decode_attention(q, K_c, V_c, make_geom(*lay), lay->dtype, cur_len_dev, max_len, sc,
+  const LenView lens{cur_len_dev, 0};
+  return launch_decode_attention(q, K_c, V_c, make_geom(*lay), lay->dtype, lens, max_len, sc,
                                  out, static_cast<char*>(scratch), plan,
                                  static_cast<cudaStream_t>(stream));
 }

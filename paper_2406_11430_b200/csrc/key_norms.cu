@@ -21,6 +21,14 @@ constexpr int kNormThreads = L2KV_NORM_THREADS;
 constexpr int kNormUnroll = 8;                 // rows per thread per step, all loads in flight
 constexpr int kNormRowsPerCta = L2KV_NORM_ROWS;
 
+// Length of a unit's compressed rows: per unit where the caller asked for that, and head 0's
+// per (b, l).
+__device__ __forceinline__ void publish_kept_len(const SelectArgs& sel, long long unit, int bl,
+                                                 int h, int keep) {
+  if (sel.kept_len_unit_dev) sel.kept_len_unit_dev[unit] = keep;
+  if (h == 0 && sel.kept_len_dev) sel.kept_len_dev[bl] = keep;
+}
+
 template <typename T, int D, int MODE>
 __global__ void __launch_bounds__(kNormThreads)
 key_norms_kernel(const T* __restrict__ K, Geom g, const int32_t* __restrict__ len_dev,
@@ -47,7 +55,7 @@ key_norms_kernel(const T* __restrict__ K, Geom g, const int32_t* __restrict__ le
         const int keep = min(len, sel.out_t_cap);
         identity_unit<kNormThreads>(len, keep, true, sel.unit_rec + unit,
                                     sel.chunk_rec + unit * sel.n_chunks);
-        if (h == 0 && tid == 0) sel.kept_len_dev[b * g.L + l] = keep;
+        if (tid == 0) publish_kept_len(sel, unit, b * g.L + l, h, keep);
       }
       return;
     }
@@ -112,9 +120,10 @@ key_norms_kernel(const T* __restrict__ K, Geom g, const int32_t* __restrict__ le
       if (!s_last) return;
       __threadfence();                                   // see the other CTAs' keys
     }
-    const int keep_req = max(0, min(sel.keep_dev[b], len));
+    const int keep_arg = sel.keep_unit_dev ? sel.keep_unit_dev[unit] : sel.keep_dev[b];
+    const int keep_req = max(0, min(keep_arg, len));
     const int keep = min(keep_req, sel.out_t_cap);       // rows that fit the output; the rest is cut
-    if (h == 0 && tid == 0) sel.kept_len_dev[b * g.L + l] = keep;
+    if (tid == 0) publish_kept_len(sel, unit, b * g.L + l, h, keep);
     if (keep_req == len) {
       identity_unit<kNormThreads>(len, keep, MODE == kKeysRandom, sel.unit_rec + unit,
                                   sel.chunk_rec + unit * sel.n_chunks);

@@ -133,10 +133,12 @@ gather_kernel(const T* __restrict__ K, const T* __restrict__ V, Geom gi, T* __re
 
 template <typename T, int D>
 static int launch_sc_t(const void* K, const void* V, const Geom& gi, const int32_t* len_dev,
-                       const int32_t* keep_dev, int max_len, const LayerMask& unc, int policy,
-                       unsigned long long seed, const float* sumsq_in, void* K_out, void* V_out,
-                       const Geom& go, int32_t* idx_out, float* sumsq_out, int32_t* kept_len_dev,
-                       char* ws, const WorkspacePlan& plan, cudaStream_t s) {
+                       const int32_t* keep_dev, const int32_t* keep_unit_dev, int max_len,
+                       const LayerMask& unc, int policy, unsigned long long seed,
+                       const float* sumsq_in, void* K_out, void* V_out, const Geom& go,
+                       int32_t* idx_out, float* sumsq_out, int32_t* kept_len_dev,
+                       int32_t* kept_len_unit_dev, char* ws, const WorkspacePlan& plan,
+                       cudaStream_t s) {
   const long long units = (long long)gi.B * gi.L * gi.H;
   if (units == 0) return L2KV_OK;
   if (plan.n_chunks > kMaxChunks) return L2KV_ERR_OUT_OF_RANGE;
@@ -156,7 +158,8 @@ static int launch_sc_t(const void* K, const void* V, const Geom& gi, const int32
     ld = gi.t_cap;
   }
   SelectArgs sel;
-  sel.keep_dev = keep_dev; sel.out_t_cap = go.t_cap;
+  sel.keep_dev = keep_dev; sel.keep_unit_dev = keep_unit_dev; sel.out_t_cap = go.t_cap;
+  sel.kept_len_unit_dev = kept_len_unit_dev;
   sel.policy = policy == L2KV_KEEP_HIGHEST_NORM ? L2KV_KEEP_HIGHEST_NORM : L2KV_KEEP_LOWEST_NORM;
   sel.seed = seed;
   sel.n_chunks = plan.n_chunks; sel.unc = unc; sel.unit_rec = urec; sel.chunk_rec = crec;
@@ -178,14 +181,17 @@ static int launch_sc_t(const void* K, const void* V, const Geom& gi, const int32
 }
 
 int launch_select_compact(const void* K, const void* V, const Geom& gi, int dtype,
-                          const int32_t* len_dev, const int32_t* keep_dev, int max_len,
+                          const int32_t* len_dev, const int32_t* keep_dev,
+                          const int32_t* keep_unit_dev, int max_len,
                           const LayerMask& unc, int policy, unsigned long long seed,
                           const float* sumsq_in, void* K_out, void* V_out, const Geom& go,
-                          int32_t* idx_out, float* sumsq_out, int32_t* kept_len_dev, char* ws,
+                          int32_t* idx_out, float* sumsq_out, int32_t* kept_len_dev,
+                          int32_t* kept_len_unit_dev, char* ws,
                           const WorkspacePlan& plan, cudaStream_t s) {
 #define L2KV_SC(T, D)                                                                           \
-  return launch_sc_t<T, D>(K, V, gi, len_dev, keep_dev, max_len, unc, policy, seed, sumsq_in,   \
-                           K_out, V_out, go, idx_out, sumsq_out, kept_len_dev, ws, plan, s)
+  return launch_sc_t<T, D>(K, V, gi, len_dev, keep_dev, keep_unit_dev, max_len, unc, policy,    \
+                           seed, sumsq_in, K_out, V_out, go, idx_out, sumsq_out, kept_len_dev,  \
+                           kept_len_unit_dev, ws, plan, s)
   if (dtype == L2KV_BF16) {
     if (gi.D == 128) L2KV_SC(__nv_bfloat16, 128);
     if (gi.D == 64) L2KV_SC(__nv_bfloat16, 64);
