@@ -567,6 +567,316 @@ prefix_attention_kernel_v2(const __nv_bfloat16* __restrict__ q, Geom g, int n_qu
                  : "memory");
 }
 
+// Third formulation: the two contractions and the softmax run concurrently.  A ninth warp
+// does nothing but fetch tiles and issue tcgen05.mma; the cache is walked in sub-blocks of
+// 64 tokens with two score buffers in tensor memory, so that S(j+1) = Q K(j+1)^T is computed
+// while the eight softmax warps work on S(j), and O += P(j) V(j) runs while they work on
+// S(j+1).  Hand-offs are mbarriers (scores ready: tcgen05.commit; weights ready: one arrival
+// per softmax thread; output quiet: tcgen05.commit), every wait on them is bounded.
+constexpr int kPf3Threads = kPfThreads + 32;    // eight softmax warps + the issuing warp
+constexpr int kPf3Sub = 64;                     // cached tokens per sub-block
+constexpr int kPf3Half = kPf3Sub * 128;         // one [64 tokens][64 bf16] swizzled tile: 8 KB
+constexpr int kPf3Tile = 2 * kPf3Half;          // both halves of the head dimension: 16 KB
+constexpr uint32_t kIdescQK64 =
+    (1u << 4) | (1u << 7) | (1u << 10) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
+
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(bar) : "memory");
+}
+// Stores 16 consecutive 32-bit columns of this thread's tensor-memory lane.  Whole warps only.
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+               "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+               :: "r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]),
+                  "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]),
+                  "r"(r[14]), "r"(r[15])
+               : "memory");
+}
+// Barrier among the 64 threads of warps w and w + 4 (the two halves of 32 query rows).
+__device__ __forceinline__ void pair_sync(int quarter) {
+  switch (quarter) {                                    // immediate ids: four named barriers in all
+    case 0: asm volatile("bar.sync 1, 64;" ::: "memory"); break;
+    case 1: asm volatile("bar.sync 2, 64;" ::: "memory"); break;
+    case 2: asm volatile("bar.sync 3, 64;" ::: "memory"); break;
+    default: asm volatile("bar.sync 4, 64;" ::: "memory"); break;
+  }
+}
+
+template <int G>
+__global__ void __launch_bounds__(kPf3Threads, 2)
+prefix_attention_kernel_v3(const __nv_bfloat16* __restrict__ q, Geom g, int n_queries,
+                           const int32_t* __restrict__ cur_len_dev, int max_len, float scale_log2e,
+                           float* __restrict__ out, float* __restrict__ lse_out,
+                           const __grid_constant__ CUtensorMap map_k,
+                           const __grid_constant__ CUtensorMap map_v,
+                           int32_t* __restrict__ status_word) {
+  constexpr int D = 128;
+  constexpr int QT = kPfRows / G;                       // queries per CTA
+  extern __shared__ unsigned char smem_raw[];
+  // [0,1] K tile landed, [2,3] V tile landed, [4,5] scores ready, [6,7] weights ready, [8] O quiet
+  __shared__ __align__(8) unsigned long long s_bar[9];
+  __shared__ uint32_t s_tmem;
+  __shared__ int s_fail;
+  __shared__ float s_x[2][2][kPfRows];                  // [sub-block parity][half][row]
+  __shared__ int s_flag[2][8];                          // [sub-block parity][softmax warp] gave up
+
+  const int q_tiles = (n_queries + QT - 1) / QT;
+  const int qt = blockIdx.x % q_tiles;
+  const long long unit = blockIdx.x / q_tiles;          // (b * L + l) * H + h
+  const int h = (int)(unit % g.H);
+  const long long bl = unit / g.H;
+  const int l = (int)(bl % g.L), b = (int)(bl / g.L);
+  const int n = max(0, min(cur_len_dev[bl], min(max_len, g.t_cap)));
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const bool softmax_thread = tid < kPfThreads;
+  // Softmax threads, two per query row: thread (row, hf) owns 32 of a sub-block's 64 score
+  // columns and output dims [64 hf, 64 hf + 64).  Warps w and w + 4 share a lane quarter.
+  const int row = tid & (kPfRows - 1), hf = (tid >> 7) & 1;
+  const int s_idx = qt * QT + row / G;                  // this row's query and head
+  const int head = h * G + row % G;
+  const bool row_valid = softmax_thread && s_idx < n_queries;
+  const long long row_off = ((bl * n_queries + s_idx) * g.Hq + head);
+  if (n == 0) {                                         // empty cache: zeros, log-sum-exp = -inf
+    if (row_valid) {
+      for (int d = 0; d < 64; ++d) out[row_off * D + hf * 64 + d] = 0.f;
+      if (lse_out && hf == 0) lse_out[row_off] = -INFINITY;
+    }
+    return;
+  }
+  // A wait that gave up in an earlier CTA marks the workspace; the rest of the grid leaves.
+  if (status_word && *reinterpret_cast<volatile int32_t*>(status_word + 2) != 0) return;
+  const int nb = (n + kPf3Sub - 1) / kPf3Sub;
+
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;   // 1024-byte aligned tiles
+  const uint32_t sQ = base, sK = base + kPfTileBytes, sV = sK + 2 * kPf3Tile;
+  const uint32_t bar0 = smem_u32(&s_bar[0]);
+  auto bar_k = [&](int i) { return bar0 + 8u * (uint32_t)i; };
+  auto bar_v = [&](int i) { return bar0 + 8u * (uint32_t)(2 + i); };
+  auto bar_s = [&](int i) { return bar0 + 8u * (uint32_t)(4 + i); };
+  auto bar_p = [&](int i) { return bar0 + 8u * (uint32_t)(6 + i); };
+  const uint32_t bar_o = bar0 + 64u;
+
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 :: "r"(smem_u32(&s_tmem)), "r"(kPfTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  if (tid == 0) {
+    for (int i = 0; i < 6; ++i) mbar_init(bar0 + 8u * i, 1);
+    mbar_init(bar_p(0), kPfThreads);
+    mbar_init(bar_p(1), kPfThreads);
+    mbar_init(bar_o, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    s_fail = 0;
+  }
+  __syncwarp();
+  if (softmax_thread) {                                 // Q rows, K-major, 128-byte swizzle
+    const uint4* src = reinterpret_cast<const uint4*>(q + row_off * D) + hf * 8;
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+      const uint4 v = row_valid ? src[c] : make_uint4(0, 0, 0, 0);
+      st_shared16(sQ + hf * kPfHalf + row * 128 + ((c ^ (row & 7)) << 4), v.x, v.y, v.z, v.w);
+    }
+  }
+  proxy_fence();
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = s_tmem;
+  bool gave_up = false;
+  float m_ref = -INFINITY, l_run = 0.f, l_exact = 0.f;  // reference maximum; sums of this half's weights
+  const uint32_t t_lane = tmem + ((uint32_t)((warp & 3) * 32) << 16);   // this warp's lane quarter
+  const uint32_t t_o = t_lane + 128 + hf * 64;          // this thread's 64 output dims
+
+  if (!softmax_thread) {
+    // ---- the issuing warp: one lane fetches tiles and issues every contraction ---------------
+    if (tid == kPfThreads) {
+      auto load_k = [&](int j) {
+        const uint32_t dst = sK + (j & 1) * kPf3Tile;
+        mbar_expect_tx(bar_k(j & 1), kPf3Tile);
+        tma_load_5d(dst, &map_k, bar_k(j & 1), 0, j * kPf3Sub, h, l, b);
+        tma_load_5d(dst + kPf3Half, &map_k, bar_k(j & 1), 64, j * kPf3Sub, h, l, b);
+      };
+      auto load_v = [&](int j) {
+        const uint32_t dst = sV + (j & 1) * kPf3Tile;
+        mbar_expect_tx(bar_v(j & 1), kPf3Tile);
+        tma_load_5d(dst, &map_v, bar_v(j & 1), 0, j * kPf3Sub, h, l, b);
+        tma_load_5d(dst + kPf3Half, &map_v, bar_v(j & 1), 64, j * kPf3Sub, h, l, b);
+      };
+      auto issue_qk = [&](int j) {                      // S[j & 1] = Q K(j)^T, then signal
+        const uint32_t kt = sK + (j & 1) * kPf3Tile;
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+          umma_bf16(tmem + (j & 1) * 64,
+                    umma_desc(sQ + (k >> 2) * kPfHalf + (k & 3) * 32, 16, 1024),
+                    umma_desc(kt + (k >> 2) * kPf3Half + (k & 3) * 32, 16, 1024), kIdescQK64, k > 0);
+        umma_commit(bar_s(j & 1));
+      };
+      bool ok = true;
+      load_k(0); load_v(0);
+      if (nb > 1) { load_k(1); load_v(1); }
+      ok = mbar_wait<kPfPolls>(bar_k(0), 0);
+      if (ok) { tc_fence_after(); issue_qk(0); }
+      if (ok && nb > 1) {
+        ok = mbar_wait<kPfPolls>(bar_k(1), 0);
+        if (ok) { tc_fence_after(); issue_qk(1); }
+      }
+      if (ok && nb > 2) {                               // the first K tile is free once S(0) is done
+        ok = mbar_wait<kPfPolls>(bar_s(0), 0);
+        if (ok) load_k(2);
+      }
+      for (int j = 0; ok && j < nb; ++j) {
+        const int s = j & 1;
+        const uint32_t par = (uint32_t)(j >> 1) & 1u;
+        ok = mbar_wait<kPfPolls>(bar_p(s), par) && mbar_wait<kPfPolls>(bar_v(s), par);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t vt = sV + s * kPf3Tile;
+#pragma unroll
+        for (int k = 0; k < 4; ++k)                     // O += P(j) V(j); slice k = tokens 16k .. 16k + 15
+          umma_bf16_ts(tmem + 128, tmem + s * 64 + (k >> 1) * 32 + (k & 1) * 8,
+                       umma_desc(vt + k * 2048, kPf3Half, 1024), kIdescPV, (j > 0 || k > 0) ? 1u : 0u);
+        umma_commit(bar_o);
+        // Q K(j+1)^T was issued before these; once it is done its K tile takes sub-block j + 3.
+        if (j + 3 < nb) {
+          ok = mbar_wait<kPfPolls>(bar_s(s ^ 1), (uint32_t)((j + 1) >> 1) & 1u);
+          if (!ok) break;
+          load_k(j + 3);
+        }
+        // P(j) V(j) done: its V tile and score buffer are free for sub-block j + 2.
+        ok = mbar_wait<kPfPolls>(bar_o, (uint32_t)j & 1u);
+        if (!ok) break;
+        if (j + 2 < nb) {
+          load_v(j + 2);
+          ok = mbar_wait<kPfPolls>(bar_k(s), (uint32_t)((j + 2) >> 1) & 1u);
+          if (!ok) break;
+          tc_fence_after();
+          issue_qk(j + 2);
+        }
+      }
+      if (!ok) s_fail = 1;
+    }
+  } else {
+    // ---- the softmax warps -------------------------------------------------------------------
+    for (int j = 0; j < nb; ++j) {
+      const int s = j & 1;
+      const int valid_all = min(kPf3Sub, n - j * kPf3Sub);   // valid tokens of this sub-block
+      const int valid = valid_all - hf * 32;                  // ... among this thread's 32
+      const uint32_t t_s = t_lane + s * 64 + hf * 32;         // this thread's scores, later its weights
+      if (!mbar_wait<kPfPolls>(bar_s(s), (uint32_t)(j >> 1) & 1u)) gave_up = true;
+      tc_fence_after();
+      float sv[32];
+      float bmax = -INFINITY;
+      {
+        uint32_t r[32];
+        tmem_ld32(t_s, r);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          sv[i] = i < valid ? __uint_as_float(r[i]) * scale_log2e : -INFINITY;
+          bmax = fmaxf(bmax, sv[i]);
+        }
+      }
+      // The two halves of a row exchange their maxima, and whether either warp gave up, so
+      // that both warps of the pair leave the loop together.
+      gave_up = __any_sync(0xffffffffu, gave_up);
+      s_x[s][hf][row] = bmax;
+      if ((tid & 31) == 0) s_flag[s][warp] = gave_up ? 1 : 0;
+      pair_sync(warp & 3);
+      if (s_flag[s][warp & 3] | s_flag[s][(warp & 3) + 4]) { gave_up = true; break; }
+      const float m_new = fmaxf(m_ref, fmaxf(s_x[s][0][row], s_x[s][1][row]));
+      if (j == 0) m_ref = m_new;
+      // ---- rescale O only when this row's maximum has drifted far from the reference --------
+      const bool need = m_new > m_ref + kPfRescaleGap;
+      if (__any_sync(0xffffffffu, need)) {
+        // O must be quiet: P(j-1) V(j-1) has to be complete (P(j) V(j) waits for this thread)
+        if (!mbar_wait<kPfPolls>(bar_o, (uint32_t)(j - 1) & 1u)) gave_up = true;
+        tc_fence_after();
+        const float factor = need ? fast_exp2(m_ref - m_new) : 1.f;
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          uint32_t r[32];
+          tmem_ld32(t_o + c * 32, r);
+#pragma unroll
+          for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * factor);
+          tmem_st32(t_o + c * 32, r);
+        }
+        if (need) { l_run *= factor; l_exact *= factor; m_ref = m_new; }
+      }
+      // ---- weights 2^(s - m_ref) as bf16 pairs over the first half of the score columns -----
+      {
+        uint32_t pk[16];
+        float rowsum = 0.f, rowsum_exact = 0.f;
+#pragma unroll
+        for (int i = 0; i < 32; i += 2) {
+          const float p0 = fast_exp2(sv[i] - m_ref), p1 = fast_exp2(sv[i + 1] - m_ref);   // -inf -> 0
+          const __nv_bfloat162 pr = __floats2bfloat162_rn(p0, p1);
+          // the normalising sum uses the rounded weights, the ones V is multiplied with
+          rowsum += __low2float(pr) + __high2float(pr);
+          rowsum_exact += p0 + p1;
+          pk[i >> 1] = *reinterpret_cast<const uint32_t*>(&pr);
+        }
+        tmem_st16(t_s, pk);
+        tmem_wait_st();
+        l_run += rowsum;
+        l_exact += rowsum_exact;
+      }
+      if (valid_all < kPf3Sub) {
+        // Last, partial sub-block: rows of the V tile past the valid length hold whatever the
+        // cache holds there; clear them so that a zero weight times Inf/NaN cannot reach O.
+        if (!mbar_wait<kPfPolls>(bar_v(s), (uint32_t)(j >> 1) & 1u)) gave_up = true;
+        if (row >= valid_all && row < kPf3Sub) {
+#pragma unroll
+          for (int c = 0; c < 8; ++c)
+            st_shared16(sV + s * kPf3Tile + hf * kPf3Half + row * 128 + (c << 4), 0, 0, 0, 0);
+        }
+        proxy_fence();
+      }
+      tc_fence_before();
+      mbar_arrive(bar_p(s));                              // this thread's weights (and O) are in place
+    }
+    // O is complete when the last P V has been committed
+    if (!gave_up && !mbar_wait<kPfPolls>(bar_o, (uint32_t)(nb - 1) & 1u)) gave_up = true;
+    if (gave_up) s_fail = 1;
+  }
+  __syncthreads();                                       // every role is done with the loop
+  tc_fence_after();
+  const bool failed = s_fail != 0;
+  // the two halves of a row share the reference maximum; their weight sums add up
+  if (softmax_thread) s_x[0][hf][row] = l_run;
+  __syncthreads();
+  const float l_tot = s_x[0][0][row] + s_x[0][1][row];
+  __syncthreads();
+  if (softmax_thread) s_x[0][hf][row] = l_exact;
+  __syncthreads();
+  const float l_tot_exact = s_x[0][0][row] + s_x[0][1][row];
+  if (!failed && softmax_thread) {
+    const float inv = 1.f / l_tot;
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+      uint32_t r[32];
+      tmem_ld32(t_o + c * 32, r);
+      if (row_valid) {
+        float4* dst = reinterpret_cast<float4*>(out + row_off * D + hf * 64 + c * 32);
+#pragma unroll
+        for (int i = 0; i < 32; i += 4)
+          dst[i >> 2] = make_float4(__uint_as_float(r[i]) * inv, __uint_as_float(r[i + 1]) * inv,
+                                    __uint_as_float(r[i + 2]) * inv, __uint_as_float(r[i + 3]) * inv);
+      }
+    }
+    if (row_valid && lse_out && hf == 0)
+      lse_out[row_off] = (m_ref + log2f(l_tot_exact)) * 0.6931471805599453f;
+  }
+  if (failed && tid == 0 && status_word) {
+    atomicExch(status_word, (int)L2KV_ERR_CUDA);
+    atomicExch(status_word + 2, 1);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0)
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem), "r"(kPfTmemCols)
+                 : "memory");
+}
+
 template <int G>
 static int launch_pf(const void* q, const void* K, const void* V, const Geom& g, int n_queries,
                      const int32_t* cur_len_dev, int max_len, float scale, float* out,
@@ -579,16 +889,19 @@ static int launch_pf(const void* q, const void* K, const void* V, const Geom& g,
   alignas(64) CUtensorMap map_k, map_v;
   std::memset(&map_k, 0, sizeof map_k);
   std::memset(&map_v, 0, sizeof map_v);
-  if (!make_cache_map(&map_k, K, g, kPfRows) || !make_cache_map(&map_v, V, g, kPfRows))
-    return L2KV_ERR_UNSUPPORTED;
   constexpr int smem_bytes = 1024 + 3 * kPfTileBytes;
-  // L2KV_PREFIX_KERNEL=v1 selects the first formulation (weights through shared memory).
+  // L2KV_PREFIX_KERNEL selects a formulation: v1 (weights through shared memory), v2 (weights
+  // in tensor memory, one role), v3 (separate issuing warp, 64-token sub-blocks).
   const char* which = std::getenv("L2KV_PREFIX_KERNEL");
   const bool v1 = which && std::strcmp(which, "v1") == 0;
-  auto kern = v1 ? prefix_attention_kernel<G> : prefix_attention_kernel_v2<G>;
+  const bool v3 = which && std::strcmp(which, "v3") == 0;
+  auto kern = v1 ? prefix_attention_kernel<G> : v3 ? prefix_attention_kernel_v3<G> : prefix_attention_kernel_v2<G>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) != cudaSuccess)
     return L2KV_ERR_CUDA;
-  kern<<<(unsigned)blocks, kPfThreads, smem_bytes, s>>>(
+  const int sub_rows = v3 ? kPf3Sub : kPfRows;
+  if (!make_cache_map(&map_k, K, g, sub_rows) || !make_cache_map(&map_v, V, g, sub_rows))
+    return L2KV_ERR_UNSUPPORTED;
+  kern<<<(unsigned)blocks, v3 ? kPf3Threads : kPfThreads, smem_bytes, s>>>(
       static_cast<const __nv_bfloat16*>(q), g, n_queries, cur_len_dev, max_len, scale * kPfLog2e, out,
       lse_out, map_k, map_v, status_word);
   return cudaGetLastError() == cudaSuccess ? L2KV_OK : L2KV_ERR_CUDA;

@@ -32,10 +32,15 @@ def run(l2, q, K, V, cur, max_len, scale=0.0):
     return out.cpu().numpy(), lse.cpu().numpy()
 
 
+KERNELS = ["v2", "v1", "v3"]      # the three formulations of the kernel; v2 is the default
+
+
+@pytest.mark.parametrize("kernel", ["v2", "v3"])
 @pytest.mark.parametrize("Hkv,Hq,n_q,T", [(2, 8, 40, 300), (2, 2, 130, 257), (1, 8, 1, 1000),
                                           (2, 4, 64, 128)])
-def test_prefix_attention_matches_oracle(Hkv, Hq, n_q, T):
+def test_prefix_attention_matches_oracle(Hkv, Hq, n_q, T, kernel, monkeypatch):
     import paper_2406_11430_b200 as l2
+    monkeypatch.setenv("L2KV_PREFIX_KERNEL", kernel)
     w = synth.WORKLOADS[2].scaled(B=2, L=2, Hkv=Hkv, Hq=Hq, T=T)
     K, V = synth.make_cache(w, DEV)
     q = make_queries(w, n_q, 3)
@@ -55,9 +60,8 @@ def test_prefix_attention_matches_oracle(Hkv, Hq, n_q, T):
         np.testing.assert_allclose(lse[b, l, s, j], scipy.special.logsumexp(z), rtol=1e-5, atol=1e-4)
 
 
-@pytest.mark.parametrize("kernel", ["v2", "v1"])
+@pytest.mark.parametrize("kernel", KERNELS)
 def test_prefix_attention_agrees_with_decode_and_ignores_rows_past_the_length(kernel, monkeypatch):
-    # both formulations of the kernel (weights in tensor memory / through shared memory)
     import paper_2406_11430_b200 as l2
     monkeypatch.setenv("L2KV_PREFIX_KERNEL", kernel)
     w = synth.WORKLOADS[2].scaled(B=1, L=2, T=700)
@@ -73,3 +77,28 @@ def test_prefix_attention_agrees_with_decode_and_ignores_rows_past_the_length(ke
     Vp[0, 1, :, 333:] = float("inf")
     out2, _ = run(l2, q, Kp, Vp, cur, 700, scale=0.07)
     assert np.array_equal(out, out2)
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+@pytest.mark.parametrize("direction", [1, -1])
+def test_prefix_attention_with_drifting_maxima(kernel, direction, monkeypatch):
+    """Scores that grow (or fall) steadily along the cache: the running maximum moves by far
+    more than the range one reference maximum can cover, so the accumulated output is rescaled
+    several times (growing), or later weights underflow to zero (falling)."""
+    import paper_2406_11430_b200 as l2
+    monkeypatch.setenv("L2KV_PREFIX_KERNEL", kernel)
+    T = 900
+    w = synth.WORKLOADS[2].scaled(B=1, L=1, Hkv=2, Hq=4, T=T)
+    K, V = synth.make_cache(w, DEV)
+    ramp = torch.arange(T, device=DEV, dtype=torch.float32) * (0.25 * direction)
+    K[0, 0, :, :, 0] = ramp.to(torch.bfloat16)
+    q = make_queries(w, 7, 21)
+    q[..., 0] = 4.0
+    cur = np.array([[T]], dtype=np.int32)
+    out, lse = run(l2, q, K, V, cur, T)
+    Kn, Vn = synth.to_numpy(K), synth.to_numpy(V)
+    for s in range(7):
+        want = oracle.attention(synth.to_numpy(q[:, :, s].contiguous()), Kn, Vn, "bf16", cur, nthreads=8)
+        assert_attention_close(out[:, :, s], want, atol=4e-3)
+    z = K[0, 0, 1].double().cpu().numpy() @ q[0, 0, 3, 2].double().cpu().numpy() / np.sqrt(w.D)
+    np.testing.assert_allclose(lse[0, 0, 3, 2], scipy.special.logsumexp(z), rtol=1e-5, atol=1e-4)
