@@ -425,7 +425,7 @@ prefix_attention_kernel_v2(const __nv_bfloat16* __restrict__ q, Geom g, int n_qu
   if (tid == 0) { load_k(0); load_v(0); }
   __syncwarp();
 
-  float m_ref = -INFINITY, l_run = 0.f, l_exact = 0.f;  // reference maximum; sums of this half's weights
+  float m_ref = -INFINITY, l_run = 0.f;                 // reference maximum; sum of this half's weights
 
   for (int kb = 0; kb < n_blocks; ++kb) {
     const int valid_all = min(kPfRows, n - kb * kPfRows);   // valid tokens of this block
@@ -451,19 +451,28 @@ prefix_attention_kernel_v2(const __nv_bfloat16* __restrict__ q, Geom g, int n_qu
     if (s_fail) break;
     tc_fence_after();
     // ---- this thread's 64 scores (log2 domain), kept in registers ---------------------------
+    // (raw products; the scale is folded into the exponent's multiply-add below)
     float sv[64];
     float bmax = -INFINITY;
 #pragma unroll
     for (int c = 0; c < 2; ++c) {
       uint32_t r[32];
       tmem_ld32(t_s + c * 32, r);
+      if (valid >= 64) {                                 // warp-uniform: only the last block masks
 #pragma unroll
-      for (int i = 0; i < 32; ++i) {
-        sv[c * 32 + i] = c * 32 + i < valid ? __uint_as_float(r[i]) * scale_log2e : -INFINITY;
-        bmax = fmaxf(bmax, sv[c * 32 + i]);
+        for (int i = 0; i < 32; ++i) {
+          sv[c * 32 + i] = __uint_as_float(r[i]);
+          bmax = fmaxf(bmax, sv[c * 32 + i]);
+        }
+      } else {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          sv[c * 32 + i] = c * 32 + i < valid ? __uint_as_float(r[i]) : -INFINITY;
+          bmax = fmaxf(bmax, sv[c * 32 + i]);
+        }
       }
     }
-    s_x[hf][row] = bmax;
+    s_x[hf][row] = bmax * scale_log2e;                   // scale > 0: the maximum commutes with it
     tc_fence_before();
     __syncthreads();                                     // maxima exchanged; every score has been read
     tc_fence_after();
@@ -482,25 +491,24 @@ prefix_attention_kernel_v2(const __nv_bfloat16* __restrict__ q, Geom g, int n_qu
         tmem_st32(t_o + c * 32, r);
       }
       tmem_wait_st();
-      if (need) { l_run *= factor; l_exact *= factor; m_ref = m_new; }
+      if (need) { l_run *= factor; m_ref = m_new; }
     }
     // ---- weights 2^(s - m_ref) as bf16 pairs over the score columns -------------------------
     {
       uint32_t pk[32];
-      float rowsum = 0.f, rowsum_exact = 0.f;
+      float rowsum0 = 0.f, rowsum1 = 0.f;
+      const float neg_m = -m_ref;
 #pragma unroll
       for (int i = 0; i < 64; i += 2) {
-        const float p0 = fast_exp2(sv[i] - m_ref), p1 = fast_exp2(sv[i + 1] - m_ref);   // -inf -> 0
-        const __nv_bfloat162 pr = __floats2bfloat162_rn(p0, p1);
-        // the normalising sum uses the rounded weights, the ones V is multiplied with
-        rowsum += __low2float(pr) + __high2float(pr);
-        rowsum_exact += p0 + p1;
-        pk[i >> 1] = *reinterpret_cast<const uint32_t*>(&pr);
+        const float p0 = fast_exp2(__fmaf_rn(sv[i], scale_log2e, neg_m));     // -inf -> 0
+        const float p1 = fast_exp2(__fmaf_rn(sv[i + 1], scale_log2e, neg_m));
+        rowsum0 += p0;
+        rowsum1 += p1;
+        pk[i >> 1] = pack_bf16(p0, p1);
       }
       tmem_st32(t_p, pk);
       tmem_wait_st();
-      l_run += rowsum;
-      l_exact += rowsum_exact;
+      l_run += rowsum0 + rowsum1;
     }
     if (valid_all < kPfRows) {
       // Last, partial block: rows of the V tile past the valid length hold whatever the cache
@@ -535,10 +543,6 @@ prefix_attention_kernel_v2(const __nv_bfloat16* __restrict__ q, Geom g, int n_qu
   s_x[hf][row] = l_run;
   __syncthreads();
   const float l_tot = s_x[0][row] + s_x[1][row];
-  __syncthreads();
-  s_x[hf][row] = l_exact;
-  __syncthreads();
-  const float l_tot_exact = s_x[0][row] + s_x[1][row];
   if (!failed) {
     const float inv = 1.f / l_tot;
 #pragma unroll
@@ -554,7 +558,7 @@ prefix_attention_kernel_v2(const __nv_bfloat16* __restrict__ q, Geom g, int n_qu
       }
     }
     if (row_valid && lse_out && hf == 0)
-      lse_out[row_off] = (m_ref + log2f(l_tot_exact)) * 0.6931471805599453f;
+      lse_out[row_off] = (m_ref + log2f(l_tot)) * 0.6931471805599453f;
   }
   if (failed && tid == 0 && status_word) {
     atomicExch(status_word, (int)L2KV_ERR_CUDA);
@@ -684,7 +688,7 @@ prefix_attention_kernel_v3(const __nv_bfloat16* __restrict__ q, Geom g, int n_qu
   tc_fence_after();
   const uint32_t tmem = s_tmem;
   bool gave_up = false;
-  float m_ref = -INFINITY, l_run = 0.f, l_exact = 0.f;  // reference maximum; sums of this half's weights
+  float m_ref = -INFINITY, l_run = 0.f;                 // reference maximum; sum of this half's weights
   const uint32_t t_lane = tmem + ((uint32_t)((warp & 3) * 32) << 16);   // this warp's lane quarter
   const uint32_t t_o = t_lane + 128 + hf * 64;          // this thread's 64 output dims
 
@@ -765,16 +769,25 @@ prefix_attention_kernel_v3(const __nv_bfloat16* __restrict__ q, Geom g, int n_qu
       const uint32_t t_s = t_lane + s * 64 + hf * 32;         // this thread's scores, later its weights
       if (!mbar_wait<kPfPolls>(bar_s(s), (uint32_t)(j >> 1) & 1u)) gave_up = true;
       tc_fence_after();
-      float sv[32];
+      float sv[32];                                       // raw products; the scale is folded in below
       float bmax = -INFINITY;
       {
         uint32_t r[32];
         tmem_ld32(t_s, r);
+        if (valid >= 32) {                                // warp-uniform: only the last sub-block masks
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          sv[i] = i < valid ? __uint_as_float(r[i]) * scale_log2e : -INFINITY;
-          bmax = fmaxf(bmax, sv[i]);
+          for (int i = 0; i < 32; ++i) {
+            sv[i] = __uint_as_float(r[i]);
+            bmax = fmaxf(bmax, sv[i]);
+          }
+        } else {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            sv[i] = i < valid ? __uint_as_float(r[i]) : -INFINITY;
+            bmax = fmaxf(bmax, sv[i]);
+          }
         }
+        bmax *= scale_log2e;                              // scale > 0: the maximum commutes with it
       }
       // The two halves of a row exchange their maxima, and whether either warp gave up, so
       // that both warps of the pair leave the loop together.
@@ -800,25 +813,24 @@ prefix_attention_kernel_v3(const __nv_bfloat16* __restrict__ q, Geom g, int n_qu
           for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * factor);
           tmem_st32(t_o + c * 32, r);
         }
-        if (need) { l_run *= factor; l_exact *= factor; m_ref = m_new; }
+        if (need) { l_run *= factor; m_ref = m_new; }
       }
       // ---- weights 2^(s - m_ref) as bf16 pairs over the first half of the score columns -----
       {
         uint32_t pk[16];
-        float rowsum = 0.f, rowsum_exact = 0.f;
+        float rowsum0 = 0.f, rowsum1 = 0.f;
+        const float neg_m = -m_ref;
 #pragma unroll
         for (int i = 0; i < 32; i += 2) {
-          const float p0 = fast_exp2(sv[i] - m_ref), p1 = fast_exp2(sv[i + 1] - m_ref);   // -inf -> 0
-          const __nv_bfloat162 pr = __floats2bfloat162_rn(p0, p1);
-          // the normalising sum uses the rounded weights, the ones V is multiplied with
-          rowsum += __low2float(pr) + __high2float(pr);
-          rowsum_exact += p0 + p1;
-          pk[i >> 1] = *reinterpret_cast<const uint32_t*>(&pr);
+          const float p0 = fast_exp2(__fmaf_rn(sv[i], scale_log2e, neg_m));     // -inf -> 0
+          const float p1 = fast_exp2(__fmaf_rn(sv[i + 1], scale_log2e, neg_m));
+          rowsum0 += p0;
+          rowsum1 += p1;
+          pk[i >> 1] = pack_bf16(p0, p1);
         }
         tmem_st16(t_s, pk);
         tmem_wait_st();
-        l_run += rowsum;
-        l_exact += rowsum_exact;
+        l_run += rowsum0 + rowsum1;
       }
       if (valid_all < kPf3Sub) {
         // Last, partial sub-block: rows of the V tile past the valid length hold whatever the
@@ -845,10 +857,6 @@ prefix_attention_kernel_v3(const __nv_bfloat16* __restrict__ q, Geom g, int n_qu
   if (softmax_thread) s_x[0][hf][row] = l_run;
   __syncthreads();
   const float l_tot = s_x[0][0][row] + s_x[0][1][row];
-  __syncthreads();
-  if (softmax_thread) s_x[0][hf][row] = l_exact;
-  __syncthreads();
-  const float l_tot_exact = s_x[0][0][row] + s_x[0][1][row];
   if (!failed && softmax_thread) {
     const float inv = 1.f / l_tot;
 #pragma unroll
@@ -864,7 +872,7 @@ prefix_attention_kernel_v3(const __nv_bfloat16* __restrict__ q, Geom g, int n_qu
       }
     }
     if (row_valid && lse_out && hf == 0)
-      lse_out[row_off] = (m_ref + log2f(l_tot_exact)) * 0.6931471805599453f;
+      lse_out[row_off] = (m_ref + log2f(l_tot)) * 0.6931471805599453f;
   }
   if (failed && tid == 0 && status_word) {
     atomicExch(status_word, (int)L2KV_ERR_CUDA);
