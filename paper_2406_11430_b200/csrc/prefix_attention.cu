@@ -327,6 +327,22 @@ prefix_attention_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n_queri
                  : "memory");
 }
 
+// Eight columns at a time: the rarely taken rescaling of O, kept small in registers.
+__device__ __forceinline__ void tmem_scale8(uint32_t taddr, float factor) {
+  uint32_t r0, r1, r2, r3, r4, r5, r6, r7;
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3), "=r"(r4), "=r"(r5), "=r"(r6), "=r"(r7)
+               : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+  r0 = __float_as_uint(__uint_as_float(r0) * factor); r1 = __float_as_uint(__uint_as_float(r1) * factor);
+  r2 = __float_as_uint(__uint_as_float(r2) * factor); r3 = __float_as_uint(__uint_as_float(r3) * factor);
+  r4 = __float_as_uint(__uint_as_float(r4) * factor); r5 = __float_as_uint(__uint_as_float(r5) * factor);
+  r6 = __float_as_uint(__uint_as_float(r6) * factor); r7 = __float_as_uint(__uint_as_float(r7) * factor);
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+               :: "r"(taddr), "r"(r0), "r"(r1), "r"(r2), "r"(r3), "r"(r4), "r"(r5), "r"(r6), "r"(r7)
+               : "memory");
+}
+
 // Second formulation of the same kernel, the one the entry point uses: the weights never go
 // to shared memory.  They are written as bf16 pairs into the tensor-memory columns that held
 // the scores and feed the second contraction from there (tcgen05.mma with A in tensor
@@ -482,14 +498,8 @@ prefix_attention_kernel_v2(const __nv_bfloat16* __restrict__ q, Geom g, int n_qu
     const bool need = m_new > m_ref + kPfRescaleGap;
     if (__any_sync(0xffffffffu, need)) {
       const float factor = need ? fast_exp2(m_ref - m_new) : 1.f;
-#pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        uint32_t r[32];
-        tmem_ld32(t_o + c * 32, r);
-#pragma unroll
-        for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * factor);
-        tmem_st32(t_o + c * 32, r);
-      }
+#pragma unroll 1
+      for (int c = 0; c < 64; c += 8) tmem_scale8(t_o + c, factor);
       tmem_wait_st();
       if (need) { l_run *= factor; m_ref = m_new; }
     }
@@ -805,14 +815,8 @@ prefix_attention_kernel_v3(const __nv_bfloat16* __restrict__ q, Geom g, int n_qu
         if (!mbar_wait<kPfPolls>(bar_o, (uint32_t)(j - 1) & 1u)) gave_up = true;
         tc_fence_after();
         const float factor = need ? fast_exp2(m_ref - m_new) : 1.f;
-#pragma unroll
-        for (int c = 0; c < 2; ++c) {
-          uint32_t r[32];
-          tmem_ld32(t_o + c * 32, r);
-#pragma unroll
-          for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * factor);
-          tmem_st32(t_o + c * 32, r);
-        }
+#pragma unroll 1
+        for (int c = 0; c < 64; c += 8) tmem_scale8(t_o + c, factor);
         if (need) { l_run *= factor; m_ref = m_new; }
       }
       // ---- weights 2^(s - m_ref) as bf16 pairs over the first half of the score columns -----
