@@ -739,10 +739,12 @@ prefix_attention_kernel_v3(const __nv_bfloat16* __restrict__ q, Geom g, int n_qu
         ok = mbar_wait<kPfPolls>(bar_s(0), 0);
         if (ok) load_k(2);
       }
+      if (ok) ok = mbar_wait<kPfPolls>(bar_v(0), 0);
+      // Waits that are expected to be over already (tiles fetched an iteration ago) are placed
+      // where this thread would otherwise idle: under the contraction it has just issued.
       for (int j = 0; ok && j < nb; ++j) {
         const int s = j & 1;
-        const uint32_t par = (uint32_t)(j >> 1) & 1u;
-        ok = mbar_wait<kPfPolls>(bar_p(s), par) && mbar_wait<kPfPolls>(bar_v(s), par);
+        ok = mbar_wait<kPfPolls>(bar_p(s), (uint32_t)(j >> 1) & 1u);
         if (!ok) break;
         tc_fence_after();
         const uint32_t vt = sV + s * kPf3Tile;
@@ -751,22 +753,18 @@ prefix_attention_kernel_v3(const __nv_bfloat16* __restrict__ q, Geom g, int n_qu
           umma_bf16_ts(tmem + 128, tmem + s * 64 + (k >> 1) * 32 + (k & 1) * 8,
                        umma_desc(vt + k * 2048, kPf3Half, 1024), kIdescPV, (j > 0 || k > 0) ? 1u : 0u);
         umma_commit(bar_o);
-        // Q K(j+1)^T was issued before these; once it is done its K tile takes sub-block j + 3.
-        if (j + 3 < nb) {
-          ok = mbar_wait<kPfPolls>(bar_s(s ^ 1), (uint32_t)((j + 1) >> 1) & 1u);
-          if (!ok) break;
-          load_k(j + 3);
-        }
-        // P(j) V(j) done: its V tile and score buffer are free for sub-block j + 2.
-        ok = mbar_wait<kPfPolls>(bar_o, (uint32_t)j & 1u);
+        if (j + 2 < nb) ok = mbar_wait<kPfPolls>(bar_k(s), (uint32_t)((j + 2) >> 1) & 1u);
+        if (ok && j + 1 < nb) ok = mbar_wait<kPfPolls>(bar_v(s ^ 1), (uint32_t)((j + 1) >> 1) & 1u);
+        // P(j) V(j) done: its V tile and score buffer are free for sub-block j + 2, and so is
+        // the K tile of Q K(j+1)^T, which was issued before it (a commit covers all earlier ones).
+        ok = ok && mbar_wait<kPfPolls>(bar_o, (uint32_t)j & 1u);
         if (!ok) break;
         if (j + 2 < nb) {
-          load_v(j + 2);
-          ok = mbar_wait<kPfPolls>(bar_k(s), (uint32_t)((j + 2) >> 1) & 1u);
-          if (!ok) break;
           tc_fence_after();
           issue_qk(j + 2);
+          load_v(j + 2);
         }
+        if (j + 3 < nb) load_k(j + 3);
       }
       if (!ok) s_fail = 1;
     }
