@@ -1199,6 +1199,277 @@ prefix_attention_kernel_v4(const __nv_bfloat16* __restrict__ q, Geom g, int n_qu
                  : "memory");
 }
 
+// Fifth formulation: the fourth with one softmax thread per query row (four warps per query
+// tile): a row's maximum and sum are thread-local, so the softmax warps never synchronise with
+// one another; they only wait for scores and hand over weights.
+constexpr int kPf5Threads = 2 * kPfRows + 4 * 32;      // softmax A, softmax B, issuer A, issuer B, K, V
+
+template <int G>
+__global__ void __launch_bounds__(kPf5Threads, 1)
+prefix_attention_kernel_v5(const __nv_bfloat16* __restrict__ q, Geom g, int n_queries,
+                           const int32_t* __restrict__ cur_len_dev, int max_len, float scale_log2e,
+                           float* __restrict__ out, float* __restrict__ lse_out,
+                           const __grid_constant__ CUtensorMap map_k,
+                           const __grid_constant__ CUtensorMap map_v,
+                           int32_t* __restrict__ status_word) {
+  constexpr int D = 128;
+  constexpr int QT = kPfRows / G;                       // queries per query tile
+  constexpr int NS = kPf4Stages;
+  extern __shared__ unsigned char smem_raw[];
+  // mbarriers: K landed [NS], V landed [NS], K tile free [NS], V tile free [NS], then per query
+  // tile: scores ready [2], weights ready [2], output quiet [1]
+  __shared__ __align__(8) unsigned long long s_bar[4 * NS + 10];
+  __shared__ uint32_t s_tmem;
+  __shared__ int s_fail;
+
+  const int q_tiles = (n_queries + QT - 1) / QT;
+  const int q_pairs = (q_tiles + 1) / 2;
+  const int qp = blockIdx.x % q_pairs;
+  const long long unit = blockIdx.x / q_pairs;          // (b * L + l) * H + h
+  const int h = (int)(unit % g.H);
+  const long long bl = unit / g.H;
+  const int l = (int)(bl % g.L), b = (int)(bl / g.L);
+  const int n = max(0, min(cur_len_dev[bl], min(max_len, g.t_cap)));
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const bool softmax_thread = tid < 2 * kPfRows;
+  const int n_tiles = (2 * qp + 1 < q_tiles) ? 2 : 1;   // query tiles of this CTA that exist
+  // Softmax threads: one per query row of query tile `tile`.
+  const int tile = softmax_thread ? tid >> 7 : warp & 1;
+  const int row = tid & (kPfRows - 1);
+  const int wq = warp & 3;                              // tensor-memory lane quarter of this warp
+  const int s_idx = (2 * qp + tile) * QT + row / G;     // this row's query and head
+  const int head = h * G + row % G;
+  const bool row_valid = softmax_thread && s_idx < n_queries;
+  const long long row_off = ((bl * n_queries + s_idx) * g.Hq + head);
+  if (n == 0) {                                         // empty cache: zeros, log-sum-exp = -inf
+    if (row_valid) {
+      for (int d = 0; d < D; ++d) out[row_off * D + d] = 0.f;
+      if (lse_out) lse_out[row_off] = -INFINITY;
+    }
+    return;
+  }
+  // A wait that gave up in an earlier CTA marks the workspace; the rest of the grid leaves.
+  if (status_word && *reinterpret_cast<volatile int32_t*>(status_word + 2) != 0) return;
+  const int nb = (n + kPf3Sub - 1) / kPf3Sub;
+
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;   // 1024-byte aligned tiles
+  const uint32_t sQ = base + (uint32_t)tile * kPfTileBytes;      // this query tile's rows
+  const uint32_t sK = base + 2 * kPfTileBytes, sV = sK + NS * kPf3Tile;
+  const uint32_t bar0 = smem_u32(&s_bar[0]);
+  auto bar_k = [&](int i) { return bar0 + 8u * (uint32_t)i; };
+  auto bar_v = [&](int i) { return bar0 + 8u * (uint32_t)(NS + i); };
+  auto bar_kfree = [&](int i) { return bar0 + 8u * (uint32_t)(2 * NS + i); };
+  auto bar_vfree = [&](int i) { return bar0 + 8u * (uint32_t)(3 * NS + i); };
+  const uint32_t bar_t = bar0 + 8u * (uint32_t)(4 * NS + 5 * tile);   // this query tile's five
+  auto bar_s = [&](int i) { return bar_t + 8u * (uint32_t)i; };
+  auto bar_p = [&](int i) { return bar_t + 8u * (uint32_t)(2 + i); };
+  const uint32_t bar_o = bar_t + 32u;
+
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 :: "r"(smem_u32(&s_tmem)), "r"(kPf4TmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  if (tid == 0) {
+    for (int i = 0; i < 2 * NS; ++i) mbar_init(bar0 + 8u * i, 1);
+    for (int i = 2 * NS; i < 4 * NS; ++i) mbar_init(bar0 + 8u * i, n_tiles);   // one commit per query tile
+    for (int t = 0; t < 2; ++t) {
+      const uint32_t bt = bar0 + 8u * (uint32_t)(4 * NS + 5 * t);
+      mbar_init(bt, 1); mbar_init(bt + 8, 1);
+      mbar_init(bt + 16, kPfRows); mbar_init(bt + 24, kPfRows);
+      mbar_init(bt + 32, 1);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    s_fail = 0;
+  }
+  __syncwarp();
+  if (softmax_thread) {                                 // Q rows, K-major, 128-byte swizzle
+    const uint4* src = reinterpret_cast<const uint4*>(q + row_off * D);
+#pragma unroll
+    for (int c = 0; c < 16; ++c) {
+      const uint4 v = row_valid ? src[c] : make_uint4(0, 0, 0, 0);
+      st_shared16(sQ + (c >> 3) * kPfHalf + row * 128 + (((c & 7) ^ (row & 7)) << 4), v.x, v.y, v.z, v.w);
+    }
+  }
+  proxy_fence();
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = s_tmem + (uint32_t)tile * 256;  // this query tile's 256 columns
+  bool gave_up = false;
+  float m_ref = -INFINITY, l_run = 0.f;                 // reference maximum; sum of this row's weights
+  const uint32_t t_lane = tmem + ((uint32_t)(wq * 32) << 16);
+  const uint32_t t_o = t_lane + 128;                    // this row's 128 output dims
+  const bool tile_active = tile < n_tiles;
+
+  if (!softmax_thread) {
+    if ((tid & 31) == 0 && warp >= 10) {
+      // ---- the two fetching threads: K tiles (warp 10), V tiles (warp 11) ---------------------
+      const bool is_k = warp == 10;
+      const CUtensorMap* map = is_k ? &map_k : &map_v;
+      bool ok = true;
+      for (int j = 0; ok && j < nb; ++j) {
+        const int st = j % NS, use = j / NS;
+        const uint32_t full = is_k ? bar_k(st) : bar_v(st);
+        if (use > 0) ok = mbar_wait<kPfPolls>(is_k ? bar_kfree(st) : bar_vfree(st), (uint32_t)(use - 1) & 1u);
+        if (!ok) break;
+        const uint32_t dst = (is_k ? sK : sV) + st * kPf3Tile;
+        mbar_expect_tx(full, kPf3Tile);
+        tma_load_5d(dst, map, full, 0, j * kPf3Sub, h, l, b);
+        tma_load_5d(dst + kPf3Half, map, full, 64, j * kPf3Sub, h, l, b);
+      }
+      if (!ok) s_fail = 1;
+    } else if ((tid & 31) == 0 && tile_active) {
+      // ---- the issuing thread of query tile `tile` ---------------------------------------------
+      auto issue_qk = [&](int j) {                      // S[j & 1] = Q K(j)^T; then the K tile is free
+        const uint32_t kt = sK + (j % NS) * kPf3Tile;
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+          umma_bf16(tmem + (j & 1) * 64,
+                    umma_desc(sQ + (k >> 2) * kPfHalf + (k & 3) * 32, 16, 1024),
+                    umma_desc(kt + (k >> 2) * kPf3Half + (k & 3) * 32, 16, 1024), kIdescQK64, k > 0);
+        umma_commit(bar_s(j & 1));
+        umma_commit(bar_kfree(j % NS));
+      };
+      bool ok = mbar_wait<kPfPolls>(bar_k(0), 0);
+      if (ok) { tc_fence_after(); issue_qk(0); }
+      if (ok && nb > 1) {
+        ok = mbar_wait<kPfPolls>(bar_k(1 % NS), 0);
+        if (ok) { tc_fence_after(); issue_qk(1); }
+      }
+      if (ok) ok = mbar_wait<kPfPolls>(bar_v(0), 0);
+      for (int j = 0; ok && j < nb; ++j) {
+        const int s = j & 1;
+        ok = mbar_wait<kPfPolls>(bar_p(s), (uint32_t)(j >> 1) & 1u);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t vt = sV + (j % NS) * kPf3Tile;
+#pragma unroll
+        for (int k = 0; k < 4; ++k)                     // O += P(j) V(j); slice k = tokens 16k .. 16k + 15
+          umma_bf16_ts(tmem + 128, tmem + s * 64 + k * 8,
+                       umma_desc(vt + k * 2048, kPf3Half, 1024), kIdescPV, (j > 0 || k > 0) ? 1u : 0u);
+        umma_commit(bar_o);
+        umma_commit(bar_vfree(j % NS));
+        // tiles fetched well ahead: these two are normally over already
+        if (j + 2 < nb) ok = mbar_wait_likely(bar_k((j + 2) % NS), (uint32_t)((j + 2) / NS) & 1u);
+        if (ok && j + 1 < nb) ok = mbar_wait_likely(bar_v((j + 1) % NS), (uint32_t)((j + 1) / NS) & 1u);
+        // P(j) V(j) done: the score buffer it read its weights from takes sub-block j + 2
+        ok = ok && mbar_wait<kPfPolls>(bar_o, (uint32_t)j & 1u);
+        if (!ok) break;
+        if (j + 2 < nb) { tc_fence_after(); issue_qk(j + 2); }
+      }
+      if (!ok) s_fail = 1;
+    }
+  } else if (tile_active) {
+    // ---- the softmax warps of query tile `tile`: one thread per row ----------------------------
+    for (int j = 0; j < nb; ++j) {
+      const int s = j & 1;
+      const int valid = min(kPf3Sub, n - j * kPf3Sub);       // valid tokens of this sub-block
+      const uint32_t t_s = t_lane + s * 64;                   // this row's scores, later its weights
+      if (!mbar_wait_likely(bar_s(s), (uint32_t)(j >> 1) & 1u)) gave_up = true;
+      tc_fence_after();
+      if (__any_sync(0xffffffffu, gave_up)) { gave_up = true; break; }
+      float sv[64];                                       // raw products; the scale is folded in below
+      float bmax = -INFINITY;
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        uint32_t r[32];
+        tmem_ld32(t_s + c * 32, r);
+        if (valid >= kPf3Sub) {                           // CTA-uniform: only the last sub-block masks
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            sv[c * 32 + i] = __uint_as_float(r[i]);
+            bmax = fmaxf(bmax, sv[c * 32 + i]);
+          }
+        } else {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            sv[c * 32 + i] = c * 32 + i < valid ? __uint_as_float(r[i]) : -INFINITY;
+            bmax = fmaxf(bmax, sv[c * 32 + i]);
+          }
+        }
+      }
+      const float m_new = fmaxf(m_ref, bmax * scale_log2e);   // scale > 0: the maximum commutes with it
+      if (j == 0) m_ref = m_new;
+      // ---- rescale O only when this row's maximum has drifted far from the reference --------
+      const bool need = m_new > m_ref + kPfRescaleGap;
+      if (__any_sync(0xffffffffu, need)) {
+        // O must be quiet: P(j-1) V(j-1) has to be complete (P(j) V(j) waits for this thread)
+        if (!mbar_wait<kPfPolls>(bar_o, (uint32_t)(j - 1) & 1u)) gave_up = true;
+        tc_fence_after();
+        const float factor = need ? fast_exp2(m_ref - m_new) : 1.f;
+#pragma unroll 1
+        for (int c = 0; c < D; c += 8) tmem_scale8(t_o + c, factor);
+        if (need) { l_run *= factor; m_ref = m_new; }
+      }
+      // ---- weights 2^(s - m_ref) as bf16 pairs over the first half of the score columns -----
+      {
+        uint32_t pk[32];
+        float rowsum0 = 0.f, rowsum1 = 0.f;
+        const float neg_m = -m_ref;
+#pragma unroll
+        for (int i = 0; i < 64; i += 2) {
+          const float p0 = fast_exp2(__fmaf_rn(sv[i], scale_log2e, neg_m));     // -inf -> 0
+          const float p1 = fast_exp2(__fmaf_rn(sv[i + 1], scale_log2e, neg_m));
+          rowsum0 += p0;
+          rowsum1 += p1;
+          pk[i >> 1] = pack_bf16(p0, p1);
+        }
+        tmem_st32(t_s, pk);
+        tmem_wait_st();
+        l_run += rowsum0 + rowsum1;
+      }
+      if (valid < kPf3Sub) {
+        // Last, partial sub-block: rows of the V tile past the valid length hold whatever the
+        // cache holds there; clear them so that a zero weight times Inf/NaN cannot reach O
+        // (both query tiles write the same zeros).
+        if (!mbar_wait<kPfPolls>(bar_v(j % NS), (uint32_t)(j / NS) & 1u)) gave_up = true;
+        if (row >= valid && row < kPf3Sub) {
+#pragma unroll
+          for (int c = 0; c < 16; ++c)
+            st_shared16(sV + (j % NS) * kPf3Tile + (c >> 3) * kPf3Half + row * 128 + ((c & 7) << 4), 0, 0, 0, 0);
+        }
+        proxy_fence();
+      }
+      tc_fence_before();
+      mbar_arrive(bar_p(s));                              // this row's weights (and O) are in place
+    }
+    // O is complete when the last P V has been committed
+    if (!gave_up && !mbar_wait<kPfPolls>(bar_o, (uint32_t)(nb - 1) & 1u)) gave_up = true;
+    if (gave_up) s_fail = 1;
+  }
+  __syncthreads();                                       // every role is done with the loop
+  tc_fence_after();
+  const bool failed = s_fail != 0;
+  const float l_tot = l_run;
+  if (!failed && softmax_thread && tile_active) {
+    const float inv = 1.f / l_tot;
+#pragma unroll 1
+    for (int c = 0; c < 4; ++c) {
+      uint32_t r[32];
+      tmem_ld32(t_o + c * 32, r);
+      if (row_valid) {
+        float4* dst = reinterpret_cast<float4*>(out + row_off * D + c * 32);
+#pragma unroll
+        for (int i = 0; i < 32; i += 4)
+          dst[i >> 2] = make_float4(__uint_as_float(r[i]) * inv, __uint_as_float(r[i + 1]) * inv,
+                                    __uint_as_float(r[i + 2]) * inv, __uint_as_float(r[i + 3]) * inv);
+      }
+    }
+    if (row_valid && lse_out)
+      lse_out[row_off] = (m_ref + log2f(l_tot)) * 0.6931471805599453f;
+  }
+  if (failed && tid == 0 && status_word) {
+    atomicExch(status_word, (int)L2KV_ERR_CUDA);
+    atomicExch(status_word + 2, 1);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0)
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(s_tmem), "r"(kPf4TmemCols)
+                 : "memory");
+}
+
 template <int G>
 static int launch_pf(const void* q, const void* K, const void* V, const Geom& g, int n_queries,
                      const int32_t* cur_len_dev, int max_len, float scale, float* out,
@@ -1217,7 +1488,8 @@ static int launch_pf(const void* q, const void* K, const void* V, const Geom& g,
   const char* which = std::getenv("L2KV_PREFIX_KERNEL");
   const bool v1 = which && std::strcmp(which, "v1") == 0;
   const bool v3 = which && std::strcmp(which, "v3") == 0;
-  const bool v4 = which && std::strcmp(which, "v4") == 0;
+  const bool v5 = which && std::strcmp(which, "v5") == 0;
+  const bool v4 = v5 || (which && std::strcmp(which, "v4") == 0);
   const int sub_rows = (v3 || v4) ? kPf3Sub : kPfRows;
   if (!make_cache_map(&map_k, K, g, sub_rows) || !make_cache_map(&map_v, V, g, sub_rows))
     return L2KV_ERR_UNSUPPORTED;
@@ -1225,10 +1497,10 @@ static int launch_pf(const void* q, const void* K, const void* V, const Geom& g,
     constexpr int smem4 = 1024 + 2 * kPfTileBytes + 2 * kPf4Stages * kPf3Tile;
     const int q_tiles = (n_queries + QT - 1) / QT;
     const long long blocks4 = units * ((q_tiles + 1) / 2);
-    auto kern4 = prefix_attention_kernel_v4<G>;
+    auto kern4 = v5 ? prefix_attention_kernel_v5<G> : prefix_attention_kernel_v4<G>;
     if (cudaFuncSetAttribute(kern4, cudaFuncAttributeMaxDynamicSharedMemorySize, smem4) != cudaSuccess)
       return L2KV_ERR_CUDA;
-    kern4<<<(unsigned)blocks4, kPf4Threads, smem4, s>>>(
+    kern4<<<(unsigned)blocks4, v5 ? kPf5Threads : kPf4Threads, smem4, s>>>(
         static_cast<const __nv_bfloat16*>(q), g, n_queries, cur_len_dev, max_len, scale * kPfLog2e, out,
         lse_out, map_k, map_v, status_word);
     return cudaGetLastError() == cudaSuccess ? L2KV_OK : L2KV_ERR_CUDA;

@@ -32,10 +32,10 @@ def run(l2, q, K, V, cur, max_len, scale=0.0):
     return out.cpu().numpy(), lse.cpu().numpy()
 
 
-KERNELS = ["v2", "v1", "v3", "v4"]      # the formulations of the kernel; v2 is the default
+KERNELS = ["v2", "v1", "v3", "v4", "v5"]      # the formulations of the kernel; v2 is the default
 
 
-@pytest.mark.parametrize("kernel", ["v2", "v3", "v4"])
+@pytest.mark.parametrize("kernel", ["v2", "v3", "v4", "v5"])
 @pytest.mark.parametrize("Hkv,Hq,n_q,T", [(2, 8, 40, 300), (2, 2, 130, 257), (1, 8, 1, 1000),
                                           (2, 4, 64, 128)])
 def test_prefix_attention_matches_oracle(Hkv, Hq, n_q, T, kernel, monkeypatch):
