@@ -3,15 +3,15 @@
 // 4 * Sq * Hq * D flop per cached token per (b, l) -- so it runs on the Blackwell tensor cores
 // (tcgen05.mma, operands in shared memory, accumulators in tensor memory).
 //
-// One CTA (256 threads, two per row) per (b, l, kv head, tile of 128 / G queries): its 128 rows are the
-// (query, head-of-the-group) pairs that share one KV head.  Per block of 128 cached tokens:
+// A query tile is 128 rows: the (query, head-of-the-group) pairs of 128 / G queries that share
+// one KV head.  For every block of cached tokens
 //   K block  -- TMA --> shared memory (128-byte swizzle)
-//   S = Q . K^T            8 x tcgen05.mma (M 128, N 128, K 16), fp32 in tensor memory
-//   the two threads of row r read it from S (tcgen05.ld): running maximum, weights 2^(s - m) as bf16 back
-//   to shared memory (over the K block, which is no longer needed), running sum
-//   V block  -- TMA --> shared memory;  O_blk = P . V   8 x tcgen05.mma (V as an N-major operand)
-//   thread r reads row r of O_blk and folds it into its fp32 accumulator row (rescaled by
-//   2^(m_old - m_new)), FlashAttention style.
+//   S = Q . K^T             tcgen05.mma (M 128, K 16 per instruction), fp32 in tensor memory
+//   softmax threads read their rows of S (tcgen05.ld): running maximum, weights 2^(s - m) as
+//   bf16 pairs written back over the score columns (tcgen05.st), running sum
+//   V block  -- TMA --> shared memory;  O += P . V   tcgen05.mma with A in tensor memory and V as
+//   an N-major operand; O stays in tensor memory and is rescaled only when a maximum has drifted.
+// Two kernels share these pieces: the pipelined one (default) and a basic single-role one.
 // Every wait on an mbarrier is bounded (a wait that gives up ends the CTA's loop and marks
 // the status word); tensor memory is released on every path.
 #include <cstdlib>
@@ -21,11 +21,11 @@
 
 namespace l2kv {
 
-constexpr int kPfThreads = 256;                // two threads per query row
+constexpr int kPfThreads = 256;                // basic kernel: two threads per query row
 constexpr int kPfRows = 128;                    // query rows per CTA, cached tokens per block
 constexpr int kPfHalf = kPfRows * 128;          // one [128 rows][64 bf16] swizzled tile: 16 KB
 constexpr int kPfTileBytes = 2 * kPfHalf;       // both halves of the head dimension: 32 KB
-constexpr int kPfTmemCols = 256;                // S: columns 0..127, O_blk: columns 128..255
+constexpr int kPfTmemCols = 256;                // basic kernel: S in columns 0..127, O in 128..255
 constexpr int kPfPolls = 18;                    // log2 of the polls a wait may take
 constexpr float kPfLog2e = 1.4426950408889634f;
 
@@ -108,225 +108,6 @@ __device__ __forceinline__ float fast_exp2(float x) {
   return y;
 }
 
-template <int G>
-__global__ void __launch_bounds__(kPfThreads, 2)
-prefix_attention_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n_queries,
-                        const int32_t* __restrict__ cur_len_dev, int max_len, float scale_log2e,
-                        float* __restrict__ out, float* __restrict__ lse_out,
-                        const __grid_constant__ CUtensorMap map_k,
-                        const __grid_constant__ CUtensorMap map_v, int32_t* __restrict__ status_word) {
-  constexpr int D = 128;
-  constexpr int QT = kPfRows / G;                       // queries per CTA
-  extern __shared__ unsigned char smem_raw[];
-  __shared__ __align__(8) unsigned long long s_bar[3];  // K landed, V landed, MMA done
-  __shared__ uint32_t s_tmem;
-  __shared__ int s_fail;
-  __shared__ float s_x[2][kPfRows];                     // row maxima / sums of the two column halves
-
-  const int q_tiles = (n_queries + QT - 1) / QT;
-  const int qt = blockIdx.x % q_tiles;
-  const long long unit = blockIdx.x / q_tiles;          // (b * L + l) * H + h
-  const int h = (int)(unit % g.H);
-  const long long bl = unit / g.H;
-  const int l = (int)(bl % g.L), b = (int)(bl / g.L);
-  const int n = max(0, min(cur_len_dev[bl], min(max_len, g.t_cap)));
-  // Two threads per query row: thread (row, hf) owns score columns and output dims
-  // [64 hf, 64 hf + 64).  Warps w and w + 4 share a tensor-memory lane quarter.
-  const int tid = threadIdx.x, warp = tid >> 5;
-  const int row = tid & (kPfRows - 1), hf = tid >> 7;
-  const int s_idx = qt * QT + row / G;                  // this row's query and head
-  const int head = h * G + row % G;
-  const bool row_valid = s_idx < n_queries;
-  const long long row_off = ((bl * n_queries + s_idx) * g.Hq + head);
-  if (n == 0) {                                         // empty cache: zeros, log-sum-exp = -inf
-    if (row_valid) {
-      for (int d = 0; d < 64; ++d) out[row_off * D + hf * 64 + d] = 0.f;
-      if (lse_out && hf == 0) lse_out[row_off] = -INFINITY;
-    }
-    return;
-  }
-  // A wait that gave up in an earlier CTA marks the workspace; the rest of the grid leaves.
-  if (status_word && *reinterpret_cast<volatile int32_t*>(status_word + 2) != 0) return;
-  const int n_blocks = (n + kPfRows - 1) / kPfRows;
-
-  // Tiles start on a 1024-byte boundary (the period of the 128-byte swizzle, which the matrix
-  // descriptors assume).
-  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t sQ = base, sKP = base + kPfTileBytes, sV = base + 2 * kPfTileBytes;
-  const uint32_t bar_k = smem_u32(&s_bar[0]), bar_v = smem_u32(&s_bar[1]), bar_m = smem_u32(&s_bar[2]);
-
-  if (warp == 0) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                 :: "r"(smem_u32(&s_tmem)), "r"(kPfTmemCols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  }
-  if (tid == 0) {
-    mbar_init(bar_k, 1); mbar_init(bar_v, 1); mbar_init(bar_m, 1);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    s_fail = 0;
-  }
-  __syncwarp();
-  // Q rows of this tile into shared memory, K-major with the 128-byte swizzle (this thread:
-  // the eight 16-byte pieces of half hf of its row).
-  {
-    const uint4* src = reinterpret_cast<const uint4*>(q + row_off * D) + hf * 8;
-#pragma unroll
-    for (int c = 0; c < 8; ++c) {
-      const uint4 v = row_valid ? src[c] : make_uint4(0, 0, 0, 0);
-      st_shared16(sQ + hf * kPfHalf + row * 128 + ((c ^ (row & 7)) << 4), v.x, v.y, v.z, v.w);
-    }
-  }
-  proxy_fence();
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem = s_tmem;
-  const uint32_t t_row = tmem + ((uint32_t)((warp & 3) * 32) << 16) + hf * 64;   // lane quarter, column half
-
-  auto load_block = [&](int kb) {                       // thread 0 only
-    mbar_expect_tx(bar_k, kPfTileBytes);
-    tma_load_5d(sKP, &map_k, bar_k, 0, kb * kPfRows, h, l, b);
-    tma_load_5d(sKP + kPfHalf, &map_k, bar_k, 64, kb * kPfRows, h, l, b);
-    mbar_expect_tx(bar_v, kPfTileBytes);
-    tma_load_5d(sV, &map_v, bar_v, 0, kb * kPfRows, h, l, b);
-    tma_load_5d(sV + kPfHalf, &map_v, bar_v, 64, kb * kPfRows, h, l, b);
-  };
-  if (tid == 0) load_block(0);
-  __syncwarp();
-
-  float o[64];
-#pragma unroll
-  for (int d = 0; d < 64; ++d) o[d] = 0.f;
-  float m_run = -INFINITY, l_run = 0.f, l_exact = 0.f;  // sums (of this half) of rounded / unrounded weights
-  uint32_t mma_phase = 0;
-
-  for (int kb = 0; kb < n_blocks; ++kb) {
-    const int valid = min(kPfRows, n - kb * kPfRows) - hf * 64;   // valid tokens among this thread's 64
-    // ---- S = Q K^T ---------------------------------------------------------------------
-    if (tid == 0) {
-      if (!mbar_wait<kPfPolls>(bar_k, kb & 1)) s_fail = 1;
-      tc_fence_after();
-#pragma unroll
-      for (int k = 0; k < 8; ++k) {
-        const uint32_t off = (k >> 2) * kPfHalf + (k & 3) * 32;
-        umma_bf16(tmem, umma_desc(sQ + off, 16, 1024), umma_desc(sKP + off, 16, 1024), kIdescQK, k > 0);
-      }
-      umma_commit(bar_m);
-      if (!mbar_wait<kPfPolls>(bar_m, mma_phase)) s_fail = 1;
-    }
-    mma_phase ^= 1;
-    __syncthreads();                                    // S is complete (thread 0 saw the commit)
-    if (s_fail) break;
-    tc_fence_after();
-    // ---- softmax of this thread's half row -------------------------------------------------
-    float bmax = -INFINITY;
-#pragma unroll
-    for (int c = 0; c < 2; ++c) {
-      uint32_t r[32];
-      tmem_ld32(t_row + c * 32, r);
-#pragma unroll
-      for (int i = 0; i < 32; ++i)
-        if (c * 32 + i < valid) bmax = fmaxf(bmax, __uint_as_float(r[i]));
-    }
-    s_x[hf][row] = bmax * scale_log2e;                  // scale > 0: the maximum commutes with it
-    __syncthreads();
-    const float m_new = fmaxf(m_run, fmaxf(s_x[0][row], s_x[1][row]));
-    const float alpha = fast_exp2(m_run - m_new);       // 0 on the first block
-    float rowsum = 0.f, rowsum_exact = 0.f;
-#pragma unroll
-    for (int c = 0; c < 2; ++c) {
-      uint32_t r[32];
-      tmem_ld32(t_row + c * 32, r);
-      uint32_t pk[16];
-#pragma unroll
-      for (int i = 0; i < 32; i += 2) {
-        const float p0 = c * 32 + i < valid ? fast_exp2(fmaf(__uint_as_float(r[i]), scale_log2e, -m_new)) : 0.f;
-        const float p1 = c * 32 + i + 1 < valid ? fast_exp2(fmaf(__uint_as_float(r[i + 1]), scale_log2e, -m_new)) : 0.f;
-        const __nv_bfloat162 pr = __floats2bfloat162_rn(p0, p1);
-        // The sum is taken over the rounded weights, the ones V is multiplied with, so that
-        // numerator and denominator stay consistent (a dominant token still gives its V row).
-        rowsum += __low2float(pr) + __high2float(pr);
-        rowsum_exact += p0 + p1;
-        pk[i >> 1] = *reinterpret_cast<const uint32_t*>(&pr);
-      }
-      // tokens 64 hf + 32 c .. + 31 of this row: four 16-byte pieces of the swizzled P tile
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const int ch = c * 4 + j;                       // piece index 0..7 inside half hf
-        st_shared16(sKP + hf * kPfHalf + row * 128 + ((ch ^ (row & 7)) << 4),
-                    pk[4 * j], pk[4 * j + 1], pk[4 * j + 2], pk[4 * j + 3]);
-      }
-    }
-    l_run = l_run * alpha + rowsum;
-    l_exact = l_exact * alpha + rowsum_exact;
-    m_run = m_new;
-    // ---- O_blk = P V -----------------------------------------------------------------------
-    if (tid == 0 && !mbar_wait<kPfPolls>(bar_v, kb & 1)) s_fail = 1;
-    __syncthreads();                                    // V landed (thread 0 saw it)
-    if (s_fail) break;
-    if (row >= min(kPfRows, n - kb * kPfRows)) {
-      // Rows past the valid length hold whatever the cache holds there: clear them so that a
-      // zero weight times Inf/NaN cannot reach the accumulators.
-#pragma unroll
-      for (int c = 0; c < 8; ++c) st_shared16(sV + hf * kPfHalf + row * 128 + (c << 4), 0, 0, 0, 0);
-    }
-    proxy_fence();                                      // P (and cleared rows) visible to the MMA
-    tc_fence_before();
-    __syncthreads();
-    if (tid == 0) {
-      tc_fence_after();
-#pragma unroll
-      for (int k = 0; k < 8; ++k) {
-        umma_bf16(tmem + 128, umma_desc(sKP + (k >> 2) * kPfHalf + (k & 3) * 32, 16, 1024),
-                  umma_desc(sV + k * 2048, kPfHalf, 1024), kIdescPV, k > 0);
-      }
-      umma_commit(bar_m);
-      if (!mbar_wait<kPfPolls>(bar_m, mma_phase)) s_fail = 1;
-      else if (kb + 1 < n_blocks) load_block(kb + 1);   // both buffers are free again
-    }
-    mma_phase ^= 1;
-    __syncthreads();                                    // O_blk is complete
-    if (s_fail) break;
-    tc_fence_after();
-#pragma unroll
-    for (int c = 0; c < 2; ++c) {
-      uint32_t r[32];
-      tmem_ld32(t_row + 128 + c * 32, r);
-#pragma unroll
-      for (int i = 0; i < 32; ++i) o[c * 32 + i] = fmaf(o[c * 32 + i], alpha, __uint_as_float(r[i]));
-    }
-    tc_fence_before();
-    __syncthreads();                                    // tensor memory free for the next block
-  }
-
-  const bool failed = s_fail != 0;
-  // the two halves of a row share the maximum; their weight sums add up
-  __syncthreads();
-  s_x[hf][row] = l_run;
-  __syncthreads();
-  const float l_tot = s_x[0][row] + s_x[1][row];
-  __syncthreads();
-  s_x[hf][row] = l_exact;
-  __syncthreads();
-  const float l_tot_exact = s_x[0][row] + s_x[1][row];
-  if (row_valid && !failed) {
-    const float inv = 1.f / l_tot;
-    float4* dst = reinterpret_cast<float4*>(out + row_off * D + hf * 64);
-#pragma unroll
-    for (int d = 0; d < 64; d += 4) dst[d >> 2] = make_float4(o[d] * inv, o[d + 1] * inv, o[d + 2] * inv, o[d + 3] * inv);
-    if (lse_out && hf == 0) lse_out[row_off] = (m_run + log2f(l_tot_exact)) * 0.6931471805599453f;
-  }
-  if (failed && tid == 0 && status_word) {
-    atomicExch(status_word, (int)L2KV_ERR_CUDA);
-    atomicExch(status_word + 2, 1);
-  }
-  tc_fence_before();
-  __syncthreads();
-  if (warp == 0)
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem), "r"(kPfTmemCols)
-                 : "memory");
-}
-
 // Eight columns at a time: the rarely taken rescaling of O, kept small in registers.
 __device__ __forceinline__ void tmem_scale8(uint32_t taddr, float factor) {
   uint32_t r0, r1, r2, r3, r4, r5, r6, r7;
@@ -343,18 +124,19 @@ __device__ __forceinline__ void tmem_scale8(uint32_t taddr, float factor) {
                : "memory");
 }
 
-// Second formulation of the same kernel, the one the entry point uses: the weights never go
-// to shared memory.  They are written as bf16 pairs into the tensor-memory columns that held
-// the scores and feed the second contraction from there (tcgen05.mma with A in tensor
-// memory), the output accumulates in tensor memory across blocks and is rescaled only when
-// a row's maximum has grown by more than 2^8 since the last rescale (weights stay <= 2^8, well
-// inside bf16 / fp32 range), and K and V each have their own shared-memory tile, so the next
-// K block is fetched while the softmax and the second contraction of the current one run.
+// The basic kernel (L2KV_PREFIX_KERNEL=basic): one role, two CTAs per SM that fill each other's
+// gaps.  The weights never go to shared memory: they are written as bf16 pairs into the
+// tensor-memory columns that held the scores and feed the second contraction from there
+// (tcgen05.mma with A in tensor memory); the output accumulates in tensor memory across
+// blocks and is rescaled only when a row's maximum has grown by more than 2^8 since the last
+// rescale (weights stay <= 2^8, well inside bf16 / fp32 range); K and V each have their own
+// shared-memory tile, so the next K block is fetched while the softmax and the second
+// contraction of the current one run.
 constexpr float kPfRescaleGap = 8.f;            // log2 units a maximum may drift before O is rescaled
 
 template <int G>
 __global__ void __launch_bounds__(kPfThreads, 2)
-prefix_attention_kernel_v2(const __nv_bfloat16* __restrict__ q, Geom g, int n_queries,
+prefix_attention_basic_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n_queries,
                            const int32_t* __restrict__ cur_len_dev, int max_len, float scale_log2e,
                            float* __restrict__ out, float* __restrict__ lse_out,
                            const __grid_constant__ CUtensorMap map_k,
@@ -581,322 +363,18 @@ prefix_attention_kernel_v2(const __nv_bfloat16* __restrict__ q, Geom g, int n_qu
                  : "memory");
 }
 
-// Third formulation: the two contractions and the softmax run concurrently.  A ninth warp
-// does nothing but fetch tiles and issue tcgen05.mma; the cache is walked in sub-blocks of
-// 64 tokens with two score buffers in tensor memory, so that S(j+1) = Q K(j+1)^T is computed
-// while the eight softmax warps work on S(j), and O += P(j) V(j) runs while they work on
-// S(j+1).  Hand-offs are mbarriers (scores ready: tcgen05.commit; weights ready: one arrival
-// per softmax thread; output quiet: tcgen05.commit), every wait on them is bounded.
-constexpr int kPf3Threads = kPfThreads + 32;    // eight softmax warps + the issuing warp
+// The pipelined kernel walks the cache in sub-blocks of 64 tokens.
 constexpr int kPf3Sub = 64;                     // cached tokens per sub-block
 constexpr int kPf3Half = kPf3Sub * 128;         // one [64 tokens][64 bf16] swizzled tile: 8 KB
 constexpr int kPf3Tile = 2 * kPf3Half;          // both halves of the head dimension: 16 KB
 constexpr uint32_t kIdescQK64 =
     (1u << 4) | (1u << 7) | (1u << 10) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
+constexpr int kPf4Stages = 4;                   // K tiles (and V tiles) in flight
+constexpr int kPf4TmemCols = 512;
 
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(bar) : "memory");
 }
-// Stores 16 consecutive 32-bit columns of this thread's tensor-memory lane.  Whole warps only.
-__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
-  asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
-               "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
-               :: "r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]),
-                  "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]),
-                  "r"(r[14]), "r"(r[15])
-               : "memory");
-}
-// Barrier among the 64 threads of warps w and w + 4 (the two halves of 32 query rows).
-__device__ __forceinline__ void pair_sync(int quarter) {
-  switch (quarter) {                                    // immediate ids: four named barriers in all
-    case 0: asm volatile("bar.sync 1, 64;" ::: "memory"); break;
-    case 1: asm volatile("bar.sync 2, 64;" ::: "memory"); break;
-    case 2: asm volatile("bar.sync 3, 64;" ::: "memory"); break;
-    default: asm volatile("bar.sync 4, 64;" ::: "memory"); break;
-  }
-}
-
-template <int G>
-__global__ void __launch_bounds__(kPf3Threads, 2)
-prefix_attention_kernel_v3(const __nv_bfloat16* __restrict__ q, Geom g, int n_queries,
-                           const int32_t* __restrict__ cur_len_dev, int max_len, float scale_log2e,
-                           float* __restrict__ out, float* __restrict__ lse_out,
-                           const __grid_constant__ CUtensorMap map_k,
-                           const __grid_constant__ CUtensorMap map_v,
-                           int32_t* __restrict__ status_word) {
-  constexpr int D = 128;
-  constexpr int QT = kPfRows / G;                       // queries per CTA
-  extern __shared__ unsigned char smem_raw[];
-  // [0,1] K tile landed, [2,3] V tile landed, [4,5] scores ready, [6,7] weights ready, [8] O quiet
-  __shared__ __align__(8) unsigned long long s_bar[9];
-  __shared__ uint32_t s_tmem;
-  __shared__ int s_fail;
-  __shared__ float s_x[2][2][kPfRows];                  // [sub-block parity][half][row]
-  __shared__ int s_flag[2][8];                          // [sub-block parity][softmax warp] gave up
-
-  const int q_tiles = (n_queries + QT - 1) / QT;
-  const int qt = blockIdx.x % q_tiles;
-  const long long unit = blockIdx.x / q_tiles;          // (b * L + l) * H + h
-  const int h = (int)(unit % g.H);
-  const long long bl = unit / g.H;
-  const int l = (int)(bl % g.L), b = (int)(bl / g.L);
-  const int n = max(0, min(cur_len_dev[bl], min(max_len, g.t_cap)));
-  const int tid = threadIdx.x, warp = tid >> 5;
-  const bool softmax_thread = tid < kPfThreads;
-  // Softmax threads, two per query row: thread (row, hf) owns 32 of a sub-block's 64 score
-  // columns and output dims [64 hf, 64 hf + 64).  Warps w and w + 4 share a lane quarter.
-  const int row = tid & (kPfRows - 1), hf = (tid >> 7) & 1;
-  const int s_idx = qt * QT + row / G;                  // this row's query and head
-  const int head = h * G + row % G;
-  const bool row_valid = softmax_thread && s_idx < n_queries;
-  const long long row_off = ((bl * n_queries + s_idx) * g.Hq + head);
-  if (n == 0) {                                         // empty cache: zeros, log-sum-exp = -inf
-    if (row_valid) {
-      for (int d = 0; d < 64; ++d) out[row_off * D + hf * 64 + d] = 0.f;
-      if (lse_out && hf == 0) lse_out[row_off] = -INFINITY;
-    }
-    return;
-  }
-  // A wait that gave up in an earlier CTA marks the workspace; the rest of the grid leaves.
-  if (status_word && *reinterpret_cast<volatile int32_t*>(status_word + 2) != 0) return;
-  const int nb = (n + kPf3Sub - 1) / kPf3Sub;
-
-  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;   // 1024-byte aligned tiles
-  const uint32_t sQ = base, sK = base + kPfTileBytes, sV = sK + 2 * kPf3Tile;
-  const uint32_t bar0 = smem_u32(&s_bar[0]);
-  auto bar_k = [&](int i) { return bar0 + 8u * (uint32_t)i; };
-  auto bar_v = [&](int i) { return bar0 + 8u * (uint32_t)(2 + i); };
-  auto bar_s = [&](int i) { return bar0 + 8u * (uint32_t)(4 + i); };
-  auto bar_p = [&](int i) { return bar0 + 8u * (uint32_t)(6 + i); };
-  const uint32_t bar_o = bar0 + 64u;
-
-  if (warp == 0) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                 :: "r"(smem_u32(&s_tmem)), "r"(kPfTmemCols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  }
-  if (tid == 0) {
-    for (int i = 0; i < 6; ++i) mbar_init(bar0 + 8u * i, 1);
-    mbar_init(bar_p(0), kPfThreads);
-    mbar_init(bar_p(1), kPfThreads);
-    mbar_init(bar_o, 1);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    s_fail = 0;
-  }
-  __syncwarp();
-  if (softmax_thread) {                                 // Q rows, K-major, 128-byte swizzle
-    const uint4* src = reinterpret_cast<const uint4*>(q + row_off * D) + hf * 8;
-#pragma unroll
-    for (int c = 0; c < 8; ++c) {
-      const uint4 v = row_valid ? src[c] : make_uint4(0, 0, 0, 0);
-      st_shared16(sQ + hf * kPfHalf + row * 128 + ((c ^ (row & 7)) << 4), v.x, v.y, v.z, v.w);
-    }
-  }
-  proxy_fence();
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem = s_tmem;
-  bool gave_up = false;
-  float m_ref = -INFINITY, l_run = 0.f;                 // reference maximum; sum of this half's weights
-  const uint32_t t_lane = tmem + ((uint32_t)((warp & 3) * 32) << 16);   // this warp's lane quarter
-  const uint32_t t_o = t_lane + 128 + hf * 64;          // this thread's 64 output dims
-
-  if (!softmax_thread) {
-    // ---- the issuing warp: one lane fetches tiles and issues every contraction ---------------
-    if (tid == kPfThreads) {
-      auto load_k = [&](int j) {
-        const uint32_t dst = sK + (j & 1) * kPf3Tile;
-        mbar_expect_tx(bar_k(j & 1), kPf3Tile);
-        tma_load_5d(dst, &map_k, bar_k(j & 1), 0, j * kPf3Sub, h, l, b);
-        tma_load_5d(dst + kPf3Half, &map_k, bar_k(j & 1), 64, j * kPf3Sub, h, l, b);
-      };
-      auto load_v = [&](int j) {
-        const uint32_t dst = sV + (j & 1) * kPf3Tile;
-        mbar_expect_tx(bar_v(j & 1), kPf3Tile);
-        tma_load_5d(dst, &map_v, bar_v(j & 1), 0, j * kPf3Sub, h, l, b);
-        tma_load_5d(dst + kPf3Half, &map_v, bar_v(j & 1), 64, j * kPf3Sub, h, l, b);
-      };
-      auto issue_qk = [&](int j) {                      // S[j & 1] = Q K(j)^T, then signal
-        const uint32_t kt = sK + (j & 1) * kPf3Tile;
-#pragma unroll
-        for (int k = 0; k < 8; ++k)
-          umma_bf16(tmem + (j & 1) * 64,
-                    umma_desc(sQ + (k >> 2) * kPfHalf + (k & 3) * 32, 16, 1024),
-                    umma_desc(kt + (k >> 2) * kPf3Half + (k & 3) * 32, 16, 1024), kIdescQK64, k > 0);
-        umma_commit(bar_s(j & 1));
-      };
-      bool ok = true;
-      load_k(0); load_v(0);
-      if (nb > 1) { load_k(1); load_v(1); }
-      ok = mbar_wait<kPfPolls>(bar_k(0), 0);
-      if (ok) { tc_fence_after(); issue_qk(0); }
-      if (ok && nb > 1) {
-        ok = mbar_wait<kPfPolls>(bar_k(1), 0);
-        if (ok) { tc_fence_after(); issue_qk(1); }
-      }
-      if (ok && nb > 2) {                               // the first K tile is free once S(0) is done
-        ok = mbar_wait<kPfPolls>(bar_s(0), 0);
-        if (ok) load_k(2);
-      }
-      if (ok) ok = mbar_wait<kPfPolls>(bar_v(0), 0);
-      // Waits that are expected to be over already (tiles fetched an iteration ago) are placed
-      // where this thread would otherwise idle: under the contraction it has just issued.
-      for (int j = 0; ok && j < nb; ++j) {
-        const int s = j & 1;
-        ok = mbar_wait<kPfPolls>(bar_p(s), (uint32_t)(j >> 1) & 1u);
-        if (!ok) break;
-        tc_fence_after();
-        const uint32_t vt = sV + s * kPf3Tile;
-#pragma unroll
-        for (int k = 0; k < 4; ++k)                     // O += P(j) V(j); slice k = tokens 16k .. 16k + 15
-          umma_bf16_ts(tmem + 128, tmem + s * 64 + (k >> 1) * 32 + (k & 1) * 8,
-                       umma_desc(vt + k * 2048, kPf3Half, 1024), kIdescPV, (j > 0 || k > 0) ? 1u : 0u);
-        umma_commit(bar_o);
-        if (j + 2 < nb) ok = mbar_wait<kPfPolls>(bar_k(s), (uint32_t)((j + 2) >> 1) & 1u);
-        if (ok && j + 1 < nb) ok = mbar_wait<kPfPolls>(bar_v(s ^ 1), (uint32_t)((j + 1) >> 1) & 1u);
-        // P(j) V(j) done: its V tile and score buffer are free for sub-block j + 2, and so is
-        // the K tile of Q K(j+1)^T, which was issued before it (a commit covers all earlier ones).
-        ok = ok && mbar_wait<kPfPolls>(bar_o, (uint32_t)j & 1u);
-        if (!ok) break;
-        if (j + 2 < nb) {
-          tc_fence_after();
-          issue_qk(j + 2);
-          load_v(j + 2);
-        }
-        if (j + 3 < nb) load_k(j + 3);
-      }
-      if (!ok) s_fail = 1;
-    }
-  } else {
-    // ---- the softmax warps -------------------------------------------------------------------
-    for (int j = 0; j < nb; ++j) {
-      const int s = j & 1;
-      const int valid_all = min(kPf3Sub, n - j * kPf3Sub);   // valid tokens of this sub-block
-      const int valid = valid_all - hf * 32;                  // ... among this thread's 32
-      const uint32_t t_s = t_lane + s * 64 + hf * 32;         // this thread's scores, later its weights
-      if (!mbar_wait<kPfPolls>(bar_s(s), (uint32_t)(j >> 1) & 1u)) gave_up = true;
-      tc_fence_after();
-      float sv[32];                                       // raw products; the scale is folded in below
-      float bmax = -INFINITY;
-      {
-        uint32_t r[32];
-        tmem_ld32(t_s, r);
-        if (valid >= 32) {                                // warp-uniform: only the last sub-block masks
-#pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            sv[i] = __uint_as_float(r[i]);
-            bmax = fmaxf(bmax, sv[i]);
-          }
-        } else {
-#pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            sv[i] = i < valid ? __uint_as_float(r[i]) : -INFINITY;
-            bmax = fmaxf(bmax, sv[i]);
-          }
-        }
-        bmax *= scale_log2e;                              // scale > 0: the maximum commutes with it
-      }
-      // The two halves of a row exchange their maxima, and whether either warp gave up, so
-      // that both warps of the pair leave the loop together.
-      gave_up = __any_sync(0xffffffffu, gave_up);
-      s_x[s][hf][row] = bmax;
-      if ((tid & 31) == 0) s_flag[s][warp] = gave_up ? 1 : 0;
-      pair_sync(warp & 3);
-      if (s_flag[s][warp & 3] | s_flag[s][(warp & 3) + 4]) { gave_up = true; break; }
-      const float m_new = fmaxf(m_ref, fmaxf(s_x[s][0][row], s_x[s][1][row]));
-      if (j == 0) m_ref = m_new;
-      // ---- rescale O only when this row's maximum has drifted far from the reference --------
-      const bool need = m_new > m_ref + kPfRescaleGap;
-      if (__any_sync(0xffffffffu, need)) {
-        // O must be quiet: P(j-1) V(j-1) has to be complete (P(j) V(j) waits for this thread)
-        if (!mbar_wait<kPfPolls>(bar_o, (uint32_t)(j - 1) & 1u)) gave_up = true;
-        tc_fence_after();
-        const float factor = need ? fast_exp2(m_ref - m_new) : 1.f;
-#pragma unroll 1
-        for (int c = 0; c < 64; c += 8) tmem_scale8(t_o + c, factor);
-        if (need) { l_run *= factor; m_ref = m_new; }
-      }
-      // ---- weights 2^(s - m_ref) as bf16 pairs over the first half of the score columns -----
-      {
-        uint32_t pk[16];
-        float rowsum0 = 0.f, rowsum1 = 0.f;
-        const float neg_m = -m_ref;
-#pragma unroll
-        for (int i = 0; i < 32; i += 2) {
-          const float p0 = fast_exp2(__fmaf_rn(sv[i], scale_log2e, neg_m));     // -inf -> 0
-          const float p1 = fast_exp2(__fmaf_rn(sv[i + 1], scale_log2e, neg_m));
-          rowsum0 += p0;
-          rowsum1 += p1;
-          pk[i >> 1] = pack_bf16(p0, p1);
-        }
-        tmem_st16(t_s, pk);
-        tmem_wait_st();
-        l_run += rowsum0 + rowsum1;
-      }
-      if (valid_all < kPf3Sub) {
-        // Last, partial sub-block: rows of the V tile past the valid length hold whatever the
-        // cache holds there; clear them so that a zero weight times Inf/NaN cannot reach O.
-        if (!mbar_wait<kPfPolls>(bar_v(s), (uint32_t)(j >> 1) & 1u)) gave_up = true;
-        if (row >= valid_all && row < kPf3Sub) {
-#pragma unroll
-          for (int c = 0; c < 8; ++c)
-            st_shared16(sV + s * kPf3Tile + hf * kPf3Half + row * 128 + (c << 4), 0, 0, 0, 0);
-        }
-        proxy_fence();
-      }
-      tc_fence_before();
-      mbar_arrive(bar_p(s));                              // this thread's weights (and O) are in place
-    }
-    // O is complete when the last P V has been committed
-    if (!gave_up && !mbar_wait<kPfPolls>(bar_o, (uint32_t)(nb - 1) & 1u)) gave_up = true;
-    if (gave_up) s_fail = 1;
-  }
-  __syncthreads();                                       // every role is done with the loop
-  tc_fence_after();
-  const bool failed = s_fail != 0;
-  // the two halves of a row share the reference maximum; their weight sums add up
-  if (softmax_thread) s_x[0][hf][row] = l_run;
-  __syncthreads();
-  const float l_tot = s_x[0][0][row] + s_x[0][1][row];
-  if (!failed && softmax_thread) {
-    const float inv = 1.f / l_tot;
-#pragma unroll
-    for (int c = 0; c < 2; ++c) {
-      uint32_t r[32];
-      tmem_ld32(t_o + c * 32, r);
-      if (row_valid) {
-        float4* dst = reinterpret_cast<float4*>(out + row_off * D + hf * 64 + c * 32);
-#pragma unroll
-        for (int i = 0; i < 32; i += 4)
-          dst[i >> 2] = make_float4(__uint_as_float(r[i]) * inv, __uint_as_float(r[i + 1]) * inv,
-                                    __uint_as_float(r[i + 2]) * inv, __uint_as_float(r[i + 3]) * inv);
-      }
-    }
-    if (row_valid && lse_out && hf == 0)
-      lse_out[row_off] = (m_ref + log2f(l_tot)) * 0.6931471805599453f;
-  }
-  if (failed && tid == 0 && status_word) {
-    atomicExch(status_word, (int)L2KV_ERR_CUDA);
-    atomicExch(status_word + 2, 1);
-  }
-  tc_fence_before();
-  __syncthreads();
-  if (warp == 0)
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem), "r"(kPfTmemCols)
-                 : "memory");
-}
-
-// Fourth formulation: one CTA per SM works on two query tiles (256 rows) that share every K
-// and V tile, which halves the traffic from L2 into shared memory and leaves room for a ring
-// of four K and four V tiles fetched well ahead.  Roles: 2 x 8 softmax warps (one set per
-// query tile, as in the third formulation), one issuing thread per query tile, one thread
-// that fetches K tiles and one that fetches V tiles.  All of tensor memory (512 columns) is
-// used: per query tile two score buffers of 64 columns and the 128 output columns.
-constexpr int kPf4Stages = 4;                   // K tiles (and V tiles) in flight
-constexpr int kPf4Threads = 2 * kPfThreads + 4 * 32;   // softmax A, softmax B, issuer A, issuer B, K, V
-constexpr int kPf4TmemCols = 512;
-
 __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
   uint32_t done;
   asm volatile("{ .reg .pred p; mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2; "
@@ -907,306 +385,26 @@ __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
 __device__ __forceinline__ bool mbar_wait_likely(uint32_t bar, uint32_t parity) {
   return mbar_test(bar, parity) || mbar_wait<kPfPolls>(bar, parity);
 }
-__device__ __forceinline__ void pair_sync8(int id) {     // ids 1..8, 64 threads each
-  switch (id) {
-    case 1: asm volatile("bar.sync 1, 64;" ::: "memory"); break;
-    case 2: asm volatile("bar.sync 2, 64;" ::: "memory"); break;
-    case 3: asm volatile("bar.sync 3, 64;" ::: "memory"); break;
-    case 4: asm volatile("bar.sync 4, 64;" ::: "memory"); break;
-    case 5: asm volatile("bar.sync 5, 64;" ::: "memory"); break;
-    case 6: asm volatile("bar.sync 6, 64;" ::: "memory"); break;
-    case 7: asm volatile("bar.sync 7, 64;" ::: "memory"); break;
-    default: asm volatile("bar.sync 8, 64;" ::: "memory"); break;
-  }
-}
 
-template <int G>
-__global__ void __launch_bounds__(kPf4Threads, 1)
-prefix_attention_kernel_v4(const __nv_bfloat16* __restrict__ q, Geom g, int n_queries,
-                           const int32_t* __restrict__ cur_len_dev, int max_len, float scale_log2e,
-                           float* __restrict__ out, float* __restrict__ lse_out,
-                           const __grid_constant__ CUtensorMap map_k,
-                           const __grid_constant__ CUtensorMap map_v,
-                           int32_t* __restrict__ status_word) {
-  constexpr int D = 128;
-  constexpr int QT = kPfRows / G;                       // queries per query tile
-  constexpr int NS = kPf4Stages;
-  extern __shared__ unsigned char smem_raw[];
-  // mbarriers: K landed [NS], V landed [NS], K tile free [NS], V tile free [NS], then per query
-  // tile: scores ready [2], weights ready [2], output quiet [1]
-  __shared__ __align__(8) unsigned long long s_bar[4 * NS + 10];
-  __shared__ uint32_t s_tmem;
-  __shared__ int s_fail;
-  __shared__ float s_x[2][2][2][kPfRows];               // [query tile][sub-block parity][half][row]
-  __shared__ int s_flag[2][2][8];                       // [query tile][parity][softmax warp] gave up
-
-  const int q_tiles = (n_queries + QT - 1) / QT;
-  const int q_pairs = (q_tiles + 1) / 2;
-  const int qp = blockIdx.x % q_pairs;
-  const long long unit = blockIdx.x / q_pairs;          // (b * L + l) * H + h
-  const int h = (int)(unit % g.H);
-  const long long bl = unit / g.H;
-  const int l = (int)(bl % g.L), b = (int)(bl / g.L);
-  const int n = max(0, min(cur_len_dev[bl], min(max_len, g.t_cap)));
-  const int tid = threadIdx.x, warp = tid >> 5;
-  const bool softmax_thread = tid < 2 * kPfThreads;
-  const int n_tiles = (2 * qp + 1 < q_tiles) ? 2 : 1;   // query tiles of this CTA that exist
-  // Softmax threads: query tile `tile`, row `row`, column half `hf` (as in the third formulation).
-  const int tile = softmax_thread ? tid >> 8 : (warp - 16) & 1;
-  const int row = tid & (kPfRows - 1), hf = (tid >> 7) & 1;
-  const int wq = warp & 3;                              // tensor-memory lane quarter of this warp
-  const int s_idx = (2 * qp + tile) * QT + row / G;     // this row's query and head
-  const int head = h * G + row % G;
-  const bool row_valid = softmax_thread && s_idx < n_queries;
-  const long long row_off = ((bl * n_queries + s_idx) * g.Hq + head);
-  if (n == 0) {                                         // empty cache: zeros, log-sum-exp = -inf
-    if (row_valid) {
-      for (int d = 0; d < 64; ++d) out[row_off * D + hf * 64 + d] = 0.f;
-      if (lse_out && hf == 0) lse_out[row_off] = -INFINITY;
-    }
-    return;
-  }
-  // A wait that gave up in an earlier CTA marks the workspace; the rest of the grid leaves.
-  if (status_word && *reinterpret_cast<volatile int32_t*>(status_word + 2) != 0) return;
-  const int nb = (n + kPf3Sub - 1) / kPf3Sub;
-
-  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;   // 1024-byte aligned tiles
-  const uint32_t sQ = base + (uint32_t)tile * kPfTileBytes;      // this query tile's rows
-  const uint32_t sK = base + 2 * kPfTileBytes, sV = sK + NS * kPf3Tile;
-  const uint32_t bar0 = smem_u32(&s_bar[0]);
-  auto bar_k = [&](int i) { return bar0 + 8u * (uint32_t)i; };
-  auto bar_v = [&](int i) { return bar0 + 8u * (uint32_t)(NS + i); };
-  auto bar_kfree = [&](int i) { return bar0 + 8u * (uint32_t)(2 * NS + i); };
-  auto bar_vfree = [&](int i) { return bar0 + 8u * (uint32_t)(3 * NS + i); };
-  const uint32_t bar_t = bar0 + 8u * (uint32_t)(4 * NS + 5 * tile);   // this query tile's five
-  auto bar_s = [&](int i) { return bar_t + 8u * (uint32_t)i; };
-  auto bar_p = [&](int i) { return bar_t + 8u * (uint32_t)(2 + i); };
-  const uint32_t bar_o = bar_t + 32u;
-
-  if (warp == 0) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                 :: "r"(smem_u32(&s_tmem)), "r"(kPf4TmemCols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  }
-  if (tid == 0) {
-    for (int i = 0; i < 2 * NS; ++i) mbar_init(bar0 + 8u * i, 1);
-    for (int i = 2 * NS; i < 4 * NS; ++i) mbar_init(bar0 + 8u * i, n_tiles);   // one commit per query tile
-    for (int t = 0; t < 2; ++t) {
-      const uint32_t bt = bar0 + 8u * (uint32_t)(4 * NS + 5 * t);
-      mbar_init(bt, 1); mbar_init(bt + 8, 1);
-      mbar_init(bt + 16, kPfThreads); mbar_init(bt + 24, kPfThreads);
-      mbar_init(bt + 32, 1);
-    }
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    s_fail = 0;
-  }
-  __syncwarp();
-  if (softmax_thread) {                                 // Q rows, K-major, 128-byte swizzle
-    const uint4* src = reinterpret_cast<const uint4*>(q + row_off * D) + hf * 8;
-#pragma unroll
-    for (int c = 0; c < 8; ++c) {
-      const uint4 v = row_valid ? src[c] : make_uint4(0, 0, 0, 0);
-      st_shared16(sQ + hf * kPfHalf + row * 128 + ((c ^ (row & 7)) << 4), v.x, v.y, v.z, v.w);
-    }
-  }
-  proxy_fence();
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem = s_tmem + (uint32_t)tile * 256;  // this query tile's 256 columns
-  bool gave_up = false;
-  float m_ref = -INFINITY, l_run = 0.f;                 // reference maximum; sum of this half's weights
-  const uint32_t t_lane = tmem + ((uint32_t)(wq * 32) << 16);
-  const uint32_t t_o = t_lane + 128 + hf * 64;          // this thread's 64 output dims
-  const bool tile_active = tile < n_tiles;
-
-  if (!softmax_thread) {
-    if ((tid & 31) == 0 && warp >= 18) {
-      // ---- the two fetching threads: K tiles (warp 18), V tiles (warp 19) ---------------------
-      const bool is_k = warp == 18;
-      const CUtensorMap* map = is_k ? &map_k : &map_v;
-      bool ok = true;
-      for (int j = 0; ok && j < nb; ++j) {
-        const int st = j % NS, use = j / NS;
-        const uint32_t full = is_k ? bar_k(st) : bar_v(st);
-        if (use > 0) ok = mbar_wait<kPfPolls>(is_k ? bar_kfree(st) : bar_vfree(st), (uint32_t)(use - 1) & 1u);
-        if (!ok) break;
-        const uint32_t dst = (is_k ? sK : sV) + st * kPf3Tile;
-        mbar_expect_tx(full, kPf3Tile);
-        tma_load_5d(dst, map, full, 0, j * kPf3Sub, h, l, b);
-        tma_load_5d(dst + kPf3Half, map, full, 64, j * kPf3Sub, h, l, b);
-      }
-      if (!ok) s_fail = 1;
-    } else if ((tid & 31) == 0 && tile_active) {
-      // ---- the issuing thread of query tile `tile` ---------------------------------------------
-      auto issue_qk = [&](int j) {                      // S[j & 1] = Q K(j)^T; then the K tile is free
-        const uint32_t kt = sK + (j % NS) * kPf3Tile;
-#pragma unroll
-        for (int k = 0; k < 8; ++k)
-          umma_bf16(tmem + (j & 1) * 64,
-                    umma_desc(sQ + (k >> 2) * kPfHalf + (k & 3) * 32, 16, 1024),
-                    umma_desc(kt + (k >> 2) * kPf3Half + (k & 3) * 32, 16, 1024), kIdescQK64, k > 0);
-        umma_commit(bar_s(j & 1));
-        umma_commit(bar_kfree(j % NS));
-      };
-      bool ok = mbar_wait<kPfPolls>(bar_k(0), 0);
-      if (ok) { tc_fence_after(); issue_qk(0); }
-      if (ok && nb > 1) {
-        ok = mbar_wait<kPfPolls>(bar_k(1 % NS), 0);
-        if (ok) { tc_fence_after(); issue_qk(1); }
-      }
-      if (ok) ok = mbar_wait<kPfPolls>(bar_v(0), 0);
-      for (int j = 0; ok && j < nb; ++j) {
-        const int s = j & 1;
-        ok = mbar_wait<kPfPolls>(bar_p(s), (uint32_t)(j >> 1) & 1u);
-        if (!ok) break;
-        tc_fence_after();
-        const uint32_t vt = sV + (j % NS) * kPf3Tile;
-#pragma unroll
-        for (int k = 0; k < 4; ++k)                     // O += P(j) V(j); slice k = tokens 16k .. 16k + 15
-          umma_bf16_ts(tmem + 128, tmem + s * 64 + (k >> 1) * 32 + (k & 1) * 8,
-                       umma_desc(vt + k * 2048, kPf3Half, 1024), kIdescPV, (j > 0 || k > 0) ? 1u : 0u);
-        umma_commit(bar_o);
-        umma_commit(bar_vfree(j % NS));
-        // tiles fetched well ahead: these two are normally over already
-        if (j + 2 < nb) ok = mbar_wait_likely(bar_k((j + 2) % NS), (uint32_t)((j + 2) / NS) & 1u);
-        if (ok && j + 1 < nb) ok = mbar_wait_likely(bar_v((j + 1) % NS), (uint32_t)((j + 1) / NS) & 1u);
-        // P(j) V(j) done: the score buffer it read its weights from takes sub-block j + 2
-        ok = ok && mbar_wait<kPfPolls>(bar_o, (uint32_t)j & 1u);
-        if (!ok) break;
-        if (j + 2 < nb) { tc_fence_after(); issue_qk(j + 2); }
-      }
-      if (!ok) s_fail = 1;
-    }
-  } else if (tile_active) {
-    // ---- the softmax warps of query tile `tile` ------------------------------------------------
-    const int wt = warp & 7;                              // warp within the query tile
-    for (int j = 0; j < nb; ++j) {
-      const int s = j & 1;
-      const int valid_all = min(kPf3Sub, n - j * kPf3Sub);   // valid tokens of this sub-block
-      const int valid = valid_all - hf * 32;                  // ... among this thread's 32
-      const uint32_t t_s = t_lane + s * 64 + hf * 32;         // this thread's scores, later its weights
-      if (!mbar_wait<kPfPolls>(bar_s(s), (uint32_t)(j >> 1) & 1u)) gave_up = true;
-      tc_fence_after();
-      float sv[32];                                       // raw products; the scale is folded in below
-      float bmax = -INFINITY;
-      {
-        uint32_t r[32];
-        tmem_ld32(t_s, r);
-        if (valid >= 32) {                                // warp-uniform: only the last sub-block masks
-#pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            sv[i] = __uint_as_float(r[i]);
-            bmax = fmaxf(bmax, sv[i]);
-          }
-        } else {
-#pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            sv[i] = i < valid ? __uint_as_float(r[i]) : -INFINITY;
-            bmax = fmaxf(bmax, sv[i]);
-          }
-        }
-        bmax *= scale_log2e;                              // scale > 0: the maximum commutes with it
-      }
-      // The two halves of a row exchange their maxima, and whether either warp gave up, so
-      // that both warps of the pair leave the loop together.
-      gave_up = __any_sync(0xffffffffu, gave_up);
-      s_x[tile][s][hf][row] = bmax;
-      if ((tid & 31) == 0) s_flag[tile][s][wt] = gave_up ? 1 : 0;
-      pair_sync8(1 + tile * 4 + wq);
-      if (s_flag[tile][s][wq] | s_flag[tile][s][wq + 4]) { gave_up = true; break; }
-      const float m_new = fmaxf(m_ref, fmaxf(s_x[tile][s][0][row], s_x[tile][s][1][row]));
-      if (j == 0) m_ref = m_new;
-      // ---- rescale O only when this row's maximum has drifted far from the reference --------
-      const bool need = m_new > m_ref + kPfRescaleGap;
-      if (__any_sync(0xffffffffu, need)) {
-        // O must be quiet: P(j-1) V(j-1) has to be complete (P(j) V(j) waits for this thread)
-        if (!mbar_wait<kPfPolls>(bar_o, (uint32_t)(j - 1) & 1u)) gave_up = true;
-        tc_fence_after();
-        const float factor = need ? fast_exp2(m_ref - m_new) : 1.f;
-#pragma unroll 1
-        for (int c = 0; c < 64; c += 8) tmem_scale8(t_o + c, factor);
-        if (need) { l_run *= factor; m_ref = m_new; }
-      }
-      // ---- weights 2^(s - m_ref) as bf16 pairs over the first half of the score columns -----
-      {
-        uint32_t pk[16];
-        float rowsum0 = 0.f, rowsum1 = 0.f;
-        const float neg_m = -m_ref;
-#pragma unroll
-        for (int i = 0; i < 32; i += 2) {
-          const float p0 = fast_exp2(__fmaf_rn(sv[i], scale_log2e, neg_m));     // -inf -> 0
-          const float p1 = fast_exp2(__fmaf_rn(sv[i + 1], scale_log2e, neg_m));
-          rowsum0 += p0;
-          rowsum1 += p1;
-          pk[i >> 1] = pack_bf16(p0, p1);
-        }
-        tmem_st16(t_s, pk);
-        tmem_wait_st();
-        l_run += rowsum0 + rowsum1;
-      }
-      if (valid_all < kPf3Sub) {
-        // Last, partial sub-block: rows of the V tile past the valid length hold whatever the
-        // cache holds there; clear them so that a zero weight times Inf/NaN cannot reach O
-        // (both query tiles write the same zeros).
-        if (!mbar_wait<kPfPolls>(bar_v(j % NS), (uint32_t)(j / NS) & 1u)) gave_up = true;
-        if (row >= valid_all && row < kPf3Sub) {
-#pragma unroll
-          for (int c = 0; c < 8; ++c)
-            st_shared16(sV + (j % NS) * kPf3Tile + hf * kPf3Half + row * 128 + (c << 4), 0, 0, 0, 0);
-        }
-        proxy_fence();
-      }
-      tc_fence_before();
-      mbar_arrive(bar_p(s));                              // this thread's weights (and O) are in place
-    }
-    // O is complete when the last P V has been committed
-    if (!gave_up && !mbar_wait<kPfPolls>(bar_o, (uint32_t)(nb - 1) & 1u)) gave_up = true;
-    if (gave_up) s_fail = 1;
-  }
-  __syncthreads();                                       // every role is done with the loop
-  tc_fence_after();
-  const bool failed = s_fail != 0;
-  // the two halves of a row share the reference maximum; their weight sums add up
-  if (softmax_thread) s_x[tile][0][hf][row] = l_run;
-  __syncthreads();
-  const float l_tot = s_x[tile][0][0][row] + s_x[tile][0][1][row];
-  if (!failed && softmax_thread && tile_active) {
-    const float inv = 1.f / l_tot;
-#pragma unroll
-    for (int c = 0; c < 2; ++c) {
-      uint32_t r[32];
-      tmem_ld32(t_o + c * 32, r);
-      if (row_valid) {
-        float4* dst = reinterpret_cast<float4*>(out + row_off * D + hf * 64 + c * 32);
-#pragma unroll
-        for (int i = 0; i < 32; i += 4)
-          dst[i >> 2] = make_float4(__uint_as_float(r[i]) * inv, __uint_as_float(r[i + 1]) * inv,
-                                    __uint_as_float(r[i + 2]) * inv, __uint_as_float(r[i + 3]) * inv);
-      }
-    }
-    if (row_valid && lse_out && hf == 0)
-      lse_out[row_off] = (m_ref + log2f(l_tot)) * 0.6931471805599453f;
-  }
-  if (failed && tid == 0 && status_word) {
-    atomicExch(status_word, (int)L2KV_ERR_CUDA);
-    atomicExch(status_word + 2, 1);
-  }
-  tc_fence_before();
-  __syncthreads();
-  if (warp == 0)
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(s_tmem), "r"(kPf4TmemCols)
-                 : "memory");
-}
-
-// Fifth formulation: the fourth with one softmax thread per query row (four warps per query
-// tile): a row's maximum and sum are thread-local, so the softmax warps never synchronise with
-// one another; they only wait for scores and hand over weights.
+// The pipelined kernel, the one the entry point uses.  The two contractions and the softmax
+// run concurrently, each in warps of its own, and one CTA per SM works on two query tiles
+// (256 rows) that share every K and V tile:
+//   - the cache is walked in sub-blocks of 64 tokens; per query tile two score buffers of 64
+//     columns and the 128 output columns live in tensor memory (2 x 256 = all 512 columns), so
+//     S(j+1) = Q K(j+1)^T is computed while the softmax works on S(j), and O += P(j) V(j) runs
+//     while it works on S(j+1);
+//   - one softmax thread per query row (four warps per query tile): a row's maximum and sum
+//     are thread-local, the softmax warps never synchronise with one another; they wait for
+//     scores and hand over weights (bf16 pairs written over the score columns);
+//   - one issuing thread per query tile, one thread that fetches K tiles and one that fetches
+//     V tiles by TMA into rings of four tiles each, freed by tcgen05.commit.
+// Hand-offs are mbarriers (scores ready / tile free / output quiet: tcgen05.commit; weights
+// ready: one arrival per softmax thread); every wait on them is bounded.
 constexpr int kPf5Threads = 2 * kPfRows + 4 * 32;      // softmax A, softmax B, issuer A, issuer B, K, V
 
 template <int G>
 __global__ void __launch_bounds__(kPf5Threads, 1)
-prefix_attention_kernel_v5(const __nv_bfloat16* __restrict__ q, Geom g, int n_queries,
+prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n_queries,
                            const int32_t* __restrict__ cur_len_dev, int max_len, float scale_log2e,
                            float* __restrict__ out, float* __restrict__ lse_out,
                            const __grid_constant__ CUtensorMap map_k,
@@ -1482,34 +680,29 @@ static int launch_pf(const void* q, const void* K, const void* V, const Geom& g,
   alignas(64) CUtensorMap map_k, map_v;
   std::memset(&map_k, 0, sizeof map_k);
   std::memset(&map_v, 0, sizeof map_v);
-  // L2KV_PREFIX_KERNEL selects a formulation: v1 (weights through shared memory), v2 (weights
-  // in tensor memory, one role), v3 (separate issuing warp, 64-token sub-blocks), v4 (two query
-  // tiles per CTA sharing the K/V tiles, one CTA per SM).
+  // L2KV_PREFIX_KERNEL=basic selects the single-role kernel; the pipelined one is the default.
   const char* which = std::getenv("L2KV_PREFIX_KERNEL");
-  const bool v1 = which && std::strcmp(which, "v1") == 0;
-  const bool v3 = which && std::strcmp(which, "v3") == 0;
-  const bool v5 = which && std::strcmp(which, "v5") == 0;
-  const bool v4 = v5 || (which && std::strcmp(which, "v4") == 0);
-  const int sub_rows = (v3 || v4) ? kPf3Sub : kPfRows;
+  const bool basic = which && std::strcmp(which, "basic") == 0;
+  const int sub_rows = basic ? kPfRows : kPf3Sub;
   if (!make_cache_map(&map_k, K, g, sub_rows) || !make_cache_map(&map_v, V, g, sub_rows))
     return L2KV_ERR_UNSUPPORTED;
-  if (v4) {
+  if (!basic) {
     constexpr int smem4 = 1024 + 2 * kPfTileBytes + 2 * kPf4Stages * kPf3Tile;
     const int q_tiles = (n_queries + QT - 1) / QT;
     const long long blocks4 = units * ((q_tiles + 1) / 2);
-    auto kern4 = v5 ? prefix_attention_kernel_v5<G> : prefix_attention_kernel_v4<G>;
+    auto kern4 = prefix_attention_pipelined_kernel<G>;
     if (cudaFuncSetAttribute(kern4, cudaFuncAttributeMaxDynamicSharedMemorySize, smem4) != cudaSuccess)
       return L2KV_ERR_CUDA;
-    kern4<<<(unsigned)blocks4, v5 ? kPf5Threads : kPf4Threads, smem4, s>>>(
+    kern4<<<(unsigned)blocks4, kPf5Threads, smem4, s>>>(
         static_cast<const __nv_bfloat16*>(q), g, n_queries, cur_len_dev, max_len, scale * kPfLog2e, out,
         lse_out, map_k, map_v, status_word);
     return cudaGetLastError() == cudaSuccess ? L2KV_OK : L2KV_ERR_CUDA;
   }
   constexpr int smem_bytes = 1024 + 3 * kPfTileBytes;
-  auto kern = v1 ? prefix_attention_kernel<G> : v3 ? prefix_attention_kernel_v3<G> : prefix_attention_kernel_v2<G>;
+  auto kern = prefix_attention_basic_kernel<G>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) != cudaSuccess)
     return L2KV_ERR_CUDA;
-  kern<<<(unsigned)blocks, v3 ? kPf3Threads : kPfThreads, smem_bytes, s>>>(
+  kern<<<(unsigned)blocks, kPfThreads, smem_bytes, s>>>(
       static_cast<const __nv_bfloat16*>(q), g, n_queries, cur_len_dev, max_len, scale * kPfLog2e, out,
       lse_out, map_k, map_v, status_word);
   return cudaGetLastError() == cudaSuccess ? L2KV_OK : L2KV_ERR_CUDA;
