@@ -108,50 +108,6 @@ __device__ __forceinline__ float fast_exp2(float x) {
   return y;
 }
 
-// 2^x on the FMA pipe, for a share of the exponentials (the MUFU unit delivers 16 per clock per SM,
-// which is as many cycles per score block as the tensor core needs for both contractions).
-// Round-to-nearest split x = n + f, f in [-0.5, 0.5], by the 1.5 * 2^23 trick; 2^f by a degree-4
-// polynomial (least-squares fit of the relative error: 2.7e-6 at most, far below the bf16
-// rounding of the weights); n goes straight into the exponent bits.  x is clamped at -125, so
-// -inf (a masked score) gives 2^-125 instead of 0: negligible against a row's largest weight,
-// which is at least 2^-8, and the V rows of masked positions are zero.
-#ifndef L2KV_PF_POLY_EVERY
-#define L2KV_PF_POLY_EVERY 4       /* one exponential in this many runs on the FMA pipe; 0: none */
-#endif
-__device__ __forceinline__ float poly_exp2(float x) {
-  x = fmaxf(x, -125.f);
-  const float t = x + 12582912.f;
-  const float f = x - (t - 12582912.f);
-  float p = 9.570082650e-03f;
-  p = __fmaf_rn(p, f, 5.591784418e-02f);
-  p = __fmaf_rn(p, f, 2.402474433e-01f);
-  p = __fmaf_rn(p, f, 6.931217909e-01f);
-  p = __fmaf_rn(p, f, 9.999992847e-01f);
-  return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
-}
-template <int I>
-__device__ __forceinline__ float weight_exp2(float x) {
-  if constexpr (L2KV_PF_POLY_EVERY > 0 && (I % (L2KV_PF_POLY_EVERY > 0 ? L2KV_PF_POLY_EVERY : 1)) == (L2KV_PF_POLY_EVERY > 0 ? L2KV_PF_POLY_EVERY : 1) - 1)
-    return poly_exp2(x);
-  else
-    return fast_exp2(x);
-}
-
-// The 64 weights of a row of a sub-block, fully unrolled so that each element's place in the
-// MUFU / FMA-pipe split is fixed at compile time.
-template <int I>
-__device__ __forceinline__ void weights_unrolled(const float (&sv)[64], float c, float neg_m, float& sum0,
-                                                 float& sum1, uint32_t (&pk)[32]) {
-  if constexpr (I < 64) {
-    const float p0 = weight_exp2<I>(__fmaf_rn(sv[I], c, neg_m));           // -inf -> 0 (or 2^-125)
-    const float p1 = weight_exp2<I + 1>(__fmaf_rn(sv[I + 1], c, neg_m));
-    sum0 += p0;
-    sum1 += p1;
-    pk[I >> 1] = pack_bf16(p0, p1);
-    weights_unrolled<I + 2>(sv, c, neg_m, sum0, sum1, pk);
-  }
-}
-
 // Eight columns at a time: the rarely taken rescaling of O, kept small in registers.
 __device__ __forceinline__ void tmem_scale8(uint32_t taddr, float factor) {
   uint32_t r0, r1, r2, r3, r4, r5, r6, r7;
@@ -649,7 +605,14 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
         uint32_t pk[32];
         float rowsum0 = 0.f, rowsum1 = 0.f;
         const float neg_m = -m_ref;
-        weights_unrolled<0>(sv, scale_log2e, neg_m, rowsum0, rowsum1, pk);
+#pragma unroll
+        for (int i = 0; i < 64; i += 2) {
+          const float p0 = fast_exp2(__fmaf_rn(sv[i], scale_log2e, neg_m));     // -inf -> 0
+          const float p1 = fast_exp2(__fmaf_rn(sv[i + 1], scale_log2e, neg_m));
+          rowsum0 += p0;
+          rowsum1 += p1;
+          pk[i >> 1] = pack_bf16(p0, p1);
+        }
         tmem_st32(t_s, pk);
         tmem_wait_st();
         l_run += rowsum0 + rowsum1;
