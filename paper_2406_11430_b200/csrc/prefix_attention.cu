@@ -399,7 +399,7 @@ __device__ __forceinline__ bool mbar_wait_likely(uint32_t bar, uint32_t parity) 
 //   - one issuing thread per query tile, one thread that fetches K tiles and one that fetches
 //     V tiles by TMA into rings of four tiles each, freed by tcgen05.commit.
 // Hand-offs are mbarriers (scores ready / tile free / output quiet: tcgen05.commit; weights
-// ready: one arrival per softmax thread); every wait on them is bounded.
+// ready: one arrival per softmax warp); every wait on them is bounded.
 constexpr int kPf5Threads = 2 * kPfRows + 4 * 32;      // softmax A, softmax B, issuer A, issuer B, K, V
 
 template <int G>
@@ -474,7 +474,7 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
     for (int t = 0; t < 2; ++t) {
       const uint32_t bt = bar0 + 8u * (uint32_t)(4 * NS + 5 * t);
       mbar_init(bt, 1); mbar_init(bt + 8, 1);
-      mbar_init(bt + 16, kPfRows); mbar_init(bt + 24, kPfRows);
+      mbar_init(bt + 16, kPfRows / 32); mbar_init(bt + 24, kPfRows / 32);   // one arrival per softmax warp
       mbar_init(bt + 32, 1);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -630,7 +630,8 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
         proxy_fence();
       }
       tc_fence_before();
-      mbar_arrive(bar_p(s));                              // this row's weights (and O) are in place
+      __syncwarp();                                       // the warp's 32 rows are in place:
+      if ((tid & 31) == 0) mbar_arrive(bar_p(s));         // one arrival per warp
     }
     // O is complete when the last P V has been committed
     if (!gave_up && !mbar_wait<kPfPolls>(bar_o, (uint32_t)(nb - 1) & 1u)) gave_up = true;
