@@ -139,6 +139,7 @@ def attention(q, K_c, V_c, dtype, cur_len, scale=0.0, nthreads=1):
 def append_evict(state, dtype, budget, uncompressed, k_new, v_new, pos_new, key_mode=0):
     """One append/evict step, in place on state = dict(K_c, V_c, idx, key, cur_len).
 
+    cur_len [B, L] with budget [B], or (a length and a budget per head) both [B, L, H].
     Returns the oracle's status (0, or -2 when a row did not fit T_cap).
     """
     K_c, V_c = state["K_c"], state["V_c"]
@@ -148,11 +149,14 @@ def append_evict(state, dtype, budget, uncompressed, k_new, v_new, pos_new, key_
     B, L, H, T_cap, D = K_c.shape
     budget, unc, pos_new = _i32(budget), _i32(list(uncompressed)), _i32(pos_new)
     assert state["idx"].dtype == np.int32 and state["key"].dtype == np.float64
-    assert state["cur_len"].dtype == np.int32 and state["cur_len"].shape == (B, L)
+    per_head = state["cur_len"].ndim == 3
+    assert state["cur_len"].dtype == np.int32
+    assert state["cur_len"].shape == ((B, L, H) if per_head else (B, L))
+    assert budget.shape == ((B, L, H) if per_head else (B,))
     return int(lib().l2kv_oracle_append_evict(
         _p(K_c), _p(V_c), _p(state["idx"]), _p(state["key"]), _DT[dtype], B, L, H, T_cap, D,
         _p(state["cur_len"]), _p(budget), _p(unc), int(unc.size), _p(k_new), _p(v_new),
-        _p(pos_new), int(key_mode)))
+        _p(pos_new), int(key_mode), int(per_head)))
 
 
 def attention_loss(q, K, dtype, cur_len, scale=0.0, key_mode=0, curves=False, nthreads=1):

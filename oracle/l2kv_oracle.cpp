@@ -396,23 +396,30 @@ int l2kv_oracle_append_evict(void* K_c, void* V_c, int32_t* idx, double* key_c, 
                              int L, int H, int T_cap, int D, int32_t* cur_len,
                              const int32_t* budget, const int32_t* uncompressed, int n_unc,
                              const void* k_new, const void* v_new, const int32_t* pos_new,
-                             int key_mode) {
+                             int key_mode, int per_head) {
+  // per_head != 0: cur_len and budget are [B, L, H] (caches compressed with a keep count per
+  // head); otherwise cur_len is [B, L] and budget [B].
   const size_t row_bytes = size_t(D) * elem_size(dtype);
   int status = 0;
   for (int b = 0; b < B; ++b) {
     for (int l = 0; l < L; ++l) {
-      const int n = cur_len[b * L + l];
-      const bool grow = in_list(uncompressed, n_unc, l) || n < budget[b];
-      if (grow && n >= T_cap) {
-        status = -2;
-        continue;
-      }
+      bool any_grow = false;
+      const int n_shared = per_head ? 0 : cur_len[b * L + l];
       for (int h = 0; h < H; ++h) {
         const int64_t u = (int64_t(b) * L + l) * H + h;
+        const int n = per_head ? cur_len[u] : n_shared;
+        const int cap = per_head ? budget[u] : budget[b];
+        const bool grow = in_list(uncompressed, n_unc, l) || n < cap;
+        if (grow && n >= T_cap) {
+          status = -2;
+          continue;
+        }
         const double s_new = row_key(k_new, dtype, u * D, D, key_mode);
         int slot;
         if (grow) {
           slot = n;
+          any_grow = true;
+          if (per_head) cur_len[u] = n + 1;
         } else {
           // arg-max of (key, position) over the stored entries and the new one
           slot = -1;  // -1 = the new token itself
@@ -437,7 +444,7 @@ int l2kv_oracle_append_evict(void* K_c, void* V_c, int32_t* idx, double* key_c, 
         idx[u * T_cap + slot] = pos_new[b];
         key_c[u * T_cap + slot] = s_new;
       }
-      if (grow) cur_len[b * L + l] = n + 1;
+      if (!per_head && any_grow) cur_len[b * L + l] = n_shared + 1;
     }
   }
   return status;

@@ -397,6 +397,37 @@ def test_streaming_eviction_equals_one_shot_selection(dtype):
                 assert np.array_equal(st["key"][b, l, h, :n][order], one["key"][b, l, h, :n])
 
 
+def test_streaming_eviction_with_a_budget_per_head():
+    """Per-head budgets: every head ends with its own `budget` lowest (norm, position) of all
+    the tokens it has seen (sort-and-cut per head); heads under budget keep growing."""
+    steps, T0 = 30, 48
+    w = synth.WORKLOADS[0].scaled(dtype="bf16", B=2, L=2, T=T0)
+    K, V = synth.make_cache(w, "cpu")
+    Kn, Vn = synth.to_numpy(K), synth.to_numpy(V)
+    rng = np.random.default_rng(2)
+    keep = rng.integers(1, T0 + 1, size=(2, 2, w.Hkv)).astype(np.int32)
+    budget = keep.copy()
+    budget[0, 0, 0] = T0 + 10                                 # still filling: appends 10, then evicts
+    budget[1, 1, 1] = T0 + steps + 5                          # never full: only appends
+    keep[0, 0, 0] = keep[1, 1, 1] = T0
+    r = oracle.compress(Kn, Vn, "bf16", [T0, T0], keep, t_cap_out=T0)
+    st = _state_from(r, T0 + steps)
+    assert st["cur_len"].shape == (2, 2, w.Hkv)
+    allK = [Kn]
+    for s in range(steps):
+        k, v = synth.make_new_kv(w, s, "cpu")
+        kn, vn = synth.to_numpy(k), synth.to_numpy(v)
+        assert oracle.append_evict(st, "bf16", budget, (), kn, vn, [T0 + s, T0 + s]) == 0
+        allK.append(kn[:, :, :, None])
+    key = oracle.key_sumsq(np.concatenate(allK, 3), "bf16")
+    T = T0 + steps
+    for b, l, h in itertools.product(range(2), range(2), range(w.Hkv)):
+        n = min(int(budget[b, l, h]), T)
+        assert st["cur_len"][b, l, h] == n
+        want = sorted(sorted(range(T), key=lambda t: (key[b, l, h, t], t))[:n])
+        assert sorted(st["idx"][b, l, h, :n].tolist()) == want
+
+
 def test_append_evict_cases():
     D = 64
     def row(c):
