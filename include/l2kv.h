@@ -151,8 +151,12 @@ int l2kv_decode_attention(const void* q, const void* K_c, const void* V_c, const
  * int32 [batch, layers, kv_heads] in place of keep_dev (0 <= keep_unit_dev[b,l,h] <=
  * len_dev[b]; layers in uncompressed_layers ignore it) and kept_len_unit_dev of the same
  * shape in place of kept_len_dev.  l2kv_decode_attention_per_head is l2kv_decode_attention
- * over rows i < cur_len_unit_dev[b,l,j/G] (dense int32 [batch, layers, kv_heads]).  All
- * other arguments, layouts, ownership and errors are those of the per-sequence calls. */
+ * over rows i < cur_len_unit_dev[b,l,j/G] (dense int32 [batch, layers, kv_heads]).
+ * l2kv_append_evict_per_head is l2kv_append_evict with cur_len_unit_dev (in/out) and
+ * budget_unit_dev dense int32 [batch, layers, kv_heads]: every head appends until it holds its
+ * own budget and evicts from then on.  l2kv_prefix_attention_per_head is
+ * l2kv_prefix_attention over rows i < cur_len_unit_dev[b,l,j/G].  All other arguments,
+ * layouts, ownership and errors are those of the per-sequence calls. */
 int l2kv_select_compact_per_head(const void* K, const void* V, const l2kv_layout* in,
                                  const int32_t* len_dev, const int32_t* keep_unit_dev,
                                  int32_t max_len, const int32_t* uncompressed_layers,
@@ -165,6 +169,17 @@ int l2kv_decode_attention_per_head(const void* q, const void* K_c, const void* V
                                    const l2kv_layout* lay, const int32_t* cur_len_unit_dev,
                                    int32_t max_len, float scale, float* out, void* workspace,
                                    size_t workspace_bytes, void* stream);
+int l2kv_append_evict_per_head(void* K_c, void* V_c, int32_t* idx, float* sumsq_c,
+                               const l2kv_layout* lay, int32_t* cur_len_unit_dev,
+                               const int32_t* budget_unit_dev, const int32_t* uncompressed_layers,
+                               int32_t n_uncompressed, const void* k_new, const void* v_new,
+                               const int32_t* pos_new_dev, void* workspace, size_t workspace_bytes,
+                               void* stream);
+int l2kv_prefix_attention_per_head(const void* q, const void* K_c, const void* V_c,
+                                   const l2kv_layout* lay, const int32_t* cur_len_unit_dev,
+                                   int32_t max_len, int32_t n_queries, float scale, float* out,
+                                   float* lse_out, void* workspace, size_t workspace_bytes,
+                                   void* stream);
 
 /* Budget-maintained cache (Section 4, "Language Modelling Tasks"): append one new
  * token per (b, l, h).  If l is uncompressed or cur_len_dev[b,l] < budget_dev[b] the

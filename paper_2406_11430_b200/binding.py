@@ -57,16 +57,19 @@ def lib():
         L.l2kv_decode_attention_per_head.argtypes = L.l2kv_decode_attention.argtypes
         L.l2kv_append_evict.argtypes = [vp, vp, vp, vp, lay, vp, vp, ctypes.POINTER(i32), i32,
                                         vp, vp, vp, vp, sz, vp]
+        L.l2kv_append_evict_per_head.argtypes = L.l2kv_append_evict.argtypes
         L.l2kv_attention_loss_workspace_bytes.argtypes = [lay, i32, ctypes.POINTER(sz)]
         L.l2kv_attention_loss.argtypes = [vp, vp, lay, vp, i32, ctypes.c_float, vp, vp, vp, vp,
                                           vp, sz, vp]
         L.l2kv_prefix_attention.argtypes = [vp, vp, vp, lay, vp, i32, i32, ctypes.c_float, vp, vp,
                                             vp, sz, vp]
+        L.l2kv_prefix_attention_per_head.argtypes = L.l2kv_prefix_attention.argtypes
         for name in ("l2kv_prefix_attention", "l2kv_attention_loss_workspace_bytes", "l2kv_attention_loss",
                      "l2kv_keep_count", "l2kv_workspace_bytes", "l2kv_read_device_status",
                      "l2kv_key_norms", "l2kv_select_compact", "l2kv_decode_attention",
                      "l2kv_append_evict", "l2kv_select_compact_per_head",
-                     "l2kv_decode_attention_per_head"):
+                     "l2kv_decode_attention_per_head", "l2kv_append_evict_per_head",
+                     "l2kv_prefix_attention_per_head"):
             getattr(L, name).restype = ctypes.c_int
         _LIB = L
     return _LIB
@@ -200,6 +203,17 @@ def append_evict(K_c, V_c, idx, sumsq_c, cur_len_dev, budget_dev, uncompressed_l
         workspace.numel(), _stream(stream)), "l2kv_append_evict")
 
 
+def append_evict_per_head(K_c, V_c, idx, sumsq_c, cur_len_unit_dev, budget_unit_dev,
+                          uncompressed_layers, k_new, v_new, pos_new_dev, workspace, stream=None):
+    """append_evict with a length (in/out) and a budget per (b, l, h)."""
+    lay = Layout(K_c)
+    arr, n = _layers(uncompressed_layers)
+    _check(lib().l2kv_append_evict_per_head(
+        _ptr(K_c), _ptr(V_c), _ptr(idx), _ptr(sumsq_c), lay.ref(), _ptr(cur_len_unit_dev),
+        _ptr(budget_unit_dev), arr, n, _ptr(k_new), _ptr(v_new), _ptr(pos_new_dev),
+        _ptr(workspace), workspace.numel(), _stream(stream)), "l2kv_append_evict_per_head")
+
+
 def decode_attention_static(q, K_c, V_c, cur_len_dev, max_len, out, scale=0.0, stream=None):
     """decode_attention for callers that cannot allocate: no workspace argument.  The partial
     results go to a fixed 16 MiB array inside the library (problems that need more raise
@@ -239,3 +253,14 @@ def prefix_attention(q, K_c, V_c, cur_len_dev, max_len, out, lse_out=None, scale
         _ptr(q), _ptr(K_c), _ptr(V_c), lay.ref(), _ptr(cur_len_dev), int(max_len), int(q.shape[2]),
         float(scale), _ptr(out), _ptr(lse_out), _ptr(workspace),
         0 if workspace is None else workspace.numel(), _stream(stream)), "l2kv_prefix_attention")
+
+
+def prefix_attention_per_head(q, K_c, V_c, cur_len_unit_dev, max_len, out, lse_out=None, scale=0.0,
+                              workspace=None, stream=None):
+    """prefix_attention with a cache length per (b, l, kv head)."""
+    lay = Layout(K_c, q_heads=q.shape[3])
+    _check(lib().l2kv_prefix_attention_per_head(
+        _ptr(q), _ptr(K_c), _ptr(V_c), lay.ref(), _ptr(cur_len_unit_dev), int(max_len),
+        int(q.shape[2]), float(scale), _ptr(out), _ptr(lse_out), _ptr(workspace),
+        0 if workspace is None else workspace.numel(), _stream(stream)),
+        "l2kv_prefix_attention_per_head")

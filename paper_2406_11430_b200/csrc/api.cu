@@ -215,11 +215,12 @@ int l2kv_decode_attention_per_head(const void* q, const void* K_c, const void* V
                                workspace, workspace_bytes, stream);
 }
 
-int l2kv_append_evict(void* K_c, void* V_c, int32_t* idx, float* sumsq_c, const l2kv_layout* lay,
-                      int32_t* cur_len_dev, const int32_t* budget_dev,
-                      const int32_t* uncompressed_layers, int32_t n_uncompressed,
-                      const void* k_new, const void* v_new, const int32_t* pos_new_dev,
-                      void* workspace, size_t workspace_bytes, void* stream) {
+static int append_evict_impl(bool per_head, void* K_c, void* V_c, int32_t* idx, float* sumsq_c,
+                             const l2kv_layout* lay, int32_t* cur_len_dev,
+                             const int32_t* budget_dev, const int32_t* uncompressed_layers,
+                             int32_t n_uncompressed, const void* k_new, const void* v_new,
+                             const int32_t* pos_new_dev, void* workspace, size_t workspace_bytes,
+                             void* stream) {
   int rc = check_layout(lay);
   if (rc != L2KV_OK) return rc;
   LayerMask unc;
@@ -238,14 +239,36 @@ int l2kv_append_evict(void* K_c, void* V_c, int32_t* idx, float* sumsq_c, const 
   return launch_append_evict(K_c, V_c, idx, sumsq_c, make_geom(*lay), lay->dtype, cur_len_dev,
                              budget_dev, unc, k_new, v_new, pos_new_dev,
                              reinterpret_cast<int32_t*>(ws),
-                             reinterpret_cast<int32_t*>(ws + plan.ticket_off),
+                             reinterpret_cast<int32_t*>(ws + plan.ticket_off), per_head ? 1 : 0,
                              static_cast<cudaStream_t>(stream));
 }
 
-int l2kv_prefix_attention(const void* q, const void* K_c, const void* V_c, const l2kv_layout* lay,
-                          const int32_t* cur_len_dev, int32_t max_len, int32_t n_queries, float scale,
-                          float* out, float* lse_out, void* workspace, size_t workspace_bytes,
-                          void* stream) {
+int l2kv_append_evict(void* K_c, void* V_c, int32_t* idx, float* sumsq_c, const l2kv_layout* lay,
+                      int32_t* cur_len_dev, const int32_t* budget_dev,
+                      const int32_t* uncompressed_layers, int32_t n_uncompressed,
+                      const void* k_new, const void* v_new, const int32_t* pos_new_dev,
+                      void* workspace, size_t workspace_bytes, void* stream) {
+  return append_evict_impl(false, K_c, V_c, idx, sumsq_c, lay, cur_len_dev, budget_dev,
+                           uncompressed_layers, n_uncompressed, k_new, v_new, pos_new_dev,
+                           workspace, workspace_bytes, stream);
+}
+
+int l2kv_append_evict_per_head(void* K_c, void* V_c, int32_t* idx, float* sumsq_c,
+                               const l2kv_layout* lay, int32_t* cur_len_unit_dev,
+                               const int32_t* budget_unit_dev, const int32_t* uncompressed_layers,
+                               int32_t n_uncompressed, const void* k_new, const void* v_new,
+                               const int32_t* pos_new_dev, void* workspace, size_t workspace_bytes,
+                               void* stream) {
+  return append_evict_impl(true, K_c, V_c, idx, sumsq_c, lay, cur_len_unit_dev, budget_unit_dev,
+                           uncompressed_layers, n_uncompressed, k_new, v_new, pos_new_dev,
+                           workspace, workspace_bytes, stream);
+}
+
+static int prefix_attention_impl(bool per_head, const void* q, const void* K_c, const void* V_c,
+                                 const l2kv_layout* lay, const int32_t* cur_len_dev,
+                                 int32_t max_len, int32_t n_queries, float scale, float* out,
+                                 float* lse_out, void* workspace, size_t workspace_bytes,
+                                 void* stream) {
   int rc = check_layout(lay);
   if (rc != L2KV_OK) return rc;
   rc = check_groups(lay);
@@ -259,9 +282,27 @@ int l2kv_prefix_attention(const void* q, const void* K_c, const void* V_c, const
     return L2KV_ERR_MISALIGNED;
   if (workspace && workspace_bytes < (size_t)kStatusBytes) return L2KV_ERR_WORKSPACE_TOO_SMALL;
   const float sc = scale > 0.f ? scale : 1.0f / std::sqrt((float)lay->head_dim);
-  return launch_prefix_attention(q, K_c, V_c, make_geom(*lay), lay->dtype, n_queries, cur_len_dev,
+  const LenView lens{cur_len_dev, per_head ? 1 : 0};
+  return launch_prefix_attention(q, K_c, V_c, make_geom(*lay), lay->dtype, n_queries, lens,
                                  max_len, sc, out, lse_out, static_cast<int32_t*>(workspace),
                                  static_cast<cudaStream_t>(stream));
+}
+
+int l2kv_prefix_attention(const void* q, const void* K_c, const void* V_c, const l2kv_layout* lay,
+                          const int32_t* cur_len_dev, int32_t max_len, int32_t n_queries, float scale,
+                          float* out, float* lse_out, void* workspace, size_t workspace_bytes,
+                          void* stream) {
+  return prefix_attention_impl(false, q, K_c, V_c, lay, cur_len_dev, max_len, n_queries, scale, out,
+                               lse_out, workspace, workspace_bytes, stream);
+}
+
+int l2kv_prefix_attention_per_head(const void* q, const void* K_c, const void* V_c,
+                                   const l2kv_layout* lay, const int32_t* cur_len_unit_dev,
+                                   int32_t max_len, int32_t n_queries, float scale, float* out,
+                                   float* lse_out, void* workspace, size_t workspace_bytes,
+                                   void* stream) {
+  return prefix_attention_impl(true, q, K_c, V_c, lay, cur_len_unit_dev, max_len, n_queries, scale,
+                               out, lse_out, workspace, workspace_bytes, stream);
 }
 
 int l2kv_attention_loss_workspace_bytes(const l2kv_layout* lay, int32_t max_len, size_t* bytes) {

@@ -21,7 +21,7 @@ append_evict_kernel(T* __restrict__ K, T* __restrict__ V, int32_t* __restrict__ 
                     const int32_t* __restrict__ budget_dev, LayerMask unc,
                     const T* __restrict__ k_new, const T* __restrict__ v_new,
                     const int32_t* __restrict__ pos_new_dev, int32_t* __restrict__ status_word,
-                    int32_t* __restrict__ tickets) {
+                    int32_t* __restrict__ tickets, int per_head) {
   constexpr int EPV = Elem<T>::kPerVec;
   constexpr int LPR = D / EPV;
   constexpr int NW = kAppendThreads / 32;
@@ -34,8 +34,9 @@ append_evict_kernel(T* __restrict__ K, T* __restrict__ V, int32_t* __restrict__ 
   const int l = (int)(bl % g.L);
   const int b = (int)(bl / g.L);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int n = max(0, min(cur_len_dev[bl], g.t_cap));
-  const bool grow = unc.test(l) || n < budget_dev[b];
+  // per_head: a length and a budget of its own for every (b, l, h)
+  const int n = max(0, min(cur_len_dev[per_head ? unit : bl], g.t_cap));
+  const bool grow = unc.test(l) || n < budget_dev[per_head ? unit : (long long)b];
   const bool overflow = grow && n >= g.t_cap;
   const int pos_new = pos_new_dev[b];
 
@@ -133,9 +134,13 @@ append_evict_kernel(T* __restrict__ K, T* __restrict__ V, int32_t* __restrict__ 
     }
   }
 
-  // Ticket of (b, l): the last of the layer's heads to finish publishes the new length.
+  // Ticket of (b, l): the last of the layer's heads to finish publishes the new length.  With
+  // a length per head every CTA publishes its own.
   __syncthreads();
-  if (tid == 0) {
+  if (tid == 0 && per_head) {
+    if (overflow) atomicExch(status_word, (int)L2KV_ERR_DEVICE_OVERFLOW);
+    else if (grow) cur_len_dev[unit] = n + 1;
+  } else if (tid == 0) {
     __threadfence();
     if (atomicAdd(tickets + bl, 1) == g.H - 1) {
       if (overflow) atomicExch(status_word, (int)L2KV_ERR_DEVICE_OVERFLOW);
@@ -149,24 +154,24 @@ template <typename T, int D>
 static int launch_ae_t(void* K, void* V, int32_t* idx, float* sumsq, const Geom& g,
                        int32_t* cur_len_dev, const int32_t* budget_dev, const LayerMask& unc,
                        const void* k_new, const void* v_new, const int32_t* pos_new_dev,
-                       int32_t* status_word, int32_t* tickets, cudaStream_t s) {
+                       int32_t* status_word, int32_t* tickets, int per_head, cudaStream_t s) {
   const long long blocks = (long long)g.B * g.L * g.H;
   if (blocks == 0) return L2KV_OK;
   if (blocks > 0x7fffffffLL) return L2KV_ERR_OUT_OF_RANGE;
   append_evict_kernel<T, D><<<(unsigned)blocks, kAppendThreads, 0, s>>>(
       static_cast<T*>(K), static_cast<T*>(V), idx, sumsq, g, cur_len_dev, budget_dev, unc,
       static_cast<const T*>(k_new), static_cast<const T*>(v_new), pos_new_dev, status_word,
-      tickets);
+      tickets, per_head);
   return cudaGetLastError() == cudaSuccess ? L2KV_OK : L2KV_ERR_CUDA;
 }
 
 int launch_append_evict(void* K, void* V, int32_t* idx, float* sumsq, const Geom& g, int dtype,
                         int32_t* cur_len_dev, const int32_t* budget_dev, const LayerMask& unc,
                         const void* k_new, const void* v_new, const int32_t* pos_new_dev,
-                        int32_t* status_word, int32_t* tickets, cudaStream_t s) {
+                        int32_t* status_word, int32_t* tickets, int per_head, cudaStream_t s) {
 #define L2KV_AE(T, D)                                                                            \
   return launch_ae_t<T, D>(K, V, idx, sumsq, g, cur_len_dev, budget_dev, unc, k_new, v_new,      \
-                           pos_new_dev, status_word, tickets, s)
+                           pos_new_dev, status_word, tickets, per_head, s)
   if (dtype == L2KV_BF16) {
     if (g.D == 128) L2KV_AE(__nv_bfloat16, 128);
     if (g.D == 64) L2KV_AE(__nv_bfloat16, 64);

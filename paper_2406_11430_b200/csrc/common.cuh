@@ -224,10 +224,10 @@ int launch_decode_attention(const void* q, const void* K, const void* V, const G
 int launch_append_evict(void* K, void* V, int32_t* idx, float* sumsq, const Geom& g, int dtype,
                         int32_t* cur_len_dev, const int32_t* budget_dev, const LayerMask& unc,
                         const void* k_new, const void* v_new, const int32_t* pos_new_dev,
-                        int32_t* status_word, int32_t* tickets, cudaStream_t s);
+                        int32_t* status_word, int32_t* tickets, int per_head, cudaStream_t s);
 
 int launch_prefix_attention(const void* q, const void* K, const void* V, const Geom& g, int dtype,
-                            int n_queries, const int32_t* cur_len_dev, int max_len, float scale,
+                            int n_queries, const LenView& cur_len_dev, int max_len, float scale,
                             float* out, float* lse_out, int32_t* status_word, cudaStream_t s);
 size_t attention_loss_workspace(const l2kv_layout& a, int max_len);
 int launch_attention_loss(const void* q, const void* K, const Geom& g, int dtype,

@@ -137,7 +137,7 @@ constexpr float kPfRescaleGap = 8.f;            // log2 units a maximum may drif
 template <int G>
 __global__ void __launch_bounds__(kPfThreads, 2)
 prefix_attention_basic_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n_queries,
-                           const int32_t* __restrict__ cur_len_dev, int max_len, float scale_log2e,
+                           LenView cur_len_dev, int max_len, float scale_log2e,
                            float* __restrict__ out, float* __restrict__ lse_out,
                            const __grid_constant__ CUtensorMap map_k,
                            const __grid_constant__ CUtensorMap map_v,
@@ -156,7 +156,7 @@ prefix_attention_basic_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n
   const int h = (int)(unit % g.H);
   const long long bl = unit / g.H;
   const int l = (int)(bl % g.L), b = (int)(bl / g.L);
-  const int n = max(0, min(cur_len_dev[bl], min(max_len, g.t_cap)));
+  const int n = max(0, min(cur_len_dev.at(bl, h, g.H), min(max_len, g.t_cap)));
   // Two threads per query row: thread (row, hf) owns score columns and output dims
   // [64 hf, 64 hf + 64).  Warps w and w + 4 share a tensor-memory lane quarter.
   const int tid = threadIdx.x, warp = tid >> 5;
@@ -405,7 +405,7 @@ constexpr int kPf5Threads = 2 * kPfRows + 4 * 32;      // softmax A, softmax B, 
 template <int G>
 __global__ void __launch_bounds__(kPf5Threads, 1)
 prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n_queries,
-                           const int32_t* __restrict__ cur_len_dev, int max_len, float scale_log2e,
+                           LenView cur_len_dev, int max_len, float scale_log2e,
                            float* __restrict__ out, float* __restrict__ lse_out,
                            const __grid_constant__ CUtensorMap map_k,
                            const __grid_constant__ CUtensorMap map_v,
@@ -427,7 +427,7 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
   const int h = (int)(unit % g.H);
   const long long bl = unit / g.H;
   const int l = (int)(bl % g.L), b = (int)(bl / g.L);
-  const int n = max(0, min(cur_len_dev[bl], min(max_len, g.t_cap)));
+  const int n = max(0, min(cur_len_dev.at(bl, h, g.H), min(max_len, g.t_cap)));
   const int tid = threadIdx.x, warp = tid >> 5;
   const bool softmax_thread = tid < 2 * kPfRows;
   const int n_tiles = (2 * qp + 1 < q_tiles) ? 2 : 1;   // query tiles of this CTA that exist
@@ -671,7 +671,7 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
 
 template <int G>
 static int launch_pf(const void* q, const void* K, const void* V, const Geom& g, int n_queries,
-                     const int32_t* cur_len_dev, int max_len, float scale, float* out,
+                     const LenView& cur_len_dev, int max_len, float scale, float* out,
                      float* lse_out, int32_t* status_word, cudaStream_t s) {
   constexpr int QT = kPfRows / G;
   const long long units = (long long)g.B * g.L * g.H;
@@ -710,7 +710,7 @@ static int launch_pf(const void* q, const void* K, const void* V, const Geom& g,
 }
 
 int launch_prefix_attention(const void* q, const void* K, const void* V, const Geom& g, int dtype,
-                            int n_queries, const int32_t* cur_len_dev, int max_len, float scale,
+                            int n_queries, const LenView& cur_len_dev, int max_len, float scale,
                             float* out, float* lse_out, int32_t* status_word, cudaStream_t s) {
   if (dtype != L2KV_BF16 || g.D != 128) return L2KV_ERR_UNSUPPORTED;
   switch (g.Hq / g.H) {

@@ -112,3 +112,83 @@ def test_per_head_pipeline_compress_then_attend(l2):
     want = oracle.attention(synth.to_numpy(q), ref["K_c"], ref["V_c"], "bf16", ref["kept_len"],
                             nthreads=8)
     assert_attention_close(out.cpu().numpy(), want)
+
+
+def _oracle_state(r, t_cap):
+    B, L, H, t0, D = r["K_c"].shape
+    st = dict(K_c=np.zeros((B, L, H, t_cap, D), r["K_c"].dtype),
+              idx=np.full((B, L, H, t_cap), -1, np.int32),
+              key=np.full((B, L, H, t_cap), np.nan), cur_len=r["kept_len"].copy())
+    st["V_c"] = np.zeros_like(st["K_c"])
+    for name in ("K_c", "V_c", "idx", "key"):
+        st[name][:, :, :, :t0] = r[name]
+    return st
+
+
+@pytest.mark.parametrize("dtype,D", [("bf16", 128), ("f32", 64)])
+def test_append_evict_with_a_budget_per_head(l2, dtype, D):
+    """A stream of appends with a length and a budget per (b, l, h): state bit-exact against the
+    oracle (fp32 key order) along the way, then decode and prefix attention over the result."""
+    steps, T0 = 40, 600
+    w = synth.WORKLOADS[4].scaled(dtype=dtype, D=D, B=2, L=3, Hkv=2, Hq=8, T=T0, ragged_lo=0)
+    K, V = synth.make_cache(w, DEV)
+    Kn, Vn = synth.to_numpy(K), synth.to_numpy(V)
+    lens = [600, 90]
+    rng = np.random.default_rng(17)
+    keep = np.stack([rng.integers(1, n + 1, size=(w.L, w.Hkv)) for n in lens]).astype(np.int32)
+    budget = keep.copy()
+    keep[1, 2, 0], budget[1, 2, 0] = 90, 100              # fills up after 10 appends, then evicts
+    keep[0, 2, 1], budget[0, 2, 1] = 600, 10_000          # never full
+    t_cap = T0 + steps
+    dev, _ = gpu_compress_per_head(l2, K, V, lens, keep, unc=(0,), t_cap_out=t_cap)
+    st = _oracle_state(oracle.compress(Kn, Vn, dtype, lens, keep, (0,), key_mode=1, t_cap_out=T0),
+                       t_cap)
+    ws = l2.new_workspace(l2.Layout(dev["K_c"], q_heads=w.Hq), t_cap, DEV)
+    bud = i32(budget)
+    for s in range(steps):
+        k, v = synth.make_new_kv(w, s, DEV)
+        pos = [n + s for n in lens]
+        l2.append_evict_per_head(dev["K_c"], dev["V_c"], dev["idx"], dev["sumsq"], dev["kept_len"],
+                                 bud, (0,), k, v, i32(pos), ws)
+        assert oracle.append_evict(st, dtype, budget, (0,), synth.to_numpy(k), synth.to_numpy(v),
+                                   pos, key_mode=1) == 0
+        if s % 13 == 12 or s == steps - 1:
+            torch.cuda.synchronize()
+            cur = dev["kept_len"].cpu().numpy()
+            assert np.array_equal(cur, st["cur_len"])
+            for b, l, h in np.ndindex(2, w.L, w.Hkv):
+                n = cur[b, l, h]
+                assert np.array_equal(dev["idx"][b, l, h, :n].cpu().numpy(), st["idx"][b, l, h, :n])
+                assert np.array_equal(synth.to_numpy(dev["K_c"][b, l, h, :n]), st["K_c"][b, l, h, :n])
+                assert np.array_equal(synth.to_numpy(dev["V_c"][b, l, h, :n]), st["V_c"][b, l, h, :n])
+                assert np.array_equal(dev["sumsq"][b, l, h, :n].cpu().numpy().astype(np.float64),
+                                      st["key"][b, l, h, :n])
+    assert l2.read_device_status(ws) == 0
+    q = synth.make_query(w, 1, DEV)
+    out = torch.full(q.shape, float("nan"), dtype=torch.float32, device=DEV)
+    l2.decode_attention_per_head(q, dev["K_c"], dev["V_c"], dev["kept_len"], t_cap, out, ws)
+    torch.cuda.synchronize()
+    want = oracle.attention(synth.to_numpy(q), st["K_c"], st["V_c"], dtype, st["cur_len"], nthreads=8)
+    assert_attention_close(out.cpu().numpy(), want)
+
+
+@pytest.mark.parametrize("kernel", ["pipelined", "basic"])
+def test_prefix_attention_with_a_length_per_head(l2, kernel, monkeypatch):
+    monkeypatch.setenv("L2KV_PREFIX_KERNEL", kernel)
+    w = synth.WORKLOADS[2].scaled(B=1, L=2, Hkv=2, Hq=8, T=700)
+    K, V = synth.make_cache(w, DEV)
+    g = torch.Generator().manual_seed(5)
+    q = torch.randn((1, 2, 37, 8, 128), generator=g).to(torch.bfloat16).to(DEV)
+    cur = np.array([[[700, 65], [0, 129]]], dtype=np.int32)
+    out = torch.full(q.shape, float("nan"), dtype=torch.float32, device=DEV)
+    lse = torch.full(q.shape[:4], float("nan"), dtype=torch.float32, device=DEV)
+    ws = torch.zeros(256, dtype=torch.uint8, device=DEV)
+    l2.prefix_attention_per_head(q, K, V, i32(cur), 700, out, lse, workspace=ws)
+    torch.cuda.synchronize()
+    assert l2.read_device_status(ws) == 0
+    got = out.cpu().numpy()
+    Kn, Vn = synth.to_numpy(K), synth.to_numpy(V)
+    for s in range(37):
+        want = oracle.attention(synth.to_numpy(q[:, :, s].contiguous()), Kn, Vn, "bf16", cur, nthreads=8)
+        assert_attention_close(got[:, :, s], want, atol=4e-3)
+    assert not got[0, 1, :, :4].any() and np.all(np.isneginf(lse[0, 1, :, :4].cpu().numpy()))
