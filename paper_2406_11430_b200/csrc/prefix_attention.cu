@@ -542,10 +542,13 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
         ok = mbar_wait<kPfPolls>(bar_k(1 % NS), 0);
         if (ok) { tc_fence_after(); issue_qk(1); }
       }
-      if (ok) ok = mbar_wait<kPfPolls>(bar_v(0), 0);
       for (int j = 0; ok && j < nb; ++j) {
         const int s = j & 1;
-        ok = mbar_wait<kPfPolls>(bar_p(s), (uint32_t)(j >> 1) & 1u);
+        // The tiles this iteration needs were fetched well ahead; checking them here, while the
+        // softmax still works on S(j), keeps the checks off the path from weights to scores.
+        ok = mbar_wait_likely(bar_v(j % NS), (uint32_t)(j / NS) & 1u);
+        if (ok && j + 2 < nb) ok = mbar_wait_likely(bar_k((j + 2) % NS), (uint32_t)((j + 2) / NS) & 1u);
+        ok = ok && mbar_wait<kPfPolls>(bar_p(s), (uint32_t)(j >> 1) & 1u);
         if (!ok) break;
         tc_fence_after();
         const uint32_t vt = sV + (j % NS) * kPf3Tile;
@@ -555,11 +558,8 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
                        umma_desc(vt + k * 2048, kPf3Half, 1024), kIdescPV, (j > 0 || k > 0) ? 1u : 0u);
         umma_commit(bar_o);
         umma_commit(bar_vfree(j % NS));
-        // tiles fetched well ahead: these two are normally over already
-        if (j + 2 < nb) ok = mbar_wait_likely(bar_k((j + 2) % NS), (uint32_t)((j + 2) / NS) & 1u);
-        if (ok && j + 1 < nb) ok = mbar_wait_likely(bar_v((j + 1) % NS), (uint32_t)((j + 1) / NS) & 1u);
         // P(j) V(j) done: the score buffer it read its weights from takes sub-block j + 2
-        ok = ok && mbar_wait<kPfPolls>(bar_o, (uint32_t)j & 1u);
+        ok = mbar_wait<kPfPolls>(bar_o, (uint32_t)j & 1u);
         if (!ok) break;
         if (j + 2 < nb) { tc_fence_after(); issue_qk(j + 2); }
       }
