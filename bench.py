@@ -328,6 +328,8 @@ def time_variants(job, w, cbytes, reps=5):
     job.compress()                     # leave the cache as the method's own policy makes it
     torch.cuda.synchronize()
     out["append_evict"] = time_append_evict(job, w)
+    if not w.append_steps:
+        out["decode_cuda_graph"] = time_decode_graph(job, w)
     # attention-loss analysis (Eqs. 5-7) of the full cache: keys from above, first query
     lens_bl = torch.full((w.B, w.L), w.T, dtype=torch.int32, device=job.dev)
     alr = torch.zeros((w.B, w.L, w.Hq), dtype=torch.float32, device=job.dev)
@@ -369,6 +371,39 @@ def time_variants(job, w, cbytes, reps=5):
     job.compress()
     torch.cuda.synchronize()
     return out
+
+
+def time_decode_graph(job, w, reps=5):
+    """The step's decode calls captured once in a CUDA graph and replayed: what a serving loop
+    does to take the launch overhead off short decode steps (the calls allocate nothing and are
+    ordered on the caller's stream, so they capture as they are)."""
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        job.decode(0)                                   # first call on this stream, outside capture
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        for s in range(w.decode_steps):
+            job.decode(s)
+
+    def timed(fn):
+        fn(); torch.cuda.synchronize()
+        t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+        t0.record()
+        for _ in range(reps):
+            fn()
+        t1.record(); torch.cuda.synchronize()
+        return t0.elapsed_time(t1) / reps / w.decode_steps
+
+    def eager():
+        for s in range(w.decode_steps):
+            job.decode(s)
+
+    ms_graph, ms_eager = timed(graph.replay), timed(eager)
+    return {"ms_per_decode_step": round(ms_graph, 5), "eager_ms_per_decode_step": round(ms_eager, 5),
+            "decode_steps_in_graph": w.decode_steps}
 
 
 def time_append_evict(job, w, reps=20):
