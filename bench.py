@@ -346,28 +346,29 @@ def time_variants(job, w, cbytes, reps=5):
                              "tokens_per_head": w.T, "mean_alr": round(float(alr.mean().item()), 2)}
     del ws_al
     # prefix attention: 128 new queries per (b, l) over the compressed cache (tensor-bound)
-    n_q = 128
-    job.compress()
-    qp = torch.randn((w.B, w.L, n_q, w.Hq, w.D), device=job.dev).to(torch.bfloat16)
-    op = torch.empty(qp.shape, dtype=torch.float32, device=job.dev)
-    job.l2.prefix_attention(qp, job.K_c, job.V_c, job.cur, job.t_cap, op)
-    t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
-    t0.record()
-    for _ in range(3):
+    if w.dtype == "bf16" and w.D == 128:             # the tensor-core kernel's types
+        n_q = 128
+        job.compress()
+        qp = torch.randn((w.B, w.L, n_q, w.Hq, w.D), device=job.dev).to(torch.bfloat16)
+        op = torch.empty(qp.shape, dtype=torch.float32, device=job.dev)
         job.l2.prefix_attention(qp, job.K_c, job.V_c, job.cur, job.t_cap, op)
-    t1.record(); torch.cuda.synchronize()
-    ms = t0.elapsed_time(t1) / 3
-    flop = 4.0 * n_q * w.Hq * w.D * float(job.cur.sum().item())
-    tf_peak = None
-    try:
-        tf_peak = float(json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))["bf16_tflops_sustained"])
-    except Exception:
-        pass
-    out["prefix_attention"] = {"ms": round(ms, 3), "queries_per_sequence": n_q,
-                               "TFLOPs": round(flop / ms / 1e9, 1), "bound": "tensor",
-                               "peak_TFLOPs_measured_sustained": tf_peak,
-                               "frac": round(flop / ms / 1e9 / tf_peak, 4) if tf_peak else None}
-    del qp, op
+        t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+        t0.record()
+        for _ in range(3):
+            job.l2.prefix_attention(qp, job.K_c, job.V_c, job.cur, job.t_cap, op)
+        t1.record(); torch.cuda.synchronize()
+        ms = t0.elapsed_time(t1) / 3
+        flop = 4.0 * n_q * w.Hq * w.D * float(job.cur.sum().item())
+        tf_peak = None
+        try:
+            tf_peak = float(json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))["bf16_tflops_sustained"])
+        except Exception:
+            pass
+        out["prefix_attention"] = {"ms": round(ms, 3), "queries_per_sequence": n_q,
+                                   "TFLOPs": round(flop / ms / 1e9, 1), "bound": "tensor",
+                                   "peak_TFLOPs_measured_sustained": tf_peak,
+                                   "frac": round(flop / ms / 1e9 / tf_peak, 4) if tf_peak else None}
+        del qp, op
     job.compress()
     torch.cuda.synchronize()
     return out
