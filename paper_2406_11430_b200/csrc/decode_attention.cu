@@ -208,13 +208,33 @@ decode_combine_kernel(const float* __restrict__ partial, LenView cur_len_dev,
   const int ns = (n + kDecodeChunk - 1) / kDecodeChunk;
   const int d = threadIdx.x;
   const float* p = partial + row * n_splits * (long long)(D + 2);
+  __shared__ float s_w[D], s_l[D], s_red[D / 32];
+  // the splits' maxima: strided over the threads, then reduced (exact in any order)
   float m = -INFINITY;
-  for (int s = 0; s < ns; ++s) m = fmaxf(m, p[s * (D + 2)]);
+  for (int s = d; s < ns; s += D) m = fmaxf(m, p[s * (D + 2)]);
+#pragma unroll
+  for (int off = 16; off >= 1; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+  if ((d & 31) == 0) s_red[d >> 5] = m;
+  __syncthreads();
+#pragma unroll
+  for (int w = 0; w < D / 32; ++w) m = fmaxf(m, s_red[w]);
+  // D splits at a time: their weights and sums go to shared memory once, then every thread adds
+  // its output element over the splits in order (independent loads, same sums as a plain loop)
   float den = 0.f, num = 0.f;
-  for (int s = 0; s < ns; ++s) {
-    const float w = exp2f(p[s * (D + 2)] - m);
-    den = fmaf(w, p[s * (D + 2) + 1], den);
-    num = fmaf(w, p[s * (D + 2) + 2 + d], num);
+  for (int s0 = 0; s0 < ns; s0 += D) {
+    const int tile = min(D, ns - s0);
+    __syncthreads();
+    if (d < tile) {
+      s_w[d] = exp2f(p[(s0 + d) * (D + 2)] - m);
+      s_l[d] = p[(s0 + d) * (D + 2) + 1];
+    }
+    __syncthreads();
+    const float* acc = p + (long long)s0 * (D + 2) + 2 + d;
+#pragma unroll 8
+    for (int t = 0; t < tile; ++t) {
+      den = fmaf(s_w[t], s_l[t], den);
+      num = fmaf(s_w[t], acc[t * (D + 2)], num);
+    }
   }
   out[row * D + d] = ns > 0 ? num / den : 0.f;
 }
