@@ -364,13 +364,13 @@ prefix_attention_basic_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n
 }
 
 // The pipelined kernel walks the cache in sub-blocks of 64 tokens.
-constexpr int kPf3Sub = 64;                     // cached tokens per sub-block
-constexpr int kPf3Half = kPf3Sub * 128;         // one [64 tokens][64 bf16] swizzled tile: 8 KB
-constexpr int kPf3Tile = 2 * kPf3Half;          // both halves of the head dimension: 16 KB
+constexpr int kPfSub = 64;                      // cached tokens per sub-block
+constexpr int kPfSubHalf = kPfSub * 128;        // one [64 tokens][64 bf16] swizzled tile: 8 KB
+constexpr int kPfSubTile = 2 * kPfSubHalf;      // both halves of the head dimension: 16 KB
 constexpr uint32_t kIdescQK64 =
     (1u << 4) | (1u << 7) | (1u << 10) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
-constexpr int kPf4Stages = 4;                   // K tiles (and V tiles) in flight
-constexpr int kPf4TmemCols = 512;
+constexpr int kPfStages = 4;                    // K tiles (and V tiles) in flight
+constexpr int kPfPipeTmemCols = 512;            // two query tiles x (2 x 64 score + 128 output columns)
 
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(bar) : "memory");
@@ -400,10 +400,10 @@ __device__ __forceinline__ bool mbar_wait_likely(uint32_t bar, uint32_t parity) 
 //     V tiles by TMA into rings of four tiles each, freed by tcgen05.commit.
 // Hand-offs are mbarriers (scores ready / tile free / output quiet: tcgen05.commit; weights
 // ready: one arrival per softmax warp); every wait on them is bounded.
-constexpr int kPf5Threads = 2 * kPfRows + 4 * 32;      // softmax A, softmax B, issuer A, issuer B, K, V
+constexpr int kPfPipeThreads = 2 * kPfRows + 4 * 32;      // softmax A, softmax B, issuer A, issuer B, K, V
 
 template <int G>
-__global__ void __launch_bounds__(kPf5Threads, 1)
+__global__ void __launch_bounds__(kPfPipeThreads, 1)
 prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n_queries,
                            LenView cur_len_dev, int max_len, float scale_log2e,
                            float* __restrict__ out, float* __restrict__ lse_out,
@@ -412,7 +412,7 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
                            int32_t* __restrict__ status_word) {
   constexpr int D = 128;
   constexpr int QT = kPfRows / G;                       // queries per query tile
-  constexpr int NS = kPf4Stages;
+  constexpr int NS = kPfStages;
   extern __shared__ unsigned char smem_raw[];
   // mbarriers: K landed [NS], V landed [NS], K tile free [NS], V tile free [NS], then per query
   // tile: scores ready [2], weights ready [2], output quiet [1]
@@ -448,11 +448,11 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
   }
   // A wait that gave up in an earlier CTA marks the workspace; the rest of the grid leaves.
   if (status_word && *reinterpret_cast<volatile int32_t*>(status_word + 2) != 0) return;
-  const int nb = (n + kPf3Sub - 1) / kPf3Sub;
+  const int nb = (n + kPfSub - 1) / kPfSub;
 
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;   // 1024-byte aligned tiles
   const uint32_t sQ = base + (uint32_t)tile * kPfTileBytes;      // this query tile's rows
-  const uint32_t sK = base + 2 * kPfTileBytes, sV = sK + NS * kPf3Tile;
+  const uint32_t sK = base + 2 * kPfTileBytes, sV = sK + NS * kPfSubTile;
   const uint32_t bar0 = smem_u32(&s_bar[0]);
   auto bar_k = [&](int i) { return bar0 + 8u * (uint32_t)i; };
   auto bar_v = [&](int i) { return bar0 + 8u * (uint32_t)(NS + i); };
@@ -465,7 +465,7 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
 
   if (warp == 0) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                 :: "r"(smem_u32(&s_tmem)), "r"(kPf4TmemCols) : "memory");
+                 :: "r"(smem_u32(&s_tmem)), "r"(kPfPipeTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   if (tid == 0) {
@@ -518,21 +518,21 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
         const uint32_t full = is_k ? bar_k(st) : bar_v(st);
         if (use > 0) ok = mbar_wait<kPfPolls>(is_k ? bar_kfree(st) : bar_vfree(st), (uint32_t)(use - 1) & 1u);
         if (!ok) break;
-        const uint32_t dst = (is_k ? sK : sV) + st * kPf3Tile;
-        mbar_expect_tx(full, kPf3Tile);
-        tma_load_5d(dst, map, full, 0, j * kPf3Sub, h, l, b);
-        tma_load_5d(dst + kPf3Half, map, full, 64, j * kPf3Sub, h, l, b);
+        const uint32_t dst = (is_k ? sK : sV) + st * kPfSubTile;
+        mbar_expect_tx(full, kPfSubTile);
+        tma_load_5d(dst, map, full, 0, j * kPfSub, h, l, b);
+        tma_load_5d(dst + kPfSubHalf, map, full, 64, j * kPfSub, h, l, b);
       }
       if (!ok) s_fail = 1;
     } else if ((tid & 31) == 0 && tile_active) {
       // ---- the issuing thread of query tile `tile` ---------------------------------------------
       auto issue_qk = [&](int j) {                      // S[j & 1] = Q K(j)^T; then the K tile is free
-        const uint32_t kt = sK + (j % NS) * kPf3Tile;
+        const uint32_t kt = sK + (j % NS) * kPfSubTile;
 #pragma unroll
         for (int k = 0; k < 8; ++k)
           umma_bf16(tmem + (j & 1) * 64,
                     umma_desc(sQ + (k >> 2) * kPfHalf + (k & 3) * 32, 16, 1024),
-                    umma_desc(kt + (k >> 2) * kPf3Half + (k & 3) * 32, 16, 1024), kIdescQK64, k > 0);
+                    umma_desc(kt + (k >> 2) * kPfSubHalf + (k & 3) * 32, 16, 1024), kIdescQK64, k > 0);
         umma_commit(bar_s(j & 1));
         umma_commit(bar_kfree(j % NS));
       };
@@ -551,11 +551,11 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
         ok = ok && mbar_wait<kPfPolls>(bar_p(s), (uint32_t)(j >> 1) & 1u);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t vt = sV + (j % NS) * kPf3Tile;
+        const uint32_t vt = sV + (j % NS) * kPfSubTile;
 #pragma unroll
         for (int k = 0; k < 4; ++k)                     // O += P(j) V(j); slice k = tokens 16k .. 16k + 15
           umma_bf16_ts(tmem + 128, tmem + s * 64 + k * 8,
-                       umma_desc(vt + k * 2048, kPf3Half, 1024), kIdescPV, (j > 0 || k > 0) ? 1u : 0u);
+                       umma_desc(vt + k * 2048, kPfSubHalf, 1024), kIdescPV, (j > 0 || k > 0) ? 1u : 0u);
         umma_commit(bar_o);
         umma_commit(bar_vfree(j % NS));
         // P(j) V(j) done: the score buffer it read its weights from takes sub-block j + 2
@@ -569,7 +569,7 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
     // ---- the softmax warps of query tile `tile`: one thread per row ----------------------------
     for (int j = 0; j < nb; ++j) {
       const int s = j & 1;
-      const int valid = min(kPf3Sub, n - j * kPf3Sub);       // valid tokens of this sub-block
+      const int valid = min(kPfSub, n - j * kPfSub);       // valid tokens of this sub-block
       const uint32_t t_s = t_lane + s * 64;                   // this row's scores, later its weights
       if (!mbar_wait_likely(bar_s(s), (uint32_t)(j >> 1) & 1u)) gave_up = true;
       tc_fence_after();
@@ -580,7 +580,7 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
       for (int c = 0; c < 2; ++c) {
         uint32_t r[32];
         tmem_ld32(t_s + c * 32, r);
-        if (valid >= kPf3Sub) {                           // CTA-uniform: only the last sub-block masks
+        if (valid >= kPfSub) {                           // CTA-uniform: only the last sub-block masks
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
             sv[c * 32 + i] = __uint_as_float(r[i]);
@@ -635,15 +635,15 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
         tmem_wait_st();
         l_run += rowsum0 + rowsum1;
       }
-      if (valid < kPf3Sub) {
+      if (valid < kPfSub) {
         // Last, partial sub-block: rows of the V tile past the valid length hold whatever the
         // cache holds there; clear them so that a zero weight times Inf/NaN cannot reach O
         // (both query tiles write the same zeros).
         if (!mbar_wait<kPfPolls>(bar_v(j % NS), (uint32_t)(j / NS) & 1u)) gave_up = true;
-        if (row >= valid && row < kPf3Sub) {
+        if (row >= valid && row < kPfSub) {
 #pragma unroll
           for (int c = 0; c < 16; ++c)
-            st_shared16(sV + (j % NS) * kPf3Tile + (c >> 3) * kPf3Half + row * 128 + ((c & 7) << 4), 0, 0, 0, 0);
+            st_shared16(sV + (j % NS) * kPfSubTile + (c >> 3) * kPfSubHalf + row * 128 + ((c & 7) << 4), 0, 0, 0, 0);
         }
         proxy_fence();
       }
@@ -683,7 +683,7 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
   tc_fence_before();
   __syncthreads();
   if (warp == 0)
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(s_tmem), "r"(kPf4TmemCols)
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(s_tmem), "r"(kPfPipeTmemCols)
                  : "memory");
 }
 
@@ -702,17 +702,17 @@ static int launch_pf(const void* q, const void* K, const void* V, const Geom& g,
   // L2KV_PREFIX_KERNEL=basic selects the single-role kernel; the pipelined one is the default.
   const char* which = std::getenv("L2KV_PREFIX_KERNEL");
   const bool basic = which && std::strcmp(which, "basic") == 0;
-  const int sub_rows = basic ? kPfRows : kPf3Sub;
+  const int sub_rows = basic ? kPfRows : kPfSub;
   if (!make_cache_map(&map_k, K, g, sub_rows) || !make_cache_map(&map_v, V, g, sub_rows))
     return L2KV_ERR_UNSUPPORTED;
   if (!basic) {
-    constexpr int smem4 = 1024 + 2 * kPfTileBytes + 2 * kPf4Stages * kPf3Tile;
+    constexpr int smem_pipe = 1024 + 2 * kPfTileBytes + 2 * kPfStages * kPfSubTile;
     const int q_tiles = (n_queries + QT - 1) / QT;
-    const long long blocks4 = units * ((q_tiles + 1) / 2);
-    auto kern4 = prefix_attention_pipelined_kernel<G>;
-    if (cudaFuncSetAttribute(kern4, cudaFuncAttributeMaxDynamicSharedMemorySize, smem4) != cudaSuccess)
+    const long long blocks_pipe = units * ((q_tiles + 1) / 2);
+    auto kern_pipe = prefix_attention_pipelined_kernel<G>;
+    if (cudaFuncSetAttribute(kern_pipe, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_pipe) != cudaSuccess)
       return L2KV_ERR_CUDA;
-    kern4<<<(unsigned)blocks4, kPf5Threads, smem4, s>>>(
+    kern_pipe<<<(unsigned)blocks_pipe, kPfPipeThreads, smem_pipe, s>>>(
         static_cast<const __nv_bfloat16*>(q), g, n_queries, cur_len_dev, max_len, scale * kPfLog2e, out,
         lse_out, map_k, map_v, status_word);
     return cudaGetLastError() == cudaSuccess ? L2KV_OK : L2KV_ERR_CUDA;
