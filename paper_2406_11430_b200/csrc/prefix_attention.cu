@@ -381,13 +381,6 @@ __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
                "selp.u32 %0, 1, 0, p; }" : "=r"(done) : "r"(bar), "r"(parity) : "memory");
   return done != 0;
 }
-// A wait by a single latency-critical thread: non-blocking tests in a loop (no suspension, so
-// the completion is seen as soon as it is visible); bounded like every other wait.
-__device__ __forceinline__ bool mbar_spin(uint32_t bar, uint32_t parity) {
-  for (int spin = 0; spin < (1 << (kPfPolls + 4)); ++spin)
-    if (mbar_test(bar, parity)) return true;
-  return false;
-}
 // A wait that is usually over already: one non-blocking test first.
 __device__ __forceinline__ bool mbar_wait_likely(uint32_t bar, uint32_t parity) {
   return mbar_test(bar, parity) || mbar_wait<kPfPolls>(bar, parity);
@@ -555,7 +548,7 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
         // softmax still works on S(j), keeps the checks off the path from weights to scores.
         ok = mbar_wait_likely(bar_v(j % NS), (uint32_t)(j / NS) & 1u);
         if (ok && j + 2 < nb) ok = mbar_wait_likely(bar_k((j + 2) % NS), (uint32_t)((j + 2) / NS) & 1u);
-        ok = ok && mbar_spin(bar_p(s), (uint32_t)(j >> 1) & 1u);
+        ok = ok && mbar_wait<kPfPolls>(bar_p(s), (uint32_t)(j >> 1) & 1u);
         if (!ok) break;
         tc_fence_after();
         const uint32_t vt = sV + (j % NS) * kPfSubTile;
@@ -566,7 +559,7 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
         umma_commit(bar_o);
         umma_commit(bar_vfree(j % NS));
         // P(j) V(j) done: the score buffer it read its weights from takes sub-block j + 2
-        ok = mbar_spin(bar_o, (uint32_t)j & 1u);
+        ok = mbar_wait<kPfPolls>(bar_o, (uint32_t)j & 1u);
         if (!ok) break;
         if (j + 2 < nb) { tc_fence_after(); issue_qk(j + 2); }
       }
