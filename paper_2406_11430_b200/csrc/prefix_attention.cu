@@ -66,17 +66,6 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
                : "r"(taddr));
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
-// 64 consecutive fp32 columns of this thread's tensor-memory lane: both loads are issued before
-// the one wait, so their latencies overlap.  Whole warps only.
-__device__ __forceinline__ void tmem_ld64(uint32_t taddr, uint32_t (&a)[32], uint32_t (&b)[32]) {
-  asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%64];\n\t"
-               "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, %48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%65];\n\t"
-               "tcgen05.wait::ld.sync.aligned;"
-               : "=r"(a[0]), "=r"(a[1]), "=r"(a[2]), "=r"(a[3]), "=r"(a[4]), "=r"(a[5]), "=r"(a[6]), "=r"(a[7]), "=r"(a[8]), "=r"(a[9]), "=r"(a[10]), "=r"(a[11]), "=r"(a[12]), "=r"(a[13]), "=r"(a[14]), "=r"(a[15]), "=r"(a[16]), "=r"(a[17]), "=r"(a[18]), "=r"(a[19]), "=r"(a[20]), "=r"(a[21]), "=r"(a[22]), "=r"(a[23]), "=r"(a[24]), "=r"(a[25]), "=r"(a[26]), "=r"(a[27]), "=r"(a[28]), "=r"(a[29]), "=r"(a[30]), "=r"(a[31]),
-                 "=r"(b[0]), "=r"(b[1]), "=r"(b[2]), "=r"(b[3]), "=r"(b[4]), "=r"(b[5]), "=r"(b[6]), "=r"(b[7]), "=r"(b[8]), "=r"(b[9]), "=r"(b[10]), "=r"(b[11]), "=r"(b[12]), "=r"(b[13]), "=r"(b[14]), "=r"(b[15]), "=r"(b[16]), "=r"(b[17]), "=r"(b[18]), "=r"(b[19]), "=r"(b[20]), "=r"(b[21]), "=r"(b[22]), "=r"(b[23]), "=r"(b[24]), "=r"(b[25]), "=r"(b[26]), "=r"(b[27]), "=r"(b[28]), "=r"(b[29]), "=r"(b[30]), "=r"(b[31])
-               : "r"(taddr), "r"(taddr + 32)
-               : "memory");
-}
 // A operand taken from tensor memory (bf16 pairs packed two per 32-bit column, row = lane).
 __device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc,
                                              uint32_t idesc, uint32_t accumulate) {
@@ -95,15 +84,6 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
                   "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]),
                   "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]),
                   "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
-               : "memory");
-}
-// Stores 16 consecutive 32-bit columns of this thread's tensor-memory lane.  Whole warps only.
-__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
-  asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
-               "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
-               :: "r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]),
-                  "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]),
-                  "r"(r[14]), "r"(r[15])
                : "memory");
 }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
@@ -436,7 +416,7 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
   extern __shared__ unsigned char smem_raw[];
   // mbarriers: K landed [NS], V landed [NS], K tile free [NS], V tile free [NS], then per query
   // tile: scores ready [2], weights ready [2], output quiet [1]
-  __shared__ __align__(8) unsigned long long s_bar[4 * NS + 10 + 8 + 4];   // + turn of A [4], turn of B [4], first half of the weights ready [2][2]
+  __shared__ __align__(8) unsigned long long s_bar[4 * NS + 10 + 8];   // + turn of A [4], turn of B [4]
   __shared__ uint32_t s_tmem;
   __shared__ int s_fail;
 
@@ -482,7 +462,6 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
   auto bar_s = [&](int i) { return bar_t + 8u * (uint32_t)i; };
   auto bar_p = [&](int i) { return bar_t + 8u * (uint32_t)(2 + i); };
   const uint32_t bar_o = bar_t + 32u;
-  auto bar_p_half = [&](int i) { return bar0 + 8u * (uint32_t)(4 * NS + 18 + 2 * tile + i); };
 
   if (warp == 0) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
@@ -499,7 +478,6 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
       mbar_init(bt + 32, 1);
     }
     for (int i = 0; i < 8; ++i) mbar_init(bar0 + 8u * (uint32_t)(4 * NS + 10 + i), 1);
-    for (int i = 0; i < 4; ++i) mbar_init(bar0 + 8u * (uint32_t)(4 * NS + 18 + i), kPfRows / 32);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     s_fail = 0;
   }
@@ -570,23 +548,14 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
         // softmax still works on S(j), keeps the checks off the path from weights to scores.
         ok = mbar_wait_likely(bar_v(j % NS), (uint32_t)(j / NS) & 1u);
         if (ok && j + 2 < nb) ok = mbar_wait_likely(bar_k((j + 2) % NS), (uint32_t)((j + 2) / NS) & 1u);
-        // O += P(j) V(j) in two halves of 32 tokens: the first runs while the softmax still works
-        // on the second half of its weights
-        const uint32_t vt = sV + (j % NS) * kPfSubTile;
-        ok = ok && mbar_wait<kPfPolls>(bar_p_half(s), (uint32_t)(j >> 1) & 1u);
+        ok = ok && mbar_wait<kPfPolls>(bar_p(s), (uint32_t)(j >> 1) & 1u);
         if (!ok) break;
         tc_fence_after();
+        const uint32_t vt = sV + (j % NS) * kPfSubTile;
 #pragma unroll
-        for (int k = 0; k < 2; ++k)                     // slice k = tokens 16k .. 16k + 15
+        for (int k = 0; k < 4; ++k)                     // O += P(j) V(j); slice k = tokens 16k .. 16k + 15
           umma_bf16_ts(tmem + 128, tmem + s * 64 + k * 8,
                        umma_desc(vt + k * 2048, kPfSubHalf, 1024), kIdescPV, (j > 0 || k > 0) ? 1u : 0u);
-        ok = mbar_wait<kPfPolls>(bar_p(s), (uint32_t)(j >> 1) & 1u);
-        if (!ok) break;
-        tc_fence_after();
-#pragma unroll
-        for (int k = 2; k < 4; ++k)
-          umma_bf16_ts(tmem + 128, tmem + s * 64 + k * 8,
-                       umma_desc(vt + k * 2048, kPfSubHalf, 1024), kIdescPV, 1u);
         umma_commit(bar_o);
         umma_commit(bar_vfree(j % NS));
         // P(j) V(j) done: the score buffer it read its weights from takes sub-block j + 2
@@ -607,22 +576,21 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
       if (__any_sync(0xffffffffu, gave_up)) { gave_up = true; break; }
       float sv[64];                                       // raw products; the scale is folded in below
       float bmax = -INFINITY;
-      {
-        uint32_t r0[32], r1[32];
-        tmem_ld64(t_s, r0, r1);
-        if (valid >= kPfSub) {                            // CTA-uniform: only the last sub-block masks
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        uint32_t r[32];
+        tmem_ld32(t_s + c * 32, r);
+        if (valid >= kPfSub) {                           // CTA-uniform: only the last sub-block masks
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
-            sv[i] = __uint_as_float(r0[i]);
-            sv[32 + i] = __uint_as_float(r1[i]);
-            bmax = fmaxf(bmax, fmaxf(sv[i], sv[32 + i]));
+            sv[c * 32 + i] = __uint_as_float(r[i]);
+            bmax = fmaxf(bmax, sv[c * 32 + i]);
           }
         } else {
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
-            sv[i] = i < valid ? __uint_as_float(r0[i]) : -INFINITY;
-            sv[32 + i] = 32 + i < valid ? __uint_as_float(r1[i]) : -INFINITY;
-            bmax = fmaxf(bmax, fmaxf(sv[i], sv[32 + i]));
+            sv[c * 32 + i] = c * 32 + i < valid ? __uint_as_float(r[i]) : -INFINITY;
+            bmax = fmaxf(bmax, sv[c * 32 + i]);
           }
         }
       }
@@ -639,20 +607,7 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
         for (int c = 0; c < D; c += 8) tmem_scale8(t_o + c, factor);
         if (need) { l_run *= factor; m_ref = m_new; }
       }
-      if (valid < kPfSub) {
-        // Last, partial sub-block: rows of the V tile past the valid length hold whatever the
-        // cache holds there; clear them so that a zero weight times Inf/NaN cannot reach O
-        // (both query tiles write the same zeros).
-        if (!mbar_wait<kPfPolls>(bar_v(j % NS), (uint32_t)(j / NS) & 1u)) gave_up = true;
-        if (row >= valid && row < kPfSub) {
-#pragma unroll
-          for (int c = 0; c < 16; ++c)
-            st_shared16(sV + (j % NS) * kPfSubTile + (c >> 3) * kPfSubHalf + row * 128 + ((c & 7) << 4), 0, 0, 0, 0);
-        }
-        proxy_fence();
-      }
-      // ---- weights 2^(s - m_ref) as bf16 pairs over the first half of the score columns, handed
-      //      over in two halves of 32 tokens --------------------------------------------------------
+      // ---- weights 2^(s - m_ref) as bf16 pairs over the first half of the score columns -----
       {
         uint32_t pk[32];
         float rowsum0 = 0.f, rowsum1 = 0.f;
@@ -664,22 +619,8 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
         float neg_m_turn = neg_m;                         // the exponentials must not be scheduled
         asm volatile("" : "+f"(neg_m_turn) :: "memory");  // ahead of the wait: they depend on this
 #pragma unroll
-        for (int i = 0; i < 32; i += 2) {
+        for (int i = 0; i < 64; i += 2) {
           const float p0 = fast_exp2(__fmaf_rn(sv[i], scale_log2e, neg_m_turn));     // -inf -> 0
-          const float p1 = fast_exp2(__fmaf_rn(sv[i + 1], scale_log2e, neg_m_turn));
-          rowsum0 += p0;
-          rowsum1 += p1;
-          pk[i >> 1] = pack_bf16(p0, p1);
-        }
-        tmem_st16(t_s, pk);
-        tmem_wait_st();
-        tc_fence_before();
-        __syncwarp();
-        if ((tid & 31) == 0) mbar_arrive(bar_p_half(s)); // tokens 0..31 of the warp's rows (and O) are in place
-        asm volatile("" : "+f"(neg_m_turn) :: "memory");  // the second half is computed after the hand-over
-#pragma unroll
-        for (int i = 32; i < 64; i += 2) {
-          const float p0 = fast_exp2(__fmaf_rn(sv[i], scale_log2e, neg_m_turn));
           const float p1 = fast_exp2(__fmaf_rn(sv[i + 1], scale_log2e, neg_m_turn));
           rowsum0 += p0;
           rowsum1 += p1;
@@ -690,9 +631,21 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
           __syncwarp();
           if ((tid & 31) == 0) mbar_arrive(bar_other_turn);
         }
-        tmem_st16(t_s + 16, pk + 16);
+        tmem_st32(t_s, pk);
         tmem_wait_st();
         l_run += rowsum0 + rowsum1;
+      }
+      if (valid < kPfSub) {
+        // Last, partial sub-block: rows of the V tile past the valid length hold whatever the
+        // cache holds there; clear them so that a zero weight times Inf/NaN cannot reach O
+        // (both query tiles write the same zeros).
+        if (!mbar_wait<kPfPolls>(bar_v(j % NS), (uint32_t)(j / NS) & 1u)) gave_up = true;
+        if (row >= valid && row < kPfSub) {
+#pragma unroll
+          for (int c = 0; c < 16; ++c)
+            st_shared16(sV + (j % NS) * kPfSubTile + (c >> 3) * kPfSubHalf + row * 128 + ((c & 7) << 4), 0, 0, 0, 0);
+        }
+        proxy_fence();
       }
       tc_fence_before();
       __syncwarp();                                       // the warp's 32 rows are in place:
