@@ -427,7 +427,7 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
   extern __shared__ unsigned char smem_raw[];
   // mbarriers: K landed [NS], V landed [NS], K tile free [NS], V tile free [NS], then per query
   // tile: scores ready [2], weights ready [2], output quiet [1]
-  __shared__ __align__(8) unsigned long long s_bar[4 * NS + 10 + 8];   // + turn of A [4], turn of B [4]
+  __shared__ __align__(8) unsigned long long s_bar[4 * NS + 10];
   __shared__ uint32_t s_tmem;
   __shared__ int s_fail;
 
@@ -488,7 +488,6 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
       mbar_init(bt + 16, kPfRows / 32); mbar_init(bt + 24, kPfRows / 32);   // one arrival per softmax warp
       mbar_init(bt + 32, 1);
     }
-    for (int i = 0; i < 8; ++i) mbar_init(bar0 + 8u * (uint32_t)(4 * NS + 10 + i), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     s_fail = 0;
   }
@@ -511,12 +510,6 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
   const uint32_t t_lane = tmem + ((uint32_t)(wq * 32) << 16);
   const uint32_t t_o = t_lane + 128;                    // this row's 128 output dims
   const bool tile_active = tile < n_tiles;
-  // The two softmax warps of a scheduler (same lane quarter, one per query tile) take turns in the
-  // exponential phase, A(0) B(0) A(1) B(1) ..., so that one has the MUFU unit to itself while
-  // the other waits for scores, loads them and takes maxima.
-  const uint32_t bar_my_turn = bar0 + 8u * (uint32_t)(4 * NS + 10 + 4 * tile + wq);
-  const uint32_t bar_other_turn = bar0 + 8u * (uint32_t)(4 * NS + 10 + 4 * (tile ^ 1) + wq);
-  const bool take_turns = n_tiles == 2;
 
   if (!softmax_thread) {
     if ((tid & 31) == 0 && warp >= 10) {
@@ -624,24 +617,13 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
         uint32_t pk[32];
         float rowsum0 = 0.f, rowsum1 = 0.f;
         const float neg_m = -m_ref;
-        if (take_turns && (tile == 1 || j > 0)) {         // A(j) follows B(j-1); B(j) follows A(j)
-          const uint32_t par = (uint32_t)(tile == 1 ? j : j - 1) & 1u;
-          if (!mbar_wait_likely(bar_my_turn, par)) gave_up = true;
-        }
-        float neg_m_turn = neg_m;                         // the exponentials must not be scheduled
-        asm volatile("" : "+f"(neg_m_turn) :: "memory");  // ahead of the wait: they depend on this
 #pragma unroll
         for (int i = 0; i < 64; i += 2) {
-          const float p0 = fast_exp2(__fmaf_rn(sv[i], scale_log2e, neg_m_turn));     // -inf -> 0
-          const float p1 = fast_exp2(__fmaf_rn(sv[i + 1], scale_log2e, neg_m_turn));
+          const float p0 = fast_exp2(__fmaf_rn(sv[i], scale_log2e, neg_m));     // -inf -> 0
+          const float p1 = fast_exp2(__fmaf_rn(sv[i + 1], scale_log2e, neg_m));
           rowsum0 += p0;
           rowsum1 += p1;
           pk[i >> 1] = pack_bf16(p0, p1);
-        }
-        if (take_turns) {
-          asm volatile("" :: "f"(rowsum0), "f"(rowsum1) : "memory");   // ... and are over before the hand-over
-          __syncwarp();
-          if ((tid & 31) == 0) mbar_arrive(bar_other_turn);
         }
         tmem_st32(t_s, pk);
         tmem_wait_st();
