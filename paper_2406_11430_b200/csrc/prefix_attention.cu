@@ -693,9 +693,15 @@ static int launch_pf(const void* q, const void* K, const void* V, const Geom& g,
   alignas(64) CUtensorMap map_k, map_v;
   std::memset(&map_k, 0, sizeof map_k);
   std::memset(&map_v, 0, sizeof map_v);
-  // L2KV_PREFIX_KERNEL=basic selects the single-role kernel; the pipelined one is the default.
+  // The pipelined kernel works on pairs of query tiles; with an odd, small number of tiles per
+  // KV head (one tile: up to 128 / G queries) too many of its CTAs would run half empty, and the
+  // single-role kernel with two CTAs per SM is the faster one.  L2KV_PREFIX_KERNEL=basic /
+  // =pipelined overrides the choice.
   const char* which = std::getenv("L2KV_PREFIX_KERNEL");
-  const bool basic = which && std::strcmp(which, "basic") == 0;
+  const int n_q_tiles = (n_queries + QT - 1) / QT;
+  bool basic = (n_q_tiles & 1) && n_q_tiles < 9;
+  if (which && std::strcmp(which, "basic") == 0) basic = true;
+  if (which && std::strcmp(which, "pipelined") == 0) basic = false;
   const int sub_rows = basic ? kPfRows : kPfSub;
   if (!make_cache_map(&map_k, K, g, sub_rows) || !make_cache_map(&map_v, V, g, sub_rows))
     return L2KV_ERR_UNSUPPORTED;
