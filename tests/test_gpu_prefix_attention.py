@@ -32,7 +32,14 @@ def run(l2, q, K, V, cur, max_len, scale=0.0):
     return out.cpu().numpy(), lse.cpu().numpy()
 
 
-KERNELS = ["pipelined", "basic"]      # the two kernels; the pipelined one is the default
+KERNELS = ["pipelined", "basic", "auto"]      # the two kernels, and the library's own choice between them
+
+
+def choose(monkeypatch, kernel):
+    if kernel == "auto":
+        monkeypatch.delenv("L2KV_PREFIX_KERNEL", raising=False)
+    else:
+        choose(monkeypatch, kernel)
 
 
 @pytest.mark.parametrize("kernel", KERNELS)
@@ -40,7 +47,7 @@ KERNELS = ["pipelined", "basic"]      # the two kernels; the pipelined one is th
                                           (2, 4, 64, 128), (2, 8, 70, 200)])
 def test_prefix_attention_matches_oracle(Hkv, Hq, n_q, T, kernel, monkeypatch):
     import paper_2406_11430_b200 as l2
-    monkeypatch.setenv("L2KV_PREFIX_KERNEL", kernel)
+    choose(monkeypatch, kernel)
     w = synth.WORKLOADS[2].scaled(B=2, L=2, Hkv=Hkv, Hq=Hq, T=T)
     K, V = synth.make_cache(w, DEV)
     q = make_queries(w, n_q, 3)
@@ -63,7 +70,7 @@ def test_prefix_attention_matches_oracle(Hkv, Hq, n_q, T, kernel, monkeypatch):
 @pytest.mark.parametrize("kernel", KERNELS)
 def test_prefix_attention_agrees_with_decode_and_ignores_rows_past_the_length(kernel, monkeypatch):
     import paper_2406_11430_b200 as l2
-    monkeypatch.setenv("L2KV_PREFIX_KERNEL", kernel)
+    choose(monkeypatch, kernel)
     w = synth.WORKLOADS[2].scaled(B=1, L=2, T=700)
     K, V = synth.make_cache(w, DEV)
     q = make_queries(w, 5, 9)
@@ -86,7 +93,7 @@ def test_prefix_attention_with_drifting_maxima(kernel, direction, monkeypatch):
     more than the range one reference maximum can cover, so the accumulated output is rescaled
     several times (growing), or later weights underflow to zero (falling)."""
     import paper_2406_11430_b200 as l2
-    monkeypatch.setenv("L2KV_PREFIX_KERNEL", kernel)
+    choose(monkeypatch, kernel)
     T = 900
     w = synth.WORKLOADS[2].scaled(B=1, L=1, Hkv=2, Hq=4, T=T)
     K, V = synth.make_cache(w, DEV)
