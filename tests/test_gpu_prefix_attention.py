@@ -39,7 +39,7 @@ def choose(monkeypatch, kernel):
     if kernel == "auto":
         monkeypatch.delenv("L2KV_PREFIX_KERNEL", raising=False)
     else:
-        choose(monkeypatch, kernel)
+        monkeypatch.setenv("L2KV_PREFIX_KERNEL", kernel)
 
 
 @pytest.mark.parametrize("kernel", KERNELS)
