@@ -213,7 +213,14 @@ int l2kv_append_evict(void* K_c, void* V_c, int32_t* idx, float* sumsq_c, const 
  * (L2KV_ERR_UNSUPPORTED otherwise, also for strides a tensor map cannot express).  Products
  * are exact, sums fp32; the softmax weights are rounded to bf16 before they multiply V, as
  * in FlashAttention.  An empty cache gives zeros and lse = -inf.  workspace may be NULL; if
- * given (>= 256 bytes, zeroed) its status word reports a copy or MMA wait that gave up. */
+ * given (>= 256 bytes, its first 256 zeroed) its status word reports a copy or MMA wait that
+ * gave up.  With a workspace of l2kv_prefix_attention_workspace_bytes(lay, max_len, n_queries)
+ * bytes the call may also split the cache into chunks handled by different thread blocks and
+ * merge their results (exact up to fp32 rounding): that keeps the GPU busy when there are few
+ * KV heads and queries per call (one layer at a time) or when lengths differ widely between
+ * (b, l) pairs.  With less room it runs unsplit. */
+int l2kv_prefix_attention_workspace_bytes(const l2kv_layout* lay, int32_t max_len,
+                                          int32_t n_queries, size_t* bytes);
 int l2kv_prefix_attention(const void* q, const void* K_c, const void* V_c, const l2kv_layout* lay,
                           const int32_t* cur_len_dev, int32_t max_len, int32_t n_queries, float scale,
                           float* out, float* lse_out, void* workspace, size_t workspace_bytes,

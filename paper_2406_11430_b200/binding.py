@@ -64,12 +64,13 @@ def lib():
         L.l2kv_prefix_attention.argtypes = [vp, vp, vp, lay, vp, i32, i32, ctypes.c_float, vp, vp,
                                             vp, sz, vp]
         L.l2kv_prefix_attention_per_head.argtypes = L.l2kv_prefix_attention.argtypes
+        L.l2kv_prefix_attention_workspace_bytes.argtypes = [lay, i32, i32, ctypes.POINTER(sz)]
         for name in ("l2kv_prefix_attention", "l2kv_attention_loss_workspace_bytes", "l2kv_attention_loss",
                      "l2kv_keep_count", "l2kv_workspace_bytes", "l2kv_read_device_status",
                      "l2kv_key_norms", "l2kv_select_compact", "l2kv_decode_attention",
                      "l2kv_append_evict", "l2kv_select_compact_per_head",
                      "l2kv_decode_attention_per_head", "l2kv_append_evict_per_head",
-                     "l2kv_prefix_attention_per_head"):
+                     "l2kv_prefix_attention_per_head", "l2kv_prefix_attention_workspace_bytes"):
             getattr(L, name).restype = ctypes.c_int
         _LIB = L
     return _LIB
@@ -243,6 +244,16 @@ def attention_loss(q, K, cur_len_dev, max_len, sumsq, alr_out, loss_out=None, lo
         _ptr(q), _ptr(K), lay.ref(), _ptr(cur_len_dev), int(max_len), float(scale), _ptr(sumsq),
         _ptr(alr_out), _ptr(loss_out), _ptr(loss_ref_out), _ptr(workspace), workspace.numel(),
         _stream(stream)), "l2kv_attention_loss")
+
+
+def prefix_attention_workspace(K_c, q, max_len, device=None):
+    """A zeroed workspace large enough for prefix_attention to split the cache into chunks."""
+    lay = Layout(K_c, q_heads=q.shape[3])
+    need = ctypes.c_size_t(0)
+    _check(lib().l2kv_prefix_attention_workspace_bytes(lay.ref(), int(max_len), int(q.shape[2]),
+                                                       ctypes.byref(need)),
+           "l2kv_prefix_attention_workspace_bytes")
+    return torch.zeros(need.value, dtype=torch.uint8, device=device or K_c.device)
 
 
 def prefix_attention(q, K_c, V_c, cur_len_dev, max_len, out, lse_out=None, scale=0.0, workspace=None,

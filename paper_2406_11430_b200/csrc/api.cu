@@ -283,9 +283,31 @@ static int prefix_attention_impl(bool per_head, const void* q, const void* K_c, 
   if (workspace && workspace_bytes < (size_t)kStatusBytes) return L2KV_ERR_WORKSPACE_TOO_SMALL;
   const float sc = scale > 0.f ? scale : 1.0f / std::sqrt((float)lay->head_dim);
   const LenView lens{cur_len_dev, per_head ? 1 : 0};
+  // beyond its status block the workspace is scratch for the per-chunk results of a split launch
+  float* scratch = nullptr;
+  size_t scratch_bytes = 0;
+  if (workspace && workspace_bytes > (size_t)kStatusBytes) {
+    scratch = reinterpret_cast<float*>(static_cast<char*>(workspace) + kStatusBytes);
+    scratch_bytes = workspace_bytes - kStatusBytes;
+  }
   return launch_prefix_attention(q, K_c, V_c, make_geom(*lay), lay->dtype, n_queries, lens,
                                  max_len, sc, out, lse_out, static_cast<int32_t*>(workspace),
-                                 static_cast<cudaStream_t>(stream));
+                                 scratch, scratch_bytes, static_cast<cudaStream_t>(stream));
+}
+
+int l2kv_prefix_attention_workspace_bytes(const l2kv_layout* lay, int32_t max_len,
+                                          int32_t n_queries, size_t* bytes) {
+  if (!bytes) return L2KV_ERR_INVALID_ARG;
+  int rc = check_layout(lay);
+  if (rc != L2KV_OK) return rc;
+  rc = check_groups(lay);
+  if (rc != L2KV_OK) return rc;
+  if (max_len < 0 || n_queries < 0) return L2KV_ERR_INVALID_ARG;
+  if (max_len > lay->t_cap) return L2KV_ERR_OUT_OF_RANGE;
+  *bytes = (size_t)kStatusBytes;
+  if (empty(lay) || n_queries == 0 || lay->dtype != L2KV_BF16 || lay->head_dim != 128) return L2KV_OK;
+  *bytes += prefix_attention_scratch(make_geom(*lay), n_queries, max_len);
+  return L2KV_OK;
 }
 
 int l2kv_prefix_attention(const void* q, const void* K_c, const void* V_c, const l2kv_layout* lay,

@@ -152,7 +152,7 @@ prefix_attention_basic_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n
                            float* __restrict__ out, float* __restrict__ lse_out,
                            const __grid_constant__ CUtensorMap map_k,
                            const __grid_constant__ CUtensorMap map_v,
-                           int32_t* __restrict__ status_word) {
+                           int32_t* __restrict__ status_word, int split_len, long long rows_total) {
   constexpr int D = 128;
   constexpr int QT = kPfRows / G;                       // queries per CTA
   extern __shared__ unsigned char smem_raw[];
@@ -167,7 +167,16 @@ prefix_attention_basic_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n
   const int h = (int)(unit % g.H);
   const long long bl = unit / g.H;
   const int l = (int)(bl % g.L), b = (int)(bl / g.L);
-  const int n = max(0, min(cur_len_dev.at(bl, h, g.H), min(max_len, g.t_cap)));
+  const int n_all = max(0, min(cur_len_dev.at(bl, h, g.H), min(max_len, g.t_cap)));
+  // blockIdx.y: the chunk of split_len cached tokens this CTA covers (one chunk = the whole cache
+  // unless the launcher split it; then out / lse_out are the per-chunk partial results)
+  const int t_base = (int)blockIdx.y * split_len;
+  const int n = gridDim.y > 1 ? min(n_all, t_base + split_len) - t_base : n_all;
+  if (gridDim.y > 1) {
+    if (n <= 0) return;                                 // nothing cached in this chunk
+    out += (long long)blockIdx.y * rows_total * 128;
+    lse_out += (long long)blockIdx.y * rows_total;
+  }
   // Two threads per query row: thread (row, hf) owns score columns and output dims
   // [64 hf, 64 hf + 64).  Warps w and w + 4 share a tensor-memory lane quarter.
   const int tid = threadIdx.x, warp = tid >> 5;
@@ -223,13 +232,13 @@ prefix_attention_basic_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n
 
   auto load_k = [&](int kb) {                           // thread 0 only
     mbar_expect_tx(bar_k, kPfTileBytes);
-    tma_load_5d(sK, &map_k, bar_k, 0, kb * kPfRows, h, l, b);
-    tma_load_5d(sK + kPfHalf, &map_k, bar_k, 64, kb * kPfRows, h, l, b);
+    tma_load_5d(sK, &map_k, bar_k, 0, t_base + kb * kPfRows, h, l, b);
+    tma_load_5d(sK + kPfHalf, &map_k, bar_k, 64, t_base + kb * kPfRows, h, l, b);
   };
   auto load_v = [&](int kb) {
     mbar_expect_tx(bar_v, kPfTileBytes);
-    tma_load_5d(sV, &map_v, bar_v, 0, kb * kPfRows, h, l, b);
-    tma_load_5d(sV + kPfHalf, &map_v, bar_v, 64, kb * kPfRows, h, l, b);
+    tma_load_5d(sV, &map_v, bar_v, 0, t_base + kb * kPfRows, h, l, b);
+    tma_load_5d(sV + kPfHalf, &map_v, bar_v, 64, t_base + kb * kPfRows, h, l, b);
   };
   if (tid == 0) { load_k(0); load_v(0); }
   __syncwarp();
@@ -420,7 +429,7 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
                            float* __restrict__ out, float* __restrict__ lse_out,
                            const __grid_constant__ CUtensorMap map_k,
                            const __grid_constant__ CUtensorMap map_v,
-                           int32_t* __restrict__ status_word) {
+                           int32_t* __restrict__ status_word, int split_len, long long rows_total) {
   constexpr int D = 128;
   constexpr int QT = kPfRows / G;                       // queries per query tile
   constexpr int NS = kPfStages;
@@ -438,7 +447,16 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
   const int h = (int)(unit % g.H);
   const long long bl = unit / g.H;
   const int l = (int)(bl % g.L), b = (int)(bl / g.L);
-  const int n = max(0, min(cur_len_dev.at(bl, h, g.H), min(max_len, g.t_cap)));
+  const int n_all = max(0, min(cur_len_dev.at(bl, h, g.H), min(max_len, g.t_cap)));
+  // blockIdx.y: the chunk of split_len cached tokens this CTA covers (one chunk = the whole cache
+  // unless the launcher split it; then out / lse_out are the per-chunk partial results)
+  const int t_base = (int)blockIdx.y * split_len;
+  const int n = gridDim.y > 1 ? min(n_all, t_base + split_len) - t_base : n_all;
+  if (gridDim.y > 1) {
+    if (n <= 0) return;                                 // nothing cached in this chunk
+    out += (long long)blockIdx.y * rows_total * 128;
+    lse_out += (long long)blockIdx.y * rows_total;
+  }
   const int tid = threadIdx.x, warp = tid >> 5;
   const bool softmax_thread = tid < 2 * kPfRows;
   const int n_tiles = (2 * qp + 1 < q_tiles) ? 2 : 1;   // query tiles of this CTA that exist
@@ -524,8 +542,8 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
         if (!ok) break;
         const uint32_t dst = (is_k ? sK : sV) + st * kPfSubTile;
         mbar_expect_tx(full, kPfSubTile);
-        tma_load_5d(dst, map, full, 0, j * kPfSub, h, l, b);
-        tma_load_5d(dst + kPfSubHalf, map, full, 64, j * kPfSub, h, l, b);
+        tma_load_5d(dst, map, full, 0, t_base + j * kPfSub, h, l, b);
+        tma_load_5d(dst + kPfSubHalf, map, full, 64, t_base + j * kPfSub, h, l, b);
       }
       if (!ok) s_fail = 1;
     } else if ((tid & 31) == 0 && tile_active) {
@@ -681,62 +699,143 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
                  : "memory");
 }
 
+// Merge of the per-chunk results of a split launch: out = sum_c w_c O_c / sum_c w_c with
+// w_c = exp(lse_c - max lse), lse = max + log(sum_c w_c), over the chunks that hold cached rows.
+__global__ void __launch_bounds__(128)
+prefix_merge_kernel(const float* __restrict__ part_out, const float* __restrict__ part_lse,
+                    LenView cur_len_dev, int max_len, int t_cap, int H, int Hq, int n_queries,
+                    int split_len, long long rows_total, float* __restrict__ out,
+                    float* __restrict__ lse_out) {
+  const long long row = blockIdx.x;                      // ((b * L + l) * n_queries + s) * Hq + head
+  const long long bl = row / ((long long)n_queries * Hq);
+  const int h = (int)(row % Hq) / (Hq / H);
+  const int n = max(0, min(cur_len_dev.at(bl, h, H), min(max_len, t_cap)));
+  const int nc = (n + split_len - 1) / split_len;        // chunks with cached rows
+  const int d = threadIdx.x;
+  float m = -INFINITY;
+  for (int c = 0; c < nc; ++c) m = fmaxf(m, part_lse[c * rows_total + row]);
+  float den = 0.f, num = 0.f;
+  for (int c = 0; c < nc; ++c) {
+    const float w = __expf(part_lse[c * rows_total + row] - m);
+    den += w;
+    num = fmaf(w, part_out[(c * rows_total + row) * 128 + d], num);
+  }
+  out[row * 128 + d] = nc > 0 ? num / den : 0.f;
+  if (lse_out && d == 0) lse_out[row] = nc > 0 ? m + logf(den) : -INFINITY;
+}
+
+// How a launch is laid out.  Kernel: the pipelined one works on pairs of query tiles; with an odd,
+// small number of tiles per KV head (one tile: up to 128 / G queries) too many of its CTAs would
+// run half empty, and the single-role kernel with two CTAs per SM is the faster one
+// (L2KV_PREFIX_KERNEL=basic / =pipelined overrides the choice).  Chunks: the cache is split over
+// blockIdx.y, with a merge pass after, when the unsplit grid would leave SMs idle (few KV heads
+// and query tiles, as in a call for one layer) or when the cache is so long that (b, l) pairs of
+// different lengths would leave a few CTAs running alone; chunks are multiples of 128 tokens
+// and at least 4096 long.
+struct PrefixPlan {
+  bool basic;
+  long long ctas;          // per chunk
+  int chunks, split_len;
+  long long rows;          // B * L * n_queries * Hq
+  size_t scratch_bytes;    // partial results of a split launch (0 when chunks == 1)
+};
+static PrefixPlan plan_prefix(const Geom& g, int n_queries, int max_len) {
+  PrefixPlan p;
+  const int G = g.Hq / g.H;
+  const int QT = kPfRows / G;
+  const int q_tiles = (n_queries + QT - 1) / QT;
+  const char* which = std::getenv("L2KV_PREFIX_KERNEL");
+  p.basic = (q_tiles & 1) && q_tiles < 9;
+  if (which && std::strcmp(which, "basic") == 0) p.basic = true;
+  if (which && std::strcmp(which, "pipelined") == 0) p.basic = false;
+  const long long units = (long long)g.B * g.L * g.H;
+  p.ctas = units * (p.basic ? q_tiles : (q_tiles + 1) / 2);
+  p.rows = (long long)g.B * g.L * n_queries * g.Hq;
+  const long long slots = 148LL * (p.basic ? 2 : 1);     // CTAs the GPU holds at once
+  long long want = p.ctas > 0 ? (2 * slots + p.ctas - 1) / p.ctas : 1;   // two waves
+  if (max_len >= 65536) want = want > (max_len + 16383) / 16384 ? want : (max_len + 16383) / 16384;
+  const long long by_len = max_len / 4096 > 1 ? max_len / 4096 : 1;
+  long long chunks = want < by_len ? want : by_len;
+  if (chunks > 64) chunks = 64;
+  if (chunks < 1) chunks = 1;
+  p.split_len = (int)round_up_ll((max_len + chunks - 1) / chunks, 128);
+  if (p.split_len < 128) p.split_len = 128;
+  p.chunks = max_len > 0 ? (max_len + p.split_len - 1) / p.split_len : 1;
+  p.scratch_bytes = p.chunks > 1 ? (size_t)p.chunks * p.rows * 129 * sizeof(float) : 0;
+  return p;
+}
+
+size_t prefix_attention_scratch(const Geom& g, int n_queries, int max_len) {
+  return plan_prefix(g, n_queries, max_len).scratch_bytes;
+}
+
 template <int G>
 static int launch_pf(const void* q, const void* K, const void* V, const Geom& g, int n_queries,
                      const LenView& cur_len_dev, int max_len, float scale, float* out,
-                     float* lse_out, int32_t* status_word, cudaStream_t s) {
-  constexpr int QT = kPfRows / G;
-  const long long units = (long long)g.B * g.L * g.H;
-  const long long blocks = units * ((n_queries + QT - 1) / QT);
-  if (blocks == 0) return L2KV_OK;
-  if (blocks > 0x7fffffffLL) return L2KV_ERR_OUT_OF_RANGE;
+                     float* lse_out, int32_t* status_word, float* scratch, size_t scratch_bytes,
+                     cudaStream_t s) {
+  PrefixPlan p = plan_prefix(g, n_queries, max_len);
+  if (p.ctas == 0) return L2KV_OK;
+  if (p.chunks > 1 && (!scratch || scratch_bytes < p.scratch_bytes)) {   // no room: one chunk
+    p.chunks = 1;
+    p.split_len = max_len > 128 ? (int)round_up_ll(max_len, 128) : 128;
+  }
+  if (p.ctas > 0x7fffffffLL) return L2KV_ERR_OUT_OF_RANGE;
   alignas(64) CUtensorMap map_k, map_v;
   std::memset(&map_k, 0, sizeof map_k);
   std::memset(&map_v, 0, sizeof map_v);
-  // The pipelined kernel works on pairs of query tiles; with an odd, small number of tiles per
-  // KV head (one tile: up to 128 / G queries) too many of its CTAs would run half empty, and the
-  // single-role kernel with two CTAs per SM is the faster one.  L2KV_PREFIX_KERNEL=basic /
-  // =pipelined overrides the choice.
-  const char* which = std::getenv("L2KV_PREFIX_KERNEL");
-  const int n_q_tiles = (n_queries + QT - 1) / QT;
-  bool basic = (n_q_tiles & 1) && n_q_tiles < 9;
-  if (which && std::strcmp(which, "basic") == 0) basic = true;
-  if (which && std::strcmp(which, "pipelined") == 0) basic = false;
-  const int sub_rows = basic ? kPfRows : kPfSub;
+  const int sub_rows = p.basic ? kPfRows : kPfSub;
   if (!make_cache_map(&map_k, K, g, sub_rows) || !make_cache_map(&map_v, V, g, sub_rows))
     return L2KV_ERR_UNSUPPORTED;
-  if (!basic) {
+  // A split launch writes per-chunk results (normalised rows, then their log-sum-exps) to the
+  // scratch; the merge pass below turns them into out / lse_out.
+  float* k_out = p.chunks > 1 ? scratch : out;
+  float* k_lse = p.chunks > 1 ? scratch + (size_t)p.chunks * p.rows * 128 : lse_out;
+  const dim3 grid((unsigned)p.ctas, (unsigned)p.chunks);
+  const __nv_bfloat16* qb = static_cast<const __nv_bfloat16*>(q);
+  if (!p.basic) {
     constexpr int smem_pipe = 1024 + 2 * kPfTileBytes + 2 * kPfStages * kPfSubTile;
-    const int q_tiles = (n_queries + QT - 1) / QT;
-    const long long blocks_pipe = units * ((q_tiles + 1) / 2);
     auto kern_pipe = prefix_attention_pipelined_kernel<G>;
     if (cudaFuncSetAttribute(kern_pipe, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_pipe) != cudaSuccess)
       return L2KV_ERR_CUDA;
-    kern_pipe<<<(unsigned)blocks_pipe, kPfPipeThreads, smem_pipe, s>>>(
-        static_cast<const __nv_bfloat16*>(q), g, n_queries, cur_len_dev, max_len, scale * kPfLog2e, out,
-        lse_out, map_k, map_v, status_word);
-    return cudaGetLastError() == cudaSuccess ? L2KV_OK : L2KV_ERR_CUDA;
+    kern_pipe<<<grid, kPfPipeThreads, smem_pipe, s>>>(qb, g, n_queries, cur_len_dev, max_len,
+                                                      scale * kPfLog2e, k_out, k_lse, map_k, map_v,
+                                                      status_word, p.split_len, p.rows);
+  } else {
+    constexpr int smem_bytes = 1024 + 3 * kPfTileBytes;
+    auto kern = prefix_attention_basic_kernel<G>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) != cudaSuccess)
+      return L2KV_ERR_CUDA;
+    kern<<<grid, kPfThreads, smem_bytes, s>>>(qb, g, n_queries, cur_len_dev, max_len, scale * kPfLog2e,
+                                              k_out, k_lse, map_k, map_v, status_word, p.split_len,
+                                              p.rows);
   }
-  constexpr int smem_bytes = 1024 + 3 * kPfTileBytes;
-  auto kern = prefix_attention_basic_kernel<G>;
-  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) != cudaSuccess)
-    return L2KV_ERR_CUDA;
-  kern<<<(unsigned)blocks, kPfThreads, smem_bytes, s>>>(
-      static_cast<const __nv_bfloat16*>(q), g, n_queries, cur_len_dev, max_len, scale * kPfLog2e, out,
-      lse_out, map_k, map_v, status_word);
-  return cudaGetLastError() == cudaSuccess ? L2KV_OK : L2KV_ERR_CUDA;
+  if (cudaGetLastError() != cudaSuccess) return L2KV_ERR_CUDA;
+  if (p.chunks > 1) {
+    if (p.rows > 0x7fffffffLL) return L2KV_ERR_OUT_OF_RANGE;
+    prefix_merge_kernel<<<(unsigned)p.rows, 128, 0, s>>>(k_out, k_lse, cur_len_dev, max_len, g.t_cap,
+                                                         g.H, g.Hq, n_queries, p.split_len, p.rows,
+                                                         out, lse_out);
+    if (cudaGetLastError() != cudaSuccess) return L2KV_ERR_CUDA;
+  }
+  return L2KV_OK;
 }
 
 int launch_prefix_attention(const void* q, const void* K, const void* V, const Geom& g, int dtype,
                             int n_queries, const LenView& cur_len_dev, int max_len, float scale,
-                            float* out, float* lse_out, int32_t* status_word, cudaStream_t s) {
+                            float* out, float* lse_out, int32_t* status_word, float* scratch,
+                            size_t scratch_bytes, cudaStream_t s) {
   if (dtype != L2KV_BF16 || g.D != 128) return L2KV_ERR_UNSUPPORTED;
+#define L2KV_PF(G)                                                                              \
+  return launch_pf<G>(q, K, V, g, n_queries, cur_len_dev, max_len, scale, out, lse_out,         \
+                      status_word, scratch, scratch_bytes, s)
   switch (g.Hq / g.H) {
-    case 1: return launch_pf<1>(q, K, V, g, n_queries, cur_len_dev, max_len, scale, out, lse_out, status_word, s);
-    case 2: return launch_pf<2>(q, K, V, g, n_queries, cur_len_dev, max_len, scale, out, lse_out, status_word, s);
-    case 4: return launch_pf<4>(q, K, V, g, n_queries, cur_len_dev, max_len, scale, out, lse_out, status_word, s);
-    case 8: return launch_pf<8>(q, K, V, g, n_queries, cur_len_dev, max_len, scale, out, lse_out, status_word, s);
+    case 1: L2KV_PF(1);
+    case 2: L2KV_PF(2);
+    case 4: L2KV_PF(4);
+    case 8: L2KV_PF(8);
   }
+#undef L2KV_PF
   return L2KV_ERR_UNSUPPORTED;
 }
 

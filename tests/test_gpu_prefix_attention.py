@@ -109,3 +109,37 @@ def test_prefix_attention_with_drifting_maxima(kernel, direction, monkeypatch):
         assert_attention_close(out[:, :, s], want, atol=4e-3)
     z = K[0, 0, 1].double().cpu().numpy() @ q[0, 0, 3, 2].double().cpu().numpy() / np.sqrt(w.D)
     np.testing.assert_allclose(lse[0, 0, 3, 2], scipy.special.logsumexp(z), rtol=1e-5, atol=1e-4)
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+@pytest.mark.parametrize("lens", [[9000, 4700], [4608, 0], [4609, 8999]])
+def test_prefix_attention_split_over_the_cache(kernel, lens, monkeypatch):
+    """Few KV heads and queries, long cache: with the workspace the library asks for, the cache
+    is split into chunks (here two of 4608 tokens) whose results are merged; lengths that end
+    inside the first chunk, at its edge, just past it and in the second one."""
+    import paper_2406_11430_b200 as l2
+    choose(monkeypatch, kernel)
+    T = 9000
+    w = synth.WORKLOADS[2].scaled(B=1, L=2, Hkv=2, Hq=8, T=T)
+    K, V = synth.make_cache(w, DEV)
+    q = make_queries(w, 24, 11)
+    cur = np.array([lens], dtype=np.int32)
+    ws = l2.prefix_attention_workspace(K, q, T)
+    assert ws.numel() > 256                                   # room for a split was asked for
+    out = torch.full(q.shape, float("nan"), dtype=torch.float32, device=DEV)
+    lse = torch.full(q.shape[:4], float("nan"), dtype=torch.float32, device=DEV)
+    l2.prefix_attention(q, K, V, i32(cur), T, out, lse, workspace=ws)
+    torch.cuda.synchronize()
+    assert l2.read_device_status(ws) == 0
+    got, got_lse = out.cpu().numpy(), lse.cpu().numpy()
+    Kn, Vn = synth.to_numpy(K), synth.to_numpy(V)
+    for s in range(0, 24, 5):
+        want = oracle.attention(synth.to_numpy(q[:, :, s].contiguous()), Kn, Vn, "bf16", cur, nthreads=8)
+        assert_attention_close(got[:, :, s], want, atol=4e-3)
+    # the unsplit launch (no room for partial results) gives the same rows up to fp32 rounding
+    out1, lse1 = run(l2, q, K, V, cur, T)
+    np.testing.assert_allclose(got, out1, rtol=1e-4, atol=2e-5)
+    np.testing.assert_allclose(got_lse, lse1, rtol=1e-5, atol=1e-5)
+    for l in range(2):
+        if lens[l] == 0:
+            assert not got[0, l].any() and np.all(np.isneginf(got_lse[0, l]))
