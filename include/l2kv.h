@@ -216,7 +216,7 @@ int l2kv_append_evict(void* K_c, void* V_c, int32_t* idx, float* sumsq_c, const 
  * given (>= 256 bytes, its first 256 zeroed) its status word reports a copy or MMA wait that
  * gave up.  With a workspace of l2kv_prefix_attention_workspace_bytes(lay, max_len, n_queries)
  * bytes the call may also split the cache into chunks handled by different thread blocks and
- * merge their results (exact up to fp32 rounding): that keeps the GPU busy when there are few
+ * merge their results (the same rows up to the bf16 rounding of the weights): that keeps the GPU busy when there are few
  * KV heads and queries per call (one layer at a time) or when lengths differ widely between
  * (b, l) pairs.  With less room it runs unsplit. */
 int l2kv_prefix_attention_workspace_bytes(const l2kv_layout* lay, int32_t max_len,

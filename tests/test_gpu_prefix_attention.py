@@ -136,9 +136,10 @@ def test_prefix_attention_split_over_the_cache(kernel, lens, monkeypatch):
     for s in range(0, 24, 5):
         want = oracle.attention(synth.to_numpy(q[:, :, s].contiguous()), Kn, Vn, "bf16", cur, nthreads=8)
         assert_attention_close(got[:, :, s], want, atol=4e-3)
-    # the unsplit launch (no room for partial results) gives the same rows up to fp32 rounding
+    # the unsplit launch (no room for partial results): same rows up to the bf16 rounding of the
+    # weights, which are taken against per-chunk maxima in the split launch; same log-sum-exps
     out1, lse1 = run(l2, q, K, V, cur, T)
-    np.testing.assert_allclose(got, out1, rtol=1e-4, atol=2e-5)
+    np.testing.assert_allclose(got, out1, rtol=1e-2, atol=2e-3)
     np.testing.assert_allclose(got_lse, lse1, rtol=1e-5, atol=1e-5)
     for l in range(2):
         if lens[l] == 0:
