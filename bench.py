@@ -354,23 +354,39 @@ def time_variants(job, w, cbytes, reps=5):
         job.compress()
         qp = torch.randn((w.B, w.L, n_q, w.Hq, w.D), device=job.dev).to(torch.bfloat16)
         op = torch.empty(qp.shape, dtype=torch.float32, device=job.dev)
-        job.l2.prefix_attention(qp, job.K_c, job.V_c, job.cur, job.t_cap, op)
-        t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
-        t0.record()
-        for _ in range(3):
-            job.l2.prefix_attention(qp, job.K_c, job.V_c, job.cur, job.t_cap, op)
-        t1.record(); torch.cuda.synchronize()
-        ms = t0.elapsed_time(t1) / 3
-        flop = 4.0 * n_q * w.Hq * w.D * float(job.cur.sum().item())
         tf_peak = None
         try:
             tf_peak = float(json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))["bf16_tflops_sustained"])
         except Exception:
             pass
-        out["prefix_attention"] = {"ms": round(ms, 3), "queries_per_sequence": n_q,
-                                   "TFLOPs": round(flop / ms / 1e9, 1), "bound": "tensor",
-                                   "peak_TFLOPs_measured_sustained": tf_peak,
-                                   "frac": round(flop / ms / 1e9 / tf_peak, 4) if tf_peak else None}
+
+        def timed(q_, K_, V_, cur_, o_, reps=3, split=True):
+            ws_ = (job.l2.prefix_attention_workspace(K_, q_, job.t_cap) if split  # room to split the cache
+                   else torch.zeros(256, dtype=torch.uint8, device=job.dev))
+            job.l2.prefix_attention(q_, K_, V_, cur_, job.t_cap, o_, workspace=ws_)
+            t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+            t0.record()
+            for _ in range(reps):
+                job.l2.prefix_attention(q_, K_, V_, cur_, job.t_cap, o_, workspace=ws_)
+            t1.record(); torch.cuda.synchronize()
+            ms_ = t0.elapsed_time(t1) / reps
+            flop_ = 4.0 * n_q * w.Hq * w.D * float(cur_.sum().item())
+            return {"ms": round(ms_, 3), "TFLOPs": round(flop_ / ms_ / 1e9, 1),
+                    "frac": round(flop_ / ms_ / 1e9 / tf_peak, 4) if tf_peak else None,
+                    "split_scratch_MiB": round((ws_.numel() - 256) / 2**20, 1)}
+
+        r = timed(qp, job.K_c, job.V_c, job.cur, op)
+        out["prefix_attention"] = {"ms": r["ms"], "queries_per_sequence": n_q, "TFLOPs": r["TFLOPs"],
+                                   "bound": "tensor", "peak_TFLOPs_measured_sustained": tf_peak,
+                                   "frac": r["frac"], "split_scratch_MiB": r["split_scratch_MiB"]}
+        # the same for one layer at a time, as a model calls it: few CTAs unless the cache is split
+        l1 = min(2, w.L - 1)
+        r1 = timed(qp[:, l1:l1 + 1].contiguous(), job.K_c[:, l1:l1 + 1], job.V_c[:, l1:l1 + 1],
+                   job.cur[:, l1:l1 + 1].contiguous(), op[:, l1:l1 + 1].contiguous(), reps=10)
+        out["prefix_attention"]["one_layer"] = r1
+        out["prefix_attention"]["one_layer_unsplit"] = timed(
+            qp[:, l1:l1 + 1].contiguous(), job.K_c[:, l1:l1 + 1], job.V_c[:, l1:l1 + 1],
+            job.cur[:, l1:l1 + 1].contiguous(), op[:, l1:l1 + 1].contiguous(), reps=10, split=False)
         del qp, op
     job.compress()
     torch.cuda.synchronize()
