@@ -731,7 +731,7 @@ prefix_merge_kernel(const float* __restrict__ part_out, const float* __restrict_
 // blockIdx.y, with a merge pass after, when the unsplit grid would leave SMs idle (few KV heads
 // and query tiles, as in a call for one layer) or when the cache is so long that (b, l) pairs of
 // different lengths would leave a few CTAs running alone; chunks are multiples of 128 tokens
-// and at least 4096 long.
+// and at least 1024 long.
 struct PrefixPlan {
   bool basic;
   long long ctas;          // per chunk
@@ -754,7 +754,7 @@ static PrefixPlan plan_prefix(const Geom& g, int n_queries, int max_len) {
   const long long slots = 148LL * (p.basic ? 2 : 1);     // CTAs the GPU holds at once
   long long want = p.ctas > 0 ? (2 * slots + p.ctas - 1) / p.ctas : 1;   // two waves
   if (max_len >= 65536) want = want > (max_len + 16383) / 16384 ? want : (max_len + 16383) / 16384;
-  const long long by_len = max_len / 4096 > 1 ? max_len / 4096 : 1;
+  const long long by_len = max_len / 1024 > 1 ? max_len / 1024 : 1;
   long long chunks = want < by_len ? want : by_len;
   if (chunks > 64) chunks = 64;
   if (chunks < 1) chunks = 1;

@@ -115,8 +115,8 @@ def test_prefix_attention_with_drifting_maxima(kernel, direction, monkeypatch):
 @pytest.mark.parametrize("lens", [[9000, 4700], [4608, 0], [4609, 8999]])
 def test_prefix_attention_split_over_the_cache(kernel, lens, monkeypatch):
     """Few KV heads and queries, long cache: with the workspace the library asks for, the cache
-    is split into chunks (here two of 4608 tokens) whose results are merged; lengths that end
-    inside the first chunk, at its edge, just past it and in the second one."""
+    is split into chunks (multiples of 128 tokens) whose results are merged; lengths that end
+    inside a chunk, at a chunk's edge, just past it, and an empty cache."""
     import paper_2406_11430_b200 as l2
     choose(monkeypatch, kernel)
     T = 9000
