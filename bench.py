@@ -361,13 +361,14 @@ def time_variants(job, w, cbytes, reps=5):
             pass
 
         def timed(q_, K_, V_, cur_, o_, reps=3, split=True):
-            ws_ = (job.l2.prefix_attention_workspace(K_, q_, job.t_cap) if split  # room to split the cache
+            max_len_ = int(cur_.max().item())               # the caller knows its longest cache
+            ws_ = (job.l2.prefix_attention_workspace(K_, q_, max_len_) if split  # room to split the cache
                    else torch.zeros(256, dtype=torch.uint8, device=job.dev))
-            job.l2.prefix_attention(q_, K_, V_, cur_, job.t_cap, o_, workspace=ws_)
+            job.l2.prefix_attention(q_, K_, V_, cur_, max_len_, o_, workspace=ws_)
             t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
             t0.record()
             for _ in range(reps):
-                job.l2.prefix_attention(q_, K_, V_, cur_, job.t_cap, o_, workspace=ws_)
+                job.l2.prefix_attention(q_, K_, V_, cur_, max_len_, o_, workspace=ws_)
             t1.record(); torch.cuda.synchronize()
             ms_ = t0.elapsed_time(t1) / reps
             flop_ = 4.0 * n_q * w.Hq * w.D * float(cur_.sum().item())
