@@ -192,3 +192,27 @@ def test_prefix_attention_with_a_length_per_head(l2, kernel, monkeypatch):
         want = oracle.attention(synth.to_numpy(q[:, :, s].contiguous()), Kn, Vn, "bf16", cur, nthreads=8)
         assert_attention_close(got[:, :, s], want, atol=4e-3)
     assert not got[0, 1, :, :4].any() and np.all(np.isneginf(lse[0, 1, :, :4].cpu().numpy()))
+
+
+def test_prefix_attention_per_head_split_over_the_cache(l2):
+    """Per-head lengths with the cache split into chunks: each head merges only the chunks that
+    hold rows of its own."""
+    T = 3100
+    w = synth.WORKLOADS[2].scaled(B=1, L=2, Hkv=2, Hq=8, T=T)
+    K, V = synth.make_cache(w, DEV)
+    g = torch.Generator().manual_seed(6)
+    q = torch.randn((1, 2, 20, 8, 128), generator=g).to(torch.bfloat16).to(DEV)
+    cur = np.array([[[3100, 900], [0, 1537]]], dtype=np.int32)
+    ws = l2.prefix_attention_workspace(K, q, T)
+    assert ws.numel() > 256
+    out = torch.full(q.shape, float("nan"), dtype=torch.float32, device=DEV)
+    lse = torch.full(q.shape[:4], float("nan"), dtype=torch.float32, device=DEV)
+    l2.prefix_attention_per_head(q, K, V, i32(cur), T, out, lse, workspace=ws)
+    torch.cuda.synchronize()
+    assert l2.read_device_status(ws) == 0
+    got = out.cpu().numpy()
+    Kn, Vn = synth.to_numpy(K), synth.to_numpy(V)
+    for s in range(0, 20, 3):
+        want = oracle.attention(synth.to_numpy(q[:, :, s].contiguous()), Kn, Vn, "bf16", cur, nthreads=8)
+        assert_attention_close(got[:, :, s], want, atol=4e-3)
+    assert not got[0, 1, :, :4].any() and np.all(np.isneginf(lse[0, 1, :, :4].cpu().numpy()))
