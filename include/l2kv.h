@@ -221,6 +221,17 @@ int l2kv_append_evict(void* K_c, void* V_c, int32_t* idx, float* sumsq_c, const 
  * (b, l) pairs.  With less room it runs unsplit. */
 int l2kv_prefix_attention_workspace_bytes(const l2kv_layout* lay, int32_t max_len,
                                           int32_t n_queries, size_t* bytes);
+/* The same for a prefill chunk whose own keys and values are already in the cache: the last
+ * n_queries cached rows of every (b, l) are the new tokens', in order, and query s attends to
+ * rows i < cur_len_dev[b,l] - n_queries + s + 1 (everything before the chunk, and the chunk up
+ * to itself) -- the causal mask of Eq. 2 as a model applies it during prefill.  Meant for
+ * caches whose tail is in position order (appended rows; not after an eviction has reused a
+ * slot).  A query with no row to see gives zeros and lse = -inf.  Everything else as above. */
+int l2kv_prefix_attention_causal(const void* q, const void* K_c, const void* V_c,
+                                 const l2kv_layout* lay, const int32_t* cur_len_dev,
+                                 int32_t max_len, int32_t n_queries, float scale, float* out,
+                                 float* lse_out, void* workspace, size_t workspace_bytes,
+                                 void* stream);
 int l2kv_prefix_attention(const void* q, const void* K_c, const void* V_c, const l2kv_layout* lay,
                           const int32_t* cur_len_dev, int32_t max_len, int32_t n_queries, float scale,
                           float* out, float* lse_out, void* workspace, size_t workspace_bytes,

@@ -64,13 +64,15 @@ def lib():
         L.l2kv_prefix_attention.argtypes = [vp, vp, vp, lay, vp, i32, i32, ctypes.c_float, vp, vp,
                                             vp, sz, vp]
         L.l2kv_prefix_attention_per_head.argtypes = L.l2kv_prefix_attention.argtypes
+        L.l2kv_prefix_attention_causal.argtypes = L.l2kv_prefix_attention.argtypes
         L.l2kv_prefix_attention_workspace_bytes.argtypes = [lay, i32, i32, ctypes.POINTER(sz)]
         for name in ("l2kv_prefix_attention", "l2kv_attention_loss_workspace_bytes", "l2kv_attention_loss",
                      "l2kv_keep_count", "l2kv_workspace_bytes", "l2kv_read_device_status",
                      "l2kv_key_norms", "l2kv_select_compact", "l2kv_decode_attention",
                      "l2kv_append_evict", "l2kv_select_compact_per_head",
                      "l2kv_decode_attention_per_head", "l2kv_append_evict_per_head",
-                     "l2kv_prefix_attention_per_head", "l2kv_prefix_attention_workspace_bytes"):
+                     "l2kv_prefix_attention_per_head", "l2kv_prefix_attention_workspace_bytes",
+                     "l2kv_prefix_attention_causal"):
             getattr(L, name).restype = ctypes.c_int
         _LIB = L
     return _LIB
@@ -264,6 +266,18 @@ def prefix_attention(q, K_c, V_c, cur_len_dev, max_len, out, lse_out=None, scale
         _ptr(q), _ptr(K_c), _ptr(V_c), lay.ref(), _ptr(cur_len_dev), int(max_len), int(q.shape[2]),
         float(scale), _ptr(out), _ptr(lse_out), _ptr(workspace),
         0 if workspace is None else workspace.numel(), _stream(stream)), "l2kv_prefix_attention")
+
+
+def prefix_attention_causal(q, K_c, V_c, cur_len_dev, max_len, out, lse_out=None, scale=0.0,
+                            workspace=None, stream=None):
+    """prefix_attention for a chunk whose own K/V are the last q.shape[2] cached rows: query s
+    sees the rows before the chunk and the chunk up to itself."""
+    lay = Layout(K_c, q_heads=q.shape[3])
+    _check(lib().l2kv_prefix_attention_causal(
+        _ptr(q), _ptr(K_c), _ptr(V_c), lay.ref(), _ptr(cur_len_dev), int(max_len), int(q.shape[2]),
+        float(scale), _ptr(out), _ptr(lse_out), _ptr(workspace),
+        0 if workspace is None else workspace.numel(), _stream(stream)),
+        "l2kv_prefix_attention_causal")
 
 
 def prefix_attention_per_head(q, K_c, V_c, cur_len_unit_dev, max_len, out, lse_out=None, scale=0.0,

@@ -264,7 +264,7 @@ int l2kv_append_evict_per_head(void* K_c, void* V_c, int32_t* idx, float* sumsq_
                            workspace, workspace_bytes, stream);
 }
 
-static int prefix_attention_impl(bool per_head, const void* q, const void* K_c, const void* V_c,
+static int prefix_attention_impl(bool per_head, bool causal, const void* q, const void* K_c, const void* V_c,
                                  const l2kv_layout* lay, const int32_t* cur_len_dev,
                                  int32_t max_len, int32_t n_queries, float scale, float* out,
                                  float* lse_out, void* workspace, size_t workspace_bytes,
@@ -292,7 +292,17 @@ static int prefix_attention_impl(bool per_head, const void* q, const void* K_c, 
   }
   return launch_prefix_attention(q, K_c, V_c, make_geom(*lay), lay->dtype, n_queries, lens,
                                  max_len, sc, out, lse_out, static_cast<int32_t*>(workspace),
-                                 scratch, scratch_bytes, static_cast<cudaStream_t>(stream));
+                                 scratch, scratch_bytes, causal ? 1 : 0,
+                                 static_cast<cudaStream_t>(stream));
+}
+
+int l2kv_prefix_attention_causal(const void* q, const void* K_c, const void* V_c,
+                                 const l2kv_layout* lay, const int32_t* cur_len_dev,
+                                 int32_t max_len, int32_t n_queries, float scale, float* out,
+                                 float* lse_out, void* workspace, size_t workspace_bytes,
+                                 void* stream) {
+  return prefix_attention_impl(false, true, q, K_c, V_c, lay, cur_len_dev, max_len, n_queries, scale,
+                               out, lse_out, workspace, workspace_bytes, stream);
 }
 
 int l2kv_prefix_attention_workspace_bytes(const l2kv_layout* lay, int32_t max_len,
@@ -314,7 +324,7 @@ int l2kv_prefix_attention(const void* q, const void* K_c, const void* V_c, const
                           const int32_t* cur_len_dev, int32_t max_len, int32_t n_queries, float scale,
                           float* out, float* lse_out, void* workspace, size_t workspace_bytes,
                           void* stream) {
-  return prefix_attention_impl(false, q, K_c, V_c, lay, cur_len_dev, max_len, n_queries, scale, out,
+  return prefix_attention_impl(false, false, q, K_c, V_c, lay, cur_len_dev, max_len, n_queries, scale, out,
                                lse_out, workspace, workspace_bytes, stream);
 }
 
@@ -323,7 +333,7 @@ int l2kv_prefix_attention_per_head(const void* q, const void* K_c, const void* V
                                    int32_t max_len, int32_t n_queries, float scale, float* out,
                                    float* lse_out, void* workspace, size_t workspace_bytes,
                                    void* stream) {
-  return prefix_attention_impl(true, q, K_c, V_c, lay, cur_len_unit_dev, max_len, n_queries, scale,
+  return prefix_attention_impl(true, false, q, K_c, V_c, lay, cur_len_unit_dev, max_len, n_queries, scale,
                                out, lse_out, workspace, workspace_bytes, stream);
 }
 

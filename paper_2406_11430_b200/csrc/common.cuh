@@ -229,7 +229,7 @@ int launch_append_evict(void* K, void* V, int32_t* idx, float* sumsq, const Geom
 int launch_prefix_attention(const void* q, const void* K, const void* V, const Geom& g, int dtype,
                             int n_queries, const LenView& cur_len_dev, int max_len, float scale,
                             float* out, float* lse_out, int32_t* status_word, float* scratch,
-                            size_t scratch_bytes, cudaStream_t s);
+                            size_t scratch_bytes, int causal, cudaStream_t s);
 size_t prefix_attention_scratch(const Geom& g, int n_queries, int max_len);
 size_t attention_loss_workspace(const l2kv_layout& a, int max_len);
 int launch_attention_loss(const void* q, const void* K, const Geom& g, int dtype,

@@ -152,7 +152,7 @@ prefix_attention_basic_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n
                            float* __restrict__ out, float* __restrict__ lse_out,
                            const __grid_constant__ CUtensorMap map_k,
                            const __grid_constant__ CUtensorMap map_v,
-                           int32_t* __restrict__ status_word, int split_len, long long rows_total) {
+                           int32_t* __restrict__ status_word, int split_len, long long rows_total, int causal) {
   constexpr int D = 128;
   constexpr int QT = kPfRows / G;                       // queries per CTA
   extern __shared__ unsigned char smem_raw[];
@@ -185,6 +185,8 @@ prefix_attention_basic_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n
   const int head = h * G + row % G;
   const bool row_valid = s_idx < n_queries;
   const long long row_off = ((bl * n_queries + s_idx) * g.Hq + head);
+  // causal: the last n_queries cached rows are the new tokens' own; query s stops at its own
+  const int n_row = causal && row_valid ? min(n, max(0, n_all - n_queries + s_idx + 1) - t_base) : n;
   if (n == 0) {                                         // empty cache: zeros, log-sum-exp = -inf
     if (row_valid) {
       for (int d = 0; d < 64; ++d) out[row_off * D + hf * 64 + d] = 0.f;
@@ -247,7 +249,7 @@ prefix_attention_basic_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n
 
   for (int kb = 0; kb < n_blocks; ++kb) {
     const int valid_all = min(kPfRows, n - kb * kPfRows);   // valid tokens of this block
-    const int valid = valid_all - hf * 64;                   // ... among this thread's 64
+    const int valid = min(valid_all, n_row - kb * kPfRows) - hf * 64;   // ... among this thread's 64
     // ---- S = Q K^T; fetch V for this block and K for the next as their tiles come free ---
     if (tid == 0) {
       if (!mbar_wait<kPfPolls>(bar_k, kb & 1)) s_fail = 1;
@@ -276,7 +278,7 @@ prefix_attention_basic_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n
     for (int c = 0; c < 2; ++c) {
       uint32_t r[32];
       tmem_ld32(t_s + c * 32, r);
-      if (valid >= 64) {                                 // warp-uniform: only the last block masks
+      if (valid >= 64) {                                 // only the last (or a causal row's own) block masks
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
           sv[c * 32 + i] = __uint_as_float(r[i]);
@@ -309,7 +311,7 @@ prefix_attention_basic_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n
     {
       uint32_t pk[32];
       float rowsum0 = 0.f, rowsum1 = 0.f;
-      const float neg_m = -m_ref;
+      const float neg_m = m_ref == -INFINITY ? 0.f : -m_ref;   // a row with nothing to see yet
 #pragma unroll
       for (int i = 0; i < 64; i += 2) {
         const float p0 = fast_exp2(__fmaf_rn(sv[i], scale_log2e, neg_m));     // -inf -> 0
@@ -356,7 +358,7 @@ prefix_attention_basic_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n
   __syncthreads();
   const float l_tot = s_x[0][row] + s_x[1][row];
   if (!failed) {
-    const float inv = 1.f / l_tot;
+    const float inv = l_tot > 0.f ? 1.f / l_tot : 0.f;   // nothing seen: zeros, log-sum-exp -inf
 #pragma unroll
     for (int c = 0; c < 2; ++c) {
       uint32_t r[32];
@@ -429,7 +431,7 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
                            float* __restrict__ out, float* __restrict__ lse_out,
                            const __grid_constant__ CUtensorMap map_k,
                            const __grid_constant__ CUtensorMap map_v,
-                           int32_t* __restrict__ status_word, int split_len, long long rows_total) {
+                           int32_t* __restrict__ status_word, int split_len, long long rows_total, int causal) {
   constexpr int D = 128;
   constexpr int QT = kPfRows / G;                       // queries per query tile
   constexpr int NS = kPfStages;
@@ -468,6 +470,8 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
   const int head = h * G + row % G;
   const bool row_valid = softmax_thread && s_idx < n_queries;
   const long long row_off = ((bl * n_queries + s_idx) * g.Hq + head);
+  // causal: the last n_queries cached rows are the new tokens' own; query s stops at its own
+  const int n_row = causal && row_valid ? min(n, max(0, n_all - n_queries + s_idx + 1) - t_base) : n;
   if (n == 0) {                                         // empty cache: zeros, log-sum-exp = -inf
     if (row_valid) {
       for (int d = 0; d < D; ++d) out[row_off * D + d] = 0.f;
@@ -601,7 +605,8 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
       {
         uint32_t r0[32], r1[32];
         tmem_ld64(t_s, r0, r1);
-        if (valid >= kPfSub) {                            // CTA-uniform: only the last sub-block masks
+        const int valid_row = min(valid, n_row - j * kPfSub);
+        if (valid_row >= kPfSub) {                        // only the last (or a causal row's own) sub-block masks
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
             sv[i] = __uint_as_float(r0[i]);
@@ -611,8 +616,8 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
         } else {
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
-            sv[i] = i < valid ? __uint_as_float(r0[i]) : -INFINITY;
-            sv[32 + i] = 32 + i < valid ? __uint_as_float(r1[i]) : -INFINITY;
+            sv[i] = i < valid_row ? __uint_as_float(r0[i]) : -INFINITY;
+            sv[32 + i] = 32 + i < valid_row ? __uint_as_float(r1[i]) : -INFINITY;
             bmax = fmaxf(bmax, fmaxf(sv[i], sv[32 + i]));
           }
         }
@@ -634,7 +639,7 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
       {
         uint32_t pk[32];
         float rowsum0 = 0.f, rowsum1 = 0.f;
-        const float neg_m = -m_ref;
+        const float neg_m = m_ref == -INFINITY ? 0.f : -m_ref;   // a row with nothing to see yet
 #pragma unroll
         for (int i = 0; i < 64; i += 2) {
           const float p0 = fast_exp2(__fmaf_rn(sv[i], scale_log2e, neg_m));     // -inf -> 0
@@ -672,7 +677,7 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
   const bool failed = s_fail != 0;
   const float l_tot = l_run;
   if (!failed && softmax_thread && tile_active) {
-    const float inv = 1.f / l_tot;
+    const float inv = l_tot > 0.f ? 1.f / l_tot : 0.f;   // nothing seen: zeros, log-sum-exp -inf
 #pragma unroll 1
     for (int c = 0; c < 4; ++c) {
       uint32_t r[32];
@@ -716,12 +721,14 @@ prefix_merge_kernel(const float* __restrict__ part_out, const float* __restrict_
   for (int c = 0; c < nc; ++c) m = fmaxf(m, part_lse[c * rows_total + row]);
   float den = 0.f, num = 0.f;
   for (int c = 0; c < nc; ++c) {
-    const float w = __expf(part_lse[c * rows_total + row] - m);
+    const float lc = part_lse[c * rows_total + row];
+    const float w = lc > -INFINITY ? __expf(lc - m) : 0.f;
     den += w;
     num = fmaf(w, part_out[(c * rows_total + row) * 128 + d], num);
   }
-  out[row * 128 + d] = nc > 0 ? num / den : 0.f;
-  if (lse_out && d == 0) lse_out[row] = nc > 0 ? m + logf(den) : -INFINITY;
+  const bool any = nc > 0 && m > -INFINITY;             // some chunk had rows this query may see
+  out[row * 128 + d] = any ? num / den : 0.f;
+  if (lse_out && d == 0) lse_out[row] = any ? m + logf(den) : -INFINITY;
 }
 
 // How a launch is laid out.  Kernel: the pipelined one works on pairs of query tiles; with an odd,
@@ -773,7 +780,7 @@ template <int G>
 static int launch_pf(const void* q, const void* K, const void* V, const Geom& g, int n_queries,
                      const LenView& cur_len_dev, int max_len, float scale, float* out,
                      float* lse_out, int32_t* status_word, float* scratch, size_t scratch_bytes,
-                     cudaStream_t s) {
+                     int causal, cudaStream_t s) {
   PrefixPlan p = plan_prefix(g, n_queries, max_len);
   if (p.ctas == 0) return L2KV_OK;
   if (p.chunks > 1 && (!scratch || scratch_bytes < p.scratch_bytes)) {   // no room: one chunk
@@ -800,7 +807,7 @@ static int launch_pf(const void* q, const void* K, const void* V, const Geom& g,
       return L2KV_ERR_CUDA;
     kern_pipe<<<grid, kPfPipeThreads, smem_pipe, s>>>(qb, g, n_queries, cur_len_dev, max_len,
                                                       scale * kPfLog2e, k_out, k_lse, map_k, map_v,
-                                                      status_word, p.split_len, p.rows);
+                                                      status_word, p.split_len, p.rows, causal);
   } else {
     constexpr int smem_bytes = 1024 + 3 * kPfTileBytes;
     auto kern = prefix_attention_basic_kernel<G>;
@@ -808,7 +815,7 @@ static int launch_pf(const void* q, const void* K, const void* V, const Geom& g,
       return L2KV_ERR_CUDA;
     kern<<<grid, kPfThreads, smem_bytes, s>>>(qb, g, n_queries, cur_len_dev, max_len, scale * kPfLog2e,
                                               k_out, k_lse, map_k, map_v, status_word, p.split_len,
-                                              p.rows);
+                                              p.rows, causal);
   }
   if (cudaGetLastError() != cudaSuccess) return L2KV_ERR_CUDA;
   if (p.chunks > 1) {
@@ -824,11 +831,11 @@ static int launch_pf(const void* q, const void* K, const void* V, const Geom& g,
 int launch_prefix_attention(const void* q, const void* K, const void* V, const Geom& g, int dtype,
                             int n_queries, const LenView& cur_len_dev, int max_len, float scale,
                             float* out, float* lse_out, int32_t* status_word, float* scratch,
-                            size_t scratch_bytes, cudaStream_t s) {
+                            size_t scratch_bytes, int causal, cudaStream_t s) {
   if (dtype != L2KV_BF16 || g.D != 128) return L2KV_ERR_UNSUPPORTED;
 #define L2KV_PF(G)                                                                              \
   return launch_pf<G>(q, K, V, g, n_queries, cur_len_dev, max_len, scale, out, lse_out,         \
-                      status_word, scratch, scratch_bytes, s)
+                      status_word, scratch, scratch_bytes, causal, s)
   switch (g.Hq / g.H) {
     case 1: L2KV_PF(1);
     case 2: L2KV_PF(2);

@@ -144,3 +144,38 @@ def test_prefix_attention_split_over_the_cache(kernel, lens, monkeypatch):
     for l in range(2):
         if lens[l] == 0:
             assert not got[0, l].any() and np.all(np.isneginf(got_lse[0, l]))
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+@pytest.mark.parametrize("T,lens,n_q,split", [(700, [700, 333], 40, False), (300, [130, 17], 24, False),
+                                               (9000, [9000, 4620], 40, True)])
+def test_prefix_attention_causal(kernel, T, lens, n_q, split, monkeypatch):
+    """The chunk's own keys are the last n_q cached rows: query s sees rows < len - n_q + s + 1.
+    Checked query by query against the oracle with that length; a cache shorter than the chunk
+    (17 rows for 24 queries) leaves the first queries with nothing to see: zeros, lse = -inf."""
+    import paper_2406_11430_b200 as l2
+    choose(monkeypatch, kernel)
+    w = synth.WORKLOADS[2].scaled(B=1, L=2, Hkv=2, Hq=8, T=T)
+    K, V = synth.make_cache(w, DEV)
+    q = make_queries(w, n_q, 13)
+    cur = np.array([lens], dtype=np.int32)
+    ws = l2.prefix_attention_workspace(K, q, T) if split else torch.zeros(256, dtype=torch.uint8, device=DEV)
+    assert (ws.numel() > 256) == split
+    out = torch.full(q.shape, float("nan"), dtype=torch.float32, device=DEV)
+    lse = torch.full(q.shape[:4], float("nan"), dtype=torch.float32, device=DEV)
+    l2.prefix_attention_causal(q, K, V, i32(cur), T, out, lse, workspace=ws)
+    torch.cuda.synchronize()
+    assert l2.read_device_status(ws) == 0
+    got, got_lse = out.cpu().numpy(), lse.cpu().numpy()
+    Kn, Vn = synth.to_numpy(K), synth.to_numpy(V)
+    Kf, qf = K.float().cpu().numpy().astype(np.float64), q.float().cpu().numpy().astype(np.float64)
+    for s in sorted(set(list(range(0, n_q, 7)) + [n_q - 1])):
+        see = np.maximum(cur - n_q + s + 1, 0).astype(np.int32)
+        want = oracle.attention(synth.to_numpy(q[:, :, s].contiguous()), Kn, Vn, "bf16", see, nthreads=8)
+        assert_attention_close(got[:, :, s], want, atol=4e-3)
+        for l in range(2):
+            if see[0, l] == 0:
+                assert not got[0, l, s].any() and np.all(np.isneginf(got_lse[0, l, s]))
+            else:
+                z = Kf[0, l, 1, :see[0, l]] @ qf[0, l, s, 5] / np.sqrt(w.D)
+                np.testing.assert_allclose(got_lse[0, l, s, 5], scipy.special.logsumexp(z), rtol=1e-5, atol=1e-4)
