@@ -14,6 +14,7 @@
 // Two kernels share these pieces: the pipelined one (default) and a basic single-role one.
 // Every wait on an mbarrier is bounded (a wait that gives up ends the CTA's loop and marks
 // the status word); tensor memory is released on every path.
+#include <cmath>
 #include <cstdlib>
 #include <cstring>
 
@@ -759,12 +760,20 @@ static PrefixPlan plan_prefix(const Geom& g, int n_queries, int max_len) {
   p.ctas = units * (p.basic ? q_tiles : (q_tiles + 1) / 2);
   p.rows = (long long)g.B * g.L * n_queries * g.Hq;
   const long long slots = 148LL * (p.basic ? 2 : 1);     // CTAs the GPU holds at once
-  long long want = p.ctas > 0 ? (2 * slots + p.ctas - 1) / p.ctas : 1;   // two waves
-  if (max_len >= 65536) want = want > (max_len + 16383) / 16384 ? want : (max_len + 16383) / 16384;
   const long long by_len = max_len / 1024 > 1 ? max_len / 1024 : 1;
-  long long chunks = want < by_len ? want : by_len;
-  if (chunks > 64) chunks = 64;
-  if (chunks < 1) chunks = 1;
+  long long chunks = 1;
+  if (p.ctas > 0 && p.ctas < 2 * slots) {
+    // few CTAs: the chunk count that fills whole waves best, a CTA's fixed cost (set-up, the
+    // first fetches, the epilogue) counted as 256 tokens' worth of work
+    double best = 0.0;
+    for (long long c = 1; c <= by_len && c <= 64; ++c) {
+      const double waves = (double)(p.ctas * c) / (double)slots;
+      const double len = (double)max_len / (double)c;
+      const double eff = waves / std::ceil(waves) * len / (len + 256.0);
+      if (eff > best * 1.02) { best = eff; chunks = c; }   // more chunks only for a real gain
+    }
+  }
+  if (max_len >= 65536 && chunks < (max_len + 16383) / 16384) chunks = (max_len + 16383) / 16384;
   p.split_len = (int)round_up_ll((max_len + chunks - 1) / chunks, 128);
   if (p.split_len < 128) p.split_len = 128;
   p.chunks = max_len > 0 ? (max_len + p.split_len - 1) / p.split_len : 1;
