@@ -738,8 +738,8 @@ prefix_merge_kernel(const float* __restrict__ part_out, const float* __restrict_
 // (L2KV_PREFIX_KERNEL=basic / =pipelined overrides the choice).  Chunks: the cache is split over
 // blockIdx.y, with a merge pass after, when the unsplit grid would leave SMs idle (few KV heads
 // and query tiles, as in a call for one layer) or when the cache is so long that (b, l) pairs of
-// different lengths would leave a few CTAs running alone; chunks are multiples of 128 tokens
-// and at least 1024 long.
+// different lengths would leave a few CTAs running alone (chunks of 16k tokens then); chunks
+// are multiples of 128 tokens and at least 1024 long.
 struct PrefixPlan {
   bool basic;
   long long ctas;          // per chunk
