@@ -153,7 +153,8 @@ prefix_attention_basic_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n
                            float* __restrict__ out, float* __restrict__ lse_out,
                            const __grid_constant__ CUtensorMap map_k,
                            const __grid_constant__ CUtensorMap map_v,
-                           int32_t* __restrict__ status_word, int split_len, long long rows_total, int causal) {
+                           int32_t* __restrict__ status_word, int split_len, long long rows_total,
+                           int causal) {
   constexpr int D = 128;
   constexpr int QT = kPfRows / G;                       // queries per CTA
   extern __shared__ unsigned char smem_raw[];
@@ -409,7 +410,8 @@ __device__ __forceinline__ bool mbar_wait_likely(uint32_t bar, uint32_t parity) 
   return mbar_test(bar, parity) || mbar_wait<kPfPolls>(bar, parity);
 }
 
-// The pipelined kernel, the one the entry point uses.  The two contractions and the softmax
+// The pipelined kernel, the launcher's choice unless the query tiles per KV head are few and
+// odd.  The two contractions and the softmax
 // run concurrently, each in warps of its own, and one CTA per SM works on two query tiles
 // (256 rows) that share every K and V tile:
 //   - the cache is walked in sub-blocks of 64 tokens; per query tile two score buffers of 64
@@ -432,7 +434,8 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
                            float* __restrict__ out, float* __restrict__ lse_out,
                            const __grid_constant__ CUtensorMap map_k,
                            const __grid_constant__ CUtensorMap map_v,
-                           int32_t* __restrict__ status_word, int split_len, long long rows_total, int causal) {
+                           int32_t* __restrict__ status_word, int split_len, long long rows_total,
+                           int causal) {
   constexpr int D = 128;
   constexpr int QT = kPfRows / G;                       // queries per query tile
   constexpr int NS = kPfStages;
