@@ -110,3 +110,30 @@ def test_validation_of_the_analysis_and_prefix_entry_points():
     with pytest.raises(l2.L2KVError) as e:          # keys are required
         l2.attention_loss(qd, K, kl, 128, None, alr, workspace=_fake((1 << 20,), torch.uint8))
     assert e.value.status == -1
+
+
+def _prefix_ws_bytes(B, L, H, Hq, t_cap, max_len, n_q, dtype=torch.bfloat16, D=128):
+    cache = torch.empty((B, L, H, t_cap, D), dtype=dtype, device="meta")
+    lay = l2.Layout(cache, q_heads=Hq)
+    out = ctypes.c_size_t(0)
+    rc = l2.lib().l2kv_prefix_attention_workspace_bytes(lay.ref(), max_len, n_q, ctypes.byref(out))
+    return rc, out.value
+
+
+def test_prefix_attention_workspace_plan():
+    """Host side of the split over the cache: room for partial results is asked for only when
+    the unsplit grid would leave SMs idle or the cache is very long; sizes follow from the plan."""
+    rows = lambda B, L, n_q, Hq: B * L * n_q * Hq
+    # the benchmark call (all 32 layers, 2048 CTAs): no split
+    assert _prefix_ws_bytes(4, 32, 8, 32, 32768, 32768, 128) == (0, 256)
+    # one layer of it: 64 CTAs -> split; scratch = chunks * rows * (128 + 1) floats
+    rc, b = _prefix_ws_bytes(4, 1, 8, 32, 32768, 16384, 128)
+    per_chunk = rows(4, 1, 128, 32) * 129 * 4
+    assert rc == 0 and b > 256 and (b - 256) % per_chunk == 0 and 2 <= (b - 256) // per_chunk <= 16
+    # a very long cache is split whatever the grid (16k-token chunks)
+    rc, b = _prefix_ws_bytes(1, 32, 8, 32, 131072, 131072, 128)
+    assert rc == 0 and (b - 256) // (rows(1, 32, 128, 32) * 129 * 4) == 8
+    # short caches are never split below 1024 tokens; unsupported types ask for the status block only
+    assert _prefix_ws_bytes(1, 1, 2, 8, 1000, 1000, 16) == (0, 256)
+    assert _prefix_ws_bytes(1, 1, 4, 4, 1024, 1024, 16, dtype=torch.float32, D=64) == (0, 256)
+    assert _prefix_ws_bytes(1, 1, 8, 32, 4096, 8192, 16)[0] == -5          # max_len beyond t_cap
