@@ -12,14 +12,15 @@
 //                          running sum, and the sum over m of the difference (fp64 sums).
 //
 // Sorting is a bitonic network on power-of-two padded arrays in global scratch, with every
-// run of steps whose distance fits a 4096-element tile done in shared memory.  This is an
+// run of steps whose distance fits a 64 KB tile done in shared memory (arrays up to the tile
+// size never leave it between load and store).  This is an
 // analysis tool, not part of the decode hot path.
 #include "common.cuh"
 
 namespace l2kv {
 
 constexpr int kLossThreads = 1024;
-constexpr int kSortTile = 4096;
+constexpr int kSortTileBytes = 64 * 1024;   // dynamic shared memory of both kernels: 2-3 CTAs per SM
 
 __host__ __device__ inline int next_pow2(int n) {
   int p = 1;
@@ -36,11 +37,11 @@ __device__ __forceinline__ void cmp_swap(K& x, K& y, int i, int k) {
 }
 
 // Sorts a[0, n2) ascending (n2 a power of two) with the whole CTA; tile = shared scratch of
-// kSortTile keys.
+// kSortTileBytes.
 template <typename K>
 __device__ void bitonic_sort(K* __restrict__ a, int n2, K* __restrict__ tile) {
   const int tid = threadIdx.x;
-  const int tile_n = min(n2, kSortTile);
+  const int tile_n = min(n2, kSortTileBytes / (int)sizeof(K));
   // Phase I: each tile sorted (in alternating directions given by its global position).
   for (int base = 0; base < n2; base += tile_n) {
     for (int i = tid; i < tile_n; i += kLossThreads) tile[i] = a[base + i];
@@ -87,7 +88,8 @@ __device__ void bitonic_sort(K* __restrict__ a, int n2, K* __restrict__ tile) {
 __global__ void __launch_bounds__(kLossThreads)
 drop_order_kernel(const float* __restrict__ sumsq, Geom g, const int32_t* __restrict__ cur_len_dev,
                   int max_len, unsigned long long* __restrict__ order, int ld_order) {
-  __shared__ unsigned long long tile[kSortTile];
+  extern __shared__ __align__(16) unsigned char sort_smem[];
+  unsigned long long* tile = reinterpret_cast<unsigned long long*>(sort_smem);
   const long long unit = blockIdx.x;
   const long long bl = unit / g.H;
   const int n = max(0, min(cur_len_dev[bl], min(max_len, g.t_cap)));
@@ -148,7 +150,8 @@ attention_loss_kernel(const T* __restrict__ q, const T* __restrict__ K, Geom g,
   constexpr int EPV = Elem<T>::kPerVec;
   constexpr int LPR = D / EPV;
   constexpr int RPS = kLossThreads / LPR;
-  __shared__ float tile[kSortTile];
+  extern __shared__ __align__(16) unsigned char sort_smem[];
+  float* tile = reinterpret_cast<float*>(sort_smem);
   __shared__ double s_warp[kLossThreads / 32];
   __shared__ float s_redf[kLossThreads / 32];
   __shared__ float s_max;
@@ -266,9 +269,15 @@ static int launch_al_t(const void* q, const void* K, const Geom& g, const int32_
   unsigned long long* order = reinterpret_cast<unsigned long long*>(ws);
   float* probs = reinterpret_cast<float*>(ws + round_up_ll(units * (long long)ld * 8, 256));
   float* sorted = probs + round_up_ll(heads * (long long)ld * 4, 256) / 4;
-  drop_order_kernel<<<(unsigned)units, kLossThreads, 0, s>>>(sumsq, g, cur_len_dev, max_len, order, ld);
+  if (cudaFuncSetAttribute(drop_order_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           kSortTileBytes) != cudaSuccess ||
+      cudaFuncSetAttribute(attention_loss_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           kSortTileBytes) != cudaSuccess)
+    return L2KV_ERR_CUDA;
+  drop_order_kernel<<<(unsigned)units, kLossThreads, kSortTileBytes, s>>>(sumsq, g, cur_len_dev, max_len,
+                                                                          order, ld);
   if (cudaGetLastError() != cudaSuccess) return L2KV_ERR_CUDA;
-  attention_loss_kernel<T, D><<<(unsigned)heads, kLossThreads, 0, s>>>(
+  attention_loss_kernel<T, D><<<(unsigned)heads, kLossThreads, kSortTileBytes, s>>>(
       static_cast<const T*>(q), static_cast<const T*>(K), g, cur_len_dev, max_len,
       scale * 1.4426950408889634f, order, ld, probs, sorted, alr_out, loss_out, loss_ref_out);
   return cudaGetLastError() == cudaSuccess ? L2KV_OK : L2KV_ERR_CUDA;
