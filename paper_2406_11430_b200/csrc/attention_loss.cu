@@ -274,11 +274,6 @@ static int launch_al_t(const void* q, const void* K, const Geom& g, const int32_
       cudaFuncSetAttribute(attention_loss_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            kSortTileBytes) != cudaSuccess)
     return L2KV_ERR_CUDA;
-  // two CTAs of 1024 threads per SM need 128 KB of shared memory: ask for the large carve-out
-  cudaFuncSetAttribute(drop_order_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
-                       cudaSharedmemCarveoutMaxShared);
-  cudaFuncSetAttribute(attention_loss_kernel<T, D>, cudaFuncAttributePreferredSharedMemoryCarveout,
-                       cudaSharedmemCarveoutMaxShared);
   drop_order_kernel<<<(unsigned)units, kLossThreads, kSortTileBytes, s>>>(sumsq, g, cur_len_dev, max_len,
                                                                           order, ld);
   if (cudaGetLastError() != cudaSuccess) return L2KV_ERR_CUDA;
