@@ -36,12 +36,98 @@ __device__ __forceinline__ void cmp_swap(K& x, K& y, int i, int k) {
   if ((x > y) == asc) { const K t = x; x = y; y = t; }
 }
 
+// A full tile (kSortTileBytes) is held E elements per thread in registers, element e of the tile
+// = thread * E + r.  Steps of distance j < E are compare-exchanges inside a thread, E <= j < 32 E
+// exchanges between lanes of a warp (shuffles), and only j >= 32 E goes through shared memory
+// (element (thread, r) at tile[r * threads + thread]: conflict-free for any partner thread).
+template <typename K>
+__device__ __forceinline__ K keep_of(K mine, K other, int i, int j, int k) {
+  const bool lower = (i & j) == 0, asc = (i & k) == 0;
+  const bool keep_min = lower == asc;
+  const K lo = mine < other ? mine : other, hi = mine < other ? other : mine;
+  return keep_min ? lo : hi;
+}
+// Steps j = j_hi .. 1 of the network for runs of size k, on the tile whose first element has
+// global index base.
+template <typename K, int E>
+__device__ __forceinline__ void tile_steps_regs(K (&x)[E], int base, int k, int j_hi,
+                                                K* __restrict__ tile) {
+  const int tid = threadIdx.x;
+  const int i0 = base + tid * E;
+  int j = j_hi;
+  for (; j >= 32 * E; j >>= 1) {                         // partner thread in another warp
+    const int pt = tid ^ (j / E);
+    __syncthreads();                                     // earlier readers of the tile are done
+#pragma unroll
+    for (int r = 0; r < E; ++r) tile[r * kLossThreads + tid] = x[r];
+    __syncthreads();
+#pragma unroll
+    for (int r = 0; r < E; ++r) x[r] = keep_of(x[r], tile[r * kLossThreads + pt], i0 + r, j, k);
+  }
+  for (; j >= E; j >>= 1) {                              // partner thread in this warp
+    const int lm = j / E;
+#pragma unroll
+    for (int r = 0; r < E; ++r) x[r] = keep_of(x[r], __shfl_xor_sync(0xffffffffu, x[r], lm), i0 + r, j, k);
+  }
+#pragma unroll
+  for (int jj = E / 2; jj > 0; jj >>= 1) {               // both elements in this thread
+    if (jj <= j) {
+#pragma unroll
+      for (int r = 0; r < E; ++r)
+        if ((r & jj) == 0) cmp_swap(x[r], x[r | jj], i0 + r, k);
+    }
+  }
+}
+
 // Sorts a[0, n2) ascending (n2 a power of two) with the whole CTA; tile = shared scratch of
 // kSortTileBytes.
 template <typename K>
 __device__ void bitonic_sort(K* __restrict__ a, int n2, K* __restrict__ tile) {
   const int tid = threadIdx.x;
-  const int tile_n = min(n2, kSortTileBytes / (int)sizeof(K));
+  constexpr int kFull = kSortTileBytes / (int)sizeof(K);
+  constexpr int E = kFull / kLossThreads;
+  const int tile_n = min(n2, kFull);
+  if (tile_n == kFull) {
+    // Full tiles: the register formulation above; global memory only for distances >= a tile.
+    auto load = [&](K (&x)[E], int base) {
+      const uint4* src = reinterpret_cast<const uint4*>(a + base + tid * E);
+      uint4* dst = reinterpret_cast<uint4*>(x);
+#pragma unroll
+      for (int v = 0; v < (int)(E * sizeof(K) / 16); ++v) dst[v] = src[v];
+    };
+    auto store = [&](const K (&x)[E], int base) {
+      uint4* dst = reinterpret_cast<uint4*>(a + base + tid * E);
+      const uint4* src = reinterpret_cast<const uint4*>(x);
+#pragma unroll
+      for (int v = 0; v < (int)(E * sizeof(K) / 16); ++v) dst[v] = src[v];
+    };
+    for (int base = 0; base < n2; base += kFull) {       // every tile sorted (direction by position)
+      K x[E];
+      load(x, base);
+      for (int k = 2; k <= kFull; k <<= 1) tile_steps_regs<K, E>(x, base, k, k >> 1, tile);
+      store(x, base);
+    }
+    __syncthreads();
+    for (int k = kFull << 1; k <= n2; k <<= 1) {         // merges of runs larger than a tile
+      for (int j = k >> 1; j >= kFull; j >>= 1) {
+        for (int t = tid; t < n2 / 2; t += kLossThreads) {
+          const int lo = ((t & ~(j - 1)) << 1) | (t & (j - 1));
+          K x = a[lo], y = a[lo | j];
+          cmp_swap(x, y, lo, k);
+          a[lo] = x; a[lo | j] = y;
+        }
+        __syncthreads();
+      }
+      for (int base = 0; base < n2; base += kFull) {
+        K x[E];
+        load(x, base);
+        tile_steps_regs<K, E>(x, base, k, kFull >> 1, tile);
+        store(x, base);
+      }
+      __syncthreads();
+    }
+    return;
+  }
   // Phase I: each tile sorted (in alternating directions given by its global position).
   for (int base = 0; base < n2; base += tile_n) {
     for (int i = tid; i < tile_n; i += kLossThreads) tile[i] = a[base + i];
@@ -57,31 +143,6 @@ __device__ void bitonic_sort(K* __restrict__ a, int n2, K* __restrict__ tile) {
     }
     for (int i = tid; i < tile_n; i += kLossThreads) a[base + i] = tile[i];
     __syncthreads();
-  }
-  // Phase II: merge runs larger than a tile: far steps in global memory, near steps per tile.
-  for (int k = tile_n << 1; k <= n2; k <<= 1) {
-    for (int j = k >> 1; j >= tile_n; j >>= 1) {
-      for (int t = tid; t < n2 / 2; t += kLossThreads) {
-        const int lo = ((t & ~(j - 1)) << 1) | (t & (j - 1));
-        K x = a[lo], y = a[lo | j];
-        cmp_swap(x, y, lo, k);
-        a[lo] = x; a[lo | j] = y;
-      }
-      __syncthreads();
-    }
-    for (int base = 0; base < n2; base += tile_n) {
-      for (int i = tid; i < tile_n; i += kLossThreads) tile[i] = a[base + i];
-      __syncthreads();
-      for (int j = tile_n >> 1; j > 0; j >>= 1) {
-        for (int t = tid; t < tile_n / 2; t += kLossThreads) {
-          const int lo = ((t & ~(j - 1)) << 1) | (t & (j - 1));
-          cmp_swap(tile[lo], tile[lo | j], base + lo, k);
-        }
-        __syncthreads();
-      }
-      for (int i = tid; i < tile_n; i += kLossThreads) a[base + i] = tile[i];
-      __syncthreads();
-    }
   }
 }
 
