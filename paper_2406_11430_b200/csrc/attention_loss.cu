@@ -7,9 +7,8 @@
 //   drop_order_kernel      one CTA per (b, l, kv head): sorts (key bits << 32 | position)
 //                          ascending; read backwards this is the method's drop order,
 //                          shared by the G query heads of the KV head.
-//   attention_loss_kernel  one CTA per (b, l, kv head): the scores of the group's query heads
-//                          (four heads per pass over K), then per query head: probabilities,
-//                          their running sum in drop order, a sort of the probabilities and its
+//   attention_loss_kernel  one CTA per (b, l, query head): scores -> probabilities, their
+//                          running sum in drop order, a sort of the probabilities and its
 //                          running sum, and the sum over m of the difference (fp64 sums).
 //
 // Sorting is a bitonic network on power-of-two padded arrays in global scratch, with every
@@ -202,7 +201,7 @@ __device__ double running_sums(int n, F f, E emit, double* s_warp) {
   return sum;
 }
 
-template <typename T, int D, int GB>                   // GB: query heads scored per pass over K
+template <typename T, int D>
 __global__ void __launch_bounds__(kLossThreads)
 attention_loss_kernel(const T* __restrict__ q, const T* __restrict__ K, Geom g,
                       const int32_t* __restrict__ cur_len_dev, int max_len, float scale_log2e,
@@ -215,129 +214,101 @@ attention_loss_kernel(const T* __restrict__ q, const T* __restrict__ K, Geom g,
   extern __shared__ __align__(16) unsigned char sort_smem[];
   float* tile = reinterpret_cast<float*>(sort_smem);
   __shared__ double s_warp[kLossThreads / 32];
+  __shared__ float s_redf[kLossThreads / 32];
+  __shared__ float s_max;
 
-  __shared__ float s_max[8];
-  __shared__ float s_redg[GB][kLossThreads / 32];
-
-  const long long unit = blockIdx.x;                     // (b * L + l) * H + h
-  const int h = (int)(unit % g.H);
-  const long long bl = unit / g.H;
+  const long long row = blockIdx.x;                      // (b * L + l) * Hq + hq
+  const int hq = (int)(row % g.Hq);
+  const long long bl = row / g.Hq;
   const int l = (int)(bl % g.L), b = (int)(bl / g.L);
   const int G = g.Hq / g.H;
-  const long long row0 = bl * g.Hq + (long long)h * G;   // first query head of the group
+  const int h = hq / G;
   const int n = max(0, min(cur_len_dev[bl], min(max_len, g.t_cap)));
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  if (n == 0) { if (tid < G) alr_out[row0 + tid] = 0.f; return; }
+  if (n == 0) { if (tid == 0) alr_out[row] = 0.f; return; }
   const int n2 = next_pow2(n);
-  const unsigned long long* ord = order + unit * ld_order;
+  float* a = probs + row * ld_order;
+  float* srt = sorted + row * ld_order;
+  const unsigned long long* ord = order + (bl * g.H + h) * ld_order;
 
-  // ---- scores (log2 domain) of the group's query heads, GB heads per pass over K: LPR adjacent
-  //      lanes own one key row and share its GB dot products (halving exchange) ---------------
+  // scores (log2 domain): LPR adjacent lanes own one key row
   const int piece = tid % LPR, sub = tid / LPR;
-  constexpr int LPG = LPR / GB;                          // lanes that end up with one head's sum
-  const int my_g = piece / LPG;                          // ... and which head that is
+  float qf[EPV];
+  {
+    const uint4 v = *reinterpret_cast<const uint4*>(q + row * D + piece * EPV);
+    Elem<T>::unpack(v, qf);
+#pragma unroll
+    for (int e = 0; e < EPV; ++e) qf[e] *= scale_log2e;
+  }
   const T* kbase = K + b * g.sb + l * g.sl + h * g.sh + (long long)piece * EPV;
-  for (int g0 = 0; g0 < G; g0 += GB) {
-    float qf[GB][EPV];
+  float mx = -INFINITY;
+  constexpr int U = 4;                                   // key rows in flight per thread
+  for (int rb = 0; rb < n; rb += RPS * U) {
+    uint4 v[U];
 #pragma unroll
-    for (int gi = 0; gi < GB; ++gi) {
-      if (g0 + gi < G) {
-        const uint4 v = *reinterpret_cast<const uint4*>(q + (row0 + g0 + gi) * D + piece * EPV);
-        Elem<T>::unpack(v, qf[gi]);
-#pragma unroll
-        for (int e = 0; e < EPV; ++e) qf[gi][e] *= scale_log2e;
-      } else {
-#pragma unroll
-        for (int e = 0; e < EPV; ++e) qf[gi][e] = 0.f;
-      }
+    for (int u = 0; u < U; ++u) {
+      const int t = rb + u * RPS + sub;
+      v[u] = t < n ? ld_stream(kbase + (long long)t * g.st) : make_uint4(0, 0, 0, 0);
     }
-    const bool writer = piece % LPG == 0 && g0 + my_g < G;
-    float* a_mine = probs + (row0 + g0 + my_g) * ld_order;
-    float mx = -INFINITY;
-    constexpr int U = 4;                                 // key rows in flight per thread
-    for (int rb = 0; rb < n; rb += RPS * U) {
-      uint4 v[U];
 #pragma unroll
-      for (int u = 0; u < U; ++u) {
-        const int t = rb + u * RPS + sub;
-        v[u] = t < n ? ld_stream(kbase + (long long)t * g.st) : make_uint4(0, 0, 0, 0);
-      }
+    for (int u = 0; u < U; ++u) {
+      const int t = rb + u * RPS + sub;
+      float x[EPV], d[1];
+      Elem<T>::unpack(v[u], x);
+      float acc = 0.f;
 #pragma unroll
-      for (int u = 0; u < U; ++u) {
-        const int t = rb + u * RPS + sub;
-        float x[EPV], d[GB];
-        Elem<T>::unpack(v[u], x);
-#pragma unroll
-        for (int gi = 0; gi < GB; ++gi) {
-          float acc = 0.f;
-#pragma unroll
-          for (int e = 0; e < EPV; ++e) acc = fmaf(qf[gi][e], x[e], acc);
-          d[gi] = acc;
-        }
-        const float sc = halving_reduce<GB, LPR>(d, piece);   // head my_g's score of row t
-        if (writer && t < n) { a_mine[t] = sc; mx = fmaxf(mx, sc); }
-      }
+      for (int e = 0; e < EPV; ++e) acc = fmaf(qf[e], x[e], acc);
+      d[0] = acc;
+      const float s = halving_reduce<1, LPR>(d, piece);
+      if (piece == 0 && t < n) { a[t] = s; mx = fmaxf(mx, s); }
     }
-    // maxima per head
-#pragma unroll
-    for (int gi = 0; gi < GB; ++gi) {
-      float v = (writer && my_g == gi) ? mx : -INFINITY;
-#pragma unroll
-      for (int off = 16; off >= 1; off >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, off));
-      if (lane == 0) s_redg[gi][warp] = v;
-    }
-    __syncthreads();
-    if (tid < GB && g0 + tid < G) {
-      float m = s_redg[tid][0];
-      for (int w = 1; w < kLossThreads / 32; ++w) m = fmaxf(m, s_redg[tid][w]);
-      s_max[g0 + tid] = m;
-    }
-    __syncthreads();
   }
-
-  // ---- per query head: probabilities, the two running sums, their difference -----------------
-  for (int gq = 0; gq < G; ++gq) {
-    const long long row = row0 + gq;                     // (b * L + l) * Hq + hq
-    float* a = probs + row * ld_order;
-    float* srt = sorted + row * ld_order;
-    const float m = s_max[gq];
-    // weights and their sum
-    double part = 0.0;
-    for (int t = tid; t < n; t += kLossThreads) {
-      const float w = exp2f(a[t] - m);
-      a[t] = w;
-      part += (double)w;
-    }
 #pragma unroll
-    for (int off = 16; off >= 1; off >>= 1) part += __shfl_xor_sync(0xffffffffu, part, off);
-    if (lane == 0) s_warp[warp] = part;
-    __syncthreads();
-    double denom = 0.0;
-    for (int w = 0; w < kLossThreads / 32; ++w) denom += s_warp[w];
-    __syncthreads();
-    const float inv = (float)(1.0 / denom);
-    for (int t = tid; t < n2; t += kLossThreads) {
-      const float p = t < n ? a[t] * inv : __uint_as_float(0x7f800000u);   // +inf pads the sort
-      if (t < n) a[t] = p;
-      srt[t] = p;
-    }
-    __syncthreads();
-
-    // L^m: running sum of the probabilities in the method's drop order (largest key first)
-    float* lo = loss_out ? loss_out + row * g.t_cap : nullptr;
-    const double sum_l = running_sums(
-        n, [&](int r) { return a[(uint32_t)(ord[n - 1 - r] & 0xffffffffull)]; },
-        [&](int r, double v) { if (lo) lo[r] = (float)v; }, s_warp);
-
-    // L^{m,ref}: running sum of the probabilities sorted ascending (non-negative floats order
-    // as their bit patterns)
-    bitonic_sort(reinterpret_cast<uint32_t*>(srt), n2, reinterpret_cast<uint32_t*>(tile));
-    float* lr = loss_ref_out ? loss_ref_out + row * g.t_cap : nullptr;
-    const double sum_ref = running_sums(
-        n, [&](int r) { return srt[r]; }, [&](int r, double v) { if (lr) lr[r] = (float)v; }, s_warp);
-    if (tid == 0) alr_out[row] = (float)(sum_l - sum_ref);
-    __syncthreads();
+  for (int off = 16; off >= 1; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+  if (lane == 0) s_redf[warp] = mx;
+  __syncthreads();
+  if (tid == 0) {
+    float m = s_redf[0];
+    for (int w = 1; w < kLossThreads / 32; ++w) m = fmaxf(m, s_redf[w]);
+    s_max = m;
   }
+  __syncthreads();
+  const float m = s_max;
+  // weights and their sum
+  double part = 0.0;
+  for (int t = tid; t < n; t += kLossThreads) {
+    const float w = exp2f(a[t] - m);
+    a[t] = w;
+    part += (double)w;
+  }
+#pragma unroll
+  for (int off = 16; off >= 1; off >>= 1) part += __shfl_xor_sync(0xffffffffu, part, off);
+  if (lane == 0) s_warp[warp] = part;
+  __syncthreads();
+  double denom = 0.0;
+  for (int w = 0; w < kLossThreads / 32; ++w) denom += s_warp[w];
+  __syncthreads();
+  const float inv = (float)(1.0 / denom);
+  for (int t = tid; t < n2; t += kLossThreads) {
+    const float p = t < n ? a[t] * inv : __uint_as_float(0x7f800000u);   // +inf pads the sort
+    if (t < n) a[t] = p;
+    srt[t] = p;
+  }
+  __syncthreads();
+
+  // L^m: running sum of the probabilities in the method's drop order (largest key first)
+  float* lo = loss_out ? loss_out + row * g.t_cap : nullptr;
+  const double sum_l = running_sums(
+      n, [&](int r) { return a[(uint32_t)(ord[n - 1 - r] & 0xffffffffull)]; },
+      [&](int r, double v) { if (lo) lo[r] = (float)v; }, s_warp);
+
+  // L^{m,ref}: running sum of the probabilities sorted ascending (non-negative floats order
+  // as their bit patterns)
+  bitonic_sort(reinterpret_cast<uint32_t*>(srt), n2, reinterpret_cast<uint32_t*>(tile));
+  float* lr = loss_ref_out ? loss_ref_out + row * g.t_cap : nullptr;
+  const double sum_ref = running_sums(
+      n, [&](int r) { return srt[r]; }, [&](int r, double v) { if (lr) lr[r] = (float)v; }, s_warp);
+  if (tid == 0) alr_out[row] = (float)(sum_l - sum_ref);
 }
 
 size_t attention_loss_workspace(const l2kv_layout& a, int max_len) {
@@ -361,20 +332,13 @@ static int launch_al_t(const void* q, const void* K, const Geom& g, const int32_
   float* sorted = probs + round_up_ll(heads * (long long)ld * 4, 256) / 4;
   if (cudaFuncSetAttribute(drop_order_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            kSortTileBytes) != cudaSuccess ||
-      cudaFuncSetAttribute(attention_loss_kernel<T, D, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           kSortTileBytes) != cudaSuccess ||
-      cudaFuncSetAttribute(attention_loss_kernel<T, D, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           kSortTileBytes) != cudaSuccess ||
-      cudaFuncSetAttribute(attention_loss_kernel<T, D, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+      cudaFuncSetAttribute(attention_loss_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            kSortTileBytes) != cudaSuccess)
     return L2KV_ERR_CUDA;
   drop_order_kernel<<<(unsigned)units, kLossThreads, kSortTileBytes, s>>>(sumsq, g, cur_len_dev, max_len,
                                                                           order, ld);
   if (cudaGetLastError() != cudaSuccess) return L2KV_ERR_CUDA;
-  const int G = g.Hq / g.H;
-  auto kern = G >= 4 ? attention_loss_kernel<T, D, 4>
-            : G >= 2 ? attention_loss_kernel<T, D, 2> : attention_loss_kernel<T, D, 1>;
-  kern<<<(unsigned)units, kLossThreads, kSortTileBytes, s>>>(
+  attention_loss_kernel<T, D><<<(unsigned)heads, kLossThreads, kSortTileBytes, s>>>(
       static_cast<const T*>(q), static_cast<const T*>(K), g, cur_len_dev, max_len,
       scale * 1.4426950408889634f, order, ld, probs, sorted, alr_out, loss_out, loss_ref_out);
   return cudaGetLastError() == cudaSuccess ? L2KV_OK : L2KV_ERR_CUDA;
