@@ -4,6 +4,11 @@ Only the tests, the smoke check and the CPU-baseline leg of the benchmark may
 import this package; the GPU library never does.  Arrays are dense and
 C-contiguous, laid out [B, L, H, T_cap, D]; bfloat16 data travels as uint16
 bit patterns (``dtype='bf16'``), fp32 as float32.
+
+The ``*_packed`` forms take ragged caches without padding: tensors [H, total_rows, D]
+(index map and keys [H, total_rows]) plus ``rows = (row_off, row_cap, total_rows)``,
+where the rows of (b, l) are [row_off[b, l], row_off[b, l] + row_cap[b, l]) for every
+head.  They compute what the dense forms compute; only the addressing differs.
 """
 import ctypes
 import os
@@ -177,3 +182,76 @@ def attention_loss(q, K, dtype, cur_len, scale=0.0, key_mode=0, curves=False, nt
     if rc != 0:
         raise ValueError(f"oracle attention_loss: bad argument ({rc})")
     return (alr, loss, ref) if curves else alr
+
+
+def _rows(rows, B, L):
+    off, cap, total = rows
+    off = np.ascontiguousarray(np.asarray(off, dtype=np.int64)).reshape(B, L)
+    cap = np.ascontiguousarray(np.asarray(cap, dtype=np.int32)).reshape(B, L)
+    assert int((off + cap).max()) <= int(total) and int(off.min()) >= 0
+    return off, cap, int(total)
+
+
+def compress_packed(K, V, dtype, in_rows, lens, keep, uncompressed, out_rows, L, key_mode=0,
+                    policy=0, nthreads=1, seed=0):
+    """compress() on packed tensors K, V [H, total_in, D]; `keep` is [B].  Returns dict(K_c, V_c
+    [H, total_out, D], idx, key [H, total_out], kept_len [B, L])."""
+    _check(K, dtype)
+    _check(V, dtype)
+    H, total_in, D = K.shape
+    lens, keep, unc = _i32(lens), _i32(keep), _i32(list(uncompressed))
+    B = lens.size
+    ioff, icap, itot = _rows(in_rows, B, L)
+    ooff, ocap, otot = _rows(out_rows, B, L)
+    assert itot == total_in
+    K_c = np.zeros((H, otot, D), dtype=K.dtype)
+    V_c = np.zeros_like(K_c)
+    idx = np.full((H, otot), -1, dtype=np.int32)
+    key = np.full((H, otot), np.nan, dtype=np.float64)
+    kept_len = np.zeros((B, L), dtype=np.int32)
+    rc = lib().l2kv_oracle_compress_packed(
+        _p(K), _p(V), _DT[dtype], B, L, H, _p(ioff), _p(icap), ctypes.c_int64(itot), D, _p(lens),
+        _p(keep), _p(unc), int(unc.size), int(key_mode), int(policy),
+        ctypes.c_uint64(int(seed) & 0xFFFFFFFFFFFFFFFF), _p(ooff), _p(ocap), ctypes.c_int64(otot),
+        _p(K_c), _p(V_c), _p(idx), _p(key), _p(kept_len), None, None, int(nthreads))
+    if rc != 0:
+        raise ValueError(f"oracle compress_packed: bad argument ({rc})")
+    return dict(K_c=K_c, V_c=V_c, idx=idx, key=key, kept_len=kept_len)
+
+
+def attention_packed(q, K_c, V_c, dtype, rows, cur_len, scale=0.0, nthreads=1):
+    """attention() over a packed cache K_c, V_c [Hkv, total_rows, D]; cur_len [B, L]."""
+    _check(q, dtype)
+    _check(K_c, dtype)
+    _check(V_c, dtype)
+    B, L, Hq, D = q.shape
+    Hkv = K_c.shape[0]
+    off, cap, tot = _rows(rows, B, L)
+    assert tot == K_c.shape[1]
+    cur_len = _i32(cur_len).reshape(B, L)
+    out = np.empty((B, L, Hq, D), dtype=np.float64)
+    rc = lib().l2kv_oracle_attention_packed(
+        _p(q), _p(K_c), _p(V_c), _DT[dtype], B, L, Hkv, Hq, _p(off), _p(cap), ctypes.c_int64(tot),
+        D, _p(cur_len), ctypes.c_double(scale), _p(out), None, int(nthreads))
+    if rc != 0:
+        raise ValueError(f"oracle attention_packed: bad argument ({rc})")
+    return out
+
+
+def append_evict_packed(state, dtype, rows, budget, uncompressed, k_new, v_new, pos_new, key_mode=0):
+    """append_evict() in place on a packed state = dict(K_c, V_c [H, total_rows, D], idx, key
+    [H, total_rows], cur_len [B, L]); budget [B]."""
+    K_c, V_c = state["K_c"], state["V_c"]
+    _check(K_c, dtype)
+    _check(k_new, dtype)
+    _check(v_new, dtype)
+    B, L, H, D = k_new.shape
+    off, cap, tot = _rows(rows, B, L)
+    assert K_c.shape == (H, tot, D) and state["idx"].shape == (H, tot)
+    budget, unc, pos_new = _i32(budget), _i32(list(uncompressed)), _i32(pos_new)
+    assert state["idx"].dtype == np.int32 and state["key"].dtype == np.float64
+    assert state["cur_len"].dtype == np.int32 and state["cur_len"].shape == (B, L)
+    return int(lib().l2kv_oracle_append_evict_packed(
+        _p(K_c), _p(V_c), _p(state["idx"]), _p(state["key"]), _DT[dtype], B, L, H, _p(off), _p(cap),
+        ctypes.c_int64(tot), D, _p(state["cur_len"]), _p(budget), _p(unc), int(unc.size),
+        _p(k_new), _p(v_new), _p(pos_new), int(key_mode), 0))

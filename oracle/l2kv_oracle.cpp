@@ -34,7 +34,11 @@
 // paper's accuracy figures) needs weights and datasets: parity unpinned, and
 // out of scope.
 //
-// Layout: every cache tensor is dense [B, L, H, T_cap, D] with D contiguous.
+// Layout: a cache tensor is dense [B, L, H, T_cap, D] with D contiguous, or, in the
+// *_packed routines, packed [H, total_rows, D]: the rows of (b, l) are the range
+// [row_off[b, l], row_off[b, l] + row_cap[b, l]) of a row axis that all sequences and
+// layers share, the same range for every head (ragged batches without padding; only
+// where rows live changes, never what is computed -- pinned against the dense form).
 // dtype 0 = IEEE fp32, dtype 1 = bfloat16 stored as raw uint16.
 
 #include <algorithm>
@@ -165,6 +169,38 @@ void for_each_unit(int64_t n, int nthreads, F fn) {
   for (auto& t : pool) t.join();
 }
 
+// Where the rows of unit u = (b * L + l) * H + h live on the row axis of a cache tensor
+// (and of the per-row index map and keys, which have the same row axis).
+struct Rows {
+  int H;
+  int64_t T_cap;              // dense: rows per unit
+  const int64_t* row_off;     // packed: [B * L] first row of (b, l); null = dense
+  const int32_t* row_cap;     // packed: [B * L] rows (b, l) may hold
+  int64_t total_rows;         // packed: extent of the shared row axis
+  int64_t first(int64_t u) const {
+    return row_off ? (u % H) * total_rows + row_off[u / H] : u * T_cap;
+  }
+  int64_t cap(int64_t u) const { return row_off ? row_cap[u / H] : T_cap; }
+};
+
+Rows dense_rows(int H, int64_t T_cap) { return Rows{H, T_cap, nullptr, nullptr, 0}; }
+Rows packed_rows(int H, const int64_t* off, const int32_t* cap, int64_t total) {
+  return Rows{H, 0, off, cap, total};
+}
+
+int compress_impl(const void* K, const void* V, int dtype, int B, int L, int H, Rows rin, int D,
+                  const int32_t* len, const int32_t* keep, const int32_t* uncompressed, int n_unc,
+                  int key_mode, int policy, uint64_t seed, Rows rout, void* K_out, void* V_out,
+                  int32_t* idx_out, double* key_out, int32_t* kept_len, const int32_t* keep_unit,
+                  int32_t* kept_len_unit, int nthreads);
+int attention_impl(const void* q, const void* K_c, const void* V_c, int dtype, int B, int L, int Hkv,
+                   int Hq, Rows rows, int D, const int32_t* cur_len, double scale, double* out,
+                   const int32_t* cur_len_unit, int nthreads);
+int append_evict_impl(void* K_c, void* V_c, int32_t* idx, double* key_c, int dtype, int B, int L,
+                      int H, Rows rows, int D, int32_t* cur_len, const int32_t* budget,
+                      const int32_t* uncompressed, int n_unc, const void* k_new, const void* v_new,
+                      const int32_t* pos_new, int key_mode, int per_head);
+
 }  // namespace
 
 extern "C" {
@@ -224,17 +260,49 @@ int l2kv_oracle_compress(const void* K, const void* V, int dtype, int B, int L, 
                          uint64_t seed, int T_cap_out, void* K_out, void* V_out, int32_t* idx_out,
                          double* key_out, int32_t* kept_len, const int32_t* keep_unit,
                          int32_t* kept_len_unit, int nthreads) {
+  return compress_impl(K, V, dtype, B, L, H, dense_rows(H, T_cap), D, len, keep, uncompressed, n_unc,
+                       key_mode, policy, seed, dense_rows(H, T_cap_out), K_out, V_out, idx_out,
+                       key_out, kept_len, keep_unit, kept_len_unit, nthreads);
+}
+
+// The same on packed tensors: K, V [H, total_in, D] with rows (in_off, in_cap); K_out, V_out
+// [H, total_out, D], idx_out / key_out [H, total_out] with rows (out_off, out_cap).
+int l2kv_oracle_compress_packed(const void* K, const void* V, int dtype, int B, int L, int H,
+                                const int64_t* in_off, const int32_t* in_cap, int64_t total_in, int D,
+                                const int32_t* len, const int32_t* keep, const int32_t* uncompressed,
+                                int n_unc, int key_mode, int policy, uint64_t seed,
+                                const int64_t* out_off, const int32_t* out_cap, int64_t total_out,
+                                void* K_out, void* V_out, int32_t* idx_out, double* key_out,
+                                int32_t* kept_len, const int32_t* keep_unit, int32_t* kept_len_unit,
+                                int nthreads) {
+  return compress_impl(K, V, dtype, B, L, H, packed_rows(H, in_off, in_cap, total_in), D, len, keep,
+                       uncompressed, n_unc, key_mode, policy, seed,
+                       packed_rows(H, out_off, out_cap, total_out), K_out, V_out, idx_out, key_out,
+                       kept_len, keep_unit, kept_len_unit, nthreads);
+}
+
+}  // extern "C"
+
+namespace {
+
+int compress_impl(const void* K, const void* V, int dtype, int B, int L, int H, Rows rin, int D,
+                  const int32_t* len, const int32_t* keep, const int32_t* uncompressed, int n_unc,
+                  int key_mode, int policy, uint64_t seed, Rows rout, void* K_out, void* V_out,
+                  int32_t* idx_out, double* key_out, int32_t* kept_len, const int32_t* keep_unit,
+                  int32_t* kept_len_unit, int nthreads) {
   if (keep_unit != nullptr && kept_len_unit == nullptr) return -1;
   for (int b = 0; b < B; ++b) {
-    if (len[b] < 0 || len[b] > T_cap) return -1;
-    if (keep_unit == nullptr) {
-      if (keep[b] < 0 || keep[b] > len[b]) return -1;
-      if (keep[b] > T_cap_out) return -1;
-    } else {
-      for (int64_t u = int64_t(b) * L * H; u < int64_t(b + 1) * L * H; ++u)
-        if (keep_unit[u] < 0 || keep_unit[u] > len[b] || keep_unit[u] > T_cap_out) return -1;
+    if (len[b] < 0) return -1;
+    if (keep_unit == nullptr && (keep[b] < 0 || keep[b] > len[b])) return -1;
+    for (int64_t u = int64_t(b) * L * H; u < int64_t(b + 1) * L * H; ++u) {
+      const int l = static_cast<int>((u / H) % L);
+      if (len[b] > rin.cap(u)) return -1;
+      if (keep_unit != nullptr && (keep_unit[u] < 0 || keep_unit[u] > len[b])) return -1;
+      const int n_out = in_list(uncompressed, n_unc, l) ? len[b]
+                        : keep_unit != nullptr          ? keep_unit[u]
+                                                        : keep[b];
+      if (n_out > rout.cap(u)) return -1;
     }
-    if (n_unc > 0 && len[b] > T_cap_out) return -1;
   }
   const int es = elem_size(dtype);
   std::vector<int32_t> unit_keep_store(size_t(B) * L * H);
@@ -255,8 +323,8 @@ int l2kv_oracle_compress(const void* K, const void* V, int dtype, int B, int L, 
     const int l = static_cast<int>((u / H) % L);
     const int T = len[b];
     const int n_keep = unit_keep[u];
-    const int64_t in_row0 = u * T_cap;        // first row of this unit, in rows
-    const int64_t out_row0 = u * T_cap_out;
+    const int64_t in_row0 = rin.first(u);     // first row of this unit, in rows
+    const int64_t out_row0 = rout.first(u);
     std::vector<double> key(T);
     for (int t = 0; t < T; ++t) key[t] = row_key(K, dtype, (in_row0 + t) * D, D, key_mode);
     std::vector<int32_t> kept(n_keep);
@@ -282,6 +350,10 @@ int l2kv_oracle_compress(const void* K, const void* V, int dtype, int B, int L, 
   return 0;
 }
 
+}  // namespace
+
+extern "C" {
+
 // a5: one query per query head over the cached rows [0, cur_len[b, l]).
 //   q [B, L, Hq, D]; K_c, V_c [B, L, Hkv, T_cap, D]; out double [B, L, Hq, D]
 // Query head j reads KV head j / (Hq / Hkv) (reading: contiguous grouping; the
@@ -292,6 +364,28 @@ int l2kv_oracle_compress(const void* K, const void* V, int dtype, int B, int L, 
 int l2kv_oracle_attention(const void* q, const void* K_c, const void* V_c, int dtype, int B, int L,
                           int Hkv, int Hq, int T_cap, int D, const int32_t* cur_len, double scale,
                           double* out, const int32_t* cur_len_unit, int nthreads) {
+  return attention_impl(q, K_c, V_c, dtype, B, L, Hkv, Hq, dense_rows(Hkv, T_cap), D, cur_len, scale,
+                        out, cur_len_unit, nthreads);
+}
+
+// The same over a packed cache: K_c, V_c [Hkv, total_rows, D] with rows (row_off, row_cap).
+int l2kv_oracle_attention_packed(const void* q, const void* K_c, const void* V_c, int dtype, int B,
+                                 int L, int Hkv, int Hq, const int64_t* row_off,
+                                 const int32_t* row_cap, int64_t total_rows, int D,
+                                 const int32_t* cur_len, double scale, double* out,
+                                 const int32_t* cur_len_unit, int nthreads) {
+  return attention_impl(q, K_c, V_c, dtype, B, L, Hkv, Hq,
+                        packed_rows(Hkv, row_off, row_cap, total_rows), D, cur_len, scale, out,
+                        cur_len_unit, nthreads);
+}
+
+}  // extern "C"
+
+namespace {
+
+int attention_impl(const void* q, const void* K_c, const void* V_c, int dtype, int B, int L, int Hkv,
+                   int Hq, Rows rows, int D, const int32_t* cur_len, double scale, double* out,
+                   const int32_t* cur_len_unit, int nthreads) {
   if (Hkv <= 0 || Hq % Hkv != 0) return -1;
   const int G = Hq / Hkv;
   const double sc = scale > 0.0 ? scale : 1.0 / std::sqrt(static_cast<double>(D));
@@ -299,7 +393,7 @@ int l2kv_oracle_attention(const void* q, const void* K_c, const void* V_c, int d
     const int hq = static_cast<int>(u % Hq);
     const int64_t bl = u / Hq;
     const int n = cur_len_unit != nullptr ? cur_len_unit[bl * Hkv + hq / G] : cur_len[bl];
-    const int64_t kv_row0 = (bl * Hkv + hq / G) * T_cap;
+    const int64_t kv_row0 = rows.first(bl * Hkv + hq / G);
     double* o = out + u * D;
     for (int d = 0; d < D; ++d) o[d] = 0.0;
     if (n <= 0) return;
@@ -324,6 +418,10 @@ int l2kv_oracle_attention(const void* q, const void* K_c, const void* V_c, int d
   });
   return 0;
 }
+
+}  // namespace
+
+extern "C" {
 
 // Attention loss of the norm-based compression against the ideal one (Section 3, Eqs. 5-7),
 // for one query per query head over the cached keys [0, cur_len[b, l]):
@@ -397,6 +495,32 @@ int l2kv_oracle_append_evict(void* K_c, void* V_c, int32_t* idx, double* key_c, 
                              const int32_t* budget, const int32_t* uncompressed, int n_unc,
                              const void* k_new, const void* v_new, const int32_t* pos_new,
                              int key_mode, int per_head) {
+  return append_evict_impl(K_c, V_c, idx, key_c, dtype, B, L, H, dense_rows(H, T_cap), D, cur_len,
+                           budget, uncompressed, n_unc, k_new, v_new, pos_new, key_mode, per_head);
+}
+
+// The same on a packed cache: K_c, V_c [H, total_rows, D], idx / key_c [H, total_rows] with rows
+// (row_off, row_cap); a row that would not fit row_cap[b, l] is the overflow case.
+int l2kv_oracle_append_evict_packed(void* K_c, void* V_c, int32_t* idx, double* key_c, int dtype,
+                                    int B, int L, int H, const int64_t* row_off,
+                                    const int32_t* row_cap, int64_t total_rows, int D,
+                                    int32_t* cur_len, const int32_t* budget,
+                                    const int32_t* uncompressed, int n_unc, const void* k_new,
+                                    const void* v_new, const int32_t* pos_new, int key_mode,
+                                    int per_head) {
+  return append_evict_impl(K_c, V_c, idx, key_c, dtype, B, L, H,
+                           packed_rows(H, row_off, row_cap, total_rows), D, cur_len, budget,
+                           uncompressed, n_unc, k_new, v_new, pos_new, key_mode, per_head);
+}
+
+}  // extern "C"
+
+namespace {
+
+int append_evict_impl(void* K_c, void* V_c, int32_t* idx, double* key_c, int dtype, int B, int L,
+                      int H, Rows rows, int D, int32_t* cur_len, const int32_t* budget,
+                      const int32_t* uncompressed, int n_unc, const void* k_new, const void* v_new,
+                      const int32_t* pos_new, int key_mode, int per_head) {
   // per_head != 0: cur_len and budget are [B, L, H] (caches compressed with a keep count per
   // head); otherwise cur_len is [B, L] and budget [B].
   const size_t row_bytes = size_t(D) * elem_size(dtype);
@@ -410,7 +534,8 @@ int l2kv_oracle_append_evict(void* K_c, void* V_c, int32_t* idx, double* key_c, 
         const int n = per_head ? cur_len[u] : n_shared;
         const int cap = per_head ? budget[u] : budget[b];
         const bool grow = in_list(uncompressed, n_unc, l) || n < cap;
-        if (grow && n >= T_cap) {
+        const int64_t row0 = rows.first(u);
+        if (grow && n >= rows.cap(u)) {
           status = -2;
           continue;
         }
@@ -426,8 +551,8 @@ int l2kv_oracle_append_evict(void* K_c, void* V_c, int32_t* idx, double* key_c, 
           double best = s_new;
           int32_t best_pos = pos_new[b];
           for (int j = 0; j < n; ++j) {
-            const double s = key_c[u * T_cap + j];
-            const int32_t p = idx[u * T_cap + j];
+            const double s = key_c[row0 + j];
+            const int32_t p = idx[row0 + j];
             if (s > best || (s == best && p > best_pos)) {
               best = s;
               best_pos = p;
@@ -436,13 +561,13 @@ int l2kv_oracle_append_evict(void* K_c, void* V_c, int32_t* idx, double* key_c, 
           }
           if (slot < 0) continue;  // the new token is the one discarded
         }
-        const int64_t dst = (u * T_cap + slot) * int64_t(row_bytes);
+        const int64_t dst = (row0 + slot) * int64_t(row_bytes);
         std::memcpy(static_cast<char*>(K_c) + dst,
                     static_cast<const char*>(k_new) + u * int64_t(row_bytes), row_bytes);
         std::memcpy(static_cast<char*>(V_c) + dst,
                     static_cast<const char*>(v_new) + u * int64_t(row_bytes), row_bytes);
-        idx[u * T_cap + slot] = pos_new[b];
-        key_c[u * T_cap + slot] = s_new;
+        idx[row0 + slot] = pos_new[b];
+        key_c[row0 + slot] = s_new;
       }
       if (!per_head && any_grow) cur_len[b * L + l] = n_shared + 1;
     }
@@ -450,4 +575,4 @@ int l2kv_oracle_append_evict(void* K_c, void* V_c, int32_t* idx, double* key_c, 
   return status;
 }
 
-}  // extern "C"
+}  // namespace

@@ -151,6 +151,66 @@ def make_new_kv(w: Workload, step, device):
     return k.to(w.torch_dtype), v.to(w.torch_dtype)
 
 
+def packing(caps):
+    """Row ranges of a packed (unpadded) cache.  caps [B, L]: rows that (b, l) may hold.  The
+    ranges lie back to back in (b, l) order on one row axis shared by all sequences and layers:
+    returns (row_off int64 [B, L], row_cap int32 [B, L], total_rows)."""
+    caps = np.asarray(caps, dtype=np.int64)
+    flat = caps.reshape(-1)
+    off = np.concatenate([[0], np.cumsum(flat)[:-1]]).reshape(caps.shape)
+    return off.astype(np.int64), caps.astype(np.int32), int(flat.sum())
+
+
+def pack_rows(dense, rows, n_rows=None):
+    """Dense [B, L, H, T, ...] (numpy or torch) -> packed [H, total_rows, ...]: the first
+    n_rows[b, l] (default: the capacity) rows of every (b, l) copied to its range."""
+    off, cap, total = rows
+    B, L, H = dense.shape[:3]
+    n_rows = cap if n_rows is None else np.broadcast_to(np.asarray(n_rows), (B, L))
+    if torch.is_tensor(dense):
+        out = torch.zeros((H, total) + tuple(dense.shape[4:]), dtype=dense.dtype, device=dense.device)
+    else:
+        out = np.zeros((H, total) + tuple(dense.shape[4:]), dtype=dense.dtype)
+    for b in range(B):
+        for l in range(L):
+            n = int(n_rows[b, l])
+            out[:, int(off[b, l]):int(off[b, l]) + n] = dense[b, l, :, :n]
+    return out
+
+
+def unpack_rows(packed, rows, B, L, t_cap):
+    """Packed [H, total_rows, ...] -> dense [B, L, H, t_cap, ...] (rows past a range's capacity
+    stay zero)."""
+    off, cap, total = rows
+    H = packed.shape[0]
+    if torch.is_tensor(packed):
+        out = torch.zeros((B, L, H, t_cap) + tuple(packed.shape[2:]), dtype=packed.dtype,
+                          device=packed.device)
+    else:
+        out = np.zeros((B, L, H, t_cap) + tuple(packed.shape[2:]), dtype=packed.dtype)
+    for b in range(B):
+        for l in range(L):
+            n = min(int(cap[b, l]), t_cap)
+            out[b, l, :, :n] = packed[:, int(off[b, l]):int(off[b, l]) + n]
+    return out
+
+
+def make_cache_packed(w: Workload, lens, device):
+    """K, V of a ragged batch without padding: [Hkv, total_rows, D], the rows of (b, l) being the
+    first lens[b] tokens of the slab make_cache would give it.  Returns (K, V, rows)."""
+    rows = packing(np.repeat(np.asarray(lens, dtype=np.int64)[:, None], w.L, axis=1))
+    off, _, total = rows
+    K = torch.zeros((w.Hkv, total, w.D), dtype=w.torch_dtype, device=device)
+    V = torch.zeros_like(K)
+    for b in range(w.B):
+        n = int(lens[b])
+        for l in range(w.L):
+            o = int(off[b, l])
+            K[:, o:o + n] = make_kv_slab(w, "K", b, l, device)[:, :n]
+            V[:, o:o + n] = make_kv_slab(w, "V", b, l, device)[:, :n]
+    return K, V, rows
+
+
 def to_numpy(t):
     """Host copy of a tensor as the oracle wants it: bf16 becomes its uint16 bit pattern."""
     t = t.detach().cpu().contiguous()
