@@ -30,6 +30,19 @@
  *     elements, head_dim 64 or 128; q_heads a multiple of kv_heads with
  *     q_heads / kv_heads in {1, 2, 4, 8}.  Query head j reads KV head
  *     j / (q_heads / kv_heads).
+ *   - Packed caches, for ragged batches without padding (the serving case of Section 4's
+ *     budget-maintained cache: sequences of very different lengths, and compressed layers
+ *     that need far fewer rows than uncompressed ones).  With row_off_dev != NULL the tensor
+ *     is [kv_heads, total_rows, head_dim] (strides stride_h, stride_t; stride_b and stride_l
+ *     are ignored) and the rows of (b, l), for every head, are the row_cap_dev[b, l] rows
+ *     starting at row row_off_dev[b, l] of that shared row axis: row t of (b, l, h) begins at
+ *     element h * stride_h + (row_off_dev[b, l] + t) * stride_t.  Ranges must not overlap and
+ *     must end at or before total_rows (not checked: the arrays live on the device).  t_cap
+ *     is then a host upper bound of row_cap_dev.  Every per-row companion array of such a
+ *     cache (idx, sumsq, the outputs of l2kv_key_norms) is dense [kv_heads, total_rows] with
+ *     the same row axis.  Accepted by l2kv_key_norms, l2kv_select_compact (input, output or
+ *     both), l2kv_decode_attention, l2kv_append_evict and their _per_head / _static forms;
+ *     the prefix-attention and attention-loss calls return L2KV_ERR_UNSUPPORTED for it.
  *   - `len_dev[b]` is the number of valid tokens of sequence b; `max_len` is a host
  *     upper bound on every length the call will meet (it sizes grids and scratch;
  *     device lengths above it are clamped to it).
@@ -82,6 +95,10 @@ typedef struct {
   int32_t dtype;                                     /* l2kv_dtype                          */
   int32_t reserved;
   int64_t stride_b, stride_l, stride_h, stride_t;    /* in elements; stride_t >= head_dim   */
+  /* Packed caches; NULL, NULL, 0 for the dense form described above. */
+  const int64_t* row_off_dev;                        /* DEVICE int64 [batch, layers]        */
+  const int32_t* row_cap_dev;                        /* DEVICE int32 [batch, layers]        */
+  int64_t total_rows;
 } l2kv_layout;
 
 /* Text for a status code (static storage, never NULL). */
@@ -236,6 +253,30 @@ int l2kv_prefix_attention(const void* q, const void* K_c, const void* V_c, const
                           const int32_t* cur_len_dev, int32_t max_len, int32_t n_queries, float scale,
                           float* out, float* lse_out, void* workspace, size_t workspace_bytes,
                           void* stream);
+/* The general form of the three calls above (Eq. 2 per query over the cache, as they state it):
+ * `flags` is any combination of
+ *   L2KV_PREFIX_CAUSAL         the chunk's own rows are the cache's last n_queries rows
+ *                              (l2kv_prefix_attention_causal);
+ *   L2KV_PREFIX_LEN_PER_HEAD   cur_len_dev is [batch, layers, kv_heads]
+ *                              (l2kv_prefix_attention_per_head);
+ *   L2KV_PREFIX_SPLIT_WEIGHTS  every softmax weight multiplies V as the sum of two bf16 terms
+ *                              (16 significant bits) instead of one rounded bf16 (8 bits).  The
+ *                              result then has the accuracy of l2kv_decode_attention (fp32
+ *                              accumulation of exact products; |error| <= 2e-3 + 1e-2 |exact|
+ *                              with a wide margin), at the price of a second P.V contraction.
+ *                              Without the flag single rounded weights are used, as fused
+ *                              attention kernels commonly do; measured |error| then stays below
+ *                              4e-3 + 1e-2 |exact| (it is largest for short caches, where few
+ *                              weights carry the sum).
+ * Any other bit gives L2KV_ERR_INVALID_ARG. */
+#define L2KV_PREFIX_CAUSAL 1u
+#define L2KV_PREFIX_LEN_PER_HEAD 2u
+#define L2KV_PREFIX_SPLIT_WEIGHTS 4u
+int l2kv_prefix_attention_flags(const void* q, const void* K_c, const void* V_c,
+                                const l2kv_layout* lay, const int32_t* cur_len_dev, int32_t max_len,
+                                int32_t n_queries, float scale, uint32_t flags, float* out,
+                                float* lse_out, void* workspace, size_t workspace_bytes,
+                                void* stream);
 
 /* Attention loss of the norm-based compression against the ideal one (Section 3,
  * Eqs. 5-7), for one query per query head over the cached keys i < cur_len_dev[b,l]:

@@ -27,7 +27,9 @@ class _CLayout(ctypes.Structure):
                 ("head_dim", ctypes.c_int32), ("t_cap", ctypes.c_int32),
                 ("dtype", ctypes.c_int32), ("reserved", ctypes.c_int32),
                 ("stride_b", ctypes.c_int64), ("stride_l", ctypes.c_int64),
-                ("stride_h", ctypes.c_int64), ("stride_t", ctypes.c_int64)]
+                ("stride_h", ctypes.c_int64), ("stride_t", ctypes.c_int64),
+                ("row_off_dev", ctypes.c_void_p), ("row_cap_dev", ctypes.c_void_p),
+                ("total_rows", ctypes.c_int64)]
 
 
 def library_path():
@@ -66,13 +68,15 @@ def lib():
         L.l2kv_prefix_attention_per_head.argtypes = L.l2kv_prefix_attention.argtypes
         L.l2kv_prefix_attention_causal.argtypes = L.l2kv_prefix_attention.argtypes
         L.l2kv_prefix_attention_workspace_bytes.argtypes = [lay, i32, i32, ctypes.POINTER(sz)]
+        L.l2kv_prefix_attention_flags.argtypes = [vp, vp, vp, lay, vp, i32, i32, ctypes.c_float,
+                                                  ctypes.c_uint32, vp, vp, vp, sz, vp]
         for name in ("l2kv_prefix_attention", "l2kv_attention_loss_workspace_bytes", "l2kv_attention_loss",
                      "l2kv_keep_count", "l2kv_workspace_bytes", "l2kv_read_device_status",
                      "l2kv_key_norms", "l2kv_select_compact", "l2kv_decode_attention",
                      "l2kv_append_evict", "l2kv_select_compact_per_head",
                      "l2kv_decode_attention_per_head", "l2kv_append_evict_per_head",
                      "l2kv_prefix_attention_per_head", "l2kv_prefix_attention_workspace_bytes",
-                     "l2kv_prefix_attention_causal"):
+                     "l2kv_prefix_attention_causal", "l2kv_prefix_attention_flags"):
             getattr(L, name).restype = ctypes.c_int
         _LIB = L
     return _LIB
@@ -87,17 +91,46 @@ def _check(rc, where):
         raise L2KVError(rc, where)
 
 
-class Layout:
-    """Geometry of a cache tensor [B, L, Hkv, t_cap, D] (D contiguous), taken from a tensor."""
+class Rows:
+    """Row ranges of a packed cache [Hkv, total_rows, D]: the rows of (b, l) are
+    [row_off[b, l], row_off[b, l] + row_cap[b, l]) for every head.  Built from host arrays
+    [B, L]; holds the device copies the library reads."""
 
-    def __init__(self, cache, q_heads=None):
-        if cache.dim() != 5 or cache.stride(4) != 1:
-            raise ValueError("cache must be [B, L, Hkv, t_cap, D] with D contiguous")
+    def __init__(self, row_off, row_cap, total_rows, device):
+        import numpy as np
+        off = np.ascontiguousarray(np.asarray(row_off, dtype=np.int64))
+        cap = np.ascontiguousarray(np.asarray(row_cap, dtype=np.int32))
+        if off.ndim != 2 or off.shape != cap.shape:
+            raise ValueError("row_off and row_cap must both be [B, L]")
+        self.B, self.L = off.shape
+        self.total_rows = int(total_rows)
+        self.t_cap = int(cap.max()) if cap.size else 0
+        self.off = torch.from_numpy(off).to(device)
+        self.cap = torch.from_numpy(cap).to(device)
+
+
+class Layout:
+    """Geometry of a cache tensor, taken from the tensor: dense [B, L, Hkv, t_cap, D], or,
+    with rows (a Rows), packed [Hkv, total_rows, D].  D contiguous."""
+
+    def __init__(self, cache, q_heads=None, rows=None):
         if cache.dtype not in _DTYPE:
             raise ValueError(f"unsupported dtype {cache.dtype}")
+        if rows is not None:
+            if cache.dim() != 3 or cache.stride(2) != 1 or cache.shape[1] != rows.total_rows:
+                raise ValueError("packed cache must be [Hkv, total_rows, D] with D contiguous")
+            H, _, D = cache.shape
+            self.c = _CLayout(rows.B, rows.L, H, H if q_heads is None else q_heads, D, rows.t_cap,
+                              _DTYPE[cache.dtype], 0, 0, 0, cache.stride(0), cache.stride(1),
+                              rows.off.data_ptr(), rows.cap.data_ptr(), rows.total_rows)
+            self.rows = rows                      # keeps the device arrays alive
+            return
+        if cache.dim() != 5 or cache.stride(4) != 1:
+            raise ValueError("cache must be [B, L, Hkv, t_cap, D] with D contiguous")
         B, L, H, T, D = cache.shape
         self.c = _CLayout(B, L, H, H if q_heads is None else q_heads, D, T, _DTYPE[cache.dtype], 0,
-                          cache.stride(0), cache.stride(1), cache.stride(2), cache.stride(3))
+                          cache.stride(0), cache.stride(1), cache.stride(2), cache.stride(3),
+                          None, None, 0)
 
     def ref(self):
         return ctypes.byref(self.c)
@@ -146,16 +179,17 @@ def read_device_status(workspace, stream=None):
     return out.value
 
 
-def key_norms(K, len_dev, max_len, sumsq_out, norm_out=None, stream=None):
-    lay = Layout(K)
+def key_norms(K, len_dev, max_len, sumsq_out, norm_out=None, stream=None, rows=None):
+    lay = Layout(K, rows=rows)
     _check(lib().l2kv_key_norms(_ptr(K), lay.ref(), _ptr(len_dev), int(max_len), _ptr(sumsq_out),
                                 _ptr(norm_out), _stream(stream)), "l2kv_key_norms")
 
 
 def select_compact(K, V, len_dev, keep_dev, max_len, uncompressed_layers, K_out, V_out, idx_out,
                    sumsq_out, kept_len_dev, workspace, policy=KEEP_LOWEST_NORM, seed=0,
-                   sumsq_in=None, stream=None):
-    lin, lout = Layout(K), Layout(K_out)
+                   sumsq_in=None, stream=None, rows_in=None, rows_out=None):
+    """rows_in / rows_out (Rows): the input / output cache is packed [Hkv, total_rows, D]."""
+    lin, lout = Layout(K, rows=rows_in), Layout(K_out, rows=rows_out)
     arr, n = _layers(uncompressed_layers)
     _check(lib().l2kv_select_compact(
         _ptr(K), _ptr(V), lin.ref(), _ptr(len_dev), _ptr(keep_dev), int(max_len), arr, n,
@@ -189,16 +223,17 @@ def decode_attention_per_head(q, K_c, V_c, cur_len_unit_dev, max_len, out, works
         "l2kv_decode_attention_per_head")
 
 
-def decode_attention(q, K_c, V_c, cur_len_dev, max_len, out, workspace, scale=0.0, stream=None):
-    lay = Layout(K_c, q_heads=q.shape[2])
+def decode_attention(q, K_c, V_c, cur_len_dev, max_len, out, workspace, scale=0.0, stream=None,
+                     rows=None):
+    lay = Layout(K_c, q_heads=q.shape[2], rows=rows)
     _check(lib().l2kv_decode_attention(
         _ptr(q), _ptr(K_c), _ptr(V_c), lay.ref(), _ptr(cur_len_dev), int(max_len), float(scale),
         _ptr(out), _ptr(workspace), workspace.numel(), _stream(stream)), "l2kv_decode_attention")
 
 
 def append_evict(K_c, V_c, idx, sumsq_c, cur_len_dev, budget_dev, uncompressed_layers, k_new, v_new,
-                 pos_new_dev, workspace, stream=None):
-    lay = Layout(K_c)
+                 pos_new_dev, workspace, stream=None, rows=None):
+    lay = Layout(K_c, rows=rows)
     arr, n = _layers(uncompressed_layers)
     _check(lib().l2kv_append_evict(
         _ptr(K_c), _ptr(V_c), _ptr(idx), _ptr(sumsq_c), lay.ref(), _ptr(cur_len_dev),
@@ -217,7 +252,8 @@ def append_evict_per_head(K_c, V_c, idx, sumsq_c, cur_len_unit_dev, budget_unit_
         _ptr(workspace), workspace.numel(), _stream(stream)), "l2kv_append_evict_per_head")
 
 
-def decode_attention_static(q, K_c, V_c, cur_len_dev, max_len, out, scale=0.0, stream=None):
+def decode_attention_static(q, K_c, V_c, cur_len_dev, max_len, out, scale=0.0, stream=None,
+                            rows=None):
     """decode_attention for callers that cannot allocate: no workspace argument.  The partial
     results go to a fixed 16 MiB array inside the library (problems that need more raise
     L2KVError with status -4).  Calls share that array, so do not let two of them overlap on
@@ -226,7 +262,7 @@ def decode_attention_static(q, K_c, V_c, cur_len_dev, max_len, out, scale=0.0, s
     vp = ctypes.c_void_p
     fn.restype = ctypes.c_int
     fn.argtypes = [vp, vp, vp, ctypes.POINTER(_CLayout), vp, ctypes.c_int32, ctypes.c_float, vp, vp]
-    lay = Layout(K_c, q_heads=q.shape[2])
+    lay = Layout(K_c, q_heads=q.shape[2], rows=rows)
     _check(fn(_ptr(q), _ptr(K_c), _ptr(V_c), lay.ref(), _ptr(cur_len_dev), int(max_len),
               float(scale), _ptr(out), _stream(stream)), "l2kv_decode_attention_static")
 
@@ -256,6 +292,22 @@ def prefix_attention_workspace(K_c, q, max_len, device=None):
                                                        ctypes.byref(need)),
            "l2kv_prefix_attention_workspace_bytes")
     return torch.zeros(need.value, dtype=torch.uint8, device=device or K_c.device)
+
+
+PREFIX_CAUSAL, PREFIX_LEN_PER_HEAD, PREFIX_SPLIT_WEIGHTS = 1, 2, 4
+
+
+def prefix_attention_flags(q, K_c, V_c, cur_len_dev, max_len, out, flags, lse_out=None, scale=0.0,
+                           workspace=None, stream=None):
+    """The general prefix-attention call: flags is a combination of PREFIX_CAUSAL,
+    PREFIX_LEN_PER_HEAD and PREFIX_SPLIT_WEIGHTS (weights as two bf16 terms: the accuracy of
+    decode attention for a second P.V contraction)."""
+    lay = Layout(K_c, q_heads=q.shape[3])
+    _check(lib().l2kv_prefix_attention_flags(
+        _ptr(q), _ptr(K_c), _ptr(V_c), lay.ref(), _ptr(cur_len_dev), int(max_len), int(q.shape[2]),
+        float(scale), int(flags), _ptr(out), _ptr(lse_out), _ptr(workspace),
+        0 if workspace is None else workspace.numel(), _stream(stream)),
+        "l2kv_prefix_attention_flags")
 
 
 def prefix_attention(q, K_c, V_c, cur_len_dev, max_len, out, lse_out=None, scale=0.0, workspace=None,

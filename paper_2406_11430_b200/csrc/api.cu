@@ -19,13 +19,25 @@ int check_layout(const l2kv_layout* a) {
   if (a->dtype != L2KV_F32 && a->dtype != L2KV_BF16) return L2KV_ERR_UNSUPPORTED;
   if (a->head_dim != 64 && a->head_dim != 128) return L2KV_ERR_UNSUPPORTED;
   if (a->layers > kMaxLayers) return L2KV_ERR_OUT_OF_RANGE;
+  const int64_t per16 = 16 / elem_bytes(a->dtype);
+  if (a->row_off_dev) {
+    // packed cache [kv_heads, total_rows, head_dim]: stride_b and stride_l are not used
+    if (!a->row_cap_dev || a->total_rows < 0) return L2KV_ERR_INVALID_ARG;
+    if (a->stride_t < a->head_dim || a->stride_h < 0) return L2KV_ERR_INVALID_ARG;
+    if (a->stride_h % per16 || a->stride_t % per16) return L2KV_ERR_MISALIGNED;
+    if ((reinterpret_cast<uintptr_t>(a->row_off_dev) & 7u) || (reinterpret_cast<uintptr_t>(a->row_cap_dev) & 3u))
+      return L2KV_ERR_MISALIGNED;
+    return L2KV_OK;
+  }
+  if (a->row_cap_dev) return L2KV_ERR_INVALID_ARG;
   if (a->stride_t < a->head_dim || a->stride_b < 0 || a->stride_l < 0 || a->stride_h < 0)
     return L2KV_ERR_INVALID_ARG;
-  const int64_t per16 = 16 / elem_bytes(a->dtype);
   if (a->stride_b % per16 || a->stride_l % per16 || a->stride_h % per16 || a->stride_t % per16)
     return L2KV_ERR_MISALIGNED;
   return L2KV_OK;
 }
+
+bool packed(const l2kv_layout* a) { return a->row_off_dev != nullptr; }
 
 int check_groups(const l2kv_layout* a) {
   if (a->kv_heads == 0) return a->q_heads == 0 ? L2KV_OK : L2KV_ERR_INVALID_ARG;
@@ -103,7 +115,8 @@ int l2kv_key_norms(const void* K, const l2kv_layout* lay, const int32_t* len_dev
   if (empty(lay) || max_len == 0) return L2KV_OK;
   if (!K || !len_dev || !sumsq_out) return L2KV_ERR_INVALID_ARG;
   if (!aligned16(K)) return L2KV_ERR_MISALIGNED;
-  return launch_key_norms(K, make_geom(*lay), lay->dtype, len_dev, max_len, sumsq_out, lay->t_cap,
+  // leading dimension -1: the outputs are laid out like the cache's rows
+  return launch_key_norms(K, make_geom(*lay), lay->dtype, len_dev, max_len, sumsq_out, -1,
                           norm_out, kKeysOnly, nullptr, static_cast<cudaStream_t>(stream));
 }
 
@@ -264,7 +277,7 @@ int l2kv_append_evict_per_head(void* K_c, void* V_c, int32_t* idx, float* sumsq_
                            workspace, workspace_bytes, stream);
 }
 
-static int prefix_attention_impl(bool per_head, bool causal, const void* q, const void* K_c, const void* V_c,
+static int prefix_attention_impl(bool per_head, bool causal, bool split_weights, const void* q, const void* K_c, const void* V_c,
                                  const l2kv_layout* lay, const int32_t* cur_len_dev,
                                  int32_t max_len, int32_t n_queries, float scale, float* out,
                                  float* lse_out, void* workspace, size_t workspace_bytes,
@@ -273,7 +286,7 @@ static int prefix_attention_impl(bool per_head, bool causal, const void* q, cons
   if (rc != L2KV_OK) return rc;
   rc = check_groups(lay);
   if (rc != L2KV_OK) return rc;
-  if (lay->dtype != L2KV_BF16 || lay->head_dim != 128) return L2KV_ERR_UNSUPPORTED;
+  if (lay->dtype != L2KV_BF16 || lay->head_dim != 128 || packed(lay)) return L2KV_ERR_UNSUPPORTED;
   if (max_len < 0 || n_queries < 0 || !(scale == scale)) return L2KV_ERR_INVALID_ARG;
   if (max_len > lay->t_cap) return L2KV_ERR_OUT_OF_RANGE;
   if (empty(lay) || n_queries == 0) return L2KV_OK;
@@ -292,7 +305,7 @@ static int prefix_attention_impl(bool per_head, bool causal, const void* q, cons
   }
   return launch_prefix_attention(q, K_c, V_c, make_geom(*lay), lay->dtype, n_queries, lens,
                                  max_len, sc, out, lse_out, static_cast<int32_t*>(workspace),
-                                 scratch, scratch_bytes, causal ? 1 : 0,
+                                 scratch, scratch_bytes, causal ? 1 : 0, split_weights ? 1 : 0,
                                  static_cast<cudaStream_t>(stream));
 }
 
@@ -301,7 +314,7 @@ int l2kv_prefix_attention_causal(const void* q, const void* K_c, const void* V_c
                                  int32_t max_len, int32_t n_queries, float scale, float* out,
                                  float* lse_out, void* workspace, size_t workspace_bytes,
                                  void* stream) {
-  return prefix_attention_impl(false, true, q, K_c, V_c, lay, cur_len_dev, max_len, n_queries, scale,
+  return prefix_attention_impl(false, true, false, q, K_c, V_c, lay, cur_len_dev, max_len, n_queries, scale,
                                out, lse_out, workspace, workspace_bytes, stream);
 }
 
@@ -315,7 +328,8 @@ int l2kv_prefix_attention_workspace_bytes(const l2kv_layout* lay, int32_t max_le
   if (max_len < 0 || n_queries < 0) return L2KV_ERR_INVALID_ARG;
   if (max_len > lay->t_cap) return L2KV_ERR_OUT_OF_RANGE;
   *bytes = (size_t)kStatusBytes;
-  if (empty(lay) || n_queries == 0 || lay->dtype != L2KV_BF16 || lay->head_dim != 128) return L2KV_OK;
+  if (empty(lay) || n_queries == 0 || lay->dtype != L2KV_BF16 || lay->head_dim != 128 || packed(lay))
+    return L2KV_OK;
   *bytes += prefix_attention_scratch(make_geom(*lay), n_queries, max_len);
   return L2KV_OK;
 }
@@ -324,7 +338,7 @@ int l2kv_prefix_attention(const void* q, const void* K_c, const void* V_c, const
                           const int32_t* cur_len_dev, int32_t max_len, int32_t n_queries, float scale,
                           float* out, float* lse_out, void* workspace, size_t workspace_bytes,
                           void* stream) {
-  return prefix_attention_impl(false, false, q, K_c, V_c, lay, cur_len_dev, max_len, n_queries, scale, out,
+  return prefix_attention_impl(false, false, false, q, K_c, V_c, lay, cur_len_dev, max_len, n_queries, scale, out,
                                lse_out, workspace, workspace_bytes, stream);
 }
 
@@ -333,8 +347,21 @@ int l2kv_prefix_attention_per_head(const void* q, const void* K_c, const void* V
                                    int32_t max_len, int32_t n_queries, float scale, float* out,
                                    float* lse_out, void* workspace, size_t workspace_bytes,
                                    void* stream) {
-  return prefix_attention_impl(true, false, q, K_c, V_c, lay, cur_len_unit_dev, max_len, n_queries, scale,
+  return prefix_attention_impl(true, false, false, q, K_c, V_c, lay, cur_len_unit_dev, max_len, n_queries, scale,
                                out, lse_out, workspace, workspace_bytes, stream);
+}
+
+int l2kv_prefix_attention_flags(const void* q, const void* K_c, const void* V_c,
+                                const l2kv_layout* lay, const int32_t* cur_len_dev, int32_t max_len,
+                                int32_t n_queries, float scale, uint32_t flags, float* out,
+                                float* lse_out, void* workspace, size_t workspace_bytes,
+                                void* stream) {
+  if (flags & ~(uint32_t)(L2KV_PREFIX_CAUSAL | L2KV_PREFIX_LEN_PER_HEAD | L2KV_PREFIX_SPLIT_WEIGHTS))
+    return L2KV_ERR_INVALID_ARG;
+  return prefix_attention_impl((flags & L2KV_PREFIX_LEN_PER_HEAD) != 0, (flags & L2KV_PREFIX_CAUSAL) != 0,
+                               (flags & L2KV_PREFIX_SPLIT_WEIGHTS) != 0, q, K_c, V_c, lay, cur_len_dev,
+                               max_len, n_queries, scale, out, lse_out, workspace, workspace_bytes,
+                               stream);
 }
 
 int l2kv_attention_loss_workspace_bytes(const l2kv_layout* lay, int32_t max_len, size_t* bytes) {
@@ -351,6 +378,7 @@ int l2kv_attention_loss(const void* q, const void* K, const l2kv_layout* lay,
                         void* workspace, size_t workspace_bytes, void* stream) {
   int rc = check_layout(lay);
   if (rc != L2KV_OK) return rc;
+  if (packed(lay)) return L2KV_ERR_UNSUPPORTED;
   if (lay->kv_heads > 0 && lay->q_heads % lay->kv_heads) return L2KV_ERR_INVALID_ARG;
   if (max_len < 0 || !(scale == scale)) return L2KV_ERR_INVALID_ARG;
   if (max_len > lay->t_cap) return L2KV_ERR_OUT_OF_RANGE;

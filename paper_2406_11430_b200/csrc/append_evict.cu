@@ -35,9 +35,11 @@ append_evict_kernel(T* __restrict__ K, T* __restrict__ V, int32_t* __restrict__ 
   const int b = (int)(bl / g.L);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   // per_head: a length and a budget of its own for every (b, l, h)
-  const int n = max(0, min(cur_len_dev[per_head ? unit : bl], g.t_cap));
+  const int cap = g.cap(bl);
+  const long long meta0 = g.meta(unit);
+  const int n = max(0, min(cur_len_dev[per_head ? unit : bl], cap));
   const bool grow = unc.test(l) || n < budget_dev[per_head ? unit : (long long)b];
-  const bool overflow = grow && n >= g.t_cap;
+  const bool overflow = grow && n >= cap;
   const int pos_new = pos_new_dev[b];
 
   if (!overflow) {
@@ -54,8 +56,8 @@ append_evict_kernel(T* __restrict__ K, T* __restrict__ V, int32_t* __restrict__ 
     }
     int slot = n;
     if (!grow) {
-      const float* key = sumsq + unit * g.t_cap;
-      const int32_t* pos = idx + unit * g.t_cap;
+      const float* key = sumsq + meta0;
+      const int32_t* pos = idx + meta0;
       unsigned long long best = 0ull;
       int best_j = -1;
       auto consider = [&](uint32_t kb, uint32_t pb, int j) {
@@ -124,12 +126,12 @@ append_evict_kernel(T* __restrict__ K, T* __restrict__ V, int32_t* __restrict__ 
       }
     }
     if (warp == 0 && slot >= 0 && lane < LPR) {
-      const long long row = b * g.sb + l * g.sl + h * g.sh + (long long)slot * g.st + lane * EPV;
+      const long long row = g.base(b, l, h) + (long long)slot * g.st + lane * EPV;
       *reinterpret_cast<uint4*>(K + row) = vk;
       *reinterpret_cast<uint4*>(V + row) = vv;
       if (lane == 0) {
-        idx[unit * g.t_cap + slot] = pos_new;
-        sumsq[unit * g.t_cap + slot] = s_new;
+        idx[meta0 + slot] = pos_new;
+        sumsq[meta0 + slot] = s_new;
       }
     }
   }

@@ -56,11 +56,17 @@ inline bool make_cache_map(CUtensorMap* map, const void* base, const Geom& g, in
     return reinterpret_cast<EncodeFn>(fn);
   }();
   if (!encode) return false;
-  if (g.st <= 0 || g.sh <= 0 || g.sl <= 0 || g.sb <= 0) return false;   // broadcast views
-  const cuuint64_t dims[5] = {128, (cuuint64_t)g.t_cap, (cuuint64_t)g.H, (cuuint64_t)g.L,
-                              (cuuint64_t)g.B};
-  const cuuint64_t strides[4] = {(cuuint64_t)g.st * 2, (cuuint64_t)g.sh * 2, (cuuint64_t)g.sl * 2,
-                                 (cuuint64_t)g.sb * 2};
+  cuuint64_t dims[5] = {128, (cuuint64_t)g.t_cap, (cuuint64_t)g.H, (cuuint64_t)g.L, (cuuint64_t)g.B};
+  cuuint64_t strides[4] = {(cuuint64_t)g.st * 2, (cuuint64_t)g.sh * 2, (cuuint64_t)g.sl * 2,
+                           (cuuint64_t)g.sb * 2};
+  if (g.row_off) {
+    // packed cache: one [H, total_rows, 128] plane; the two outer dimensions have extent 1
+    if (g.st <= 0 || g.sh <= 0 || g.total_rows <= 0 || g.total_rows > 0x7fffffffLL) return false;
+    dims[1] = (cuuint64_t)g.total_rows; dims[3] = 1; dims[4] = 1;
+    strides[2] = strides[1]; strides[3] = strides[1];
+  } else if (g.st <= 0 || g.sh <= 0 || g.sl <= 0 || g.sb <= 0) {
+    return false;                                                       // broadcast views
+  }
   const cuuint32_t box[5] = {64, (cuuint32_t)box_rows, 1, 1, 1};
   const cuuint32_t elem[5] = {1, 1, 1, 1, 1};
   return encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(base), dims, strides,

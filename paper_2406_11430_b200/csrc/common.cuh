@@ -20,10 +20,28 @@ constexpr int kMaxChunks = 4096;       // kGatherChunk * kMaxChunks tokens per u
 #endif
 constexpr int kDecodeChunk = L2KV_DECODE_CHUNK;   // cached tokens per split of decode attention
 
-// Cache geometry handed to kernels by value (strides in elements).
+// Cache geometry handed to kernels by value (strides in elements).  Dense caches are
+// [B, L, H, t_cap, D]; packed caches (row_off != null) are [H, total_rows, D] with the rows of
+// (b, l) at [row_off[b * L + l], + row_cap[b * L + l]) of the shared row axis, for every head.
+// The per-row index map and keys follow the cache: [B, L, H, t_cap] or [H, total_rows].
 struct Geom {
   int B, L, H, Hq, D, t_cap;
   long long sb, sl, sh, st;
+  const long long* row_off;
+  const int32_t* row_cap;
+  long long total_rows;
+  // element offset of row 0 of unit (b, l, h)
+  __device__ __forceinline__ long long base(int b, int l, int h) const {
+    return row_off ? h * sh + row_off[(long long)b * L + l] * st : b * sb + l * sl + h * sh;
+  }
+  // rows that (b, l) may hold
+  __device__ __forceinline__ int cap(long long bl) const { return row_off ? row_cap[bl] : t_cap; }
+  // first entry of unit = (b * L + l) * H + h in the index map / key arrays
+  __device__ __forceinline__ long long meta(long long unit) const {
+    return row_off ? (unit % H) * total_rows + row_off[unit / H] : unit * (long long)t_cap;
+  }
+  // first row of (b, l) on the row axis of a packed cache (0 for dense ones)
+  __device__ __forceinline__ long long row0(long long bl) const { return row_off ? row_off[bl] : 0; }
 };
 
 // Result of the selection for one (b, l, h) unit, consumed by the gather kernel.
@@ -51,6 +69,9 @@ inline Geom make_geom(const l2kv_layout& a) {
   g.B = a.batch; g.L = a.layers; g.H = a.kv_heads; g.Hq = a.q_heads; g.D = a.head_dim;
   g.t_cap = a.t_cap;
   g.sb = a.stride_b; g.sl = a.stride_l; g.sh = a.stride_h; g.st = a.stride_t;
+  g.row_off = reinterpret_cast<const long long*>(a.row_off_dev);
+  g.row_cap = a.row_cap_dev;
+  g.total_rows = a.total_rows;
   return g;
 }
 
@@ -200,6 +221,7 @@ struct SelectArgs {
   const int32_t* keep_unit_dev;               // [B, L, H] or null
   int32_t* kept_len_unit_dev;                 // [B, L, H] or null
   int out_t_cap, policy, n_chunks;            // policy: how key bits order (lowest / highest)
+  const int32_t* out_row_cap;                 // packed output: rows per (b, l), else null
   unsigned long long seed;                    // kKeysRandom
   LayerMask unc;
   UnitRec* unit_rec;
@@ -229,7 +251,7 @@ int launch_append_evict(void* K, void* V, int32_t* idx, float* sumsq, const Geom
 int launch_prefix_attention(const void* q, const void* K, const void* V, const Geom& g, int dtype,
                             int n_queries, const LenView& cur_len_dev, int max_len, float scale,
                             float* out, float* lse_out, int32_t* status_word, float* scratch,
-                            size_t scratch_bytes, int causal, cudaStream_t s);
+                            size_t scratch_bytes, int causal, int split_weights, cudaStream_t s);
 size_t prefix_attention_scratch(const Geom& g, int n_queries, int max_len);
 size_t attention_loss_workspace(const l2kv_layout& a, int max_len);
 int launch_attention_loss(const void* q, const void* K, const Geom& g, int dtype,

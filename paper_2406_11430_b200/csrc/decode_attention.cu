@@ -42,7 +42,7 @@ decode_split_kernel(const T* __restrict__ q, const T* __restrict__ K, const T* _
   const long long bl = unit / g.H;
   const int l = (int)(bl % g.L);
   const int b = (int)(bl / g.L);
-  const int n = max(0, min(cur_len_dev.at(bl, h, g.H), min(max_len, g.t_cap)));
+  const int n = max(0, min(cur_len_dev.at(bl, h, g.H), min(max_len, g.cap(bl))));
   const int t0 = split * kDecodeChunk;
   if (t0 >= n) return;
   const int t_end = min(n, t0 + kDecodeChunk);
@@ -50,7 +50,7 @@ decode_split_kernel(const T* __restrict__ q, const T* __restrict__ K, const T* _
 
   const int tid = threadIdx.x, piece = tid % LPR, sub = tid / LPR;
   const int warp = tid >> 5, lane = tid & 31;
-  const long long kv_base = b * g.sb + l * g.sl + h * g.sh + (long long)piece * EPV;
+  const long long kv_base = g.base(b, l, h) + (long long)piece * EPV;
 
   // ---- phase 1: scores ------------------------------------------------------------
   float qf[G][EPV];
@@ -199,12 +199,12 @@ decode_split_kernel(const T* __restrict__ q, const T* __restrict__ K, const T* _
 template <int D>
 __global__ void __launch_bounds__(D)
 decode_combine_kernel(const float* __restrict__ partial, LenView cur_len_dev,
-                      int max_len, int t_cap, int H, int Hq, int n_splits,
-                      float* __restrict__ out) {
+                      int max_len, Geom g, int n_splits, float* __restrict__ out) {
+  const int H = g.H, Hq = g.Hq;
   const long long row = blockIdx.x;                      // (b * L + l) * Hq + hq
   const long long bl = row / Hq;
   const int h = (int)(row % Hq) / (Hq / H);
-  const int n = max(0, min(cur_len_dev.at(bl, h, H), min(max_len, t_cap)));
+  const int n = max(0, min(cur_len_dev.at(bl, h, H), min(max_len, g.cap(bl))));
   const int ns = (n + kDecodeChunk - 1) / kDecodeChunk;
   const int d = threadIdx.x;
   const float* p = partial + row * n_splits * (long long)(D + 2);
@@ -337,7 +337,7 @@ decode_split_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16
   const long long bl = unit / g.H;
   const int l = (int)(bl % g.L);
   const int b = (int)(bl / g.L);
-  const int n = max(0, min(cur_len_dev.at(bl, h, g.H), min(max_len, g.t_cap)));
+  const int n = max(0, min(cur_len_dev.at(bl, h, g.H), min(max_len, g.cap(bl))));
   const int t0 = split * kDecodeChunk;
   if (t0 >= n) return;
   if constexpr (TMA) {
@@ -351,8 +351,12 @@ decode_split_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int fr = lane >> 2, fc = lane & 3;               // fragment row / column-pair indices
-  const __nv_bfloat16* Kb = K + b * g.sb + l * g.sl + h * g.sh + (long long)t0 * g.st;
-  const __nv_bfloat16* Vb = V + b * g.sb + l * g.sl + h * g.sh + (long long)t0 * g.st;
+  const __nv_bfloat16* Kb = K + g.base(b, l, h) + (long long)t0 * g.st;
+  const __nv_bfloat16* Vb = V + g.base(b, l, h) + (long long)t0 * g.st;
+  // Tensor-map coordinates of this unit: (token, head, layer, batch) for a dense cache; a packed
+  // cache is one [H, total_rows] plane, so the unit's first row joins the token coordinate.
+  [[maybe_unused]] const int tm_row = (int)g.row0(bl) + t0;
+  [[maybe_unused]] const int tm_l = g.row_off ? 0 : l, tm_b = g.row_off ? 0 : b;
   const uint32_t stage0 = smem_u32(s_stage);
 
   // Copy plan of this thread, fixed for the whole kernel: it moves the 16-byte piece c_ch of
@@ -377,8 +381,8 @@ decode_split_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16
         const uint32_t dst = stage0 + (s % kStages) * kStageBytes;
         const CUtensorMap* map = s < n_st ? &map_k : &map_v;
         mbar_expect_tx(bar, kStageBytes);
-        tma_load_5d(dst, map, bar, 0, t0 + st * kStageTok, h, l, b);
-        tma_load_5d(dst + kStageTok * 128, map, bar, 64, t0 + st * kStageTok, h, l, b);
+        tma_load_5d(dst, map, bar, 0, tm_row + st * kStageTok, h, tm_l, tm_b);
+        tma_load_5d(dst + kStageTok * 128, map, bar, 64, tm_row + st * kStageTok, h, tm_l, tm_b);
       }
     } else {
       const char* src = (s < n_st ? c_k : c_v) + (long long)st * kStageTok * row_bytes;
@@ -624,7 +628,7 @@ static int launch_dec_mma(const void* q, const void* K, const void* V, const Geo
     if (cudaGetLastError() != cudaSuccess) return L2KV_ERR_CUDA;
   }
   decode_combine_kernel<128><<<(unsigned)((long long)g.B * g.L * g.Hq), 128, 0, s>>>(
-      partial, cur_len_dev, max_len, g.t_cap, g.H, g.Hq, plan.n_splits, out);
+      partial, cur_len_dev, max_len, g, plan.n_splits, out);
   return cudaGetLastError() == cudaSuccess ? L2KV_OK : L2KV_ERR_CUDA;
 }
 
@@ -643,7 +647,7 @@ static int launch_dec_t(const void* q, const void* K, const void* V, const Geom&
     if (cudaGetLastError() != cudaSuccess) return L2KV_ERR_CUDA;
   }
   decode_combine_kernel<D><<<(unsigned)((long long)g.B * g.L * g.Hq), D, 0, s>>>(
-      partial, cur_len_dev, max_len, g.t_cap, g.H, g.Hq, plan.n_splits, out);
+      partial, cur_len_dev, max_len, g, plan.n_splits, out);
   return cudaGetLastError() == cudaSuccess ? L2KV_OK : L2KV_ERR_CUDA;
 }
 

@@ -45,14 +45,16 @@ key_norms_kernel(const T* __restrict__ K, Geom g, const int32_t* __restrict__ le
   const int l = (int)((unit / g.H) % g.L);
   const int b = (int)(unit / ((long long)g.H * g.L));
   const int tid = threadIdx.x;
-  const int len = max(0, min(len_dev[b], min(max_len, g.t_cap)));
+  const long long bl = (long long)b * g.L + l;
+  const int len = max(0, min(len_dev[b], min(max_len, g.cap(bl))));
+  [[maybe_unused]] const int out_cap = SEL ? (sel.out_row_cap ? sel.out_row_cap[bl] : sel.out_t_cap) : 0;
 
   if constexpr (SEL) {
     // Units that need no keys: copied layers and empty sequences get their record here.
     const bool whole = sel.unc.test(l);
     if (whole || len == 0) {
       if (chunk == 0) {
-        const int keep = min(len, sel.out_t_cap);
+        const int keep = min(len, out_cap);
         identity_unit<kNormThreads>(len, keep, true, sel.unit_rec + unit,
                                     sel.chunk_rec + unit * sel.n_chunks);
         if (tid == 0) publish_kept_len(sel, unit, b * g.L + l, h, keep);
@@ -60,7 +62,7 @@ key_norms_kernel(const T* __restrict__ K, Geom g, const int32_t* __restrict__ le
       return;
     }
   }
-  float* out = sumsq + unit * ld;
+  float* out = sumsq + (ld >= 0 ? unit * ld : g.meta(unit));   // ld < 0: laid out like the cache
   if constexpr (MODE != kKeysGiven) {
     const int row0 = chunk * kNormRowsPerCta;
     if (row0 >= len) return;
@@ -72,8 +74,8 @@ key_norms_kernel(const T* __restrict__ K, Geom g, const int32_t* __restrict__ le
     } else {
       const int piece = tid % LPR;
       const int sub = tid / LPR;
-      const T* base = K + b * g.sb + l * g.sl + h * g.sh + (long long)piece * Elem<T>::kPerVec;
-      float* nout = norm_out ? norm_out + unit * ld : nullptr;
+      const T* base = K + g.base(b, l, h) + (long long)piece * Elem<T>::kPerVec;
+      float* nout = norm_out ? norm_out + (ld >= 0 ? unit * ld : g.meta(unit)) : nullptr;
       const int my_row = piece / (LPR / U);              // which of its U rows this lane reports
       const bool writer = (piece % (LPR / U)) == 0;
 
@@ -122,7 +124,7 @@ key_norms_kernel(const T* __restrict__ K, Geom g, const int32_t* __restrict__ le
     }
     const int keep_arg = sel.keep_unit_dev ? sel.keep_unit_dev[unit] : sel.keep_dev[b];
     const int keep_req = max(0, min(keep_arg, len));
-    const int keep = min(keep_req, sel.out_t_cap);       // rows that fit the output; the rest is cut
+    const int keep = min(keep_req, out_cap);             // rows that fit the output; the rest is cut
     if (tid == 0) publish_kept_len(sel, unit, b * g.L + l, h, keep);
     if (keep_req == len) {
       identity_unit<kNormThreads>(len, keep, MODE == kKeysRandom, sel.unit_rec + unit,

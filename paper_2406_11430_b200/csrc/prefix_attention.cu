@@ -127,6 +127,12 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<const uint32_t*>(&v);
 }
 
+// The part of a weight pair that its bf16 rounding `packed` left out, again as a bf16 pair:
+// hi + lo carries 16 significant bits of each weight.
+__device__ __forceinline__ uint32_t pack_bf16_rest(float lo, float hi, uint32_t packed) {
+  return pack_bf16(lo - __uint_as_float(packed << 16), hi - __uint_as_float(packed & 0xffff0000u));
+}
+
 // 2^x by the hardware approximation (one MUFU instruction; x <= 0 here, -inf gives 0).
 __device__ __forceinline__ float fast_exp2(float x) {
   float y;
@@ -160,7 +166,7 @@ __device__ __forceinline__ void tmem_scale8(uint32_t taddr, float factor) {
 // contraction of the current one run.
 constexpr float kPfRescaleGap = 8.f;            // log2 units a maximum may drift before O is rescaled
 
-template <int G>
+template <int G, bool SW>
 __global__ void __launch_bounds__(kPfThreads, 2)
 prefix_attention_basic_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n_queries,
                            LenView cur_len_dev, int max_len, float scale_log2e,
@@ -326,6 +332,7 @@ prefix_attention_basic_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n
     // ---- weights 2^(s - m_ref) as bf16 pairs over the score columns -------------------------
     {
       uint32_t pk[32];
+      [[maybe_unused]] uint32_t pr[SW ? 32 : 1];
       float rowsum0 = 0.f, rowsum1 = 0.f;
       const float neg_m = m_ref == -INFINITY ? 0.f : -m_ref;   // a row with nothing to see yet
 #pragma unroll
@@ -335,8 +342,10 @@ prefix_attention_basic_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n
         rowsum0 += p0;
         rowsum1 += p1;
         pk[i >> 1] = pack_bf16(p0, p1);
+        if constexpr (SW) pr[i >> 1] = pack_bf16_rest(p0, p1, pk[i >> 1]);
       }
       tmem_st32(t_p, pk);
+      if constexpr (SW) tmem_st32(t_p + 64, pr);          // second terms: columns 64..127
       tmem_wait_st();
       l_run += rowsum0 + rowsum1;
     }
@@ -358,9 +367,12 @@ prefix_attention_basic_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n
       if (valid_all == kPfRows && !mbar_wait<kPfPolls>(bar_v, kb & 1)) s_fail = 1;
       tc_fence_after();
 #pragma unroll
-      for (int k = 0; k < 8; ++k)
+      for (int k = 0; k < 8; ++k) {
         umma_bf16_ts(tmem + 128, tmem + k * 8, umma_desc(sV + k * 2048, kPfHalf, 1024), kIdescPV,
                      (kb > 0 || k > 0) ? 1u : 0u);
+        if constexpr (SW)
+          umma_bf16_ts(tmem + 128, tmem + 64 + k * 8, umma_desc(sV + k * 2048, kPfHalf, 1024), kIdescPV, 1u);
+      }
       umma_commit(bar_o);
     }
   }
@@ -441,7 +453,7 @@ __device__ __forceinline__ bool mbar_wait_likely(uint32_t bar, uint32_t parity) 
 // ready: one arrival per softmax warp); every wait on them is bounded.
 constexpr int kPfPipeThreads = 2 * kPfRows + 4 * 32;      // softmax A, softmax B, issuer A, issuer B, K, V
 
-template <int G>
+template <int G, bool SW>
 __global__ void __launch_bounds__(kPfPipeThreads, 1)
 prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n_queries,
                            LenView cur_len_dev, int max_len, float scale_log2e,
@@ -597,9 +609,13 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
         tc_fence_after();
         const uint32_t vt = sV + (j % NS) * kPfSubTile;
 #pragma unroll
-        for (int k = 0; k < 4; ++k)                     // O += P(j) V(j); slice k = tokens 16k .. 16k + 15
+        for (int k = 0; k < 4; ++k) {                   // O += P(j) V(j); slice k = tokens 16k .. 16k + 15
           umma_bf16_ts(tmem + 128, tmem + s * 64 + k * 8,
                        umma_desc(vt + k * 2048, kPfSubHalf, 1024), kIdescPV, (j > 0 || k > 0) ? 1u : 0u);
+          if constexpr (SW)                             // the weights' second terms: columns 32..63
+            umma_bf16_ts(tmem + 128, tmem + s * 64 + 32 + k * 8,
+                         umma_desc(vt + k * 2048, kPfSubHalf, 1024), kIdescPV, 1u);
+        }
         umma_commit(bar_o);
         umma_commit(bar_vfree(j % NS));
         // P(j) V(j) done: the score buffer it read its weights from takes sub-block j + 2
@@ -656,6 +672,7 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
       // ---- weights 2^(s - m_ref) as bf16 pairs over the first half of the score columns -----
       {
         uint32_t pk[32];
+        [[maybe_unused]] uint32_t pr[SW ? 32 : 1];
         float rowsum0 = 0.f, rowsum1 = 0.f;
         const float neg_m = m_ref == -INFINITY ? 0.f : -m_ref;   // a row with nothing to see yet
 #pragma unroll
@@ -665,8 +682,10 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
           rowsum0 += p0;
           rowsum1 += p1;
           pk[i >> 1] = pack_bf16(p0, p1);
+          if constexpr (SW) pr[i >> 1] = pack_bf16_rest(p0, p1, pk[i >> 1]);
         }
         tmem_st32(t_s, pk);
+        if constexpr (SW) tmem_st32(t_s + 32, pr);        // second terms: the other half of the buffer
         tmem_wait_st();
         l_run += rowsum0 + rowsum1;
       }
@@ -802,7 +821,7 @@ size_t prefix_attention_scratch(const Geom& g, int n_queries, int max_len) {
   return plan_prefix(g, n_queries, max_len).scratch_bytes;
 }
 
-template <int G>
+template <int G, bool SW>
 static int launch_pf(const void* q, const void* K, const void* V, const Geom& g, int n_queries,
                      const LenView& cur_len_dev, int max_len, float scale, float* out,
                      float* lse_out, int32_t* status_word, float* scratch, size_t scratch_bytes,
@@ -828,7 +847,7 @@ static int launch_pf(const void* q, const void* K, const void* V, const Geom& g,
   const __nv_bfloat16* qb = static_cast<const __nv_bfloat16*>(q);
   if (!p.basic) {
     constexpr int smem_pipe = 1024 + 2 * kPfTileBytes + 2 * kPfStages * kPfSubTile;
-    auto kern_pipe = prefix_attention_pipelined_kernel<G>;
+    auto kern_pipe = prefix_attention_pipelined_kernel<G, SW>;
     if (cudaFuncSetAttribute(kern_pipe, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_pipe) != cudaSuccess)
       return L2KV_ERR_CUDA;
     kern_pipe<<<grid, kPfPipeThreads, smem_pipe, s>>>(qb, g, n_queries, cur_len_dev, max_len,
@@ -836,7 +855,7 @@ static int launch_pf(const void* q, const void* K, const void* V, const Geom& g,
                                                       status_word, p.split_len, p.rows, causal);
   } else {
     constexpr int smem_bytes = 1024 + 3 * kPfTileBytes;
-    auto kern = prefix_attention_basic_kernel<G>;
+    auto kern = prefix_attention_basic_kernel<G, SW>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) != cudaSuccess)
       return L2KV_ERR_CUDA;
     kern<<<grid, kPfThreads, smem_bytes, s>>>(qb, g, n_queries, cur_len_dev, max_len, scale * kPfLog2e,
@@ -857,11 +876,14 @@ static int launch_pf(const void* q, const void* K, const void* V, const Geom& g,
 int launch_prefix_attention(const void* q, const void* K, const void* V, const Geom& g, int dtype,
                             int n_queries, const LenView& cur_len_dev, int max_len, float scale,
                             float* out, float* lse_out, int32_t* status_word, float* scratch,
-                            size_t scratch_bytes, int causal, cudaStream_t s) {
+                            size_t scratch_bytes, int causal, int split_weights, cudaStream_t s) {
   if (dtype != L2KV_BF16 || g.D != 128) return L2KV_ERR_UNSUPPORTED;
 #define L2KV_PF(G)                                                                              \
-  return launch_pf<G>(q, K, V, g, n_queries, cur_len_dev, max_len, scale, out, lse_out,         \
-                      status_word, scratch, scratch_bytes, causal, s)
+  return split_weights                                                                          \
+      ? launch_pf<G, true>(q, K, V, g, n_queries, cur_len_dev, max_len, scale, out, lse_out,    \
+                           status_word, scratch, scratch_bytes, causal, s)                      \
+      : launch_pf<G, false>(q, K, V, g, n_queries, cur_len_dev, max_len, scale, out, lse_out,   \
+                            status_word, scratch, scratch_bytes, causal, s)
   switch (g.Hq / g.H) {
     case 1: L2KV_PF(1);
     case 2: L2KV_PF(2);

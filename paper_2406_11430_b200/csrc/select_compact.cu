@@ -36,7 +36,8 @@ gather_kernel(const T* __restrict__ K, const T* __restrict__ V, Geom gi, T* __re
   const int h = (int)(unit % gi.H);
   const int l = (int)((unit / gi.H) % gi.L);
   const int b = (int)(unit / ((long long)gi.H * gi.L));
-  const int len = max(0, min(len_dev[b], min(max_len, gi.t_cap)));
+  const long long bl = (long long)b * gi.L + l;
+  const int len = max(0, min(len_dev[b], min(max_len, gi.cap(bl))));
   const int t0 = chunk * kGatherChunk;
   if (t0 >= len) return;
   const int t_end = min(len, t0 + kGatherChunk);
@@ -44,7 +45,7 @@ gather_kernel(const T* __restrict__ K, const T* __restrict__ V, Geom gi, T* __re
   if (ur.n_keep == 0) return;
   const int2 cr = chunk_rec[unit * n_chunks + chunk];
   const int tid = threadIdx.x;
-  const float* key = sumsq + unit * ld;
+  const float* key = sumsq + (ld >= 0 ? unit * ld : gi.meta(unit));
   const bool identity = ur.flags & kFlagIdentity;
 
   int n_kept;
@@ -92,9 +93,10 @@ gather_kernel(const T* __restrict__ K, const T* __restrict__ V, Geom gi, T* __re
 
   // Copy the kept rows: LPR adjacent lanes move one row as 16-byte pieces.
   const int piece = tid % LPR, sub = tid / LPR;
-  const long long in_base = b * gi.sb + l * gi.sl + h * gi.sh + (long long)piece * Elem<T>::kPerVec;
-  const long long out_base = b * go.sb + l * go.sl + h * go.sh + (long long)piece * Elem<T>::kPerVec;
-  const long long meta_base = unit * (long long)go.t_cap;
+  const long long in_base = gi.base(b, l, h) + (long long)piece * Elem<T>::kPerVec;
+  const long long out_base = go.base(b, l, h) + (long long)piece * Elem<T>::kPerVec;
+  const long long meta_base = go.meta(unit);
+  const int out_cap = go.cap(bl);
   const bool no_keys = ur.flags & kFlagNoKeys;
   const int slot0 = cr.x;
   for (int jb = 0; jb < n_kept; jb += RPS * kGatherUnroll) {
@@ -118,7 +120,7 @@ gather_kernel(const T* __restrict__ K, const T* __restrict__ V, Geom gi, T* __re
       if (no_keys) s = piece_sumsq_reduce<T, LPR>(vk[i]);      // CTA-uniform branch
       if (src[i] >= 0) {
         const long long slot = slot0 + j;
-        if (slot < go.t_cap) {
+        if (slot < out_cap) {
           st_stream(K_out + out_base + slot * go.st, vk[i]);
           st_stream(V_out + out_base + slot * go.st, vv[i]);
           if (piece == 0) {
@@ -155,10 +157,11 @@ static int launch_sc_t(const void* K, const void* V, const Geom& gi, const int32
   } else if (sumsq_in) {
     key_mode = kKeysGiven;
     keys = const_cast<float*>(sumsq_in);                 // read-only in this mode
-    ld = gi.t_cap;
+    ld = -1;                                             // laid out like the input cache
   }
   SelectArgs sel;
   sel.keep_dev = keep_dev; sel.keep_unit_dev = keep_unit_dev; sel.out_t_cap = go.t_cap;
+  sel.out_row_cap = go.row_cap;
   sel.kept_len_unit_dev = kept_len_unit_dev;
   sel.policy = policy == L2KV_KEEP_HIGHEST_NORM ? L2KV_KEEP_HIGHEST_NORM : L2KV_KEEP_LOWEST_NORM;
   sel.seed = seed;

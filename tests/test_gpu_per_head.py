@@ -172,8 +172,9 @@ def test_append_evict_with_a_budget_per_head(l2, dtype, D):
     assert_attention_close(out.cpu().numpy(), want)
 
 
+@pytest.mark.parametrize("weights", ["split", "single"])
 @pytest.mark.parametrize("kernel", ["pipelined", "basic"])
-def test_prefix_attention_with_a_length_per_head(l2, kernel, monkeypatch):
+def test_prefix_attention_with_a_length_per_head(l2, kernel, weights, monkeypatch):
     monkeypatch.setenv("L2KV_PREFIX_KERNEL", kernel)
     w = synth.WORKLOADS[2].scaled(B=1, L=2, Hkv=2, Hq=8, T=700)
     K, V = synth.make_cache(w, DEV)
@@ -183,14 +184,19 @@ def test_prefix_attention_with_a_length_per_head(l2, kernel, monkeypatch):
     out = torch.full(q.shape, float("nan"), dtype=torch.float32, device=DEV)
     lse = torch.full(q.shape[:4], float("nan"), dtype=torch.float32, device=DEV)
     ws = torch.zeros(256, dtype=torch.uint8, device=DEV)
-    l2.prefix_attention_per_head(q, K, V, i32(cur), 700, out, lse, workspace=ws)
+    if weights == "single":
+        l2.prefix_attention_per_head(q, K, V, i32(cur), 700, out, lse, workspace=ws)
+    else:
+        l2.prefix_attention_flags(q, K, V, i32(cur), 700, out, l2.PREFIX_LEN_PER_HEAD | l2.PREFIX_SPLIT_WEIGHTS,
+                                  lse_out=lse, workspace=ws)
     torch.cuda.synchronize()
     assert l2.read_device_status(ws) == 0
     got = out.cpu().numpy()
     Kn, Vn = synth.to_numpy(K), synth.to_numpy(V)
     for s in range(37):
         want = oracle.attention(synth.to_numpy(q[:, :, s].contiguous()), Kn, Vn, "bf16", cur, nthreads=8)
-        assert_attention_close(got[:, :, s], want, atol=4e-3)
+        # one rounded bf16 weight: the documented 4e-3 reading; two terms: the decode path's bound
+        assert_attention_close(got[:, :, s], want, atol=4e-3 if weights == "single" else 2e-3)
     assert not got[0, 1, :, :4].any() and np.all(np.isneginf(lse[0, 1, :, :4].cpu().numpy()))
 
 
@@ -207,12 +213,13 @@ def test_prefix_attention_per_head_split_over_the_cache(l2):
     assert ws.numel() > 256
     out = torch.full(q.shape, float("nan"), dtype=torch.float32, device=DEV)
     lse = torch.full(q.shape[:4], float("nan"), dtype=torch.float32, device=DEV)
-    l2.prefix_attention_per_head(q, K, V, i32(cur), T, out, lse, workspace=ws)
+    l2.prefix_attention_flags(q, K, V, i32(cur), T, out, l2.PREFIX_LEN_PER_HEAD | l2.PREFIX_SPLIT_WEIGHTS,
+                              lse_out=lse, workspace=ws)
     torch.cuda.synchronize()
     assert l2.read_device_status(ws) == 0
     got = out.cpu().numpy()
     Kn, Vn = synth.to_numpy(K), synth.to_numpy(V)
     for s in range(0, 20, 3):
         want = oracle.attention(synth.to_numpy(q[:, :, s].contiguous()), Kn, Vn, "bf16", cur, nthreads=8)
-        assert_attention_close(got[:, :, s], want, atol=4e-3)
+        assert_attention_close(got[:, :, s], want)
     assert not got[0, 1, :, :4].any() and np.all(np.isneginf(lse[0, 1, :, :4].cpu().numpy()))
