@@ -71,7 +71,9 @@ typedef enum {
   L2KV_ERR_WORKSPACE_TOO_SMALL = -4,
   L2KV_ERR_OUT_OF_RANGE = -5,        /* max_len > t_cap, layer index outside [0, layers)   */
   L2KV_ERR_CUDA = -6,                /* a CUDA runtime call failed                         */
-  L2KV_ERR_DEVICE_OVERFLOW = -7      /* device status: a row did not fit t_cap             */
+  L2KV_ERR_DEVICE_OVERFLOW = -7,     /* device status: a row did not fit t_cap             */
+  L2KV_ERR_TIMEOUT = -8,             /* device status: a bounded wait in a kernel gave up  */
+  L2KV_ERR_DEBUG_BOUNDS = -9         /* device status, debug build only: an index check    */
 } l2kv_status;
 
 typedef enum { L2KV_F32 = 0, L2KV_BF16 = 1 } l2kv_dtype;
@@ -115,9 +117,36 @@ int l2kv_keep_count(int32_t len, double keep_ratio, int32_t* keep);
  * the workspace once before first use.  Host only. */
 int l2kv_workspace_bytes(const l2kv_layout* lay, int32_t max_len, size_t* bytes);
 
-/* Reads (and waits for) the device status word of a workspace: *status becomes
- * L2KV_OK or L2KV_ERR_DEVICE_OVERFLOW.  Synchronises `stream`. */
+/* Reads (and waits for) the device status word of a workspace.  Synchronises `stream`.
+ * *status becomes
+ *   L2KV_OK                   nothing happened;
+ *   L2KV_ERR_DEVICE_OVERFLOW  l2kv_append_evict had no row left for an append (the row was
+ *                             dropped, everything else went ahead);
+ *   L2KV_ERR_TIMEOUT          a kernel of l2kv_decode_attention or l2kv_prefix_attention gave up
+ *                             waiting for a copy or a tensor-core operation (every such wait
+ *                             is bounded so that a fault cannot hang the GPU).  The kernel
+ *                             also sets a mark in the status block at which the rest of its
+ *                             grid, and EVERY LATER decode / prefix call on this workspace,
+ *                             leaves at once without writing its output;
+ *   L2KV_ERR_DEBUG_BOUNDS     only from a library built with -DL2KV_DEBUG: an index check
+ *                             failed (the access was skipped).
+ * The word keeps the last anomaly until the workspace is cleared: after any non-zero status,
+ * and after any call that returned L2KV_ERR_CUDA (a launch that died may leave the per-unit
+ * completion counters of l2kv_select_compact / l2kv_append_evict non-zero, and the next call
+ * would then skip a unit's selection), call l2kv_workspace_reset or zero the workspace. */
 int l2kv_read_device_status(const void* workspace, void* stream, int32_t* status);
+
+/* Puts a workspace back into its initial state in stream order: zeroes the status block
+ * and the completion counters (the first l2kv_workspace_bytes(lay, 0) bytes; scratch beyond
+ * them never needs clearing).  Allocates nothing. */
+int l2kv_workspace_reset(void* workspace, size_t workspace_bytes, const l2kv_layout* lay,
+                         void* stream);
+
+/* Self-test of the give-up path, for test suites: one thread block waits, with a small poll
+ * limit, on a barrier that nothing will ever complete (no copy is in flight, nothing faults),
+ * gives up, and records L2KV_ERR_TIMEOUT and the abort mark in `workspace` exactly as the
+ * decode and prefix kernels do.  The paper has no counterpart. */
+int l2kv_selftest_wait_timeout(void* workspace, size_t workspace_bytes, void* stream);
 
 /* Key norms (Abstract; Section 3): for every valid token t < len_dev[b] of every
  * (b, l, h), sumsq_out[b,l,h,t] = sum_d K[b,l,h,t,d]^2 in the fixed order above, and,
@@ -311,13 +340,20 @@ int l2kv_attention_loss(const void* q, const void* K, const l2kv_layout* lay,
  * pool is already handed out) and that has no spare buffer to pass as a workspace.
  *
  *   - Limit: batch * layers * q_heads * ceil(max_len / 1024) * (head_dim + 2) * 4 bytes must
- *     not exceed L2KV_STATIC_SCRATCH_BYTES (16 MiB: e.g. one layer of 32 query heads at
+ *     not exceed L2KV_STATIC_SCRATCH_BYTES - 256 (16 MiB less the status block: e.g. one layer of 32 query heads at
  *     batch 4 up to a cache of about 250k tokens, or a whole 32-layer model at batch 4 up to 7k
  *     tokens).  Beyond it the call returns L2KV_ERR_WORKSPACE_TOO_SMALL and launches
  *     nothing: call per layer, or use l2kv_decode_attention with your own workspace.
- *   - The first call on each device looks up the array's device address (a runtime
- *     query, not an allocation), with the current device taken as the one `stream`
- *     belongs to; make that first call outside any stream capture.
+ *   - The first call on each device looks up the array's device address, with the current
+ *     device taken as the one `stream` belongs to.  The library calls no allocator, but that
+ *     first call is where the CUDA runtime loads this part of the library onto the device, and
+ *     the 16 MiB of the array are reserved then: make the call once at start-up, outside any
+ *     stream capture, and expect L2KV_ERR_CUDA from it if the device has no memory left.
+ *   - The first 256 bytes of the array are its status block, the rest holds the partial
+ *     results.  l2kv_decode_attention_static_status reads the status word as
+ *     l2kv_read_device_status does for a workspace (L2KV_OK or L2KV_ERR_TIMEOUT) and, with
+ *     reset != 0, then zeroes the status block in stream order, which a call needs after a
+ *     L2KV_ERR_TIMEOUT before it will write results again.
  *   - All calls on a device share the one array, which simply keeps what the last call
  *     left in it (nothing in it needs clearing between calls).  Two calls whose kernels can
  *     overlap on the GPU -- different streams, no dependency -- race on it and give wrong
@@ -326,6 +362,7 @@ int l2kv_attention_loss(const void* q, const void* K, const l2kv_layout* lay,
 int l2kv_decode_attention_static(const void* q, const void* K_c, const void* V_c,
                                  const l2kv_layout* lay, const int32_t* cur_len_dev,
                                  int32_t max_len, float scale, float* out, void* stream);
+int l2kv_decode_attention_static_status(void* stream, int32_t* status, int32_t reset);
 
 #ifdef __cplusplus
 }

@@ -68,6 +68,9 @@ def lib():
         L.l2kv_prefix_attention_per_head.argtypes = L.l2kv_prefix_attention.argtypes
         L.l2kv_prefix_attention_causal.argtypes = L.l2kv_prefix_attention.argtypes
         L.l2kv_prefix_attention_workspace_bytes.argtypes = [lay, i32, i32, ctypes.POINTER(sz)]
+        L.l2kv_workspace_reset.argtypes = [vp, sz, lay, vp]
+        L.l2kv_selftest_wait_timeout.argtypes = [vp, sz, vp]
+        L.l2kv_decode_attention_static_status.argtypes = [vp, ctypes.POINTER(i32), i32]
         L.l2kv_prefix_attention_flags.argtypes = [vp, vp, vp, lay, vp, i32, i32, ctypes.c_float,
                                                   ctypes.c_uint32, vp, vp, vp, sz, vp]
         for name in ("l2kv_prefix_attention", "l2kv_attention_loss_workspace_bytes", "l2kv_attention_loss",
@@ -76,7 +79,9 @@ def lib():
                      "l2kv_append_evict", "l2kv_select_compact_per_head",
                      "l2kv_decode_attention_per_head", "l2kv_append_evict_per_head",
                      "l2kv_prefix_attention_per_head", "l2kv_prefix_attention_workspace_bytes",
-                     "l2kv_prefix_attention_causal", "l2kv_prefix_attention_flags"):
+                     "l2kv_prefix_attention_causal", "l2kv_prefix_attention_flags",
+                     "l2kv_workspace_reset", "l2kv_selftest_wait_timeout",
+                     "l2kv_decode_attention_static_status"):
             getattr(L, name).restype = ctypes.c_int
         _LIB = L
     return _LIB
@@ -176,6 +181,26 @@ def read_device_status(workspace, stream=None):
     out = ctypes.c_int32(0)
     _check(lib().l2kv_read_device_status(_ptr(workspace), _stream(stream), ctypes.byref(out)),
            "l2kv_read_device_status")
+    return out.value
+
+
+def workspace_reset(workspace, layout, stream=None):
+    """Zeroes the status block and the completion counters of a workspace, in stream order."""
+    _check(lib().l2kv_workspace_reset(_ptr(workspace), workspace.numel(), layout.ref(), _stream(stream)),
+           "l2kv_workspace_reset")
+
+
+def selftest_wait_timeout(workspace, stream=None):
+    """Makes one bounded wait run out on purpose (nothing faults) and records it in workspace."""
+    _check(lib().l2kv_selftest_wait_timeout(_ptr(workspace), workspace.numel(), _stream(stream)),
+           "l2kv_selftest_wait_timeout")
+
+
+def decode_attention_static_status(reset=False, stream=None):
+    """Status word of the built-in scratch of decode_attention_static; reset=True clears it."""
+    out = ctypes.c_int32(0)
+    _check(lib().l2kv_decode_attention_static_status(_stream(stream), ctypes.byref(out), int(bool(reset))),
+           "l2kv_decode_attention_static_status")
     return out.value
 
 

@@ -15,6 +15,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libl2kv.so")
+DEBUG_LIB = os.path.join(HERE, "libl2kv_debug.so")      # the same library with index checks
 OBJ_DIR = os.path.join(HERE, "_build")
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
@@ -60,5 +61,13 @@ def build(force=False, verbose=False, out=None, defines=()):
     return out
 
 
+def build_debug(force=False):
+    """The bounds-checked variant: every index check that -DL2KV_DEBUG adds records
+    L2KV_ERR_DEBUG_BOUNDS in the workspace and skips the access (nothing traps)."""
+    return build(force=force, out=DEBUG_LIB, defines=["L2KV_DEBUG"])
+
+
 if __name__ == "__main__":
     print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    if "--debug" in sys.argv:
+        print(build_debug(force="--force" in sys.argv))

@@ -1,11 +1,19 @@
 // The C entry points: argument checks on the host, then the kernel launchers.
 #include <cmath>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "common.cuh"
 
 namespace {
 
 using namespace l2kv;
+
+// One NVTX range per entry point (no cost unless a profiler is attached).
+struct Range {
+  explicit Range(const char* name) { nvtxRangePushA(name); }
+  ~Range() { nvtxRangePop(); }
+};
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -73,6 +81,8 @@ const char* l2kv_status_string(int status) {
     case L2KV_ERR_OUT_OF_RANGE: return "length, capacity or layer index out of range";
     case L2KV_ERR_CUDA: return "CUDA runtime error";
     case L2KV_ERR_DEVICE_OVERFLOW: return "a cache row did not fit t_cap (device status)";
+    case L2KV_ERR_TIMEOUT: return "a bounded wait inside a kernel gave up (device status)";
+    case L2KV_ERR_DEBUG_BOUNDS: return "an index check of the debug build failed (device status)";
   }
   return "unknown status";
 }
@@ -106,8 +116,20 @@ int l2kv_read_device_status(const void* workspace, void* stream, int32_t* status
   return L2KV_OK;
 }
 
+int l2kv_workspace_reset(void* workspace, size_t workspace_bytes, const l2kv_layout* lay,
+                         void* stream) {
+  const int rc = check_layout(lay);
+  if (rc != L2KV_OK) return rc;
+  if (!workspace) return L2KV_ERR_INVALID_ARG;
+  const size_t head = plan_workspace(*lay, 0).sumsq_off;   // status block + completion counters
+  if (workspace_bytes < head) return L2KV_ERR_WORKSPACE_TOO_SMALL;
+  return cudaMemsetAsync(workspace, 0, head, static_cast<cudaStream_t>(stream)) == cudaSuccess
+             ? L2KV_OK : L2KV_ERR_CUDA;
+}
+
 int l2kv_key_norms(const void* K, const l2kv_layout* lay, const int32_t* len_dev, int32_t max_len,
                    float* sumsq_out, float* norm_out, void* stream) {
+  const Range nvtx_range("l2kv_key_norms");
   int rc = check_layout(lay);
   if (rc != L2KV_OK) return rc;
   if (max_len < 0) return L2KV_ERR_INVALID_ARG;
@@ -129,6 +151,7 @@ static int select_compact_impl(bool per_head, const void* K, const void* V, cons
                                void* V_out, const l2kv_layout* out, int32_t* idx_out,
                                float* sumsq_out, int32_t* kept_len_dev, void* workspace,
                                size_t workspace_bytes, void* stream) {
+  const Range nvtx_range("l2kv_select_compact");
   int rc = check_layout(in);
   if (rc != L2KV_OK) return rc;
   rc = check_layout(out);
@@ -194,6 +217,7 @@ static int decode_attention_impl(bool per_head, const void* q, const void* K_c, 
                                  const l2kv_layout* lay, const int32_t* cur_len_dev,
                                  int32_t max_len, float scale, float* out, void* workspace,
                                  size_t workspace_bytes, void* stream) {
+  const Range nvtx_range("l2kv_decode_attention");
   int rc = check_layout(lay);
   if (rc != L2KV_OK) return rc;
   rc = check_groups(lay);
@@ -234,6 +258,7 @@ static int append_evict_impl(bool per_head, void* K_c, void* V_c, int32_t* idx, 
                              int32_t n_uncompressed, const void* k_new, const void* v_new,
                              const int32_t* pos_new_dev, void* workspace, size_t workspace_bytes,
                              void* stream) {
+  const Range nvtx_range("l2kv_append_evict");
   int rc = check_layout(lay);
   if (rc != L2KV_OK) return rc;
   LayerMask unc;
@@ -282,6 +307,7 @@ static int prefix_attention_impl(bool per_head, bool causal, bool split_weights,
                                  int32_t max_len, int32_t n_queries, float scale, float* out,
                                  float* lse_out, void* workspace, size_t workspace_bytes,
                                  void* stream) {
+  const Range nvtx_range("l2kv_prefix_attention");
   int rc = check_layout(lay);
   if (rc != L2KV_OK) return rc;
   rc = check_groups(lay);
@@ -376,6 +402,7 @@ int l2kv_attention_loss(const void* q, const void* K, const l2kv_layout* lay,
                         const int32_t* cur_len_dev, int32_t max_len, float scale,
                         const float* sumsq, float* alr_out, float* loss_out, float* loss_ref_out,
                         void* workspace, size_t workspace_bytes, void* stream) {
+  const Range nvtx_range("l2kv_attention_loss");
   int rc = check_layout(lay);
   if (rc != L2KV_OK) return rc;
   if (packed(lay)) return L2KV_ERR_UNSUPPORTED;

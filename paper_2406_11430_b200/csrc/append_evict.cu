@@ -125,7 +125,7 @@ append_evict_kernel(T* __restrict__ K, T* __restrict__ V, int32_t* __restrict__ 
         if (slot < 0 || c_new > top) slot = -1;          // the newcomer is the one discarded
       }
     }
-    if (warp == 0 && slot >= 0 && lane < LPR) {
+    if (warp == 0 && slot >= 0 && lane < LPR && L2KV_BOUNDS(slot < cap && slot <= n, status_word)) {
       const long long row = g.base(b, l, h) + (long long)slot * g.st + lane * EPV;
       *reinterpret_cast<uint4*>(K + row) = vk;
       *reinterpret_cast<uint4*>(V + row) = vv;

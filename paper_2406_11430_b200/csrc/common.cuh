@@ -113,6 +113,28 @@ inline WorkspacePlan plan_workspace(const l2kv_layout& a, int max_len) {
   return p;
 }
 
+// ---- device status -------------------------------------------------------------------
+// Word 0 of a workspace: the first anomaly a kernel saw (an l2kv_status); word 2: abort mark,
+// set together with L2KV_ERR_TIMEOUT so that the remaining CTAs of a grid leave at once.
+__device__ __forceinline__ void record_timeout(int32_t* status_word) {
+  if (!status_word) return;
+  atomicExch(status_word, (int)L2KV_ERR_TIMEOUT);
+  atomicExch(status_word + 2, 1);
+}
+
+// Index checks of the debug build (-DL2KV_DEBUG): L2KV_BOUNDS(ok, status_word) is true when the
+// access may go ahead; when it may not, the debug build records L2KV_ERR_DEBUG_BOUNDS and the
+// caller skips the access (nothing traps).  The release build compiles the check away.
+#ifdef L2KV_DEBUG
+__device__ __forceinline__ bool debug_bounds(bool ok, int32_t* status_word) {
+  if (!ok && status_word) atomicExch(status_word, (int)L2KV_ERR_DEBUG_BOUNDS);
+  return ok;
+}
+#define L2KV_BOUNDS(ok, status_word) (::l2kv::debug_bounds((ok), (status_word)))
+#else
+#define L2KV_BOUNDS(ok, status_word) (true)
+#endif
+
 // ---- element access ------------------------------------------------------------------
 
 template <typename T> struct Elem;
@@ -228,6 +250,7 @@ struct SelectArgs {
   int2* chunk_rec;
   int32_t* tickets;
   int32_t* kept_len_dev;                      // [B, L] (head 0's length) or null
+  int32_t* status_word;                       // workspace status word, or null
 };
 int launch_key_norms(const void* K, const Geom& g, int dtype, const int32_t* len_dev, int max_len,
                      float* sumsq, long long ld_sumsq, float* norm_out, int key_mode,

@@ -199,7 +199,10 @@ decode_split_kernel(const T* __restrict__ q, const T* __restrict__ K, const T* _
 template <int D>
 __global__ void __launch_bounds__(D)
 decode_combine_kernel(const float* __restrict__ partial, LenView cur_len_dev,
-                      int max_len, Geom g, int n_splits, float* __restrict__ out) {
+                      int max_len, Geom g, int n_splits, float* __restrict__ out,
+                      const int32_t* __restrict__ status_word) {
+  // a split kernel that gave up left partial results behind that mean nothing: write no output
+  if (status_word && status_word[2] != 0) return;
   const int H = g.H, Hq = g.Hq;
   const long long row = blockIdx.x;                      // (b * L + l) * Hq + hq
   const long long bl = row / Hq;
@@ -570,10 +573,7 @@ decode_split_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16
     }
   }
   if constexpr (TMA) {
-    if (!copy_ok && tid == 0 && status_word) {
-      atomicExch(status_word, (int)L2KV_ERR_CUDA);
-      atomicExch(status_word + 2, 1);                      // abort mark read by later CTAs
-    }
+    if (!copy_ok && tid == 0) record_timeout(status_word);   // also marks the grid for leaving
   } else {
     cp_async_wait<0>();
   }
@@ -584,6 +584,7 @@ decode_split_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16
     const int head = 2 * fc + e;
     if (head < G) {
       float* p = partial + ((bl * g.Hq + h * G + head) * n_splits + split) * (long long)(D + 2);
+      if (!L2KV_BOUNDS(split < n_splits && t0 + nt <= g.cap(bl), status_word)) continue;
 #pragma unroll
       for (int db = 0; db < kDbw; ++db) {
         p[2 + 16 * (warp * kDbw + db) + fr] = oacc[db][e];
@@ -628,7 +629,8 @@ static int launch_dec_mma(const void* q, const void* K, const void* V, const Geo
     if (cudaGetLastError() != cudaSuccess) return L2KV_ERR_CUDA;
   }
   decode_combine_kernel<128><<<(unsigned)((long long)g.B * g.L * g.Hq), 128, 0, s>>>(
-      partial, cur_len_dev, max_len, g, plan.n_splits, out);
+      partial, cur_len_dev, max_len, g, plan.n_splits, out,
+      plan.partial_off >= (size_t)kStatusBytes ? reinterpret_cast<const int32_t*>(ws) : nullptr);
   return cudaGetLastError() == cudaSuccess ? L2KV_OK : L2KV_ERR_CUDA;
 }
 
@@ -647,7 +649,7 @@ static int launch_dec_t(const void* q, const void* K, const void* V, const Geom&
     if (cudaGetLastError() != cudaSuccess) return L2KV_ERR_CUDA;
   }
   decode_combine_kernel<D><<<(unsigned)((long long)g.B * g.L * g.Hq), D, 0, s>>>(
-      partial, cur_len_dev, max_len, g, plan.n_splits, out);
+      partial, cur_len_dev, max_len, g, plan.n_splits, out, nullptr);
   return cudaGetLastError() == cudaSuccess ? L2KV_OK : L2KV_ERR_CUDA;
 }
 

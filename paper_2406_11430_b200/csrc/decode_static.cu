@@ -60,20 +60,33 @@ extern "C" int l2kv_decode_attention_static(const void* q, const void* K_c, cons
   if (!q || !K_c || !V_c || !cur_len_dev || !out) return L2KV_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(K_c) || !aligned16(V_c)) return L2KV_ERR_MISALIGNED;
 
-  // Only the partial results need scratch: [B * L * Hq][splits][D + 2] floats.
+  // Only the partial results need scratch: [B * L * Hq][splits][D + 2] floats, placed after
+  // the status block that starts the array as it starts every workspace.
   WorkspacePlan plan = plan_workspace(*lay, max_len);
   const size_t need = plan.total - plan.partial_off;
-  if (need > (size_t)L2KV_STATIC_SCRATCH_BYTES) return L2KV_ERR_WORKSPACE_TOO_SMALL;
-  plan.partial_off = 0;
+  if (need > (size_t)L2KV_STATIC_SCRATCH_BYTES - kStatusBytes) return L2KV_ERR_WORKSPACE_TOO_SMALL;
+  plan.partial_off = kStatusBytes;
 
   void* scratch = nullptr;
   rc = scratch_address(&scratch);
   if (rc != L2KV_OK) return rc;
   const float sc = scale > 0.f ? scale : 1.0f / sqrtf((float)lay->head_dim);
-  // Nothing in the scratch has to start at zero: every partial that the merge step reads is
-  // written by the split step of the same call.
+  // The status block starts at zero (the array is zero-initialised when it is loaded) and
+  // changes only if a wait gives up; nothing else in the scratch has to start at zero: every
+  // partial that the merge step reads is written by the split step of the same call.
   const LenView lens{cur_len_dev, 0};
   return launch_decode_attention(q, K_c, V_c, make_geom(*lay), lay->dtype, lens, max_len, sc,
                                  out, static_cast<char*>(scratch), plan,
                                  static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int l2kv_decode_attention_static_status(void* stream, int32_t* status, int32_t reset) {
+  if (!status) return L2KV_ERR_INVALID_ARG;
+  void* scratch = nullptr;
+  int rc = scratch_address(&scratch);
+  if (rc != L2KV_OK) return rc;
+  rc = l2kv_read_device_status(scratch, stream, status);
+  if (rc != L2KV_OK || !reset) return rc;
+  return cudaMemsetAsync(scratch, 0, l2kv::kStatusBytes, static_cast<cudaStream_t>(stream)) ==
+                 cudaSuccess ? L2KV_OK : L2KV_ERR_CUDA;
 }

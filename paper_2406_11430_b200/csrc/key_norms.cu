@@ -100,7 +100,7 @@ key_norms_kernel(const T* __restrict__ K, Geom g, const int32_t* __restrict__ le
         }
         const float s = halving_reduce<U, LPR>(p, piece);
         const int t = t0 + my_row;
-        if (writer && t < row_end) {
+        if (writer && t < row_end && L2KV_BOUNDS(t >= 0 && t < g.cap(bl), sel.status_word)) {
           out[t] = s;
           if (nout) nout[t] = sqrtf(s);
         }

@@ -402,10 +402,7 @@ prefix_attention_basic_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n
     if (row_valid && lse_out && hf == 0)
       lse_out[row_off] = (m_ref + log2f(l_tot)) * 0.6931471805599453f;
   }
-  if (failed && tid == 0 && status_word) {
-    atomicExch(status_word, (int)L2KV_ERR_CUDA);
-    atomicExch(status_word + 2, 1);
-  }
+  if (failed && tid == 0) record_timeout(status_word);
   tc_fence_before();
   __syncthreads();
   if (warp == 0)
@@ -730,10 +727,7 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
     if (row_valid && lse_out)
       lse_out[row_off] = (m_ref + log2f(l_tot)) * 0.6931471805599453f;
   }
-  if (failed && tid == 0 && status_word) {
-    atomicExch(status_word, (int)L2KV_ERR_CUDA);
-    atomicExch(status_word + 2, 1);
-  }
+  if (failed && tid == 0) record_timeout(status_word);
   tc_fence_before();
   __syncthreads();
   if (warp == 0)
@@ -747,7 +741,8 @@ __global__ void __launch_bounds__(128)
 prefix_merge_kernel(const float* __restrict__ part_out, const float* __restrict__ part_lse,
                     LenView cur_len_dev, int max_len, int t_cap, int H, int Hq, int n_queries,
                     int split_len, long long rows_total, float* __restrict__ out,
-                    float* __restrict__ lse_out) {
+                    float* __restrict__ lse_out, const int32_t* __restrict__ status_word) {
+  if (status_word && status_word[2] != 0) return;       // a chunk gave up: no output
   const long long row = blockIdx.x;                      // ((b * L + l) * n_queries + s) * Hq + head
   const long long bl = row / ((long long)n_queries * Hq);
   const int h = (int)(row % Hq) / (Hq / H);
@@ -867,7 +862,7 @@ static int launch_pf(const void* q, const void* K, const void* V, const Geom& g,
     if (p.rows > 0x7fffffffLL) return L2KV_ERR_OUT_OF_RANGE;
     prefix_merge_kernel<<<(unsigned)p.rows, 128, 0, s>>>(k_out, k_lse, cur_len_dev, max_len, g.t_cap,
                                                          g.H, g.Hq, n_queries, p.split_len, p.rows,
-                                                         out, lse_out);
+                                                         out, lse_out, status_word);
     if (cudaGetLastError() != cudaSuccess) return L2KV_ERR_CUDA;
   }
   return L2KV_OK;

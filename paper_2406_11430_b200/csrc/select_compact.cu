@@ -23,7 +23,8 @@ gather_kernel(const T* __restrict__ K, const T* __restrict__ V, Geom gi, T* __re
               T* __restrict__ V_out, Geom go, const int32_t* __restrict__ len_dev, int max_len,
               const float* __restrict__ sumsq, long long ld, int policy,
               const UnitRec* __restrict__ unit_rec, const int2* __restrict__ chunk_rec,
-              int n_chunks, int32_t* __restrict__ idx_out, float* __restrict__ sumsq_out) {
+              int n_chunks, int32_t* __restrict__ idx_out, float* __restrict__ sumsq_out,
+              [[maybe_unused]] int32_t* __restrict__ status_word) {
   constexpr int LPR = D / Elem<T>::kPerVec;
   constexpr int RPS = kGatherThreads / LPR;              // rows per copy step of the CTA
   constexpr int TPT = kGatherChunk / kGatherThreads;     // tokens ranked per thread
@@ -108,6 +109,7 @@ gather_kernel(const T* __restrict__ K, const T* __restrict__ V, Geom gi, T* __re
       src[i] = j < n_kept ? (identity ? t0 + j : s_src[j]) : -1;
       vk[i] = make_uint4(0, 0, 0, 0);
       vv[i] = make_uint4(0, 0, 0, 0);
+      if (src[i] >= 0 && !L2KV_BOUNDS(src[i] >= t0 && src[i] < t_end, status_word)) src[i] = -1;
       if (src[i] >= 0) {
         vk[i] = ld_stream(K + in_base + (long long)src[i] * gi.st);
         vv[i] = ld_stream(V + in_base + (long long)src[i] * gi.st);
@@ -120,7 +122,7 @@ gather_kernel(const T* __restrict__ K, const T* __restrict__ V, Geom gi, T* __re
       if (no_keys) s = piece_sumsq_reduce<T, LPR>(vk[i]);      // CTA-uniform branch
       if (src[i] >= 0) {
         const long long slot = slot0 + j;
-        if (slot < out_cap) {
+        if (slot < out_cap && L2KV_BOUNDS(slot >= 0 && slot < ur.n_keep, status_word)) {
           st_stream(K_out + out_base + slot * go.st, vk[i]);
           st_stream(V_out + out_base + slot * go.st, vv[i]);
           if (piece == 0) {
@@ -168,6 +170,7 @@ static int launch_sc_t(const void* K, const void* V, const Geom& gi, const int32
   sel.n_chunks = plan.n_chunks; sel.unc = unc; sel.unit_rec = urec; sel.chunk_rec = crec;
   sel.tickets = reinterpret_cast<int32_t*>(ws + plan.ticket_off);
   sel.kept_len_dev = kept_len_dev;
+  sel.status_word = reinterpret_cast<int32_t*>(ws);
   // Keys of the layers that are compressed (the others are copied whole), and, as each
   // unit's last chunk of keys lands, its selection.
   const int rc = launch_key_norms(K, gi, Elem<T>::kDtype, len_dev, max_len, keys, ld, nullptr,
@@ -177,7 +180,7 @@ static int launch_sc_t(const void* K, const void* V, const Geom& gi, const int32
     gather_kernel<T, D><<<(unsigned)(units * plan.n_chunks), kGatherThreads, 0, s>>>(
         static_cast<const T*>(K), static_cast<const T*>(V), gi, static_cast<T*>(K_out),
         static_cast<T*>(V_out), go, len_dev, max_len, keys, ld, sel.policy, urec, crec,
-        plan.n_chunks, idx_out, sumsq_out);
+        plan.n_chunks, idx_out, sumsq_out, reinterpret_cast<int32_t*>(ws));
     if (cudaGetLastError() != cudaSuccess) return L2KV_ERR_CUDA;
   }
   return L2KV_OK;

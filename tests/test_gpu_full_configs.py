@@ -123,6 +123,39 @@ def test_config2_llama3_8b_32k(l2):
         q = synth.make_query(w, step, DEV)
         check_sampled_attention(l2, w, out, q, w.T, units + [(0, 0, 1), (3, 1, 6)])
     _free()
+    check_sampled_prefix_attention(l2, w, out, [(0, 2, 0, 0), (1, 17, 5, 127), (3, 31, 7, 64), (2, 9, 3, 31),
+                                               (0, 0, 1, 100), (3, 1, 6, 5)])
+    _free()
+
+
+def check_sampled_prefix_attention(l2, w, out, samples, n_q=128):
+    """Prefix attention in the launch the benchmark times (128 queries per (b, l) over the whole
+    compressed cache), plain and causal, both forms of the weights; the oracle recomputes the
+    sampled (b, l, kv head, query) rows with that row's own length."""
+    g = torch.Generator().manual_seed(17)
+    q = torch.randn((w.B, w.L, n_q, w.Hq, w.D), generator=g).to(torch.bfloat16).to(DEV)
+    res = torch.empty(q.shape, dtype=torch.float32, device=DEV)
+    ws = torch.zeros(256, dtype=torch.uint8, device=DEV)
+    G = w.Hq // w.Hkv
+    cur = out["cur"].cpu().numpy()
+    for causal in (False, True):
+        for weights, atol in (("split", 2e-3), ("single", 4e-3)):
+            flags = (l2.PREFIX_CAUSAL if causal else 0) | (l2.PREFIX_SPLIT_WEIGHTS if weights == "split" else 0)
+            res.fill_(float("nan"))
+            l2.prefix_attention_flags(q, out["K_c"], out["V_c"], out["cur"], w.T, res, flags, workspace=ws)
+            torch.cuda.synchronize()
+            assert l2.read_device_status(ws) == 0
+            assert bool(torch.isfinite(res).all())
+            worst = 0.0
+            for (b, l, h, s) in samples:
+                n = int(cur[b, l]) - (n_q - s - 1 if causal else 0)
+                Kn = synth.to_numpy(out["K_c"][b, l, h, :n])[None, None, None]
+                Vn = synth.to_numpy(out["V_c"][b, l, h, :n])[None, None, None]
+                qn = synth.to_numpy(q[b, l, s, h * G:(h + 1) * G])[None, None]
+                want = oracle.attention(qn, Kn, Vn, w.dtype, [[n]], nthreads=8)
+                got = res[b, l, s, h * G:(h + 1) * G].cpu().numpy()[None, None]
+                worst = max(worst, assert_attention_close(got, want, atol=atol))
+            print(f"prefix attention at full size, causal={causal}, {weights} weights: worst error {worst:.2e}")
 
 
 def test_config3_extreme_128k(l2):

@@ -113,6 +113,52 @@ def test_compress_exact_ties(l2):
     check_compress(l2, w, K, V, Kn, Vn, [1300], [300], policy=1)
 
 
+def near_tie_pair(seed=0):
+    """Two bf16 key rows A, B with fp64 sums ordered A < B (by ~1e-10 relative) and the
+    library's documented fp32 sums ordered the other way.  B is A's elements in another order
+    (only rounding differs) with one small element nudged up by one bf16 step."""
+    def bf16(x):
+        return (torch.from_numpy(x).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16))[None]
+    rng = np.random.default_rng(seed)
+    for _ in range(2000):
+        a = rng.standard_normal(128).astype(np.float32)
+        a[5] = 2.0 ** -10                                   # the element that gets nudged
+        b = a[rng.permutation(128)].copy()
+        b[np.argmin(np.abs(b - 2.0 ** -10))] = 2.0 ** -10 * (1 + 2.0 ** -7)
+        A, B = bf16(a), bf16(b)
+        if (oracle.key_sumsq(A, "bf16")[0] < oracle.key_sumsq(B, "bf16")[0]
+                and oracle.key_sumsq_f32(A, "bf16")[0] > oracle.key_sumsq_f32(B, "bf16")[0]):
+            return A[0], B[0]
+    raise AssertionError("no near-tie pair found")
+
+
+def test_near_tie_is_decided_in_fp32_and_reported_as_a_swap_inside_the_band(l2):
+    """A directed near-tie: the fp64 definition keeps row A, the fp32 keys keep row B.  The GPU
+    must agree bit for bit with the oracle run on the fp32-ordered keys, and differ from the
+    fp64 selection by exactly this one swap, which lies inside the 1e-6 norm band."""
+    A, B = near_tie_pair()
+    T, pa, pb = 96, 30, 61
+    w = synth.WORKLOADS[2].scaled(B=1, L=1, Hkv=1, Hq=1, T=T)
+    K, V, Kn, Vn = make(w)
+    Kn = Kn.copy()
+    # every other token: clearly smaller (first half) or clearly larger (second half) norms
+    base = (torch.from_numpy(A.view(np.int16).copy()).view(torch.bfloat16).float()).numpy()
+    for t in range(T):
+        f = 0.25 + 0.5 * t / T if t < T // 2 else 1.5 + t / T
+        row = torch.from_numpy((base * f).astype(np.float32)).to(torch.bfloat16)
+        Kn[0, 0, 0, t] = row.view(torch.int16).numpy().view(np.uint16)
+    Kn[0, 0, 0, pa], Kn[0, 0, 0, pb] = A, B
+    K = torch.from_numpy(Kn.view(np.int16)).view(torch.bfloat16).to(DEV)
+    keep = sum(1 for t in range(T // 2) if t != pa) + 1     # the smaller-norm tokens, then one of A / B
+    got, swaps = check_compress(l2, w, K, V, Kn, Vn, [T], [keep])
+    assert swaps == 1
+    kept = set(got["idx"][0, 0, 0, :keep].tolist())
+    assert pb in kept and pa not in kept                    # fp32 keys: B is the smaller
+    ref = oracle.compress(Kn, Vn, "bf16", [T], [keep])
+    kept64 = set(ref["idx"][0, 0, 0, :keep].tolist())
+    assert pa in kept64 and pb not in kept64                # fp64 keys: A is the smaller
+
+
 @pytest.mark.parametrize("T,keep", [(1, 1), (2, 1), (33, 17), (512, 512), (513, 1), (1024, 0)])
 def test_compress_edge_sizes(l2, T, keep):
     w = synth.WORKLOADS[0].scaled(T=T)

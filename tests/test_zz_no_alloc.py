@@ -8,6 +8,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 import synth
 from gpu_util import DEV, i32, gpu_attention, assert_attention_close
 
@@ -34,6 +35,9 @@ def test_static_scratch_matches_workspace_variant_twice_in_a_row():
         got = _static(l2, q, K, V, cur_dev, w.T)
         assert_attention_close(got, want.astype(np.float64))
         np.testing.assert_allclose(got, want, rtol=1e-6, atol=1e-7)
+        # and against the definition itself, not only the other entry point
+        ref = oracle.attention(synth.to_numpy(q), synth.to_numpy(K), synth.to_numpy(V), w.dtype, cur, nthreads=8)
+        assert_attention_close(got, ref)
     # fp32 caches go through the other kernel family; same contract
     w32 = synth.WORKLOADS[0].scaled(T=1500)
     K32, V32 = synth.make_cache(w32, DEV)
