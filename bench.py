@@ -36,19 +36,17 @@ GIB = 1 << 30
 METRIC = "compress + decode GB/s of KV read and % of B200 HBM peak; decode tokens/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
-# DRAM bytes (read + written) per algorithmic byte of the dominant kernel, from the ncu capture
-# summarised in profiles/decode_split_mma_kernel_llama3-8b-32k_4layers.md (a 4-layer case; the
-# traffic is proportional to the tokens streamed).  Set to None whenever that kernel changes.
+# DRAM bytes (read + written) per algorithmic byte of the dominant kernel, from an ncu capture of
+# the decode split kernel on a 4-layer case of the benchmark workload (the traffic is
+# proportional to the tokens streamed).  Set to None whenever that kernel changes.
 DECODE_TRAFFIC_RATIO = 1.0058
 
 
 def workload(args):
     """The benchmark workload: configuration 2 (Llama-3-8B, 32k context) unless --workload
-    picks another of the five; the serving workload is cut to 8 of its 32 layers, since all 32
-    padded to the longest sequence do not fit one GPU next to their compressed copy."""
+    picks another of the five.  The ragged serving workload runs on packed (unpadded) caches,
+    so all of its 32 layers fit one GPU."""
     w = synth.WORKLOADS[args.workload]
-    if w.append_steps and not args.layers:
-        w = w.scaled(L=8)
     if args.layers:
         w = w.scaled(L=args.layers)
     if args.context:
@@ -157,30 +155,50 @@ def barrier(world):
 # ------------------------------------------------------------------------------ GPU arm
 
 class Job:
-    """Device-resident state of one rank: the full cache, the compressed cache, queries."""
+    """Device-resident state of one rank: the full cache, the compressed cache, queries.
+    Ragged workloads use packed caches (no padding): the input holds len_b rows per (b, l); in
+    the compressed cache an uncompressed layer has room for len_b + steps rows and a compressed
+    one for its keep count."""
 
     def __init__(self, w, device, rank):
         import paper_2406_11430_b200 as l2
         self.l2, self.w, self.dev = l2, w, device
         ws = w.scaled(seed=w.seed + 1000 * rank)          # each rank its own batch
-        self.K, self.V = synth.make_cache(ws, device)
         self.lens_host = synth.ragged_lengths(ws)
         self.keep_host = np.ceil(w.keep_ratio * self.lens_host.astype(np.float64)).astype(np.int32)
+        self.unc = tuple(l for l in w.uncompressed if l < w.L)
+        self.packed = bool(w.ragged_lo)
         self.t_cap = w.T + w.append_steps                 # uncompressed layers grow by one per step
-        shape = (w.B, w.L, w.Hkv, self.t_cap, w.D)
-        self.K_c = torch.zeros(shape, dtype=w.torch_dtype, device=device)
+        if self.packed:
+            self.K, self.V, rin = synth.make_cache_packed(ws, self.lens_host, device)
+            self.rin_host, self.rin = rin, l2.Rows(*rin, device)
+            caps = [[int(self.lens_host[b]) + w.append_steps if l in self.unc else int(self.keep_host[b])
+                     for l in range(w.L)] for b in range(w.B)]
+            self.rows_host = synth.packing(caps)
+            self.rows = l2.Rows(*self.rows_host, device)
+            total = self.rows_host[2]
+            self.K_c = torch.zeros((w.Hkv, total, w.D), dtype=w.torch_dtype, device=device)
+            meta = (w.Hkv, total)
+        else:
+            self.K, self.V = synth.make_cache(ws, device)
+            self.rin = self.rows = None
+            shape = (w.B, w.L, w.Hkv, self.t_cap, w.D)
+            self.K_c = torch.zeros(shape, dtype=w.torch_dtype, device=device)
+            meta = shape[:4]
         self.V_c = torch.zeros_like(self.K_c)
-        self.idx = torch.zeros(shape[:4], dtype=torch.int32, device=device)
-        self.sumsq = torch.zeros(shape[:4], dtype=torch.float32, device=device)
+        self.idx = torch.zeros(meta, dtype=torch.int32, device=device)
+        self.sumsq = torch.zeros(meta, dtype=torch.float32, device=device)
         self.cur = torch.zeros((w.B, w.L), dtype=torch.int32, device=device)
         self.keep_n = int(self.keep_host.max())
+        self.max_in = int(self.lens_host.max())           # longest sequence handed to compression
+        self.max_dec = self.rows.t_cap if self.packed else self.t_cap   # longest cache decode may meet
         self.lens = torch.tensor(self.lens_host, dtype=torch.int32, device=device)
         self.keep = torch.tensor(self.keep_host, dtype=torch.int32, device=device)
-        self.unc = tuple(l for l in w.uncompressed if l < w.L)
         self.q = torch.stack([synth.make_query(ws, s, device) for s in range(w.decode_steps)])
         self.out = torch.zeros((w.decode_steps, w.B, w.L, w.Hq, w.D), dtype=torch.float32,
                                device=device)
-        self.ws = l2.new_workspace(l2.Layout(self.K_c, q_heads=w.Hq), self.t_cap, device)
+        self.ws = l2.new_workspace(l2.Layout(self.K_c, q_heads=w.Hq, rows=self.rows),
+                                   max(self.max_dec, self.max_in), device)
         self.new_rows, self.new_pos = [], []
         for s in range(w.append_steps):                   # budget-maintained serving loop
             self.new_rows.append(synth.make_new_kv(ws, s, device))
@@ -189,25 +207,31 @@ class Job:
         # one append/evict launch when the workload maintains a budget
         self.launches_per_step = 2 + (3 if w.append_steps else 2) * w.decode_steps
 
+    def kv_bytes(self):
+        return 2 * self.K.numel() * self.w.elem_bytes
+
     def compress(self, b=None):
-        """The whole batch, or (b given) sequence b alone: every tensor of one sequence is dense."""
-        i = slice(None) if b is None else slice(b, b + 1)
-        self.l2.select_compact(self.K[i], self.V[i], self.lens[i], self.keep[i], self.w.T, self.unc,
-                               self.K_c[i], self.V_c[i], self.idx[i], self.sumsq[i], self.cur[i], self.ws)
+        """The whole batch, or (b given; dense caches) sequence b alone: every tensor of one
+        sequence is dense."""
+        i = slice(None) if b is None or self.packed else slice(b, b + 1)
+        self.l2.select_compact(self.K[i], self.V[i], self.lens[i], self.keep[i], self.max_in, self.unc,
+                               self.K_c[i], self.V_c[i], self.idx[i], self.sumsq[i], self.cur[i], self.ws,
+                               rows_in=self.rin, rows_out=self.rows)
 
     def compress_variant(self, policy=0, sumsq_in=None):
-        self.l2.select_compact(self.K, self.V, self.lens, self.keep, self.w.T, self.unc, self.K_c,
+        self.l2.select_compact(self.K, self.V, self.lens, self.keep, self.max_in, self.unc, self.K_c,
                                self.V_c, self.idx, self.sumsq, self.cur, self.ws, policy=policy,
-                               seed=1, sumsq_in=sumsq_in)
+                               seed=1, sumsq_in=sumsq_in, rows_in=self.rin, rows_out=self.rows)
 
     def decode(self, s, b=None):
-        i = slice(None) if b is None else slice(b, b + 1)
+        i = slice(None) if b is None or self.packed else slice(b, b + 1)
         if self.w.append_steps:
             k, v = self.new_rows[s]
             self.l2.append_evict(self.K_c[i], self.V_c[i], self.idx[i], self.sumsq[i], self.cur[i],
-                                 self.keep[i], self.unc, k[i], v[i], self.new_pos[s][i], self.ws)
-        self.l2.decode_attention(self.q[s][i], self.K_c[i], self.V_c[i], self.cur[i], self.t_cap,
-                                 self.out[s][i], self.ws)
+                                 self.keep[i], self.unc, k[i], v[i], self.new_pos[s][i], self.ws,
+                                 rows=self.rows)
+        self.l2.decode_attention(self.q[s][i], self.K_c[i], self.V_c[i], self.cur[i], self.max_dec,
+                                 self.out[s][i], self.ws, rows=self.rows)
 
     def step(self, ev=None):
         """One pass of the whole path.  ev: optional list collecting (start, mid, end) events."""
@@ -222,26 +246,26 @@ class Job:
             e2 = torch.cuda.Event(enable_timing=True); e2.record()
             ev.append((e0, e1, e2))
 
+    def unit_input_rows(self, b, l, h):
+        """K rows of unit (b, l, h) of the input cache (device view) and its kept positions."""
+        n_in, keep = int(self.lens_host[b]), int(self.keep_host[b])
+        if self.packed:
+            i0, o0 = int(self.rin_host[0][b, l]), int(self.rows_host[0][b, l])
+            return self.K[h, i0:i0 + n_in], self.idx[h, o0:o0 + keep]
+        return self.K[b, l, h, :n_in], self.idx[b, l, h, :keep]
 
-def run_gpu(args):
-    rank, world, local = dist_setup(args.gpus)
-    device = torch.device("cuda", local)
-    torch.cuda.set_device(device)
-    w = workload(args)
-    job = Job(w, device, rank)
-    cbytes, dbytes_all, abytes_all = algorithmic_bytes(w, job.lens_host)
-    dbytes = (dbytes_all + abytes_all) / w.decode_steps   # per decode step (with its append, if any)
-    step_bytes = cbytes + dbytes_all + abytes_all
-    keep = job.keep_n
 
-    for _ in range(max(args.warmup, 3)):
+def measure(job, w, steps, warmup, world, device, rank, local):
+    """warmup untimed steps, then `steps` timed ones between barriers; device times, max over
+    ranks; SM clocks sampled during the timed region (rank 0)."""
+    for _ in range(warmup):
         job.step()
     barrier(world)
     sampler = ClockSampler(local) if rank == 0 else None
     ev = []
     t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
     t0.record()
-    for _ in range(args.steps):
+    for _ in range(steps):
         job.step(ev)
     t1.record()
     barrier(world)
@@ -249,39 +273,16 @@ def run_gpu(args):
     clocks = sampler.stop() if sampler else None
     c_ms = statistics.mean(a.elapsed_time(b) for a, b, _ in ev)
     d_ms = statistics.mean(b.elapsed_time(c) for _, b, c in ev) / w.decode_steps
-    c_ms = max_over_ranks(c_ms, world, device)
-    d_ms = max_over_ranks(d_ms, world, device)
+    return (total_ms, max_over_ranks(c_ms, world, device), max_over_ranks(d_ms, world, device), clocks)
 
-    variants = None
-    if rank == 0 and not args.no_variants and not w.append_steps and not w.ragged_lo:
-        variants = time_variants(job, w, cbytes)
 
-    # end to end: inputs start in pinned host memory, results end there
-    e2e = None
-    if not args.no_e2e:
-        e2e = run_e2e(job, w, step_bytes, world, device, args)
-
-    if rank != 0:
-        return
-    ms_per_step = total_ms / args.steps
-    value = world * step_bytes / (ms_per_step * 1e-3) / 1e9
-    peak, peak_kind = measured_peak()
+def stage_report(w, job, c_ms, d_ms, world, peak, peak_kind):
+    """The per-stage numbers of one workload: ms, algorithmic GB/s, fractions of both peaks."""
+    cbytes, dbytes_all, abytes_all = algorithmic_bytes(w, job.lens_host)
+    dbytes = (dbytes_all + abytes_all) / w.decode_steps   # per decode step (with its append, if any)
     dec_gbs = dbytes / (d_ms * 1e-3) / 1e9
     cmp_gbs = cbytes / (c_ms * 1e-3) / 1e9
-    line = {
-        "metric": METRIC, "value": round(value, 1), "unit": "GB/s", "n_gpus": world,
-        "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": round(ms_per_step, 3),
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
-        "data": "synthetic",
-        "config": {"workload": w.name, "batch": w.B, "layers": w.L, "kv_heads": w.Hkv,
-                   "q_heads": w.Hq, "head_dim": w.D, "context": w.T, "storage": w.dtype,
-                   "ragged_lengths": bool(w.ragged_lo),
-                   "append_evict_per_decode_step": bool(w.append_steps),
-                   "keep_ratio": w.keep_ratio, "keep_per_head": keep,
-                   "uncompressed_layers": list(job.unc), "decode_steps_per_step": w.decode_steps,
-                   "l2": f"inputs larger than L2 ({dbytes / GIB:.1f} GiB read per decode step, "
-                         f"{2 * job.K.numel() * w.elem_bytes / GIB:.0f} GiB of K and V per compress)",
-                   "parallelism": f"independent replicas x{world}, no collective"},
+    return {
         "compress": {"ms": round(c_ms, 3), "GBps": round(cmp_gbs, 1), "bytes": int(cbytes),
                      "frac_of_8TBps": round(cmp_gbs / NOMINAL_HBM_GBS, 4),
                      f"frac_of_{peak_kind}": round(cmp_gbs / peak, 4)},
@@ -289,23 +290,101 @@ def run_gpu(args):
                    "frac_of_8TBps": round(dec_gbs / NOMINAL_HBM_GBS, 4),
                    f"frac_of_{peak_kind}": round(dec_gbs / peak, 4),
                    "tokens_per_s": round(world * w.B / (d_ms * 1e-3), 1)},
-        "roofline": {"bound": "hbm", "kernel": "decode_split_mma_kernel (+ combine, timed together)",
-                     "achieved": round(dec_gbs, 1), "peak": peak, "peak_kind": peak_kind,
-                     "unit": "GB/s", "frac": round(dec_gbs / peak, 4),
-                     "traffic": args.traffic if args.traffic is not None else
-                     (round(DECODE_TRAFFIC_RATIO * dbytes)
-                      if DECODE_TRAFFIC_RATIO and args.workload == 2 and not w.append_steps else None)},
-        "gpu_launches": job.launches_per_step * args.steps,
-        "clocks": clocks,
-    }
-    if variants:
-        line["variants"] = variants
-    if e2e:
-        line["e2e"] = e2e
-    if not args.no_cpu_baseline and world == 1:
-        line["cpu_baseline"] = cpu_baseline(w, target_s=args.cpu_seconds)
-        line["tie_band"] = tie_band_report(job, w)
-    print(json.dumps(line))
+    }, cbytes + dbytes_all + abytes_all, dbytes, dec_gbs
+
+
+def workload_config(w, job, world):
+    return {"workload": w.name, "batch": w.B, "layers": w.L, "kv_heads": w.Hkv,
+            "q_heads": w.Hq, "head_dim": w.D, "context": w.T, "storage": w.dtype,
+            "ragged_lengths": bool(w.ragged_lo), "cache_layout": "packed" if job.packed else "dense",
+            "append_evict_per_decode_step": bool(w.append_steps),
+            "keep_ratio": w.keep_ratio, "keep_per_head": job.keep_n,
+            "uncompressed_layers": list(job.unc), "decode_steps_per_step": w.decode_steps}
+
+
+def run_gpu(args):
+    rank, world, local = dist_setup(args.gpus)
+    device = torch.device("cuda", local)
+    torch.cuda.set_device(device)
+    w = workload(args)
+    job = Job(w, device, rank)
+    peak, peak_kind = measured_peak()
+    warmup = max(args.warmup, 3)
+    total_ms, c_ms, d_ms, clocks = measure(job, w, args.steps, warmup, world, device, rank, local)
+    stages, step_bytes, dbytes, dec_gbs = stage_report(w, job, c_ms, d_ms, world, peak, peak_kind)
+    cbytes = stages["compress"]["bytes"]
+
+    variants = None
+    if rank == 0 and not args.no_variants and not w.append_steps and not w.ragged_lo:
+        variants = time_variants(job, w, cbytes)
+
+    # end to end: inputs start in pinned host memory, results end there
+    e2e = None
+    if not args.no_e2e and not job.packed:
+        e2e = run_e2e(job, w, step_bytes, world, device, args)
+
+    line = None
+    if rank == 0:
+        ms_per_step = total_ms / args.steps
+        value = world * step_bytes / (ms_per_step * 1e-3) / 1e9
+        cfg = workload_config(w, job, world)
+        cfg["l2"] = (f"inputs larger than L2 ({dbytes / GIB:.1f} GiB read per decode step, "
+                     f"{job.kv_bytes() / GIB:.0f} GiB of K and V per compress)")
+        cfg["parallelism"] = f"independent replicas x{world}, no collective"
+        line = {
+            "metric": METRIC, "value": round(value, 1), "unit": "GB/s", "n_gpus": world,
+            "steps": args.steps, "warmup": warmup, "ms_per_step": round(ms_per_step, 3),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic", "config": cfg,
+            "compress": stages["compress"], "decode": stages["decode"],
+            "roofline": {"bound": "hbm", "kernel": "decode_split_mma_kernel (+ combine, timed together)",
+                         "achieved": round(dec_gbs, 1), "peak": peak, "peak_kind": peak_kind,
+                         "unit": "GB/s", "frac": round(dec_gbs / peak, 4),
+                         "traffic": args.traffic if args.traffic is not None else
+                         (round(DECODE_TRAFFIC_RATIO * dbytes)
+                          if DECODE_TRAFFIC_RATIO and args.workload == 2 and not w.append_steps else None)},
+            "gpu_launches": job.launches_per_step * args.steps,
+            "clocks": clocks,
+        }
+        if variants:
+            line["variants"] = variants
+        if e2e:
+            line["e2e"] = e2e
+        if not args.no_cpu_baseline and world == 1:
+            line["cpu_baseline"] = cpu_baseline(w, target_s=args.cpu_seconds)
+            line["tie_band"] = tie_band_report(job, w)
+
+    # the other four configurations, a few steps each (same job, same measurement)
+    if not args.no_other_configs and args.workload == 2 and not (args.layers or args.context):
+        del job
+        free_device_memory()
+        others = {}
+        for i, wo in enumerate(synth.WORKLOADS):
+            if i == args.workload:
+                continue
+            jo = Job(wo, device, rank)
+            n = 2 if wo.append_steps else 5
+            _, c2, d2, clk = measure(jo, wo, n, 3, world, device, rank, local)
+            if rank == 0:
+                st, _, _, _ = stage_report(wo, jo, c2, d2, world, peak, peak_kind)
+                entry = {"config": workload_config(wo, jo, world), "steps": n, "warmup": 3,
+                         "compress": st["compress"], "decode": st["decode"], "clocks": clk,
+                         "gpu_launches": jo.launches_per_step * n}
+                if not args.no_cpu_baseline and world == 1:
+                    entry["tie_band"] = tie_band_report(jo, wo)
+                others[wo.name] = entry
+            del jo
+            free_device_memory()
+        if rank == 0:
+            line["configs"] = others
+    if rank == 0:
+        print(json.dumps(line))
+
+
+def free_device_memory():
+    import gc
+    gc.collect()
+    torch.cuda.empty_cache()
 
 
 def time_variants(job, w, cbytes, reps=5):
@@ -543,11 +622,18 @@ def cpu_baseline(w, target_s=15.0):
     # the uncompressed layer of the pair costs about two compressed ones (twice the rows)
     n_comp = int(max(1, min(w.L - len(w.uncompressed), round(3 * target_s / max(probe, 1e-3) - 2))))
     dt, nbytes, nthreads, layers = oracle_sample_step(w, n_dec=w.decode_steps, n_comp=n_comp)
+    # the same oracle on one thread, on a smaller sample (one layer pair, a few decode steps)
+    n1 = min(4, w.decode_steps)
+    dt1, nbytes1, _, layers1 = oracle_sample_step(w, n_dec=n1, n_comp=1, nthreads=1)
     return {"value": round(nbytes / dt / 1e9, 4), "unit": "GB/s", "cores": nthreads,
             "kind": "oracle", "seconds": round(dt, 2),
             "sample": f"sequence 0, layers {layers} (first one uncompressed), all {w.Hkv} KV "
                       f"heads, full {w.T}-token context: one compression pass + "
-                      f"{w.decode_steps} decode steps"}
+                      f"{w.decode_steps} decode steps",
+            "single_thread": {"value": round(nbytes1 / dt1 / 1e9, 4), "unit": "GB/s", "cores": 1,
+                              "seconds": round(dt1, 2),
+                              "sample": f"sequence 0, layers {layers1}, all {w.Hkv} KV heads, full "
+                                        f"{w.T}-token context: one compression pass + {n1} decode steps"}}
 
 
 def tie_band_report(job, w, n_units=6, band=1e-6):
@@ -563,11 +649,11 @@ def tie_band_report(job, w, n_units=6, band=1e-6):
     swaps = bad = 0
     for i in range(n_units):
         b, l, h = i % w.B, comp[(i * 7) % len(comp)], (i * 3) % w.Hkv
-        n_in, keep = int(job.lens_host[b]), int(job.keep_host[b])
-        Kn = synth.to_numpy(job.K[b, l, h, :n_in])[None, None, None]
-        key = oracle.key_sumsq(Kn, w.dtype)[0, 0, 0]
+        keep = int(job.keep_host[b])
+        rows, kept = job.unit_input_rows(b, l, h)
+        key = oracle.key_sumsq(np.ascontiguousarray(synth.to_numpy(rows)), w.dtype)
         want = set(oracle.select(key, keep).tolist())
-        got = set(job.idx[b, l, h, :keep].cpu().tolist())
+        got = set(kept.cpu().tolist())
         norm = np.sqrt(key)
         thr = np.sort(norm)[keep - 1]
         for t in got ^ want:
@@ -617,6 +703,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-variants", action="store_true")
+    ap.add_argument("--no-other-configs", action="store_true",
+                    help="skip the short runs of the other four configurations")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--workload", type=int, default=2, choices=range(len(synth.WORKLOADS)),
                     help="which of the five configurations (default 2: llama3-8b-32k)")

@@ -41,13 +41,26 @@ key_norms_kernel(const T* __restrict__ K, Geom g, const int32_t* __restrict__ le
   static_assert(U <= LPR, "the halving reduction needs at least as many lanes as rows");
   const long long unit = blockIdx.x / chunks_per_unit;
   const int chunk = blockIdx.x % chunks_per_unit;
-  const int h = (int)(unit % g.H);
-  const int l = (int)((unit / g.H) % g.L);
-  const int b = (int)(unit / ((long long)g.H * g.L));
   const int tid = threadIdx.x;
-  const long long bl = (long long)b * g.L + l;
-  const int len = max(0, min(len_dev[b], min(max_len, g.cap(bl))));
-  [[maybe_unused]] const int out_cap = SEL ? (sel.out_row_cap ? sel.out_row_cap[bl] : sel.out_t_cap) : 0;
+  // Where this unit lives: worked out by one thread and handed round through shared memory, so
+  // that the streaming loop below is compiled free of the addressing arithmetic (dense or packed).
+  __shared__ long long s_kbase, s_keyoff;
+  __shared__ int s_ctx[6];
+  if (tid == 0) {
+    const int h0 = (int)(unit % g.H);
+    const int l0 = (int)((unit / g.H) % g.L);
+    const int b0 = (int)(unit / ((long long)g.H * g.L));
+    const long long bl0 = (long long)b0 * g.L + l0;
+    s_ctx[0] = h0; s_ctx[1] = l0; s_ctx[2] = b0;
+    s_ctx[3] = max(0, min(len_dev[b0], min(max_len, g.cap(bl0))));
+    s_ctx[4] = SEL ? (sel.out_row_cap ? sel.out_row_cap[bl0] : sel.out_t_cap) : 0;
+    s_kbase = g.base(b0, l0, h0);
+    s_keyoff = ld >= 0 ? unit * ld : g.meta(unit);         // ld < 0: keys laid out like the cache
+  }
+  __syncthreads();
+  const int h = s_ctx[0], l = s_ctx[1], b = s_ctx[2], len = s_ctx[3];
+  [[maybe_unused]] const int out_cap = s_ctx[4];
+  [[maybe_unused]] const long long bl = (long long)b * g.L + l;
 
   if constexpr (SEL) {
     // Units that need no keys: copied layers and empty sequences get their record here.
@@ -62,7 +75,7 @@ key_norms_kernel(const T* __restrict__ K, Geom g, const int32_t* __restrict__ le
       return;
     }
   }
-  float* out = sumsq + (ld >= 0 ? unit * ld : g.meta(unit));   // ld < 0: laid out like the cache
+  float* out = sumsq + s_keyoff;
   if constexpr (MODE != kKeysGiven) {
     const int row0 = chunk * kNormRowsPerCta;
     if (row0 >= len) return;
@@ -74,8 +87,8 @@ key_norms_kernel(const T* __restrict__ K, Geom g, const int32_t* __restrict__ le
     } else {
       const int piece = tid % LPR;
       const int sub = tid / LPR;
-      const T* base = K + g.base(b, l, h) + (long long)piece * Elem<T>::kPerVec;
-      float* nout = norm_out ? norm_out + (ld >= 0 ? unit * ld : g.meta(unit)) : nullptr;
+      const T* base = K + s_kbase + (long long)piece * Elem<T>::kPerVec;
+      float* nout = norm_out ? norm_out + s_keyoff : nullptr;
       const int my_row = piece / (LPR / U);              // which of its U rows this lane reports
       const bool writer = (piece % (LPR / U)) == 0;
 
