@@ -139,7 +139,7 @@ int l2kv_key_norms(const void* K, const l2kv_layout* lay, const int32_t* len_dev
   if (!aligned16(K)) return L2KV_ERR_MISALIGNED;
   // leading dimension -1: the outputs are laid out like the cache's rows
   return launch_key_norms(K, make_geom(*lay), lay->dtype, len_dev, max_len, sumsq_out, -1,
-                          norm_out, kKeysOnly, nullptr, static_cast<cudaStream_t>(stream));
+                          norm_out, kKeysOnly, nullptr, nullptr, static_cast<cudaStream_t>(stream));
 }
 
 // Both forms of the compression call: keep counts and result lengths per sequence

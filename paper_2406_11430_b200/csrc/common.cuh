@@ -48,6 +48,7 @@ struct Geom {
 struct UnitRec { uint32_t thr; int32_t admit; int32_t n_keep; uint32_t flags; };
 constexpr uint32_t kFlagIdentity = 1u;           // every valid token is kept
 constexpr uint32_t kFlagNoKeys = 2u;             // keys were not precomputed for this unit
+constexpr uint32_t kFlagCopied = 4u;             // the norm pass copies this unit itself (see CopyArgs)
 
 struct LayerMask {
   uint32_t w[kMaxLayers / 32];
@@ -252,9 +253,23 @@ struct SelectArgs {
   int32_t* kept_len_dev;                      // [B, L] (head 0's length) or null
   int32_t* status_word;                       // workspace status word, or null
 };
+// Uncompressed layers inside l2kv_select_compact: their whole-unit copies run as the LAST blocks
+// of the norm pass's grid, so that they fill the GPU while the selections of the last compressed
+// units (one block each, after the stream of K has ended) are still running.
+struct CopyArgs {
+  const void* V;
+  void* K_out;
+  void* V_out;
+  int32_t* idx_out;
+  float* sumsq_out;
+  Geom go;
+  int n_blocks;                               // trailing copy blocks of the grid (0 = none)
+  int n_unc;                                  // uncompressed layers
+  int chunks;                                 // kGatherChunk-row chunks per unit
+};
 int launch_key_norms(const void* K, const Geom& g, int dtype, const int32_t* len_dev, int max_len,
                      float* sumsq, long long ld_sumsq, float* norm_out, int key_mode,
-                     const SelectArgs* select, cudaStream_t s);
+                     const SelectArgs* select, const CopyArgs* copy, cudaStream_t s);
 int launch_select_compact(const void* K, const void* V, const Geom& gi, int dtype,
                           const int32_t* len_dev, const int32_t* keep_dev,
                           const int32_t* keep_unit_dev, int max_len,

@@ -29,16 +29,93 @@ __device__ __forceinline__ void publish_kept_len(const SelectArgs& sel, long lon
   if (h == 0 && sel.kept_len_dev) sel.kept_len_dev[bl] = keep;
 }
 
+// One kGatherChunk-row chunk of an uncompressed unit, copied whole: K and V rows to the same
+// slots of the output cache, idx = the row's own position, key computed from the row on the way.
+template <typename T, int D>
+__device__ __forceinline__ void copy_whole_chunk(const T* __restrict__ K, const T* __restrict__ V,
+                                                 const Geom& gi, const CopyArgs& cp,
+                                                 const int32_t* __restrict__ len_dev, int max_len,
+                                                 const LayerMask& unc, int c) {
+  constexpr int EPV = Elem<T>::kPerVec;
+  constexpr int LPR = D / EPV;
+  constexpr int RPS = kNormThreads / LPR;
+  constexpr int U = 4;
+  __shared__ long long s_cin, s_cout, s_cmeta;
+  __shared__ int s_c[3];
+  const int tid = threadIdx.x;
+  if (tid == 0) {
+    const int chunk = c % cp.chunks;
+    const long long uu = c / cp.chunks;
+    const int h = (int)(uu % gi.H);
+    const int li = (int)((uu / gi.H) % cp.n_unc);
+    const int b = (int)(uu / ((long long)gi.H * cp.n_unc));
+    int l = 0, seen = -1;                               // the li-th layer of the list
+    for (int x = 0; x < gi.L; ++x)
+      if (unc.test(x) && ++seen == li) { l = x; break; }
+    const long long bl = (long long)b * gi.L + l;
+    const int len = max(0, min(len_dev[b], min(max_len, gi.cap(bl))));
+    s_c[0] = chunk * kGatherChunk;
+    s_c[1] = min(len, s_c[0] + kGatherChunk);
+    s_c[2] = cp.go.cap(bl);
+    s_cin = gi.base(b, l, h);
+    s_cout = cp.go.base(b, l, h);
+    s_cmeta = cp.go.meta(bl * gi.H + h);
+  }
+  __syncthreads();
+  const int t0 = s_c[0], t_end = s_c[1], out_cap = s_c[2];
+  if (t0 >= t_end) return;
+  const int piece = tid % LPR, sub = tid / LPR;
+  const T* kin = K + s_cin + (long long)piece * EPV;
+  const T* vin = V + s_cin + (long long)piece * EPV;
+  T* kout = static_cast<T*>(cp.K_out) + s_cout + (long long)piece * EPV;
+  T* vout = static_cast<T*>(cp.V_out) + s_cout + (long long)piece * EPV;
+  const long long meta = s_cmeta;
+  for (int jb = t0; jb < t_end; jb += RPS * U) {         // bounds uniform over the block
+    uint4 vk[U], vv[U];
+#pragma unroll
+    for (int i = 0; i < U; ++i) {
+      const int t = jb + i * RPS + sub;
+      vk[i] = make_uint4(0, 0, 0, 0);
+      vv[i] = make_uint4(0, 0, 0, 0);
+      if (t < t_end) {
+        vk[i] = ld_stream(kin + (long long)t * gi.st);
+        vv[i] = ld_stream(vin + (long long)t * gi.st);
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < U; ++i) {
+      const int t = jb + i * RPS + sub;
+      const float s = piece_sumsq_reduce<T, LPR>(vk[i]);
+      if (t < t_end && t < out_cap) {
+        st_stream(kout + (long long)t * cp.go.st, vk[i]);
+        st_stream(vout + (long long)t * cp.go.st, vv[i]);
+        if (piece == 0) {
+          cp.idx_out[meta + t] = t;
+          cp.sumsq_out[meta + t] = s;
+        }
+      }
+    }
+  }
+}
+
 template <typename T, int D, int MODE>
 __global__ void __launch_bounds__(kNormThreads)
 key_norms_kernel(const T* __restrict__ K, Geom g, const int32_t* __restrict__ len_dev,
                  float* __restrict__ sumsq, long long ld, float* __restrict__ norm_out,
-                 int chunks_per_unit, int max_len, SelectArgs sel) {
+                 int chunks_per_unit, int max_len, SelectArgs sel, CopyArgs cp) {
   constexpr int LPR = D / Elem<T>::kPerVec;            // lanes per row
   constexpr int RPS = kNormThreads / LPR;              // row groups of the CTA
   constexpr int U = kNormUnroll;
   constexpr bool SEL = MODE != kKeysOnly;
   static_assert(U <= LPR, "the halving reduction needs at least as many lanes as rows");
+  if constexpr (MODE == kKeysFromK) {
+    const int norm_blocks = (int)gridDim.x - cp.n_blocks;
+    if ((int)blockIdx.x >= norm_blocks) {                // trailing blocks: uncompressed layers
+      copy_whole_chunk<T, D>(K, static_cast<const T*>(cp.V), g, cp, len_dev, max_len, sel.unc,
+                             (int)blockIdx.x - norm_blocks);
+      return;
+    }
+  }
   const long long unit = blockIdx.x / chunks_per_unit;
   const int chunk = blockIdx.x % chunks_per_unit;
   const int tid = threadIdx.x;
@@ -69,7 +146,8 @@ key_norms_kernel(const T* __restrict__ K, Geom g, const int32_t* __restrict__ le
       if (chunk == 0) {
         const int keep = min(len, out_cap);
         identity_unit<kNormThreads>(len, keep, true, sel.unit_rec + unit,
-                                    sel.chunk_rec + unit * sel.n_chunks);
+                                    sel.chunk_rec + unit * sel.n_chunks,
+                                    MODE == kKeysFromK && whole && cp.n_blocks > 0);
         if (tid == 0) publish_kept_len(sel, unit, b * g.L + l, h, keep);
       }
       return;
@@ -159,29 +237,31 @@ key_norms_kernel(const T* __restrict__ K, Geom g, const int32_t* __restrict__ le
 template <typename T, int D>
 static int launch_norms_t(const void* K, const Geom& g, const int32_t* len_dev, int max_len,
                           float* sumsq, long long ld, float* norm_out, int key_mode,
-                          const SelectArgs* select, cudaStream_t s) {
+                          const SelectArgs* select, const CopyArgs* copy, cudaStream_t s) {
   const long long units = (long long)g.B * g.L * g.H;
   int chunks = (max_len + kNormRowsPerCta - 1) / kNormRowsPerCta;
   if (key_mode != kKeysOnly && chunks < 1) chunks = 1;   // records are written even for max_len 0
   if (key_mode == kKeysGiven) chunks = 1;                // one CTA per unit: selection only
   if (units == 0 || chunks == 0) return L2KV_OK;
-  const long long blocks = units * chunks;
+  CopyArgs cp = copy ? *copy : CopyArgs{};
+  if (key_mode != kKeysFromK) cp.n_blocks = 0;
+  const long long blocks = units * chunks + cp.n_blocks;
   if (blocks > 0x7fffffffLL) return L2KV_ERR_OUT_OF_RANGE;
   const T* Kt = static_cast<const T*>(K);
   const SelectArgs sa = select ? *select : SelectArgs{};
   const unsigned nb = (unsigned)blocks;
   switch (key_mode) {
     case kKeysOnly:
-      key_norms_kernel<T, D, kKeysOnly><<<nb, kNormThreads, 0, s>>>(Kt, g, len_dev, sumsq, ld, norm_out, chunks, max_len, sa);
+      key_norms_kernel<T, D, kKeysOnly><<<nb, kNormThreads, 0, s>>>(Kt, g, len_dev, sumsq, ld, norm_out, chunks, max_len, sa, cp);
       break;
     case kKeysFromK:
-      key_norms_kernel<T, D, kKeysFromK><<<nb, kNormThreads, 0, s>>>(Kt, g, len_dev, sumsq, ld, norm_out, chunks, max_len, sa);
+      key_norms_kernel<T, D, kKeysFromK><<<nb, kNormThreads, 0, s>>>(Kt, g, len_dev, sumsq, ld, norm_out, chunks, max_len, sa, cp);
       break;
     case kKeysRandom:
-      key_norms_kernel<T, D, kKeysRandom><<<nb, kNormThreads, 0, s>>>(Kt, g, len_dev, sumsq, ld, norm_out, chunks, max_len, sa);
+      key_norms_kernel<T, D, kKeysRandom><<<nb, kNormThreads, 0, s>>>(Kt, g, len_dev, sumsq, ld, norm_out, chunks, max_len, sa, cp);
       break;
     case kKeysGiven:
-      key_norms_kernel<T, D, kKeysGiven><<<nb, kNormThreads, 0, s>>>(Kt, g, len_dev, sumsq, ld, norm_out, chunks, max_len, sa);
+      key_norms_kernel<T, D, kKeysGiven><<<nb, kNormThreads, 0, s>>>(Kt, g, len_dev, sumsq, ld, norm_out, chunks, max_len, sa, cp);
       break;
     default:
       return L2KV_ERR_INVALID_ARG;
@@ -191,9 +271,9 @@ static int launch_norms_t(const void* K, const Geom& g, const int32_t* len_dev, 
 
 int launch_key_norms(const void* K, const Geom& g, int dtype, const int32_t* len_dev, int max_len,
                      float* sumsq, long long ld_sumsq, float* norm_out, int key_mode,
-                     const SelectArgs* select, cudaStream_t s) {
+                     const SelectArgs* select, const CopyArgs* copy, cudaStream_t s) {
 #define L2KV_KN(T, D) \
-  return launch_norms_t<T, D>(K, g, len_dev, max_len, sumsq, ld_sumsq, norm_out, key_mode, select, s)
+  return launch_norms_t<T, D>(K, g, len_dev, max_len, sumsq, ld_sumsq, norm_out, key_mode, select, copy, s)
   if (dtype == L2KV_BF16) {
     if (g.D == 128) L2KV_KN(__nv_bfloat16, 128);
     if (g.D == 64) L2KV_KN(__nv_bfloat16, 64);

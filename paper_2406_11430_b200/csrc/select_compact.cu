@@ -43,7 +43,7 @@ gather_kernel(const T* __restrict__ K, const T* __restrict__ V, Geom gi, T* __re
   if (t0 >= len) return;
   const int t_end = min(len, t0 + kGatherChunk);
   const UnitRec ur = unit_rec[unit];
-  if (ur.n_keep == 0) return;
+  if (ur.n_keep == 0 || (ur.flags & kFlagCopied)) return;   // nothing kept, or copied by the norm pass
   const int2 cr = chunk_rec[unit * n_chunks + chunk];
   const int tid = threadIdx.x;
   const float* key = sumsq + (ld >= 0 ? unit * ld : gi.meta(unit));
@@ -173,8 +173,16 @@ static int launch_sc_t(const void* K, const void* V, const Geom& gi, const int32
   sel.status_word = reinterpret_cast<int32_t*>(ws);
   // Keys of the layers that are compressed (the others are copied whole), and, as each
   // unit's last chunk of keys lands, its selection.
+  CopyArgs cp{};
+  int n_unc = 0;
+  for (int l = 0; l < gi.L; ++l) n_unc += unc.test(l) ? 1 : 0;
+  const long long copy_blocks = (long long)gi.B * n_unc * gi.H * plan.n_chunks;
+  if (key_mode == kKeysFromK && max_len > 0 && copy_blocks > 0 && copy_blocks < 0x3fffffffLL) {
+    cp.V = V; cp.K_out = K_out; cp.V_out = V_out; cp.idx_out = idx_out; cp.sumsq_out = sumsq_out;
+    cp.go = go; cp.n_blocks = (int)copy_blocks; cp.n_unc = n_unc; cp.chunks = plan.n_chunks;
+  }
   const int rc = launch_key_norms(K, gi, Elem<T>::kDtype, len_dev, max_len, keys, ld, nullptr,
-                                  key_mode, &sel, s);
+                                  key_mode, &sel, &cp, s);
   if (rc != L2KV_OK) return rc;
   if (max_len > 0) {
     gather_kernel<T, D><<<(unsigned)(units * plan.n_chunks), kGatherThreads, 0, s>>>(

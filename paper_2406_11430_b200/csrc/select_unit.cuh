@@ -180,11 +180,11 @@ __device__ void select_unit(SelectSmem& sm, const float* __restrict__ key, int l
 // Record of a unit whose valid tokens are all kept (uncompressed layer, or keep == len).
 template <int NT>
 __device__ void identity_unit(int len, int keep, bool keys_missing, UnitRec* __restrict__ rec,
-                              int2* __restrict__ crec) {
+                              int2* __restrict__ crec, bool copied = false) {
   const int my_chunks = (len + kGatherChunk - 1) / kGatherChunk;
   if (threadIdx.x == 0) {
     UnitRec r; r.thr = 0xffffffffu; r.admit = 0; r.n_keep = keep;
-    r.flags = kFlagIdentity | (keys_missing ? kFlagNoKeys : 0u);
+    r.flags = kFlagIdentity | (keys_missing ? kFlagNoKeys : 0u) | (copied ? kFlagCopied : 0u);
     *rec = r;
   }
   for (int c = threadIdx.x; c < my_chunks; c += NT) crec[c] = make_int2(c * kGatherChunk, 0);
