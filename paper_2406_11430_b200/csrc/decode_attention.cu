@@ -320,7 +320,8 @@ decode_split_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16
                         LenView cur_len_dev, int max_len, float scale_log2e,
                         float* __restrict__ partial, int n_splits,
                         const __grid_constant__ CUtensorMap map_k,
-                        const __grid_constant__ CUtensorMap map_v, int32_t* __restrict__ status_word) {
+                        const __grid_constant__ CUtensorMap map_v, int32_t* __restrict__ status_word,
+                        int32_t* __restrict__ tickets, float* __restrict__ out) {
   constexpr int D = 128;
   constexpr int NW = kMmaWarps;
   constexpr int TPT = kDecodeChunk / kMmaThreads;        // tokens per thread in phase 2
@@ -342,7 +343,12 @@ decode_split_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16
   const int b = (int)(bl / g.L);
   const int n = max(0, min(cur_len_dev.at(bl, h, g.H), min(max_len, g.cap(bl))));
   const int t0 = split * kDecodeChunk;
-  if (t0 >= n) return;
+  if (t0 >= n) {
+    // an empty cache has no split to merge: with the merge inside this kernel, split 0 writes the zeros
+    if (tickets && split == 0 && n == 0)
+      for (int o = threadIdx.x; o < G * D; o += kMmaThreads) out[(bl * g.Hq + h * G) * D + o] = 0.f;
+    return;
+  }
   if constexpr (TMA) {
     // A copy that timed out in an earlier CTA marks the workspace; the rest of the grid
     // then leaves at once instead of timing out CTA by CTA.
@@ -597,6 +603,49 @@ decode_split_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16
     p[0] = s_m[tid];
     p[1] = s_l[tid];
   }
+  if (!tickets) return;                                    // the caller merges with a kernel of its own
+
+  // ---- merge, by the split that finishes last (a ticket per unit; nobody waits) ----------------
+  // out = sum_s 2^(m_s - m) acc_s / sum_s 2^(m_s - m) l_s over the unit's splits, in split order:
+  // the same sums as decode_combine_kernel, whichever block happens to form them.
+  __shared__ int s_last;
+  __threadfence();                                         // this split's partial is visible device-wide
+  __syncthreads();
+  const int ns = (n + kDecodeChunk - 1) / kDecodeChunk;    // splits of this unit that hold tokens
+  if (tid == 0) s_last = (ns == 1) || (atomicAdd(tickets + unit, 1) == ns - 1);
+  __syncthreads();
+  if (!s_last) return;
+  if constexpr (TMA) {
+    // a split of this grid gave up: its partial means nothing, so no output (the status is set)
+    if (!copy_ok || (status_word && *reinterpret_cast<volatile int32_t*>(status_word + 2) != 0)) return;
+  }
+  __threadfence();                                         // see the other splits' partials
+  float* s_w = s_sc;                                       // [G][ns] weights, then [G] denominators
+  for (int i = tid; i < G * ns; i += kMmaThreads) {
+    const int head = i / ns, sp = i % ns;
+    s_w[i] = __ldcg(partial + ((bl * g.Hq + h * G + head) * n_splits + sp) * (long long)(D + 2));
+  }
+  __syncthreads();
+  if (tid < G) {
+    float m = -INFINITY;
+    for (int sp = 0; sp < ns; ++sp) m = fmaxf(m, s_w[tid * ns + sp]);
+    s_m[tid] = m;
+  }
+  __syncthreads();
+  for (int i = tid; i < G * ns; i += kMmaThreads) s_w[i] = exp2f(s_w[i] - s_m[i / ns]);
+  __syncthreads();
+  for (int o = tid; o < G * D; o += kMmaThreads) {
+    const int head = o / D, d = o % D;
+    const float* p = partial + (bl * g.Hq + h * G + head) * n_splits * (long long)(D + 2);
+    float den = 0.f, num = 0.f;
+    for (int sp = 0; sp < ns; ++sp) {
+      const float wgt = s_w[head * ns + sp];
+      den = fmaf(wgt, __ldcg(p + sp * (D + 2) + 1), den);
+      num = fmaf(wgt, __ldcg(p + sp * (D + 2) + 2 + d), num);
+    }
+    out[(bl * g.Hq + h * G + head) * D + d] = num / den;
+  }
+  if (tid == 0 && ns > 1) tickets[unit] = 0;               // counters rest at zero between calls
 }
 
 template <int G>
@@ -607,6 +656,12 @@ static int launch_dec_mma(const void* q, const void* K, const void* V, const Geo
   if (units == 0) return L2KV_OK;
   if (units * plan.n_splits > 0x7fffffffLL) return L2KV_ERR_OUT_OF_RANGE;
   float* partial = reinterpret_cast<float*>(ws + plan.partial_off);
+  // The per-unit completion counters of the workspace let the last split of a unit merge its
+  // partials inside the split kernel; a scratch without them (the built-in one) gets the merge
+  // kernel instead.  The weights of the merge reuse the score buffer: G * splits floats.
+  int32_t* tickets = plan.ticket_off + (size_t)units * 4 <= plan.partial_off && plan.n_splits <= kDecodeChunk
+                         ? reinterpret_cast<int32_t*>(ws + plan.ticket_off) : nullptr;
+  if (std::getenv("L2KV_DECODE_MERGE_KERNEL")) tickets = nullptr;   // the two-kernel form, for comparison
   constexpr int smem_bytes = 128 + kStages * kStageTok * kRowBytes + G * kScLd * 4;
   if (max_len > 0) {
     // K and V rows reach shared memory through TMA tensor maps; L2KV_DECODE_COPY=cpasync (or a
@@ -625,8 +680,10 @@ static int launch_dec_mma(const void* q, const void* K, const void* V, const Geo
         static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(K),
         static_cast<const __nv_bfloat16*>(V), g, cur_len_dev, max_len, scale * kLog2e, partial,
         plan.n_splits, map_k, map_v,
-        plan.partial_off >= (size_t)kStatusBytes ? reinterpret_cast<int32_t*>(ws) : nullptr);
+        plan.partial_off >= (size_t)kStatusBytes ? reinterpret_cast<int32_t*>(ws) : nullptr,
+        tickets, out);
     if (cudaGetLastError() != cudaSuccess) return L2KV_ERR_CUDA;
+    if (tickets) return L2KV_OK;                           // merged by the last split of every unit
   }
   decode_combine_kernel<128><<<(unsigned)((long long)g.B * g.L * g.Hq), 128, 0, s>>>(
       partial, cur_len_dev, max_len, g, plan.n_splits, out,

@@ -66,6 +66,7 @@ extern "C" int l2kv_decode_attention_static(const void* q, const void* K_c, cons
   const size_t need = plan.total - plan.partial_off;
   if (need > (size_t)L2KV_STATIC_SCRATCH_BYTES - kStatusBytes) return L2KV_ERR_WORKSPACE_TOO_SMALL;
   plan.partial_off = kStatusBytes;
+  plan.ticket_off = plan.partial_off;         // no completion counters here: the merge is a kernel
 
   void* scratch = nullptr;
   rc = scratch_address(&scratch);

@@ -269,6 +269,22 @@ def test_attention_copy_paths_agree(l2, monkeypatch):
         assert np.array_equal(gpu_attention(l2, q, Kp, Vp, cur), a)
 
 
+def test_attention_merge_inside_the_split_kernel_equals_the_merge_kernel(l2, monkeypatch):
+    """The partial results of a unit's splits are merged by whichever split finishes last; the
+    sums are formed in split order either way, so the result has the bits of the two-kernel form
+    (split kernel, then merge kernel).  Ragged lengths: 0, 1, exactly one split, many splits."""
+    w = synth.WORKLOADS[2].scaled(B=2, L=3, T=5000)
+    K, V, _, _ = make(w)
+    q = synth.make_query(w, 0, DEV)
+    cur = [[5000, 0, 1024], [1, 1025, 3333]]
+    a = gpu_attention(l2, q, K, V, cur)
+    b = gpu_attention(l2, q, K, V, cur)                      # and it is deterministic
+    monkeypatch.setenv("L2KV_DECODE_MERGE_KERNEL", "1")
+    c = gpu_attention(l2, q, K, V, cur)
+    assert np.array_equal(a, b) and np.array_equal(a, c)
+    assert not a[0, 1].any()
+
+
 def test_attention_special_cases(l2):
     w = synth.WORKLOADS[2].scaled(B=1, L=1, T=2048)
     K, V, Kn, Vn = make(w)
