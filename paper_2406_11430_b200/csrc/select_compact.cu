@@ -3,7 +3,7 @@
 //   selection       runs inside the norm pass (key_norms.cu, select_unit.cuh): exact k-th
 //                   smallest of the ordering keys by a most-significant-digit radix select
 //                   (4 passes of 8 bits), then per-chunk slot bases by a scan.
-//   gather_kernel   one CTA per (unit, chunk of input tokens): rebuilds the keep flags
+//   gather_kernel   one CTA per (unit, chunk of input tokens; two chunks where little is kept): rebuilds the keep flags
 //                   from the threshold, ranks the kept tokens with a block scan and copies
 //                   their K and V rows (16-byte pieces, LPR lanes per row) to the dense,
 //                   position-ordered output together with the index map and the keys.
@@ -16,6 +16,16 @@ namespace l2kv {
 
 constexpr int kGatherThreads = 256;
 constexpr int kGatherUnroll = 4;
+// Chunks of kGatherChunk input tokens that one CTA may take.  The grid has one CTA per chunk.  In
+// a unit that keeps at most a quarter of its tokens a CTA would move few rows between three
+// dependent round trips to memory (keys, rows in, rows out) and the kernel would idle on latency
+// (keep 0.1: 4.4 TB/s), so there the CTAs of even chunks take the next chunk as well and the odd
+// ones leave at once; elsewhere one chunk per CTA measured fastest.
+#ifndef L2KV_GATHER_GROUP
+#define L2KV_GATHER_GROUP 2
+#endif
+constexpr int kGatherGroup = L2KV_GATHER_GROUP;
+constexpr int kGatherSpan = kGatherGroup * kGatherChunk;   // input tokens per CTA
 
 template <typename T, int D>
 __global__ void __launch_bounds__(kGatherThreads)
@@ -27,13 +37,14 @@ gather_kernel(const T* __restrict__ K, const T* __restrict__ V, Geom gi, T* __re
               [[maybe_unused]] int32_t* __restrict__ status_word) {
   constexpr int LPR = D / Elem<T>::kPerVec;
   constexpr int RPS = kGatherThreads / LPR;              // rows per copy step of the CTA
-  constexpr int TPT = kGatherChunk / kGatherThreads;     // tokens ranked per thread
-  __shared__ int s_src[kGatherChunk];                    // kept tokens of this chunk, in order
+  constexpr int TPT = kGatherSpan / kGatherThreads;      // tokens ranked per thread
+  static_assert(kGatherSpan < 65536, "the packed (below, equal) counts hold 16 bits each");
+  __shared__ int s_src[kGatherSpan];                     // kept tokens of this CTA's span, in order
   __shared__ int s_warp[kGatherThreads / 32];
   __shared__ int s_total;
 
   const long long unit = blockIdx.x / n_chunks;
-  const int chunk = blockIdx.x % n_chunks;
+  const int chunk = blockIdx.x % n_chunks;               // first (or only) chunk of this CTA
   const int h = (int)(unit % gi.H);
   const int l = (int)((unit / gi.H) % gi.L);
   const int b = (int)(unit / ((long long)gi.H * gi.L));
@@ -41,9 +52,11 @@ gather_kernel(const T* __restrict__ K, const T* __restrict__ V, Geom gi, T* __re
   const int len = max(0, min(len_dev[b], min(max_len, gi.cap(bl))));
   const int t0 = chunk * kGatherChunk;
   if (t0 >= len) return;
-  const int t_end = min(len, t0 + kGatherChunk);
   const UnitRec ur = unit_rec[unit];
   if (ur.n_keep == 0 || (ur.flags & kFlagCopied)) return;   // nothing kept, or copied by the norm pass
+  const int my_chunks = (long long)ur.n_keep * 4 <= len ? kGatherGroup : 1;
+  if (chunk % my_chunks) return;                         // a neighbour takes this chunk
+  const int t_end = min(len, t0 + my_chunks * kGatherChunk);
   const int2 cr = chunk_rec[unit * n_chunks + chunk];
   const int tid = threadIdx.x;
   const float* key = sumsq + (ld >= 0 ? unit * ld : gi.meta(unit));
@@ -56,10 +69,34 @@ gather_kernel(const T* __restrict__ K, const T* __restrict__ V, Geom gi, T* __re
     // Rank this chunk's tokens: packed (below, equal) counts, one exclusive block scan.
     uint32_t kb[TPT];
     int cnt = 0;                                         // low 16 bits: equal, high: below
+    // a thread's TPT tokens are consecutive: 16-byte key loads where the array allows them
+    [[maybe_unused]] const bool vec = (reinterpret_cast<uintptr_t>(key + t0) & 15u) == 0;
+#pragma unroll
+    for (int i = 0; i < TPT; ++i) kb[i] = 0xffffffffu;
+    if constexpr (TPT % 4 == 0) {
+#pragma unroll
+      for (int i = 0; i < TPT; i += 4) {
+        const int t = t0 + tid * TPT + i;
+        if (vec && t + 3 < t_end) {
+          const float4 v = *reinterpret_cast<const float4*>(key + t);
+          kb[i] = order_bits(v.x, policy);     kb[i + 1] = order_bits(v.y, policy);
+          kb[i + 2] = order_bits(v.z, policy); kb[i + 3] = order_bits(v.w, policy);
+        } else {
+#pragma unroll
+          for (int j = 0; j < 4; ++j)
+            if (t + j < t_end) kb[i + j] = order_bits(key[t + j], policy);
+        }
+      }
+    } else {
+#pragma unroll
+      for (int i = 0; i < TPT; ++i) {
+        const int t = t0 + tid * TPT + i;
+        if (t < t_end) kb[i] = order_bits(key[t], policy);
+      }
+    }
 #pragma unroll
     for (int i = 0; i < TPT; ++i) {
       const int t = t0 + tid * TPT + i;
-      kb[i] = t < t_end ? order_bits(key[t], policy) : 0xffffffffu;
       if (t < t_end) cnt += (kb[i] < ur.thr ? 0x10000 : 0) + (kb[i] == ur.thr ? 1 : 0);
     }
     int inc = cnt;
