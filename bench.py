@@ -39,7 +39,7 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes (read + written) per algorithmic byte of the dominant kernel, from an ncu capture of
 # the decode split kernel on a 4-layer case of the benchmark workload (the traffic is
 # proportional to the tokens streamed).  Set to None whenever that kernel changes.
-DECODE_TRAFFIC_RATIO = 1.0058
+DECODE_TRAFFIC_RATIO = 1.0069
 
 
 def workload(args):
