@@ -417,6 +417,12 @@ constexpr int kPfSubTile = 2 * kPfSubHalf;      // both halves of the head dimen
 constexpr uint32_t kIdescQK64 =
     (1u << 4) | (1u << 7) | (1u << 10) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
 constexpr int kPfStages = 4;                    // K tiles (and V tiles) in flight
+// 1 (default): Q K(j+2)^T is issued right behind P(j) V(j) although it overwrites the columns that
+// P(j) V(j) reads its weights from -- see the issuing thread.  0: wait for P(j) V(j) to be
+// committed first (8-12 % slower; the form to fall back to if the assumption is ever in doubt).
+#ifndef L2KV_PREFIX_MMA_IN_ORDER
+#define L2KV_PREFIX_MMA_IN_ORDER 1
+#endif
 constexpr int kPfPipeTmemCols = 512;            // two query tiles x (2 x 64 score + 128 output columns)
 
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
@@ -615,10 +621,18 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
         }
         umma_commit(bar_o);
         umma_commit(bar_vfree(j % NS));
+#if L2KV_PREFIX_MMA_IN_ORDER
+        // The score buffer that P(j) V(j) reads its weights from takes sub-block j + 2.  The two
+        // operations are issued by this one thread to this CTA's tensor core, which executes
+        // what it is given in issue order: Q K(j+2)^T is queued right behind P(j) V(j) and
+        // cannot overwrite the weights before they have been read.
+        if (j + 2 < nb) issue_qk(j + 2);
+#else
         // P(j) V(j) done: the score buffer it read its weights from takes sub-block j + 2
         ok = mbar_wait<kPfPolls>(bar_o, (uint32_t)j & 1u);
         if (!ok) break;
         if (j + 2 < nb) { tc_fence_after(); issue_qk(j + 2); }
+#endif
       }
       if (!ok) s_fail = 1;
     }
