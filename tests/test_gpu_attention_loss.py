@@ -26,7 +26,9 @@ def run(l2, q, K, cur, max_len, curves=True):
 
 @pytest.mark.parametrize("dtype,D,Hkv,Hq,T", [("bf16", 128, 2, 8, 5000), ("f32", 64, 4, 4, 1024),
                                              ("bf16", 64, 2, 2, 4097), ("f32", 128, 1, 2, 700),
-                                             ("bf16", 128, 1, 2, 20000), ("bf16", 128, 1, 1, 70000)])
+                                             ("bf16", 128, 1, 2, 20000), ("bf16", 128, 1, 1, 70000),
+                                             ("bf16", 128, 1, 12, 3000), ("f32", 64, 2, 6, 2500),
+                                             ("bf16", 128, 1, 3, 33000), ("bf16", 128, 2, 4, 32768)])
 def test_attention_loss_matches_oracle(dtype, D, Hkv, Hq, T):
     import paper_2406_11430_b200 as l2
     w = synth.WORKLOADS[2].scaled(dtype=dtype, D=D, Hkv=Hkv, Hq=Hq, B=2, L=2, T=T)
