@@ -340,7 +340,7 @@ def run_gpu(args):
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
             "data": "synthetic", "config": cfg,
             "compress": stages["compress"], "decode": stages["decode"],
-            "roofline": {"bound": "hbm", "kernel": "decode_split_mma_kernel (+ combine, timed together)",
+            "roofline": {"bound": "hbm", "kernel": "decode_split_mma_kernel (the merge of the splits runs inside it)",
                          "achieved": round(dec_gbs, 1), "peak": peak, "peak_kind": peak_kind,
                          "unit": "GB/s", "frac": round(dec_gbs / peak, 4),
                          "traffic": args.traffic if args.traffic is not None else
