@@ -394,6 +394,46 @@ def test_append_evict_stream(l2, dtype, D):
     assert l2.read_device_status(ws) == 0
 
 
+def test_append_evict_stream_against_fp64_keys(l2):
+    """The same stream against the oracle with its fp64 keys: after every append the kept sets
+    must agree outside the 1e-6 tie band around the threshold norm (the kernel decides in fp32)."""
+    steps, T0 = 64, 600
+    w = synth.WORKLOADS[4].scaled(B=2, L=3, Hkv=2, Hq=8, T=T0, ragged_lo=0)
+    K, V, Kn, Vn = make(w)
+    lens, budget = [600, 250], [300, 125]
+    t_cap = T0 + steps
+    dev, _ = gpu_compress(l2, K, V, lens, budget, unc=(0,), t_cap_out=t_cap)
+    st = _oracle_state(oracle.compress(Kn, Vn, w.dtype, lens, budget, (0,), key_mode=0, t_cap_out=T0),
+                       t_cap)
+    ws = l2.new_workspace(l2.Layout(dev["K_c"], q_heads=w.Hq), t_cap, DEV)
+    bud = i32(budget)
+    rows = [[Kn[b, :, :, :lens[b]]] for b in range(w.B)]          # every key a unit has seen, by position
+    swaps = 0
+    for s in range(steps):
+        k, v = synth.make_new_kv(w, s, DEV)
+        kn, vn = synth.to_numpy(k), synth.to_numpy(v)
+        pos = [n + s for n in lens]
+        l2.append_evict(dev["K_c"], dev["V_c"], dev["idx"], dev["sumsq"], dev["kept_len"], bud,
+                        (0,), k, v, i32(pos), ws)
+        assert oracle.append_evict(st, w.dtype, budget, (0,), kn, vn, pos, key_mode=0) == 0
+        for b in range(w.B):
+            rows[b].append(kn[b][:, :, None, :])
+    torch.cuda.synchronize()
+    assert l2.read_device_status(ws) == 0
+    cur = dev["kept_len"].cpu().numpy()
+    assert np.array_equal(cur, st["cur_len"])
+    for b in range(w.B):
+        seen = np.concatenate(rows[b], axis=2)                    # [L, H, lens[b] + steps, D]
+        key64 = oracle.key_sumsq(seen[None], w.dtype)[0]
+        for l in range(1, w.L):                                   # layer 0 is uncompressed
+            n = int(cur[b, l])
+            assert n == budget[b]
+            for h in range(w.Hkv):
+                swaps += compare_with_band(dev["idx"][b, l, h, :n].cpu().numpy(), st["idx"][b, l, h, :n],
+                                           key64[l, h], n)
+    print(f"append/evict against fp64 keys: {swaps} swaps inside the tie band")
+
+
 def test_append_evict_overflow_sets_status(l2):
     w = synth.WORKLOADS[4].scaled(B=1, L=2, Hkv=2, Hq=8, T=64, ragged_lo=0)
     K, V, Kn, Vn = make(w)
