@@ -320,8 +320,10 @@ int l2kv_prefix_attention_flags(const void* q, const void* K_c, const void* V_c,
  * [batch, layers, q_heads, t_cap] receiving L^m / L^{m,ref} at index m - 1 (entries at
  * and beyond n untouched).  Sums are fp64 internally.  An empty cache gives Y = 0.
  * The workspace needs l2kv_attention_loss_workspace_bytes(lay, max_len) bytes (it is
- * separate from, and much larger than, the one of the other calls; no zeroing needed).
- * An analysis tool: it sorts every head's scores and is not tuned like the decode path. */
+ * separate from, and much larger than, the one of the other calls: about 8 bytes per cached
+ * token and query head; no zeroing needed).  The query heads of a KV head are scored from one
+ * read of its keys; every head's scores are then sorted (radix sort), so this is an analysis
+ * tool with the cost of a sort per head, not a step of the decode path. */
 int l2kv_attention_loss_workspace_bytes(const l2kv_layout* lay, int32_t max_len, size_t* bytes);
 int l2kv_attention_loss(const void* q, const void* K, const l2kv_layout* lay,
                         const int32_t* cur_len_dev, int32_t max_len, float scale,
