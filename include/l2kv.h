@@ -41,8 +41,8 @@
  *     is then a host upper bound of row_cap_dev.  Every per-row companion array of such a
  *     cache (idx, sumsq, the outputs of l2kv_key_norms) is dense [kv_heads, total_rows] with
  *     the same row axis.  Accepted by l2kv_key_norms, l2kv_select_compact (input, output or
- *     both), l2kv_decode_attention, l2kv_append_evict and their _per_head / _static forms;
- *     the prefix-attention and attention-loss calls return L2KV_ERR_UNSUPPORTED for it.
+ *     both), l2kv_decode_attention, l2kv_append_evict, their _per_head / _static forms and the
+ *     prefix-attention calls; l2kv_attention_loss returns L2KV_ERR_UNSUPPORTED for it.
  *   - `len_dev[b]` is the number of valid tokens of sequence b; `max_len` is a host
  *     upper bound on every length the call will meet (it sizes grids and scratch;
  *     device lengths above it are clamped to it).

@@ -309,9 +309,9 @@ def attention_loss(q, K, cur_len_dev, max_len, sumsq, alr_out, loss_out=None, lo
         _stream(stream)), "l2kv_attention_loss")
 
 
-def prefix_attention_workspace(K_c, q, max_len, device=None):
+def prefix_attention_workspace(K_c, q, max_len, device=None, rows=None):
     """A zeroed workspace large enough for prefix_attention to split the cache into chunks."""
-    lay = Layout(K_c, q_heads=q.shape[3])
+    lay = Layout(K_c, q_heads=q.shape[3], rows=rows)
     need = ctypes.c_size_t(0)
     _check(lib().l2kv_prefix_attention_workspace_bytes(lay.ref(), int(max_len), int(q.shape[2]),
                                                        ctypes.byref(need)),
@@ -323,11 +323,11 @@ PREFIX_CAUSAL, PREFIX_LEN_PER_HEAD, PREFIX_SPLIT_WEIGHTS = 1, 2, 4
 
 
 def prefix_attention_flags(q, K_c, V_c, cur_len_dev, max_len, out, flags, lse_out=None, scale=0.0,
-                           workspace=None, stream=None):
+                           workspace=None, stream=None, rows=None):
     """The general prefix-attention call: flags is a combination of PREFIX_CAUSAL,
     PREFIX_LEN_PER_HEAD and PREFIX_SPLIT_WEIGHTS (weights as two bf16 terms: the accuracy of
-    decode attention for a second P.V contraction)."""
-    lay = Layout(K_c, q_heads=q.shape[3])
+    decode attention for a second P.V contraction).  rows (Rows): the cache is packed."""
+    lay = Layout(K_c, q_heads=q.shape[3], rows=rows)
     _check(lib().l2kv_prefix_attention_flags(
         _ptr(q), _ptr(K_c), _ptr(V_c), lay.ref(), _ptr(cur_len_dev), int(max_len), int(q.shape[2]),
         float(scale), int(flags), _ptr(out), _ptr(lse_out), _ptr(workspace),

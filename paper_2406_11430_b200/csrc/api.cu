@@ -312,7 +312,7 @@ static int prefix_attention_impl(bool per_head, bool causal, bool split_weights,
   if (rc != L2KV_OK) return rc;
   rc = check_groups(lay);
   if (rc != L2KV_OK) return rc;
-  if (lay->dtype != L2KV_BF16 || lay->head_dim != 128 || packed(lay)) return L2KV_ERR_UNSUPPORTED;
+  if (lay->dtype != L2KV_BF16 || lay->head_dim != 128) return L2KV_ERR_UNSUPPORTED;
   if (max_len < 0 || n_queries < 0 || !(scale == scale)) return L2KV_ERR_INVALID_ARG;
   if (max_len > lay->t_cap) return L2KV_ERR_OUT_OF_RANGE;
   if (empty(lay) || n_queries == 0) return L2KV_OK;
@@ -354,7 +354,7 @@ int l2kv_prefix_attention_workspace_bytes(const l2kv_layout* lay, int32_t max_le
   if (max_len < 0 || n_queries < 0) return L2KV_ERR_INVALID_ARG;
   if (max_len > lay->t_cap) return L2KV_ERR_OUT_OF_RANGE;
   *bytes = (size_t)kStatusBytes;
-  if (empty(lay) || n_queries == 0 || lay->dtype != L2KV_BF16 || lay->head_dim != 128 || packed(lay))
+  if (empty(lay) || n_queries == 0 || lay->dtype != L2KV_BF16 || lay->head_dim != 128)
     return L2KV_OK;
   *bytes += prefix_attention_scratch(make_geom(*lay), n_queries, max_len);
   return L2KV_OK;

@@ -189,10 +189,14 @@ prefix_attention_basic_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n
   const int h = (int)(unit % g.H);
   const long long bl = unit / g.H;
   const int l = (int)(bl % g.L), b = (int)(bl / g.L);
-  const int n_all = max(0, min(cur_len_dev.at(bl, h, g.H), min(max_len, g.t_cap)));
+  const int n_all = max(0, min(cur_len_dev.at(bl, h, g.H), min(max_len, g.cap(bl))));
   // blockIdx.y: the chunk of split_len cached tokens this CTA covers (one chunk = the whole cache
   // unless the launcher split it; then out / lse_out are the per-chunk partial results)
   const int t_base = (int)blockIdx.y * split_len;
+  // tensor-map coordinates: (token, head, layer, batch) of a dense cache; a packed cache is one
+  // [H, total_rows] plane, so the first row of (b, l) joins the token coordinate
+  const int tm_row = (int)g.row0(bl) + t_base;
+  const int tm_l = g.row_off ? 0 : l, tm_b = g.row_off ? 0 : b;
   const int n = gridDim.y > 1 ? min(n_all, t_base + split_len) - t_base : n_all;
   if (gridDim.y > 1) {
     if (n <= 0) return;                                 // nothing cached in this chunk
@@ -256,13 +260,13 @@ prefix_attention_basic_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n
 
   auto load_k = [&](int kb) {                           // thread 0 only
     mbar_expect_tx(bar_k, kPfTileBytes);
-    tma_load_5d(sK, &map_k, bar_k, 0, t_base + kb * kPfRows, h, l, b);
-    tma_load_5d(sK + kPfHalf, &map_k, bar_k, 64, t_base + kb * kPfRows, h, l, b);
+    tma_load_5d(sK, &map_k, bar_k, 0, tm_row + kb * kPfRows, h, tm_l, tm_b);
+    tma_load_5d(sK + kPfHalf, &map_k, bar_k, 64, tm_row + kb * kPfRows, h, tm_l, tm_b);
   };
   auto load_v = [&](int kb) {
     mbar_expect_tx(bar_v, kPfTileBytes);
-    tma_load_5d(sV, &map_v, bar_v, 0, t_base + kb * kPfRows, h, l, b);
-    tma_load_5d(sV + kPfHalf, &map_v, bar_v, 64, t_base + kb * kPfRows, h, l, b);
+    tma_load_5d(sV, &map_v, bar_v, 0, tm_row + kb * kPfRows, h, tm_l, tm_b);
+    tma_load_5d(sV + kPfHalf, &map_v, bar_v, 64, tm_row + kb * kPfRows, h, tm_l, tm_b);
   };
   if (tid == 0) { load_k(0); load_v(0); }
   __syncwarp();
@@ -482,10 +486,14 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
   const int h = (int)(unit % g.H);
   const long long bl = unit / g.H;
   const int l = (int)(bl % g.L), b = (int)(bl / g.L);
-  const int n_all = max(0, min(cur_len_dev.at(bl, h, g.H), min(max_len, g.t_cap)));
+  const int n_all = max(0, min(cur_len_dev.at(bl, h, g.H), min(max_len, g.cap(bl))));
   // blockIdx.y: the chunk of split_len cached tokens this CTA covers (one chunk = the whole cache
   // unless the launcher split it; then out / lse_out are the per-chunk partial results)
   const int t_base = (int)blockIdx.y * split_len;
+  // tensor-map coordinates: (token, head, layer, batch) of a dense cache; a packed cache is one
+  // [H, total_rows] plane, so the first row of (b, l) joins the token coordinate
+  const int tm_row = (int)g.row0(bl) + t_base;
+  const int tm_l = g.row_off ? 0 : l, tm_b = g.row_off ? 0 : b;
   const int n = gridDim.y > 1 ? min(n_all, t_base + split_len) - t_base : n_all;
   if (gridDim.y > 1) {
     if (n <= 0) return;                                 // nothing cached in this chunk
@@ -579,8 +587,8 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
         if (!ok) break;
         const uint32_t dst = (is_k ? sK : sV) + st * kPfSubTile;
         mbar_expect_tx(full, kPfSubTile);
-        tma_load_5d(dst, map, full, 0, t_base + j * kPfSub, h, l, b);
-        tma_load_5d(dst + kPfSubHalf, map, full, 64, t_base + j * kPfSub, h, l, b);
+        tma_load_5d(dst, map, full, 0, tm_row + j * kPfSub, h, tm_l, tm_b);
+        tma_load_5d(dst + kPfSubHalf, map, full, 64, tm_row + j * kPfSub, h, tm_l, tm_b);
       }
       if (!ok) s_fail = 1;
     } else if ((tid & 31) == 0 && tile_active) {
@@ -753,14 +761,14 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
 // w_c = exp(lse_c - max lse), lse = max + log(sum_c w_c), over the chunks that hold cached rows.
 __global__ void __launch_bounds__(128)
 prefix_merge_kernel(const float* __restrict__ part_out, const float* __restrict__ part_lse,
-                    LenView cur_len_dev, int max_len, int t_cap, int H, int Hq, int n_queries,
+                    LenView cur_len_dev, int max_len, Geom g, int H, int Hq, int n_queries,
                     int split_len, long long rows_total, float* __restrict__ out,
                     float* __restrict__ lse_out, const int32_t* __restrict__ status_word) {
   if (status_word && status_word[2] != 0) return;       // a chunk gave up: no output
   const long long row = blockIdx.x;                      // ((b * L + l) * n_queries + s) * Hq + head
   const long long bl = row / ((long long)n_queries * Hq);
   const int h = (int)(row % Hq) / (Hq / H);
-  const int n = max(0, min(cur_len_dev.at(bl, h, H), min(max_len, t_cap)));
+  const int n = max(0, min(cur_len_dev.at(bl, h, H), min(max_len, g.cap(bl))));
   const int nc = (n + split_len - 1) / split_len;        // chunks with cached rows
   const int d = threadIdx.x;
   float m = -INFINITY;
@@ -874,7 +882,7 @@ static int launch_pf(const void* q, const void* K, const void* V, const Geom& g,
   if (cudaGetLastError() != cudaSuccess) return L2KV_ERR_CUDA;
   if (p.chunks > 1) {
     if (p.rows > 0x7fffffffLL) return L2KV_ERR_OUT_OF_RANGE;
-    prefix_merge_kernel<<<(unsigned)p.rows, 128, 0, s>>>(k_out, k_lse, cur_len_dev, max_len, g.t_cap,
+    prefix_merge_kernel<<<(unsigned)p.rows, 128, 0, s>>>(k_out, k_lse, cur_len_dev, max_len, g,
                                                          g.H, g.Hq, n_queries, p.split_len, p.rows,
                                                          out, lse_out, status_word);
     if (cudaGetLastError() != cudaSuccess) return L2KV_ERR_CUDA;

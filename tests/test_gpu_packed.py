@@ -184,7 +184,7 @@ def test_packed_overflow_sets_status_and_leaves_neighbours_alone(l2):
         assert np.array_equal(before["idx"][:, sl], after["idx"][:, sl])
 
 
-def test_packed_static_decode_and_unsupported_calls(l2):
+def test_packed_static_decode_and_unsupported_call(l2):
     w = synth.WORKLOADS[2].scaled(B=2, L=2, T=1300)
     pc, st = run_packed_pipeline(l2, w, lens=[1300, 700], keep=[650, 350], unc=(0,), steps=1)
     q = synth.make_query(w, 7, DEV)
@@ -196,9 +196,45 @@ def test_packed_static_decode_and_unsupported_calls(l2):
     assert torch.equal(got, want)
     import ctypes
     lay = l2.Layout(pc.K_c, q_heads=w.Hq, rows=pc.rows)
-    qp = torch.zeros((2, 2, 4, w.Hq, w.D), dtype=torch.bfloat16, device=DEV)
-    op = torch.zeros(qp.shape, dtype=torch.float32, device=DEV)
-    rc = l2.lib().l2kv_prefix_attention(qp.data_ptr(), pc.K_c.data_ptr(), pc.V_c.data_ptr(), lay.ref(),
-                                        pc.cur.data_ptr(), 100, 4, ctypes.c_float(0.0), op.data_ptr(),
-                                        None, None, 0, None)
-    assert rc == -2                                          # prefix attention takes dense caches only
+    need = ctypes.c_size_t(0)
+    rc = l2.lib().l2kv_attention_loss_workspace_bytes(lay.ref(), 100, ctypes.byref(need))
+    assert rc == 0
+    scratch = torch.empty(need.value, dtype=torch.uint8, device=DEV)
+    alr = torch.zeros((2, 2, w.Hq), dtype=torch.float32, device=DEV)
+    rc = l2.lib().l2kv_attention_loss(q.data_ptr(), pc.K_c.data_ptr(), lay.ref(), pc.cur.data_ptr(), 100,
+                                      ctypes.c_float(0.0), pc.sumsq.data_ptr(), alr.data_ptr(), None, None,
+                                      scratch.data_ptr(), scratch.numel(), None)
+    assert rc == -2                                          # the attention-loss analysis takes dense caches only
+
+def test_packed_prefix_attention(l2):
+    """Several new queries per (b, l) over a packed compressed cache, plain and causal, both weight
+    precisions, against the packed oracle query by query; lengths differ per (b, l)."""
+    B, L, Hkv, Hq, D, Sq = 3, 2, 2, 8, 128, 40
+    w = synth.WORKLOADS[2].scaled(B=B, L=L, Hkv=Hkv, Hq=Hq, T=64)
+    caps = [[700, 90], [300, 1], [64, 1500]]
+    cur = np.array([[650, 90], [300, 0], [40, 1500]], dtype=np.int32)
+    rows_host = synth.packing(caps)
+    off, cap, total = rows_host
+    rows = l2.Rows(off, cap, total, DEV)
+    g = torch.Generator(device="cpu").manual_seed(7)
+    K = torch.randn((Hkv, total, D), generator=g).to(torch.bfloat16).to(DEV)
+    V = torch.randn((Hkv, total, D), generator=g).to(torch.bfloat16).to(DEV)
+    q = torch.randn((B, L, Sq, Hq, D), generator=g).to(torch.bfloat16).to(DEV)
+    Kn, Vn = synth.to_numpy(K), synth.to_numpy(V)
+    max_len = int(cap.max())
+    for causal in (False, True):
+        for weights, atol in (("split", 2e-3), ("single", 4e-3)):
+            flags = (l2.PREFIX_CAUSAL if causal else 0) | (l2.PREFIX_SPLIT_WEIGHTS if weights == "split" else 0)
+            out = torch.full(q.shape, float("nan"), dtype=torch.float32, device=DEV)
+            lse = torch.full(q.shape[:4], float("nan"), dtype=torch.float32, device=DEV)
+            ws = l2.prefix_attention_workspace(K, q, max_len, rows=rows)
+            l2.prefix_attention_flags(q, K, V, i32(cur), max_len, out, flags, lse_out=lse, workspace=ws, rows=rows)
+            torch.cuda.synchronize()
+            assert l2.read_device_status(ws) == 0
+            got = out.cpu().numpy()
+            for s in range(Sq):
+                n_s = np.maximum(cur - Sq + s + 1, 0) if causal else cur
+                want = oracle.attention_packed(synth.to_numpy(q[:, :, s].contiguous()), Kn, Vn, "bf16", rows_host,
+                                               n_s, nthreads=4)
+                assert_attention_close(got[:, :, s], want, atol=atol)
+            assert np.all(np.isneginf(lse.cpu().numpy()[1, 1]))      # the empty cache
