@@ -16,6 +16,9 @@
  *   - Pointers named *_dev, and all tensor pointers (K, V, q, outputs, workspace),
  *     are DEVICE pointers owned by the caller.  `const l2kv_layout*` and the
  *     `uncompressed_layers` list are HOST pointers read before the call returns.
+ *     Any memory the device can address will do: l2kv_select_compact, for one, may be given a
+ *     V cache that lies in mapped pinned host memory, and then reads only the rows it keeps
+ *     over the link.
  *   - The library allocates nothing and keeps no state.  Calls enqueue work on
  *     `stream` (a cudaStream_t passed as void*; NULL = the default stream) and
  *     return at once; outputs are valid in stream order.

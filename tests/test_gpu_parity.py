@@ -341,6 +341,20 @@ def test_compress_then_attend_pipeline(l2):
         assert_attention_close(out, want)
 
 
+def test_compress_reads_v_from_pinned_host_memory(l2):
+    """V left in pinned host memory: the compression reads the rows it keeps in place; same result."""
+    w = synth.WORKLOADS[2].scaled(B=2, L=3, T=1500)
+    K, V, Kn, Vn = make(w)
+    lens, keep = [1500, 900], [700, 450]
+    dev, host = gpu_compress(l2, K, V, lens, keep, unc=(0,))
+    V_host = torch.empty(V.shape, dtype=V.dtype, pin_memory=True)
+    V_host.copy_(V)
+    torch.cuda.synchronize()
+    dev2, host2 = gpu_compress(l2, K, V_host, lens, keep, unc=(0,))
+    for name in ("K_c", "V_c", "idx", "kept_len"):
+        assert np.array_equal(host[name], host2[name]), name
+
+
 # -------------------------------------------------------------- append/evict
 
 def _oracle_state(r, t_cap):
