@@ -197,6 +197,8 @@ class Job:
         self.q = torch.stack([synth.make_query(ws, s, device) for s in range(w.decode_steps)])
         self.out = torch.zeros((w.decode_steps, w.B, w.L, w.Hq, w.D), dtype=torch.float32,
                                device=device)
+        self.q_step = list(self.q.unbind(0))              # views made once, not per call
+        self.out_step = list(self.out.unbind(0))
         self.ws = l2.new_workspace(l2.Layout(self.K_c, q_heads=w.Hq, rows=self.rows),
                                    max(self.max_dec, self.max_in), device)
         self.new_rows, self.new_pos = [], []
@@ -229,7 +231,15 @@ class Job:
                                seed=1, sumsq_in=sumsq_in, rows_in=self.rin, rows_out=self.rows)
 
     def decode(self, s, b=None):
-        i = slice(None) if b is None or self.packed else slice(b, b + 1)
+        if b is None or self.packed:                      # the whole batch: no views to make
+            if self.w.append_steps:
+                k, v = self.new_rows[s]
+                self.l2.append_evict(self.K_c, self.V_c, self.idx, self.sumsq, self.cur, self.keep, self.unc,
+                                     k, v, self.new_pos[s], self.ws, rows=self.rows)
+            self.l2.decode_attention(self.q_step[s], self.K_c, self.V_c, self.cur, self.max_dec,
+                                     self.out_step[s], self.ws, rows=self.rows)
+            return
+        i = slice(b, b + 1)
         if self.w.append_steps:
             k, v = self.new_rows[s]
             self.l2.append_evict(self.K_c[i], self.V_c[i], self.idx[i], self.sumsq[i], self.cur[i],
