@@ -34,8 +34,9 @@ def make(w, t_cap=None):
 
 def check_compress(l2, w, K, V, Kn, Vn, lens, keep, unc=(), policy=0, t_cap_out=None, seed=0,
                    sumsq_in=None):
-    _, got = gpu_compress(l2, K, V, lens, keep, unc, policy, t_cap_out, seed=seed,
-                          sumsq_in=sumsq_in)
+    dev, got = gpu_compress(l2, K, V, lens, keep, unc, policy, t_cap_out, seed=seed,
+                            sumsq_in=sumsq_in)
+    got["_dev"] = dev                                   # the device tensors, for callers that go on
     exact = oracle.compress(Kn, Vn, w.dtype, lens, keep, unc, key_mode=1, policy=policy,
                             t_cap_out=t_cap_out, nthreads=8, seed=seed)
     assert np.array_equal(got["kept_len"], exact["kept_len"])
@@ -98,6 +99,33 @@ def test_compress_ragged_multi_chunk(l2, dtype, D):
     w = synth.WORKLOADS[1].scaled(dtype=dtype, D=D, B=3, L=3, Hkv=2, Hq=2, T=2500)
     K, V, Kn, Vn = make(w, t_cap=2560)
     check_compress(l2, w, K, V, Kn, Vn, [2500, 777, 1], [1250, 100, 1], unc=(1,), t_cap_out=2500)
+
+
+@pytest.mark.parametrize("case", range(10))
+def test_compress_and_attention_random_shapes(l2, case):
+    """Seeded random shapes, lengths, keep counts, layer lists, policies and element types: the whole
+    path (compression, then decode attention over the result) against the oracle."""
+    rng = np.random.default_rng(1000 + case)
+    dtype = ("bf16", "f32")[int(rng.integers(0, 2))]
+    D = (64, 128)[int(rng.integers(0, 2))]
+    Hkv = int(rng.integers(1, 4))
+    G = (1, 2, 4, 8)[int(rng.integers(0, 4))]
+    B, L = int(rng.integers(1, 4)), int(rng.integers(1, 4))
+    T = int(rng.integers(1, 3000))
+    w = synth.WORKLOADS[2].scaled(dtype=dtype, D=D, B=B, L=L, Hkv=Hkv, Hq=Hkv * G, T=T, seed=50 + case)
+    t_cap = T + int(rng.integers(0, 70))
+    K, V, Kn, Vn = make(w, t_cap=t_cap)
+    lens = [int(rng.integers(0, T + 1)) for _ in range(B)]
+    lens[0] = T
+    keep = [int(rng.integers(0, n + 1)) for n in lens]
+    unc = tuple(sorted(set(int(x) for x in rng.integers(0, L, size=int(rng.integers(0, 2))))))
+    policy = int(rng.integers(0, 3))
+    got, _ = check_compress(l2, w, K, V, Kn, Vn, lens, keep, unc=unc, policy=policy, seed=case)
+    q = synth.make_query(w, case, DEV)
+    dev = got["_dev"]
+    out = gpu_attention(l2, q, dev["K_c"], dev["V_c"], dev["kept_len"])
+    want = oracle.attention(synth.to_numpy(q), got["K_c"], got["V_c"], dtype, got["kept_len"], nthreads=8)
+    assert_attention_close(out, want)
 
 
 def test_compress_exact_ties(l2):
