@@ -44,8 +44,8 @@
  *     is then a host upper bound of row_cap_dev.  Every per-row companion array of such a
  *     cache (idx, sumsq, the outputs of l2kv_key_norms) is dense [kv_heads, total_rows] with
  *     the same row axis.  Accepted by l2kv_key_norms, l2kv_select_compact (input, output or
- *     both), l2kv_decode_attention, l2kv_append_evict, their _per_head / _static forms and the
- *     prefix-attention calls; l2kv_attention_loss returns L2KV_ERR_UNSUPPORTED for it.
+ *     both), l2kv_decode_attention, l2kv_append_evict, their _per_head / _static forms, the
+ *     prefix-attention calls and l2kv_attention_loss.
  *   - `len_dev[b]` is the number of valid tokens of sequence b; `max_len` is a host
  *     upper bound on every length the call will meet (it sizes grids and scratch;
  *     device lengths above it are clamped to it).
@@ -318,7 +318,7 @@ int l2kv_prefix_attention_flags(const void* q, const void* K_c, const void* V_c,
  *   L^{m,ref} = sum of the m smallest a_p (the ideal compression)
  *   Y         = sum_{m=1..n} (L^m - L^{m,ref})                     (Eqs. 6, 7)
  * sumsq holds the keys of K as l2kv_key_norms writes them (dense fp32
- * [batch, layers, kv_heads, t_cap]).  alr_out is dense fp32 [batch, layers, q_heads].
+ * [batch, layers, kv_heads, t_cap]; [kv_heads, total_rows] for a packed cache).  alr_out is dense fp32 [batch, layers, q_heads].
  * loss_out / loss_ref_out may be NULL; otherwise dense fp32
  * [batch, layers, q_heads, t_cap] receiving L^m / L^{m,ref} at index m - 1 (entries at
  * and beyond n untouched).  Sums are fp64 internally.  An empty cache gives Y = 0.
@@ -332,6 +332,13 @@ int l2kv_attention_loss(const void* q, const void* K, const l2kv_layout* lay,
                         const int32_t* cur_len_dev, int32_t max_len, float scale,
                         const float* sumsq, float* alr_out, float* loss_out, float* loss_ref_out,
                         void* workspace, size_t workspace_bytes, void* stream);
+/* The same with a cache length per (b, l, kv head): cur_len_unit_dev dense int32
+ * [batch, layers, kv_heads], as l2kv_select_compact_per_head leaves it. */
+int l2kv_attention_loss_per_head(const void* q, const void* K, const l2kv_layout* lay,
+                                 const int32_t* cur_len_unit_dev, int32_t max_len, float scale,
+                                 const float* sumsq, float* alr_out, float* loss_out,
+                                 float* loss_ref_out, void* workspace, size_t workspace_bytes,
+                                 void* stream);
 
 /* Decode attention without a workspace -- the paper has no counterpart to this entry
  * point; it exists for the callers of this library that cannot allocate device memory.

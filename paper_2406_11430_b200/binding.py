@@ -63,6 +63,7 @@ def lib():
         L.l2kv_attention_loss_workspace_bytes.argtypes = [lay, i32, ctypes.POINTER(sz)]
         L.l2kv_attention_loss.argtypes = [vp, vp, lay, vp, i32, ctypes.c_float, vp, vp, vp, vp,
                                           vp, sz, vp]
+        L.l2kv_attention_loss_per_head.argtypes = L.l2kv_attention_loss.argtypes
         L.l2kv_prefix_attention.argtypes = [vp, vp, vp, lay, vp, i32, i32, ctypes.c_float, vp, vp,
                                             vp, sz, vp]
         L.l2kv_prefix_attention_per_head.argtypes = L.l2kv_prefix_attention.argtypes
@@ -81,7 +82,7 @@ def lib():
                      "l2kv_prefix_attention_per_head", "l2kv_prefix_attention_workspace_bytes",
                      "l2kv_prefix_attention_causal", "l2kv_prefix_attention_flags",
                      "l2kv_workspace_reset", "l2kv_selftest_wait_timeout",
-                     "l2kv_decode_attention_static_status"):
+                     "l2kv_decode_attention_static_status", "l2kv_attention_loss_per_head"):
             getattr(L, name).restype = ctypes.c_int
         _LIB = L
     return _LIB
@@ -293,17 +294,19 @@ def decode_attention_static(q, K_c, V_c, cur_len_dev, max_len, out, scale=0.0, s
 
 
 def attention_loss(q, K, cur_len_dev, max_len, sumsq, alr_out, loss_out=None, loss_ref_out=None,
-                   scale=0.0, workspace=None, stream=None):
+                   scale=0.0, workspace=None, stream=None, rows=None, per_head=False):
     """Attention loss of norm-based vs ideal compression (Eqs. 5-7); see l2kv_attention_loss.
-    Allocates the (large) scratch itself unless a workspace tensor is passed."""
-    lay = Layout(K, q_heads=q.shape[2])
+    Allocates the (large) scratch itself unless a workspace tensor is passed.  rows (Rows): the
+    cache is packed; per_head: cur_len_dev holds a length per (b, l, kv head)."""
+    lay = Layout(K, q_heads=q.shape[2], rows=rows)
     if workspace is None:
         need = ctypes.c_size_t(0)
         _check(lib().l2kv_attention_loss_workspace_bytes(lay.ref(), int(max_len),
                                                          ctypes.byref(need)),
                "l2kv_attention_loss_workspace_bytes")
         workspace = torch.empty(need.value, dtype=torch.uint8, device=K.device)
-    _check(lib().l2kv_attention_loss(
+    fn = lib().l2kv_attention_loss_per_head if per_head else lib().l2kv_attention_loss
+    _check(fn(
         _ptr(q), _ptr(K), lay.ref(), _ptr(cur_len_dev), int(max_len), float(scale), _ptr(sumsq),
         _ptr(alr_out), _ptr(loss_out), _ptr(loss_ref_out), _ptr(workspace), workspace.numel(),
         _stream(stream)), "l2kv_attention_loss")

@@ -45,8 +45,6 @@ int check_layout(const l2kv_layout* a) {
   return L2KV_OK;
 }
 
-bool packed(const l2kv_layout* a) { return a->row_off_dev != nullptr; }
-
 int check_groups(const l2kv_layout* a) {
   if (a->kv_heads == 0) return a->q_heads == 0 ? L2KV_OK : L2KV_ERR_INVALID_ARG;
   if (a->q_heads % a->kv_heads) return L2KV_ERR_INVALID_ARG;
@@ -398,14 +396,14 @@ int l2kv_attention_loss_workspace_bytes(const l2kv_layout* lay, int32_t max_len,
   return L2KV_OK;
 }
 
-int l2kv_attention_loss(const void* q, const void* K, const l2kv_layout* lay,
-                        const int32_t* cur_len_dev, int32_t max_len, float scale,
-                        const float* sumsq, float* alr_out, float* loss_out, float* loss_ref_out,
-                        void* workspace, size_t workspace_bytes, void* stream) {
+static int attention_loss_impl(bool per_head, const void* q, const void* K, const l2kv_layout* lay,
+                               const int32_t* cur_len_dev, int32_t max_len, float scale,
+                               const float* sumsq, float* alr_out, float* loss_out,
+                               float* loss_ref_out, void* workspace, size_t workspace_bytes,
+                               void* stream) {
   const Range nvtx_range("l2kv_attention_loss");
   int rc = check_layout(lay);
   if (rc != L2KV_OK) return rc;
-  if (packed(lay)) return L2KV_ERR_UNSUPPORTED;
   if (lay->kv_heads > 0 && lay->q_heads % lay->kv_heads) return L2KV_ERR_INVALID_ARG;
   if (max_len < 0 || !(scale == scale)) return L2KV_ERR_INVALID_ARG;
   if (max_len > lay->t_cap) return L2KV_ERR_OUT_OF_RANGE;
@@ -415,9 +413,27 @@ int l2kv_attention_loss(const void* q, const void* K, const l2kv_layout* lay,
   if (!aligned16(q) || !aligned16(K) || !aligned16(workspace)) return L2KV_ERR_MISALIGNED;
   if (workspace_bytes < attention_loss_workspace(*lay, max_len)) return L2KV_ERR_WORKSPACE_TOO_SMALL;
   const float sc = scale > 0.f ? scale : 1.0f / std::sqrt((float)lay->head_dim);
-  return launch_attention_loss(q, K, make_geom(*lay), lay->dtype, cur_len_dev, max_len, sc, sumsq,
+  const LenView lens{cur_len_dev, per_head ? 1 : 0};
+  return launch_attention_loss(q, K, make_geom(*lay), lay->dtype, lens, max_len, sc, sumsq,
                                alr_out, loss_out, loss_ref_out, static_cast<char*>(workspace),
                                static_cast<cudaStream_t>(stream));
+}
+
+int l2kv_attention_loss(const void* q, const void* K, const l2kv_layout* lay,
+                        const int32_t* cur_len_dev, int32_t max_len, float scale,
+                        const float* sumsq, float* alr_out, float* loss_out, float* loss_ref_out,
+                        void* workspace, size_t workspace_bytes, void* stream) {
+  return attention_loss_impl(false, q, K, lay, cur_len_dev, max_len, scale, sumsq, alr_out, loss_out,
+                             loss_ref_out, workspace, workspace_bytes, stream);
+}
+
+int l2kv_attention_loss_per_head(const void* q, const void* K, const l2kv_layout* lay,
+                                 const int32_t* cur_len_unit_dev, int32_t max_len, float scale,
+                                 const float* sumsq, float* alr_out, float* loss_out,
+                                 float* loss_ref_out, void* workspace, size_t workspace_bytes,
+                                 void* stream) {
+  return attention_loss_impl(true, q, K, lay, cur_len_unit_dev, max_len, scale, sumsq, alr_out, loss_out,
+                             loss_ref_out, workspace, workspace_bytes, stream);
 }
 
 }  // extern "C"

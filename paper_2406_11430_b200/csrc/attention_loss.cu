@@ -411,7 +411,7 @@ __device__ void scores_plain(const T* __restrict__ q_unit, const T* __restrict__
 template <typename T, int D, bool SMALL>
 __global__ void __launch_bounds__(kLossThreads)
 attention_loss_kernel(const T* __restrict__ q, const T* __restrict__ K, Geom g,
-                      const int32_t* __restrict__ cur_len_dev, int max_len, float scale_log2e,
+                      LenView cur_len_dev, int max_len, float scale_log2e,
                       const float* __restrict__ sumsq, uint32_t* order, uint32_t* order_tmp,
                       long long ld, float* probs, float* sorted, float* alr_out, float* loss_out,
                       float* loss_ref_out) {
@@ -431,7 +431,7 @@ attention_loss_kernel(const T* __restrict__ q, const T* __restrict__ K, Geom g,
   const long long bl = unit / g.H;
   const int l = (int)(bl % g.L), b = (int)(bl / g.L);
   const int G = g.Hq / g.H;
-  const int n = max(0, min(cur_len_dev[bl], min(max_len, g.t_cap)));
+  const int n = max(0, min(cur_len_dev.at(bl, h, g.H), min(max_len, g.cap(bl))));
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const long long row0 = bl * g.Hq + (long long)h * G;   // first query head of this KV head
   if (n == 0) {
@@ -447,8 +447,8 @@ attention_loss_kernel(const T* __restrict__ q, const T* __restrict__ K, Geom g,
   // keys end up in position order.
   uint32_t* ord = order + unit * ld;
   uint32_t* ord_tmp = SMALL ? s_buf : order_tmp + unit * ld;
-  const KeyOfPosition key_of{sumsq + unit * g.t_cap, n, &s_bad};
-  const T* Kb = K + b * g.sb + l * g.sl + h * g.sh;
+  const KeyOfPosition key_of{sumsq + g.meta(unit), n, &s_bad};
+  const T* Kb = K + g.base(b, l, h);
   // The blocks of a wave start together and do the same work, so they would all stream K at the
   // same time and all sort at the same time.  Every other block therefore takes the two steps
   // in the other order: half of the GPU reads K while the other half sorts.
@@ -556,7 +556,7 @@ size_t attention_loss_workspace(const l2kv_layout& a, int max_len) {
 }
 
 template <typename T, int D>
-static int launch_al_t(const void* q, const void* K, const Geom& g, const int32_t* cur_len_dev,
+static int launch_al_t(const void* q, const void* K, const Geom& g, const LenView& cur_len_dev,
                        int max_len, float scale, const float* sumsq, float* alr_out, float* loss_out,
                        float* loss_ref_out, char* ws, cudaStream_t s) {
   const long long units = (long long)g.B * g.L * g.H;
@@ -582,7 +582,7 @@ static int launch_al_t(const void* q, const void* K, const Geom& g, const int32_
 }
 
 int launch_attention_loss(const void* q, const void* K, const Geom& g, int dtype,
-                          const int32_t* cur_len_dev, int max_len, float scale, const float* sumsq,
+                          const LenView& cur_len_dev, int max_len, float scale, const float* sumsq,
                           float* alr_out, float* loss_out, float* loss_ref_out, char* ws,
                           cudaStream_t s) {
 #define L2KV_AL(T, D) \

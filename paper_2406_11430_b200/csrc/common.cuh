@@ -293,7 +293,7 @@ int launch_prefix_attention(const void* q, const void* K, const void* V, const G
 size_t prefix_attention_scratch(const Geom& g, int n_queries, int max_len);
 size_t attention_loss_workspace(const l2kv_layout& a, int max_len);
 int launch_attention_loss(const void* q, const void* K, const Geom& g, int dtype,
-                          const int32_t* cur_len_dev, int max_len, float scale, const float* sumsq,
+                          const LenView& cur_len_dev, int max_len, float scale, const float* sumsq,
                           float* alr_out, float* loss_out, float* loss_ref_out, char* ws,
                           cudaStream_t s);
 

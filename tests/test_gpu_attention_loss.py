@@ -66,3 +66,58 @@ def test_attention_loss_planted_structure():
     K[0, 0, 0, :, 1] = torch.linspace(9.0, 1.0, n, device=DEV)
     alr3, _, _ = run(l2, q, K, [[n]], n, curves=False)
     assert alr3[0, 0, 0] > 100.0
+
+
+def test_attention_loss_per_head_lengths_and_packed_cache():
+    """A length per (b, l, kv head), and a packed cache: each unit against the oracle run on that
+    unit alone (its rows, its length, its query heads)."""
+    import paper_2406_11430_b200 as l2
+    B, L, Hkv, Hq, D, T = 2, 2, 2, 8, 128, 900
+    G = Hq // Hkv
+    w = synth.WORKLOADS[2].scaled(B=B, L=L, Hkv=Hkv, Hq=Hq, T=T)
+    K, _ = synth.make_cache(w, DEV)
+    q = synth.make_query(w, 3, DEV)
+    Kn, qn = synth.to_numpy(K), synth.to_numpy(q)
+
+    def unit_oracle(rows, n, qs):
+        return oracle.attention_loss(np.ascontiguousarray(qs[None, None]), np.ascontiguousarray(rows[None, None, None]),
+                                     "bf16", [[n]], key_mode=1)[0, 0]
+
+    # per-head lengths on the dense cache
+    cur = np.array([[[900, 333], [1, 0]], [[512, 777], [64, 899]]], dtype=np.int32)
+    lens = i32(np.full(B, T))
+    sumsq = torch.zeros((B, L, Hkv, T), dtype=torch.float32, device=DEV)
+    l2.key_norms(K, lens, T, sumsq)
+    alr = torch.full((B, L, Hq), float("nan"), dtype=torch.float32, device=DEV)
+    l2.attention_loss(q, K, i32(cur), T, sumsq, alr, per_head=True)
+    torch.cuda.synchronize()
+    got = alr.cpu().numpy()
+    for b in range(B):
+        for l in range(L):
+            for h in range(Hkv):
+                n = int(cur[b, l, h])
+                want = unit_oracle(Kn[b, l, h, :max(n, 1)], n, qn[b, l, h * G:(h + 1) * G])
+                np.testing.assert_allclose(got[b, l, h * G:(h + 1) * G], want, rtol=2e-4, atol=1e-4 * max(n, 1))
+
+    # the same cache packed: (b, l) ranges of different sizes on one row axis
+    caps = [[900, 400], [64, 700]]
+    cur_bl = np.array([[900, 350], [0, 700]], dtype=np.int32)
+    off, cap, total = synth.packing(caps)
+    rows = l2.Rows(off, cap, total, DEV)
+    Kp = torch.zeros((Hkv, total, D), dtype=K.dtype, device=DEV)
+    for b in range(B):
+        for l in range(L):
+            o, c = int(off[b, l]), int(cap[b, l])
+            Kp[:, o:o + c] = K[b, l, :, :c]
+    ss = torch.zeros((Hkv, total), dtype=torch.float32, device=DEV)
+    l2.key_norms(Kp, i32([900, 700]), 900, ss, rows=rows)
+    alr2 = torch.full((B, L, Hq), float("nan"), dtype=torch.float32, device=DEV)
+    l2.attention_loss(q, Kp, i32(cur_bl), 900, ss, alr2, rows=rows)
+    torch.cuda.synchronize()
+    got2 = alr2.cpu().numpy()
+    for b in range(B):
+        for l in range(L):
+            n = int(cur_bl[b, l])
+            for h in range(Hkv):
+                want = unit_oracle(Kn[b, l, h, :max(n, 1)], n, qn[b, l, h * G:(h + 1) * G])
+                np.testing.assert_allclose(got2[b, l, h * G:(h + 1) * G], want, rtol=2e-4, atol=1e-4 * max(n, 1))

@@ -184,7 +184,7 @@ def test_packed_overflow_sets_status_and_leaves_neighbours_alone(l2):
         assert np.array_equal(before["idx"][:, sl], after["idx"][:, sl])
 
 
-def test_packed_static_decode_and_unsupported_call(l2):
+def test_packed_static_decode(l2):
     w = synth.WORKLOADS[2].scaled(B=2, L=2, T=1300)
     pc, st = run_packed_pipeline(l2, w, lens=[1300, 700], keep=[650, 350], unc=(0,), steps=1)
     q = synth.make_query(w, 7, DEV)
@@ -194,17 +194,7 @@ def test_packed_static_decode_and_unsupported_call(l2):
     l2.decode_attention_static(q, pc.K_c, pc.V_c, pc.cur, pc.max_len, got, rows=pc.rows)
     torch.cuda.synchronize()
     assert torch.equal(got, want)
-    import ctypes
-    lay = l2.Layout(pc.K_c, q_heads=w.Hq, rows=pc.rows)
-    need = ctypes.c_size_t(0)
-    rc = l2.lib().l2kv_attention_loss_workspace_bytes(lay.ref(), 100, ctypes.byref(need))
-    assert rc == 0
-    scratch = torch.empty(need.value, dtype=torch.uint8, device=DEV)
-    alr = torch.zeros((2, 2, w.Hq), dtype=torch.float32, device=DEV)
-    rc = l2.lib().l2kv_attention_loss(q.data_ptr(), pc.K_c.data_ptr(), lay.ref(), pc.cur.data_ptr(), 100,
-                                      ctypes.c_float(0.0), pc.sumsq.data_ptr(), alr.data_ptr(), None, None,
-                                      scratch.data_ptr(), scratch.numel(), None)
-    assert rc == -2                                          # the attention-loss analysis takes dense caches only
+
 
 def test_packed_prefix_attention(l2):
     """Several new queries per (b, l) over a packed compressed cache, plain and causal, both weight
