@@ -403,6 +403,8 @@ def run_gpu(args):
                          "gpu_launches": jo.launches_per_step * n}
                 if not args.no_cpu_baseline and world == 1:
                     entry["tie_band"] = tie_band_report(jo, wo)
+                if jo.packed and wo.dtype == "bf16" and wo.D == 128:
+                    entry["prefix_attention"] = time_packed_prefix(jo, wo)
                 others[wo.name] = entry
             del jo
             free_device_memory()
@@ -410,6 +412,29 @@ def run_gpu(args):
             line["configs"] = others
     if rank == 0:
         print(json.dumps(line))
+
+
+def time_packed_prefix(job, w, n_q=128, reps=3):
+    """A block of n_q new queries per sequence over the packed, ragged compressed caches (a chunk of
+    a chunked prefill in a serving batch): prefix attention on the tensor cores, cache split over
+    the grid where the lengths call for it."""
+    q = torch.randn((w.B, w.L, n_q, w.Hq, w.D), dtype=torch.bfloat16, device=job.dev)
+    out = torch.empty(q.shape, dtype=torch.float32, device=job.dev)
+    ws = job.l2.prefix_attention_workspace(job.K_c, q, job.max_dec, rows=job.rows)
+    call = lambda: job.l2.prefix_attention_flags(q, job.K_c, job.V_c, job.cur, job.max_dec, out, 0,
+                                                 workspace=ws, rows=job.rows)
+    call()
+    torch.cuda.synchronize()
+    t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(reps):
+        call()
+    t1.record(); torch.cuda.synchronize()
+    ms = t0.elapsed_time(t1) / reps
+    flops = 4.0 * n_q * w.Hq * w.D * float(job.cur.sum().item())
+    status = job.l2.read_device_status(ws)
+    return {"ms": round(ms, 3), "queries_per_sequence": n_q, "TFLOPs": round(flops / ms / 1e9, 1),
+            "cached_rows": int(job.cur.sum().item()), "device_status": status}
 
 
 def free_device_memory():
