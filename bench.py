@@ -590,6 +590,22 @@ def time_append_evict(job, w, reps=20):
             "stored_entries": stored}
 
 
+def host_memory_is_device_addressable(device_index):
+    """True when kernels may read pinned host memory through its host pointer (unified addressing
+    with mapped host memory), which the V-on-demand schedule relies on."""
+    try:
+        try:
+            from cuda.bindings import runtime as cudart
+        except ImportError:
+            from cuda import cudart
+        a = cudart.cudaDeviceAttr
+        e1, ua = cudart.cudaDeviceGetAttribute(a.cudaDevAttrUnifiedAddressing, device_index)
+        e2, mh = cudart.cudaDeviceGetAttribute(a.cudaDevAttrCanMapHostMemory, device_index)
+        return int(e1) == 0 and int(e2) == 0 and bool(ua) and bool(mh)
+    except Exception:
+        return False
+
+
 def run_e2e(job, w, step_bytes, world, device, args):
     """The same step with the cache arriving from pinned host memory and the attention outputs
     returning to it, all inside the timed region.  Two schedules are timed.  "copy everything":
@@ -654,6 +670,13 @@ def run_e2e(job, w, step_bytes, world, device, args):
         return max_over_ranks(t0.elapsed_time(t1), world, device) / n, n, same
 
     ms_all, n, same_all = timed(True)
+    if not host_memory_is_device_addressable(job.K.device.index or 0):
+        # no mapped host memory on this system: only the copying schedule can run
+        del Kh, Vh
+        return {"value": round(world * step_bytes / (ms_all * 1e-3) / 1e9, 1), "unit": "GB/s",
+                "ms_per_step": round(ms_all, 2), "steps": n, "h2d_bytes_per_step": 2 * kv_bytes + q_bytes,
+                "d2h_bytes_per_step": d2h, "outputs_equal_device_resident_step": same_all,
+                "schedule": "per sequence: upload of sequence b+1 overlaps compress + decode of sequence b"}
     ms_dem, _, same_dem = timed(False)
     del Kh, Vh
     rate = lambda ms: round(world * step_bytes / (ms * 1e-3) / 1e9, 1)
