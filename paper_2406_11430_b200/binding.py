@@ -134,9 +134,9 @@ class Layout:
         if cache.dim() != 5 or cache.stride(4) != 1:
             raise ValueError("cache must be [B, L, Hkv, t_cap, D] with D contiguous")
         B, L, H, T, D = cache.shape
+        sb, sl, sh, st, _ = cache.stride()
         self.c = _CLayout(B, L, H, H if q_heads is None else q_heads, D, T, _DTYPE[cache.dtype], 0,
-                          cache.stride(0), cache.stride(1), cache.stride(2), cache.stride(3),
-                          None, None, 0)
+                          sb, sl, sh, st, None, None, 0)
 
     def ref(self):
         return ctypes.byref(self.c)
@@ -146,12 +146,24 @@ def _ptr(t):
     return ctypes.c_void_p(0 if t is None else t.data_ptr())
 
 
-def _stream(stream):
-    if stream is None:
-        if not torch.cuda.is_available():        # host-only calls (argument checks) need no stream
+_RAW_STREAM = getattr(torch._C, "_cuda_getCurrentRawStream", None)
+
+
+def _stream(stream, ref=None):
+    """Handle of the CUDA stream a call is ordered on: the given torch stream, else the current
+    stream of the device that holds `ref` (a tensor of the call); 0 for host-only calls
+    (argument checks on host tensors, or no GPU at all)."""
+    if stream is not None:
+        return ctypes.c_void_p(stream.cuda_stream)
+    if ref is not None:
+        if not ref.is_cuda:
             return ctypes.c_void_p(0)
-        stream = torch.cuda.current_stream()
-    return ctypes.c_void_p(stream.cuda_stream)
+        if _RAW_STREAM is not None:              # the handle without building a Stream object
+            return ctypes.c_void_p(_RAW_STREAM(ref.device.index))
+        return ctypes.c_void_p(torch.cuda.current_stream(ref.device).cuda_stream)
+    if not torch.cuda.is_available():
+        return ctypes.c_void_p(0)
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
 
 
 def _layers(layers):
@@ -180,20 +192,20 @@ def new_workspace(layout, max_len, device):
 
 def read_device_status(workspace, stream=None):
     out = ctypes.c_int32(0)
-    _check(lib().l2kv_read_device_status(_ptr(workspace), _stream(stream), ctypes.byref(out)),
+    _check(lib().l2kv_read_device_status(_ptr(workspace), _stream(stream, workspace), ctypes.byref(out)),
            "l2kv_read_device_status")
     return out.value
 
 
 def workspace_reset(workspace, layout, stream=None):
     """Zeroes the status block and the completion counters of a workspace, in stream order."""
-    _check(lib().l2kv_workspace_reset(_ptr(workspace), workspace.numel(), layout.ref(), _stream(stream)),
+    _check(lib().l2kv_workspace_reset(_ptr(workspace), workspace.numel(), layout.ref(), _stream(stream, workspace)),
            "l2kv_workspace_reset")
 
 
 def selftest_wait_timeout(workspace, stream=None):
     """Makes one bounded wait run out on purpose (nothing faults) and records it in workspace."""
-    _check(lib().l2kv_selftest_wait_timeout(_ptr(workspace), workspace.numel(), _stream(stream)),
+    _check(lib().l2kv_selftest_wait_timeout(_ptr(workspace), workspace.numel(), _stream(stream, workspace)),
            "l2kv_selftest_wait_timeout")
 
 
@@ -208,7 +220,7 @@ def decode_attention_static_status(reset=False, stream=None):
 def key_norms(K, len_dev, max_len, sumsq_out, norm_out=None, stream=None, rows=None):
     lay = Layout(K, rows=rows)
     _check(lib().l2kv_key_norms(_ptr(K), lay.ref(), _ptr(len_dev), int(max_len), _ptr(sumsq_out),
-                                _ptr(norm_out), _stream(stream)), "l2kv_key_norms")
+                                _ptr(norm_out), _stream(stream, K)), "l2kv_key_norms")
 
 
 def select_compact(K, V, len_dev, keep_dev, max_len, uncompressed_layers, K_out, V_out, idx_out,
@@ -221,7 +233,7 @@ def select_compact(K, V, len_dev, keep_dev, max_len, uncompressed_layers, K_out,
         _ptr(K), _ptr(V), lin.ref(), _ptr(len_dev), _ptr(keep_dev), int(max_len), arr, n,
         int(policy), ctypes.c_uint64(int(seed) & 0xFFFFFFFFFFFFFFFF), _ptr(sumsq_in), _ptr(K_out),
         _ptr(V_out), lout.ref(), _ptr(idx_out), _ptr(sumsq_out),
-        _ptr(kept_len_dev), _ptr(workspace), workspace.numel(), _stream(stream)),
+        _ptr(kept_len_dev), _ptr(workspace), workspace.numel(), _stream(stream, K)),
         "l2kv_select_compact")
 
 
@@ -235,7 +247,7 @@ def select_compact_per_head(K, V, len_dev, keep_unit_dev, max_len, uncompressed_
         _ptr(K), _ptr(V), lin.ref(), _ptr(len_dev), _ptr(keep_unit_dev), int(max_len), arr, n,
         int(policy), ctypes.c_uint64(int(seed) & 0xFFFFFFFFFFFFFFFF), _ptr(sumsq_in), _ptr(K_out),
         _ptr(V_out), lout.ref(), _ptr(idx_out), _ptr(sumsq_out),
-        _ptr(kept_len_unit_dev), _ptr(workspace), workspace.numel(), _stream(stream)),
+        _ptr(kept_len_unit_dev), _ptr(workspace), workspace.numel(), _stream(stream, K)),
         "l2kv_select_compact_per_head")
 
 
@@ -245,7 +257,7 @@ def decode_attention_per_head(q, K_c, V_c, cur_len_unit_dev, max_len, out, works
     lay = Layout(K_c, q_heads=q.shape[2])
     _check(lib().l2kv_decode_attention_per_head(
         _ptr(q), _ptr(K_c), _ptr(V_c), lay.ref(), _ptr(cur_len_unit_dev), int(max_len),
-        float(scale), _ptr(out), _ptr(workspace), workspace.numel(), _stream(stream)),
+        float(scale), _ptr(out), _ptr(workspace), workspace.numel(), _stream(stream, q)),
         "l2kv_decode_attention_per_head")
 
 
@@ -254,7 +266,7 @@ def decode_attention(q, K_c, V_c, cur_len_dev, max_len, out, workspace, scale=0.
     lay = Layout(K_c, q_heads=q.shape[2], rows=rows)
     _check(lib().l2kv_decode_attention(
         _ptr(q), _ptr(K_c), _ptr(V_c), lay.ref(), _ptr(cur_len_dev), int(max_len), float(scale),
-        _ptr(out), _ptr(workspace), workspace.numel(), _stream(stream)), "l2kv_decode_attention")
+        _ptr(out), _ptr(workspace), workspace.numel(), _stream(stream, q)), "l2kv_decode_attention")
 
 
 def append_evict(K_c, V_c, idx, sumsq_c, cur_len_dev, budget_dev, uncompressed_layers, k_new, v_new,
@@ -264,7 +276,7 @@ def append_evict(K_c, V_c, idx, sumsq_c, cur_len_dev, budget_dev, uncompressed_l
     _check(lib().l2kv_append_evict(
         _ptr(K_c), _ptr(V_c), _ptr(idx), _ptr(sumsq_c), lay.ref(), _ptr(cur_len_dev),
         _ptr(budget_dev), arr, n, _ptr(k_new), _ptr(v_new), _ptr(pos_new_dev), _ptr(workspace),
-        workspace.numel(), _stream(stream)), "l2kv_append_evict")
+        workspace.numel(), _stream(stream, K_c)), "l2kv_append_evict")
 
 
 def append_evict_per_head(K_c, V_c, idx, sumsq_c, cur_len_unit_dev, budget_unit_dev,
@@ -275,7 +287,7 @@ def append_evict_per_head(K_c, V_c, idx, sumsq_c, cur_len_unit_dev, budget_unit_
     _check(lib().l2kv_append_evict_per_head(
         _ptr(K_c), _ptr(V_c), _ptr(idx), _ptr(sumsq_c), lay.ref(), _ptr(cur_len_unit_dev),
         _ptr(budget_unit_dev), arr, n, _ptr(k_new), _ptr(v_new), _ptr(pos_new_dev),
-        _ptr(workspace), workspace.numel(), _stream(stream)), "l2kv_append_evict_per_head")
+        _ptr(workspace), workspace.numel(), _stream(stream, K_c)), "l2kv_append_evict_per_head")
 
 
 def decode_attention_static(q, K_c, V_c, cur_len_dev, max_len, out, scale=0.0, stream=None,
@@ -290,7 +302,7 @@ def decode_attention_static(q, K_c, V_c, cur_len_dev, max_len, out, scale=0.0, s
     fn.argtypes = [vp, vp, vp, ctypes.POINTER(_CLayout), vp, ctypes.c_int32, ctypes.c_float, vp, vp]
     lay = Layout(K_c, q_heads=q.shape[2], rows=rows)
     _check(fn(_ptr(q), _ptr(K_c), _ptr(V_c), lay.ref(), _ptr(cur_len_dev), int(max_len),
-              float(scale), _ptr(out), _stream(stream)), "l2kv_decode_attention_static")
+              float(scale), _ptr(out), _stream(stream, q)), "l2kv_decode_attention_static")
 
 
 def attention_loss(q, K, cur_len_dev, max_len, sumsq, alr_out, loss_out=None, loss_ref_out=None,
@@ -309,7 +321,7 @@ def attention_loss(q, K, cur_len_dev, max_len, sumsq, alr_out, loss_out=None, lo
     _check(fn(
         _ptr(q), _ptr(K), lay.ref(), _ptr(cur_len_dev), int(max_len), float(scale), _ptr(sumsq),
         _ptr(alr_out), _ptr(loss_out), _ptr(loss_ref_out), _ptr(workspace), workspace.numel(),
-        _stream(stream)), "l2kv_attention_loss")
+        _stream(stream, q)), "l2kv_attention_loss")
 
 
 def prefix_attention_workspace(K_c, q, max_len, device=None, rows=None):
@@ -334,7 +346,7 @@ def prefix_attention_flags(q, K_c, V_c, cur_len_dev, max_len, out, flags, lse_ou
     _check(lib().l2kv_prefix_attention_flags(
         _ptr(q), _ptr(K_c), _ptr(V_c), lay.ref(), _ptr(cur_len_dev), int(max_len), int(q.shape[2]),
         float(scale), int(flags), _ptr(out), _ptr(lse_out), _ptr(workspace),
-        0 if workspace is None else workspace.numel(), _stream(stream)),
+        0 if workspace is None else workspace.numel(), _stream(stream, q)),
         "l2kv_prefix_attention_flags")
 
 
@@ -345,7 +357,7 @@ def prefix_attention(q, K_c, V_c, cur_len_dev, max_len, out, lse_out=None, scale
     _check(lib().l2kv_prefix_attention(
         _ptr(q), _ptr(K_c), _ptr(V_c), lay.ref(), _ptr(cur_len_dev), int(max_len), int(q.shape[2]),
         float(scale), _ptr(out), _ptr(lse_out), _ptr(workspace),
-        0 if workspace is None else workspace.numel(), _stream(stream)), "l2kv_prefix_attention")
+        0 if workspace is None else workspace.numel(), _stream(stream, q)), "l2kv_prefix_attention")
 
 
 def prefix_attention_causal(q, K_c, V_c, cur_len_dev, max_len, out, lse_out=None, scale=0.0,
@@ -356,7 +368,7 @@ def prefix_attention_causal(q, K_c, V_c, cur_len_dev, max_len, out, lse_out=None
     _check(lib().l2kv_prefix_attention_causal(
         _ptr(q), _ptr(K_c), _ptr(V_c), lay.ref(), _ptr(cur_len_dev), int(max_len), int(q.shape[2]),
         float(scale), _ptr(out), _ptr(lse_out), _ptr(workspace),
-        0 if workspace is None else workspace.numel(), _stream(stream)),
+        0 if workspace is None else workspace.numel(), _stream(stream, q)),
         "l2kv_prefix_attention_causal")
 
 
@@ -367,5 +379,5 @@ def prefix_attention_per_head(q, K_c, V_c, cur_len_unit_dev, max_len, out, lse_o
     _check(lib().l2kv_prefix_attention_per_head(
         _ptr(q), _ptr(K_c), _ptr(V_c), lay.ref(), _ptr(cur_len_unit_dev), int(max_len),
         int(q.shape[2]), float(scale), _ptr(out), _ptr(lse_out), _ptr(workspace),
-        0 if workspace is None else workspace.numel(), _stream(stream)),
+        0 if workspace is None else workspace.numel(), _stream(stream, q)),
         "l2kv_prefix_attention_per_head")
