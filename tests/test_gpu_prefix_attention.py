@@ -216,3 +216,46 @@ def test_prefix_attention_causal(kernel, T, lens, n_q, split, weights, monkeypat
             else:
                 z = Kf[0, l, 1, :see[0, l]] @ qf[0, l, s, 5] / np.sqrt(w.D)
                 np.testing.assert_allclose(got_lse[0, l, s, 5], scipy.special.logsumexp(z), rtol=1e-5, atol=1e-4)
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_prefix_attention_random_shapes(seed, monkeypatch):
+    """Seeded random cases: group size, query count, cache lengths (empty ones included), scale,
+    causal or not, either form of the weights, with or without room to split the cache; a sample
+    of the queries is compared with the oracle run at the length that query may see."""
+    import paper_2406_11430_b200 as l2
+    monkeypatch.delenv("L2KV_PREFIX_KERNEL", raising=False)
+    rng = np.random.default_rng(1000 + seed)
+    G = int(rng.choice([1, 2, 4, 8]))
+    Hkv = int(rng.integers(1, 4))
+    B, L = int(rng.integers(1, 3)), int(rng.integers(1, 4))
+    T = int(rng.choice([65, 200, 777, 1500, 5000]))
+    n_q = int(rng.integers(1, 150))
+    causal = bool(rng.integers(0, 2))
+    weights = WEIGHTS[int(rng.integers(0, 2))]
+    split = bool(rng.integers(0, 2))
+    scale = float(rng.choice([0.0, 0.05, 0.2]))
+    w = synth.WORKLOADS[2].scaled(B=B, L=L, Hkv=Hkv, Hq=Hkv * G, T=T, seed=77 + seed)
+    K, V = synth.make_cache(w, DEV)
+    q = make_queries(w, n_q, 100 + seed)
+    cur = rng.integers(0, T + 1, size=(B, L)).astype(np.int32)
+    cur[0, 0] = T
+    if B * L > 1:
+        cur[-1, -1] = int(rng.choice([0, 1, min(T, n_q - 1) if n_q > 1 else 0]))
+    ws = l2.prefix_attention_workspace(K, q, T) if split else torch.zeros(256, dtype=torch.uint8, device=DEV)
+    out = torch.full(q.shape, float("nan"), dtype=torch.float32, device=DEV)
+    lse = torch.full(q.shape[:4], float("nan"), dtype=torch.float32, device=DEV)
+    call(l2, weights, q, K, V, i32(cur), T, out, lse, scale=scale, workspace=ws, causal=causal)
+    torch.cuda.synchronize()
+    assert l2.read_device_status(ws) == 0
+    got, got_lse = out.cpu().numpy(), lse.cpu().numpy()
+    assert not np.isnan(got).any() and not np.isnan(got_lse).any()
+    Kn, Vn = synth.to_numpy(K), synth.to_numpy(V)
+    for s in sorted(set(rng.integers(0, n_q, size=5).tolist() + [0, n_q - 1])):
+        see = (np.maximum(cur - n_q + s + 1, 0) if causal else cur).astype(np.int32)
+        want = oracle.attention(synth.to_numpy(q[:, :, s].contiguous()), Kn, Vn, "bf16", see, scale=scale,
+                                nthreads=8)
+        assert_attention_close(got[:, :, s], want, atol=ATOL[weights])
+        empty = see == 0
+        assert not got[:, :, s][empty].any() and np.all(np.isneginf(got_lse[:, :, s][empty]))
+        assert np.all(np.isfinite(got_lse[:, :, s][~empty]))
