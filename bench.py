@@ -629,29 +629,48 @@ def run_e2e(job, w, step_bytes, world, device, args):
     v_rows = sum((n_unc * int(n) + (w.L - n_unc) * int(k)) for n, k in zip(job.lens_host, job.keep_host))
     v_read = v_rows * w.Hkv * w.D * w.elem_bytes
 
-    # Sequence by sequence: the upload of sequence b + 1 (copy stream) runs under the compression
-    # and the decode steps of sequence b (the caller's stream); one sequence's tensors are dense,
-    # so the same entry points take them as a batch of one.
+    # Part by part -- a part is a group of consecutive layers of one sequence, whose tensors are
+    # dense, so the same entry points take it as a batch of one with fewer layers: the upload of
+    # the next part (copy stream) runs under the compression and the decode steps of this one
+    # (the caller's stream).  The smaller the parts, the less of the step runs with the link idle
+    # (the first upload, the last part's decode steps).
     comp = torch.cuda.current_stream()
     copy = torch.cuda.Stream()
+    n_groups = max(1, min(w.L, args.e2e_layer_groups))
+    bounds = [round(i * w.L / n_groups) for i in range(n_groups + 1)]
+    parts = [(b, l0, l1) for b in range(w.B) for l0, l1 in zip(bounds[:-1], bounds[1:]) if l1 > l0]
+    l2 = job.l2
+
+    def run_part(b, l0, l1, V):
+        i, ls = slice(b, b + 1), slice(l0, l1)
+        unc = tuple(l - l0 for l in job.unc if l0 <= l < l1)
+        l2.select_compact(job.K[i, ls], V[i, ls], job.lens[i], job.keep[i], job.max_in, unc,
+                          job.K_c[i, ls], job.V_c[i, ls], job.idx[i, ls], job.sumsq[i, ls], job.cur[i, ls],
+                          job.ws)
+        for s in range(w.decode_steps):
+            if w.append_steps:
+                k, v = job.new_rows[s]
+                l2.append_evict(job.K_c[i, ls], job.V_c[i, ls], job.idx[i, ls], job.sumsq[i, ls],
+                                job.cur[i, ls], job.keep[i], unc, k[i, ls], v[i, ls], job.new_pos[s][i],
+                                job.ws)
+            l2.decode_attention(job.q_step[s][i, ls], job.K_c[i, ls], job.V_c[i, ls], job.cur[i, ls],
+                                job.max_dec, job.out_step[s][i, ls], job.ws)
 
     def step(copy_v):
         copy.wait_stream(comp)                          # the last step is done with the buffers
         landed = []
         with torch.cuda.stream(copy):
             job.q.copy_(qh, non_blocking=True)
-            for b in range(w.B):
-                job.K[b].copy_(Kh[b], non_blocking=True)
+            for b, l0, l1 in parts:
+                job.K[b, l0:l1].copy_(Kh[b, l0:l1], non_blocking=True)
                 if copy_v:
-                    job.V[b].copy_(Vh[b], non_blocking=True)
+                    job.V[b, l0:l1].copy_(Vh[b, l0:l1], non_blocking=True)
                 ev = torch.cuda.Event()
                 ev.record(copy)
                 landed.append(ev)
-        for b in range(w.B):
-            comp.wait_event(landed[b])
-            job.compress(b, V=None if copy_v else Vh)
-            for s in range(w.decode_steps):
-                job.decode(s, b)
+        for ev, (b, l0, l1) in zip(landed, parts):
+            comp.wait_event(ev)
+            run_part(b, l0, l1, job.V if copy_v else Vh)
         oh.copy_(job.out, non_blocking=True)
 
     def timed(copy_v):
@@ -676,15 +695,19 @@ def run_e2e(job, w, step_bytes, world, device, args):
         return {"value": round(world * step_bytes / (ms_all * 1e-3) / 1e9, 1), "unit": "GB/s",
                 "ms_per_step": round(ms_all, 2), "steps": n, "h2d_bytes_per_step": 2 * kv_bytes + q_bytes,
                 "d2h_bytes_per_step": d2h, "outputs_equal_device_resident_step": same_all,
-                "schedule": "per sequence: upload of sequence b+1 overlaps compress + decode of sequence b"}
+                "parts_per_step": len(parts),
+                "schedule": "per part (some layers of one sequence): the upload of the next part overlaps "
+                            "compress + decode of this one"}
     ms_dem, _, same_dem = timed(False)
     del Kh, Vh
     rate = lambda ms: round(world * step_bytes / (ms * 1e-3) / 1e9, 1)
     return {"value": rate(ms_dem), "unit": "GB/s", "ms_per_step": round(ms_dem, 2), "steps": n,
             "h2d_bytes_per_step": kv_bytes + q_bytes + v_read, "d2h_bytes_per_step": d2h,
             "outputs_equal_device_resident_step": same_dem,
-            "schedule": "per sequence: upload of K of sequence b+1 overlaps compress + decode of sequence b; "
-                        "V stays in pinned host memory and the compression reads only the rows it keeps",
+            "parts_per_step": len(parts),
+            "schedule": "per part (some layers of one sequence): the upload of K of the next part overlaps "
+                        "compress + decode of this one; V stays in pinned host memory and the compression "
+                        "reads only the rows it keeps",
             "copy_everything": {"value": rate(ms_all), "ms_per_step": round(ms_all, 2),
                                 "h2d_bytes_per_step": 2 * kv_bytes + q_bytes,
                                 "outputs_equal_device_resident_step": same_all}}
@@ -803,6 +826,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="l2kv", choices=["l2kv", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--e2e-layer-groups", type=int, default=4,
+                    help="the end-to-end schedule cuts every sequence into this many groups of layers")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-variants", action="store_true")
