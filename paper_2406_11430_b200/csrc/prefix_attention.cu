@@ -14,6 +14,7 @@
 // Two kernels share these pieces: the pipelined one (default) and a basic single-role one.
 // Every wait on an mbarrier is bounded (a wait that gives up ends the CTA's loop and marks
 // the status word); tensor memory is released on every path.
+#include <climits>
 #include <cmath>
 #include <cstdlib>
 #include <cstring>
@@ -474,8 +475,8 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
   constexpr int NS = kPfStages;
   extern __shared__ unsigned char smem_raw[];
   // mbarriers: K landed [NS], V landed [NS], K tile free [NS], V tile free [NS], then per query
-  // tile: scores ready [2], weights ready [2], output quiet [1]
-  __shared__ __align__(8) unsigned long long s_bar[4 * NS + 10];
+  // tile: scores ready [2], weights ready [2], output quiet [1], output complete [1]
+  __shared__ __align__(8) unsigned long long s_bar[4 * NS + 12];
   __shared__ uint32_t s_tmem;
   __shared__ int s_fail;
 
@@ -532,10 +533,13 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
   auto bar_v = [&](int i) { return bar0 + 8u * (uint32_t)(NS + i); };
   auto bar_kfree = [&](int i) { return bar0 + 8u * (uint32_t)(2 * NS + i); };
   auto bar_vfree = [&](int i) { return bar0 + 8u * (uint32_t)(3 * NS + i); };
-  const uint32_t bar_t = bar0 + 8u * (uint32_t)(4 * NS + 5 * tile);   // this query tile's five
+  const uint32_t bar_t = bar0 + 8u * (uint32_t)(4 * NS + 6 * tile);   // this query tile's six
   auto bar_s = [&](int i) { return bar_t + 8u * (uint32_t)i; };
   auto bar_p = [&](int i) { return bar_t + 8u * (uint32_t)(2 + i); };
-  const uint32_t bar_o = bar_t + 32u;
+  // bar_o completes a phase per P V (a waiter that is two phases behind would read its parity
+  // wrongly, so only the rescaling path, which is at most one behind, waits on it); bar_done
+  // completes once, behind the last P V
+  const uint32_t bar_o = bar_t + 32u, bar_done = bar_t + 40u;
 
   if (warp == 0) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
@@ -546,10 +550,10 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
     for (int i = 0; i < 2 * NS; ++i) mbar_init(bar0 + 8u * i, 1);
     for (int i = 2 * NS; i < 4 * NS; ++i) mbar_init(bar0 + 8u * i, n_tiles);   // one commit per query tile
     for (int t = 0; t < 2; ++t) {
-      const uint32_t bt = bar0 + 8u * (uint32_t)(4 * NS + 5 * t);
+      const uint32_t bt = bar0 + 8u * (uint32_t)(4 * NS + 6 * t);
       mbar_init(bt, 1); mbar_init(bt + 8, 1);
       mbar_init(bt + 16, kPfRows / 32); mbar_init(bt + 24, kPfRows / 32);   // one arrival per softmax warp
-      mbar_init(bt + 32, 1);
+      mbar_init(bt + 32, 1); mbar_init(bt + 40, 1);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     s_fail = 0;
@@ -642,6 +646,7 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
         if (j + 2 < nb) { tc_fence_after(); issue_qk(j + 2); }
 #endif
       }
+      if (ok) umma_commit(bar_done);                    // behind every P V of this query tile
       if (!ok) s_fail = 1;
     }
   } else if (tile_active) {
@@ -724,8 +729,8 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
       __syncwarp();                                       // the warp's 32 rows are in place:
       if ((tid & 31) == 0) mbar_arrive(bar_p(s));         // one arrival per warp
     }
-    // O is complete when the last P V has been committed
-    if (!gave_up && !mbar_wait<kPfPolls>(bar_o, (uint32_t)(nb - 1) & 1u)) gave_up = true;
+    // O is complete when the commit behind the last P V has arrived
+    if (!gave_up && !mbar_wait<kPfPolls>(bar_done, 0)) gave_up = true;
     if (gave_up) s_fail = 1;
   }
   __syncthreads();                                       // every role is done with the loop
@@ -750,6 +755,506 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
       lse_out[row_off] = (m_ref + log2f(l_tot)) * 0.6931471805599453f;
   }
   if (failed && tid == 0) record_timeout(status_word);
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0)
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(s_tmem), "r"(kPfPipeTmemCols)
+                 : "memory");
+}
+
+// The persistent, work-balanced kernel (L2KV_PREFIX_KERNEL=persistent; needs a workspace with
+// room for its partial results).  The pipelined kernel's roles and hand-offs, but a fixed grid of
+// kPfPersistCtas CTAs, each of which stays on its SM and walks an equal share of the call's work:
+//   - a work item is (pair of query tiles, unit); its cost is its number of 64-token sub-blocks.
+//     Every CTA adds up the costs of all items (the lengths live in device memory) and takes the
+//     range [c P, (c + 1) P) of the running total, P = ceil(total / CTAs): whole items, plus at
+//     most one item cut at its start and one cut at its end;
+//   - an item that lies in one CTA's range is written straight to out / lse_out; the pieces of a
+//     cut item go, normalised and with their log-sum-exp, to two slots per CTA in the workspace
+//     (slot 2c: the piece that is CTA c's first segment; 2c + 1: a piece that begins inside its
+//     range); the CTA that hands in an item's last piece (a counter per cut item) adds them up;
+//   - tensor memory, the mbarriers and the K / V rings are set up once; the fetching threads run
+//     ahead across item boundaries; between two segments the softmax threads write the next
+//     query rows into shared memory and tell the issuing thread (one more mbarrier per tile).
+constexpr int kPfPersistCtas = 148;
+constexpr int kPfSlotRows = 2 * kPfRows;         // rows of one partial result: both query tiles
+constexpr int kPfMinShare = 16;                  // sub-blocks: no share below 1024 tokens
+
+template <int G, bool SW>
+__global__ void __launch_bounds__(kPfPipeThreads, 1)
+prefix_attention_persistent_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n_queries,
+                           LenView cur_len_dev, int max_len, float scale_log2e,
+                           float* __restrict__ out, float* __restrict__ lse_out,
+                           const __grid_constant__ CUtensorMap map_k,
+                           const __grid_constant__ CUtensorMap map_v,
+                           int32_t* __restrict__ status_word, float* __restrict__ part_out,
+                           float* __restrict__ part_lse, int* __restrict__ tickets, int causal) {
+  constexpr int D = 128;
+  constexpr int QT = kPfRows / G;                       // queries per query tile
+  constexpr int NS = kPfStages;
+  constexpr int NT = kPfPipeThreads;
+  extern __shared__ unsigned char smem_raw[];
+  // mbarriers: K landed [NS], V landed [NS], K tile free [NS], V tile free [NS], then per query
+  // tile: scores ready [2], weights ready [2], output quiet [1], query rows ready [1], the
+  // segment's output complete [1]; then: a piece's rows written [1], its turn known [1]
+  __shared__ __align__(8) unsigned long long s_bar[4 * NS + 16];
+  __shared__ int s_merge;                               // this CTA handed in the item's last piece
+  __shared__ uint32_t s_tmem;
+  __shared__ int s_fail;
+  __shared__ int s_sum[NT / 32];
+  __shared__ unsigned long long s_first;                // first item of this CTA's walk
+  __shared__ int s_first_at;                            // running total before that item
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int cta = (int)blockIdx.x, n_cta = (int)gridDim.x;
+  const int q_tiles = (n_queries + QT - 1) / QT;
+  const int q_pairs = (q_tiles + 1) / 2;
+  // items are numbered pair-major (item = pair * units + unit): CTAs a whole number of units apart
+  // then walk the same K and V rows at about the same time, and the second read hits the L2
+  const long long units = (long long)g.B * g.L * g.H;
+  const long long items = units * q_pairs;
+  // A wait that gave up in an earlier call marks the workspace; nothing runs until it is cleared.
+  if (status_word && *reinterpret_cast<volatile int32_t*>(status_word + 2) != 0) return;
+
+  // cached rows of item `it`, and its cost in sub-blocks
+  auto item_rows = [&](long long it) {
+    const long long unit = it % units, bl = unit / g.H;
+    return max(0, min(cur_len_dev.at(bl, (int)(unit % g.H), g.H), min(max_len, g.cap(bl))));
+  };
+  auto item_cost = [&](long long it) { return (item_rows(it) + kPfSub - 1) / kPfSub; };
+
+  // ---- every CTA adds up all costs: thread t takes the items [t chunk, (t + 1) chunk) -----------
+  const long long chunk = (items + NT - 1) / NT;
+  const long long c_lo = min(items, (long long)tid * chunk), c_hi = min(items, c_lo + chunk);
+  int mine = 0;
+  for (long long it = c_lo; it < c_hi; ++it) mine += item_cost(it);
+  int incl = mine;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const int o = __shfl_up_sync(0xffffffffu, incl, off);
+    if (lane >= off) incl += o;
+  }
+  if (lane == 31) s_sum[warp] = incl;
+  if (tid == 0) { s_first = ~0ull; s_first_at = 0; s_fail = 0; }
+  __syncthreads();
+  int before = incl - mine, total = 0;
+  for (int w = 0; w < NT / 32; ++w) {
+    if (w < warp) before += s_sum[w];
+    total += s_sum[w];
+  }
+  // The CTAs are dealt out in equal groups, one per pair of query tiles (every pair's items cost
+  // the same: the costs depend on the unit alone), when the grid divides that way: CTA c of one
+  // group and CTA c of the next then walk the same K and V rows at the same time, and one of the
+  // two reads hits the L2.  Otherwise one group takes everything.
+  const int groups = (total > 0 && n_cta % q_pairs == 0) ? q_pairs : 1;
+  const int per_group = n_cta / groups, group_total = total / groups;
+  const int share = max(kPfMinShare, (group_total + per_group - 1) / per_group);
+  // first position of CTA c's range, and the CTA whose range holds position x (x < total)
+  auto lo_of = [&](int c) {                              // (a group's surplus CTAs get its end: nothing)
+    const long long g0 = (long long)(c / per_group) * group_total;
+    return (int)min(g0 + (long long)(c % per_group) * share, g0 + group_total);
+  };
+  auto cta_of = [&](int x) {
+    const int grp = min(groups - 1, x / max(group_total, 1));
+    return grp * per_group + min(per_group - 1, (x - grp * group_total) / share);
+  };
+  // this CTA's range of the running total; the last CTA's is open-ended (trailing empty items)
+  const int lo = lo_of(cta);
+  const int hi = cta == n_cta - 1 ? INT_MAX
+               : (cta % per_group == per_group - 1 ? (cta / per_group + 1) * group_total
+                                                  : min(lo_of(cta) + share, (cta / per_group + 1) * group_total));
+  // the walk starts at the first item that reaches past lo, or begins at or after it
+  {
+    int at = before;
+    for (long long it = c_lo; it < c_hi; ++it) {
+      const int c = item_cost(it);
+      if (at + c > lo || at >= lo) { atomicMin(&s_first, (unsigned long long)it); break; }
+      at += c;
+    }
+  }
+  __syncthreads();
+  {
+    int at = before;
+    for (long long it = c_lo; it < c_hi; ++it) {
+      if ((unsigned long long)it == s_first) { s_first_at = at; break; }
+      at += item_cost(it);
+    }
+  }
+
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;   // 1024-byte aligned tiles
+  const bool softmax_thread = tid < 2 * kPfRows;
+  const int tile = softmax_thread ? tid >> 7 : warp & 1;
+  const int row = tid & (kPfRows - 1);
+  const int wq = warp & 3;                              // tensor-memory lane quarter of this warp
+  const uint32_t sQ = base + (uint32_t)tile * kPfTileBytes;
+  const uint32_t sK = base + 2 * kPfTileBytes, sV = sK + NS * kPfSubTile;
+  const uint32_t bar0 = smem_u32(&s_bar[0]);
+  auto bar_k = [&](int i) { return bar0 + 8u * (uint32_t)i; };
+  auto bar_v = [&](int i) { return bar0 + 8u * (uint32_t)(NS + i); };
+  auto bar_kfree = [&](int i) { return bar0 + 8u * (uint32_t)(2 * NS + i); };
+  auto bar_vfree = [&](int i) { return bar0 + 8u * (uint32_t)(3 * NS + i); };
+  const uint32_t bar_t = bar0 + 8u * (uint32_t)(4 * NS + 7 * tile);   // this query tile's seven
+  auto bar_s = [&](int i) { return bar_t + 8u * (uint32_t)i; };
+  auto bar_p = [&](int i) { return bar_t + 8u * (uint32_t)(2 + i); };
+  const uint32_t bar_o = bar_t + 32u, bar_q = bar_t + 40u, bar_done = bar_t + 48u;
+  const uint32_t bar_piece = bar0 + 8u * (uint32_t)(4 * NS + 14), bar_turn = bar_piece + 8u;
+
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 :: "r"(smem_u32(&s_tmem)), "r"(kPfPipeTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  if (tid == 0) {
+    for (int i = 0; i < 2 * NS; ++i) mbar_init(bar0 + 8u * i, 1);
+    for (int i = 2 * NS; i < 4 * NS; ++i) mbar_init(bar0 + 8u * i, 2);     // one arrival per query tile
+    for (int t = 0; t < 2; ++t) {
+      const uint32_t bt = bar0 + 8u * (uint32_t)(4 * NS + 7 * t);
+      mbar_init(bt, 1); mbar_init(bt + 8, 1);
+      mbar_init(bt + 16, kPfRows / 32); mbar_init(bt + 24, kPfRows / 32);   // one arrival per softmax warp
+      mbar_init(bt + 32, 1);
+      mbar_init(bt + 40, kPfRows / 32);
+      mbar_init(bt + 48, 1);
+    }
+    mbar_init(bar_piece, 2 * kPfRows / 32);               // one arrival per softmax warp, both tiles
+    mbar_init(bar_turn, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = s_tmem + (uint32_t)tile * 256;  // this query tile's 256 columns
+  const uint32_t t_lane = tmem + ((uint32_t)(wq * 32) << 16);
+  const uint32_t t_o = t_lane + 128;                    // this row's 128 output dims
+
+  // Every thread that has a role walks the same segments: (item, sub-blocks [j0, j1) of it).
+  long long w_it = (long long)s_first;
+  int w_at = s_first_at;
+  long long it = 0;                                     // the segment's item
+  int at = 0, cost = 0, j0 = 0, j1 = 0;                 // its place in the total, cost, sub-block range
+  auto next_segment = [&]() {
+    if (w_it < 0 || w_it >= items || w_at >= hi) return false;
+    it = w_it; at = w_at; cost = item_cost(it);
+    j0 = max(0, lo - at); j1 = min(cost, hi - at);
+    ++w_it; w_at += cost;
+    return true;
+  };
+  int jj = 0;                                           // sub-blocks this CTA has been through
+  bool gave_up = false;
+
+  if (!softmax_thread) {
+    if (lane == 0 && warp >= 10) {
+      // ---- the two fetching threads: K tiles (warp 10), V tiles (warp 11) ---------------------
+      const bool is_k = warp == 10;
+      const CUtensorMap* map = is_k ? &map_k : &map_v;
+      bool ok = true;
+      while (ok && next_segment()) {
+        const long long unit = it % units, bl = unit / g.H;
+        const int h = (int)(unit % g.H);
+        const int tm_row = (int)g.row0(bl);
+        const int tm_l = g.row_off ? 0 : (int)(bl % g.L), tm_b = g.row_off ? 0 : (int)(bl / g.L);
+        for (int j = j0; ok && j < j1; ++j, ++jj) {
+          const int st = jj % NS, use = jj / NS;
+          const uint32_t full = is_k ? bar_k(st) : bar_v(st);
+          if (use > 0) ok = mbar_wait<kPfPolls>(is_k ? bar_kfree(st) : bar_vfree(st), (uint32_t)(use - 1) & 1u);
+          if (!ok) break;
+          const uint32_t dst = (is_k ? sK : sV) + st * kPfSubTile;
+          mbar_expect_tx(full, kPfSubTile);
+          tma_load_5d(dst, map, full, 0, tm_row + j * kPfSub, h, tm_l, tm_b);
+          tma_load_5d(dst + kPfSubHalf, map, full, 64, tm_row + j * kPfSub, h, tm_l, tm_b);
+        }
+      }
+      if (!ok) s_fail = 1;
+    } else if (lane == 0) {
+      // ---- the issuing thread of query tile `tile` ---------------------------------------------
+      // S[a & 1] = Q K^T for the K tile at ring position x; a counts this query tile's sub-blocks
+      auto issue_qk = [&](int x, int a) {
+        const uint32_t kt = sK + (x % NS) * kPfSubTile;
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+          umma_bf16(tmem + (a & 1) * 64,
+                    umma_desc(sQ + (k >> 2) * kPfHalf + (k & 3) * 32, 16, 1024),
+                    umma_desc(kt + (k >> 2) * kPfSubHalf + (k & 3) * 32, 16, 1024), kIdescQK64, k > 0);
+        umma_commit(bar_s(a & 1));
+        umma_commit(bar_kfree(x % NS));
+      };
+      bool ok = true;
+      int seg = 0, ja = 0;                              // segments / sub-blocks this tile took part in
+      while (ok && next_segment()) {
+        const int nbs = j1 - j0;
+        if (nbs <= 0) continue;
+        const int qp = (int)(it / units);
+        if (2 * qp + tile >= q_tiles) {
+          // this query tile does not exist in the item: hand every K and V tile back as it lands
+          for (int x = jj; ok && x < jj + nbs; ++x) {
+            ok = mbar_wait<kPfPolls>(bar_k(x % NS), (uint32_t)(x / NS) & 1u);
+            if (ok) mbar_arrive(bar_kfree(x % NS));
+            ok = ok && mbar_wait<kPfPolls>(bar_v(x % NS), (uint32_t)(x / NS) & 1u);
+            if (ok) mbar_arrive(bar_vfree(x % NS));
+          }
+          jj += nbs;
+          continue;
+        }
+        ok = mbar_wait<kPfPolls>(bar_q, (uint32_t)seg & 1u);          // the segment's query rows
+        ++seg;
+        if (ok) ok = mbar_wait<kPfPolls>(bar_k(jj % NS), (uint32_t)(jj / NS) & 1u);
+        if (ok) { tc_fence_after(); issue_qk(jj, ja); }
+        if (ok && nbs > 1) {
+          ok = mbar_wait<kPfPolls>(bar_k((jj + 1) % NS), (uint32_t)((jj + 1) / NS) & 1u);
+          if (ok) { tc_fence_after(); issue_qk(jj + 1, ja + 1); }
+        }
+        const int end = jj + nbs;
+        for (int x = jj; ok && x < end; ++x) {
+          const int a = ja + (x - jj), s = a & 1;
+          ok = mbar_wait_likely(bar_v(x % NS), (uint32_t)(x / NS) & 1u);
+          if (ok && x + 2 < end) ok = mbar_wait_likely(bar_k((x + 2) % NS), (uint32_t)((x + 2) / NS) & 1u);
+          ok = ok && mbar_wait<kPfPolls>(bar_p(s), (uint32_t)(a >> 1) & 1u);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t vt = sV + (x % NS) * kPfSubTile;
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {                 // O += P V; slice k = tokens 16k .. 16k + 15
+            umma_bf16_ts(tmem + 128, tmem + s * 64 + k * 8,
+                         umma_desc(vt + k * 2048, kPfSubHalf, 1024), kIdescPV, (x > jj || k > 0) ? 1u : 0u);
+            if constexpr (SW)
+              umma_bf16_ts(tmem + 128, tmem + s * 64 + 32 + k * 8,
+                           umma_desc(vt + k * 2048, kPfSubHalf, 1024), kIdescPV, 1u);
+          }
+          umma_commit(bar_o);
+          umma_commit(bar_vfree(x % NS));
+          // queued right behind P V, whose weights it overwrites: the tensor core executes this
+          // thread's operations in issue order (see the pipelined kernel)
+          if (x + 2 < end) issue_qk(x + 2, a + 2);
+        }
+        if (ok) umma_commit(bar_done);                  // behind every P V of the segment
+        jj = end;
+        ja += nbs;
+      }
+      if (!ok) s_fail = 1;
+    }
+  } else {
+    // ---- the softmax warps of query tile `tile`: one thread per row ------------------------------
+    int seg = 0, ja = 0;                                // segments / sub-blocks this tile took part in
+    int pieces = 0;                                     // partial results this CTA has written
+    while (!gave_up && next_segment()) {
+      const long long unit = it % units, bl = unit / g.H;
+      const int qp = (int)(it / units), h = (int)(unit % g.H);
+      const int s_idx = (2 * qp + tile) * QT + row / G;     // this row's query and head
+      const int head = h * G + row % G;
+      const bool row_valid = s_idx < n_queries;
+      const long long row_off = ((bl * n_queries + s_idx) * g.Hq + head);
+      if (cost == 0) {                                    // empty cache: zeros, log-sum-exp = -inf
+        if (row_valid) {
+          for (int d = 0; d < D; ++d) out[row_off * D + d] = 0.f;
+          if (lse_out) lse_out[row_off] = -INFINITY;
+        }
+        continue;
+      }
+      const int nbs = j1 - j0;
+      if (nbs <= 0) continue;
+      const bool partial = j0 > 0 || j1 < cost;
+      const int slot = (j0 > 0 || at == lo) ? 2 * cta : 2 * cta + 1;
+      const bool active = 2 * qp + tile < q_tiles;
+      if (!active) jj += nbs;
+      if (active) {
+      const int n_all = item_rows(it);
+      // causal: the last n_queries cached rows are the new tokens' own; query s stops at its own
+      const int n_row = causal && row_valid ? min(n_all, max(0, n_all - n_queries + s_idx + 1)) : n_all;
+      {                                                   // Q row, K-major, 128-byte swizzle
+        const uint4* src = reinterpret_cast<const uint4*>(q + row_off * D);
+#pragma unroll
+        for (int c = 0; c < 16; ++c) {
+          const uint4 v = row_valid ? src[c] : make_uint4(0, 0, 0, 0);
+          st_shared16(sQ + (c >> 3) * kPfHalf + row * 128 + (((c & 7) ^ (row & 7)) << 4), v.x, v.y, v.z, v.w);
+        }
+        proxy_fence();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_q);
+      }
+      float m_ref = -INFINITY, l_run = 0.f;               // reference maximum; sum of this row's weights
+      const int end = jj + nbs;
+      for (int x = jj; x < end; ++x) {
+        const int j = j0 + (x - jj);                      // sub-block of the item
+        const int a = ja + (x - jj), s = a & 1;
+        const int valid = min(kPfSub, n_all - j * kPfSub);   // valid tokens of this sub-block
+        const uint32_t t_s = t_lane + s * 64;               // this row's scores, later its weights
+        if (!mbar_wait_likely(bar_s(s), (uint32_t)(a >> 1) & 1u)) gave_up = true;
+        tc_fence_after();
+        if (__any_sync(0xffffffffu, gave_up)) { gave_up = true; break; }
+        float sv[64];                                     // raw products; the scale is folded in below
+        float bmax = -INFINITY;
+        {
+          uint32_t r0[32], r1[32];
+          tmem_ld64(t_s, r0, r1);
+          const int valid_row = min(valid, n_row - j * kPfSub);
+          if (valid_row >= kPfSub) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              sv[i] = __uint_as_float(r0[i]);
+              sv[32 + i] = __uint_as_float(r1[i]);
+              bmax = fmaxf(bmax, fmaxf(sv[i], sv[32 + i]));
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              sv[i] = i < valid_row ? __uint_as_float(r0[i]) : -INFINITY;
+              sv[32 + i] = 32 + i < valid_row ? __uint_as_float(r1[i]) : -INFINITY;
+              bmax = fmaxf(bmax, fmaxf(sv[i], sv[32 + i]));
+            }
+          }
+        }
+        const float m_new = fmaxf(m_ref, bmax * scale_log2e);
+        if (x == jj) m_ref = m_new;
+        const bool need = m_new > m_ref + kPfRescaleGap;
+        if (__any_sync(0xffffffffu, need)) {
+          // O must be quiet: the previous P V has to be complete (this one waits for this thread)
+          if (!mbar_wait<kPfPolls>(bar_o, (uint32_t)(a - 1) & 1u)) gave_up = true;
+          tc_fence_after();
+          const float factor = need ? fast_exp2(m_ref - m_new) : 1.f;
+#pragma unroll 1
+          for (int c = 0; c < D; c += 8) tmem_scale8(t_o + c, factor);
+          if (need) { l_run *= factor; m_ref = m_new; }
+        }
+        {
+          uint32_t pk[32];
+          [[maybe_unused]] uint32_t pr[SW ? 32 : 1];
+          float rowsum0 = 0.f, rowsum1 = 0.f;
+          const float neg_m = m_ref == -INFINITY ? 0.f : -m_ref;   // a row with nothing to see yet
+#pragma unroll
+          for (int i = 0; i < 64; i += 2) {
+            const float p0 = fast_exp2(__fmaf_rn(sv[i], scale_log2e, neg_m));     // -inf -> 0
+            const float p1 = fast_exp2(__fmaf_rn(sv[i + 1], scale_log2e, neg_m));
+            rowsum0 += p0;
+            rowsum1 += p1;
+            pk[i >> 1] = pack_bf16(p0, p1);
+            if constexpr (SW) pr[i >> 1] = pack_bf16_rest(p0, p1, pk[i >> 1]);
+          }
+          tmem_st32(t_s, pk);
+          if constexpr (SW) tmem_st32(t_s + 32, pr);
+          tmem_wait_st();
+          l_run += rowsum0 + rowsum1;
+        }
+        if (valid < kPfSub) {
+          // partial sub-block: clear the V rows past the valid length (both query tiles write
+          // the same zeros) so that a zero weight times Inf/NaN cannot reach O
+          if (!mbar_wait<kPfPolls>(bar_v(x % NS), (uint32_t)(x / NS) & 1u)) gave_up = true;
+          if (row >= valid && row < kPfSub) {
+#pragma unroll
+            for (int c = 0; c < 16; ++c)
+              st_shared16(sV + (x % NS) * kPfSubTile + (c >> 3) * kPfSubHalf + row * 128 + ((c & 7) << 4), 0, 0, 0, 0);
+          }
+          proxy_fence();
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_p(s));             // one arrival per warp
+      }
+      if (gave_up) break;
+      // the segment's O is complete when the commit behind its last P V has arrived
+      if (!mbar_wait<kPfPolls>(bar_done, (uint32_t)seg & 1u)) { gave_up = true; break; }
+      ++seg;
+      tc_fence_after();
+      jj = end;
+      ja += nbs;
+      {
+        const float inv = l_run > 0.f ? 1.f / l_run : 0.f;   // nothing seen: zeros, log-sum-exp -inf
+        const long long p_row = (long long)slot * kPfSlotRows + tile * kPfRows + row;
+        float* dst_row = partial ? part_out + p_row * D : out + row_off * D;
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+          uint32_t r[32];
+          tmem_ld32(t_o + c * 32, r);
+          if (row_valid) {
+            float4* dst = reinterpret_cast<float4*>(dst_row + c * 32);
+#pragma unroll
+            for (int i = 0; i < 32; i += 4)
+              dst[i >> 2] = make_float4(__uint_as_float(r[i]) * inv, __uint_as_float(r[i + 1]) * inv,
+                                        __uint_as_float(r[i + 2]) * inv, __uint_as_float(r[i + 3]) * inv);
+          }
+        }
+        const float lse = (m_ref + log2f(l_run)) * 0.6931471805599453f;
+        if (row_valid) {
+          if (partial) part_lse[p_row] = lse;
+          else if (lse_out) lse_out[row_off] = lse;
+        }
+        tc_fence_before();                                // O has been read before the next segment's P V
+      }
+      }
+      if (gave_up) break;
+      if (partial) {
+        // A piece of a cut item: once both tiles' rows are in the workspace, this CTA takes a
+        // ticket of the item (counter of the CTA the item starts in); whoever takes the last one
+        // adds the pieces up.  Nobody waits for another CTA; the counter goes back to zero.
+        const int c_first = cta_of(at), c_last = cta_of(at + cost - 1);
+        __threadfence();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_piece);
+        if (!mbar_wait<kPfPolls>(bar_piece, (uint32_t)pieces & 1u)) { gave_up = true; break; }
+        if (tid == 0) {
+          const int turn = atomicAdd(tickets + c_first, 1);
+          s_merge = turn == c_last - c_first;
+          if (s_merge) tickets[c_first] = 0;
+          __threadfence();
+          mbar_arrive(bar_turn);
+        }
+        if (!mbar_wait<kPfPolls>(bar_turn, (uint32_t)pieces & 1u)) { gave_up = true; break; }
+        ++pieces;
+        if (s_merge && active) {
+          // A warp adds up its 32 rows together: every lane works out the weights of its own
+          // row's pieces, then the lanes go through the rows side by side (a row is 32 float4),
+          // 8 rows' loads in flight at a time.
+          __threadfence();
+          const int r = tile * kPfRows + row;
+          auto slot_of = [&](int p) { return p == c_first ? (at == lo_of(c_first) ? 2 * p : 2 * p + 1) : 2 * p; };
+          float m = -INFINITY;
+          if (row_valid)
+            for (int p = c_first; p <= c_last; ++p)
+              m = fmaxf(m, __ldcg(part_lse + (long long)slot_of(p) * kPfSlotRows + r));
+          float den = 0.f;
+          if (row_valid)
+            for (int p = c_first; p <= c_last; ++p) {
+              const float lp = __ldcg(part_lse + (long long)slot_of(p) * kPfSlotRows + r);
+              den += lp > -INFINITY ? __expf(lp - m) : 0.f;
+            }
+          const bool any = m > -INFINITY;                 // some piece had rows this query may see
+          const float inv = any ? 1.f / den : 0.f;
+          const uint32_t valid_rows = __ballot_sync(0xffffffffu, row_valid);
+          const int r_warp = r - lane;                    // first row of this warp
+#pragma unroll 1
+          for (int part = 0; part < 4; ++part) {
+            float4 acc[8] = {};
+            for (int p = c_first; p <= c_last; ++p) {
+              const long long pr = (long long)slot_of(p) * kPfSlotRows + r;
+              const float lp = row_valid ? __ldcg(part_lse + pr) : -INFINITY;
+              const float w = lp > -INFINITY ? __expf(lp - m) * inv : 0.f;
+              const float4* src = reinterpret_cast<const float4*>(
+                  part_out + ((long long)slot_of(p) * kPfSlotRows + r_warp + part * 8) * D) + lane;
+              float4 v[8];
+#pragma unroll
+              for (int rr = 0; rr < 8; ++rr)
+                v[rr] = (valid_rows >> (part * 8 + rr)) & 1u ? __ldcg(src + rr * (D / 4))
+                                                              : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+              for (int rr = 0; rr < 8; ++rr) {
+                const float wr = __shfl_sync(0xffffffffu, w, part * 8 + rr);
+                acc[rr].x = fmaf(wr, v[rr].x, acc[rr].x); acc[rr].y = fmaf(wr, v[rr].y, acc[rr].y);
+                acc[rr].z = fmaf(wr, v[rr].z, acc[rr].z); acc[rr].w = fmaf(wr, v[rr].w, acc[rr].w);
+              }
+            }
+#pragma unroll
+            for (int rr = 0; rr < 8; ++rr) {
+              const long long ro = __shfl_sync(0xffffffffu, row_off, part * 8 + rr);
+              if ((valid_rows >> (part * 8 + rr)) & 1u)
+                reinterpret_cast<float4*>(out + ro * D)[lane] = acc[rr];
+            }
+          }
+          if (row_valid && lse_out) lse_out[row_off] = any ? m + logf(den) : -INFINITY;
+        }
+      }
+    }
+    if (gave_up) s_fail = 1;
+  }
+  __syncthreads();                                       // every role is done
+  if (s_fail != 0 && tid == 0) record_timeout(status_word);
   tc_fence_before();
   __syncthreads();
   if (warp == 0)
@@ -790,11 +1295,14 @@ prefix_merge_kernel(const float* __restrict__ part_out, const float* __restrict_
 // run half empty, and the single-role kernel with two CTAs per SM is the faster one
 // (L2KV_PREFIX_KERNEL=basic / =pipelined overrides the choice).  Chunks: the cache is split over
 // blockIdx.y, with a merge pass after, when the unsplit grid would leave SMs idle (few KV heads
-// and query tiles, as in a call for one layer) or when the cache is so long that (b, l) pairs of
-// different lengths would leave a few CTAs running alone (chunks of 16k tokens then); chunks
-// are multiples of 128 tokens and at least 1024 long.
+// and query tiles, as in a call for one layer); chunks are multiples of 128 tokens and at least
+// 1024 long.  A cache so long that (b, l) pairs of different lengths would leave a few CTAs
+// running alone at the end goes to the work-balanced persistent kernel instead
+// (L2KV_PREFIX_KERNEL=persistent asks for it anywhere), or, without the workspace it needs, is
+// split into chunks of 16k tokens if there is room for that.
 struct PrefixPlan {
   bool basic;
+  bool persistent;         // the work-balanced kernel was asked for and its totals fit 32 bits
   long long ctas;          // per chunk
   int chunks, split_len;
   long long rows;          // B * L * n_queries * Hq
@@ -809,6 +1317,13 @@ static PrefixPlan plan_prefix(const Geom& g, int n_queries, int max_len) {
   p.basic = (q_tiles & 1) && q_tiles < 9;
   if (which && std::strcmp(which, "basic") == 0) p.basic = true;
   if (which && std::strcmp(which, "pipelined") == 0) p.basic = false;
+  const long long pairs_all = (long long)g.B * g.L * g.H * ((q_tiles + 1) / 2);
+  // the work-balanced kernel: on request, and by itself for very long caches, where (b, l) pairs
+  // of different lengths would otherwise leave a few CTAs running alone at the end
+  const bool fits = pairs_all * ((long long)max_len / kPfSub + 1) < (long long)INT_MAX / 2;
+  if (which && std::strcmp(which, "persistent") == 0) p.basic = false;
+  p.persistent = fits && !p.basic &&
+                 ((which && std::strcmp(which, "persistent") == 0) || (!which && max_len >= 65536));
   const long long units = (long long)g.B * g.L * g.H;
   p.ctas = units * (p.basic ? q_tiles : (q_tiles + 1) / 2);
   p.rows = (long long)g.B * g.L * n_queries * g.Hq;
@@ -834,8 +1349,15 @@ static PrefixPlan plan_prefix(const Geom& g, int n_queries, int max_len) {
   return p;
 }
 
+// Scratch of the persistent kernel: a ticket counter per CTA, then the log-sum-exps and the rows
+// of the two partial results a CTA may write.
+constexpr size_t kPfCutBytes = (kPfPersistCtas * sizeof(int) + 255) / 256 * 256;   // the tickets
+constexpr size_t kPfPartLseBytes = (size_t)2 * kPfPersistCtas * kPfSlotRows * sizeof(float);
+constexpr size_t kPfPersistBytes = kPfCutBytes + kPfPartLseBytes * (1 + 128);
+
 size_t prefix_attention_scratch(const Geom& g, int n_queries, int max_len) {
-  return plan_prefix(g, n_queries, max_len).scratch_bytes;
+  const PrefixPlan p = plan_prefix(g, n_queries, max_len);
+  return p.persistent ? kPfPersistBytes : p.scratch_bytes;
 }
 
 template <int G, bool SW>
@@ -862,6 +1384,21 @@ static int launch_pf(const void* q, const void* K, const void* V, const Geom& g,
   float* k_lse = p.chunks > 1 ? scratch + (size_t)p.chunks * p.rows * 128 : lse_out;
   const dim3 grid((unsigned)p.ctas, (unsigned)p.chunks);
   const __nv_bfloat16* qb = static_cast<const __nv_bfloat16*>(q);
+  if (p.persistent && scratch && scratch_bytes >= kPfPersistBytes) {
+    constexpr int smem_pipe = 1024 + 2 * kPfTileBytes + 2 * kPfStages * kPfSubTile;
+    auto kern = prefix_attention_persistent_kernel<G, SW>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_pipe) != cudaSuccess)
+      return L2KV_ERR_CUDA;
+    char* sc = reinterpret_cast<char*>(scratch);
+    int* tickets = reinterpret_cast<int*>(sc);
+    if (cudaMemsetAsync(tickets, 0, kPfCutBytes, s) != cudaSuccess) return L2KV_ERR_CUDA;
+    float* part_lse = reinterpret_cast<float*>(sc + kPfCutBytes);
+    float* part_out = reinterpret_cast<float*>(sc + kPfCutBytes + kPfPartLseBytes);
+    kern<<<kPfPersistCtas, kPfPipeThreads, smem_pipe, s>>>(qb, g, n_queries, cur_len_dev, max_len,
+                                                          scale * kPfLog2e, out, lse_out, map_k, map_v,
+                                                          status_word, part_out, part_lse, tickets, causal);
+    return cudaGetLastError() == cudaSuccess ? L2KV_OK : L2KV_ERR_CUDA;
+  }
   if (!p.basic) {
     constexpr int smem_pipe = 1024 + 2 * kPfTileBytes + 2 * kPfStages * kPfSubTile;
     auto kern_pipe = prefix_attention_pipelined_kernel<G, SW>;

@@ -7,6 +7,8 @@ as two bf16 terms (16 significant bits) -- held to the decode path's bound
 weight, the usual arrangement of fused attention kernels) -- a documented reading with the
 absolute term 4e-3 (the error is largest for caches of a few hundred tokens, where few
 weights carry the sum); the RMS error is bounded separately."""
+import os
+
 import numpy as np
 import pytest
 import scipy.special
@@ -40,13 +42,16 @@ def run(l2, q, K, V, cur, max_len, scale=0.0, weights="single"):
     out = torch.full(q.shape, float("nan"), dtype=torch.float32, device=DEV)
     lse = torch.full(q.shape[:4], float("nan"), dtype=torch.float32, device=DEV)
     ws = torch.zeros(256, dtype=torch.uint8, device=DEV)
+    if os.environ.get("L2KV_PREFIX_KERNEL") == "persistent":      # that kernel needs room for cut items
+        ws = l2.prefix_attention_workspace(K, q, max_len)
     call(l2, weights, q, K, V, i32(np.asarray(cur)), max_len, out, lse, scale=scale, workspace=ws)
     torch.cuda.synchronize()
     assert l2.read_device_status(ws) == 0
     return out.cpu().numpy(), lse.cpu().numpy()
 
 
-KERNELS = ["pipelined", "basic", "auto"]      # the two kernels, and the library's own choice between them
+# the three kernels, and the library's own choice between them
+KERNELS = ["pipelined", "basic", "persistent", "auto"]
 
 
 def test_plain_entry_points_are_the_flagless_call():
@@ -196,8 +201,11 @@ def test_prefix_attention_causal(kernel, T, lens, n_q, split, weights, monkeypat
     K, V = synth.make_cache(w, DEV)
     q = make_queries(w, n_q, 13)
     cur = np.array([lens], dtype=np.int32)
-    ws = l2.prefix_attention_workspace(K, q, T) if split else torch.zeros(256, dtype=torch.uint8, device=DEV)
-    assert (ws.numel() > 256) == split
+    if kernel == "persistent":
+        ws = l2.prefix_attention_workspace(K, q, T)
+    else:
+        ws = l2.prefix_attention_workspace(K, q, T) if split else torch.zeros(256, dtype=torch.uint8, device=DEV)
+        assert (ws.numel() > 256) == split
     out = torch.full(q.shape, float("nan"), dtype=torch.float32, device=DEV)
     lse = torch.full(q.shape[:4], float("nan"), dtype=torch.float32, device=DEV)
     call(l2, weights, q, K, V, i32(cur), T, out, lse, workspace=ws, causal=True)
