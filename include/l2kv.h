@@ -264,10 +264,12 @@ int l2kv_append_evict(void* K_c, void* V_c, int32_t* idx, float* sumsq_c, const 
  * in FlashAttention.  An empty cache gives zeros and lse = -inf.  workspace may be NULL; if
  * given (>= 256 bytes, its first 256 zeroed) its status word reports a copy or MMA wait that
  * gave up.  With a workspace of l2kv_prefix_attention_workspace_bytes(lay, max_len, n_queries)
- * bytes the call may also split the cache into chunks handled by different thread blocks and
- * merge their results (the same rows up to the bf16 rounding of the weights): that keeps the GPU busy when there are few
- * KV heads and queries per call (one layer at a time) or when lengths differ widely between
- * (b, l) pairs.  With less room it runs unsplit. */
+ * bytes the call may also split the cache into pieces handled by different thread blocks and
+ * merge their results (the same rows up to the bf16 rounding of the weights): that keeps the
+ * GPU busy when there are few KV heads and queries per call (one layer at a time), and for
+ * very long caches (max_len >= 65536), whose (b, l) pairs may differ widely in length, the
+ * work is dealt out in equal shares to a fixed grid of resident thread blocks.  With less
+ * room it runs unsplit.  Beyond its first 256 bytes the workspace needs no initial contents. */
 int l2kv_prefix_attention_workspace_bytes(const l2kv_layout* lay, int32_t max_len,
                                           int32_t n_queries, size_t* bytes);
 /* The same for a prefill chunk whose own keys and values are already in the cache: the last
