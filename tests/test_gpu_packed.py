@@ -196,9 +196,15 @@ def test_packed_static_decode(l2):
     assert torch.equal(got, want)
 
 
-def test_packed_prefix_attention(l2):
+@pytest.mark.parametrize("kernel", ["auto", "persistent"])
+def test_packed_prefix_attention(l2, kernel, monkeypatch):
     """Several new queries per (b, l) over a packed compressed cache, plain and causal, both weight
-    precisions, against the packed oracle query by query; lengths differ per (b, l)."""
+    precisions, against the packed oracle query by query; lengths differ per (b, l).  With the
+    library's own choice of kernel and with the work-balanced one."""
+    if kernel == "auto":
+        monkeypatch.delenv("L2KV_PREFIX_KERNEL", raising=False)
+    else:
+        monkeypatch.setenv("L2KV_PREFIX_KERNEL", kernel)
     B, L, Hkv, Hq, D, Sq = 3, 2, 2, 8, 128, 40
     w = synth.WORKLOADS[2].scaled(B=B, L=L, Hkv=Hkv, Hq=Hq, T=64)
     caps = [[700, 90], [300, 1], [64, 1500]]

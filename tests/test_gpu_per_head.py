@@ -173,7 +173,7 @@ def test_append_evict_with_a_budget_per_head(l2, dtype, D):
 
 
 @pytest.mark.parametrize("weights", ["split", "single"])
-@pytest.mark.parametrize("kernel", ["pipelined", "basic"])
+@pytest.mark.parametrize("kernel", ["pipelined", "basic", "persistent"])
 def test_prefix_attention_with_a_length_per_head(l2, kernel, weights, monkeypatch):
     monkeypatch.setenv("L2KV_PREFIX_KERNEL", kernel)
     w = synth.WORKLOADS[2].scaled(B=1, L=2, Hkv=2, Hq=8, T=700)
@@ -184,6 +184,8 @@ def test_prefix_attention_with_a_length_per_head(l2, kernel, weights, monkeypatc
     out = torch.full(q.shape, float("nan"), dtype=torch.float32, device=DEV)
     lse = torch.full(q.shape[:4], float("nan"), dtype=torch.float32, device=DEV)
     ws = torch.zeros(256, dtype=torch.uint8, device=DEV)
+    if kernel == "persistent":                            # needs room for the pieces of cut items
+        ws = l2.prefix_attention_workspace(K, q, 700)
     if weights == "single":
         l2.prefix_attention_per_head(q, K, V, i32(cur), 700, out, lse, workspace=ws)
     else:
