@@ -128,14 +128,17 @@ def test_config2_llama3_8b_32k(l2):
     _free()
 
 
-def check_sampled_prefix_attention(l2, w, out, samples, n_q=128):
+def check_sampled_prefix_attention(l2, w, out, samples, n_q=128, room=False):
     """Prefix attention in the launch the benchmark times (128 queries per (b, l) over the whole
     compressed cache), plain and causal, both forms of the weights; the oracle recomputes the
-    sampled (b, l, kv head, query) rows with that row's own length."""
+    sampled (b, l, kv head, query) rows with that row's own length.  room: with the workspace
+    the library asks for (very long caches then go to the work-balanced kernel)."""
     g = torch.Generator().manual_seed(17)
     q = torch.randn((w.B, w.L, n_q, w.Hq, w.D), generator=g).to(torch.bfloat16).to(DEV)
     res = torch.empty(q.shape, dtype=torch.float32, device=DEV)
-    ws = torch.zeros(256, dtype=torch.uint8, device=DEV)
+    ws = (l2.prefix_attention_workspace(out["K_c"], q, w.T) if room
+          else torch.zeros(256, dtype=torch.uint8, device=DEV))
+    assert (ws.numel() > 256) == room
     G = w.Hq // w.Hkv
     cur = out["cur"].cpu().numpy()
     for causal in (False, True):
@@ -176,6 +179,11 @@ def test_config3_extreme_128k(l2):
     _free()
     q = synth.make_query(w, 0, DEV)
     check_sampled_attention(l2, w, out, q, w.T, units + [(0, 1, 2)])
+    _free()
+    # 128 queries over the whole compressed cache (two layers of 131072 rows, thirty of 13108):
+    # the work-balanced kernel, every item cut across several thread blocks
+    check_sampled_prefix_attention(l2, w, out, [(0, 0, 0, 0), (0, 1, 7, 127), (0, 2, 0, 64), (0, 30, 7, 31),
+                                               (0, 13, 4, 100)], room=True)
     _free()
 
 
