@@ -415,6 +415,40 @@ prefix_attention_basic_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n
                  : "memory");
 }
 
+// Epilogue of the kernels with one softmax thread per query row: this warp's 32 rows of O (128
+// fp32 each, in tensor memory at t_o, one row per lane) times the lane's `inv`, written to the
+// rows at `dst` (the lane's own destination row; nullptr: the row does not exist).  A thread
+// that stored its own row would put 16 bytes into each of 32 different 128-byte lines per
+// instruction; instead the rows go through 4 KB of shared memory (`stage`, this warp's own), 32
+// columns at a time, and leave as 128-byte pieces, four rows per instruction.
+constexpr int kPfStageBytes = 4096;
+__device__ __forceinline__ void store_rows_via_stage(uint32_t t_o, float inv, float* dst, float4* stage) {
+  const int lane = threadIdx.x & 31;
+  float* dst_k[8];                                      // destination rows 4k + (lane >> 3)
+#pragma unroll
+  for (int k = 0; k < 8; ++k)
+    dst_k[k] = reinterpret_cast<float*>(__shfl_sync(0xffffffffu, reinterpret_cast<unsigned long long>(dst),
+                                                    4 * k + (lane >> 3)));
+#pragma unroll 1
+  for (int c = 0; c < 4; ++c) {
+    uint32_t r[32];
+    tmem_ld32(t_o + c * 32, r);
+#pragma unroll
+    for (int i = 0; i < 8; ++i)                         // piece i of row `lane`, swizzled by the row
+      stage[lane * 8 + (i ^ (lane & 7))] =
+          make_float4(__uint_as_float(r[4 * i]) * inv, __uint_as_float(r[4 * i + 1]) * inv,
+                      __uint_as_float(r[4 * i + 2]) * inv, __uint_as_float(r[4 * i + 3]) * inv);
+    __syncwarp();
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      const int rr = 4 * k + (lane >> 3);
+      const float4 v = stage[rr * 8 + ((lane & 7) ^ (rr & 7))];
+      if (dst_k[k]) reinterpret_cast<float4*>(dst_k[k] + c * 32)[lane & 7] = v;
+    }
+    __syncwarp();
+  }
+}
+
 // The pipelined kernel walks the cache in sub-blocks of 64 tokens.
 constexpr int kPfSub = 64;                      // cached tokens per sub-block
 constexpr int kPfSubHalf = kPfSub * 128;        // one [64 tokens][64 bf16] swizzled tile: 8 KB
@@ -528,6 +562,8 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;   // 1024-byte aligned tiles
   const uint32_t sQ = base + (uint32_t)tile * kPfTileBytes;      // this query tile's rows
   const uint32_t sK = base + 2 * kPfTileBytes, sV = sK + NS * kPfSubTile;
+  // behind the tiles: 4 KB per softmax warp for the epilogue's way out
+  unsigned char* const stage_base = smem_raw + (base - smem_u32(smem_raw)) + 2 * kPfTileBytes + 2 * NS * kPfSubTile;
   const uint32_t bar0 = smem_u32(&s_bar[0]);
   auto bar_k = [&](int i) { return bar0 + 8u * (uint32_t)i; };
   auto bar_v = [&](int i) { return bar0 + 8u * (uint32_t)(NS + i); };
@@ -739,18 +775,8 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
   const float l_tot = l_run;
   if (!failed && softmax_thread && tile_active) {
     const float inv = l_tot > 0.f ? 1.f / l_tot : 0.f;   // nothing seen: zeros, log-sum-exp -inf
-#pragma unroll 1
-    for (int c = 0; c < 4; ++c) {
-      uint32_t r[32];
-      tmem_ld32(t_o + c * 32, r);
-      if (row_valid) {
-        float4* dst = reinterpret_cast<float4*>(out + row_off * D + c * 32);
-#pragma unroll
-        for (int i = 0; i < 32; i += 4)
-          dst[i >> 2] = make_float4(__uint_as_float(r[i]) * inv, __uint_as_float(r[i + 1]) * inv,
-                                    __uint_as_float(r[i + 2]) * inv, __uint_as_float(r[i + 3]) * inv);
-      }
-    }
+    store_rows_via_stage(t_o, inv, row_valid ? out + row_off * D : nullptr,
+                         reinterpret_cast<float4*>(stage_base + warp * kPfStageBytes));
     if (row_valid && lse_out)
       lse_out[row_off] = (m_ref + log2f(l_tot)) * 0.6931471805599453f;
   }
@@ -765,7 +791,8 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
 // The persistent, work-balanced kernel (L2KV_PREFIX_KERNEL=persistent; needs a workspace with
 // room for its partial results).  The pipelined kernel's roles and hand-offs, but a fixed grid of
 // kPfPersistCtas CTAs, each of which stays on its SM and walks an equal share of the call's work:
-//   - a work item is (pair of query tiles, unit); its cost is its number of 64-token sub-blocks.
+//   - a work item is (pair of query tiles, unit); its cost is its number of 64-token sub-blocks
+//     plus kPfItemOverhead (what starting and finishing an item costs, in sub-blocks' time).
 //     Every CTA adds up the costs of all items (the lengths live in device memory) and takes the
 //     range [c P, (c + 1) P) of the running total, P = ceil(total / CTAs): whole items, plus at
 //     most one item cut at its start and one cut at its end;
@@ -779,6 +806,8 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
 constexpr int kPfPersistCtas = 148;
 constexpr int kPfSlotRows = 2 * kPfRows;         // rows of one partial result: both query tiles
 constexpr int kPfMinShare = 16;                  // sub-blocks: no share below 1024 tokens
+constexpr int kPfAutoShare = 48;                 // sub-blocks per CTA from which a small grid is dealt out this way
+constexpr int kPfItemOverhead = 10;              // measured: about 20 k cycles against 1.9 k per sub-block
 
 template <int G, bool SW>
 __global__ void __launch_bounds__(kPfPipeThreads, 1)
@@ -821,7 +850,11 @@ prefix_attention_persistent_kernel(const __nv_bfloat16* __restrict__ q, Geom g, 
     const long long unit = it % units, bl = unit / g.H;
     return max(0, min(cur_len_dev.at(bl, (int)(unit % g.H), g.H), min(max_len, g.cap(bl))));
   };
-  auto item_cost = [&](long long it) { return (item_rows(it) + kPfSub - 1) / kPfSub; };
+  // (the overhead comes first in an item's range of the running total, its sub-blocks after it)
+  auto item_cost = [&](long long it) {
+    const int nb_it = (item_rows(it) + kPfSub - 1) / kPfSub;
+    return nb_it > 0 ? nb_it + kPfItemOverhead : 0;
+  };
 
   // ---- every CTA adds up all costs: thread t takes the items [t chunk, (t + 1) chunk) -----------
   const long long chunk = (items + NT - 1) / NT;
@@ -888,6 +921,8 @@ prefix_attention_persistent_kernel(const __nv_bfloat16* __restrict__ q, Geom g, 
   const int wq = warp & 3;                              // tensor-memory lane quarter of this warp
   const uint32_t sQ = base + (uint32_t)tile * kPfTileBytes;
   const uint32_t sK = base + 2 * kPfTileBytes, sV = sK + NS * kPfSubTile;
+  // behind the tiles: 4 KB per softmax warp for the epilogue's way out
+  unsigned char* const stage_base = smem_raw + (base - smem_u32(smem_raw)) + 2 * kPfTileBytes + 2 * NS * kPfSubTile;
   const uint32_t bar0 = smem_u32(&s_bar[0]);
   auto bar_k = [&](int i) { return bar0 + 8u * (uint32_t)i; };
   auto bar_v = [&](int i) { return bar0 + 8u * (uint32_t)(NS + i); };
@@ -930,11 +965,12 @@ prefix_attention_persistent_kernel(const __nv_bfloat16* __restrict__ q, Geom g, 
   long long w_it = (long long)s_first;
   int w_at = s_first_at;
   long long it = 0;                                     // the segment's item
-  int at = 0, cost = 0, j0 = 0, j1 = 0;                 // its place in the total, cost, sub-block range
+  int at = 0, cost = 0, nb_it = 0, j0 = 0, j1 = 0;      // its place in the total, cost, sub-blocks, range
   auto next_segment = [&]() {
     if (w_it < 0 || w_it >= items || w_at >= hi) return false;
     it = w_it; at = w_at; cost = item_cost(it);
-    j0 = max(0, lo - at); j1 = min(cost, hi - at);
+    nb_it = max(0, cost - kPfItemOverhead);
+    j0 = max(0, lo - at - kPfItemOverhead); j1 = min(nb_it, hi - at - kPfItemOverhead);
     ++w_it; w_at += cost;
     return true;
   };
@@ -1051,8 +1087,10 @@ prefix_attention_persistent_kernel(const __nv_bfloat16* __restrict__ q, Geom g, 
       }
       const int nbs = j1 - j0;
       if (nbs <= 0) continue;
-      const bool partial = j0 > 0 || j1 < cost;
-      const int slot = (j0 > 0 || at == lo) ? 2 * cta : 2 * cta + 1;
+      const bool partial = j0 > 0 || j1 < nb_it;
+      // a piece that is this CTA's first segment (the item begins at or before the range) takes
+      // slot 2c, one that begins inside the range slot 2c + 1
+      const int slot = at <= lo ? 2 * cta : 2 * cta + 1;
       const bool active = 2 * qp + tile < q_tiles;
       if (!active) jj += nbs;
       if (active) {
@@ -1159,18 +1197,8 @@ prefix_attention_persistent_kernel(const __nv_bfloat16* __restrict__ q, Geom g, 
         const float inv = l_run > 0.f ? 1.f / l_run : 0.f;   // nothing seen: zeros, log-sum-exp -inf
         const long long p_row = (long long)slot * kPfSlotRows + tile * kPfRows + row;
         float* dst_row = partial ? part_out + p_row * D : out + row_off * D;
-#pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
-          uint32_t r[32];
-          tmem_ld32(t_o + c * 32, r);
-          if (row_valid) {
-            float4* dst = reinterpret_cast<float4*>(dst_row + c * 32);
-#pragma unroll
-            for (int i = 0; i < 32; i += 4)
-              dst[i >> 2] = make_float4(__uint_as_float(r[i]) * inv, __uint_as_float(r[i + 1]) * inv,
-                                        __uint_as_float(r[i + 2]) * inv, __uint_as_float(r[i + 3]) * inv);
-          }
-        }
+        store_rows_via_stage(t_o, inv, row_valid ? dst_row : nullptr,
+                             reinterpret_cast<float4*>(stage_base + warp * kPfStageBytes));
         const float lse = (m_ref + log2f(l_run)) * 0.6931471805599453f;
         if (row_valid) {
           if (partial) part_lse[p_row] = lse;
@@ -1184,7 +1212,7 @@ prefix_attention_persistent_kernel(const __nv_bfloat16* __restrict__ q, Geom g, 
         // A piece of a cut item: once both tiles' rows are in the workspace, this CTA takes a
         // ticket of the item (counter of the CTA the item starts in); whoever takes the last one
         // adds the pieces up.  Nobody waits for another CTA; the counter goes back to zero.
-        const int c_first = cta_of(at), c_last = cta_of(at + cost - 1);
+        const int c_first = cta_of(at + kPfItemOverhead), c_last = cta_of(at + cost - 1);   // CTAs with sub-blocks
         __threadfence();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_piece);
@@ -1204,7 +1232,7 @@ prefix_attention_persistent_kernel(const __nv_bfloat16* __restrict__ q, Geom g, 
           // 8 rows' loads in flight at a time.
           __threadfence();
           const int r = tile * kPfRows + row;
-          auto slot_of = [&](int p) { return p == c_first ? (at == lo_of(c_first) ? 2 * p : 2 * p + 1) : 2 * p; };
+          auto slot_of = [&](int p) { return p == c_first && at > lo_of(c_first) ? 2 * p + 1 : 2 * p; };
           float m = -INFINITY;
           if (row_valid)
             for (int p = c_first; p <= c_last; ++p)
@@ -1318,12 +1346,17 @@ static PrefixPlan plan_prefix(const Geom& g, int n_queries, int max_len) {
   if (which && std::strcmp(which, "basic") == 0) p.basic = true;
   if (which && std::strcmp(which, "pipelined") == 0) p.basic = false;
   const long long pairs_all = (long long)g.B * g.L * g.H * ((q_tiles + 1) / 2);
-  // the work-balanced kernel: on request, and by itself for very long caches, where (b, l) pairs
-  // of different lengths would otherwise leave a few CTAs running alone at the end
-  const bool fits = pairs_all * ((long long)max_len / kPfSub + 1) < (long long)INT_MAX / 2;
+  // the work-balanced kernel: on request, and by itself (a) for very long caches, where (b, l)
+  // pairs of different lengths would otherwise leave a few CTAs running alone at the end, and
+  // (b) for grids of less than two waves whose work still gives each of its CTAs a share of at
+  // least kPfAutoShare sub-blocks (measured: below that its set-up and the merging of many short
+  // pieces cost more than the even shares gain)
+  const bool fits = pairs_all * ((long long)max_len / kPfSub + 1 + kPfItemOverhead) < (long long)INT_MAX / 2;
   if (which && std::strcmp(which, "persistent") == 0) p.basic = false;
+  const bool small_grid = pairs_all < 2 * 148 &&
+                          pairs_all * (((long long)max_len + kPfSub - 1) / kPfSub) >= (long long)kPfAutoShare * kPfPersistCtas;
   p.persistent = fits && !p.basic &&
-                 ((which && std::strcmp(which, "persistent") == 0) || (!which && max_len >= 65536));
+                 ((which && std::strcmp(which, "persistent") == 0) || (!which && (max_len >= 65536 || small_grid)));
   const long long units = (long long)g.B * g.L * g.H;
   p.ctas = units * (p.basic ? q_tiles : (q_tiles + 1) / 2);
   p.rows = (long long)g.B * g.L * n_queries * g.Hq;
@@ -1385,7 +1418,7 @@ static int launch_pf(const void* q, const void* K, const void* V, const Geom& g,
   const dim3 grid((unsigned)p.ctas, (unsigned)p.chunks);
   const __nv_bfloat16* qb = static_cast<const __nv_bfloat16*>(q);
   if (p.persistent && scratch && scratch_bytes >= kPfPersistBytes) {
-    constexpr int smem_pipe = 1024 + 2 * kPfTileBytes + 2 * kPfStages * kPfSubTile;
+    constexpr int smem_pipe = 1024 + 2 * kPfTileBytes + 2 * kPfStages * kPfSubTile + (2 * kPfRows / 32) * kPfStageBytes;
     auto kern = prefix_attention_persistent_kernel<G, SW>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_pipe) != cudaSuccess)
       return L2KV_ERR_CUDA;
@@ -1400,7 +1433,7 @@ static int launch_pf(const void* q, const void* K, const void* V, const Geom& g,
     return cudaGetLastError() == cudaSuccess ? L2KV_OK : L2KV_ERR_CUDA;
   }
   if (!p.basic) {
-    constexpr int smem_pipe = 1024 + 2 * kPfTileBytes + 2 * kPfStages * kPfSubTile;
+    constexpr int smem_pipe = 1024 + 2 * kPfTileBytes + 2 * kPfStages * kPfSubTile + (2 * kPfRows / 32) * kPfStageBytes;
     auto kern_pipe = prefix_attention_pipelined_kernel<G, SW>;
     if (cudaFuncSetAttribute(kern_pipe, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_pipe) != cudaSuccess)
       return L2KV_ERR_CUDA;

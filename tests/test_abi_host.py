@@ -124,16 +124,19 @@ def test_prefix_attention_workspace_plan():
     """Host side of the split over the cache: room for partial results is asked for only when
     the unsplit grid would leave SMs idle or the cache is very long; sizes follow from the plan."""
     rows = lambda B, L, n_q, Hq: B * L * n_q * Hq
+    persistent = 256 + 768 + 2 * 148 * 256 * 129 * 4
     # the benchmark call (all 32 layers, 2048 CTAs): no split
     assert _prefix_ws_bytes(4, 32, 8, 32, 32768, 32768, 128) == (0, 256)
-    # one layer of it: 64 CTAs -> split; scratch = chunks * rows * (128 + 1) floats
-    rc, b = _prefix_ws_bytes(4, 1, 8, 32, 32768, 16384, 128)
+    # one layer of it (64 CTAs unsplit, 256 sub-blocks each): the work-balanced kernel -- a counter
+    # and two partial results of 256 rows (129 floats each) per CTA of its fixed grid of 148
+    assert _prefix_ws_bytes(4, 1, 8, 32, 32768, 16384, 128) == (0, persistent)
+    # a small grid with little work per CTA is cut into chunks: scratch = chunks * rows * (128 + 1) floats
+    rc, b = _prefix_ws_bytes(4, 1, 8, 32, 4096, 4096, 128)
     per_chunk = rows(4, 1, 128, 32) * 129 * 4
     assert rc == 0 and b > 256 and (b - 256) % per_chunk == 0 and 2 <= (b - 256) // per_chunk <= 16
-    # a very long cache goes to the work-balanced kernel: a counter and two partial results of
-    # 256 rows (129 floats each) per CTA of its fixed grid of 148, whatever the call's size
-    assert _prefix_ws_bytes(1, 32, 8, 32, 131072, 131072, 128) == (0, 256 + 768 + 2 * 148 * 256 * 129 * 4)
-    assert _prefix_ws_bytes(2, 4, 8, 32, 70000, 70000, 64)[1] == 256 + 768 + 2 * 148 * 256 * 129 * 4
+    # a very long cache goes to the work-balanced kernel whatever the grid
+    assert _prefix_ws_bytes(1, 32, 8, 32, 131072, 131072, 128) == (0, persistent)
+    assert _prefix_ws_bytes(2, 4, 8, 32, 70000, 70000, 64)[1] == persistent
     # short caches are never split below 1024 tokens; unsupported types ask for the status block only
     assert _prefix_ws_bytes(1, 1, 2, 8, 1000, 1000, 16) == (0, 256)
     assert _prefix_ws_bytes(1, 1, 4, 4, 1024, 1024, 16, dtype=torch.float32, D=64) == (0, 256)
