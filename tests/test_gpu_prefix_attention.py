@@ -267,3 +267,41 @@ def test_prefix_attention_random_shapes(seed, monkeypatch):
         empty = see == 0
         assert not got[:, :, s][empty].any() and np.all(np.isneginf(got_lse[:, :, s][empty]))
         assert np.all(np.isfinite(got_lse[:, :, s][~empty]))
+
+
+def test_persistent_kernel_many_calls_on_one_workspace(monkeypatch):
+    """The work-balanced kernel keeps counters and partial results in the workspace: a dozen
+    calls of different shapes and lengths reuse one workspace back to back (no clearing in
+    between); sampled queries of every call are compared with the oracle."""
+    import paper_2406_11430_b200 as l2
+    monkeypatch.setenv("L2KV_PREFIX_KERNEL", "persistent")
+    rng = np.random.default_rng(4242)
+    ws = None
+    for call_no in range(12):
+        G = int(rng.choice([2, 4, 8]))
+        Hkv = int(rng.integers(1, 3))
+        B, L = int(rng.integers(1, 4)), int(rng.integers(1, 4))
+        T = int(rng.choice([900, 3000, 6000]))
+        n_q = int(rng.choice([2 * 128 // G, 3 * 128 // G + 1, 150]))      # two or more query tiles
+        causal = bool(rng.integers(0, 2))
+        w = synth.WORKLOADS[2].scaled(B=B, L=L, Hkv=Hkv, Hq=Hkv * G, T=T, seed=500 + call_no)
+        K, V = synth.make_cache(w, DEV)
+        q = make_queries(w, n_q, 600 + call_no)
+        cur = rng.integers(0, T + 1, size=(B, L)).astype(np.int32)
+        cur[0, 0] = T
+        need = l2.prefix_attention_workspace(K, q, T).numel()
+        if ws is None:
+            ws = torch.zeros(need, dtype=torch.uint8, device=DEV)
+        assert need == ws.numel()                        # that kernel's ask does not depend on the call
+        out = torch.full(q.shape, float("nan"), dtype=torch.float32, device=DEV)
+        lse = torch.full(q.shape[:4], float("nan"), dtype=torch.float32, device=DEV)
+        call(l2, "split", q, K, V, i32(cur), T, out, lse, workspace=ws, causal=causal)
+        torch.cuda.synchronize()
+        assert l2.read_device_status(ws) == 0
+        got = out.cpu().numpy()
+        assert not np.isnan(got).any()
+        Kn, Vn = synth.to_numpy(K), synth.to_numpy(V)
+        for s in sorted(set(rng.integers(0, n_q, size=3).tolist() + [n_q - 1])):
+            see = (np.maximum(cur - n_q + s + 1, 0) if causal else cur).astype(np.int32)
+            want = oracle.attention(synth.to_numpy(q[:, :, s].contiguous()), Kn, Vn, "bf16", see, nthreads=8)
+            assert_attention_close(got[:, :, s], want, atol=ATOL["split"])
