@@ -403,8 +403,8 @@ def run_gpu(args):
                          "gpu_launches": jo.launches_per_step * n}
                 if not args.no_cpu_baseline and world == 1:
                     entry["tie_band"] = tie_band_report(jo, wo)
-                if jo.packed and wo.dtype == "bf16" and wo.D == 128:
-                    entry["prefix_attention"] = time_packed_prefix(jo, wo)
+                if wo.dtype == "bf16" and wo.D == 128:
+                    entry["prefix_attention"] = time_prefix_over_compressed(jo, wo)
                 others[wo.name] = entry
             del jo
             free_device_memory()
@@ -414,14 +414,15 @@ def run_gpu(args):
         print(json.dumps(line))
 
 
-def time_packed_prefix(job, w, n_q=128, reps=3):
-    """A block of n_q new queries per sequence over the packed, ragged compressed caches (a chunk of
-    a chunked prefill in a serving batch): prefix attention on the tensor cores, cache split over
-    the grid where the lengths call for it."""
+def time_prefix_over_compressed(job, w, n_q=128, reps=3):
+    """A block of n_q new queries per sequence over the compressed caches as they stand (dense, or
+    packed and ragged: a chunk of a chunked prefill in a serving batch): prefix attention on the
+    tensor cores with the workspace the library asks for, so that it may cut the caches up."""
     q = torch.randn((w.B, w.L, n_q, w.Hq, w.D), dtype=torch.bfloat16, device=job.dev)
     out = torch.empty(q.shape, dtype=torch.float32, device=job.dev)
-    ws = job.l2.prefix_attention_workspace(job.K_c, q, job.max_dec, rows=job.rows)
-    call = lambda: job.l2.prefix_attention_flags(q, job.K_c, job.V_c, job.cur, job.max_dec, out, 0,
+    max_len = int(job.cur.max().item())                  # the caller knows its longest cache
+    ws = job.l2.prefix_attention_workspace(job.K_c, q, max_len, rows=job.rows)
+    call = lambda: job.l2.prefix_attention_flags(q, job.K_c, job.V_c, job.cur, max_len, out, 0,
                                                  workspace=ws, rows=job.rows)
     call()
     torch.cuda.synchronize()
@@ -434,7 +435,8 @@ def time_packed_prefix(job, w, n_q=128, reps=3):
     flops = 4.0 * n_q * w.Hq * w.D * float(job.cur.sum().item())
     status = job.l2.read_device_status(ws)
     return {"ms": round(ms, 3), "queries_per_sequence": n_q, "TFLOPs": round(flops / ms / 1e9, 1),
-            "cached_rows": int(job.cur.sum().item()), "device_status": status}
+            "cached_rows": int(job.cur.sum().item()), "workspace_MiB": round(ws.numel() / 2**20, 1),
+            "device_status": status}
 
 
 def free_device_memory():
