@@ -305,3 +305,23 @@ def test_persistent_kernel_many_calls_on_one_workspace(monkeypatch):
             see = (np.maximum(cur - n_q + s + 1, 0) if causal else cur).astype(np.int32)
             want = oracle.attention(synth.to_numpy(q[:, :, s].contiguous()), Kn, Vn, "bf16", see, nthreads=8)
             assert_attention_close(got[:, :, s], want, atol=ATOL["split"])
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_prefix_attention_all_caches_empty(kernel, monkeypatch):
+    """Nothing cached anywhere: zeros and lse = -inf for every query, from every kernel."""
+    import paper_2406_11430_b200 as l2
+    choose(monkeypatch, kernel)
+    w = synth.WORKLOADS[2].scaled(B=2, L=3, Hkv=2, Hq=8, T=300)
+    K, V = synth.make_cache(w, DEV)
+    q = make_queries(w, 70, 21)
+    cur = np.zeros((2, 3), dtype=np.int32)
+    out = torch.full(q.shape, float("nan"), dtype=torch.float32, device=DEV)
+    lse = torch.full(q.shape[:4], float("nan"), dtype=torch.float32, device=DEV)
+    ws = l2.prefix_attention_workspace(K, q, 300)
+    if ws.numel() == 256 and kernel == "persistent":
+        pytest.skip("no room asked for")
+    call(l2, "single", q, K, V, i32(cur), 300, out, lse, workspace=ws)
+    torch.cuda.synchronize()
+    assert l2.read_device_status(ws) == 0
+    assert not out.cpu().numpy().any() and np.all(np.isneginf(lse.cpu().numpy()))
