@@ -157,6 +157,27 @@ __device__ __forceinline__ void tmem_scale8(uint32_t taddr, float factor) {
                : "memory");
 }
 
+// Query rows of one tile into shared memory (K-major, 128-byte swizzle), by one warp: rows
+// row0 .. row0 + 31 of the tile, pieces [16 first, 16 first + 16 count) of the 32 instruction
+// slots (slot i: rows row0 + 2i and row0 + 2i + 1).  Lanes 0-15 and 16-31 each read one whole
+// 256-byte row per instruction, so a request touches 4 lines instead of 32.  Row r of tile
+// number `tile_no` of the unit is query tile_no * (128 / G) + r / G, head h * G + r % G.
+template <int G>
+__device__ __forceinline__ void load_query_rows(const __nv_bfloat16* __restrict__ q, long long bl,
+                                                int n_queries, int Hq, int h, int tile_no, int row0,
+                                                uint32_t sQ, int first, int count) {
+  constexpr int QT = kPfRows / G;
+  const int lane = threadIdx.x & 31, c = lane & 15;
+#pragma unroll 8
+  for (int i = first; i < first + count; ++i) {
+    const int r = row0 + 2 * i + (lane >> 4);
+    const int s_idx = tile_no * QT + r / G;
+    const long long off = ((bl * n_queries + s_idx) * Hq + h * G + r % G) * 128 + c * 8;
+    const uint4 v = s_idx < n_queries ? *reinterpret_cast<const uint4*>(q + off) : make_uint4(0, 0, 0, 0);
+    st_shared16(sQ + (c >> 3) * kPfHalf + r * 128 + (((c & 7) ^ (r & 7)) << 4), v.x, v.y, v.z, v.w);
+  }
+}
+
 // The basic kernel (L2KV_PREFIX_KERNEL=basic): one role, two CTAs per SM that fill each other's
 // gaps.  The weights never go to shared memory: they are written as bf16 pairs into the
 // tensor-memory columns that held the scores and feed the second contraction from there
@@ -241,14 +262,8 @@ prefix_attention_basic_kernel(const __nv_bfloat16* __restrict__ q, Geom g, int n
     s_fail = 0;
   }
   __syncwarp();
-  {                                                     // Q rows, K-major, 128-byte swizzle
-    const uint4* src = reinterpret_cast<const uint4*>(q + row_off * D) + hf * 8;
-#pragma unroll
-    for (int c = 0; c < 8; ++c) {
-      const uint4 v = row_valid ? src[c] : make_uint4(0, 0, 0, 0);
-      st_shared16(sQ + hf * kPfHalf + row * 128 + ((c ^ (row & 7)) << 4), v.x, v.y, v.z, v.w);
-    }
-  }
+  // Q rows: warps w and w + 4 share rows 32 (w & 3) .. + 31 and load half of them each
+  load_query_rows<G>(q, bl, n_queries, g.Hq, h, qt, (warp & 3) * 32, sQ, hf * 8, 8);
   proxy_fence();
   tc_fence_before();
   __syncthreads();
@@ -595,14 +610,8 @@ prefix_attention_pipelined_kernel(const __nv_bfloat16* __restrict__ q, Geom g, i
     s_fail = 0;
   }
   __syncwarp();
-  if (softmax_thread) {                                 // Q rows, K-major, 128-byte swizzle
-    const uint4* src = reinterpret_cast<const uint4*>(q + row_off * D);
-#pragma unroll
-    for (int c = 0; c < 16; ++c) {
-      const uint4 v = row_valid ? src[c] : make_uint4(0, 0, 0, 0);
-      st_shared16(sQ + (c >> 3) * kPfHalf + row * 128 + (((c & 7) ^ (row & 7)) << 4), v.x, v.y, v.z, v.w);
-    }
-  }
+  if (softmax_thread)                                   // every softmax warp loads its own 32 rows
+    load_query_rows<G>(q, bl, n_queries, g.Hq, h, 2 * qp + tile, wq * 32, sQ, 0, 16);
   proxy_fence();
   tc_fence_before();
   __syncthreads();
@@ -1097,13 +1106,8 @@ prefix_attention_persistent_kernel(const __nv_bfloat16* __restrict__ q, Geom g, 
       const int n_all = item_rows(it);
       // causal: the last n_queries cached rows are the new tokens' own; query s stops at its own
       const int n_row = causal && row_valid ? min(n_all, max(0, n_all - n_queries + s_idx + 1)) : n_all;
-      {                                                   // Q row, K-major, 128-byte swizzle
-        const uint4* src = reinterpret_cast<const uint4*>(q + row_off * D);
-#pragma unroll
-        for (int c = 0; c < 16; ++c) {
-          const uint4 v = row_valid ? src[c] : make_uint4(0, 0, 0, 0);
-          st_shared16(sQ + (c >> 3) * kPfHalf + row * 128 + (((c & 7) ^ (row & 7)) << 4), v.x, v.y, v.z, v.w);
-        }
+      {                                                   // this warp's 32 query rows
+        load_query_rows<G>(q, bl, n_queries, g.Hq, h, 2 * qp + tile, wq * 32, sQ, 0, 16);
         proxy_fence();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_q);
