@@ -816,6 +816,9 @@ constexpr int kPfPersistCtas = 148;
 constexpr int kPfSlotRows = 2 * kPfRows;         // rows of one partial result: both query tiles
 constexpr int kPfMinShare = 16;                  // sub-blocks: no share below 1024 tokens
 constexpr int kPfAutoShare = 48;                 // sub-blocks per CTA from which a small grid is dealt out this way
+constexpr int kPfTicketWord = 16;                // first word of the ticket bytes in the status block
+static_assert(kPfTicketWord * 4 + kPfPersistCtas <= kStatusBytes && kPfPersistCtas < 256,
+              "a ticket byte per CTA inside the status block; a count fits its byte");
 constexpr int kPfItemOverhead = 10;              // measured: about 20 k cycles against 1.9 k per sub-block
 
 template <int G, bool SW>
@@ -826,7 +829,7 @@ prefix_attention_persistent_kernel(const __nv_bfloat16* __restrict__ q, Geom g, 
                            const __grid_constant__ CUtensorMap map_k,
                            const __grid_constant__ CUtensorMap map_v,
                            int32_t* __restrict__ status_word, float* __restrict__ part_out,
-                           float* __restrict__ part_lse, int* __restrict__ tickets, int causal) {
+                           float* __restrict__ part_lse, int causal) {
   constexpr int D = 128;
   constexpr int QT = kPfRows / G;                       // queries per query tile
   constexpr int NS = kPfStages;
@@ -1222,9 +1225,13 @@ prefix_attention_persistent_kernel(const __nv_bfloat16* __restrict__ q, Geom g, 
         if (lane == 0) mbar_arrive(bar_piece);
         if (!mbar_wait<kPfPolls>(bar_piece, (uint32_t)pieces & 1u)) { gave_up = true; break; }
         if (tid == 0) {
-          const int turn = atomicAdd(tickets + c_first, 1);
+          // the counters: one byte per CTA, four to a word, in the workspace's status block (zero
+          // before the call like the rest of the block, and zero again after the last ticket)
+          unsigned int* const word = reinterpret_cast<unsigned int*>(status_word) + kPfTicketWord + (c_first >> 2);
+          const int shift = (c_first & 3) * 8;
+          const int turn = (int)((atomicAdd(word, 1u << shift) >> shift) & 0xffu);
           s_merge = turn == c_last - c_first;
-          if (s_merge) tickets[c_first] = 0;
+          if (s_merge) atomicSub(word, (unsigned int)(c_last - c_first + 1) << shift);
           __threadfence();
           mbar_arrive(bar_turn);
         }
@@ -1386,11 +1393,10 @@ static PrefixPlan plan_prefix(const Geom& g, int n_queries, int max_len) {
   return p;
 }
 
-// Scratch of the persistent kernel: a ticket counter per CTA, then the log-sum-exps and the rows
-// of the two partial results a CTA may write.
-constexpr size_t kPfCutBytes = (kPfPersistCtas * sizeof(int) + 255) / 256 * 256;   // the tickets
+// Scratch of the persistent kernel: the log-sum-exps and the rows of the two partial results a
+// CTA may write (its ticket counters live in the status block).
 constexpr size_t kPfPartLseBytes = (size_t)2 * kPfPersistCtas * kPfSlotRows * sizeof(float);
-constexpr size_t kPfPersistBytes = kPfCutBytes + kPfPartLseBytes * (1 + 128);
+constexpr size_t kPfPersistBytes = kPfPartLseBytes * (1 + 128);
 
 size_t prefix_attention_scratch(const Geom& g, int n_queries, int max_len) {
   const PrefixPlan p = plan_prefix(g, n_queries, max_len);
@@ -1421,19 +1427,17 @@ static int launch_pf(const void* q, const void* K, const void* V, const Geom& g,
   float* k_lse = p.chunks > 1 ? scratch + (size_t)p.chunks * p.rows * 128 : lse_out;
   const dim3 grid((unsigned)p.ctas, (unsigned)p.chunks);
   const __nv_bfloat16* qb = static_cast<const __nv_bfloat16*>(q);
-  if (p.persistent && scratch && scratch_bytes >= kPfPersistBytes) {
+  if (p.persistent && status_word && scratch && scratch_bytes >= kPfPersistBytes) {
     constexpr int smem_pipe = 1024 + 2 * kPfTileBytes + 2 * kPfStages * kPfSubTile + (2 * kPfRows / 32) * kPfStageBytes;
     auto kern = prefix_attention_persistent_kernel<G, SW>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_pipe) != cudaSuccess)
       return L2KV_ERR_CUDA;
     char* sc = reinterpret_cast<char*>(scratch);
-    int* tickets = reinterpret_cast<int*>(sc);
-    if (cudaMemsetAsync(tickets, 0, kPfCutBytes, s) != cudaSuccess) return L2KV_ERR_CUDA;
-    float* part_lse = reinterpret_cast<float*>(sc + kPfCutBytes);
-    float* part_out = reinterpret_cast<float*>(sc + kPfCutBytes + kPfPartLseBytes);
+    float* part_lse = reinterpret_cast<float*>(sc);
+    float* part_out = reinterpret_cast<float*>(sc + kPfPartLseBytes);
     kern<<<kPfPersistCtas, kPfPipeThreads, smem_pipe, s>>>(qb, g, n_queries, cur_len_dev, max_len,
                                                           scale * kPfLog2e, out, lse_out, map_k, map_v,
-                                                          status_word, part_out, part_lse, tickets, causal);
+                                                          status_word, part_out, part_lse, causal);
     return cudaGetLastError() == cudaSuccess ? L2KV_OK : L2KV_ERR_CUDA;
   }
   if (!p.basic) {

@@ -124,11 +124,11 @@ def test_prefix_attention_workspace_plan():
     """Host side of the split over the cache: room for partial results is asked for only when
     the unsplit grid would leave SMs idle or the cache is very long; sizes follow from the plan."""
     rows = lambda B, L, n_q, Hq: B * L * n_q * Hq
-    persistent = 256 + 768 + 2 * 148 * 256 * 129 * 4
+    persistent = 256 + 2 * 148 * 256 * 129 * 4
     # the benchmark call (all 32 layers, 2048 CTAs): no split
     assert _prefix_ws_bytes(4, 32, 8, 32, 32768, 32768, 128) == (0, 256)
-    # one layer of it (64 CTAs unsplit, 256 sub-blocks each): the work-balanced kernel -- a counter
-    # and two partial results of 256 rows (129 floats each) per CTA of its fixed grid of 148
+    # one layer of it (64 CTAs unsplit, 256 sub-blocks each): the work-balanced kernel -- two
+    # partial results of 256 rows (129 floats each) per CTA of its fixed grid of 148
     assert _prefix_ws_bytes(4, 1, 8, 32, 32768, 16384, 128) == (0, persistent)
     # a small grid with little work per CTA is cut into chunks: scratch = chunks * rows * (128 + 1) floats
     rc, b = _prefix_ws_bytes(4, 1, 8, 32, 4096, 4096, 128)
