@@ -1106,113 +1106,113 @@ prefix_attention_persistent_kernel(const __nv_bfloat16* __restrict__ q, Geom g, 
       const bool active = 2 * qp + tile < q_tiles;
       if (!active) jj += nbs;
       if (active) {
-      const int n_all = item_rows(it);
-      // causal: the last n_queries cached rows are the new tokens' own; query s stops at its own
-      const int n_row = causal && row_valid ? min(n_all, max(0, n_all - n_queries + s_idx + 1)) : n_all;
-      {                                                   // this warp's 32 query rows
-        load_query_rows<G>(q, bl, n_queries, g.Hq, h, 2 * qp + tile, wq * 32, sQ, 0, 16);
-        proxy_fence();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar_q);
-      }
-      float m_ref = -INFINITY, l_run = 0.f;               // reference maximum; sum of this row's weights
-      const int end = jj + nbs;
-      for (int x = jj; x < end; ++x) {
-        const int j = j0 + (x - jj);                      // sub-block of the item
-        const int a = ja + (x - jj), s = a & 1;
-        const int valid = min(kPfSub, n_all - j * kPfSub);   // valid tokens of this sub-block
-        const uint32_t t_s = t_lane + s * 64;               // this row's scores, later its weights
-        if (!mbar_wait_likely(bar_s(s), (uint32_t)(a >> 1) & 1u)) gave_up = true;
-        tc_fence_after();
-        if (__any_sync(0xffffffffu, gave_up)) { gave_up = true; break; }
-        float sv[64];                                     // raw products; the scale is folded in below
-        float bmax = -INFINITY;
-        {
-          uint32_t r0[32], r1[32];
-          tmem_ld64(t_s, r0, r1);
-          const int valid_row = min(valid, n_row - j * kPfSub);
-          if (valid_row >= kPfSub) {
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              sv[i] = __uint_as_float(r0[i]);
-              sv[32 + i] = __uint_as_float(r1[i]);
-              bmax = fmaxf(bmax, fmaxf(sv[i], sv[32 + i]));
-            }
-          } else {
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              sv[i] = i < valid_row ? __uint_as_float(r0[i]) : -INFINITY;
-              sv[32 + i] = 32 + i < valid_row ? __uint_as_float(r1[i]) : -INFINITY;
-              bmax = fmaxf(bmax, fmaxf(sv[i], sv[32 + i]));
-            }
-          }
-        }
-        const float m_new = fmaxf(m_ref, bmax * scale_log2e);
-        if (x == jj) m_ref = m_new;
-        const bool need = m_new > m_ref + kPfRescaleGap;
-        if (__any_sync(0xffffffffu, need)) {
-          // O must be quiet: the previous P V has to be complete (this one waits for this thread)
-          if (!mbar_wait<kPfPolls>(bar_o, (uint32_t)(a - 1) & 1u)) gave_up = true;
-          tc_fence_after();
-          const float factor = need ? fast_exp2(m_ref - m_new) : 1.f;
-#pragma unroll 1
-          for (int c = 0; c < D; c += 8) tmem_scale8(t_o + c, factor);
-          if (need) { l_run *= factor; m_ref = m_new; }
-        }
-        {
-          uint32_t pk[32];
-          [[maybe_unused]] uint32_t pr[SW ? 32 : 1];
-          float rowsum0 = 0.f, rowsum1 = 0.f;
-          const float neg_m = m_ref == -INFINITY ? 0.f : -m_ref;   // a row with nothing to see yet
-#pragma unroll
-          for (int i = 0; i < 64; i += 2) {
-            const float p0 = fast_exp2(__fmaf_rn(sv[i], scale_log2e, neg_m));     // -inf -> 0
-            const float p1 = fast_exp2(__fmaf_rn(sv[i + 1], scale_log2e, neg_m));
-            rowsum0 += p0;
-            rowsum1 += p1;
-            pk[i >> 1] = pack_bf16(p0, p1);
-            if constexpr (SW) pr[i >> 1] = pack_bf16_rest(p0, p1, pk[i >> 1]);
-          }
-          tmem_st32(t_s, pk);
-          if constexpr (SW) tmem_st32(t_s + 32, pr);
-          tmem_wait_st();
-          l_run += rowsum0 + rowsum1;
-        }
-        if (valid < kPfSub) {
-          // partial sub-block: clear the V rows past the valid length (both query tiles write
-          // the same zeros) so that a zero weight times Inf/NaN cannot reach O
-          if (!mbar_wait<kPfPolls>(bar_v(x % NS), (uint32_t)(x / NS) & 1u)) gave_up = true;
-          if (row >= valid && row < kPfSub) {
-#pragma unroll
-            for (int c = 0; c < 16; ++c)
-              st_shared16(sV + (x % NS) * kPfSubTile + (c >> 3) * kPfSubHalf + row * 128 + ((c & 7) << 4), 0, 0, 0, 0);
-          }
+        const int n_all = item_rows(it);
+        // causal: the last n_queries cached rows are the new tokens' own; query s stops at its own
+        const int n_row = causal && row_valid ? min(n_all, max(0, n_all - n_queries + s_idx + 1)) : n_all;
+        {                                                   // this warp's 32 query rows
+          load_query_rows<G>(q, bl, n_queries, g.Hq, h, 2 * qp + tile, wq * 32, sQ, 0, 16);
           proxy_fence();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_q);
         }
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar_p(s));             // one arrival per warp
-      }
-      if (gave_up) break;
-      // the segment's O is complete when the commit behind its last P V has arrived
-      if (!mbar_wait<kPfPolls>(bar_done, (uint32_t)seg & 1u)) { gave_up = true; break; }
-      ++seg;
-      tc_fence_after();
-      jj = end;
-      ja += nbs;
-      {
-        const float inv = l_run > 0.f ? 1.f / l_run : 0.f;   // nothing seen: zeros, log-sum-exp -inf
-        const long long p_row = (long long)slot * kPfSlotRows + tile * kPfRows + row;
-        float* dst_row = partial ? part_out + p_row * D : out + row_off * D;
-        store_rows_via_stage(t_o, inv, row_valid ? dst_row : nullptr,
-                             reinterpret_cast<float4*>(stage_base + warp * kPfStageBytes));
-        const float lse = (m_ref + log2f(l_run)) * 0.6931471805599453f;
-        if (row_valid) {
-          if (partial) part_lse[p_row] = lse;
-          else if (lse_out) lse_out[row_off] = lse;
+        float m_ref = -INFINITY, l_run = 0.f;               // reference maximum; sum of this row's weights
+        const int end = jj + nbs;
+        for (int x = jj; x < end; ++x) {
+          const int j = j0 + (x - jj);                      // sub-block of the item
+          const int a = ja + (x - jj), s = a & 1;
+          const int valid = min(kPfSub, n_all - j * kPfSub);   // valid tokens of this sub-block
+          const uint32_t t_s = t_lane + s * 64;               // this row's scores, later its weights
+          if (!mbar_wait_likely(bar_s(s), (uint32_t)(a >> 1) & 1u)) gave_up = true;
+          tc_fence_after();
+          if (__any_sync(0xffffffffu, gave_up)) { gave_up = true; break; }
+          float sv[64];                                     // raw products; the scale is folded in below
+          float bmax = -INFINITY;
+          {
+            uint32_t r0[32], r1[32];
+            tmem_ld64(t_s, r0, r1);
+            const int valid_row = min(valid, n_row - j * kPfSub);
+            if (valid_row >= kPfSub) {
+#pragma unroll
+              for (int i = 0; i < 32; ++i) {
+                sv[i] = __uint_as_float(r0[i]);
+                sv[32 + i] = __uint_as_float(r1[i]);
+                bmax = fmaxf(bmax, fmaxf(sv[i], sv[32 + i]));
+              }
+            } else {
+#pragma unroll
+              for (int i = 0; i < 32; ++i) {
+                sv[i] = i < valid_row ? __uint_as_float(r0[i]) : -INFINITY;
+                sv[32 + i] = 32 + i < valid_row ? __uint_as_float(r1[i]) : -INFINITY;
+                bmax = fmaxf(bmax, fmaxf(sv[i], sv[32 + i]));
+              }
+            }
+          }
+          const float m_new = fmaxf(m_ref, bmax * scale_log2e);
+          if (x == jj) m_ref = m_new;
+          const bool need = m_new > m_ref + kPfRescaleGap;
+          if (__any_sync(0xffffffffu, need)) {
+            // O must be quiet: the previous P V has to be complete (this one waits for this thread)
+            if (!mbar_wait<kPfPolls>(bar_o, (uint32_t)(a - 1) & 1u)) gave_up = true;
+            tc_fence_after();
+            const float factor = need ? fast_exp2(m_ref - m_new) : 1.f;
+#pragma unroll 1
+            for (int c = 0; c < D; c += 8) tmem_scale8(t_o + c, factor);
+            if (need) { l_run *= factor; m_ref = m_new; }
+          }
+          {
+            uint32_t pk[32];
+            [[maybe_unused]] uint32_t pr[SW ? 32 : 1];
+            float rowsum0 = 0.f, rowsum1 = 0.f;
+            const float neg_m = m_ref == -INFINITY ? 0.f : -m_ref;   // a row with nothing to see yet
+#pragma unroll
+            for (int i = 0; i < 64; i += 2) {
+              const float p0 = fast_exp2(__fmaf_rn(sv[i], scale_log2e, neg_m));     // -inf -> 0
+              const float p1 = fast_exp2(__fmaf_rn(sv[i + 1], scale_log2e, neg_m));
+              rowsum0 += p0;
+              rowsum1 += p1;
+              pk[i >> 1] = pack_bf16(p0, p1);
+              if constexpr (SW) pr[i >> 1] = pack_bf16_rest(p0, p1, pk[i >> 1]);
+            }
+            tmem_st32(t_s, pk);
+            if constexpr (SW) tmem_st32(t_s + 32, pr);
+            tmem_wait_st();
+            l_run += rowsum0 + rowsum1;
+          }
+          if (valid < kPfSub) {
+            // partial sub-block: clear the V rows past the valid length (both query tiles write
+            // the same zeros) so that a zero weight times Inf/NaN cannot reach O
+            if (!mbar_wait<kPfPolls>(bar_v(x % NS), (uint32_t)(x / NS) & 1u)) gave_up = true;
+            if (row >= valid && row < kPfSub) {
+#pragma unroll
+              for (int c = 0; c < 16; ++c)
+                st_shared16(sV + (x % NS) * kPfSubTile + (c >> 3) * kPfSubHalf + row * 128 + ((c & 7) << 4), 0, 0, 0, 0);
+            }
+            proxy_fence();
+          }
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_p(s));             // one arrival per warp
         }
-        tc_fence_before();                                // O has been read before the next segment's P V
-      }
+        if (gave_up) break;
+        // the segment's O is complete when the commit behind its last P V has arrived
+        if (!mbar_wait<kPfPolls>(bar_done, (uint32_t)seg & 1u)) { gave_up = true; break; }
+        ++seg;
+        tc_fence_after();
+        jj = end;
+        ja += nbs;
+        {
+          const float inv = l_run > 0.f ? 1.f / l_run : 0.f;   // nothing seen: zeros, log-sum-exp -inf
+          const long long p_row = (long long)slot * kPfSlotRows + tile * kPfRows + row;
+          float* dst_row = partial ? part_out + p_row * D : out + row_off * D;
+          store_rows_via_stage(t_o, inv, row_valid ? dst_row : nullptr,
+                               reinterpret_cast<float4*>(stage_base + warp * kPfStageBytes));
+          const float lse = (m_ref + log2f(l_run)) * 0.6931471805599453f;
+          if (row_valid) {
+            if (partial) part_lse[p_row] = lse;
+            else if (lse_out) lse_out[row_off] = lse;
+          }
+          tc_fence_before();                                // O has been read before the next segment's P V
+        }
       }
       if (gave_up) break;
       if (partial) {
